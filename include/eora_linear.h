@@ -1,0 +1,169 @@
+/*
+ * eora_linear.h -- C ABI of the EoRA compensated linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper Eq. 4 / Algorithm 1 step 7, written row-vector style):
+ *
+ *     Y = X . deq(Wq) + (X . A) . B
+ *
+ *   X  [M][d_in]      activations (fp16 or bf16), row-major
+ *   Wq [d_in][d_out]  frozen compressed backbone: group-wise asymmetric 3/4-bit codes
+ *                     (paper Section 4.1 "asymmetric quantization"; group size 128 in the
+ *                     group-wise appendix) or 2:4 structured-sparse fp16 (Section 1 / 4.2)
+ *   A  [d_in][rank], B [rank][d_out]   the EoRA low-rank residual (Algorithm 1 output), in
+ *                     fp16 or quantised to 4-bit group-wise / 8-bit per-channel (Section 4.5)
+ *   Y  [M][d_out]     written once (Section 4.5: the output shared by the backbone product and
+ *                     the product with B never leaves the chip in between)
+ *
+ * The paper's column-vector form  W^ X + B' A X  maps as d_in = k, d_out = d, A = A_paper^T,
+ * B = B'_paper^T.
+ *
+ * All pointers are DEVICE pointers unless a parameter is named *_host.  Nothing here is a
+ * torch type.  Every function returns an int status (0 = EORA_OK, negative = error); nothing
+ * throws, aborts or traps.  The library targets one GPU; there is no CPU fallback.
+ *
+ * Interchange layout of the weights handed to eora_linear_create (all little-endian):
+ *   b-bit codes (b = w_bits = 3 or 4): LSB-first bit stream along d_in for each column n;
+ *       the code of (k, n) is stream bits [b*k, b*k+b); word i of the stream is
+ *       w_codes[i * d_out + n]  (uint32 [b*d_in/32][d_out]).  For b = 4: 8 codes per uint32,
+ *       code k%8 in bits 4*(k%8).  For b = 3: 32 codes per 3 words, codes 10 and 21 straddle.
+ *   scales: fp16 [d_in/w_group][d_out].
+ *   zeros : the same b-bit stream along n for each group row: uint32 [d_in/w_group][b*d_out/32];
+ *       the stored value is the zero-point itself;  w = (q - z) * s.
+ *   fp16 A: [d_in][rank] row-major; fp16 B: [rank][d_out] row-major.
+ *   4-bit A (ab_format 1): a [d_in x rank] weight in the layout above (codes uint32 [d_in/8][rank],
+ *       scales fp16 [d_in/ab_group][rank], zeros uint32 [d_in/ab_group][rank/8]); 4-bit B: a
+ *       [rank x d_out] weight with groups of min(ab_group, rank) along rank.
+ *   8-bit A/B (ab_format 2): uint8 codes [d_in][rank] / [rank][d_out], one fp16 scale and one
+ *       uint8 zero per column (rank of them for A, d_out for B).
+ *   2:4 backbone (w_format 1): w_codes = fp16 values [d_out][d_in/2] (the two kept values of each
+ *       quad of consecutive k in increasing-k order), w_zeros = uint32 meta [d_out][d_in/32]:
+ *       quad j owns nibble (meta[n][j/8] >> 4*(j%8)) & 0xF = p0 | p1<<2, 0 <= p0 < p1 <= 3;
+ *       w_scales is unused (may be NULL).
+ */
+#ifndef EORA_LINEAR_H_
+#define EORA_LINEAR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct eora_linear* eora_linear_t;   /* opaque handle, owned by the library */
+
+enum {
+  EORA_OK = 0,
+  EORA_ERR_NULL_ARG = -1,
+  EORA_ERR_BAD_SHAPE = -2,
+  EORA_ERR_UNSUPPORTED = -3,
+  EORA_ERR_MISALIGNED = -4,
+  EORA_ERR_M_TOO_LARGE = -5,
+  EORA_ERR_CUDA = -6,
+  EORA_ERR_DEVICE_TIMEOUT = -7
+};
+
+enum { EORA_W_QUANT = 0, EORA_W_SPARSE24 = 1 };
+enum { EORA_AB_F16 = 0, EORA_AB_Q4 = 1, EORA_AB_Q8 = 2 };
+enum { EORA_X_F16 = 0, EORA_X_BF16 = 1 };
+enum { EORA_Y_F16 = 0, EORA_Y_BF16 = 1, EORA_Y_F32 = 2 };
+/* kernel families reported by eora_linear_path */
+enum { EORA_PATH_GENERIC = 0, EORA_PATH_DECODE = 1, EORA_PATH_PREFILL = 2 };
+/* kernel_policy */
+enum { EORA_POLICY_AUTO = 0, EORA_POLICY_GENERIC = 1 };
+
+/* Plain-old-data, caller-owned, copied by create. */
+typedef struct {
+  int32_t d_in;        /* K; multiple of 128 */
+  int32_t d_out;       /* N; multiple of 32 */
+  int32_t rank;        /* r >= 0, multiple of 8 (0 = no adapter: the plain compressed layer) */
+  int32_t w_format;    /* EORA_W_QUANT or EORA_W_SPARSE24 */
+  int32_t w_bits;      /* 3 or 4 (EORA_W_QUANT) */
+  int32_t w_group;     /* group size along d_in: multiple of 64 dividing d_in (d_in = channel-wise) */
+  int32_t ab_format;   /* EORA_AB_F16 / EORA_AB_Q4 / EORA_AB_Q8 */
+  int32_t ab_group;    /* group size for EORA_AB_Q4 (128); B uses min(ab_group, rank) */
+  int32_t x_dtype;     /* EORA_X_F16 or EORA_X_BF16 */
+  int32_t y_dtype;     /* EORA_Y_F16, EORA_Y_BF16 or EORA_Y_F32 */
+  int32_t max_m;       /* largest M forward will be called with (sizes the scratch memory) */
+  int32_t kernel_policy; /* EORA_POLICY_AUTO, or EORA_POLICY_GENERIC to force the simple kernels */
+} eora_linear_config;
+
+/* Device pointers, interchange layout (see the top of this file); 16-byte aligned. */
+typedef struct {
+  const void* w_codes;   /* codes, or 2:4 values */
+  const void* w_scales;  /* fp16 scales (NULL for 2:4) */
+  const void* w_zeros;   /* packed zero-points, or 2:4 metadata */
+  const void* a;         /* fp16 A, or its codes */
+  const void* a_scales;  /* NULL when ab_format == EORA_AB_F16 */
+  const void* a_zeros;
+  const void* b;
+  const void* b_scales;
+  const void* b_zeros;
+} eora_linear_weights;
+
+/*
+ * Build a layer (Eq. 4 operands).  Reads the caller's weight buffers on `stream` (a cudaStream_t,
+ * may be NULL for the default stream), re-tiles them into library-owned device memory laid out
+ * for 128-bit loads, and allocates the scratch memory forward needs.  The call synchronises
+ * `stream` before returning, so the caller may free its buffers afterwards.  The handle is
+ * immutable; it owns scratch memory, so two forwards on the same handle must not overlap on the
+ * GPU (stream order is enough).  Errors: NULL_ARG, BAD_SHAPE, UNSUPPORTED, MISALIGNED, CUDA;
+ * on error *out is NULL and nothing is leaked.
+ */
+int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights* w,
+                       void* stream, eora_linear_t* out);
+
+/*
+ * Y[M][d_out] = X[M][d_in] . deq(Wq) + (X . A) . B   (Eq. 4), enqueued on `stream`.
+ * x, y: device pointers, row-major, 16-byte aligned, caller-owned; 1 <= m <= max_m; m == 0 is a
+ * no-op returning EORA_OK.  Never synchronises and never allocates.  M <= 64 runs the decode
+ * kernel family, larger M the tensor-core (tcgen05) prefill family.  Asynchronous device-side
+ * problems (a bounded wait that ran out) are latched in a status word readable with
+ * eora_linear_last_device_status after the caller has synchronised.
+ */
+int eora_linear_forward(eora_linear_t h, const void* x, int32_t m, void* y, void* stream);
+
+/*
+ * The same forward for callers whose activations live in HOST memory: copies x_host (pinned or
+ * pageable, [m][d_in]) to a library-owned device staging buffer, runs the forward, copies the
+ * result back to y_host ([m][d_out]) and synchronises `stream` before returning.
+ */
+int eora_linear_forward_host(eora_linear_t h, const void* x_host, int32_t m, void* y_host, void* stream);
+
+/* Free everything the handle owns.  NULL is a no-op.  The caller must have synchronised. */
+int eora_linear_destroy(eora_linear_t h);
+
+/* Which kernel family (EORA_PATH_*) forward would run for this m; negative status on error. */
+int eora_linear_path(eora_linear_t h, int32_t m);
+
+/* How many of this library's kernels one forward(m) launches; negative status on error. */
+int eora_linear_launches(eora_linear_t h, int32_t m);
+
+/*
+ * Debug read-back of the library's internal (re-tiled) copy, for bit-exact unpack / dequant
+ * checks of steps a1/a2:  what = 0: backbone codes as int32 [d_in][d_out] (quantised backbones);
+ * 1: backbone dequantised to fp32 [d_in][d_out], exactly (float)(q - z) * (float)s, or the
+ * expanded 2:4 matrix; 2: A as fp32 [d_in][rank]; 3: B as fp32 [rank][d_out].
+ * `out` is a device buffer of that size; enqueued on `stream`.
+ */
+int eora_linear_dump(eora_linear_t h, int32_t what, void* out, void* stream);
+
+/*
+ * Status word latched by the kernels (0 = fine, EORA_ERR_DEVICE_TIMEOUT = a bounded wait ran
+ * out).  Reads device memory with a blocking copy: call after synchronising.  Clears the word.
+ */
+int eora_linear_last_device_status(eora_linear_t h);
+
+/* Bytes of device memory the handle owns: re-tiled weights, and scratch. */
+int64_t eora_linear_weight_bytes(eora_linear_t h);
+int64_t eora_linear_scratch_bytes(eora_linear_t h);
+
+/* Human-readable name of a status code; never NULL. */
+const char* eora_status_string(int status);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int eora_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EORA_LINEAR_H_ */

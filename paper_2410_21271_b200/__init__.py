@@ -1,0 +1,276 @@
+"""Thin Python binding of libeora_linear (the C ABI in include/eora_linear.h).
+
+Argument marshalling only: every step of the layer runs in the library's CUDA kernels.
+torch is used for device memory and streams.  There is no CPU fallback: if the shared
+library has not been built (``python -m paper_2410_21271_b200.build``) loading fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_int, c_int32, c_int64, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libeora_linear.so")
+HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "eora_linear.h")
+
+# status codes / enums (mirrors of include/eora_linear.h)
+EORA_OK = 0
+EORA_ERR_NULL_ARG, EORA_ERR_BAD_SHAPE, EORA_ERR_UNSUPPORTED, EORA_ERR_MISALIGNED = -1, -2, -3, -4
+EORA_ERR_M_TOO_LARGE, EORA_ERR_CUDA, EORA_ERR_DEVICE_TIMEOUT = -5, -6, -7
+EORA_W_QUANT, EORA_W_SPARSE24 = 0, 1
+EORA_AB_F16, EORA_AB_Q4, EORA_AB_Q8 = 0, 1, 2
+EORA_X_F16, EORA_X_BF16 = 0, 1
+EORA_Y_F16, EORA_Y_BF16, EORA_Y_F32 = 0, 1, 2
+EORA_PATH_GENERIC, EORA_PATH_DECODE, EORA_PATH_PREFILL = 0, 1, 2
+EORA_POLICY_AUTO, EORA_POLICY_GENERIC = 0, 1
+
+
+class eora_linear_config(Structure):
+    _fields_ = [(n, c_int32) for n in ("d_in", "d_out", "rank", "w_format", "w_bits", "w_group", "ab_format",
+                                       "ab_group", "x_dtype", "y_dtype", "max_m", "kernel_policy")]
+
+
+class eora_linear_weights(Structure):
+    _fields_ = [(n, c_void_p) for n in ("w_codes", "w_scales", "w_zeros", "a", "a_scales", "a_zeros",
+                                        "b", "b_scales", "b_zeros")]
+
+
+class EoraError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {eora_status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_21271_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.eora_linear_create.argtypes = [POINTER(eora_linear_config), POINTER(eora_linear_weights), c_void_p,
+                                         POINTER(c_void_p)]
+        L.eora_linear_create.restype = c_int
+        L.eora_linear_forward.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_forward.restype = c_int
+        L.eora_linear_forward_host.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_forward_host.restype = c_int
+        L.eora_linear_destroy.argtypes = [c_void_p]
+        L.eora_linear_destroy.restype = c_int
+        L.eora_linear_path.argtypes = [c_void_p, c_int32]
+        L.eora_linear_path.restype = c_int
+        L.eora_linear_launches.argtypes = [c_void_p, c_int32]
+        L.eora_linear_launches.restype = c_int
+        L.eora_linear_dump.argtypes = [c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_dump.restype = c_int
+        L.eora_linear_last_device_status.argtypes = [c_void_p]
+        L.eora_linear_last_device_status.restype = c_int
+        L.eora_linear_weight_bytes.argtypes = [c_void_p]
+        L.eora_linear_weight_bytes.restype = c_int64
+        L.eora_linear_scratch_bytes.argtypes = [c_void_p]
+        L.eora_linear_scratch_bytes.restype = c_int64
+        L.eora_status_string.argtypes = [c_int]
+        L.eora_status_string.restype = c_char_p
+        L.eora_version.argtypes = []
+        L.eora_version.restype = c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> int | None:
+    """Raw address of a torch tensor / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int | None:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def eora_status_string(status: int) -> str:
+    return lib().eora_status_string(int(status)).decode()
+
+
+def eora_version() -> int:
+    return lib().eora_version()
+
+
+def eora_linear_create(cfg: eora_linear_config, weights: eora_linear_weights, stream=None) -> int:
+    """Returns the opaque handle (an address).  Raises EoraError on a non-zero status."""
+    out = c_void_p()
+    st = lib().eora_linear_create(byref(cfg), byref(weights), _stream(stream), byref(out))
+    if st != EORA_OK:
+        raise EoraError(st, "eora_linear_create")
+    return out.value
+
+
+def eora_linear_create_status(cfg, weights, stream=0) -> int:
+    """create, returning only the status (for argument-checking tests; no handle is kept on error)."""
+    out = c_void_p()
+    st = lib().eora_linear_create(byref(cfg) if cfg is not None else None,
+                                  byref(weights) if weights is not None else None, stream, byref(out))
+    if st == EORA_OK:
+        lib().eora_linear_destroy(out)
+    return st
+
+
+def eora_linear_forward(handle: int, x, m: int, y, stream=None, check: bool = True) -> int:
+    st = lib().eora_linear_forward(handle, _ptr(x), int(m), _ptr(y), _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward")
+    return st
+
+
+def eora_linear_forward_host(handle: int, x_host, m: int, y_host, stream=None, check: bool = True) -> int:
+    st = lib().eora_linear_forward_host(handle, _ptr(x_host), int(m), _ptr(y_host), _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward_host")
+    return st
+
+
+def eora_linear_destroy(handle: int) -> int:
+    return lib().eora_linear_destroy(handle)
+
+
+def eora_linear_path(handle: int, m: int) -> int:
+    return lib().eora_linear_path(handle, int(m))
+
+
+def eora_linear_launches(handle: int, m: int) -> int:
+    return lib().eora_linear_launches(handle, int(m))
+
+
+def eora_linear_dump(handle: int, what: int, out, stream=None) -> int:
+    st = lib().eora_linear_dump(handle, int(what), _ptr(out), _stream(stream))
+    if st != EORA_OK:
+        raise EoraError(st, "eora_linear_dump")
+    return st
+
+
+def eora_linear_last_device_status(handle: int) -> int:
+    return lib().eora_linear_last_device_status(handle)
+
+
+def eora_linear_weight_bytes(handle: int) -> int:
+    return lib().eora_linear_weight_bytes(handle)
+
+
+def eora_linear_scratch_bytes(handle: int) -> int:
+    return lib().eora_linear_scratch_bytes(handle)
+
+
+# ---------------------------------------------------------------------------------------------
+# marshalling helper: numpy weight descriptions (as made by eora_inputs) -> device buffers -> handle
+# ---------------------------------------------------------------------------------------------
+def _dev(arr, device):
+    import numpy as np
+    import torch
+    a = np.ascontiguousarray(arr)
+    if a.dtype == np.uint32:
+        a = a.view(np.int32)
+    elif a.dtype == np.uint16:
+        a = a.view(np.int16)
+    return torch.from_numpy(a).to(device)
+
+
+class Layer:
+    """Owns a library handle plus nothing else (the uploaded interchange buffers are dropped after
+    create).  Methods only marshal arguments."""
+
+    def __init__(self, w_fmt: dict, a_fmt: dict | None, b_fmt: dict | None, *, max_m: int, x_dtype: str = "f16",
+                 y_dtype: str = "f16", kernel_policy: int = EORA_POLICY_AUTO, device="cuda:0"):
+        import torch
+        cfg = eora_linear_config()
+        wts = eora_linear_weights()
+        keep = []
+        cfg.d_in, cfg.d_out = w_fmt["rows"], w_fmt["cols"]
+        if w_fmt["kind"] == "quant":
+            cfg.w_format, cfg.w_bits, cfg.w_group = EORA_W_QUANT, w_fmt["bits"], w_fmt["group"]
+            bufs = [_dev(w_fmt["codes"], device), _dev(w_fmt["scales"], device), _dev(w_fmt["zeros"], device)]
+        elif w_fmt["kind"] == "sparse24":
+            cfg.w_format = EORA_W_SPARSE24
+            bufs = [_dev(w_fmt["values"], device), None, _dev(w_fmt["meta"], device)]
+        else:
+            raise ValueError(w_fmt["kind"])
+        keep += bufs
+        wts.w_codes, wts.w_scales, wts.w_zeros = [_ptr(b) for b in bufs]
+        cfg.rank = 0
+        cfg.ab_format, cfg.ab_group = EORA_AB_F16, 128
+        if a_fmt is not None and b_fmt is not None:
+            kind = a_fmt["kind"]
+            if kind == "f16":
+                cfg.rank = a_fmt["data"].shape[1]
+                ab = [_dev(a_fmt["data"], device), None, None, _dev(b_fmt["data"], device), None, None]
+            elif kind == "quant":
+                cfg.rank, cfg.ab_format, cfg.ab_group = a_fmt["cols"], EORA_AB_Q4, a_fmt["group"]
+                ab = [_dev(f[k], device) for f in (a_fmt, b_fmt) for k in ("codes", "scales", "zeros")]
+            elif kind == "q8":
+                cfg.rank, cfg.ab_format = a_fmt["cols"], EORA_AB_Q8
+                ab = [_dev(f[k], device) for f in (a_fmt, b_fmt) for k in ("codes", "scales", "zeros")]
+            else:
+                raise ValueError(kind)
+            keep += ab
+            (wts.a, wts.a_scales, wts.a_zeros, wts.b, wts.b_scales, wts.b_zeros) = [_ptr(b) for b in ab]
+        cfg.x_dtype = {"f16": EORA_X_F16, "bf16": EORA_X_BF16}[x_dtype]
+        cfg.y_dtype = {"f16": EORA_Y_F16, "bf16": EORA_Y_BF16, "f32": EORA_Y_F32}[y_dtype]
+        cfg.max_m, cfg.kernel_policy = max_m, kernel_policy
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.y_torch_dtype = {"f16": torch.float16, "bf16": torch.bfloat16, "f32": torch.float32}[y_dtype]
+        with torch.cuda.device(self.device):
+            self.handle = eora_linear_create(cfg, wts)
+        del keep
+
+    def forward(self, x, y=None, stream=None):
+        import torch
+        m = x.shape[0]
+        if y is None:
+            y = torch.empty((m, self.cfg.d_out), dtype=self.y_torch_dtype, device=x.device)
+        eora_linear_forward(self.handle, x, m, y, stream)
+        return y
+
+    def forward_host(self, x_host, y_host, stream=None):
+        eora_linear_forward_host(self.handle, x_host, x_host.shape[0], y_host, stream)
+        return y_host
+
+    def path(self, m: int) -> int:
+        return eora_linear_path(self.handle, m)
+
+    def launches(self, m: int) -> int:
+        return eora_linear_launches(self.handle, m)
+
+    def dump(self, what: int):
+        import torch
+        c = self.cfg
+        shape, dt = {0: ((c.d_in, c.d_out), torch.int32), 1: ((c.d_in, c.d_out), torch.float32),
+                     2: ((c.d_in, c.rank), torch.float32), 3: ((c.rank, c.d_out), torch.float32)}[what]
+        out = torch.empty(shape, dtype=dt, device=self.device)
+        eora_linear_dump(self.handle, what, out)
+        return out
+
+    def device_status(self) -> int:
+        return eora_linear_last_device_status(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            eora_linear_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

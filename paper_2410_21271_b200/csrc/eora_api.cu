@@ -1,0 +1,282 @@
+// C ABI of libeora_linear (declared in include/eora_linear.h): argument checking, memory
+// ownership and dispatch.  All arithmetic of the layer lives in the kernels of the other files.
+#include <new>
+#include "eora_common.cuh"
+
+using namespace eora;
+
+struct eora_linear {
+  Handle h;
+};
+
+namespace {
+
+inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Carve {
+  char* base;
+  int64_t off;
+  template <typename T>
+  T* take(int64_t bytes) {
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += align_up(bytes, 256);
+    return p;
+  }
+};
+
+void wmat_shape(WMat& m, int fmt, int rows, int k_red, int group) {
+  m.fmt = fmt;
+  m.n_rows = (int)align_up(rows, 16);
+  m.k_red = (int)align_up(k_red, 64);
+  m.group = group > 0 ? group : m.k_red;
+  if (m.group > m.k_red) m.group = m.k_red;
+  m.nt = m.n_rows / 16;
+  m.kc = m.k_red / 64;
+  m.ng = m.k_red / m.group;
+  m.q = nullptr; m.q2 = nullptr; m.sc = nullptr; m.zz = nullptr;
+}
+
+void wmat_carve(WMat& m, Carve& c) {
+  if (m.fmt == FMT_NONE) return;
+  m.q = c.take<void>(wmat_q_bytes(m.fmt, m.nt, m.kc));
+  if (wmat_q2_bytes(m.fmt, m.nt, m.kc)) m.q2 = c.take<uint32_t>(wmat_q2_bytes(m.fmt, m.nt, m.kc));
+  if (m.fmt == FMT_Q4 || m.fmt == FMT_Q3 || m.fmt == FMT_Q8) {
+    m.sc = c.take<uint32_t>((int64_t)m.nt * m.ng * 8 * 4);
+    m.zz = c.take<uint16_t>((int64_t)m.nt * m.ng * 8 * 2);
+  }
+}
+
+int check_config(const eora_linear_config& c) {
+  if (c.d_in <= 0 || c.d_out <= 0 || c.rank < 0 || c.max_m < 1) return EORA_ERR_BAD_SHAPE;
+  if (c.d_in % 128 || c.d_out % 32 || c.rank % 8) return EORA_ERR_BAD_SHAPE;
+  if (c.w_format == EORA_W_QUANT) {
+    if (c.w_bits != 3 && c.w_bits != 4) return EORA_ERR_UNSUPPORTED;
+    if (c.w_group <= 0 || c.w_group % 64 || c.d_in % c.w_group) return EORA_ERR_BAD_SHAPE;
+  } else if (c.w_format != EORA_W_SPARSE24) {
+    return EORA_ERR_UNSUPPORTED;
+  }
+  if (c.ab_format != EORA_AB_F16 && c.ab_format != EORA_AB_Q4 && c.ab_format != EORA_AB_Q8) return EORA_ERR_UNSUPPORTED;
+  if (c.rank > 0 && c.ab_format == EORA_AB_Q4) {
+    if (c.rank % 64 || c.ab_group <= 0 || c.ab_group % 64 || c.d_in % c.ab_group) return EORA_ERR_BAD_SHAPE;
+    int gb = c.ab_group < c.rank ? c.ab_group : c.rank;
+    if (c.rank % gb) return EORA_ERR_BAD_SHAPE;
+  }
+  if (c.x_dtype != EORA_X_F16 && c.x_dtype != EORA_X_BF16) return EORA_ERR_UNSUPPORTED;
+  if (c.y_dtype != EORA_Y_F16 && c.y_dtype != EORA_Y_BF16 && c.y_dtype != EORA_Y_F32) return EORA_ERR_UNSUPPORTED;
+  if (c.kernel_policy != EORA_POLICY_AUTO && c.kernel_policy != EORA_POLICY_GENERIC) return EORA_ERR_UNSUPPORTED;
+  return EORA_OK;
+}
+
+int y_elem_bytes(int y_dtype) { return y_dtype == EORA_Y_F32 ? 4 : 2; }
+
+int pick_path(const Handle* h, int m) {
+  if (h->cfg.kernel_policy == EORA_POLICY_GENERIC) return EORA_PATH_GENERIC;
+  if (m <= 64 && decode_supported(h, m)) return EORA_PATH_DECODE;
+  if (m > 64 && prefill_supported(h, m)) return EORA_PATH_PREFILL;
+  return EORA_PATH_GENERIC;
+}
+
+}  // namespace
+
+extern "C" {
+
+int eora_version(void) { return 100; }
+
+const char* eora_status_string(int s) {
+  switch (s) {
+    case EORA_OK: return "ok";
+    case EORA_ERR_NULL_ARG: return "null argument";
+    case EORA_ERR_BAD_SHAPE: return "bad shape";
+    case EORA_ERR_UNSUPPORTED: return "unsupported format or option";
+    case EORA_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+    case EORA_ERR_M_TOO_LARGE: return "m exceeds max_m";
+    case EORA_ERR_CUDA: return "CUDA runtime error";
+    case EORA_ERR_DEVICE_TIMEOUT: return "bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights* wts, void* stream, eora_linear_t* out) {
+  if (out) *out = nullptr;
+  if (!cfg || !wts || !out) return EORA_ERR_NULL_ARG;
+  int st = check_config(*cfg);
+  if (st != EORA_OK) return st;
+  const eora_linear_config& c = *cfg;
+  bool quant_w = c.w_format == EORA_W_QUANT;
+  if (!wts->w_codes || !wts->w_zeros || (quant_w && !wts->w_scales)) return EORA_ERR_NULL_ARG;
+  if (!aligned16(wts->w_codes) || !aligned16(wts->w_zeros) || !aligned16(wts->w_scales)) return EORA_ERR_MISALIGNED;
+  if (c.rank > 0) {
+    if (!wts->a || !wts->b) return EORA_ERR_NULL_ARG;
+    if (!aligned16(wts->a) || !aligned16(wts->b)) return EORA_ERR_MISALIGNED;
+    if (c.ab_format != EORA_AB_F16) {
+      if (!wts->a_scales || !wts->a_zeros || !wts->b_scales || !wts->b_zeros) return EORA_ERR_NULL_ARG;
+      if (!aligned16(wts->a_scales) || !aligned16(wts->a_zeros) || !aligned16(wts->b_scales) || !aligned16(wts->b_zeros))
+        return EORA_ERR_MISALIGNED;
+    }
+  }
+
+  eora_linear* obj = new (std::nothrow) eora_linear();
+  if (!obj) return EORA_ERR_CUDA;
+  Handle* h = &obj->h;
+  *h = Handle();
+  h->cfg = c;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  auto fail = [&](int code) {
+    if (h->prefill_state) prefill_free(h);
+    if (h->weight_mem) cudaFree(h->weight_mem);
+    if (h->scratch_mem) cudaFree(h->scratch_mem);
+    delete obj;
+    return code;
+  };
+  if (cudaGetDevice(&h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
+
+  h->r_pad = (int)align_up(c.rank, 64);
+  int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : FMT_Q8;
+  wmat_shape(h->w, quant_w ? (c.w_bits == 4 ? FMT_Q4 : FMT_Q3) : FMT_SP24, c.d_out, c.d_in, quant_w ? c.w_group : 0);
+  if (c.rank > 0) {
+    int ga = c.ab_format == EORA_AB_Q4 ? c.ab_group : 0;
+    int gb = c.ab_format == EORA_AB_Q4 ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 0;
+    wmat_shape(h->a, ab_fmt, h->r_pad, c.d_in, ga);
+    wmat_shape(h->b, ab_fmt, c.d_out, h->r_pad, gb);
+  } else {
+    wmat_shape(h->a, FMT_NONE, 0, 0, 0);
+    wmat_shape(h->b, FMT_NONE, 0, 0, 0);
+  }
+
+  // ---- weights: one allocation
+  Carve sizing{nullptr, 0};
+  { WMat tw = h->w, ta = h->a, tb = h->b; wmat_carve(tw, sizing); wmat_carve(ta, sizing); wmat_carve(tb, sizing); }
+  h->weight_bytes = sizing.off;
+  if (cudaMalloc(&h->weight_mem, (size_t)h->weight_bytes) != cudaSuccess) { h->weight_mem = nullptr; return fail(EORA_ERR_CUDA); }
+  Carve wc{reinterpret_cast<char*>(h->weight_mem), 0};
+  wmat_carve(h->w, wc); wmat_carve(h->a, wc); wmat_carve(h->b, wc);
+
+  // ---- scratch: one allocation, zero-initialised
+  decode_make_plan(h);
+  int m_dec = c.max_m < 64 ? c.max_m : 64;
+  int64_t n_counters = h->w.nt + h->a.nt + 64;
+  for (int pass = 0; pass < 2; ++pass) {
+    Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
+    h->t_ws = sc.take<float>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 4);
+    h->y_ws = sc.take<float>((int64_t)m_dec * c.d_out * 4);
+    h->t16 = sc.take<__half>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 2);
+    h->counters = sc.take<uint32_t>(n_counters * 4);
+    h->dev_status = sc.take<int>(256);
+    h->x_stage = sc.take<void>((int64_t)c.max_m * c.d_in * 2);
+    h->y_stage = sc.take<void>((int64_t)c.max_m * c.d_out * y_elem_bytes(c.y_dtype));
+    if (pass == 0) {
+      h->scratch_bytes = sc.off;
+      if (cudaMalloc(&h->scratch_mem, (size_t)h->scratch_bytes) != cudaSuccess) { h->scratch_mem = nullptr; return fail(EORA_ERR_CUDA); }
+    }
+  }
+  if (cudaMemsetAsync(h->scratch_mem, 0, (size_t)h->scratch_bytes, s) != cudaSuccess) return fail(EORA_ERR_CUDA);
+
+  // ---- re-tile
+  cudaError_t e = cudaSuccess;
+  if (quant_w) e = launch_repack_quant(h->w, wts->w_codes, wts->w_scales, wts->w_zeros, c.w_bits, c.d_out, c.d_in, s);
+  else e = launch_repack_sp24(h->w, wts->w_codes, wts->w_zeros, c.d_out, c.d_in, s);
+  if (e == cudaSuccess && c.rank > 0) {
+    if (c.ab_format == EORA_AB_F16) {
+      e = launch_repack_f16(h->a, wts->a, c.rank, c.d_in, s);
+      if (e == cudaSuccess) e = launch_repack_f16(h->b, wts->b, c.d_out, c.rank, s);
+    } else if (c.ab_format == EORA_AB_Q4) {
+      e = launch_repack_quant(h->a, wts->a, wts->a_scales, wts->a_zeros, 4, c.rank, c.d_in, s);
+      if (e == cudaSuccess) e = launch_repack_quant(h->b, wts->b, wts->b_scales, wts->b_zeros, 4, c.d_out, c.rank, s);
+    } else {
+      e = launch_repack_q8(h->a, wts->a, wts->a_scales, wts->a_zeros, c.rank, c.d_in, s);
+      if (e == cudaSuccess) e = launch_repack_q8(h->b, wts->b, wts->b_scales, wts->b_zeros, c.d_out, c.rank, s);
+    }
+  }
+  if (e != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (prefill_init(h) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  *out = obj;
+  return EORA_OK;
+}
+
+int eora_linear_destroy(eora_linear_t obj) {
+  if (!obj) return EORA_OK;
+  Handle* h = &obj->h;
+  int rc = EORA_OK;
+  if (h->prefill_state) prefill_free(h);
+  if (h->weight_mem && cudaFree(h->weight_mem) != cudaSuccess) rc = EORA_ERR_CUDA;
+  if (h->scratch_mem && cudaFree(h->scratch_mem) != cudaSuccess) rc = EORA_ERR_CUDA;
+  delete obj;
+  return rc;
+}
+
+int eora_linear_path(eora_linear_t obj, int32_t m) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (m < 1) return EORA_ERR_BAD_SHAPE;
+  if (m > obj->h.cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  return pick_path(&obj->h, m);
+}
+
+int eora_linear_launches(eora_linear_t obj, int32_t m) {
+  int p = eora_linear_path(obj, m);
+  if (p < 0) return p;
+  if (p == EORA_PATH_DECODE) return decode_launch_count(&obj->h, m);
+  if (p == EORA_PATH_PREFILL) return prefill_launch_count(&obj->h, m);
+  return generic_launch_count(&obj->h);
+}
+
+int eora_linear_forward(eora_linear_t obj, const void* x, int32_t m, void* y, void* stream) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (m == 0) return EORA_OK;
+  if (m < 0) return EORA_ERR_BAD_SHAPE;
+  if (!x || !y) return EORA_ERR_NULL_ARG;
+  if (!aligned16(x) || !aligned16(y)) return EORA_ERR_MISALIGNED;
+  Handle* h = &obj->h;
+  if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int p = pick_path(h, m);
+  cudaError_t e;
+  if (p == EORA_PATH_DECODE) e = launch_decode_forward(h, x, m, y, s);
+  else if (p == EORA_PATH_PREFILL) e = launch_prefill_forward(h, x, m, y, s);
+  else e = launch_generic_forward(h, x, m, y, s);
+  return e == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
+}
+
+int eora_linear_forward_host(eora_linear_t obj, const void* x_host, int32_t m, void* y_host, void* stream) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (m == 0) return EORA_OK;
+  if (m < 0) return EORA_ERR_BAD_SHAPE;
+  if (!x_host || !y_host) return EORA_ERR_NULL_ARG;
+  Handle* h = &obj->h;
+  if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  size_t xb = (size_t)m * h->cfg.d_in * 2, yb = (size_t)m * h->cfg.d_out * y_elem_bytes(h->cfg.y_dtype);
+  if (cudaMemcpyAsync(h->x_stage, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EORA_ERR_CUDA;
+  int rc = eora_linear_forward(obj, h->x_stage, m, h->y_stage, stream);
+  if (rc != EORA_OK) return rc;
+  if (cudaMemcpyAsync(y_host, h->y_stage, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EORA_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return EORA_ERR_CUDA;
+  return EORA_OK;
+}
+
+int eora_linear_dump(eora_linear_t obj, int32_t what, void* outp, void* stream) {
+  if (!obj || !outp) return EORA_ERR_NULL_ARG;
+  Handle* h = &obj->h;
+  if (what < 0 || what > 3) return EORA_ERR_UNSUPPORTED;
+  if (what == 0 && h->cfg.w_format != EORA_W_QUANT) return EORA_ERR_UNSUPPORTED;
+  if (what >= 2 && h->cfg.rank == 0) return EORA_ERR_BAD_SHAPE;
+  return launch_dump(h, what, outp, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
+}
+
+int eora_linear_last_device_status(eora_linear_t obj) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  int v = 0;
+  if (cudaMemcpy(&v, obj->h.dev_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EORA_ERR_CUDA;
+  if (v != 0) {
+    int z = 0;
+    if (cudaMemcpy(obj->h.dev_status, &z, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return EORA_ERR_CUDA;
+  }
+  return v;
+}
+
+int64_t eora_linear_weight_bytes(eora_linear_t obj) { return obj ? obj->h.weight_bytes : 0; }
+int64_t eora_linear_scratch_bytes(eora_linear_t obj) { return obj ? obj->h.scratch_bytes : 0; }
+
+}  // extern "C"
