@@ -1,0 +1,160 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Integer work (unpack) and dequantisation are compared bit for bit; outputs within
+rel. Frobenius <= 2e-3 and max|diff| <= 1e-2 * max|y| of the float64 oracle."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from oracle import eora_oracle as orc
+import eora_inputs as gen
+import paper_2410_21271_b200 as eora
+from helpers import make_case, run_layer, check_parity, x_to_torch
+
+
+# --------------------------------------------------------------------------- a1 / a2 bit-exact
+@pytest.mark.parametrize("w,K,N,group", [("q4", 256, 64, 128), ("q3", 256, 64, 128), ("q4", 512, 96, 64),
+                                         ("q3", 384, 32, 384), ("q4", 4096, 1024, 128), ("q3", 4096, 1024, 128)])
+def test_unpack_and_dequant_bit_exact(w, K, N, group):
+    wf, _, _ = make_case(11, K, N, 0, w=w, group=group)
+    L = eora.Layer(wf, None, None, max_m=1)
+    codes = L.dump(0).cpu().numpy()
+    q = orc.unpack_codes(wf["codes"], wf["bits"], K)
+    assert np.array_equal(codes, q)
+    deq = L.dump(1).cpu().numpy()
+    z = orc.unpack_zeros(wf["zeros"], wf["bits"], N)
+    assert np.array_equal(deq, orc.deq_fp32(q, z, wf["scales"], group))
+    L.close()
+
+
+@pytest.mark.parametrize("ab,r", [("f16", 64), ("f16", 24), ("q4", 64), ("q4", 256), ("q8", 64), ("q8", 40)])
+def test_adapter_storage_bit_exact(ab, r):
+    K, N = 256, 96
+    wf, af, bf = make_case(12, K, N, r, ab=ab)
+    L = eora.Layer(wf, af, bf, max_m=1)
+    A = L.dump(2).cpu().numpy().astype(np.float64)
+    B = L.dump(3).cpu().numpy().astype(np.float64)
+    assert np.array_equal(A, orc.dequant_matrix(af).astype(np.float32).astype(np.float64))
+    assert np.array_equal(B, orc.dequant_matrix(bf).astype(np.float32).astype(np.float64))
+    L.close()
+
+
+def test_sparse24_expansion_bit_exact():
+    K, N = 256, 64
+    wf, _, _ = make_case(13, K, N, 0, w="sp24")
+    L = eora.Layer(wf, None, None, max_m=1)
+    assert np.array_equal(L.dump(1).cpu().numpy().astype(np.float64), orc.dequant_matrix(wf))
+    L.close()
+
+
+# --------------------------------------------------------------------------- forward parity
+SMALL = [
+    # w, ab, K, N, r, M, x_dtype
+    ("q4", "f16", 256, 64, 64, 1, "f16"),
+    ("q4", "f16", 512, 96, 128, 3, "f16"),
+    ("q3", "f16", 384, 160, 64, 8, "f16"),
+    ("q3", "f16", 1024, 224, 128, 16, "bf16"),
+    ("q4", "f16", 256, 64, 0, 5, "f16"),
+    ("q4", "f16", 256, 64, 24, 7, "f16"),
+    ("q4", "q4", 512, 96, 128, 1, "f16"),
+    ("q4", "q4", 512, 96, 512, 16, "f16"),
+    ("q4", "q8", 512, 96, 128, 64, "f16"),
+    ("q4", "q8", 256, 64, 40, 2, "f16"),
+    ("sp24", "f16", 512, 96, 128, 1, "f16"),
+    ("sp24", "f16", 256, 64, 64, 9, "bf16"),
+    ("q4", "f16", 1152, 352, 128, 63, "f16"),
+    ("q3", "f16", 1152, 352, 128, 65, "f16"),
+    ("q4", "f16", 640, 160, 64, 200, "f16"),
+    ("q4", "f16", 1024, 512, 128, 300, "bf16"),
+]
+
+
+@pytest.mark.parametrize("policy", [eora.EORA_POLICY_GENERIC, eora.EORA_POLICY_AUTO])
+@pytest.mark.parametrize("w,ab,K,N,r,M,xd", SMALL)
+def test_forward_matches_oracle_small(policy, w, ab, K, N, r, M, xd):
+    wf, af, bf = make_case(21, K, N, r, w=w, ab=ab)
+    x = gen.make_x(22, M, K, xd)
+    L = eora.Layer(wf, af, bf, max_m=M, x_dtype=xd, kernel_policy=policy)
+    y = run_layer(L, x, xd)
+    y_ref = orc.forward(x, xd, wf, af, bf)
+    check_parity(y, y_ref, f"{w}/{ab} K{K} N{N} r{r} M{M} path{L.path(M)}")
+    # second call on the same handle: scratch state must have been restored
+    y2 = run_layer(L, x, xd)
+    check_parity(y2, y_ref, "second call")
+    L.close()
+
+
+@pytest.mark.parametrize("yd", ["f16", "bf16", "f32"])
+def test_output_dtypes(yd):
+    K, N, r, M = 512, 96, 64, 4
+    wf, af, bf = make_case(23, K, N, r)
+    x = gen.make_x(24, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M, y_dtype=yd)
+    y = run_layer(L, x, "f16")
+    rel, _ = orc.parity_errors(y, orc.forward(x, "f16", wf, af, bf))
+    # bf16 output alone costs ~1.7e-3 of the 2e-3 budget; fp16/fp32 outputs are far inside it
+    assert rel <= (2e-3 if yd == "bf16" else 6e-4)
+    L.close()
+
+
+@pytest.mark.parametrize("w", ["q4", "q3"])
+def test_one_hot_rows_read_back_exact_weights(w):
+    """X = e_k, rank 0, fp32 output: y[n] is a single product, so the fast path's own unpack and
+    dequantisation are checked bit for bit against the oracle."""
+    K, N = 512, 96
+    wf, _, _ = make_case(25, K, N, 0, w=w)
+    ks = [0, 1, 10, 21, 63, 64, 127, 128, 300, 511]
+    x = np.zeros((len(ks), K), dtype=np.float16)
+    for i, k in enumerate(ks):
+        x[i, k] = 1.0
+    L = eora.Layer(wf, None, None, max_m=len(ks), y_dtype="f32")
+    y = run_layer(L, x, "f16")
+    q = orc.unpack_codes(wf["codes"], wf["bits"], K); z = orc.unpack_zeros(wf["zeros"], wf["bits"], N)
+    W = orc.deq_fp32(q, z, wf["scales"], 128).astype(np.float64)
+    assert np.array_equal(y, W[ks])
+    L.close()
+
+
+def test_forward_argument_errors():
+    import torch
+    K, N = 256, 64
+    wf, af, bf = make_case(26, K, N, 64)
+    L = eora.Layer(wf, af, bf, max_m=4)
+    x = torch.zeros((8, K), dtype=torch.float16, device="cuda:0")
+    y = torch.zeros((8, N), dtype=torch.float16, device="cuda:0")
+    assert eora.eora_linear_forward(L.handle, x, 0, y, check=False) == eora.EORA_OK
+    assert eora.eora_linear_forward(L.handle, x, 5, y, check=False) == eora.EORA_ERR_M_TOO_LARGE
+    assert eora.eora_linear_forward(L.handle, x, -1, y, check=False) == eora.EORA_ERR_BAD_SHAPE
+    assert eora.eora_linear_forward(L.handle, None, 1, y, check=False) == eora.EORA_ERR_NULL_ARG
+    assert eora.eora_linear_forward(L.handle, x.data_ptr() + 2, 1, y, check=False) == eora.EORA_ERR_MISALIGNED
+    assert eora.eora_linear_path(L.handle, 5) == eora.EORA_ERR_M_TOO_LARGE
+    assert eora.eora_linear_weight_bytes(L.handle) > 0 and eora.eora_linear_scratch_bytes(L.handle) > 0
+    torch.cuda.synchronize()
+    L.close()
+
+
+def test_forward_host_roundtrip():
+    import torch
+    K, N, r, M = 512, 96, 64, 3
+    wf, af, bf = make_case(27, K, N, r)
+    x = gen.make_x(28, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.empty((M, N), dtype=torch.float16).pin_memory()
+    L.forward_host(xh, yh)
+    check_parity(yh.float().numpy().astype(np.float64), orc.forward(x, "f16", wf, af, bf), "forward_host")
+    L.close()
+
+
+def test_adapter_off_equals_rank0_and_linearity():
+    """Toggling the adapter off restores the plain compressed layer (rank 0 = zero adapter)."""
+    K, N, M = 512, 96, 4
+    wf, af, bf = make_case(29, K, N, 64)
+    x = gen.make_x(30, M, K)
+    L0 = eora.Layer(wf, None, None, max_m=M, y_dtype="f32")
+    zA = {"kind": "f16", "data": np.zeros_like(af["data"])}
+    Lz = eora.Layer(wf, zA, bf, max_m=M, y_dtype="f32")
+    y0, yz = run_layer(L0, x, "f16"), run_layer(Lz, x, "f16")
+    assert np.allclose(y0, yz, rtol=0, atol=1e-6 * np.abs(y0).max())
+    L0.close(); Lz.close()
