@@ -153,6 +153,17 @@ int eora_linear_dump(eora_linear_t h, int32_t what, void* out, void* stream);
  */
 int eora_linear_last_device_status(eora_linear_t h);
 
+/*
+ * Diagnostics of the decode kernel.  eora_linear_decode_grid: how many CTAs forward(m) launches
+ * (0 if m is not served by the decode family).  eora_linear_set_trace: give the handle a device
+ * buffer of 16 x uint64 per CTA (or NULL to switch tracing off); every decode forward then
+ * records, per CTA, %globaltimer nanoseconds at fixed points of the kernel (0 start, 1 weight
+ * copies issued, 2 dependency wait over, 3 X staged, 4 own slice done, 5 t available, 6 t staged,
+ * 7 B extension done, 8 warps summed, 9 end).  The buffer is caller-owned.
+ */
+int eora_linear_decode_grid(eora_linear_t h, int32_t m);
+int eora_linear_set_trace(eora_linear_t h, void* trace_buf);
+
 /* Bytes of device memory the handle owns: re-tiled weights, and scratch. */
 int64_t eora_linear_weight_bytes(eora_linear_t h);
 int64_t eora_linear_scratch_bytes(eora_linear_t h);

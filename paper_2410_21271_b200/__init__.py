@@ -70,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.eora_linear_dump.restype = c_int
         L.eora_linear_last_device_status.argtypes = [c_void_p]
         L.eora_linear_last_device_status.restype = c_int
+        L.eora_linear_set_trace.argtypes = [c_void_p, c_void_p]
+        L.eora_linear_set_trace.restype = c_int
+        L.eora_linear_decode_grid.argtypes = [c_void_p, c_int32]
+        L.eora_linear_decode_grid.restype = c_int
         L.eora_linear_weight_bytes.argtypes = [c_void_p]
         L.eora_linear_weight_bytes.restype = c_int64
         L.eora_linear_scratch_bytes.argtypes = [c_void_p]
@@ -162,6 +166,14 @@ def eora_linear_dump(handle: int, what: int, out, stream=None) -> int:
 
 def eora_linear_last_device_status(handle: int) -> int:
     return lib().eora_linear_last_device_status(handle)
+
+
+def eora_linear_set_trace(handle: int, buf) -> int:
+    return lib().eora_linear_set_trace(handle, _ptr(buf))
+
+
+def eora_linear_decode_grid(handle: int, m: int) -> int:
+    return lib().eora_linear_decode_grid(handle, int(m))
 
 
 def eora_linear_weight_bytes(handle: int) -> int:

@@ -6,20 +6,23 @@
 // elements of the backbone product with t in the place of X, so Y is written exactly once.
 //
 // Work decomposition.  A CTA (8 warps) owns one unit = (matrix, 16-row tile, reduction slice).
-// Units of A come first in blockIdx order, backbone units after them.  Inside a unit each warp
-// streams whole quantisation quanta (<= 128 reduction elements sharing one scale / zero-point)
-// of packed weights with 128-bit loads, turns the codes into exact fp16 integers (q - z) in
-// registers, multiplies them with the activations on the tensor cores (mma.m16n8k16, weights as
-// the 16-row operand, fp32 accumulate) and applies the scale once per quantum in fp32.
-// The 8 warps are then summed through shared memory.
+// Units of A come first in blockIdx order, backbone units after them.  The packed weights of a
+// unit are one contiguous byte range; one thread brings them into shared memory with a few bulk
+// async copies (cp.async.bulk + mbarrier, no multicast) issued at the very start of the CTA, so
+// a whole layer is in flight at once and no registers are spent on prefetch.  Each warp then
+// walks its quanta (<= 128 reduction elements sharing one scale / zero-point): codes become the
+// exact fp16 integers (q - z) in registers, are multiplied with the activations on the tensor
+// cores (mma.m16n8k16, weights as the 16-row operand, fp32 accumulate) and the scale is applied
+// once per quantum in fp32.  The 8 warps are then summed through shared memory.
 //   A unit       : adds its partial t to the fp32 buffer t_ws (red.add), then bumps T_DONE.
 //   backbone unit: the last reduction slice of each row tile also owns the B extension: it waits
 //                  (bounded) for T_DONE, reads t, splits it into fp16 hi + lo parts and runs the
-//                  B tiles against them.  With one slice per row tile the result goes straight
-//                  to Y; otherwise slices add into y_ws and the last one to arrive converts.
+//                  B tiles (prefetched with the weights) against them.  With one slice per row
+//                  tile the result goes straight to Y; otherwise slices add into y_ws and the
+//                  last one to arrive converts.
 // All scratch words are returned to zero before the kernel ends, so calls need no memset.
 //
-// Programmatic dependent launch: the first batch of weight loads is issued before
+// Programmatic dependent launch: the bulk copies of the weights are issued before
 // griddepcontrol.wait, i.e. while the previous kernel in the stream is still draining;
 // activations and scratch are touched only after it.
 #include "eora_common.cuh"
@@ -29,28 +32,41 @@ namespace {
 
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
-constexpr int kXPad = 32;                // halves of padding per activation row in shared memory
-constexpr int kXSmemBudget = 64 * 1024;  // bytes of staged activations per CTA
+constexpr int kXPad = 32;                 // halves of padding per activation row in shared memory
+constexpr int kChunks = 4;                // bulk-copy chunks (one mbarrier each) per unit
+constexpr int kUnitBytes = 32 * 1024;     // largest packed-weight slice of one unit
+constexpr int kXSmemBudget = 64 * 1024;   // bytes of staged activations per CTA
+constexpr int kMaxSmem = 200 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 21;
 
 enum { CNT_T_DONE = 0, CNT_T_CONSUMED = 1, CNT_TILE0 = 2 };
 
-// ------------------------------------------------------------------------------------------ loads
-__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
+// ------------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ uint2 ldg_stream(const uint2* p) {
-  uint2 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
-  return v;
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ uint32_t ldg_stream(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
-  return v;
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false (and latches the status word) if the copy never lands.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* dev_status) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+  }
+  atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
+  return false;
+}
+// global -> shared bulk copy of `bytes` (multiple of 16; both addresses 16-byte aligned)
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
   uint32_t v;
@@ -65,31 +81,6 @@ __device__ __forceinline__ float ld_cg(const float* p) {
 __device__ __forceinline__ void red_add(float* p, float v) {
   asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
-
-template <int FMT> struct TileRegs;
-template <> struct TileRegs<FMT_Q4> { uint4 v; };
-template <> struct TileRegs<FMT_Q3> { uint2 v; uint32_t w2; };
-template <> struct TileRegs<FMT_Q8> { uint4 v[2]; };
-template <> struct TileRegs<FMT_F16> { uint4 v[4]; };
-template <> struct TileRegs<FMT_NONE> { int unused; };
-
-template <int FMT>
-__device__ __forceinline__ void tile_load(TileRegs<FMT>& r, const WMat& m, int64_t ti, int lane) {
-  if constexpr (FMT == FMT_Q4) {
-    r.v = ldg_stream(reinterpret_cast<const uint4*>(m.q) + ti * 32 + lane);
-  } else if constexpr (FMT == FMT_Q3) {
-    r.v = ldg_stream(reinterpret_cast<const uint2*>(m.q) + ti * 32 + lane);
-    r.w2 = ldg_stream(m.q2 + ti * 32 + lane);
-  } else if constexpr (FMT == FMT_Q8) {
-    r.v[0] = ldg_stream(reinterpret_cast<const uint4*>(m.q) + (ti * 2 + 0) * 32 + lane);
-    r.v[1] = ldg_stream(reinterpret_cast<const uint4*>(m.q) + (ti * 2 + 1) * 32 + lane);
-  } else if constexpr (FMT == FMT_F16) {
-#pragma unroll
-    for (int p = 0; p < 4; ++p) r.v[p] = ldg_stream(reinterpret_cast<const uint4*>(m.q) + (ti * 4 + p) * 32 + lane);
-  }
-}
-
-// ------------------------------------------------------------------------------------------ dequant
 __device__ __forceinline__ uint32_t h2sub(uint32_t a, uint32_t b) {
   uint32_t d;
   asm("sub.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
@@ -100,9 +91,15 @@ __device__ __forceinline__ uint32_t h2fma(uint32_t a, uint32_t b, uint32_t c) {
   asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
+// ------------------------------------------------------------------------------------------ dequant
 // Per-quantum constants of the two rows a lane owns: fp16x2 values that turn the magic-number
-// form of a code into the exact integer q - z.
+// form of a code (1024 + q * 2^s as fp16) into the exact integer q - z.
 struct ZC { uint32_t c[2][3]; };
 
 template <int FMT>
@@ -121,11 +118,15 @@ __device__ __forceinline__ void make_zc(ZC& zc, uint32_t zz) {
 
 constexpr uint32_t kMagic = 0x64006400u;   // fp16x2 (1024, 1024)
 
-// a[i][*]: the A-operand registers of mma i (i = 2*blk + sub) for this lane; entries are fp16x2.
+template <int FMT> constexpr bool is_quant() { return FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8; }
+
+// Build the A-operand registers of the four mma of one tile from its blob in shared memory.
+// a[i][*]: mma i = 2*blk + sub; entries are fp16x2.
 template <int FMT>
-__device__ __forceinline__ void tile_frags(const TileRegs<FMT>& r, const ZC& zc, uint32_t (&a)[4][4]) {
+__device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const ZC& zc, uint32_t (&a)[4][4]) {
   if constexpr (FMT == FMT_Q4) {
-    const uint32_t w[4] = {r.v.x, r.v.y, r.v.z, r.v.w};
+    const uint4 v = *reinterpret_cast<const uint4*>(blob + lane * 16);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int part = 0; part < 4; ++part) {
       const int hf = part & 1, blk = part >> 1;
@@ -138,8 +139,10 @@ __device__ __forceinline__ void tile_frags(const TileRegs<FMT>& r, const ZC& zc,
       a[blk * 2 + 1][hf + 2] = h2fma(h3, 0x2C002C00u, zc.c[hf][1]);
     }
   } else if constexpr (FMT == FMT_Q3) {
-    const uint32_t w[3] = {r.v.x, r.v.y, r.w2};
-    const uint32_t ws[3] = {r.v.x >> 9, r.v.y >> 9, r.w2 >> 9};
+    const uint2 v01 = *reinterpret_cast<const uint2*>(blob + lane * 8);
+    const uint32_t v2 = *reinterpret_cast<const uint32_t*>(blob + 256 + lane * 4);
+    const uint32_t w[3] = {v01.x, v01.y, v2};
+    const uint32_t ws[3] = {v01.x >> 9, v01.y >> 9, v2 >> 9};
 #pragma unroll
     for (int p = 0; p < 16; ++p) {
       const int part = p >> 2, j = p & 3, hf = part & 1, blk = part >> 1;
@@ -161,117 +164,106 @@ __device__ __forceinline__ void tile_frags(const TileRegs<FMT>& r, const ZC& zc,
     }
   } else if constexpr (FMT == FMT_Q8) {
 #pragma unroll
-    for (int part = 0; part < 4; ++part) {
-      const int hf = part & 1, blk = part >> 1;
-      const uint4 u = r.v[part >> 1];
-      const uint32_t w0 = (part & 1) ? u.z : u.x, w1 = (part & 1) ? u.w : u.y;
-      a[blk * 2 + 0][hf] = h2sub((w0 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-      a[blk * 2 + 0][hf + 2] = h2sub(((w0 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-      a[blk * 2 + 1][hf] = h2sub((w1 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-      a[blk * 2 + 1][hf + 2] = h2sub(((w1 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+    for (int pl = 0; pl < 2; ++pl) {
+      const uint4 u = *reinterpret_cast<const uint4*>(blob + pl * 512 + lane * 16);
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const uint32_t w0 = hf ? u.z : u.x, w1 = hf ? u.w : u.y;
+        a[pl * 2 + 0][hf] = h2sub((w0 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[pl * 2 + 0][hf + 2] = h2sub(((w0 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[pl * 2 + 1][hf] = h2sub((w1 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[pl * 2 + 1][hf + 2] = h2sub(((w1 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+      }
     }
   } else if constexpr (FMT == FMT_F16) {
 #pragma unroll
     for (int part = 0; part < 4; ++part) {
       const int hf = part & 1, blk = part >> 1;
-      a[blk * 2 + 0][hf] = r.v[part].x;
-      a[blk * 2 + 0][hf + 2] = r.v[part].y;
-      a[blk * 2 + 1][hf] = r.v[part].z;
-      a[blk * 2 + 1][hf + 2] = r.v[part].w;
+      const uint4 u = *reinterpret_cast<const uint4*>(blob + part * 512 + lane * 16);
+      a[blk * 2 + 0][hf] = u.x;
+      a[blk * 2 + 0][hf + 2] = u.y;
+      a[blk * 2 + 1][hf] = u.z;
+      a[blk * 2 + 1][hf + 2] = u.w;
     }
   }
 }
 
-__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-template <int FMT> constexpr bool is_quant() { return FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8; }
-template <int FMT> constexpr int prefetch_quanta() { return FMT == FMT_F16 ? 2 : 4; }
-
-// Stream the quanta [q0, q1) of row tile `tile` of matrix `m` against NX activation sources held in
-// shared memory (source s at xs + s * xsrc_stride; row `token` at + token * xrow; the element for
-// reduction index k at + (k - k_base)).  QT = tiles per quantum.  Quanta are dealt round-robin to
-// the warps.  `pre` / `have_pre`: the first batch, already loaded by the caller.
-template <int FMT, int MT, int QT, int NX>
-struct Streamer {
-  static constexpr int PF = prefetch_quanta<FMT>();
-  TileRegs<FMT> regs[PF][QT];
-  uint32_t sc[PF];
-  uint32_t zz[PF];
-
-  __device__ __forceinline__ void issue(const WMat& m, int tile, int qfirst, int q1, int warp, int lane) {
-#pragma unroll
-    for (int j = 0; j < PF; ++j) {
-      int qi = qfirst + warp + kWarps * j;
-      if (qi < q1) {
-#pragma unroll
-        for (int tt = 0; tt < QT; ++tt) tile_load<FMT>(regs[j][tt], m, (int64_t)tile * m.kc + (int64_t)qi * QT + tt, lane);
-        if constexpr (is_quant<FMT>()) {
-          int grp = (qi * QT * 64) / m.group;
-          int64_t si = ((int64_t)tile * m.ng + grp) * 8 + (lane >> 2);
-          sc[j] = __ldg(m.sc + si);
-          zz[j] = __ldg(m.zz + si);
-        }
-      }
-    }
-  }
-
-  __device__ __forceinline__ void compute(int qfirst, int q1, int warp, int lane, const __half* xs, int xrow,
-                                          int xsrc_stride, int k_base, int m_rows, float (&acc)[MT][4]) {
-    const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-    for (int j = 0; j < PF; ++j) {
-      int qi = qfirst + warp + kWarps * j;
-      if (qi < q1) {
-        float gacc[MT][4];
-        if constexpr (is_quant<FMT>()) {
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) { gacc[mt][0] = gacc[mt][1] = gacc[mt][2] = gacc[mt][3] = 0.f; }
-        }
-        ZC zc;
-        if constexpr (is_quant<FMT>()) make_zc<FMT>(zc, zz[j]);
-#pragma unroll
-        for (int tt = 0; tt < QT; ++tt) {
-          uint32_t a[4][4];
-          tile_frags<FMT>(regs[j][tt], zc, a);
-          const int koff = (qi * QT + tt) * 64 - k_base + 8 * t;
-#pragma unroll
-          for (int s = 0; s < NX; ++s) {
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-              const int token = mt * 8 + g;
-              uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
-              if (token < m_rows) {
-                const __half* p = xs + s * xsrc_stride + token * xrow + koff;
-                x0 = *reinterpret_cast<const uint4*>(p);
-                x1 = *reinterpret_cast<const uint4*>(p + 32);
-              }
-              float(&d)[4] = is_quant<FMT>() ? gacc[mt] : acc[mt];
-              mma16816(d, a[0], x0.x, x0.y);
-              mma16816(d, a[1], x0.z, x0.w);
-              mma16816(d, a[2], x1.x, x1.y);
-              mma16816(d, a[3], x1.z, x1.w);
-            }
-          }
-        }
-        if constexpr (is_quant<FMT>()) {
-          const float sa = __half2float(__ushort_as_half((unsigned short)(sc[j] & 0xffffu)));
-          const float sb = __half2float(__ushort_as_half((unsigned short)(sc[j] >> 16)));
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            acc[mt][0] = fmaf(sa, gacc[mt][0], acc[mt][0]);
-            acc[mt][1] = fmaf(sa, gacc[mt][1], acc[mt][1]);
-            acc[mt][2] = fmaf(sb, gacc[mt][2], acc[mt][2]);
-            acc[mt][3] = fmaf(sb, gacc[mt][3], acc[mt][3]);
-          }
-        }
-      }
-    }
-  }
+// What one CTA streams: a slice of nq quanta of one row tile, (being) copied to shared memory.
+struct SliceView {
+  const uint8_t* wbuf;      // tile blobs of the slice, first tile of the slice at offset 0
+  const uint32_t* sc;       // scales from the first group the slice touches (8 words per group)
+  const uint16_t* zz;
+  uint64_t* bars;           // kChunks barriers, chunk c covers quanta [c*cq, (c+1)*cq) of the slice
+  int nq;                   // quanta in the slice
+  int qt;                   // tiles per quantum
+  int cq;                   // quanta per chunk
+  int group_tiles;          // tiles per quantisation group
+  int gofs;                 // tiles between the start of that first group and the slice start
 };
+
+// Accumulate the slice against NX activation sources in shared memory (source s at
+// xs + s * xsrc_stride halves; row `token` at + token * xrow; reduction index 0 = slice start).
+template <int FMT, int MT, int NX>
+__device__ __forceinline__ void run_slice(const SliceView& sv, int warp, int lane, const __half* xs, int xrow,
+                                          int xsrc_stride, int m_rows, int* dev_status, float (&acc)[MT][4]) {
+  constexpr int TB = FMT == FMT_Q4 ? 512 : FMT == FMT_Q3 ? 384 : FMT == FMT_Q8 ? 1024 : 2048;
+  const int g = lane >> 2, t = lane & 3;
+  int chunk_ready = -1;
+#pragma unroll 1
+  for (int q = warp; q < sv.nq; q += kWarps) {
+    const int chunk = q / sv.cq;
+    if (chunk > chunk_ready) {
+      mbar_wait(sv.bars + chunk, 0, dev_status);
+      chunk_ready = chunk;
+    }
+    float gacc[MT][4];
+    ZC zc;
+    uint32_t sc2 = 0;
+    if constexpr (is_quant<FMT>()) {
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) gacc[mt][0] = gacc[mt][1] = gacc[mt][2] = gacc[mt][3] = 0.f;
+      const int gi = (sv.gofs + q * sv.qt) / sv.group_tiles;
+      sc2 = sv.sc[gi * 8 + g];
+      make_zc<FMT>(zc, sv.zz[gi * 8 + g]);
+    }
+#pragma unroll 1
+    for (int tt = 0; tt < sv.qt; ++tt) {
+      const int tile = q * sv.qt + tt;
+      uint32_t a[4][4];
+      tile_frags<FMT>(sv.wbuf + tile * TB, lane, zc, a);
+      const int koff = tile * 64 + 8 * t;
+#pragma unroll
+      for (int s = 0; s < NX; ++s) {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const int token = mt * 8 + g;
+          uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
+          if (token < m_rows) {
+            const __half* p = xs + s * xsrc_stride + token * xrow + koff;
+            x0 = *reinterpret_cast<const uint4*>(p);
+            x1 = *reinterpret_cast<const uint4*>(p + 32);
+          }
+          float(&d)[4] = is_quant<FMT>() ? gacc[mt] : acc[mt];
+          mma16816(d, a[0], x0.x, x0.y);
+          mma16816(d, a[1], x0.z, x0.w);
+          mma16816(d, a[2], x1.x, x1.y);
+          mma16816(d, a[3], x1.z, x1.w);
+        }
+      }
+    }
+    if constexpr (is_quant<FMT>()) {
+      const float sa = __half2float(__ushort_as_half((unsigned short)(sc2 & 0xffffu)));
+      const float sb = __half2float(__ushort_as_half((unsigned short)(sc2 >> 16)));
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        acc[mt][0] = fmaf(sa, gacc[mt][0], acc[mt][0]);
+        acc[mt][1] = fmaf(sa, gacc[mt][1], acc[mt][1]);
+        acc[mt][2] = fmaf(sb, gacc[mt][2], acc[mt][2]);
+        acc[mt][3] = fmaf(sb, gacc[mt][3], acc[mt][3]);
+      }
+    }
+  }
+}
 
 struct DecodeArgs {
   WMat w, a, b;
@@ -285,7 +277,17 @@ struct DecodeArgs {
   int x_dtype, y_dtype;
   int a_units, a_split, w_split;
   int qt_w, qt_a, qt_b;     // tiles per quantum of each matrix
+  // shared-memory carve-up (byte offsets from the dynamic shared memory base)
+  int off_sc, off_zz, off_b, off_bsc, off_bzz, off_x, off_red;
+  unsigned long long* trace;   // optional: 16 timestamps (ns) per CTA, see eora_linear_set_trace
 };
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define EORA_TRACE(slot) do { if (p.trace && threadIdx.x == 0) p.trace[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
 
 __device__ __forceinline__ void store_y(void* y, int dtype, int64_t i, float v) {
   if (dtype == EORA_Y_F16) reinterpret_cast<__half*>(y)[i] = __float2half_rn(v);
@@ -296,64 +298,61 @@ __device__ __forceinline__ void store_y(void* y, int dtype, int64_t i, float v) 
 // Stage activation rows [0, m) x reduction range [k0, k0 + len) into shared memory as fp16.
 __device__ __forceinline__ void stage_x(__half* xs, int xrow, const void* x, int x_dtype, int m, int d_in, int k0, int len) {
   const int chunks = len >> 3;   // 16-byte chunks per row
-  for (int i = threadIdx.x; i < m * chunks; i += kThreads) {
-    int row = i / chunks, c = i - row * chunks;
-    uint4 v = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(x) + (int64_t)row * d_in + k0 + c * 8);
-    if (x_dtype == EORA_X_BF16) {
-      uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
+  for (int row = 0; row < m; ++row) {
+    for (int c = threadIdx.x; c < chunks; c += kThreads) {
+      uint4 v = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(x) + (int64_t)row * d_in + k0 + c * 8);
+      if (x_dtype == EORA_X_BF16) {
+        uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        __nv_bfloat162 b2 = *reinterpret_cast<__nv_bfloat162*>(&pv[j]);
-        float2 f = __bfloat1622float2(b2);
-        __half2 h2 = __floats2half2_rn(f.x, f.y);
-        pv[j] = *reinterpret_cast<uint32_t*>(&h2);
+        for (int j = 0; j < 4; ++j) {
+          __nv_bfloat162 b2 = *reinterpret_cast<__nv_bfloat162*>(&pv[j]);
+          float2 f = __bfloat1622float2(b2);
+          __half2 h2 = __floats2half2_rn(f.x, f.y);
+          pv[j] = *reinterpret_cast<uint32_t*>(&h2);
+        }
       }
-    }
-    *reinterpret_cast<uint4*>(xs + row * xrow + c * 8) = v;
-  }
-}
-
-template <int FMT, int MT, int NX>
-__device__ __forceinline__ void stream_range(const WMat& m, int qt, int tile, int q0, int q1, int warp, int lane,
-                                             const __half* xs, int xrow, int xsrc_stride, int k_base, int m_rows,
-                                             float (&acc)[MT][4]) {
-  if (qt == 2) {
-    Streamer<FMT, MT, 2, NX> s;
-    for (int qf = q0; qf < q1; qf += kWarps * s.PF) {
-      s.issue(m, tile, qf, q1, warp, lane);
-      s.compute(qf, q1, warp, lane, xs, xrow, xsrc_stride, k_base, m_rows, acc);
-    }
-  } else {
-    Streamer<FMT, MT, 1, NX> s;
-    for (int qf = q0; qf < q1; qf += kWarps * s.PF) {
-      s.issue(m, tile, qf, q1, warp, lane);
-      s.compute(qf, q1, warp, lane, xs, xrow, xsrc_stride, k_base, m_rows, acc);
+      *reinterpret_cast<uint4*>(xs + row * xrow + c * 8) = v;
     }
   }
 }
 
-// Same, but the first batch is loaded before `sync_point()` (the dependent-launch wait and the
-// activation staging) runs, so that weight traffic overlaps the previous kernel.
-template <int FMT, int MT, int QT, typename F>
-__device__ __forceinline__ void stream_first(const WMat& m, int tile, int q0, int q1, int warp, int lane, F&& sync_point,
-                                             const __half* xs, int xrow, int k_base, int m_rows, float (&acc)[MT][4]) {
-  Streamer<FMT, MT, QT, 1> s;
-  s.issue(m, tile, q0, q1, warp, lane);
-  sync_point();
-  s.compute(q0, q1, warp, lane, xs, xrow, 0, k_base, m_rows, acc);
-  for (int qf = q0 + kWarps * s.PF; qf < q1; qf += kWarps * s.PF) {
-    s.issue(m, tile, qf, q1, warp, lane);
-    s.compute(qf, q1, warp, lane, xs, xrow, 0, k_base, m_rows, acc);
+// Issue the bulk copies of one slice (quanta [q0, q0 + nq) of row tile `tile`) in kChunks pieces,
+// plus (with the first piece) the scales and zero-points of the groups the slice touches.
+// Returns the tile offset of the slice start inside its first group.
+__device__ __forceinline__ int issue_slice(const WMat& m, int tile, int q0, int nq, int qt, int cq, uint8_t* wbuf,
+                                           uint32_t* sc_s, uint16_t* zz_s, uint64_t* bars) {
+  const int tb = tile_bytes(m.fmt);
+  const uint8_t* src = m.q + ((int64_t)tile * m.kc + (int64_t)q0 * qt) * tb;
+  const bool quant = m.fmt == FMT_Q4 || m.fmt == FMT_Q3 || m.fmt == FMT_Q8;
+  const int gt = m.group / 64;
+  const int g0 = (q0 * qt) / gt;
+  for (int c = 0; c < kChunks; ++c) {
+    int qa = c * cq, qb = (c + 1) * cq < nq ? (c + 1) * cq : nq;
+    uint32_t bytes = qb > qa ? (uint32_t)(qb - qa) * qt * tb : 0u;
+    uint32_t extra_sc = 0, extra_zz = 0;
+    if (c == 0 && quant) {
+      const int g1 = ((q0 + nq) * qt + gt - 1) / gt;
+      extra_sc = (uint32_t)(g1 - g0) * 32u;
+      extra_zz = (uint32_t)(g1 - g0) * 16u;
+    }
+    mbar_expect_tx(bars + c, bytes + extra_sc + extra_zz);
+    if (bytes) bulk_g2s(wbuf + (size_t)qa * qt * tb, src + (size_t)qa * qt * tb, bytes, bars + c);
+    if (extra_sc) {
+      bulk_g2s(sc_s, m.sc + ((int64_t)tile * m.ng + g0) * 8, extra_sc, bars + c);
+      bulk_g2s(zz_s, m.zz + ((int64_t)tile * m.ng + g0) * 8, extra_zz, bars + c);
+    }
   }
+  return q0 * qt - g0 * gt;
 }
 
 template <int WF, int ABF, int MT>
-__global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const DecodeArgs p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ float red[kWarps][MT * 4 * 32];
+__global__ void __launch_bounds__(kThreads, MT == 1 ? 3 : (MT == 2 ? 2 : 1)) k_decode(const DecodeArgs p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t bars[2 * kChunks];
   __shared__ uint32_t s_flag;
 
   asm volatile("griddepcontrol.launch_dependents;");
+  EORA_TRACE(0);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int unit = blockIdx.x;
@@ -363,34 +362,58 @@ __global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const Deco
   else { int u = unit - p.a_units; tile = u / p.w_split; slice = u % p.w_split; split = p.w_split; }
   const WMat& mat = is_a ? p.a : p.w;
   const int qt = is_a ? p.qt_a : p.qt_w;
-  const int nq = mat.kc / qt;                       // quanta per row tile
-  const int q0 = (int)((int64_t)nq * slice / split), q1 = (int)((int64_t)nq * (slice + 1) / split);
-  const int k_base = q0 * qt * 64, k_len = (q1 - q0) * qt * 64;
+  const int nq_all = mat.kc / qt;                   // quanta per row tile
+  const int q0 = (int)((int64_t)nq_all * slice / split), q1 = (int)((int64_t)nq_all * (slice + 1) / split);
+  const int nq = q1 - q0;
+  const int cq = (nq + kChunks - 1) / kChunks;
+  const int k_base = q0 * qt * 64, k_len = nq * qt * 64;
   const int xrow = k_len + kXPad;
-  __half* xs = reinterpret_cast<__half*>(smem_raw);
+  const bool owns_b = !is_a && slice == split - 1 && p.a_units > 0;
+  const int nqb = owns_b ? p.b.kc / p.qt_b : 0;
+  const int cqb = owns_b ? (nqb + kChunks - 1) / kChunks : 1;
+
+  uint8_t* wbuf = smem;
+  uint32_t* sc_s = reinterpret_cast<uint32_t*>(smem + p.off_sc);
+  uint16_t* zz_s = reinterpret_cast<uint16_t*>(smem + p.off_zz);
+  uint8_t* bbuf = smem + p.off_b;
+  uint32_t* bsc_s = reinterpret_cast<uint32_t*>(smem + p.off_bsc);
+  uint16_t* bzz_s = reinterpret_cast<uint16_t*>(smem + p.off_bzz);
+  __half* xs = reinterpret_cast<__half*>(smem + p.off_x);
+  float* red = reinterpret_cast<float*>(smem + p.off_red);
+
+  // the slice start inside its first quantisation group, in tiles (same formula as issue_slice)
+  const int gofs = q0 * qt - ((q0 * qt) / (mat.group / 64)) * (mat.group / 64);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2 * kChunks; ++i) mbar_init(bars + i, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // weights are immutable: their copies may start before the previous kernel has finished
+    issue_slice(mat, tile, q0, nq, qt, cq, wbuf, sc_s, zz_s, bars);
+    if (owns_b) issue_slice(p.b, tile, 0, nqb, p.qt_b, cqb, bbuf, bsc_s, bzz_s, bars + kChunks);
+  }
+  EORA_TRACE(1);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  EORA_TRACE(2);
+  stage_x(xs, xrow, p.x, p.x_dtype, p.m, p.d_in, k_base, k_len);
+  __syncthreads();      // barriers initialised, X staged
+  EORA_TRACE(3);
 
   float acc[MT][4];
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
 
-  auto sync_point = [&]() {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    stage_x(xs, xrow, p.x, p.x_dtype, p.m, p.d_in, k_base, k_len);
-    __syncthreads();
-  };
-
+  SliceView sv;
+  sv.wbuf = wbuf; sv.sc = sc_s; sv.zz = zz_s; sv.bars = bars; sv.nq = nq; sv.qt = qt; sv.cq = cq;
+  sv.group_tiles = mat.group / 64; sv.gofs = gofs;
   if (is_a) {
-    if constexpr (ABF != FMT_NONE) {
-      if (qt == 2) stream_first<ABF, MT, 2>(mat, tile, q0, q1, warp, lane, sync_point, xs, xrow, k_base, p.m, acc);
-      else stream_first<ABF, MT, 1>(mat, tile, q0, q1, warp, lane, sync_point, xs, xrow, k_base, p.m, acc);
-    }
+    if constexpr (ABF != FMT_NONE) run_slice<ABF, MT, 1>(sv, warp, lane, xs, xrow, 0, p.m, p.dev_status, acc);
   } else {
-    if (qt == 2) stream_first<WF, MT, 2>(mat, tile, q0, q1, warp, lane, sync_point, xs, xrow, k_base, p.m, acc);
-    else stream_first<WF, MT, 1>(mat, tile, q0, q1, warp, lane, sync_point, xs, xrow, k_base, p.m, acc);
+    run_slice<WF, MT, 1>(sv, warp, lane, xs, xrow, 0, p.m, p.dev_status, acc);
   }
 
+  EORA_TRACE(4);
   // ---- B extension: the last slice of a backbone row tile adds (X.A).B for its 16 output columns
-  const bool owns_b = !is_a && slice == split - 1 && p.a_units > 0;
   if constexpr (ABF != FMT_NONE) {
     if (owns_b) {
       __syncthreads();                                   // everyone is done reading the staged X
@@ -398,20 +421,22 @@ __global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const Deco
         uint32_t it = 0;
         while (ld_acquire(p.counters + CNT_T_DONE) < (uint32_t)p.a_units) {
           if (++it > kSpinLimit) { atomicExch(p.dev_status, EORA_ERR_DEVICE_TIMEOUT); break; }
-          __nanosleep(64);
+          __nanosleep(32);
         }
       }
       __syncthreads();
+      EORA_TRACE(5);
       // t -> fp16 hi + lo in shared memory (two sources), rows padded like X
       const int trow = p.r_pad + kXPad;
       __half* ts = xs;
-      for (int i = threadIdx.x; i < p.m * p.r_pad; i += kThreads) {
-        int row = i / p.r_pad, j = i - row * p.r_pad;
-        float v = ld_cg(p.t_ws + (int64_t)row * p.r_pad + j);
-        __half hi = __float2half_rn(v);
-        __half lo = __float2half_rn(v - __half2float(hi));
-        ts[row * trow + j] = hi;
-        ts[p.m * trow + row * trow + j] = lo;
+      for (int row = 0; row < p.m; ++row) {
+        for (int j = threadIdx.x; j < p.r_pad; j += kThreads) {
+          float v = ld_cg(p.t_ws + (int64_t)row * p.r_pad + j);
+          __half hi = __float2half_rn(v);
+          __half lo = __float2half_rn(v - __half2float(hi));
+          ts[row * trow + j] = hi;
+          ts[(p.m + row) * trow + j] = lo;
+        }
       }
       __syncthreads();
       // all reads of t by this CTA are done: the last consumer returns t_ws and the counters to zero
@@ -425,17 +450,22 @@ __global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const Deco
         for (int i = threadIdx.x; i < p.m * p.r_pad; i += kThreads) p.t_ws[i] = 0.f;
         if (threadIdx.x == 0) { p.counters[CNT_T_DONE] = 0; p.counters[CNT_T_CONSUMED] = 0; }
       }
-      const int nqb = p.b.kc / p.qt_b;
-      stream_range<ABF, MT, 2>(p.b, p.qt_b, tile, 0, nqb, warp, lane, ts, trow, p.m * trow, 0, p.m, acc);
+      EORA_TRACE(6);
+      SliceView sb;
+      sb.wbuf = bbuf; sb.sc = bsc_s; sb.zz = bzz_s; sb.bars = bars + kChunks; sb.nq = nqb; sb.qt = p.qt_b; sb.cq = cqb;
+      sb.group_tiles = p.b.group / 64; sb.gofs = 0;
+      run_slice<ABF, MT, 2>(sb, warp, lane, ts, trow, p.m * trow, p.m, p.dev_status, acc);
     }
   }
 
+  EORA_TRACE(7);
   // ---- sum the 8 warps
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) red[warp][(mt * 4 + c) * 32 + lane] = acc[mt][c];
+    for (int c = 0; c < 4; ++c) red[warp * (MT * 128) + (mt * 4 + c) * 32 + lane] = acc[mt][c];
   __syncthreads();
+  EORA_TRACE(8);
 
   // outputs of this unit: 16 rows x 8*MT tokens; element idx of the warp sums is
   // (mt, c, lane) = (idx >> 7, (idx >> 5) & 3, idx & 31)
@@ -447,7 +477,7 @@ __global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const Deco
   auto warp_sum = [&](int idx) {
     float v = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) v += red[w][idx];
+    for (int w = 0; w < kWarps; ++w) v += red[w * (MT * 128) + idx];
     return v;
   };
 
@@ -460,6 +490,7 @@ __global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const Deco
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) atomicAdd(p.counters + CNT_T_DONE, 1u);
+    EORA_TRACE(9);
     return;
   }
   if (split == 1) {
@@ -468,6 +499,7 @@ __global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const Deco
       out_pos(idx, token, row);
       if (token < p.m) store_y(p.y, p.y_dtype, (int64_t)token * p.d_out + row, warp_sum(idx));
     }
+    EORA_TRACE(9);
     return;
   }
   for (int idx = threadIdx.x; idx < MT * 128; idx += kThreads) {
@@ -495,58 +527,80 @@ __global__ void __launch_bounds__(kThreads, MT <= 2 ? 2 : 1) k_decode(const Deco
     }
     if (threadIdx.x == 0) p.counters[CNT_TILE0 + tile] = 0;
   }
+  EORA_TRACE(9);
 }
 
+// ------------------------------------------------------------------------------------------ host
 int quantum_tiles(const WMat& m) {
   if (m.fmt == FMT_F16) return 1;
   return (m.group % 128 == 0) ? 2 : 1;
 }
 
-struct Plan { int a_units, a_split, w_split, smem; };
+struct Plan {
+  int a_units, a_split, w_split, smem;
+  int off_sc, off_zz, off_b, off_bsc, off_bzz, off_x, off_red;
+};
+
+inline int align_up_i(int v, int a) { return (v + a - 1) / a * a; }
 
 Plan make_plan(const Handle* h, int m) {
-  Plan pl;
-  const int slots = 2 * h->sm_count;
-  const int max_slice_k = (kXSmemBudget / (2 * m)) & ~127;          // activations staged per CTA
+  Plan pl = {};
+  const int slots = 3 * h->sm_count;
+  const int mt = m <= 8 ? 1 : m <= 16 ? 2 : m <= 32 ? 4 : 8;
+  const int max_slice_k_x = (kXSmemBudget / (2 * m)) & ~127;          // activations staged per CTA
+  auto max_slice_k = [&](const WMat& mat) {
+    int by_bytes = ((kUnitBytes / tile_bytes(mat.fmt)) * 64) & ~127;
+    return by_bytes < max_slice_k_x ? by_bytes : max_slice_k_x;
+  };
   auto split_for = [&](const WMat& mat, int want) {
     int qt = quantum_tiles(mat), nq = mat.kc / qt;
-    int min_split = (mat.k_red + max_slice_k - 1) / max_slice_k;
+    int msk = max_slice_k(mat);
+    int min_split = (mat.k_red + msk - 1) / msk;
     int s = want > min_split ? want : min_split;
     if (s > nq) s = nq;
     if (s < 1) s = 1;
     return s;
   };
-  int want_w = (h->w.nt * 4 >= slots * 3) ? 1 : (slots + h->w.nt - 1) / h->w.nt;
-  pl.w_split = split_for(h->w, want_w);
-  pl.a_units = 0; pl.a_split = 1;
-  if (h->cfg.rank > 0) {
-    // size A units like backbone units (in bytes streamed)
-    int64_t w_unit_bytes = wmat_q_bytes(h->w.fmt, 1, h->w.kc) / pl.w_split;
-    if (w_unit_bytes < 8192) w_unit_bytes = 8192;
-    int64_t a_tile_bytes = wmat_q_bytes(h->a.fmt, 1, h->a.kc);
-    int want_a = (int)((a_tile_bytes + w_unit_bytes - 1) / w_unit_bytes);
-    pl.a_split = split_for(h->a, want_a);
-    pl.a_units = h->a.nt * pl.a_split;
-  }
-  // shared memory: the staged X slice, or the hi/lo copies of t
-  int64_t max_k = 0;
-  auto slice_len = [&](const WMat& mat, int split) {
-    int qt = quantum_tiles(mat), nq = mat.kc / qt;
-    int best = 0;
+  auto slice_len = [&](const WMat& mat, int split) {      // longest slice in reduction elements
+    int qt = quantum_tiles(mat), nq = mat.kc / qt, best = 0;
     for (int s = 0; s < split; ++s) {
       int l = (int)(((int64_t)nq * (s + 1) / split) - ((int64_t)nq * s / split)) * qt * 64;
       if (l > best) best = l;
     }
     return best;
   };
-  max_k = slice_len(h->w, pl.w_split);
-  if (h->cfg.rank > 0) {
-    int la = slice_len(h->a, pl.a_split);
-    if (la > max_k) max_k = la;
+  int want_w = (h->w.nt * 4 >= slots * 3) ? 1 : (slots + h->w.nt - 1) / h->w.nt;
+  pl.w_split = split_for(h->w, want_w);
+  const bool ab = h->cfg.rank > 0;
+  if (ab) {
+    // size A units like backbone units (in bytes streamed)
+    int64_t w_unit_bytes = wmat_q_bytes(h->w.fmt, 1, h->w.kc) / pl.w_split;
+    if (w_unit_bytes < 8192) w_unit_bytes = 8192;
+    int64_t a_tile_bytes = wmat_q_bytes(h->a.fmt, 1, h->a.kc);
+    pl.a_split = split_for(h->a, (int)((a_tile_bytes + w_unit_bytes - 1) / w_unit_bytes));
+    pl.a_units = h->a.nt * pl.a_split;
+  } else {
+    pl.a_split = 1;
   }
-  int64_t xb = (int64_t)m * (max_k + kXPad) * 2;
-  int64_t tb = h->cfg.rank > 0 ? (int64_t)2 * m * (h->r_pad + kXPad) * 2 : 0;
-  pl.smem = (int)(xb > tb ? xb : tb);
+  int lw = slice_len(h->w, pl.w_split), la = ab ? slice_len(h->a, pl.a_split) : 0;
+  int wbytes = lw / 64 * tile_bytes(h->w.fmt);
+  if (ab && la / 64 * tile_bytes(h->a.fmt) > wbytes) wbytes = la / 64 * tile_bytes(h->a.fmt);
+  int max_k = lw > la ? lw : la;
+  int groups_w = lw / h->w.group + 2;
+  int groups_a = ab ? la / h->a.group + 2 : 0;
+  int groups = groups_w > groups_a ? groups_w : groups_a;
+  int off = align_up_i(wbytes, 128);
+  pl.off_sc = off; off += align_up_i(groups * 32, 128);
+  pl.off_zz = off; off += align_up_i(groups * 16, 128);
+  pl.off_b = off; off += ab ? align_up_i(h->b.kc * tile_bytes(h->b.fmt), 128) : 0;
+  pl.off_bsc = off; off += ab ? align_up_i((h->b.ng + 1) * 32, 128) : 0;
+  pl.off_bzz = off; off += ab ? align_up_i((h->b.ng + 1) * 16, 128) : 0;
+  pl.off_x = off;
+  int xb = m * (max_k + kXPad) * 2;
+  int tb = ab ? 2 * m * (h->r_pad + kXPad) * 2 : 0;
+  off += align_up_i(xb > tb ? xb : tb, 128);
+  pl.off_red = off; off += kWarps * mt * 128 * 4;
+  pl.smem = off;
   return pl;
 }
 
@@ -554,7 +608,7 @@ template <auto KERNEL>
 cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const DecodeArgs& args) {
   static bool attr_set = false;   // one per kernel (KERNEL is a template argument)
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -598,12 +652,17 @@ bool decode_supported(const Handle* h, int m) {
   if (h->w.fmt != FMT_Q4 && h->w.fmt != FMT_Q3) return false;
   if (h->w.group % 64) return false;
   Plan pl = make_plan(h, m);
-  return pl.smem <= 160 * 1024;
+  return pl.smem <= kMaxSmem;
 }
 
 void decode_make_plan(Handle* h) { h->plan = DecodePlan(); }
 
 int decode_launch_count(const Handle*, int) { return 1; }
+
+int decode_grid(const Handle* h, int m) {
+  Plan pl = make_plan(h, m);
+  return pl.a_units + h->w.nt * pl.w_split;
+}
 
 cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st) {
   Plan pl = make_plan(h, m);
@@ -617,6 +676,9 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y
   a.qt_w = quantum_tiles(h->w);
   a.qt_a = h->cfg.rank > 0 ? quantum_tiles(h->a) : 1;
   a.qt_b = h->cfg.rank > 0 ? quantum_tiles(h->b) : 1;
+  a.off_sc = pl.off_sc; a.off_zz = pl.off_zz; a.off_b = pl.off_b; a.off_bsc = pl.off_bsc; a.off_bzz = pl.off_bzz;
+  a.off_x = pl.off_x; a.off_red = pl.off_red;
+  a.trace = reinterpret_cast<unsigned long long*>(h->trace);
   int grid = pl.a_units + h->w.nt * pl.w_split;
   int mt = m <= 8 ? 1 : m <= 16 ? 2 : m <= 32 ? 4 : 8;
   int abf = h->cfg.rank > 0 ? h->a.fmt : FMT_NONE;

@@ -34,13 +34,12 @@ void wmat_shape(WMat& m, int fmt, int rows, int k_red, int group) {
   m.nt = m.n_rows / 16;
   m.kc = m.k_red / 64;
   m.ng = m.k_red / m.group;
-  m.q = nullptr; m.q2 = nullptr; m.sc = nullptr; m.zz = nullptr;
+  m.q = nullptr; m.sc = nullptr; m.zz = nullptr;
 }
 
 void wmat_carve(WMat& m, Carve& c) {
   if (m.fmt == FMT_NONE) return;
-  m.q = c.take<void>(wmat_q_bytes(m.fmt, m.nt, m.kc));
-  if (wmat_q2_bytes(m.fmt, m.nt, m.kc)) m.q2 = c.take<uint32_t>(wmat_q2_bytes(m.fmt, m.nt, m.kc));
+  m.q = c.take<uint8_t>(wmat_q_bytes(m.fmt, m.nt, m.kc));
   if (m.fmt == FMT_Q4 || m.fmt == FMT_Q3 || m.fmt == FMT_Q8) {
     m.sc = c.take<uint32_t>((int64_t)m.nt * m.ng * 8 * 4);
     m.zz = c.take<uint16_t>((int64_t)m.nt * m.ng * 8 * 2);
@@ -274,6 +273,19 @@ int eora_linear_last_device_status(eora_linear_t obj) {
     if (cudaMemcpy(obj->h.dev_status, &z, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return EORA_ERR_CUDA;
   }
   return v;
+}
+
+int eora_linear_set_trace(eora_linear_t obj, void* buf) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  obj->h.trace = buf;
+  return EORA_OK;
+}
+
+int eora_linear_decode_grid(eora_linear_t obj, int32_t m) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (m < 1 || m > 64) return EORA_ERR_BAD_SHAPE;
+  if (pick_path(&obj->h, m) != EORA_PATH_DECODE) return 0;
+  return decode_grid(&obj->h, m);
 }
 
 int64_t eora_linear_weight_bytes(eora_linear_t obj) { return obj ? obj->h.weight_bytes : 0; }

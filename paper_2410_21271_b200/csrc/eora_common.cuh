@@ -23,19 +23,23 @@ namespace eora {
 // 16-byte chunk of a K-major tensor-core operand, so the same layout feeds the prefill kernel.
 // Tiles of one row-tile are contiguous along the reduction axis: index = tile * kc + c.
 //
-// Per format, the payload of lane L in tile (tile, c):
-//   Q4  : one uint4; word `part` holds the 8 codes of that part, element e in nibble
+// Every tile is one contiguous blob of tile_bytes(fmt) bytes, so the tiles a CTA needs are one
+// contiguous byte range that a single bulk copy can bring into shared memory.
+// Per format, the payload of lane L inside the blob of tile (tile, c):
+//   Q4  : 512 B: one uint4 per lane; word `part` holds the 8 codes of that part, element e in nibble
 //         (e & 1) * 4 + (e >> 1)   (so that (w & 0x000f000f) is the pair (e0, e1), ...).
-//   Q3  : three words w0, w1 (a uint2 in `q`) and w2 (in `q2`).  The 32 codes form 16 pairs,
+//   Q3  : 384 B: three words; w0, w1 as a uint2 per lane in bytes [0, 256), w2 as one word per lane
+//         in bytes [256, 384).  The 32 codes form 16 pairs,
 //         pair p = part*4 + e/2; for p < 15 the pair lives in word p/5, field f = p%5: the even
 //         element in bits [3f, 3f+3), the odd one in bits [16+3f, 16+3f+3).  Pair 15 is spread
 //         over the spare bits: bit i of the even element is bit 15 of word i, bit i of the odd
 //         element is bit 31 of word i.
-//   Q8  : two uint4 (index part/2); words 2*(part%2) and 2*(part%2)+1 hold elements 0..3 and
-//         4..7; inside a word element i sits in byte {0, 2, 1, 3}[i].
-//   F16 : four uint4 (index = part), 8 fp16 in natural order.
-//   SP24: values: two uint4 (index part/2), the half (part%2) holds the 4 kept fp16 values of
-//         the part's two quads; meta: one uint32 in `q2`, byte `part` = nibble(quad0) | nibble(quad1)<<4.
+//   Q8  : 1024 B: two planes of one uint4 per lane (plane = part/2); words 2*(part%2) and 2*(part%2)+1
+//         hold elements 0..3 and 4..7; inside a word element i sits in byte {0, 2, 1, 3}[i].
+//   F16 : 2048 B: four planes of one uint4 per lane (plane = part), 8 fp16 in natural order.
+//   SP24: 1152 B: values in two planes of one uint4 per lane (plane = part/2), the half (part%2) holds
+//         the 4 kept fp16 values of the part's two quads; then one word per lane in bytes [1024, 1152),
+//         byte `part` = nibble(quad0) | nibble(quad1)<<4.
 // Scales / zero-points (Q4, Q3, Q8): sc[(tile*G + grp)*8 + g] = half2(s[n_a], s[n_b]),
 //   zz[(tile*G + grp)*8 + g] = z[n_a] | z[n_b] << 8, with grp = k / group.
 // ---------------------------------------------------------------------------------------------
@@ -49,27 +53,22 @@ struct WMat {
   int nt;          // n_rows / 16
   int kc;          // k_red / 64
   int ng;          // k_red / group
-  const void* q;         // main payload
-  const uint32_t* q2;    // Q3 third word / SP24 metadata
+  const uint8_t* q;      // tile blobs
   const uint32_t* sc;    // half2 scales
   const uint16_t* zz;    // u8x2 zero-points
 };
 
-__host__ __device__ inline int64_t wmat_q_bytes(int fmt, int nt, int kc) {
-  int64_t tiles = (int64_t)nt * kc;
+__host__ __device__ inline int tile_bytes(int fmt) {
   switch (fmt) {
-    case FMT_Q4: return tiles * 512;
-    case FMT_Q3: return tiles * 256;
-    case FMT_Q8: return tiles * 1024;
-    case FMT_F16: return tiles * 2048;
-    case FMT_SP24: return tiles * 1024;
+    case FMT_Q4: return 512;
+    case FMT_Q3: return 384;
+    case FMT_Q8: return 1024;
+    case FMT_F16: return 2048;
+    case FMT_SP24: return 1152;
     default: return 0;
   }
 }
-__host__ __device__ inline int64_t wmat_q2_bytes(int fmt, int nt, int kc) {
-  int64_t tiles = (int64_t)nt * kc;
-  return (fmt == FMT_Q3 || fmt == FMT_SP24) ? tiles * 128 : 0;
-}
+__host__ __device__ inline int64_t wmat_q_bytes(int fmt, int nt, int kc) { return (int64_t)nt * kc * tile_bytes(fmt); }
 
 // nibble / byte positions (shared by the repack kernels and the accessors below)
 __host__ __device__ inline int q4_nibble(int e) { return (e & 1) * 4 + (e >> 1); }
@@ -80,20 +79,17 @@ __device__ inline int wmat_code(const WMat& w, int k, int n) {
   int tile = n >> 4, g = n & 7, half = (n >> 3) & 1;
   int c = k >> 6, blk = (k >> 5) & 1, t = (k >> 3) & 3, e = k & 7;
   int lane = g * 4 + t, part = blk * 2 + half;
-  int64_t ti = (int64_t)tile * w.kc + c;
+  const uint32_t* blob = reinterpret_cast<const uint32_t*>(w.q + ((int64_t)tile * w.kc + c) * tile_bytes(w.fmt));
   if (w.fmt == FMT_Q4) {
-    const uint32_t* p = reinterpret_cast<const uint32_t*>(w.q) + (ti * 32 + lane) * 4;
-    return (p[part] >> (4 * q4_nibble(e))) & 15;
+    return (blob[lane * 4 + part] >> (4 * q4_nibble(e))) & 15;
   } else if (w.fmt == FMT_Q3) {
-    const uint32_t* p01 = reinterpret_cast<const uint32_t*>(w.q) + (ti * 32 + lane) * 2;
-    uint32_t wd[3] = {p01[0], p01[1], w.q2[ti * 32 + lane]};
+    uint32_t wd[3] = {blob[lane * 2], blob[lane * 2 + 1], blob[64 + lane]};
     int pr = part * 4 + (e >> 1), hi = (e & 1) * 16;
     if (pr < 15) return (wd[pr / 5] >> (3 * (pr % 5) + hi)) & 7;
     int b = 15 + hi;
     return ((wd[0] >> b) & 1) | (((wd[1] >> b) & 1) << 1) | (((wd[2] >> b) & 1) << 2);
   } else {  // FMT_Q8
-    const uint32_t* p = reinterpret_cast<const uint32_t*>(w.q) + ((ti * 2 + (part >> 1)) * 32 + lane) * 4;
-    uint32_t wd = p[2 * (part & 1) + (e >> 2)];
+    uint32_t wd = blob[(part >> 1) * 128 + lane * 4 + 2 * (part & 1) + (e >> 2)];
     return (wd >> (8 * q8_byte(e & 3))) & 255;
   }
 }
@@ -112,14 +108,14 @@ __device__ inline float wmat_elem(const WMat& w, int k, int n) {
   }
   int c = k >> 6, blk = (k >> 5) & 1, t = (k >> 3) & 3, e = k & 7;
   int lane = g * 4 + t, part = blk * 2 + half;
-  int64_t ti = (int64_t)tile * w.kc + c;
+  const uint8_t* blob = w.q + ((int64_t)tile * w.kc + c) * tile_bytes(w.fmt);
   if (w.fmt == FMT_F16) {
-    const __half* p = reinterpret_cast<const __half*>(w.q) + ((ti * 4 + part) * 32 + lane) * 8;
+    const __half* p = reinterpret_cast<const __half*>(blob) + (part * 32 + lane) * 8;
     return __half2float(p[e]);
   }
   // FMT_SP24
-  const __half* v = reinterpret_cast<const __half*>(w.q) + ((ti * 2 + (part >> 1)) * 32 + lane) * 8 + 4 * (part & 1);
-  uint32_t meta = (w.q2[ti * 32 + lane] >> (8 * part)) & 255;
+  const __half* v = reinterpret_cast<const __half*>(blob) + ((part >> 1) * 32 + lane) * 8 + 4 * (part & 1);
+  uint32_t meta = (reinterpret_cast<const uint32_t*>(blob + 1024)[lane] >> (8 * part)) & 255;
   int quad = e >> 2, pos = e & 3;
   uint32_t nib = (meta >> (4 * quad)) & 15;
   int p0 = nib & 3, p1 = nib >> 2;
@@ -156,6 +152,7 @@ struct Handle {
   DecodePlan plan;
   int sm_count;
   void* prefill_state;   // owned by prefill.cu (tensor maps), may be NULL
+  void* trace;           // optional caller-owned timestamp buffer (decode kernel), may be NULL
 };
 
 // kernels / launchers implemented in the other translation units ------------------------------
@@ -174,6 +171,7 @@ bool decode_supported(const Handle* h, int m);
 void decode_make_plan(Handle* h);
 cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
 int decode_launch_count(const Handle* h, int m);
+int decode_grid(const Handle* h, int m);
 
 bool prefill_supported(const Handle* h, int m);
 cudaError_t prefill_init(Handle* h);

@@ -54,7 +54,7 @@ __global__ void k_repack_q4(WMat d, const uint32_t* codes, const uint32_t* zeros
         w |= padded_code(codes, zeros, 4, k0 + e, n, rows_src, k_src, d.group, ldz) << (4 * q4_nibble(e));
       out[part] = w;
     }
-    reinterpret_cast<uint4*>(const_cast<void*>(d.q))[idx] = make_uint4(out[0], out[1], out[2], out[3]);
+    reinterpret_cast<uint4*>(const_cast<uint8_t*>(d.q))[idx] = make_uint4(out[0], out[1], out[2], out[3]);
   }
 }
 
@@ -76,8 +76,10 @@ __global__ void k_repack_q3(WMat d, const uint32_t* codes, const uint32_t* zeros
         }
       }
     }
-    reinterpret_cast<uint2*>(const_cast<void*>(d.q))[idx] = make_uint2(wd[0], wd[1]);
-    const_cast<uint32_t*>(d.q2)[idx] = wd[2];
+    uint32_t* blob = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(d.q) + (idx >> 5) * 384);
+    blob[p.lane * 2] = wd[0];
+    blob[p.lane * 2 + 1] = wd[1];
+    blob[64 + p.lane] = wd[2];
   }
 }
 
@@ -95,7 +97,7 @@ __global__ void k_repack_q8(WMat d, const uint8_t* codes, const uint8_t* zeros, 
         if (n < rows_src) q = (k0 + e < k_src) ? codes[(int64_t)(k0 + e) * rows_src + n] : zeros[n];
         w2[e >> 2] |= q << (8 * q8_byte(e & 3));
       }
-      uint32_t* dst = reinterpret_cast<uint32_t*>(const_cast<void*>(d.q)) + ((ti * 2 + (part >> 1)) * 32 + p.lane) * 4;
+      uint32_t* dst = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(d.q)) + ((ti * 2 + (part >> 1)) * 32 + p.lane) * 4;
       dst[2 * (part & 1)] = w2[0];
       dst[2 * (part & 1) + 1] = w2[1];
     }
@@ -111,7 +113,7 @@ __global__ void k_repack_f16(WMat d, const __half* src, int rows_src, int k_src)
     for (int part = 0; part < 4; ++part) {
       int n = p.tile * 16 + p.g + 8 * (part & 1);
       int k0 = p.c * 64 + (part >> 1) * 32 + 8 * p.t;
-      __half* dst = reinterpret_cast<__half*>(const_cast<void*>(d.q)) + ((ti * 4 + part) * 32 + p.lane) * 8;
+      __half* dst = reinterpret_cast<__half*>(const_cast<uint8_t*>(d.q)) + ((ti * 4 + part) * 32 + p.lane) * 8;
       for (int e = 0; e < 8; ++e) {
         int k = k0 + e;
         dst[e] = (n < rows_src && k < k_src) ? src[(int64_t)k * rows_src + n] : __float2half(0.f);
@@ -130,7 +132,7 @@ __global__ void k_repack_sp24(WMat d, const __half* values, const uint32_t* meta
       int n = p.tile * 16 + p.g + 8 * (part & 1);
       int k0 = p.c * 64 + (part >> 1) * 32 + 8 * p.t;
       int j0 = k0 >> 2;   // first of the part's two quads
-      __half* dst = reinterpret_cast<__half*>(const_cast<void*>(d.q)) + ((ti * 2 + (part >> 1)) * 32 + p.lane) * 8 + 4 * (part & 1);
+      __half* dst = reinterpret_cast<__half*>(const_cast<uint8_t*>(d.q) + ti * 1152) + ((part >> 1) * 32 + p.lane) * 8 + 4 * (part & 1);
       uint32_t mb = 0x44;  // positions (0,1) with zero values outside the source
       if (n < rows_src && k0 < k_src) {
         for (int i = 0; i < 4; ++i) dst[i] = values[(int64_t)n * (k_src / 2) + 2 * j0 + i];
@@ -140,7 +142,7 @@ __global__ void k_repack_sp24(WMat d, const __half* values, const uint32_t* meta
       }
       m |= mb << (8 * part);
     }
-    const_cast<uint32_t*>(d.q2)[idx] = m;
+    reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(d.q) + ti * 1152 + 1024)[p.lane] = m;
   }
 }
 
