@@ -25,9 +25,10 @@
 // Programmatic dependent launch: the bulk copies of the weights are issued before
 // griddepcontrol.wait, i.e. while the previous kernel in the stream is still draining;
 // activations and scratch are touched only after it.
-#include "eora_common.cuh"
+#include "decode_common.cuh"
 
 namespace eora {
+using namespace dec;
 namespace {
 
 constexpr int kWarps = 8;
@@ -37,156 +38,7 @@ constexpr int kChunks = 4;                // bulk-copy chunks (one mbarrier each
 constexpr int kUnitBytes = 32 * 1024;     // largest packed-weight slice of one unit
 constexpr int kXSmemBudget = 64 * 1024;   // bytes of staged activations per CTA
 constexpr int kMaxSmem = 200 * 1024;
-constexpr uint32_t kSpinLimit = 1u << 21;
 
-enum { CNT_T_DONE = 0, CNT_T_CONSUMED = 1, CNT_TILE0 = 2 };
-
-// ------------------------------------------------------------------------------------------ PTX
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: returns false (and latches the status word) if the copy never lands.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* dev_status) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-  }
-  atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
-  return false;
-}
-// global -> shared bulk copy of `bytes` (multiple of 16; both addresses 16-byte aligned)
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ float ld_cg(const float* p) {
-  float v;
-  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void red_add(float* p, float v) {
-  asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
-}
-__device__ __forceinline__ uint32_t h2sub(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("sub.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t h2fma(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// ------------------------------------------------------------------------------------------ dequant
-// Per-quantum constants of the two rows a lane owns: fp16x2 values that turn the magic-number
-// form of a code (1024 + q * 2^s as fp16) into the exact integer q - z.
-struct ZC { uint32_t c[2][3]; };
-
-template <int FMT>
-__device__ __forceinline__ void make_zc(ZC& zc, uint32_t zz) {
-#pragma unroll
-  for (int hf = 0; hf < 2; ++hf) {
-    uint32_t z = (zz >> (8 * hf)) & 255u;
-    zc.c[hf][0] = (0x6400u | z) * 0x00010001u;                                      //  1024 + z
-    if constexpr (FMT == FMT_Q4) zc.c[hf][1] = (0xD400u | (z << 4)) * 0x00010001u;   // -(64 + z)
-    if constexpr (FMT == FMT_Q3) {
-      zc.c[hf][1] = (0xD800u | (z << 3)) * 0x00010001u;                              // -(128 + z)
-      zc.c[hf][2] = (0xCC00u | (z << 6)) * 0x00010001u;                              // -(16 + z)
-    }
-  }
-}
-
-constexpr uint32_t kMagic = 0x64006400u;   // fp16x2 (1024, 1024)
-
-template <int FMT> constexpr bool is_quant() { return FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8; }
-
-// Build the A-operand registers of the four mma of one tile from its blob in shared memory.
-// a[i][*]: mma i = 2*blk + sub; entries are fp16x2.
-template <int FMT>
-__device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const ZC& zc, uint32_t (&a)[4][4]) {
-  if constexpr (FMT == FMT_Q4) {
-    const uint4 v = *reinterpret_cast<const uint4*>(blob + lane * 16);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int part = 0; part < 4; ++part) {
-      const int hf = part & 1, blk = part >> 1;
-      uint32_t lo = w[part], hi = w[part] >> 8;
-      uint32_t h0 = (lo & 0x000f000fu) | kMagic, h1 = (lo & 0x00f000f0u) | kMagic;
-      uint32_t h2 = (hi & 0x000f000fu) | kMagic, h3 = (hi & 0x00f000f0u) | kMagic;
-      a[blk * 2 + 0][hf] = h2sub(h0, zc.c[hf][0]);
-      a[blk * 2 + 0][hf + 2] = h2fma(h1, 0x2C002C00u, zc.c[hf][1]);   // * 1/16
-      a[blk * 2 + 1][hf] = h2sub(h2, zc.c[hf][0]);
-      a[blk * 2 + 1][hf + 2] = h2fma(h3, 0x2C002C00u, zc.c[hf][1]);
-    }
-  } else if constexpr (FMT == FMT_Q3) {
-    const uint2 v01 = *reinterpret_cast<const uint2*>(blob + lane * 8);
-    const uint32_t v2 = *reinterpret_cast<const uint32_t*>(blob + 256 + lane * 4);
-    const uint32_t w[3] = {v01.x, v01.y, v2};
-    const uint32_t ws[3] = {v01.x >> 9, v01.y >> 9, v2 >> 9};
-#pragma unroll
-    for (int p = 0; p < 16; ++p) {
-      const int part = p >> 2, j = p & 3, hf = part & 1, blk = part >> 1;
-      uint32_t v;
-      if (p < 15) {
-        const int wi = p / 5, f = p % 5, ff = f >= 3 ? f - 3 : f;
-        const uint32_t src = f >= 3 ? ws[wi] : w[wi];
-        const uint32_t h = (src & (0x00070007u << (3 * ff))) | kMagic;
-        if (ff == 0) v = h2sub(h, zc.c[hf][0]);
-        else if (ff == 1) v = h2fma(h, 0x30003000u, zc.c[hf][1]);   // * 1/8
-        else v = h2fma(h, 0x24002400u, zc.c[hf][2]);                // * 1/64
-      } else {
-        uint32_t h = ((w[0] >> 15) & 0x00010001u) | kMagic;
-        h |= (w[1] >> 14) & 0x00020002u;
-        h |= (w[2] >> 13) & 0x00040004u;
-        v = h2sub(h, zc.c[hf][0]);
-      }
-      a[blk * 2 + (j >> 1)][hf + 2 * (j & 1)] = v;
-    }
-  } else if constexpr (FMT == FMT_Q8) {
-#pragma unroll
-    for (int pl = 0; pl < 2; ++pl) {
-      const uint4 u = *reinterpret_cast<const uint4*>(blob + pl * 512 + lane * 16);
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        const uint32_t w0 = hf ? u.z : u.x, w1 = hf ? u.w : u.y;
-        a[pl * 2 + 0][hf] = h2sub((w0 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[pl * 2 + 0][hf + 2] = h2sub(((w0 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[pl * 2 + 1][hf] = h2sub((w1 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[pl * 2 + 1][hf + 2] = h2sub(((w1 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-      }
-    }
-  } else if constexpr (FMT == FMT_F16) {
-#pragma unroll
-    for (int part = 0; part < 4; ++part) {
-      const int hf = part & 1, blk = part >> 1;
-      const uint4 u = *reinterpret_cast<const uint4*>(blob + part * 512 + lane * 16);
-      a[blk * 2 + 0][hf] = u.x;
-      a[blk * 2 + 0][hf + 2] = u.y;
-      a[blk * 2 + 1][hf] = u.z;
-      a[blk * 2 + 1][hf + 2] = u.w;
-    }
-  }
-}
 
 // What one CTA streams: a slice of nq quanta of one row tile, (being) copied to shared memory.
 struct SliceView {
@@ -282,18 +134,7 @@ struct DecodeArgs {
   unsigned long long* trace;   // optional: 16 timestamps (ns) per CTA, see eora_linear_set_trace
 };
 
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
 #define EORA_TRACE(slot) do { if (p.trace && threadIdx.x == 0) p.trace[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
-
-__device__ __forceinline__ void store_y(void* y, int dtype, int64_t i, float v) {
-  if (dtype == EORA_Y_F16) reinterpret_cast<__half*>(y)[i] = __float2half_rn(v);
-  else if (dtype == EORA_Y_BF16) reinterpret_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
-  else reinterpret_cast<float*>(y)[i] = v;
-}
 
 // Stage activation rows [0, m) x reduction range [k0, k0 + len) into shared memory as fp16.
 __device__ __forceinline__ void stage_x(__half* xs, int xrow, const void* x, int x_dtype, int m, int d_in, int k0, int len) {
@@ -418,11 +259,7 @@ __global__ void __launch_bounds__(kThreads, MT == 1 ? 3 : (MT == 2 ? 2 : 1)) k_d
     if (owns_b) {
       __syncthreads();                                   // everyone is done reading the staged X
       if (threadIdx.x == 0) {
-        uint32_t it = 0;
-        while (ld_acquire(p.counters + CNT_T_DONE) < (uint32_t)p.a_units) {
-          if (++it > kSpinLimit) { atomicExch(p.dev_status, EORA_ERR_DEVICE_TIMEOUT); break; }
-          __nanosleep(32);
-        }
+        counter_wait(p.counters + CNT_T_DONE, (uint32_t)p.a_units, p.dev_status);
       }
       __syncthreads();
       EORA_TRACE(5);
@@ -531,11 +368,6 @@ __global__ void __launch_bounds__(kThreads, MT == 1 ? 3 : (MT == 2 ? 2 : 1)) k_d
 }
 
 // ------------------------------------------------------------------------------------------ host
-int quantum_tiles(const WMat& m) {
-  if (m.fmt == FMT_F16) return 1;
-  return (m.group % 128 == 0) ? 2 : 1;
-}
-
 struct Plan {
   int a_units, a_split, w_split, smem;
   int off_sc, off_zz, off_b, off_bsc, off_bzz, off_x, off_red;
@@ -660,11 +492,13 @@ void decode_make_plan(Handle* h) { h->plan = DecodePlan(); }
 int decode_launch_count(const Handle*, int) { return 1; }
 
 int decode_grid(const Handle* h, int m) {
+  if (decode_stream_supported(h, m)) return decode_stream_grid(h, m);
   Plan pl = make_plan(h, m);
   return pl.a_units + h->w.nt * pl.w_split;
 }
 
 cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st) {
+  if (decode_stream_supported(h, m)) return launch_decode_stream(h, x, m, y, st);
   Plan pl = make_plan(h, m);
   DecodeArgs a;
   a.w = h->w; a.a = h->a; a.b = h->b;

@@ -172,6 +172,9 @@ void decode_make_plan(Handle* h);
 cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
 int decode_launch_count(const Handle* h, int m);
 int decode_grid(const Handle* h, int m);
+bool decode_stream_supported(const Handle* h, int m);
+int decode_stream_grid(const Handle* h, int m);
+cudaError_t launch_decode_stream(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
 
 bool prefill_supported(const Handle* h, int m);
 cudaError_t prefill_init(Handle* h);
