@@ -164,6 +164,35 @@ int eora_linear_last_device_status(eora_linear_t h);
 int eora_linear_decode_grid(eora_linear_t h, int32_t m);
 int eora_linear_set_trace(eora_linear_t h, void* trace_buf);
 
+/*
+ * The same layer for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a deployment convenience of the library.)
+ *
+ * Everything else in this header works on a handle, and eora_linear_create calls cudaMalloc.  Code
+ * that runs after another framework has taken all device memory into its own pool, code in a
+ * latency-critical loop that must not risk the stall an allocation can cause, or a plug-in that is
+ * only ever handed buffers and a stream, cannot do that.  This call needs no handle: it reads the
+ * weights directly from the caller's buffers in the interchange layout (top of this file) and keeps
+ * its only scratch, t = X.A as fp32, in a fixed array of EORA_NOALLOC_MAX_T_ELEMS floats (256 KB)
+ * that is part of the library image: every GPU that loads the library holds it until the process
+ * exits.  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * Supported: quantised backbone (3/4-bit), fp16 A and B (or rank 0), any x/y dtype of the config;
+ * cfg->max_m and cfg->kernel_policy are ignored.  m * cfg->rank must not exceed
+ * EORA_NOALLOC_MAX_T_ELEMS, otherwise EORA_ERR_M_TOO_LARGE is returned and nothing is launched.
+ * Other errors as for create / forward.  It runs two simple kernels and is much slower than the
+ * handle-based forward.
+ *
+ * The first call on a device looks up the device address of the scratch array
+ * (cudaGetSymbolAddress) with that device current; make that first call outside any stream capture.
+ * All calls on a device share the one array, which keeps whatever the previous call left in it; each
+ * call overwrites the part it uses before reading it, so nothing has to be cleared, but two calls
+ * that overlap on the GPU (different streams) race on it: keep them in stream order.
+ */
+#define EORA_NOALLOC_MAX_T_ELEMS 65536
+int eora_linear_forward_noalloc(const eora_linear_config* cfg, const eora_linear_weights* w, const void* x,
+                                int32_t m, void* y, void* stream);
+
 /* Bytes of device memory the handle owns: re-tiled weights, and scratch. */
 int64_t eora_linear_weight_bytes(eora_linear_t h);
 int64_t eora_linear_scratch_bytes(eora_linear_t h);

@@ -74,6 +74,9 @@ def lib() -> ctypes.CDLL:
         L.eora_linear_set_trace.restype = c_int
         L.eora_linear_decode_grid.argtypes = [c_void_p, c_int32]
         L.eora_linear_decode_grid.restype = c_int
+        L.eora_linear_forward_noalloc.argtypes = [POINTER(eora_linear_config), POINTER(eora_linear_weights), c_void_p,
+                                                  c_int32, c_void_p, c_void_p]
+        L.eora_linear_forward_noalloc.restype = c_int
         L.eora_linear_weight_bytes.argtypes = [c_void_p]
         L.eora_linear_weight_bytes.restype = c_int64
         L.eora_linear_scratch_bytes.argtypes = [c_void_p]
@@ -174,6 +177,19 @@ def eora_linear_set_trace(handle: int, buf) -> int:
 
 def eora_linear_decode_grid(handle: int, m: int) -> int:
     return lib().eora_linear_decode_grid(handle, int(m))
+
+
+EORA_NOALLOC_MAX_T_ELEMS = 65536
+
+
+def eora_linear_forward_noalloc(cfg: eora_linear_config, weights: eora_linear_weights, x, m: int, y, stream=None,
+                                check: bool = True) -> int:
+    """Handle-free forward for callers that cannot allocate device memory: weights are read from the
+    caller's interchange-layout buffers, scratch lives in a fixed array inside the library."""
+    st = lib().eora_linear_forward_noalloc(byref(cfg), byref(weights), _ptr(x), int(m), _ptr(y), _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward_noalloc")
+    return st
 
 
 def eora_linear_weight_bytes(handle: int) -> int:
