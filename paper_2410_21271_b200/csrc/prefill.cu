@@ -1,9 +1,539 @@
-// Prefill kernel family (large M, tcgen05).
-#include "eora_common.cuh"
+// Prefill kernel family (M > 64): Y = X.deq(Wq) + (X.A).B  (paper Eq. 4) as a tcgen05 GEMM.
+//
+// The paper measures only batch-1 decoding (Section 4.5); for many tokens the layer is a dense
+// contraction, so it runs on the 5th-generation tensor cores:
+//   * activations (M x K, K-major) arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle, no
+//     multicast) into a ring of shared-memory stages;
+//   * the packed weights are read by eight "dequant" warps straight from global memory (the tiles of
+//     the shared layout are 512-byte contiguous per warp), turned into fp16 RN((q - z) * s) in
+//     registers and stored as the K-major, 128-byte-swizzled B operand of the same stage;
+//   * one thread issues tcgen05.mma (M = 128, N = BN, K = 16) with the fp32 accumulator in tensor
+//     memory; tcgen05.commit releases a stage when its MMAs have drained;
+//   * the low-rank term is a K-extension: after the d_in/64 backbone k-blocks come r/64 k-blocks whose
+//     activation operand is t = X.A (fp16, from a first launch of the same kernel with A as the
+//     weight) and whose weight operand is B, so (X.A).B lands in the same accumulator and Y is
+//     written once by the epilogue (tcgen05.ld -> convert -> global).
+// Launches per forward: 1 (rank 0) or 2 (t = X.A, then the main product), plus a conversion launch
+// when X is bf16 (the f16 MMA kind needs both operands in fp16; weights are kept fp16 because
+// bf16 weights alone cost 1.7e-3 of the 2e-3 error budget).
+#include <cuda.h>
+#include "decode_common.cuh"
+
 namespace eora {
-bool prefill_supported(const Handle*, int) { return false; }
-cudaError_t prefill_init(Handle*) { return cudaSuccess; }
-void prefill_free(Handle*) {}
-cudaError_t launch_prefill_forward(const Handle*, const void*, int, void*, cudaStream_t) { return cudaErrorNotSupported; }
-int prefill_launch_count(const Handle*, int) { return 2; }
+using namespace dec;
+namespace {
+
+constexpr int BM = 128, BK = 64;
+constexpr int kDqWarps = 8;                     // dequant warps (warps 4..11); warps 4..7 are also the epilogue
+constexpr int kThreadsP = (4 + kDqWarps) * 32;  // warp 0: TMA, warp 1: MMA, warp 2: TMEM alloc, warp 3: idle
+constexpr int kMaxStagesP = 6;
+constexpr int kPrefetch = 4;                    // k-blocks of packed weights held in registers ahead of use
+
+struct PrefillArgs {
+  WMat w;            // weight operand of the first nkb_w k-blocks (rows = output columns)
+  WMat b;            // weight operand of the K-extension (FMT_NONE if none)
+  void* out;         // [m][ld_out]
+  int out_dtype;     // EORA_Y_*
+  int ld_out;        // leading dimension of out (elements)
+  int n_valid;       // columns of out to write
+  int m;
+  int bn;            // N tile: 64, 128 or 256
+  int nkb_w, nkb_b;  // k-blocks of each part
+  int stages;
+  int stage_bytes;   // BM*128 + bn*128
+  int* dev_status;
+};
+
+struct PrefillState {
+  __half* x16;       // fp16 copy of a bf16 X, [max_m][d_in]
+};
+
+// ---------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(tm), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+               "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                 "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                 "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                 "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+               : "r"(taddr) : "memory");
+}
+
+// K-major, 128-byte swizzle operand descriptor: rows of 128 B, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_desc(const void* smem_ptr) {
+  const uint32_t addr = smem_u32(smem_ptr);
+  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | (1u << 16);            // start address, leading byte offset (unused) = 1
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);           // stride byte offset, descriptor version 1, SWIZZLE_128B
+  return ((uint64_t)hi << 32) | lo;
+}
+
+// packed tile payload of one lane, by format
+template <int FMT> struct Packed;
+template <> struct Packed<FMT_Q4> { uint4 v; };
+template <> struct Packed<FMT_Q3> { uint2 v; uint32_t w2; };
+template <> struct Packed<FMT_Q8> { uint4 v[2]; };
+template <> struct Packed<FMT_F16> { uint4 v[4]; };
+template <> struct Packed<FMT_SP24> { uint4 v[2]; uint32_t meta; };
+
+template <int FMT>
+__device__ __forceinline__ void load_packed(Packed<FMT>& r, const uint8_t* blob, int lane) {
+  if constexpr (FMT == FMT_Q4) r.v = __ldg(reinterpret_cast<const uint4*>(blob) + lane);
+  else if constexpr (FMT == FMT_Q3) {
+    r.v = __ldg(reinterpret_cast<const uint2*>(blob) + lane);
+    r.w2 = __ldg(reinterpret_cast<const uint32_t*>(blob + 256) + lane);
+  } else if constexpr (FMT == FMT_Q8) {
+    r.v[0] = __ldg(reinterpret_cast<const uint4*>(blob) + lane);
+    r.v[1] = __ldg(reinterpret_cast<const uint4*>(blob + 512) + lane);
+  } else if constexpr (FMT == FMT_F16) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) r.v[p] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * p) + lane);
+  } else {
+    r.v[0] = __ldg(reinterpret_cast<const uint4*>(blob) + lane);
+    r.v[1] = __ldg(reinterpret_cast<const uint4*>(blob + 512) + lane);
+    r.meta = __ldg(reinterpret_cast<const uint32_t*>(blob + 1024) + lane);
+  }
+}
+
+__device__ __forceinline__ uint32_t h2mul(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+
+// Dequantise one 16 x 64 tile to fp16 RN((q - z) * s) and store this lane's four 16-byte chunks
+// (8 consecutive reduction elements of one row each) into the swizzled B operand.
+// btile: start of the stage's B operand; row0: first row of the tile inside the operand.
+template <int FMT>
+__device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2, uint32_t zz2, uint8_t* btile, int row0, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  uint32_t out[4][4];     // [part][pair]
+  if constexpr (FMT == FMT_F16) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) { out[p][0] = r.v[p].x; out[p][1] = r.v[p].y; out[p][2] = r.v[p].z; out[p][3] = r.v[p].w; }
+  } else if constexpr (FMT == FMT_SP24) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const uint4 u = r.v[p >> 1];
+      const uint32_t v01 = (p & 1) ? u.z : u.x, v23 = (p & 1) ? u.w : u.y;   // (val0,val1) of quad 0, of quad 1
+      const uint32_t mb = (r.meta >> (8 * p)) & 255u;
+#pragma unroll
+      for (int quad = 0; quad < 2; ++quad) {
+        const uint32_t vv = quad ? v23 : v01;
+        const uint32_t nib = (mb >> (4 * quad)) & 15u, p0 = nib & 3u, p1 = nib >> 2;
+        const uint32_t v0 = vv & 0xffffu, v1 = vv >> 16;
+        uint32_t e[4];
+#pragma unroll
+        for (uint32_t pos = 0; pos < 4; ++pos) e[pos] = (pos == p0) ? v0 : (pos == p1) ? v1 : 0u;
+        out[p][2 * quad] = e[0] | (e[1] << 16);
+        out[p][2 * quad + 1] = e[2] | (e[3] << 16);
+      }
+    }
+  } else {
+    ZC zc;
+    make_zc<FMT>(zc, zz2);
+    uint32_t a[4][4];
+    if constexpr (FMT == FMT_Q4) {
+      const uint32_t w[4] = {r.v.x, r.v.y, r.v.z, r.v.w};
+#pragma unroll
+      for (int part = 0; part < 4; ++part) {
+        const int hf = part & 1;
+        uint32_t lo = w[part], hi = w[part] >> 8;
+        a[part][0] = h2sub((lo & 0x000f000fu) | kMagic, zc.c[hf][0]);
+        a[part][1] = h2fma((lo & 0x00f000f0u) | kMagic, 0x2C002C00u, zc.c[hf][1]);
+        a[part][2] = h2sub((hi & 0x000f000fu) | kMagic, zc.c[hf][0]);
+        a[part][3] = h2fma((hi & 0x00f000f0u) | kMagic, 0x2C002C00u, zc.c[hf][1]);
+      }
+    } else if constexpr (FMT == FMT_Q3) {
+      const uint32_t w[3] = {r.v.x, r.v.y, r.w2};
+      const uint32_t ws[3] = {r.v.x >> 9, r.v.y >> 9, r.w2 >> 9};
+#pragma unroll
+      for (int p = 0; p < 16; ++p) {
+        const int part = p >> 2, j = p & 3, hf = part & 1;
+        uint32_t v;
+        if (p < 15) {
+          const int wi = p / 5, f = p % 5, ff = f >= 3 ? f - 3 : f;
+          const uint32_t src = f >= 3 ? ws[wi] : w[wi];
+          const uint32_t h = (src & (0x00070007u << (3 * ff))) | kMagic;
+          if (ff == 0) v = h2sub(h, zc.c[hf][0]);
+          else if (ff == 1) v = h2fma(h, 0x30003000u, zc.c[hf][1]);
+          else v = h2fma(h, 0x24002400u, zc.c[hf][2]);
+        } else {
+          uint32_t h = ((w[0] >> 15) & 0x00010001u) | kMagic;
+          h |= (w[1] >> 14) & 0x00020002u;
+          h |= (w[2] >> 13) & 0x00040004u;
+          v = h2sub(h, zc.c[hf][0]);
+        }
+        a[part][j] = v;
+      }
+    } else {   // FMT_Q8
+#pragma unroll
+      for (int part = 0; part < 4; ++part) {
+        const int hf = part & 1;
+        const uint4 u = r.v[part >> 1];
+        const uint32_t w0 = hf ? u.z : u.x, w1 = hf ? u.w : u.y;
+        a[part][0] = h2sub((w0 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[part][1] = h2sub(((w0 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[part][2] = h2sub((w1 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[part][3] = h2sub(((w1 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+      }
+    }
+    const uint32_t s_a = (sc2 & 0xffffu) * 0x00010001u, s_b = (sc2 >> 16) * 0x00010001u;
+#pragma unroll
+    for (int part = 0; part < 4; ++part)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) out[part][j] = h2mul(a[part][j], (part & 1) ? s_b : s_a);
+  }
+#pragma unroll
+  for (int part = 0; part < 4; ++part) {
+    const int row = row0 + g + 8 * (part & 1);
+    const int chunk = (part >> 1) * 4 + t;                      // 16-byte chunk index along K inside the 128-byte row
+    uint8_t* dst = btile + row * 128 + ((chunk ^ (row & 7)) << 4);
+    *reinterpret_cast<uint4*>(dst) = make_uint4(out[part][0], out[part][1], out[part][2], out[part][3]);
+  }
+}
+
+// One part (W or the K-extension B) of the dequant warps' work: k-blocks [0, nkb) of `mat`, landing in
+// pipeline iterations kb0 .. kb0 + nkb - 1.
+template <int FMT>
+__device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int bn, int nkb, int kb0, int dw, int lane,
+                                             uint8_t* smem, const PrefillArgs& p, uint64_t* full_w, uint64_t* empty) {
+  if constexpr (FMT == FMT_NONE) {
+    return true;
+  } else {
+    const int tiles_per_warp = bn / (16 * kDqWarps) > 0 ? bn / (16 * kDqWarps) : 1;   // 2 (bn 256) or 1
+    const int my_first = dw * tiles_per_warp;
+    const bool active = my_first * 16 < bn;
+    const int g = lane >> 2;
+    constexpr bool quant = FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8;
+    const int tb = tile_bytes(FMT);
+    const int gt = mat.group / 64;
+    Packed<FMT> pk[kPrefetch][2];
+    auto issue = [&](int kb, int slot) {
+      if (!active || kb >= nkb) return;
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (i < tiles_per_warp) {
+          const int rt = (n0 >> 4) + my_first + i;
+          if (rt < mat.nt) load_packed<FMT>(pk[slot][i], mat.q + ((int64_t)rt * mat.kc + kb) * tb, lane);
+        }
+      }
+    };
+#pragma unroll
+    for (int j = 0; j < kPrefetch; ++j) issue(j, j);
+    for (int kbb = 0; kbb < nkb; kbb += kPrefetch) {
+#pragma unroll
+      for (int j = 0; j < kPrefetch; ++j) {
+        const int kb = kbb + j;
+        if (kb < nkb) {
+          const int it = kb0 + kb, s = it % p.stages;
+          if (it >= p.stages && !mbar_wait(empty + s, ((it / p.stages) - 1) & 1, p.dev_status)) return false;
+          if (active) {
+            uint8_t* btile = smem + (size_t)s * p.stage_bytes + BM * 128;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+              if (i < tiles_per_warp) {
+                const int rt = (n0 >> 4) + my_first + i;
+                if (rt < mat.nt) {
+                  uint32_t sc2 = 0, zz2 = 0;
+                  if constexpr (quant) {
+                    const int64_t si = ((int64_t)rt * mat.ng + kb / gt) * 8 + g;
+                    sc2 = __ldg(mat.sc + si); zz2 = __ldg(mat.zz + si);
+                  }
+                  dequant_store<FMT>(pk[j][i], sc2, zz2, btile, (my_first + i) * 16, lane);
+                }
+              }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(full_w + s);
+          issue(kb + kPrefetch, j);
+        }
+      }
+    }
+    return true;
+  }
+}
+
+template <int WF, int BF>
+__global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant__ CUtensorMap tm_x,
+                                                          const __grid_constant__ CUtensorMap tm_t, const PrefillArgs p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_x[kMaxStagesP], full_w[kMaxStagesP], empty[kMaxStagesP], acc_full;
+  __shared__ uint32_t tmem_base_s;
+  // 1024-byte alignment of the operand tiles (the swizzle pattern is anchored at 1 KB)
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * p.bn;
+  const int nkb = p.nkb_w + p.nkb_b;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.stages; ++i) { mbar_init(full_x + i, 1); mbar_init(full_w + i, kDqWarps); mbar_init(empty + i, 1); }
+    mbar_init(&acc_full, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 2) {   // tensor memory: 256 fp32 columns x 128 lanes for the accumulator
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(256u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_d = tmem_base_s;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (activations)
+    if (lane == 0) {
+      for (int it = 0; it < nkb; ++it) {
+        const int s = it % p.stages;
+        if (it >= p.stages && !mbar_wait(empty + s, ((it / p.stages) - 1) & 1, p.dev_status)) break;
+        mbar_expect_tx(full_x + s, BM * 128);
+        uint8_t* xt = smem + (size_t)s * p.stage_bytes;
+        if (it < p.nkb_w) tma_load_2d(xt, &tm_x, it * BK, m0, full_x + s);
+        else tma_load_2d(xt, &tm_t, (it - p.nkb_w) * BK, m0, full_x + s);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, fp16 x fp16, both operands K-major, N = bn, M = 128
+      const uint32_t idesc = (1u << 4) | ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < nkb && ok; ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        ok = mbar_wait(full_x + s, ph, p.dev_status) && mbar_wait(full_w + s, ph, p.dev_status);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint8_t* xt = smem + (size_t)s * p.stage_bytes;
+        const uint64_t adesc = make_desc(xt), bdesc = make_desc(xt + BM * 128);
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k)          // 32 bytes (16 fp16) further along K per step: +2 in the address field
+          umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+        umma_commit(empty + s);                     // arrives when these MMAs have finished reading the stage
+      }
+      umma_commit(&acc_full);                       // arrives when every MMA above has completed
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ dequant warps, then epilogue
+    const int dw = warp - 4;
+    bool ok = dequant_part<WF>(p.w, n0, p.bn, p.nkb_w, 0, dw, lane, smem, p, full_w, empty);
+    if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, p.bn, p.nkb_b, p.nkb_w, dw, lane, smem, p, full_w, empty);
+    if (dw < 4) {
+      // epilogue: warp dw owns accumulator rows 32*dw .. 32*dw+31 (= its TMEM lanes)
+      if (ok) ok = mbar_wait(&acc_full, 0, p.dev_status);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int row = m0 + dw * 32 + lane;
+      if (ok) {
+        for (int c0 = 0; c0 < p.bn; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem_d + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          const int col = n0 + c0;
+          if (row < p.m && col < p.n_valid) {
+            if (p.out_dtype == EORA_Y_F32) {
+              float* o = reinterpret_cast<float*>(p.out) + (int64_t)row * p.ld_out + col;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                if (col + j < p.n_valid)
+                  *reinterpret_cast<float4*>(o + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+            } else {
+              uint16_t* o = reinterpret_cast<uint16_t*>(p.out) + (int64_t)row * p.ld_out + col;
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                if (col + j < p.n_valid) {
+                  uint32_t h[4];
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    const float f0 = __uint_as_float(v[j + 2 * q]), f1 = __uint_as_float(v[j + 2 * q + 1]);
+                    if (p.out_dtype == EORA_Y_F16) {
+                      __half2 hh = __floats2half2_rn(f0, f1);
+                      h[q] = *reinterpret_cast<uint32_t*>(&hh);
+                    } else {
+                      __nv_bfloat162 bb = __floats2bfloat162_rn(f0, f1);
+                      h[q] = *reinterpret_cast<uint32_t*>(&bb);
+                    }
+                  }
+                  *reinterpret_cast<uint4*>(o + j) = make_uint4(h[0], h[1], h[2], h[3]);
+                }
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(256u) : "memory");
+}
+
+__global__ void k_bf16_to_f16(const __nv_bfloat16* in, __half* out, int64_t n) {
+  for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 2; i < n; i += (int64_t)gridDim.x * blockDim.x * 2) {
+    float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(in + i));
+    *reinterpret_cast<__half2*>(out + i) = __floats2half2_rn(f.x, f.y);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || !p) return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// fp16 [rows][cols] row-major, box = 64 columns x 128 rows, 128-byte swizzle, zero fill out of bounds
+bool make_map(CUtensorMap* tm, const void* base, int rows, int cols, int ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kSmemP = 225 * 1024;
+
+template <auto KERNEL>
+cudaError_t launch_p(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt, const PrefillArgs& a) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  KERNEL<<<grid, kThreadsP, smem, st>>>(tx, tt, a);
+  return cudaGetLastError();
+}
+
+template <int WF>
+cudaError_t launch_bf(int bf, dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt,
+                      const PrefillArgs& a) {
+  switch (bf) {
+    case FMT_F16: return launch_p<k_prefill<WF, FMT_F16>>(grid, smem, st, tx, tt, a);
+    case FMT_Q4: return launch_p<k_prefill<WF, FMT_Q4>>(grid, smem, st, tx, tt, a);
+    case FMT_Q8: return launch_p<k_prefill<WF, FMT_Q8>>(grid, smem, st, tx, tt, a);
+    default: return launch_p<k_prefill<WF, FMT_NONE>>(grid, smem, st, tx, tt, a);
+  }
+}
+
+cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt,
+                       const PrefillArgs& a) {
+  switch (wf) {
+    case FMT_Q4: return launch_bf<FMT_Q4>(bf, grid, smem, st, tx, tt, a);
+    case FMT_Q3: return launch_bf<FMT_Q3>(bf, grid, smem, st, tx, tt, a);
+    case FMT_SP24: return launch_bf<FMT_SP24>(bf, grid, smem, st, tx, tt, a);
+    // A as the weight of the first launch (t = X.A): no K-extension there
+    case FMT_F16: return launch_p<k_prefill<FMT_F16, FMT_NONE>>(grid, smem, st, tx, tt, a);
+    case FMT_Q8: return launch_p<k_prefill<FMT_Q8, FMT_NONE>>(grid, smem, st, tx, tt, a);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+void fill_stages(PrefillArgs& a) {
+  a.stage_bytes = BM * 128 + a.bn * 128;
+  a.stages = (kSmemP - 2048) / a.stage_bytes;
+  if (a.stages > kMaxStagesP) a.stages = kMaxStagesP;
+}
+
+}  // namespace
+
+bool prefill_supported(const Handle* h, int m) {
+  if (m <= 64) return false;
+  if (h->w.group % 64) return false;
+  return encode_fn() != nullptr;
+}
+
+int prefill_launch_count(const Handle* h, int) {
+  return (h->cfg.rank > 0 ? 2 : 1) + (h->cfg.x_dtype == EORA_X_BF16 ? 1 : 0);
+}
+
+cudaError_t prefill_init(Handle* h) {
+  h->prefill_state = nullptr;
+  if (h->cfg.max_m <= 64 || h->cfg.x_dtype != EORA_X_BF16) return cudaSuccess;
+  PrefillState* ps = new PrefillState();
+  cudaError_t e = cudaMalloc(&ps->x16, (size_t)h->cfg.max_m * h->cfg.d_in * 2);
+  if (e != cudaSuccess) { delete ps; return e; }
+  h->prefill_state = ps;
+  return cudaSuccess;
+}
+
+void prefill_free(Handle* h) {
+  PrefillState* ps = reinterpret_cast<PrefillState*>(h->prefill_state);
+  if (!ps) return;
+  cudaFree(ps->x16);
+  delete ps;
+  h->prefill_state = nullptr;
+}
+
+cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st) {
+  const eora_linear_config& c = h->cfg;
+  const void* x16 = x;
+  if (c.x_dtype == EORA_X_BF16) {
+    PrefillState* ps = reinterpret_cast<PrefillState*>(h->prefill_state);
+    if (!ps) return cudaErrorInvalidValue;
+    int64_t n = (int64_t)m * c.d_in;
+    int64_t blocks = (n / 2 + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    k_bf16_to_f16<<<(int)blocks, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), ps->x16, n);
+    x16 = ps->x16;
+  }
+  CUtensorMap tm_x, tm_t;
+  if (!make_map(&tm_x, x16, m, c.d_in, c.d_in)) return cudaErrorInvalidValue;
+  const bool ab = c.rank > 0;
+  if (ab) {
+    if (!make_map(&tm_t, h->t16, m, h->r_pad, h->r_pad)) return cudaErrorInvalidValue;
+    // launch 1: t = X.A  (A as the weight: rows = r_pad, fp16 output into t16)
+    PrefillArgs a = {};
+    a.w = h->a; a.b = WMat(); a.b.fmt = FMT_NONE;
+    a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m;
+    a.bn = (h->r_pad % 128 == 0) ? 128 : 64;
+    a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status;
+    fill_stages(a);
+    dim3 grid(h->r_pad / a.bn, (m + BM - 1) / BM);
+    cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, a.stages * a.stage_bytes + 1024, st, tm_x, tm_x, a);
+    if (e != cudaSuccess) return e;
+  } else {
+    tm_t = tm_x;
+  }
+  PrefillArgs a = {};
+  a.w = h->w; a.b = h->b;
+  if (!ab) a.b.fmt = FMT_NONE;
+  a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m;
+  a.bn = 256;
+  a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
+  fill_stages(a);
+  dim3 grid((c.d_out + a.bn - 1) / a.bn, (m + BM - 1) / BM);
+  return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, a.stages * a.stage_bytes + 1024, st, tm_x, tm_t, a);
+}
+
 }  // namespace eora
