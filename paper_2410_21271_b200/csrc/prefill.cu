@@ -24,10 +24,11 @@ using namespace dec;
 namespace {
 
 constexpr int BM = 128, BK = 64;
-constexpr int kDqWarps = 8;                     // dequant warps (warps 4..11); warps 4..7 are also the epilogue
+constexpr int kDqWarps = 16;                    // dequant warps (warps 4..19); warps 4..7 are also the epilogue
 constexpr int kThreadsP = (4 + kDqWarps) * 32;  // warp 0: TMA, warp 1: MMA, warp 2: TMEM alloc, warp 3: idle
-constexpr int kMaxStagesP = 6;
-constexpr int kPrefetch = 4;                    // k-blocks of packed weights held in registers ahead of use
+constexpr int kMaxXStages = 8;                   // ring of activation tiles (TMA latency is long: deep)
+constexpr int kMaxBStages = 4;                   // ring of dequantised weight tiles (produced on chip: shallow)
+constexpr int kPrefetch = 4;                    // k-blocks of packed weights held in registers ahead of use (2 for fp16)
 
 struct PrefillArgs {
   WMat w;            // weight operand of the first nkb_w k-blocks (rows = output columns)
@@ -39,10 +40,13 @@ struct PrefillArgs {
   int m;
   int bn;            // N tile: 64, 128 or 256
   int nkb_w, nkb_b;  // k-blocks of each part
-  int stages;
-  int stage_bytes;   // BM*128 + bn*128
+  int sx, sb;        // stages of the activation ring / of the weight ring
+  int b_off;         // byte offset of the weight ring (after sx activation tiles of BM*128 bytes)
   int* dev_status;
+  long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (dequant start, B ready, X ready, MMA issued)
 };
+
+#define PTRACE(it, slot) do { if (p.trace && blockIdx.x == 0 && blockIdx.y == 0) p.trace[(it) * 4 + (slot)] = clock64(); } while (0)
 
 struct PrefillState {
   __half* x16;       // fp16 copy of a bf16 X, [max_m][d_in]
@@ -207,61 +211,50 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
 }
 
 // One part (W or the K-extension B) of the dequant warps' work: k-blocks [0, nkb) of `mat`, landing in
-// pipeline iterations kb0 .. kb0 + nkb - 1.
+// pipeline iterations kb0 .. kb0 + nkb - 1.  Each active warp owns one 16-row tile of the N tile; packed
+// weights, scales and zero-points are loaded PF k-blocks ahead into registers.
 template <int FMT>
 __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int bn, int nkb, int kb0, int dw, int lane,
                                              uint8_t* smem, const PrefillArgs& p, uint64_t* full_w, uint64_t* empty) {
   if constexpr (FMT == FMT_NONE) {
     return true;
   } else {
-    const int tiles_per_warp = bn / (16 * kDqWarps) > 0 ? bn / (16 * kDqWarps) : 1;   // 2 (bn 256) or 1
-    const int my_first = dw * tiles_per_warp;
-    const bool active = my_first * 16 < bn;
-    const int g = lane >> 2;
+    constexpr int PF = FMT == FMT_F16 ? 2 : kPrefetch;
     constexpr bool quant = FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8;
+    const int rt = (n0 >> 4) + dw;                       // this warp's row tile
+    const bool active = dw * 16 < bn && rt < mat.nt;
+    const int g = lane >> 2;
     const int tb = tile_bytes(FMT);
     const int gt = mat.group / 64;
-    Packed<FMT> pk[kPrefetch][2];
+    Packed<FMT> pk[PF];
+    uint32_t scq[PF], zzq[PF];
     auto issue = [&](int kb, int slot) {
       if (!active || kb >= nkb) return;
-#pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        if (i < tiles_per_warp) {
-          const int rt = (n0 >> 4) + my_first + i;
-          if (rt < mat.nt) load_packed<FMT>(pk[slot][i], mat.q + ((int64_t)rt * mat.kc + kb) * tb, lane);
-        }
+      load_packed<FMT>(pk[slot], mat.q + ((int64_t)rt * mat.kc + kb) * tb, lane);
+      if constexpr (quant) {
+        const int64_t si = ((int64_t)rt * mat.ng + kb / gt) * 8 + g;
+        scq[slot] = __ldg(mat.sc + si);
+        zzq[slot] = __ldg(mat.zz + si);
       }
     };
 #pragma unroll
-    for (int j = 0; j < kPrefetch; ++j) issue(j, j);
-    for (int kbb = 0; kbb < nkb; kbb += kPrefetch) {
+    for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(j, j); }
+    for (int kbb = 0; kbb < nkb; kbb += PF) {
 #pragma unroll
-      for (int j = 0; j < kPrefetch; ++j) {
+      for (int j = 0; j < PF; ++j) {
         const int kb = kbb + j;
         if (kb < nkb) {
-          const int it = kb0 + kb, s = it % p.stages;
-          if (it >= p.stages && !mbar_wait(empty + s, ((it / p.stages) - 1) & 1, p.dev_status)) return false;
+          const int it = kb0 + kb, s = it % p.sb;
+          if (it >= p.sb && !mbar_wait(empty + s, ((it / p.sb) - 1) & 1, p.dev_status)) return false;
+          if (dw == 0 && lane == 0) PTRACE(it, 0);
           if (active) {
-            uint8_t* btile = smem + (size_t)s * p.stage_bytes + BM * 128;
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              if (i < tiles_per_warp) {
-                const int rt = (n0 >> 4) + my_first + i;
-                if (rt < mat.nt) {
-                  uint32_t sc2 = 0, zz2 = 0;
-                  if constexpr (quant) {
-                    const int64_t si = ((int64_t)rt * mat.ng + kb / gt) * 8 + g;
-                    sc2 = __ldg(mat.sc + si); zz2 = __ldg(mat.zz + si);
-                  }
-                  dequant_store<FMT>(pk[j][i], sc2, zz2, btile, (my_first + i) * 16, lane);
-                }
-              }
-            }
+            uint8_t* btile = smem + p.b_off + (size_t)s * p.bn * 128;
+            dequant_store<FMT>(pk[j], scq[j], zzq[j], btile, dw * 16, lane);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
           }
           __syncwarp();
-          if (lane == 0) mbar_arrive(full_w + s);
-          issue(kb + kPrefetch, j);
+          if (lane == 0) { mbar_arrive(full_w + s); if (dw == 0) PTRACE(it, 1); }
+          issue(kb + PF, j);
         }
       }
     }
@@ -273,7 +266,7 @@ template <int WF, int BF>
 __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant__ CUtensorMap tm_x,
                                                           const __grid_constant__ CUtensorMap tm_t, const PrefillArgs p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_x[kMaxStagesP], full_w[kMaxStagesP], empty[kMaxStagesP], acc_full;
+  __shared__ __align__(8) uint64_t full_x[kMaxXStages], empty_x[kMaxXStages], full_w[kMaxBStages], empty_w[kMaxBStages], acc_full;
   __shared__ uint32_t tmem_base_s;
   // 1024-byte alignment of the operand tiles (the swizzle pattern is anchored at 1 KB)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -283,7 +276,8 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   const int nkb = p.nkb_w + p.nkb_b;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < p.stages; ++i) { mbar_init(full_x + i, 1); mbar_init(full_w + i, kDqWarps); mbar_init(empty + i, 1); }
+    for (int i = 0; i < p.sx; ++i) { mbar_init(full_x + i, 1); mbar_init(empty_x + i, 1); }
+    for (int i = 0; i < p.sb; ++i) { mbar_init(full_w + i, kDqWarps); mbar_init(empty_w + i, 1); }
     mbar_init(&acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -301,10 +295,10 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
     // ------------------------------------------------------------------ TMA producer (activations)
     if (lane == 0) {
       for (int it = 0; it < nkb; ++it) {
-        const int s = it % p.stages;
-        if (it >= p.stages && !mbar_wait(empty + s, ((it / p.stages) - 1) & 1, p.dev_status)) break;
+        const int s = it % p.sx;
+        if (it >= p.sx && !mbar_wait(empty_x + s, ((it / p.sx) - 1) & 1, p.dev_status)) break;
         mbar_expect_tx(full_x + s, BM * 128);
-        uint8_t* xt = smem + (size_t)s * p.stage_bytes;
+        uint8_t* xt = smem + (size_t)s * (BM * 128);
         if (it < p.nkb_w) tma_load_2d(xt, &tm_x, it * BK, m0, full_x + s);
         else tma_load_2d(xt, &tm_t, (it - p.nkb_w) * BK, m0, full_x + s);
       }
@@ -316,25 +310,29 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       const uint32_t idesc = (1u << 4) | ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       bool ok = true;
       for (int it = 0; it < nkb && ok; ++it) {
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
-        ok = mbar_wait(full_x + s, ph, p.dev_status) && mbar_wait(full_w + s, ph, p.dev_status);
+        const int sx = it % p.sx, sb = it % p.sb;
+        ok = mbar_wait(full_x + sx, (it / p.sx) & 1, p.dev_status);
+        if (!ok) break;
+        PTRACE(it, 2);
+        ok = mbar_wait(full_w + sb, (it / p.sb) & 1, p.dev_status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint8_t* xt = smem + (size_t)s * p.stage_bytes;
-        const uint64_t adesc = make_desc(xt), bdesc = make_desc(xt + BM * 128);
+        const uint64_t adesc = make_desc(smem + (size_t)sx * (BM * 128));
+        const uint64_t bdesc = make_desc(smem + p.b_off + (size_t)sb * p.bn * 128);
 #pragma unroll
         for (int k = 0; k < BK / 16; ++k)          // 32 bytes (16 fp16) further along K per step: +2 in the address field
           umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
-        umma_commit(empty + s);                     // arrives when these MMAs have finished reading the stage
+        umma_commit(empty_x + sx);                  // both arrive when these MMAs have finished reading their operands
+        umma_commit(empty_w + sb);
+        PTRACE(it, 3);
       }
       umma_commit(&acc_full);                       // arrives when every MMA above has completed
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ dequant warps, then epilogue
     const int dw = warp - 4;
-    bool ok = dequant_part<WF>(p.w, n0, p.bn, p.nkb_w, 0, dw, lane, smem, p, full_w, empty);
-    if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, p.bn, p.nkb_b, p.nkb_w, dw, lane, smem, p, full_w, empty);
+    bool ok = dequant_part<WF>(p.w, n0, p.bn, p.nkb_w, 0, dw, lane, smem, p, full_w, empty_w);
+    if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, p.bn, p.nkb_b, p.nkb_w, dw, lane, smem, p, full_w, empty_w);
     if (dw < 4) {
       // epilogue: warp dw owns accumulator rows 32*dw .. 32*dw+31 (= its TMEM lanes)
       if (ok) ok = mbar_wait(&acc_full, 0, p.dev_status);
@@ -459,10 +457,13 @@ cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, con
   }
 }
 
-void fill_stages(PrefillArgs& a) {
-  a.stage_bytes = BM * 128 + a.bn * 128;
-  a.stages = (kSmemP - 2048) / a.stage_bytes;
-  if (a.stages > kMaxStagesP) a.stages = kMaxStagesP;
+int fill_stages(PrefillArgs& a) {      // returns the dynamic shared memory to request
+  a.sb = 3;
+  const int b_bytes = a.sb * a.bn * 128;
+  a.sx = (kSmemP - 3072 - b_bytes) / (BM * 128);
+  if (a.sx > kMaxXStages) a.sx = kMaxXStages;
+  a.b_off = a.sx * BM * 128;
+  return a.b_off + b_bytes + 1024;
 }
 
 }  // namespace
@@ -518,9 +519,9 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m;
     a.bn = (h->r_pad % 128 == 0) ? 128 : 64;
     a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status;
-    fill_stages(a);
+    const int smem_t = fill_stages(a);
     dim3 grid(h->r_pad / a.bn, (m + BM - 1) / BM);
-    cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, a.stages * a.stage_bytes + 1024, st, tm_x, tm_x, a);
+    cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_x, tm_x, a);
     if (e != cudaSuccess) return e;
   } else {
     tm_t = tm_x;
@@ -531,9 +532,10 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m;
   a.bn = 256;
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
-  fill_stages(a);
+  a.trace = reinterpret_cast<long long*>(h->trace);
+  const int smem_y = fill_stages(a);
   dim3 grid((c.d_out + a.bn - 1) / a.bn, (m + BM - 1) / BM);
-  return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, a.stages * a.stage_bytes + 1024, st, tm_x, tm_t, a);
+  return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, a);
 }
 
 }  // namespace eora
