@@ -1,18 +1,22 @@
 // Prefill kernel family (M > 64): Y = X.deq(Wq) + (X.A).B  (paper Eq. 4) as a tcgen05 GEMM.
 //
 // The paper measures only batch-1 decoding (Section 4.5); for many tokens the layer is a dense
-// contraction, so it runs on the 5th-generation tensor cores:
-//   * activations (M x K, K-major) arrive by TMA (cp.async.bulk.tensor, 128-byte swizzle, no
-//     multicast) into a ring of shared-memory stages;
-//   * the packed weights are read by eight "dequant" warps straight from global memory (the tiles of
-//     the shared layout are 512-byte contiguous per warp), turned into fp16 RN((q - z) * s) in
-//     registers and stored as the K-major, 128-byte-swizzled B operand of the same stage;
-//   * one thread issues tcgen05.mma (M = 128, N = BN, K = 16) with the fp32 accumulator in tensor
-//     memory; tcgen05.commit releases a stage when its MMAs have drained;
+// contraction, so it runs on the 5th-generation tensor cores.  The product is computed transposed,
+// Yt[n][m] = sum_k w[n][k] X[m][k], so that the operand that has to be produced on chip is the small one:
+//   * MMA "A" operand (128 rows): a tile of 128 output columns n of the weights.  Sixteen dequant warps
+//     read the packed tiles of the shared layout straight from global memory (512 contiguous bytes per
+//     warp), turn them into fp16 RN((q - z) * s) in registers and store them as a K-major,
+//     128-byte-swizzled operand tile (bank-conflict-free stores);
+//   * MMA "B" operand (up to 256 rows): a tile of tokens of X, K-major, brought in by TMA
+//     (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a deep ring, because TMA latency is
+//     several k-blocks long;
+//   * one thread issues tcgen05.mma (M = 128, N = tokens, K = 16) with the fp32 accumulator in tensor
+//     memory; tcgen05.commit releases the ring slots when the MMAs have drained;
 //   * the low-rank term is a K-extension: after the d_in/64 backbone k-blocks come r/64 k-blocks whose
-//     activation operand is t = X.A (fp16, from a first launch of the same kernel with A as the
-//     weight) and whose weight operand is B, so (X.A).B lands in the same accumulator and Y is
-//     written once by the epilogue (tcgen05.ld -> convert -> global).
+//     token operand is t = X.A (fp16, from a first launch of the same kernel with A as the weight) and
+//     whose weight operand is B, so (X.A).B lands in the same accumulator;
+//   * epilogue: tcgen05.ld -> fp16/bf16/fp32 -> transpose through shared memory -> 16-byte row stores,
+//     so Y is written once.
 // Launches per forward: 1 (rank 0) or 2 (t = X.A, then the main product), plus a conversion launch
 // when X is bf16 (the f16 MMA kind needs both operands in fp16; weights are kept fp16 because
 // bf16 weights alone cost 1.7e-3 of the 2e-3 error budget).
@@ -23,11 +27,11 @@ namespace eora {
 using namespace dec;
 namespace {
 
-constexpr int BM = 128, BK = 64;
-constexpr int kDqWarps = 16;                    // dequant warps (warps 4..19); warps 4..7 are also the epilogue
+constexpr int BN_W = 128, BK = 64;               // weight rows per CTA tile (the MMA M), k-block
+constexpr int kDqWarps = 16;                    // dequant warps (warps 4..19): 8 row tiles x 2 k-block parities
 constexpr int kThreadsP = (4 + kDqWarps) * 32;  // warp 0: TMA, warp 1: MMA, warp 2: TMEM alloc, warp 3: idle
-constexpr int kMaxXStages = 8;                   // ring of activation tiles (TMA latency is long: deep)
-constexpr int kMaxBStages = 4;                   // ring of dequantised weight tiles (produced on chip: shallow)
+constexpr int kMaxXStages = 8;                  // ring of token tiles (TMA latency is long: deep)
+constexpr int kMaxWStages = 4;                  // ring of dequantised weight tiles (produced on chip: shallow)
 constexpr int kPrefetch = 4;                    // k-blocks of packed weights held in registers ahead of use (2 for fp16)
 
 struct PrefillArgs {
@@ -38,12 +42,12 @@ struct PrefillArgs {
   int ld_out;        // leading dimension of out (elements)
   int n_valid;       // columns of out to write
   int m;
-  int bn;            // N tile: 64, 128 or 256
+  int bt;            // token tile (the MMA N): multiple of 16, at most 256
   int nkb_w, nkb_b;  // k-blocks of each part
-  int sx, sb;        // stages of the activation ring / of the weight ring
-  int b_off;         // byte offset of the weight ring (after sx activation tiles of BM*128 bytes)
+  int sx, sw;        // stages of the token ring / of the weight ring
+  int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
   int* dev_status;
-  long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (dequant start, B ready, X ready, MMA issued)
+  long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (dequant start, W ready, X ready, MMA issued)
 };
 
 #define PTRACE(it, slot) do { if (p.trace && blockIdx.x == 0 && blockIdx.y == 0) p.trace[(it) * 4 + (slot)] = clock64(); } while (0)
@@ -201,31 +205,41 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
 #pragma unroll
       for (int j = 0; j < 4; ++j) out[part][j] = h2mul(a[part][j], (part & 1) ? s_b : s_a);
   }
+  // Store order: in step k lanes with even g write their blk = k/2 part and lanes with odd g the other
+  // one, so that the 8 lanes of a quarter warp (two rows) hit 8 different 16-byte columns of the swizzle.
+  const int odd = g & 1;
 #pragma unroll
-  for (int part = 0; part < 4; ++part) {
-    const int row = row0 + g + 8 * (part & 1);
-    const int chunk = (part >> 1) * 4 + t;                      // 16-byte chunk index along K inside the 128-byte row
+  for (int k = 0; k < 4; ++k) {
+    const int hf = k & 1, blk_even = k >> 1;
+    const int blk = blk_even ^ odd;
+    const int pe = blk_even * 2 + hf, po = (blk_even ^ 1) * 2 + hf;
+    const uint4 v = odd ? make_uint4(out[po][0], out[po][1], out[po][2], out[po][3])
+                        : make_uint4(out[pe][0], out[pe][1], out[pe][2], out[pe][3]);
+    const int row = row0 + g + 8 * hf;
+    const int chunk = blk * 4 + t;                              // 16-byte chunk index along K inside the 128-byte row
     uint8_t* dst = btile + row * 128 + ((chunk ^ (row & 7)) << 4);
-    *reinterpret_cast<uint4*>(dst) = make_uint4(out[part][0], out[part][1], out[part][2], out[part][3]);
+    *reinterpret_cast<uint4*>(dst) = v;
   }
 }
 
-// One part (W or the K-extension B) of the dequant warps' work: k-blocks [0, nkb) of `mat`, landing in
-// pipeline iterations kb0 .. kb0 + nkb - 1.  Each active warp owns one 16-row tile of the N tile; packed
-// weights, scales and zero-points are loaded PF k-blocks ahead into registers.
+// One part (W or the K-extension B) of a dequant warp's work.  The warp owns row tile `tile` (0..7) of
+// the CTA's 128 weight rows and the k-blocks of `mat` with kb = par (mod 2); k-block kb lands in pipeline
+// iteration kb0 + kb.  Packed weights, scales and zero-points are loaded PF of its k-blocks ahead.
 template <int FMT>
-__device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int bn, int nkb, int kb0, int dw, int lane,
-                                             uint8_t* smem, const PrefillArgs& p, uint64_t* full_w, uint64_t* empty) {
+__device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int nkb, int kb0, int tile, int par, int lane,
+                                             uint8_t* smem, const PrefillArgs& p, uint64_t* full_w, uint64_t* empty_w) {
   if constexpr (FMT == FMT_NONE) {
     return true;
   } else {
     constexpr int PF = FMT == FMT_F16 ? 2 : kPrefetch;
     constexpr bool quant = FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8;
-    const int rt = (n0 >> 4) + dw;                       // this warp's row tile
-    const bool active = dw * 16 < bn && rt < mat.nt;
+    const int rt = (n0 >> 4) + tile;                     // this warp's row tile of the matrix
+    const bool active = rt < mat.nt;
     const int g = lane >> 2;
     const int tb = tile_bytes(FMT);
     const int gt = mat.group / 64;
+    // the warp's k-blocks are kb = first, first + 2, ... where first has the parity that makes (kb0 + kb) % 2 == par
+    const int first = (par ^ (kb0 & 1)) & 1;
     Packed<FMT> pk[PF];
     uint32_t scq[PF], zzq[PF];
     auto issue = [&](int kb, int slot) {
@@ -238,23 +252,30 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int bn, in
       }
     };
 #pragma unroll
-    for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(j, j); }
-    for (int kbb = 0; kbb < nkb; kbb += PF) {
+    for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(first + 2 * j, j); }
+    for (int kbb = first; kbb < nkb; kbb += 2 * PF) {
 #pragma unroll
       for (int j = 0; j < PF; ++j) {
-        const int kb = kbb + j;
+        const int kb = kbb + 2 * j;
         if (kb < nkb) {
-          const int it = kb0 + kb, s = it % p.sb;
-          if (it >= p.sb && !mbar_wait(empty + s, ((it / p.sb) - 1) & 1, p.dev_status)) return false;
-          if (dw == 0 && lane == 0) PTRACE(it, 0);
+          const int it = kb0 + kb, s = it % p.sw;
+          if (it >= p.sw && !mbar_wait(empty_w + s, ((it / p.sw) - 1) & 1, p.dev_status)) return false;
+          if (tile == 0 && lane == 0) PTRACE(it, 0);
+          uint8_t* wt = smem + p.w_off + (size_t)s * (BN_W * 128);
           if (active) {
-            uint8_t* btile = smem + p.b_off + (size_t)s * p.bn * 128;
-            dequant_store<FMT>(pk[j], scq[j], zzq[j], btile, dw * 16, lane);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
+            dequant_store<FMT>(pk[j], scq[j], zzq[j], wt, tile * 16, lane);
+          } else {                                        // rows past the matrix: keep the operand finite
+            const int gg = lane >> 2, tt = lane & 3;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const int row = tile * 16 + gg + 8 * (k & 1), chunk = (k >> 1) * 4 + tt;
+              *reinterpret_cast<uint4*>(wt + row * 128 + ((chunk ^ (row & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+            }
           }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
           __syncwarp();
-          if (lane == 0) { mbar_arrive(full_w + s); if (dw == 0) PTRACE(it, 1); }
-          issue(kb + PF, j);
+          if (lane == 0) { mbar_arrive(full_w + s); if (tile == 0) PTRACE(it, 1); }
+          issue(kb + 2 * PF, j);
         }
       }
     }
@@ -266,18 +287,19 @@ template <int WF, int BF>
 __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant__ CUtensorMap tm_x,
                                                           const __grid_constant__ CUtensorMap tm_t, const PrefillArgs p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_x[kMaxXStages], empty_x[kMaxXStages], full_w[kMaxBStages], empty_w[kMaxBStages], acc_full;
+  __shared__ __align__(8) uint64_t full_x[kMaxXStages], empty_x[kMaxXStages], full_w[kMaxWStages], empty_w[kMaxWStages], acc_full;
   __shared__ uint32_t tmem_base_s;
   // 1024-byte alignment of the operand tiles (the swizzle pattern is anchored at 1 KB)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * p.bn;
+  const int n0 = blockIdx.x * BN_W, m0 = blockIdx.y * p.bt;
   const int nkb = p.nkb_w + p.nkb_b;
+  const uint32_t xbytes = (uint32_t)p.bt * 128;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.sx; ++i) { mbar_init(full_x + i, 1); mbar_init(empty_x + i, 1); }
-    for (int i = 0; i < p.sb; ++i) { mbar_init(full_w + i, kDqWarps); mbar_init(empty_w + i, 1); }
+    for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8); mbar_init(empty_w + i, 1); }
     mbar_init(&acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -292,13 +314,13 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   const uint32_t tmem_d = tmem_base_s;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer (activations)
+    // ------------------------------------------------------------------ TMA producer (token tiles)
     if (lane == 0) {
       for (int it = 0; it < nkb; ++it) {
         const int s = it % p.sx;
         if (it >= p.sx && !mbar_wait(empty_x + s, ((it / p.sx) - 1) & 1, p.dev_status)) break;
-        mbar_expect_tx(full_x + s, BM * 128);
-        uint8_t* xt = smem + (size_t)s * (BM * 128);
+        mbar_expect_tx(full_x + s, xbytes);
+        uint8_t* xt = smem + (size_t)s * xbytes;
         if (it < p.nkb_w) tma_load_2d(xt, &tm_x, it * BK, m0, full_x + s);
         else tma_load_2d(xt, &tm_t, (it - p.nkb_w) * BK, m0, full_x + s);
       }
@@ -306,75 +328,66 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      // instruction descriptor: fp32 accumulate, fp16 x fp16, both operands K-major, N = bn, M = 128
-      const uint32_t idesc = (1u << 4) | ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      // instruction descriptor: fp32 accumulate, fp16 x fp16, both operands K-major, M = 128 weight rows, N = bt tokens
+      const uint32_t idesc = (1u << 4) | ((uint32_t)(p.bt >> 3) << 17) | ((uint32_t)(BN_W >> 4) << 24);
       bool ok = true;
       for (int it = 0; it < nkb && ok; ++it) {
-        const int sx = it % p.sx, sb = it % p.sb;
+        const int sx = it % p.sx, sw = it % p.sw;
         ok = mbar_wait(full_x + sx, (it / p.sx) & 1, p.dev_status);
         if (!ok) break;
         PTRACE(it, 2);
-        ok = mbar_wait(full_w + sb, (it / p.sb) & 1, p.dev_status);
+        ok = mbar_wait(full_w + sw, (it / p.sw) & 1, p.dev_status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t adesc = make_desc(smem + (size_t)sx * (BM * 128));
-        const uint64_t bdesc = make_desc(smem + p.b_off + (size_t)sb * p.bn * 128);
+        const uint64_t adesc = make_desc(smem + p.w_off + (size_t)sw * (BN_W * 128));
+        const uint64_t bdesc = make_desc(smem + (size_t)sx * xbytes);
 #pragma unroll
         for (int k = 0; k < BK / 16; ++k)          // 32 bytes (16 fp16) further along K per step: +2 in the address field
           umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
         umma_commit(empty_x + sx);                  // both arrive when these MMAs have finished reading their operands
-        umma_commit(empty_w + sb);
+        umma_commit(empty_w + sw);
         PTRACE(it, 3);
       }
       umma_commit(&acc_full);                       // arrives when every MMA above has completed
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ dequant warps, then epilogue
-    const int dw = warp - 4;
-    bool ok = dequant_part<WF>(p.w, n0, p.bn, p.nkb_w, 0, dw, lane, smem, p, full_w, empty_w);
-    if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, p.bn, p.nkb_b, p.nkb_w, dw, lane, smem, p, full_w, empty_w);
+    const int dw = warp - 4, tile = dw & 7, par = dw >> 3;
+    bool ok = dequant_part<WF>(p.w, n0, p.nkb_w, 0, tile, par, lane, smem, p, full_w, empty_w);
+    if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, p.nkb_b, p.nkb_w, tile, par, lane, smem, p, full_w, empty_w);
     if (dw < 4) {
-      // epilogue: warp dw owns accumulator rows 32*dw .. 32*dw+31 (= its TMEM lanes)
+      // Epilogue (4 warps).  Warp dw owns accumulator rows (= weight rows n) 32*dw .. 32*dw+31, its TMEM lanes;
+      // columns are tokens.  Chunks of 32 tokens go through shared memory as [token][128 n] so that the global
+      // stores are 16-byte pieces of rows of Y.  The token ring is free by now (every MMA has completed).
       if (ok) ok = mbar_wait(&acc_full, 0, p.dev_status);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int row = m0 + dw * 32 + lane;
-      if (ok) {
-        for (int c0 = 0; c0 < p.bn; c0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(tmem_d + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          const int col = n0 + c0;
+      const int esz = p.out_dtype == EORA_Y_F32 ? 4 : 2;
+      uint8_t* tbuf = smem;                              // 32 tokens x 128 n x esz bytes (<= 16 KB)
+      const int et = threadIdx.x - 128;                  // 0..127 among the epilogue threads
+      for (int c0 = 0; c0 < p.bt && ok; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem_d + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        const int nl = dw * 32 + lane;                   // local weight row
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float f = __uint_as_float(v[j]);
+          if (p.out_dtype == EORA_Y_F32) reinterpret_cast<float*>(tbuf)[j * BN_W + nl] = f;
+          else if (p.out_dtype == EORA_Y_F16) reinterpret_cast<__half*>(tbuf)[j * BN_W + nl] = __float2half_rn(f);
+          else reinterpret_cast<__nv_bfloat16*>(tbuf)[j * BN_W + nl] = __float2bfloat16_rn(f);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        // 32 token rows of 128*esz bytes each -> 16-byte stores
+        const int per_row = BN_W * esz / 16;             // 16 or 32 pieces per token row
+        for (int i = et; i < 32 * per_row; i += 128) {
+          const int tok = i / per_row, piece = i - tok * per_row;
+          const int row = m0 + c0 + tok, col = n0 + piece * (16 / esz);
           if (row < p.m && col < p.n_valid) {
-            if (p.out_dtype == EORA_Y_F32) {
-              float* o = reinterpret_cast<float*>(p.out) + (int64_t)row * p.ld_out + col;
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                if (col + j < p.n_valid)
-                  *reinterpret_cast<float4*>(o + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                                  __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-            } else {
-              uint16_t* o = reinterpret_cast<uint16_t*>(p.out) + (int64_t)row * p.ld_out + col;
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                if (col + j < p.n_valid) {
-                  uint32_t h[4];
-#pragma unroll
-                  for (int q = 0; q < 4; ++q) {
-                    const float f0 = __uint_as_float(v[j + 2 * q]), f1 = __uint_as_float(v[j + 2 * q + 1]);
-                    if (p.out_dtype == EORA_Y_F16) {
-                      __half2 hh = __floats2half2_rn(f0, f1);
-                      h[q] = *reinterpret_cast<uint32_t*>(&hh);
-                    } else {
-                      __nv_bfloat162 bb = __floats2bfloat162_rn(f0, f1);
-                      h[q] = *reinterpret_cast<uint32_t*>(&bb);
-                    }
-                  }
-                  *reinterpret_cast<uint4*>(o + j) = make_uint4(h[0], h[1], h[2], h[3]);
-                }
-              }
-            }
+            const uint4 val = *reinterpret_cast<const uint4*>(tbuf + (size_t)tok * BN_W * esz + piece * 16);
+            *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + ((int64_t)row * p.ld_out + col) * esz) = val;
           }
         }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
       }
     }
   }
@@ -406,13 +419,13 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// fp16 [rows][cols] row-major, box = 64 columns x 128 rows, 128-byte swizzle, zero fill out of bounds
-bool make_map(CUtensorMap* tm, const void* base, int rows, int cols, int ld) {
+// fp16 [rows][cols] row-major, box = 64 columns x box_rows rows, 128-byte swizzle, zero fill out of bounds
+bool make_map(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -458,12 +471,17 @@ cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, con
 }
 
 int fill_stages(PrefillArgs& a) {      // returns the dynamic shared memory to request
-  a.sb = 3;
-  const int b_bytes = a.sb * a.bn * 128;
-  a.sx = (kSmemP - 3072 - b_bytes) / (BM * 128);
+  a.sw = 3;
+  const int w_bytes = a.sw * BN_W * 128;
+  a.sx = (kSmemP - 3072 - w_bytes) / (a.bt * 128);
   if (a.sx > kMaxXStages) a.sx = kMaxXStages;
-  a.b_off = a.sx * BM * 128;
-  return a.b_off + b_bytes + 1024;
+  a.w_off = a.sx * a.bt * 128;
+  return a.w_off + w_bytes + 1024;
+}
+
+int token_tile(int m) {                // the MMA N: a multiple of 16 up to 256
+  if (m >= 256) return 256;
+  return (m + 15) / 16 * 16;
 }
 
 }  // namespace
@@ -508,19 +526,19 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     k_bf16_to_f16<<<(int)blocks, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), ps->x16, n);
     x16 = ps->x16;
   }
+  const int bt = token_tile(m);
   CUtensorMap tm_x, tm_t;
-  if (!make_map(&tm_x, x16, m, c.d_in, c.d_in)) return cudaErrorInvalidValue;
+  if (!make_map(&tm_x, x16, m, c.d_in, c.d_in, bt)) return cudaErrorInvalidValue;
   const bool ab = c.rank > 0;
   if (ab) {
-    if (!make_map(&tm_t, h->t16, m, h->r_pad, h->r_pad)) return cudaErrorInvalidValue;
+    if (!make_map(&tm_t, h->t16, m, h->r_pad, h->r_pad, bt)) return cudaErrorInvalidValue;
     // launch 1: t = X.A  (A as the weight: rows = r_pad, fp16 output into t16)
     PrefillArgs a = {};
     a.w = h->a; a.b = WMat(); a.b.fmt = FMT_NONE;
-    a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m;
-    a.bn = (h->r_pad % 128 == 0) ? 128 : 64;
-    a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status;
+    a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt;
+    a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status; a.trace = nullptr;
     const int smem_t = fill_stages(a);
-    dim3 grid(h->r_pad / a.bn, (m + BM - 1) / BM);
+    dim3 grid((h->r_pad + BN_W - 1) / BN_W, (m + bt - 1) / bt);
     cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_x, tm_x, a);
     if (e != cudaSuccess) return e;
   } else {
@@ -529,12 +547,11 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   PrefillArgs a = {};
   a.w = h->w; a.b = h->b;
   if (!ab) a.b.fmt = FMT_NONE;
-  a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m;
-  a.bn = 256;
+  a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m; a.bt = bt;
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
   a.trace = reinterpret_cast<long long*>(h->trace);
   const int smem_y = fill_stages(a);
-  dim3 grid((c.d_out + a.bn - 1) / a.bn, (m + BM - 1) / BM);
+  dim3 grid((c.d_out + BN_W - 1) / BN_W, (m + bt - 1) / bt);
   return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, a);
 }
 
