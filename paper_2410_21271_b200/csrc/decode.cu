@@ -65,7 +65,7 @@ __device__ __forceinline__ void run_slice(const SliceView& sv, int warp, int lan
   for (int q = warp; q < sv.nq; q += kWarps) {
     const int chunk = q / sv.cq;
     if (chunk > chunk_ready) {
-      mbar_wait(sv.bars + chunk, 0, dev_status);
+      mbar_wait_warp(sv.bars + chunk, 0, dev_status, lane);
       chunk_ready = chunk;
     }
     float gacc[MT][4];

@@ -18,9 +18,8 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
-  // the last operand lets the hardware park the thread for up to ~4 us instead of spinning
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(4000u) : "memory");
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
@@ -42,6 +41,32 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* d
   atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
   return false;
 }
+// The same wait for a whole warp.  Only lane 0 polls, and it backs off between polls: a warp-wide
+// spin costs a shared-memory access per poll, and a dozen spinning warps are enough to starve the
+// bulk-copy engine and the tensor core of shared-memory bandwidth.  Once lane 0 has seen the phase
+// complete, every lane tests it once itself (which succeeds at once) so that each thread has its own
+// acquire of the data behind the barrier.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, int* dev_status, int lane) {
+  if (mbar_try_wait(bar, parity)) return true;
+  int ok = 1;
+  if (lane == 0) {
+    const unsigned long long t0 = globaltimer_ns();
+    ok = 0;
+    for (;;) {
+#pragma unroll 1
+      for (int it = 0; it < 64 && !ok; ++it) {
+        __nanosleep(40);
+        ok = mbar_try_wait(bar, parity) ? 1 : 0;
+      }
+      if (ok || globaltimer_ns() - t0 > kWaitLimitNs) break;
+    }
+    if (!ok) atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
+  }
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  if (ok) { while (!mbar_try_wait(bar, parity)) {} }
+  return ok != 0;
+}
+
 // Bounded spin on a global counter reaching `target`.
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p);
 __device__ __forceinline__ bool counter_wait(const uint32_t* cnt, uint32_t target, int* dev_status) {

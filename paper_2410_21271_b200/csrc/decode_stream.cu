@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
         sc2 = __ldg(scp + gi * 8); zz2 = __ldg(zzp + gi * 8);
       }
       for (int q = 0; q < u.nq; q += cq) {
-        if (!mbar_wait(full + s, ph, p.dev_status)) { alive = false; break; }
+        if (!mbar_wait_warp(full + s, ph, p.dev_status, lane)) { alive = false; break; }
         const int myq = q + warp;
         if (warp < cq && myq < u.nq) {
           uint32_t sc_n = 0, zz_n = 0;               // prefetch for this warp's quantum of the next chunk
@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
         if (++s == p.stages) { s = 0; ph ^= 1; }
       }
       if (!alive) break;
-      if (i >= kRed && !mbar_wait(red_free + rb, rph ^ 1, p.dev_status)) break;
+      if (i >= kRed && !mbar_wait_warp(red_free + rb, rph ^ 1, p.dev_status, lane)) break;
       float* r = red + (rb * kCW + warp) * 128;
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) r[cc * 32 + lane] = acc[cc];
@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
   for (int i = 0; i < n_mine; ++i, eit.next(p, G)) {
     const int rb = i & (kRed - 1);
     const Unit u = eit.get(p);
-    if (!mbar_wait(red_full + rb, (i / kRed) & 1, p.dev_status)) break;
+    if (!mbar_wait_warp(red_full + rb, (i / kRed) & 1, p.dev_status, lane)) break;
     float acc[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -420,7 +420,7 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
         if (!t_staged) stage_t();
         const int slot = b_used % kBRing;
         const uint8_t* bb = smem + p.off_b + (size_t)slot * p.b_bytes;
-        if (!mbar_wait(b_full + slot, (b_used / kBRing) & 1, p.dev_status)) break;
+        if (!mbar_wait_warp(b_full + slot, (b_used / kBRing) & 1, p.dev_status, lane)) break;
         run_b<ABF>(bb, reinterpret_cast<const uint32_t*>(bb + p.b_sc_off), reinterpret_cast<const uint16_t*>(bb + p.b_zz_off),
                    p.b.kc, p.qt_b, p.b.group / 64, lane, ts, trow, p.m, acc);
         __syncwarp();

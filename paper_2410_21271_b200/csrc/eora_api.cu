@@ -160,6 +160,7 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
     Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
     h->t_ws = sc.take<float>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 4);
     h->y_ws = sc.take<float>((int64_t)m_dec * c.d_out * 4);
+    h->t_gen = sc.take<float>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 4);
     h->t16 = sc.take<__half>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 2);
     h->counters = sc.take<uint32_t>(n_counters * 4);
     h->dev_status = sc.take<int>(256);

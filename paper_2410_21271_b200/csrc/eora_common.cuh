@@ -142,7 +142,8 @@ struct Handle {
   int64_t weight_bytes;
   void* scratch_mem;     // one allocation: t, split-K sums, counters, staging
   int64_t scratch_bytes;
-  float* t_ws;           // [max_m][r_pad] fp32
+  float* t_ws;           // [max_m][r_pad] fp32 sums of the fast kernels; zero between calls
+  float* t_gen;          // [max_m][r_pad] fp32, simple kernels only
   float* y_ws;           // [min(max_m,64)][d_out] fp32 split-K sums (decode)
   __half* t16;           // [max_m][r_pad] fp16 (prefill)
   uint32_t* counters;    // see decode.cu

@@ -71,9 +71,9 @@ cudaError_t launch_generic_forward(const Handle* h, const void* x, int m, void* 
   const eora_linear_config& c = h->cfg;
   bool has_ab = c.rank > 0;
   if (has_ab)
-    k_generic_t<<<grid_for((int64_t)m * h->r_pad, 128), 128, 0, st>>>(h->a, x, c.x_dtype, m, c.d_in, h->t_ws, h->r_pad);
+    k_generic_t<<<grid_for((int64_t)m * h->r_pad, 128), 128, 0, st>>>(h->a, x, c.x_dtype, m, c.d_in, h->t_gen, h->r_pad);
   k_generic_y<<<grid_for((int64_t)m * c.d_out, 128), 128, 0, st>>>(h->w, h->b, has_ab, x, c.x_dtype, m, c.d_in, c.d_out,
-                                                                  h->t_ws, h->r_pad, y, c.y_dtype);
+                                                                  h->t_gen, h->r_pad, y, c.y_dtype);
   return cudaGetLastError();
 }
 

@@ -27,8 +27,8 @@ namespace eora {
 using namespace dec;
 namespace {
 
-constexpr int BN_W = 128, BK = 64;               // weight rows per CTA tile (the MMA M), k-block
-constexpr int kDqWarps = 16;                    // dequant warps (warps 4..19): 8 row tiles x 2 k-block parities
+constexpr int BN_W = 128, BK = 64;               // weight rows per MMA (its M), k-block; a CTA owns up to two such halves
+constexpr int kDqWarps = 16;                    // dequant warps (warps 4..19): one 16-row tile of the 256 weight rows each
 constexpr int kThreadsP = (4 + kDqWarps) * 32;  // warp 0: TMA, warp 1: MMA, warp 2: TMEM alloc, warp 3: idle
 constexpr int kMaxXStages = 8;                  // ring of token tiles (TMA latency is long: deep)
 constexpr int kMaxWStages = 4;                  // ring of dequantised weight tiles (produced on chip: shallow)
@@ -45,6 +45,7 @@ struct PrefillArgs {
   int bt;            // token tile (the MMA N): multiple of 16, at most 256
   int nkb_w, nkb_b;  // k-blocks of each part
   int sx, sw;        // stages of the token ring / of the weight ring
+  int split_k;       // gridDim.z: each z handles a slice of the k-blocks and adds into a fp32 `out` (out_dtype 3)
   int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
   int* dev_status;
   long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (dequant start, W ready, X ready, MMA issued)
@@ -222,11 +223,11 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
   }
 }
 
-// One part (W or the K-extension B) of a dequant warp's work.  The warp owns row tile `tile` (0..7) of
-// the CTA's 128 weight rows and the k-blocks of `mat` with kb = par (mod 2); k-block kb lands in pipeline
-// iteration kb0 + kb.  Packed weights, scales and zero-points are loaded PF of its k-blocks ahead.
+// One part (W or the K-extension B) of a dequant warp's work.  The warp owns row tile `tile` (0..15) of
+// the CTA's 256 weight rows; k-blocks [kb_lo, kb_hi) of `mat` land in pipeline iterations it0, it0 + 1, ...
+// Packed weights, scales and zero-points are loaded PF k-blocks ahead.
 template <int FMT>
-__device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int nkb, int kb0, int tile, int par, int lane,
+__device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo, int kb_hi, int it0, int tile, int lane,
                                              uint8_t* smem, const PrefillArgs& p, uint64_t* full_w, uint64_t* empty_w) {
   if constexpr (FMT == FMT_NONE) {
     return true;
@@ -238,12 +239,10 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int nkb, i
     const int g = lane >> 2;
     const int tb = tile_bytes(FMT);
     const int gt = mat.group / 64;
-    // the warp's k-blocks are kb = first, first + 2, ... where first has the parity that makes (kb0 + kb) % 2 == par
-    const int first = (par ^ (kb0 & 1)) & 1;
     Packed<FMT> pk[PF];
     uint32_t scq[PF], zzq[PF];
     auto issue = [&](int kb, int slot) {
-      if (!active || kb >= nkb) return;
+      if (!active || kb >= kb_hi) return;
       load_packed<FMT>(pk[slot], mat.q + ((int64_t)rt * mat.kc + kb) * tb, lane);
       if constexpr (quant) {
         const int64_t si = ((int64_t)rt * mat.ng + kb / gt) * 8 + g;
@@ -252,16 +251,15 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int nkb, i
       }
     };
 #pragma unroll
-    for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(first + 2 * j, j); }
-    for (int kbb = first; kbb < nkb; kbb += 2 * PF) {
+    for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(kb_lo + j, j); }
+    for (int kbb = kb_lo; kbb < kb_hi; kbb += PF) {
 #pragma unroll
       for (int j = 0; j < PF; ++j) {
-        const int kb = kbb + 2 * j;
-        if (kb < nkb) {
-          const int it = kb0 + kb, s = it % p.sw;
-          if (it >= p.sw && !mbar_wait(empty_w + s, ((it / p.sw) - 1) & 1, p.dev_status)) return false;
-          if (tile == 0 && lane == 0) PTRACE(it, 0);
-          uint8_t* wt = smem + p.w_off + (size_t)s * (BN_W * 128);
+        const int kb = kbb + j;
+        if (kb < kb_hi) {
+          const int it = it0 + (kb - kb_lo), s = it % p.sw;
+          if (it >= p.sw && !mbar_wait_warp(empty_w + s, ((it / p.sw) - 1) & 1, p.dev_status, lane)) return false;
+          uint8_t* wt = smem + p.w_off + (size_t)s * (2 * BN_W * 128);
           if (active) {
             dequant_store<FMT>(pk[j], scq[j], zzq[j], wt, tile * 16, lane);
           } else {                                        // rows past the matrix: keep the operand finite
@@ -275,7 +273,7 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int nkb, i
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
           __syncwarp();
           if (lane == 0) { mbar_arrive(full_w + s); if (tile == 0) PTRACE(it, 1); }
-          issue(kb + 2 * PF, j);
+          issue(kb + PF, j);
         }
       }
     }
@@ -293,19 +291,23 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * BN_W, m0 = blockIdx.y * p.bt;
-  const int nkb = p.nkb_w + p.nkb_b;
+  const int n0 = blockIdx.x * (2 * BN_W), m0 = blockIdx.y * p.bt;
+  const int nh = (p.n_valid - n0 > BN_W) ? 2 : 1;          // 128-row halves of this CTA that hold real rows
+  // this CTA's slice of the k-blocks (split-K over gridDim.z; the K-extension only exists without split)
+  const int kw_lo = (int)((int64_t)p.nkb_w * blockIdx.z / p.split_k), kw_hi = (int)((int64_t)p.nkb_w * (blockIdx.z + 1) / p.split_k);
+  const int nkw = kw_hi - kw_lo;
+  const int nkb = nkw + p.nkb_b;
   const uint32_t xbytes = (uint32_t)p.bt * 128;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.sx; ++i) { mbar_init(full_x + i, 1); mbar_init(empty_x + i, 1); }
-    for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8); mbar_init(empty_w + i, 1); }
+    for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8 * nh); mbar_init(empty_w + i, 1); }
     mbar_init(&acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 2) {   // tensor memory: 256 fp32 columns x 128 lanes for the accumulator
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(256u) : "memory");
+  if (warp == 2) {   // tensor memory: two accumulators of 128 lanes x 256 fp32 columns
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -319,10 +321,11 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       for (int it = 0; it < nkb; ++it) {
         const int s = it % p.sx;
         if (it >= p.sx && !mbar_wait(empty_x + s, ((it / p.sx) - 1) & 1, p.dev_status)) break;
+        PTRACE(it, 0);
         mbar_expect_tx(full_x + s, xbytes);
         uint8_t* xt = smem + (size_t)s * xbytes;
-        if (it < p.nkb_w) tma_load_2d(xt, &tm_x, it * BK, m0, full_x + s);
-        else tma_load_2d(xt, &tm_t, (it - p.nkb_w) * BK, m0, full_x + s);
+        if (it < nkw) tma_load_2d(xt, &tm_x, (kw_lo + it) * BK, m0, full_x + s);
+        else tma_load_2d(xt, &tm_t, (it - nkw) * BK, m0, full_x + s);
       }
     }
   } else if (warp == 1) {
@@ -339,11 +342,13 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
         ok = mbar_wait(full_w + sw, (it / p.sw) & 1, p.dev_status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t adesc = make_desc(smem + p.w_off + (size_t)sw * (BN_W * 128));
         const uint64_t bdesc = make_desc(smem + (size_t)sx * xbytes);
+        for (int hh = 0; hh < nh; ++hh) {
+          const uint64_t adesc = make_desc(smem + p.w_off + (size_t)sw * (2 * BN_W * 128) + hh * (BN_W * 128));
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k)          // 32 bytes (16 fp16) further along K per step: +2 in the address field
-          umma_f16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK / 16; ++k)        // 32 bytes (16 fp16) further along K per step: +2 in the address field
+            umma_f16(tmem_d + hh * 256, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+        }
         umma_commit(empty_x + sx);                  // both arrive when these MMAs have finished reading their operands
         umma_commit(empty_w + sw);
         PTRACE(it, 3);
@@ -352,48 +357,80 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ dequant warps, then epilogue
-    const int dw = warp - 4, tile = dw & 7, par = dw >> 3;
-    bool ok = dequant_part<WF>(p.w, n0, p.nkb_w, 0, tile, par, lane, smem, p, full_w, empty_w);
-    if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, p.nkb_b, p.nkb_w, tile, par, lane, smem, p, full_w, empty_w);
+    const int dw = warp - 4;
+    bool ok = true;
+    if (dw < 8 * nh) {
+      ok = dequant_part<WF>(p.w, n0, kw_lo, kw_hi, 0, dw, lane, smem, p, full_w, empty_w);
+      if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, 0, p.nkb_b, nkw, dw, lane, smem, p, full_w, empty_w);
+    }
     if (dw < 4) {
-      // Epilogue (4 warps).  Warp dw owns accumulator rows (= weight rows n) 32*dw .. 32*dw+31, its TMEM lanes;
-      // columns are tokens.  Chunks of 32 tokens go through shared memory as [token][128 n] so that the global
-      // stores are 16-byte pieces of rows of Y.  The token ring is free by now (every MMA has completed).
-      if (ok) ok = mbar_wait(&acc_full, 0, p.dev_status);
+      // Epilogue (4 warps).  Warp dw owns accumulator rows (= weight rows n) 32*dw .. 32*dw+31 of each half,
+      // its TMEM lanes; columns are tokens.
+      if (ok) ok = mbar_wait_warp(&acc_full, 0, p.dev_status, lane);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int esz = p.out_dtype == EORA_Y_F32 ? 4 : 2;
-      uint8_t* tbuf = smem;                              // 32 tokens x 128 n x esz bytes (<= 16 KB)
-      const int et = threadIdx.x - 128;                  // 0..127 among the epilogue threads
-      for (int c0 = 0; c0 < p.bt && ok; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(tmem_d + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        const int nl = dw * 32 + lane;                   // local weight row
+      const int nl = dw * 32 + lane;                     // local weight row inside the half
+      if (p.out_dtype == 3) {
+        // split-K partial: add fp32 into out[token][n]; lanes hold consecutive n, so each red is a 128-byte row piece
+        for (int hh = 0; hh < nh && ok; ++hh) {
+          const int col = n0 + hh * BN_W + nl;
+          for (int c0 = 0; c0 < p.bt; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_d + hh * 256 + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (col < p.n_valid) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float f = __uint_as_float(v[j]);
-          if (p.out_dtype == EORA_Y_F32) reinterpret_cast<float*>(tbuf)[j * BN_W + nl] = f;
-          else if (p.out_dtype == EORA_Y_F16) reinterpret_cast<__half*>(tbuf)[j * BN_W + nl] = __float2half_rn(f);
-          else reinterpret_cast<__nv_bfloat16*>(tbuf)[j * BN_W + nl] = __float2bfloat16_rn(f);
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        // 32 token rows of 128*esz bytes each -> 16-byte stores
-        const int per_row = BN_W * esz / 16;             // 16 or 32 pieces per token row
-        for (int i = et; i < 32 * per_row; i += 128) {
-          const int tok = i / per_row, piece = i - tok * per_row;
-          const int row = m0 + c0 + tok, col = n0 + piece * (16 / esz);
-          if (row < p.m && col < p.n_valid) {
-            const uint4 val = *reinterpret_cast<const uint4*>(tbuf + (size_t)tok * BN_W * esz + piece * 16);
-            *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + ((int64_t)row * p.ld_out + col) * esz) = val;
+              for (int j = 0; j < 32; ++j) {
+                const int row = m0 + c0 + j;
+                if (row < p.m) red_add(reinterpret_cast<float*>(p.out) + (int64_t)row * p.ld_out + col, __uint_as_float(v[j]));
+              }
+            }
           }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+      } else {
+        // Chunks of 32 tokens go through shared memory as [token][128 n] so that the global stores are 16-byte
+        // pieces of rows of Y.  The token ring is free by now (every MMA has completed).
+        const int esz = p.out_dtype == EORA_Y_F32 ? 4 : 2;
+        uint8_t* tbuf = smem;                            // 32 tokens x 128 n x esz bytes (<= 16 KB)
+        const int et = threadIdx.x - 128;                // 0..127 among the epilogue threads
+        for (int hh = 0; hh < nh && ok; ++hh) {
+          for (int c0 = 0; c0 < p.bt; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem_d + hh * 256 + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float f = __uint_as_float(v[j]);
+              if (p.out_dtype == EORA_Y_F32) reinterpret_cast<float*>(tbuf)[j * BN_W + nl] = f;
+              else if (p.out_dtype == EORA_Y_F16) reinterpret_cast<__half*>(tbuf)[j * BN_W + nl] = __float2half_rn(f);
+              else reinterpret_cast<__nv_bfloat16*>(tbuf)[j * BN_W + nl] = __float2bfloat16_rn(f);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const int per_row = BN_W * esz / 16;         // 16 or 32 pieces per token row
+            for (int i = et; i < 32 * per_row; i += 128) {
+              const int tok = i / per_row, piece = i - tok * per_row;
+              const int row = m0 + c0 + tok, col = n0 + hh * BN_W + piece * (16 / esz);
+              if (row < p.m && col < p.n_valid) {
+                const uint4 val = *reinterpret_cast<const uint4*>(tbuf + (size_t)tok * BN_W * esz + piece * 16);
+                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + ((int64_t)row * p.ld_out + col) * esz) = val;
+              }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+          }
+        }
       }
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(256u) : "memory");
+  if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(512u) : "memory");
+}
+
+// t (fp32 split-K sums) -> fp16 operand of the K-extension; the sums are returned to zero for the next call
+__global__ void k_t32_to_f16(float* t32, __half* t16, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    t16[i] = __float2half_rn(t32[i]);
+    t32[i] = 0.f;
+  }
 }
 
 __global__ void k_bf16_to_f16(const __nv_bfloat16* in, __half* out, int64_t n) {
@@ -472,8 +509,8 @@ cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, con
 
 int fill_stages(PrefillArgs& a) {      // returns the dynamic shared memory to request
   a.sw = 3;
-  const int w_bytes = a.sw * BN_W * 128;
-  a.sx = (kSmemP - 3072 - w_bytes) / (a.bt * 128);
+  const int w_bytes = a.sw * 2 * BN_W * 128;
+  a.sx = (kSmemP - 1024 - w_bytes) / (a.bt * 128);
   if (a.sx > kMaxXStages) a.sx = kMaxXStages;
   a.w_off = a.sx * a.bt * 128;
   return a.w_off + w_bytes + 1024;
@@ -493,7 +530,7 @@ bool prefill_supported(const Handle* h, int m) {
 }
 
 int prefill_launch_count(const Handle* h, int) {
-  return (h->cfg.rank > 0 ? 2 : 1) + (h->cfg.x_dtype == EORA_X_BF16 ? 1 : 0);
+  return (h->cfg.rank > 0 ? 3 : 1) + (h->cfg.x_dtype == EORA_X_BF16 ? 1 : 0);
 }
 
 cudaError_t prefill_init(Handle* h) {
@@ -532,15 +569,23 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   const bool ab = c.rank > 0;
   if (ab) {
     if (!make_map(&tm_t, h->t16, m, h->r_pad, h->r_pad, bt)) return cudaErrorInvalidValue;
-    // launch 1: t = X.A  (A as the weight: rows = r_pad, fp16 output into t16)
+    // launch 1: t = X.A with A as the weight (rows = r_pad), split over K so that the small product fills the
+    // GPU; partial sums are added into the fp32 buffer t_ws (zero between calls); launch 2 rounds them to fp16.
     PrefillArgs a = {};
     a.w = h->a; a.b = WMat(); a.b.fmt = FMT_NONE;
-    a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt;
+    a.out = h->t_ws; a.out_dtype = 3; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt;
     a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status; a.trace = nullptr;
     const int smem_t = fill_stages(a);
-    dim3 grid((h->r_pad + BN_W - 1) / BN_W, (m + bt - 1) / bt);
+    const int tiles = ((h->r_pad + 2 * BN_W - 1) / (2 * BN_W)) * ((m + bt - 1) / bt);
+    int split = h->sm_count / tiles;
+    if (split > a.nkb_w / 2) split = a.nkb_w / 2;
+    if (split < 1) split = 1;
+    a.split_k = split;
+    dim3 grid((h->r_pad + 2 * BN_W - 1) / (2 * BN_W), (m + bt - 1) / bt, split);
     cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_x, tm_x, a);
     if (e != cudaSuccess) return e;
+    const int64_t nt = (int64_t)m * h->r_pad;
+    k_t32_to_f16<<<(int)((nt + 255) / 256 > 1184 ? 1184 : (nt + 255) / 256), 256, 0, st>>>(h->t_ws, h->t16, nt);
   } else {
     tm_t = tm_x;
   }
@@ -550,8 +595,9 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m; a.bt = bt;
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
   a.trace = reinterpret_cast<long long*>(h->trace);
+  a.split_k = 1;
   const int smem_y = fill_stages(a);
-  dim3 grid((c.d_out + BN_W - 1) / BN_W, (m + bt - 1) / bt);
+  dim3 grid((c.d_out + 2 * BN_W - 1) / (2 * BN_W), (m + bt - 1) / bt, 1);
   return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, a);
 }
 
