@@ -6,8 +6,8 @@
 //
 // A CTA has 10 warps and owns the units  blockIdx.x, blockIdx.x + gridDim.x, ...  (a unit is a
 // 16-row tile x reduction slice of A or of the backbone; A units come first).
-//   producer warp (1 lane): walks the CTA's units chunk by chunk (a chunk = one quantum per compute
-//       warp, at most 8 KB) and bulk-copies the packed tiles into a ring of shared-memory slots
+//   producer warp (1 lane): walks the CTA's units chunk by chunk (a chunk = up to two quanta per compute
+//       warp, at most 16 KB) and bulk-copies the packed tiles into a ring of shared-memory slots
 //       (cp.async.bulk + mbarrier, no multicast).  Weights never change, so it starts before the
 //       dependency wait of programmatic dependent launch and keeps the whole ring in flight.
 //   8 compute warps: per chunk, wait for the slot, dequantise their quantum in registers to the
@@ -30,7 +30,7 @@ constexpr int kEpiWarp = kCW, kProdWarp = kCW + 1;
 constexpr int kThreadsS = (kCW + 2) * 32;
 constexpr int kXPad = 32;
 constexpr int kMaxStages = 12;
-constexpr int kSlotBytes = 8 * 1024;           // one ring slot = one chunk
+constexpr int kSlotBytes = 16 * 1024;          // one ring slot = one chunk (up to two quanta per compute warp)
 constexpr int kRed = 4;                        // reduction-slot ring depth
 constexpr int kBRing = 2;
 constexpr int kSmemPerCta = 110 * 1024;        // two CTAs per SM
@@ -100,41 +100,106 @@ __device__ __forceinline__ int group_of(int quantum, int shift, int qpg) {
 
 #define STRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
 
-// One quantum (QT tiles sharing one scale / zero-point) for one compute warp.  blob: its tiles in
-// shared memory; xl: this lane's activations for the quantum's first reduction element.
-template <int FMT, int QT>
-__device__ __forceinline__ void run_quantum(const uint8_t* blob, uint32_t sc2, uint32_t zz2, int lane, const __half* xl,
-                                            bool have_x, float (&acc)[4]) {
+// NQ quanta (QT tiles each, sharing one scale / zero-point per quantum) for one compute warp, in one
+// straight-line block so that the independent dequant / MMA chains of the quanta interleave.
+// Quantum j: tiles at blob + j * blob_stride, activations at xl + j * x_stride (halves).
+template <int FMT, int QT, int NQ>
+__device__ __forceinline__ void run_quanta(const uint8_t* blob, int blob_stride, const uint32_t (&sc2)[2], const uint32_t (&zz2)[2],
+                                           int lane, const __half* xl, int x_stride, bool have_x, float (&acc)[4]) {
   constexpr int TB = FMT == FMT_Q4 ? 512 : FMT == FMT_Q3 ? 384 : FMT == FMT_Q8 ? 1024 : 2048;
-  float gacc[QT][4];
-  ZC zc;
-  if constexpr (is_quant<FMT>()) make_zc<FMT>(zc, zz2);
+  float gacc[NQ][QT][4];
 #pragma unroll
-  for (int tt = 0; tt < QT; ++tt) {
-    gacc[tt][0] = gacc[tt][1] = gacc[tt][2] = gacc[tt][3] = 0.f;
-    uint32_t a[4][4];
-    tile_frags<FMT>(blob + tt * TB, lane, zc, a);
-    uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
-    if (have_x) {
-      x0 = *reinterpret_cast<const uint4*>(xl + tt * 64);
-      x1 = *reinterpret_cast<const uint4*>(xl + tt * 64 + 32);
+  for (int j = 0; j < NQ; ++j) {
+    ZC zc;
+    if constexpr (is_quant<FMT>()) make_zc<FMT>(zc, zz2[j]);
+#pragma unroll
+    for (int tt = 0; tt < QT; ++tt) {
+      gacc[j][tt][0] = gacc[j][tt][1] = gacc[j][tt][2] = gacc[j][tt][3] = 0.f;
+      uint32_t a[4][4];
+      tile_frags<FMT>(blob + j * blob_stride + tt * TB, lane, zc, a);
+      uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
+      if (have_x) {
+        x0 = *reinterpret_cast<const uint4*>(xl + j * x_stride + tt * 64);
+        x1 = *reinterpret_cast<const uint4*>(xl + j * x_stride + tt * 64 + 32);
+      }
+      mma16816(gacc[j][tt], a[0], x0.x, x0.y);
+      mma16816(gacc[j][tt], a[1], x0.z, x0.w);
+      mma16816(gacc[j][tt], a[2], x1.x, x1.y);
+      mma16816(gacc[j][tt], a[3], x1.z, x1.w);
     }
-    mma16816(gacc[tt], a[0], x0.x, x0.y);
-    mma16816(gacc[tt], a[1], x0.z, x0.w);
-    mma16816(gacc[tt], a[2], x1.x, x1.y);
-    mma16816(gacc[tt], a[3], x1.z, x1.w);
-  }
-  float sa = 1.f, sb = 1.f;
-  if constexpr (is_quant<FMT>()) {
-    sa = __half2float(__ushort_as_half((unsigned short)(sc2 & 0xffffu)));
-    sb = __half2float(__ushort_as_half((unsigned short)(sc2 >> 16)));
   }
 #pragma unroll
-  for (int tt = 0; tt < QT; ++tt) {
-    acc[0] = fmaf(sa, gacc[tt][0], acc[0]);
-    acc[1] = fmaf(sa, gacc[tt][1], acc[1]);
-    acc[2] = fmaf(sb, gacc[tt][2], acc[2]);
-    acc[3] = fmaf(sb, gacc[tt][3], acc[3]);
+  for (int j = 0; j < NQ; ++j) {
+    float sa = 1.f, sb = 1.f;
+    if constexpr (is_quant<FMT>()) {
+      sa = __half2float(__ushort_as_half((unsigned short)(sc2[j] & 0xffffu)));
+      sb = __half2float(__ushort_as_half((unsigned short)(sc2[j] >> 16)));
+    }
+#pragma unroll
+    for (int tt = 0; tt < QT; ++tt) {
+      acc[0] = fmaf(sa, gacc[j][tt][0], acc[0]);
+      acc[1] = fmaf(sa, gacc[j][tt][1], acc[1]);
+      acc[2] = fmaf(sb, gacc[j][tt][2], acc[2]);
+      acc[3] = fmaf(sb, gacc[j][tt][3], acc[3]);
+    }
+  }
+}
+
+template <int FMT>
+__device__ __forceinline__ void run_chunk(int qt, int nq_here, const uint8_t* blob, int blob_stride, const uint32_t (&sc2)[2],
+                                          const uint32_t (&zz2)[2], int lane, const __half* xl, int x_stride, bool have_x,
+                                          float (&acc)[4]) {
+  if constexpr (FMT != FMT_NONE) {
+    if (qt == 2) {
+      if (nq_here == 2) run_quanta<FMT, 2, 2>(blob, blob_stride, sc2, zz2, lane, xl, x_stride, have_x, acc);
+      else run_quanta<FMT, 2, 1>(blob, blob_stride, sc2, zz2, lane, xl, x_stride, have_x, acc);
+    } else {
+      if (nq_here == 2) run_quanta<FMT, 1, 2>(blob, blob_stride, sc2, zz2, lane, xl, x_stride, have_x, acc);
+      else run_quanta<FMT, 1, 1>(blob, blob_stride, sc2, zz2, lane, xl, x_stride, have_x, acc);
+    }
+  }
+}
+
+// What a compute warp needs to know about the matrix of a unit.  The two possible matrices (A and the
+// backbone) are turned into registers once per kernel: picking between two kernel-parameter structs at run
+// time costs a chain of dependent constant-bank loads at every unit boundary.
+struct MatInfo {
+  const uint32_t* scp;      // scales of the unit's row tile (+ g), set per unit
+  const uint16_t* zzp;
+  const uint32_t* sc_base;  // matrix base (+ g)
+  const uint16_t* zz_base;
+  int ng8;                  // words per row tile in sc / zz
+  int qt, cq, tb, qsh, qpg;
+  bool quant;
+};
+__device__ __forceinline__ MatInfo mat_base(const WMat& mat, int qt, int cq, int qsh, int g) {
+  MatInfo m;
+  m.qt = qt; m.cq = cq; m.qsh = qsh;
+  m.tb = tile_bytes(mat.fmt);
+  m.qpg = mat.fmt == FMT_NONE ? 1 : mat.group / (64 * qt);
+  m.quant = mat.fmt != FMT_F16;
+  m.sc_base = mat.sc + g; m.zz_base = mat.zz + g;
+  m.ng8 = mat.ng * 8;
+  m.scp = m.sc_base; m.zzp = m.zz_base;
+  return m;
+}
+__device__ __forceinline__ MatInfo mat_info(const MatInfo& ma, const MatInfo& mw, const Unit& u) {
+  MatInfo m = u.is_a ? ma : mw;
+  m.scp = m.sc_base + (int64_t)u.tile * m.ng8;
+  m.zzp = m.zz_base + (int64_t)u.tile * m.ng8;
+  return m;
+}
+// scales / zero-points of this warp's (up to two) quanta of the chunk that starts at quantum q of unit u
+__device__ __forceinline__ void load_sz(const MatInfo& m, const Unit& u, int q, int warp, uint32_t (&sc)[2], uint32_t (&zz)[2]) {
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const int lq = j * kCW + warp, qq = q + lq;
+    sc[j] = 0; zz[j] = 0;
+    if (m.quant && lq < m.cq && qq < u.nq) {
+      const int gi = group_of(u.q0 + qq, m.qsh, m.qpg);
+      sc[j] = __ldg(m.scp + gi * 8);
+      zz[j] = __ldg(m.zzp + gi * 8);
+    }
   }
 }
 
@@ -265,55 +330,51 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
     const int g = lane >> 2;
     const bool have_x = g < p.m;
     const __half* xlane = xs + g * xrow + 8 * (lane & 3);
+    int cstamp = 0;                                 // per-chunk trace stamps of CTA 0 (see eora_linear_set_trace)
     int s = 0, ph = 0;                              // ring slot and phase, in step with the producer
     int rb = 0, rph = 0;                            // reduction slot and phase
     bool alive = true;
     UnitIter it;
     it.init(p, (int)blockIdx.x);
-    for (int i = 0; i < n_mine && alive; ++i, it.next(p, G)) {
-      const Unit u = it.get(p);
-      const WMat& mat = u.is_a ? p.a : p.w;
-      const int qt = u.is_a ? p.qt_a : p.qt_w, cq = u.is_a ? p.cq_a : p.cq_w;
-      const int tb = tile_bytes(mat.fmt);
-      const int qsh = u.is_a ? p.qpg_shift_a : p.qpg_shift_w;
-      const int qpg = mat.group / (64 * qt);
-      const bool quant = mat.fmt != FMT_F16;
-      const uint32_t* scp = mat.sc + (int64_t)u.tile * mat.ng * 8 + g;
-      const uint16_t* zzp = mat.zz + (int64_t)u.tile * mat.ng * 8 + g;
+    const MatInfo base_a = mat_base(p.a, p.qt_a, p.cq_a, p.qpg_shift_a, g);
+    const MatInfo base_w = mat_base(p.w, p.qt_w, p.cq_w, p.qpg_shift_w, g);
+    Unit u = it.get(p);
+    MatInfo mi = mat_info(base_a, base_w, u);
+    uint32_t sc2[2], zz2[2];
+    load_sz(mi, u, 0, warp, sc2, zz2);            // weights are immutable: plain cached loads, always one chunk ahead
+    for (int i = 0; i < n_mine && alive; ++i) {
+      UnitIter itn = it;
+      itn.next(p, G);
+      const bool have_next = i + 1 < n_mine;
+      Unit un = u;
+      MatInfo mn = mi;
+      if (have_next) { un = itn.get(p); mn = mat_info(base_a, base_w, un); }
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
-      // scale / zero-point of this warp's first quantum (weights are immutable: plain cached loads)
-      uint32_t sc2 = 0, zz2 = 0;
-      if (quant && warp < cq && warp < u.nq) {
-        const int gi = group_of(u.q0 + warp, qsh, qpg);
-        sc2 = __ldg(scp + gi * 8); zz2 = __ldg(zzp + gi * 8);
-      }
-      for (int q = 0; q < u.nq; q += cq) {
+      for (int q = 0; q < u.nq; q += mi.cq) {
+        if (threadIdx.x == 0 && p.trace && blockIdx.x == 0 && cstamp < 500) p.trace[(size_t)gridDim.x * 16 + cstamp * 4 + 0] = clock64();
         if (!mbar_wait_warp(full + s, ph, p.dev_status, lane)) { alive = false; break; }
-        const int myq = q + warp;
-        if (warp < cq && myq < u.nq) {
-          uint32_t sc_n = 0, zz_n = 0;               // prefetch for this warp's quantum of the next chunk
-          if (quant && myq + cq < u.nq) {
-            const int gi = group_of(u.q0 + myq + cq, qsh, qpg);
-            sc_n = __ldg(scp + gi * 8); zz_n = __ldg(zzp + gi * 8);
-          }
-          const uint8_t* blob = smem + (size_t)s * kSlotBytes + warp * qt * tb;
-          const __half* xl = xlane + (u.q0 + myq) * qt * 64;
-          if (u.is_a) {
-            if constexpr (ABF != FMT_NONE) {
-              if (qt == 2) run_quantum<ABF, 2>(blob, sc2, zz2, lane, xl, have_x, acc);
-              else run_quantum<ABF, 1>(blob, sc2, zz2, lane, xl, have_x, acc);
-            }
-          } else {
-            if (qt == 2) run_quantum<WF, 2>(blob, sc2, zz2, lane, xl, have_x, acc);
-            else run_quantum<WF, 1>(blob, sc2, zz2, lane, xl, have_x, acc);
-          }
-          sc2 = sc_n; zz2 = zz_n;
+        if (threadIdx.x == 0 && p.trace && blockIdx.x == 0 && cstamp < 500) p.trace[(size_t)gridDim.x * 16 + cstamp * 4 + 1] = clock64();
+        uint32_t sc_n[2] = {0, 0}, zz_n[2] = {0, 0};
+        if (q + mi.cq < u.nq) load_sz(mi, u, q + mi.cq, warp, sc_n, zz_n);
+        else if (have_next) load_sz(mn, un, 0, warp, sc_n, zz_n);
+        // this warp's quanta of the chunk: local indices warp and warp + 8
+        int nq_here = 0;
+        if (warp < mi.cq && q + warp < u.nq) nq_here = (warp + kCW < mi.cq && q + warp + kCW < u.nq) ? 2 : 1;
+        if (nq_here) {
+          const int qbytes = mi.qt * mi.tb;
+          const uint8_t* blob = smem + (size_t)s * kSlotBytes + warp * qbytes;
+          const __half* xl = xlane + (u.q0 + q + warp) * mi.qt * 64;
+          if (u.is_a) run_chunk<ABF>(mi.qt, nq_here, blob, kCW * qbytes, sc2, zz2, lane, xl, kCW * mi.qt * 64, have_x, acc);
+          else run_chunk<WF>(mi.qt, nq_here, blob, kCW * qbytes, sc2, zz2, lane, xl, kCW * mi.qt * 64, have_x, acc);
         }
+        sc2[0] = sc_n[0]; sc2[1] = sc_n[1]; zz2[0] = zz_n[0]; zz2[1] = zz_n[1];
+        if (threadIdx.x == 0 && p.trace && blockIdx.x == 0 && cstamp < 500) { p.trace[(size_t)gridDim.x * 16 + cstamp * 4 + 2] = clock64(); ++cstamp; }
         __syncwarp();
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(empty + s)) : "memory");
         if (++s == p.stages) { s = 0; ph ^= 1; }
       }
       if (!alive) break;
+      if (threadIdx.x == 0 && p.trace && blockIdx.x == 0 && cstamp > 0 && cstamp <= 500) p.trace[(size_t)gridDim.x * 16 + (cstamp - 1) * 4 + 3] = clock64();
       if (i >= kRed && !mbar_wait_warp(red_free + rb, rph ^ 1, p.dev_status, lane)) break;
       float* r = red + (rb * kCW + warp) * 128;
 #pragma unroll
@@ -321,6 +382,7 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(red_full + rb)) : "memory");
       if (++rb == kRed) { rb = 0; rph ^= 1; }
+      it = itn; u = un; mi = mn;
     }
     if (threadIdx.x == 0) STRACE(4);
     return;
@@ -385,6 +447,25 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
     if (have_ab && lane == 0) issue_b();
   }
   const int g = lane >> 2, t4 = lane & 3;
+  bool pend = false;            // a split-K ticket whose count has not been looked at yet
+  uint32_t pend_cnt = 0;
+  int pend_tile = 0, pend_split = 0;
+  auto settle = [&]() {         // the last slice to arrive converts the sums of its row tile and clears them
+    if (!pend) return;
+    pend = false;
+    const uint32_t last = __shfl_sync(0xffffffffu, (pend_cnt == (uint32_t)pend_split - 1) ? 1u : 0u, 0);
+    if (!last) return;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int tok = 2 * t4 + (c & 1), row = pend_tile * 16 + g + 8 * (c >> 1);
+      if (tok < p.m) {
+        float* src = p.y_ws + (int64_t)tok * p.d_out + row;
+        store_y(p.y, p.y_dtype, (int64_t)tok * p.d_out + row, ld_cg(src));
+        *src = 0.f;
+      }
+    }
+    if (lane == 0) p.counters[CNT_TILE0 + pend_tile] = 0;
+  };
   UnitIter eit;
   eit.init(p, (int)blockIdx.x);
   for (int i = 0; i < n_mine; ++i, eit.next(p, G)) {
@@ -410,9 +491,8 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
         const int tok = tok0 + (c & 1), row = row0 + 8 * (c >> 1);
         if (tok < p.m) red_add(p.t_ws + (int64_t)tok * p.r_pad + row, acc[c]);
       }
-      __threadfence();
-      __syncwarp();
-      if (lane == 0) atomicAdd(p.counters + CNT_T_DONE, 1u);
+      __syncwarp();      // every lane's adds happen-before lane 0's release
+      if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.counters + CNT_T_DONE) : "memory");
       continue;
     }
     if constexpr (ABF != FMT_NONE) {
@@ -441,25 +521,15 @@ __global__ void __launch_bounds__(kThreadsS, 2) k_decode_stream(const StreamArgs
       const int tok = tok0 + (c & 1), row = row0 + 8 * (c >> 1);
       if (tok < p.m) red_add(p.y_ws + (int64_t)tok * p.d_out + row, acc[c]);
     }
-    __threadfence();
-    __syncwarp();
-    uint32_t last = 0;
-    if (lane == 0) last = (atomicAdd(p.counters + CNT_TILE0 + u.tile, 1u) == (uint32_t)u.split - 1) ? 1u : 0u;
-    last = __shfl_sync(0xffffffffu, last, 0);
-    if (last) {
-      __threadfence();
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int tok = tok0 + (c & 1), row = row0 + 8 * (c >> 1);
-        if (tok < p.m) {
-          float* src = p.y_ws + (int64_t)tok * p.d_out + row;
-          store_y(p.y, p.y_dtype, (int64_t)tok * p.d_out + row, ld_cg(src));
-          *src = 0.f;
-        }
-      }
-      if (lane == 0) p.counters[CNT_TILE0 + u.tile] = 0;
-    }
+    // Split-K ticket.  The counter round trip is long, so its result is only looked at after the next
+    // unit has been summed: first settle the previous ticket, then take this one.
+    settle();
+    __syncwarp();        // every lane's adds happen-before lane 0's release
+    if (lane == 0)
+      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(pend_cnt) : "l"(p.counters + CNT_TILE0 + u.tile) : "memory");
+    pend = true; pend_tile = u.tile; pend_split = u.split;
   }
+  settle();
   // a CTA without a B-owning unit still takes part in the hand-back of t_ws
   if constexpr (ABF != FMT_NONE) {
     if (have_ab && !t_staged) stage_t();
@@ -488,7 +558,7 @@ SPlan make_splan(const Handle* h, int m) {
   a.qt_b = ab ? quantum_tiles(h->b) : 1;
   auto chunk_quanta = [](const WMat& mat, int qt) {
     int cq = kSlotBytes / (qt * tile_bytes(mat.fmt));
-    return cq > kCW ? kCW : cq;
+    return cq > 2 * kCW ? 2 * kCW : cq;
   };
   a.cq_w = chunk_quanta(h->w, a.qt_w);
   a.cq_a = ab ? chunk_quanta(h->a, a.qt_a) : 1;
@@ -528,9 +598,11 @@ SPlan make_splan(const Handle* h, int m) {
     int ubytes = (nq_w / s) * a.qt_w * tbw;
     if (s > 1 && ubytes < 8192) break;
     int units = h->w.nt * s;
-    int G = units < G_max ? units : G_max;
-    double eff = ((double)units / G) / (double)((units + G - 1) / G);
-    if (s > 1) eff -= 0.03 * (s - 1);                          // split-K has a price
+    // two CTAs share an SM and its issue slots, so what has to balance is units per SM
+    int sms = h->sm_count;
+    double per_sm = (double)units / sms;
+    double eff = per_sm >= 1.0 ? per_sm / (double)((units + sms - 1) / sms) : per_sm;
+    if (s > 1) eff -= 0.02 * (s - 1);                          // split-K has a price
     if (eff > best_eff) { best_eff = eff; best_split = s; }
   }
   a.w_split = best_split;
