@@ -1,0 +1,130 @@
+"""GPU parity at the full LLaMA3-8B layer sizes, in the launch configuration bench.py times.
+
+Decode cases (M <= 64) are compared element by element with the float64 oracle (its forward is cheap at
+small M).  Prefill cases (M = 2048) are compared on sampled outputs that the oracle computes one by one
+(forward_at), plus the whole output for the smallest shape.  Tolerances as everywhere: rel. Frobenius
+<= 2e-3, max|diff| <= 1e-2 * max|y| (for sampled checks the norms run over the samples)."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from oracle import eora_oracle as orc
+import eora_inputs as gen
+import paper_2410_21271_b200 as eora
+from helpers import make_case, run_layer, check_parity, x_to_torch
+
+SHAPES = gen.LLAMA3_8B_SHAPES
+
+
+def sampled_check(L, wf, af, bf, x, xd, n_samples=96, seed=0):
+    y = run_layer(L, x, xd)
+    rng = np.random.default_rng(seed)
+    M, N = y.shape
+    mi = rng.integers(0, M, n_samples)
+    ni = rng.integers(0, N, n_samples)
+    mi[:4] = [0, M - 1, 0, M - 1]; ni[:4] = [0, 0, N - 1, N - 1]          # corners: first / last tile edges
+    ref = orc.forward_at(x, xd, wf, af, bf, mi, ni)
+    got = y[mi, ni]
+    d = got - ref
+    assert np.all(np.isfinite(y))
+    assert np.linalg.norm(d) / np.linalg.norm(ref) <= 2e-3
+    assert np.abs(d).max() <= 1e-2 * np.abs(ref).max()
+
+
+# config 1 and 2: 4-bit / 3-bit backbone, fp16 rank-128 adapter, decode
+@pytest.mark.parametrize("name", ["q", "k", "gate", "down"])
+@pytest.mark.parametrize("w,M", [("q4", 1), ("q3", 1), ("q3", 8), ("q3", 16)])
+def test_decode_fullsize(name, w, M):
+    K, N = SHAPES[name]
+    wf, af, bf = make_case(31, K, N, 128, w=w)
+    x = gen.make_x(32, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    assert L.path(M) == eora.EORA_PATH_DECODE
+    y = run_layer(L, x, "f16")
+    rel, _ = check_parity(y, orc.forward(x, "f16", wf, af, bf), f"{name} {w} M{M}")
+    assert 5e-5 < rel < 1e-3          # fp16 output rounding alone is ~2e-4: far off means a harness bug
+    L.close()
+
+
+# config 3: quantised adapter
+@pytest.mark.parametrize("name,ab,r,M", [("q", "q4", 128, 1), ("k", "q4", 512, 16), ("q", "q8", 128, 64),
+                                         ("down", "q4", 128, 1), ("gate", "q8", 512, 1)])
+def test_decode_quantised_adapter_fullsize(name, ab, r, M):
+    K, N = SHAPES[name]
+    wf, af, bf = make_case(33, K, N, r, w="q4", ab=ab)
+    x = gen.make_x(34, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    assert L.path(M) == eora.EORA_PATH_DECODE
+    check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} {ab} r{r} M{M}")
+    L.close()
+
+
+# config 4: prefill
+def test_prefill_fullsize_whole_output():
+    K, N = SHAPES["k"]
+    M = 2048
+    wf, af, bf = make_case(35, K, N, 128, w="q4")
+    x = gen.make_x(36, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    assert L.path(M) == eora.EORA_PATH_PREFILL
+    rel, _ = check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), "k prefill")
+    assert 5e-5 < rel < 1e-3
+    L.close()
+
+
+@pytest.mark.parametrize("name,r,xd", [("q", 128, "f16"), ("q", 512, "bf16"), ("gate", 64, "f16"), ("down", 128, "bf16")])
+def test_prefill_fullsize_sampled(name, r, xd):
+    K, N = SHAPES[name]
+    M = 2048
+    wf, af, bf = make_case(37, K, N, r, w="q4")
+    x = gen.make_x(38, M, K, xd)
+    L = eora.Layer(wf, af, bf, max_m=M, x_dtype=xd)
+    assert L.path(M) == eora.EORA_PATH_PREFILL
+    sampled_check(L, wf, af, bf, x, xd)
+    L.close()
+
+
+def test_prefill_weights_are_the_rounded_dequantised_values():
+    """X = identity block, rank 0, fp32 out: Y is the fp16-rounded dequantised weight, bit for bit."""
+    K, N = 512, 256
+    wf, _, _ = make_case(39, K, N, 0, w="q4")
+    x = np.eye(K, dtype=np.float16)
+    L = eora.Layer(wf, None, None, max_m=K, y_dtype="f32")
+    assert L.path(K) == eora.EORA_PATH_PREFILL
+    y = run_layer(L, x, "f16")
+    q = orc.unpack_codes(wf["codes"], 4, K); z = orc.unpack_zeros(wf["zeros"], 4, N)
+    assert np.array_equal(y, orc.deq_fp16(q, z, wf["scales"], 128).astype(np.float64))
+    L.close()
+
+
+# config 5: 2:4 backbone
+@pytest.mark.parametrize("name,M", [("k", 1), ("q", 1), ("k", 2048)])
+def test_sparse24_fullsize(name, M):
+    K, N = SHAPES[name]
+    wf, af, bf = make_case(41, K, N, 128, w="sp24")
+    x = gen.make_x(42, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    if M == 1:
+        check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} sp24 M1")
+    else:
+        assert L.path(M) == eora.EORA_PATH_PREFILL
+        sampled_check(L, wf, af, bf, x, "f16")
+    L.close()
+
+
+def test_prefill_small_formats():
+    """Every adapter format and odd sizes through the tensor-core path."""
+    for (w, ab, K, N, r, M, yd) in [("q3", "q4", 512, 352, 128, 130, "f16"), ("q4", "q8", 640, 96, 64, 257, "bf16"),
+                                    ("sp24", "f16", 384, 288, 24, 100, "f32"), ("q3", "f16", 1024, 512, 0, 300, "f16")]:
+        wf, af, bf = make_case(43, K, N, r, w=w, ab=ab)
+        x = gen.make_x(44, M, K)
+        L = eora.Layer(wf, af, bf, max_m=M, y_dtype=yd)
+        assert L.path(M) == eora.EORA_PATH_PREFILL
+        y = run_layer(L, x, "f16")
+        rel, mabs = orc.parity_errors(y, orc.forward(x, "f16", wf, af, bf))
+        assert rel <= 2e-3 and mabs <= 1e-2, (w, ab, rel, mabs)
+        y2 = run_layer(L, x, "f16")           # scratch (the split-K sums of t) must have been restored
+        rel2, mabs2 = orc.parity_errors(y2, orc.forward(x, "f16", wf, af, bf))
+        assert rel2 <= 2e-3 and mabs2 <= 1e-2, (w, ab, rel2, mabs2)
+        L.close()
