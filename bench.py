@@ -60,7 +60,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -109,33 +109,63 @@ def build_layer_set(blocks: int, device: str, seed0: int = 1000):
             layers.append((name, K, N, eora.Layer(wf, af, bf, max_m=M_DECODE, device=device)))
     xs, ys = {}, {}
     for name, (K, N) in LAYERS:
-        xs[K] = torch.from_numpy(gen.make_x(7, M_DECODE, K)).to(device)
-        ys[N] = torch.empty((M_DECODE, N), dtype=torch.float16, device=device)
+        xs[name] = torch.from_numpy(gen.make_x(7, M_DECODE, K)).to(device)
+        ys[name] = torch.empty((M_DECODE, N), dtype=torch.float16, device=device)
     return layers, xs, ys
 
 
-def run_step(layers, xs, ys):
+# Inside a transformer block q, k, v read the same hidden state and gate, up the same one, so those launches
+# do not depend on each other: they go to side streams and join before o / down.  Everything else is in
+# stream order (each layer's input is the previous layer's output in the real model).
+CONCURRENT_WITH_PREVIOUS = {"k", "v", "up"}
+
+
+def run_step(layers, xs, ys, side=None):
+    import torch
     import paper_2410_21271_b200 as eora
-    for _, K, N, L in layers:
-        eora.eora_linear_forward(L.handle, xs[K], M_DECODE, ys[N])
+    main = torch.cuda.current_stream()
+    pending = []
+    i = 0
+    while i < len(layers):
+        group = [layers[i]]
+        while i + len(group) < len(layers) and layers[i + len(group)][0] in CONCURRENT_WITH_PREVIOUS:
+            group.append(layers[i + len(group)])
+        i += len(group)
+        if side is None or len(group) == 1:
+            for name, K, N, L in group:
+                eora.eora_linear_forward(L.handle, xs[name], M_DECODE, ys[name], main)
+            continue
+        fork = main.record_event()
+        for j, (name, K, N, L) in enumerate(group):
+            st = main if j == 0 else side[(j - 1) % len(side)]
+            if j:
+                st.wait_event(fork)
+            eora.eora_linear_forward(L.handle, xs[name], M_DECODE, ys[name], st)
+            if j:
+                pending.append(st.record_event())
+        for ev in pending:
+            main.wait_event(ev)
+        pending = []
 
 
-def time_decode(layers, xs, ys, steps: int, warmup: int, device_index: int, use_graph: bool = True):
+def time_decode(layers, xs, ys, steps: int, warmup: int, device_index: int, use_graph: bool = True,
+                use_streams: bool = True):
     """Device-timed steps (CUDA events on the launching stream).  Returns (ms per step, clocks)."""
     import torch
     stream = torch.cuda.Stream()
+    side = [torch.cuda.Stream(), torch.cuda.Stream()] if use_streams else None
     graph = None
     with torch.cuda.stream(stream):
-        run_step(layers, xs, ys)
-        stream.synchronize()
+        run_step(layers, xs, ys, side)
+        torch.cuda.synchronize()
         if use_graph:
             try:
                 graph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(graph, stream=stream):
-                    run_step(layers, xs, ys)
+                    run_step(layers, xs, ys, side)
             except Exception:
                 graph = None
-        launch = graph.replay if graph is not None else (lambda: run_step(layers, xs, ys))
+        launch = graph.replay if graph is not None else (lambda: run_step(layers, xs, ys, side))
         for _ in range(warmup):
             launch()
         stream.synchronize()
@@ -159,11 +189,11 @@ def time_decode(layers, xs, ys, steps: int, warmup: int, device_index: int, use_
 def time_e2e(layers, steps: int, warmup: int):
     """The same step through eora_linear_forward_host: pinned host X in, host Y out, per layer."""
     import torch
-    hx = {K: torch.from_numpy(gen.make_x(7, M_DECODE, K)).pin_memory() for _, (K, N) in LAYERS}
-    hy = {N: torch.empty((M_DECODE, N), dtype=torch.float16).pin_memory() for _, (K, N) in LAYERS}
+    hx = {name: torch.from_numpy(gen.make_x(7, M_DECODE, K)).pin_memory() for name, (K, N) in LAYERS}
+    hy = {name: torch.empty((M_DECODE, N), dtype=torch.float16).pin_memory() for name, (K, N) in LAYERS}
     def step():
-        for _, K, N, L in layers:
-            L.forward_host(hx[K], hy[N])
+        for name, K, N, L in layers:
+            L.forward_host(hx[name], hy[name])
     for _ in range(max(1, warmup)):
         step()
     torch.cuda.synchronize()
@@ -264,18 +294,21 @@ def aggregate(ms_local: float, tokens_per_step_per_rank: int, world: int) -> tup
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--blocks", type=int, default=gen.LLAMA3_8B_BLOCKS, help=argparse.SUPPRESS)
     ap.add_argument("--no-extras", action="store_true", help="skip the prefill / e2e / cpu legs")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--single-stream", action="store_true", help="launch all layers of a block in stream order")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     config = {"workload": WORKLOAD, "blocks": args.blocks, "layers_per_block": 7, "M": M_DECODE,
-              "l2": "weights of one step (3.4 GB) exceed L2, no flush needed", "parallelism": f"replicas x{world}"}
+              "l2": "weights of one step (3.4 GB) exceed L2, no flush needed", "parallelism": f"replicas x{world}",
+              "streams": ("stream order" if args.single_stream else
+                          "q,k,v and gate,up of a block are independent and run on 3 / 2 streams; the rest in stream order")}
 
     if args.impl == "reference":
         if rank != 0:
@@ -307,7 +340,8 @@ def main():
 
     layers, xs, ys = build_layer_set(args.blocks, device)
     n_launch_step = sum(L.launches(M_DECODE) for _, _, _, L in layers)
-    ms_local, clocks, graphed = time_decode(layers, xs, ys, args.steps, args.warmup, local_rank, not args.no_graph)
+    ms_local, clocks, graphed = time_decode(layers, xs, ys, args.steps, args.warmup, local_rank, not args.no_graph,
+                                             not args.single_stream)
     value, ms = aggregate(ms_local, M_DECODE, world)
     peaks, peak_kind = measured_peaks()
     bytes_step = step_bytes(args.blocks)
@@ -331,7 +365,7 @@ def main():
         L.close()
     if not args.no_extras and rank == 0:
         if world == 1:
-            line["cpu_baseline"] = cpu_oracle_sample(3)[0]
+            line["cpu_baseline"] = cpu_oracle_sample(8)[0]
         try:
             line["prefill"] = time_prefill(device)
             line["prefill"]["frac_of_measured_bf16_burst"] = line["prefill"]["tflops"] / peaks["bf16_tflops"]
