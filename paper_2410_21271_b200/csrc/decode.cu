@@ -1,480 +1,432 @@
-// Decode kernel family (M <= 64): one launch computes  Y = X.deq(Wq) + (X.A).B  (paper Eq. 4).
+// Decode path (m <= 8 tokens per launch): one kernel computes Eq. 4 for a whole layer,
+//     Y = X . deq(Wq) + (X . A) . B,
+// streaming every weight byte exactly once.
 //
-// Section 4.5 of the paper fuses only the product with B into the quantised mat-vec kernel and
-// leaves t = A.x to a separate op.  Here the whole layer is one pass: A is treated as `rank`
-// more output rows of the same streaming product over X, and B as `rank` more reduction
-// elements of the backbone product with t in the place of X, so Y is written exactly once.
+// Work decomposition.  All three matrices are stored as blobs of 16 rows x 128 reduction elements,
+// ordered pair-major (see eora_common.cuh), and every blob is an independent piece of work: a warp
+// multiplies it with the 128 activations it needs (kept in registers as tensor-core operand
+// fragments, tokens as the n8 side of mma.m16n8k16) and adds the 16 x m partial sums to an fp32
+// accumulator array in global memory with red.add.  Warps are fully independent: each owns a
+// contiguous run of blobs of up to three matrices, fetches it with its own bulk copies into its own
+// shared-memory ring and never synchronises with another warp of its CTA.
 //
-// Work decomposition.  A CTA (8 warps) owns one unit = (matrix, 16-row tile, reduction slice).
-// Units of A come first in blockIdx order, backbone units after them.  The packed weights of a
-// unit are one contiguous byte range; one thread brings them into shared memory with a few bulk
-// async copies (cp.async.bulk + mbarrier, no multicast) issued at the very start of the CTA, so
-// a whole layer is in flight at once and no registers are spent on prefetch.  Each warp then
-// walks its quanta (<= 128 reduction elements sharing one scale / zero-point): codes become the
-// exact fp16 integers (q - z) in registers, are multiplied with the activations on the tensor
-// cores (mma.m16n8k16, weights as the 16-row operand, fp32 accumulate) and the scale is applied
-// once per quantum in fp32.  The 8 warps are then summed through shared memory.
-//   A unit       : adds its partial t to the fp32 buffer t_ws (red.add), then bumps T_DONE.
-//   backbone unit: the last reduction slice of each row tile also owns the B extension: it waits
-//                  (bounded) for T_DONE, reads t, splits it into fp16 hi + lo parts and runs the
-//                  B tiles (prefetched with the weights) against them.  With one slice per row
-//                  tile the result goes straight to Y; otherwise slices add into y_ws and the
-//                  last one to arrive converts.
-// All scratch words are returned to zero before the kernel ends, so calls need no memset.
+//   * warps [0, n_a) ("A owners") take A first (t += X . A, sums in d_t) and then a share of W,
+//   * the other warps take their share of W first and then a share of B, for which the activations are
+//     t (read back as fp32 and split into an fp16 high and low part, so that t keeps fp32-like accuracy).
+// The only wait in the kernel is the one before the B share: all of A must have been added to t.  A
+// owners never wait, and they sit in the CTAs with the lowest indices, which are dispatched first, so a
+// waiting warp never holds the slot of a CTA it is waiting for.  The wait is bounded like every other.
 //
-// Programmatic dependent launch: the bulk copies of the weights are issued before
-// griddepcontrol.wait, i.e. while the previous kernel in the stream is still draining;
-// activations and scratch are touched only after it.
+// Completion.  Every blob of W or B that has been added to y_ws bumps the ticket of its row tile; the
+// warp that brings a ticket to its final count converts the 16 x m sums to the output type, writes Y and
+// puts the sums and the ticket back to zero.  The warp that finishes the last row tile also clears t
+// and the counters, so all scratch is back to zero when the kernel ends.
+//
+// Programmatic dependent launch: the first bulk copies (weights never change) are issued before
+// griddepcontrol.wait, i.e. while the previous kernel in the stream is still draining; activations
+// and scratch are only touched after it.
 #include "decode_common.cuh"
 
 namespace eora {
-using namespace dec;
 namespace {
+using namespace dec;
 
-constexpr int kWarps = 8;
+constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
-constexpr int kXPad = 32;                 // halves of padding per activation row in shared memory
-constexpr int kChunks = 4;                // bulk-copy chunks (one mbarrier each) per unit
-constexpr int kUnitBytes = 32 * 1024;     // largest packed-weight slice of one unit
-constexpr int kXSmemBudget = 64 * 1024;   // bytes of staged activations per CTA
-constexpr int kMaxSmem = 200 * 1024;
+constexpr int kCtasPerSm = 4;
+constexpr int kRing = 3;                  // bulk copies in flight per warp
+constexpr int kSlotBytes = 4352;          // one ring slot = one bulk copy (a run of whole blobs)
+constexpr int kSmemBytes = kWarps * kRing * kSlotBytes + kWarps * kRing * 8;
 
+enum { CNT_A_DONE = 0, CNT_TILES_DONE = 1, CNT_TICKET0 = 2 };
 
-// What one CTA streams: a slice of nq quanta of one row tile, (being) copied to shared memory.
-struct SliceView {
-  const uint8_t* wbuf;      // tile blobs of the slice, first tile of the slice at offset 0
-  const uint32_t* sc;       // scales from the first group the slice touches (8 words per group)
-  const uint16_t* zz;
-  uint64_t* bars;           // kChunks barriers, chunk c covers quanta [c*cq, (c+1)*cq) of the slice
-  int nq;                   // quanta in the slice
-  int qt;                   // tiles per quantum
-  int cq;                   // quanta per chunk
-  int group_tiles;          // tiles per quantisation group
-  int gofs;                 // tiles between the start of that first group and the slice start
-};
-
-// Accumulate the slice against NX activation sources in shared memory (source s at
-// xs + s * xsrc_stride halves; row `token` at + token * xrow; reduction index 0 = slice start).
-template <int FMT, int MT, int NX>
-__device__ __forceinline__ void run_slice(const SliceView& sv, int warp, int lane, const __half* xs, int xrow,
-                                          int xsrc_stride, int m_rows, int* dev_status, float (&acc)[MT][4]) {
-  constexpr int TB = FMT == FMT_Q4 ? 512 : FMT == FMT_Q3 ? 384 : FMT == FMT_Q8 ? 1024 : 2048;
-  const int g = lane >> 2, t = lane & 3;
-  int chunk_ready = -1;
-#pragma unroll 1
-  for (int q = warp; q < sv.nq; q += kWarps) {
-    const int chunk = q / sv.cq;
-    if (chunk > chunk_ready) {
-      mbar_wait_warp(sv.bars + chunk, 0, dev_status, lane);
-      chunk_ready = chunk;
-    }
-    float gacc[MT][4];
-    ZC zc;
-    uint32_t sc2 = 0;
-    if constexpr (is_quant<FMT>()) {
-#pragma unroll
-      for (int mt = 0; mt < MT; ++mt) gacc[mt][0] = gacc[mt][1] = gacc[mt][2] = gacc[mt][3] = 0.f;
-      const int gi = (sv.gofs + q * sv.qt) / sv.group_tiles;
-      sc2 = sv.sc[gi * 8 + g];
-      make_zc<FMT>(zc, sv.zz[gi * 8 + g]);
-    }
-#pragma unroll 1
-    for (int tt = 0; tt < sv.qt; ++tt) {
-      const int tile = q * sv.qt + tt;
-      uint32_t a[4][4];
-      tile_frags<FMT>(sv.wbuf + tile * TB, lane, zc, a);
-      const int koff = tile * 64 + 8 * t;
-#pragma unroll
-      for (int s = 0; s < NX; ++s) {
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-          const int token = mt * 8 + g;
-          uint4 x0 = make_uint4(0, 0, 0, 0), x1 = make_uint4(0, 0, 0, 0);
-          if (token < m_rows) {
-            const __half* p = xs + s * xsrc_stride + token * xrow + koff;
-            x0 = *reinterpret_cast<const uint4*>(p);
-            x1 = *reinterpret_cast<const uint4*>(p + 32);
-          }
-          float(&d)[4] = is_quant<FMT>() ? gacc[mt] : acc[mt];
-          mma16816(d, a[0], x0.x, x0.y);
-          mma16816(d, a[1], x0.z, x0.w);
-          mma16816(d, a[2], x1.x, x1.y);
-          mma16816(d, a[3], x1.z, x1.w);
-        }
-      }
-    }
-    if constexpr (is_quant<FMT>()) {
-      const float sa = __half2float(__ushort_as_half((unsigned short)(sc2 & 0xffffu)));
-      const float sb = __half2float(__ushort_as_half((unsigned short)(sc2 >> 16)));
-#pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        acc[mt][0] = fmaf(sa, gacc[mt][0], acc[mt][0]);
-        acc[mt][1] = fmaf(sa, gacc[mt][1], acc[mt][1]);
-        acc[mt][2] = fmaf(sb, gacc[mt][2], acc[mt][2]);
-        acc[mt][3] = fmaf(sb, gacc[mt][3], acc[mt][3]);
-      }
-    }
-  }
-}
+struct Share { uint32_t per, rem; };      // blobs of a matrix dealt to n warps: warp i gets per + (i < rem)
 
 struct DecodeArgs {
-  WMat w, a, b;
-  const void* x;
-  void* y;
-  float* t_ws;
-  float* y_ws;
-  uint32_t* counters;
-  int* dev_status;
-  int m, d_in, d_out, r_pad;
-  int x_dtype, y_dtype;
-  int a_units, a_split, w_split;
-  int qt_w, qt_a, qt_b;     // tiles per quantum of each matrix
-  // shared-memory carve-up (byte offsets from the dynamic shared memory base)
-  int off_sc, off_zz, off_b, off_bsc, off_bzz, off_x, off_red;
-  unsigned long long* trace;   // optional: 16 timestamps (ns) per CTA, see eora_linear_set_trace
+  const uint8_t* a_q; const uint8_t* w_q; const uint8_t* b_q;
+  uint32_t a_nt, w_nt;                    // row tiles of A and of W (= of B)
+  uint32_t a_blobs, w1_blobs;             // all of A; the part of W that the A owners take
+  uint32_t a_per_copy, w_per_copy, b_per_copy;   // blobs per bulk copy
+  uint32_t a_sz2, w_sz2, b_sz2;
+  uint32_t n_a;                           // number of A-owner warps
+  Share sh_a, sh_w1, sh_w2, sh_b;
+  uint32_t tile_target;                   // blobs per output row tile: pairs of W + pairs of B
+  const void* x; void* y;
+  float* d_t; float* y_ws; uint32_t* counters; int* dev_status;
+  int m, d_in, d_out, r_pad, n_pad, x_dtype, y_dtype;
+  unsigned long long* trace;
 };
 
-#define EORA_TRACE(slot) do { if (p.trace && threadIdx.x == 0) p.trace[(size_t)blockIdx.x * 16 + (slot)] = globaltimer_ns(); } while (0)
+__device__ __forceinline__ uint32_t share_lo(const Share& s, uint32_t i) { return i * s.per + (i < s.rem ? i : s.rem); }
+__device__ __forceinline__ uint32_t share_n(const Share& s, uint32_t i) { return s.per + (i < s.rem ? 1u : 0u); }
 
-// Stage activation rows [0, m) x reduction range [k0, k0 + len) into shared memory as fp16.
-__device__ __forceinline__ void stage_x(__half* xs, int xrow, const void* x, int x_dtype, int m, int d_in, int k0, int len) {
-  const int chunks = len >> 3;   // 16-byte chunks per row
-  for (int row = 0; row < m; ++row) {
-    for (int c = threadIdx.x; c < chunks; c += kThreads) {
-      uint4 v = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(x) + (int64_t)row * d_in + k0 + c * 8);
-      if (x_dtype == EORA_X_BF16) {
-        uint32_t* pv = reinterpret_cast<uint32_t*>(&v);
+__device__ __forceinline__ uint4 ld_cg_u4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t pack_h2(float a, float b) {
+  __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t bf2_to_h2(uint32_t v) {
+  return pack_h2(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+}
+
+// Activation fragments of one pair (128 reduction elements) for lane (g, t): token g, elements
+// 64*c + 32*blk + 8*t + [0, 8) in xr[8*c + 4*blk + 0..3].
+__device__ __forceinline__ void load_x_pair(uint32_t (&xr)[16], const DecodeArgs& p, uint32_t pair, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  if (g < p.m) {
+    const uint16_t* src = reinterpret_cast<const uint16_t*>(p.x) + (size_t)g * p.d_in + pair * 128 + 8 * t;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          __nv_bfloat162 b2 = *reinterpret_cast<__nv_bfloat162*>(&pv[j]);
-          float2 f = __bfloat1622float2(b2);
-          __half2 h2 = __floats2half2_rn(f.x, f.y);
-          pv[j] = *reinterpret_cast<uint32_t*>(&h2);
+    for (int i = 0; i < 4; ++i) {
+      uint4 v = ld_cg_u4(src + 32 * i);
+      if (p.x_dtype == EORA_X_BF16) { v.x = bf2_to_h2(v.x); v.y = bf2_to_h2(v.y); v.z = bf2_to_h2(v.z); v.w = bf2_to_h2(v.w); }
+      xr[4 * i] = v.x; xr[4 * i + 1] = v.y; xr[4 * i + 2] = v.z; xr[4 * i + 3] = v.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) xr[i] = 0u;
+  }
+}
+
+// The same for t (fp32 sums in d_t [8][r_pad]), split into high and low fp16 parts.
+__device__ __forceinline__ void load_t_pair(uint32_t (&xh)[16], uint32_t (&xl)[16], const DecodeArgs& p, uint32_t pair, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  const float* src = p.d_t + (size_t)g * p.r_pad + pair * 128 + 8 * t;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+#pragma unroll
+    for (int hq = 0; hq < 2; ++hq) {
+      const uint4 u = ld_cg_u4(src + 32 * i + 4 * hq);
+      const float f[4] = {__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w)};
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const __half h0 = __float2half_rn(f[2 * j]), h1 = __float2half_rn(f[2 * j + 1]);
+        const __half2 hi = __halves2half2(h0, h1);
+        xh[4 * i + 2 * hq + j] = *reinterpret_cast<const uint32_t*>(&hi);
+        xl[4 * i + 2 * hq + j] = pack_h2(f[2 * j] - __half2float(h0), f[2 * j + 1] - __half2float(h1));
+      }
+    }
+  }
+}
+
+// One blob: 16 rows x 128 reduction elements times the activation fragments -> tot (this lane's four
+// entries of the 16 x 8 result: rows g / g + 8, tokens 2t / 2t + 1).
+template <int FMT, bool HILO>
+__device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint32_t sz2, const uint32_t (&xr)[16],
+                                             const uint32_t (&xl)[16], float (&tot)[4]) {
+  constexpr int tb = tile_bytes(FMT);
+  constexpr bool quant = fmt_quantised(FMT);
+  const int g = lane >> 2;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  tot[0] = tot[1] = tot[2] = tot[3] = 0.f;
+  ZC zc;
+  float s_a = 0.f, s_b = 0.f;
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    if constexpr (quant) {
+      if (c == 0 || sz2) {
+        const uint8_t* sz = blob + 2 * tb + c * kSzEntryBytes;      // c != 0 only with two entries
+        const uint32_t s2 = reinterpret_cast<const uint32_t*>(sz)[g];
+        const uint32_t z2 = reinterpret_cast<const uint16_t*>(sz + 32)[g];
+        make_zc<FMT>(zc, z2);
+        s_a = __half2float(__ushort_as_half((unsigned short)(s2 & 0xffffu)));
+        s_b = __half2float(__ushort_as_half((unsigned short)(s2 >> 16)));
+      }
+    }
+    uint32_t a[4][4];
+    tile_frags<FMT>(blob + c * tb, lane, zc, a);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      mma16816(acc, a[i], xr[8 * c + 2 * i], xr[8 * c + 2 * i + 1]);
+      if constexpr (HILO) mma16816(acc, a[i], xl[8 * c + 2 * i], xl[8 * c + 2 * i + 1]);
+    }
+    if constexpr (quant) {
+      if (c == 1 || sz2) {
+        tot[0] = fmaf(acc[0], s_a, tot[0]); tot[1] = fmaf(acc[1], s_a, tot[1]);
+        tot[2] = fmaf(acc[2], s_b, tot[2]); tot[3] = fmaf(acc[3], s_b, tot[3]);
+        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+      }
+    }
+  }
+  if constexpr (!quant) { tot[0] = acc[0]; tot[1] = acc[1]; tot[2] = acc[2]; tot[3] = acc[3]; }
+}
+
+// tot -> sums[token][ld] for rows 16 * tile + {g, g + 8}
+__device__ __forceinline__ void flush_sums(float* sums, int ld, uint32_t tile, const float (&tot)[4], int m, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  float* base = sums + (size_t)(2 * t) * ld + tile * 16 + g;
+  if (2 * t < m) { red_add(base, tot[0]); red_add(base + 8, tot[2]); }
+  if (2 * t + 1 < m) { red_add(base + ld, tot[1]); red_add(base + ld + 8, tot[3]); }
+}
+
+__device__ __forceinline__ uint32_t atom_add_acq_rel(uint32_t* p, uint32_t v) {
+  uint32_t old;
+  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+__device__ __forceinline__ void red_add_release(uint32_t* p, uint32_t v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Per-warp state of the copy ring.  All lanes keep the same copy of it; lane 0 issues.
+struct Ring {
+  uint8_t* slots;
+  uint64_t* bars;
+  // producer side: the run of blobs still to be requested, over up to three segments
+  const uint8_t* ptr[3];
+  uint32_t rem[3], blob[3], per[3];
+  int pseg;
+  // consumer side
+  int slot;
+  uint32_t parity;
+};
+
+__device__ __forceinline__ void ring_issue(Ring& r, int slot, int lane) {
+  if (r.pseg == 0 && r.rem[0] == 0) r.pseg = 1;
+  if (r.pseg == 1 && r.rem[1] == 0) r.pseg = 2;
+  if (r.pseg == 2 && r.rem[2] == 0) r.pseg = 3;
+  if (r.pseg >= 3) return;
+  // runtime-indexed reads of three-element arrays would go to local memory: select instead
+  const int s = r.pseg;
+  const uint8_t* src = s == 0 ? r.ptr[0] : s == 1 ? r.ptr[1] : r.ptr[2];
+  const uint32_t rem = s == 0 ? r.rem[0] : s == 1 ? r.rem[1] : r.rem[2];
+  const uint32_t blob = s == 0 ? r.blob[0] : s == 1 ? r.blob[1] : r.blob[2];
+  const uint32_t per = s == 0 ? r.per[0] : s == 1 ? r.per[1] : r.per[2];
+  const uint32_t n = rem < per ? rem : per;
+  const uint32_t bytes = n * blob;
+  if (lane == 0) {
+    mbar_expect_tx(r.bars + slot, bytes);
+    bulk_g2s(r.slots + slot * kSlotBytes, src, bytes, r.bars + slot);
+  }
+  if (s == 0) { r.ptr[0] = src + bytes; r.rem[0] = rem - n; }
+  else if (s == 1) { r.ptr[1] = src + bytes; r.rem[1] = rem - n; }
+  else { r.ptr[2] = src + bytes; r.rem[2] = rem - n; }
+}
+
+enum { OUT_T = 0, OUT_Y = 1 };
+
+__device__ __forceinline__ void st_zero4(float* p) {
+  *reinterpret_cast<float4*>(p) = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// Row tile `tile` of the output is complete.  Called by ONE lane (the one whose ticket was the last);
+// it converts the tile's 16 x m sums, stores them and puts the scratch back to zero.  Several lanes of a
+// warp may each be finishing a tile of their own at the same time.
+__device__ __forceinline__ void finish_row_tile(const DecodeArgs& p, uint32_t tile) {
+  for (int token = 0; token < p.m; ++token) {
+    float* s = p.y_ws + (size_t)token * p.n_pad + tile * 16;
+    uint4 u[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) u[i] = ld_cg_u4(s + 4 * i);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) st_zero4(s + 4 * i);
+    const float v[16] = {__uint_as_float(u[0].x), __uint_as_float(u[0].y), __uint_as_float(u[0].z), __uint_as_float(u[0].w),
+                         __uint_as_float(u[1].x), __uint_as_float(u[1].y), __uint_as_float(u[1].z), __uint_as_float(u[1].w),
+                         __uint_as_float(u[2].x), __uint_as_float(u[2].y), __uint_as_float(u[2].z), __uint_as_float(u[2].w),
+                         __uint_as_float(u[3].x), __uint_as_float(u[3].y), __uint_as_float(u[3].z), __uint_as_float(u[3].w)};
+    const int64_t o = (int64_t)token * p.d_out + tile * 16;       // d_out is a multiple of 32: the 16 outputs exist
+    if (p.y_dtype == EORA_Y_F32) {
+      float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.y) + o);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    } else {
+      uint32_t h[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (p.y_dtype == EORA_Y_F16) {
+          h[i] = pack_h2(v[2 * i], v[2 * i + 1]);
+        } else {
+          const __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+          h[i] = *reinterpret_cast<const uint32_t*>(&b);
         }
       }
-      *reinterpret_cast<uint4*>(xs + row * xrow + c * 8) = v;
+      uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(p.y) + o);
+      dst[0] = make_uint4(h[0], h[1], h[2], h[3]);
+      dst[1] = make_uint4(h[4], h[5], h[6], h[7]);
     }
+  }
+  p.counters[CNT_TICKET0 + tile] = 0u;
+}
+
+// One segment: `n` consecutive blobs of one matrix starting at blob index b0.
+template <int FMT, bool HILO, int OUT>
+__device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32_t b0, uint32_t n, uint32_t nt, uint32_t blob_b,
+                                            uint32_t per_copy, uint32_t sz2, int lane) {
+  if constexpr (FMT == FMT_NONE) {
+    return true;
+  } else {
+    if (n == 0) return true;
+    uint32_t pair = b0 / nt, tile = b0 - pair * nt;
+    uint32_t xr[16], xl[16];
+    if constexpr (HILO) {
+      // all of A must be in t
+      int ok = 1;
+      if (lane == 0) ok = counter_wait(p.counters + CNT_A_DONE, p.a_blobs, p.dev_status) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) return false;
+      __syncwarp();
+      load_t_pair(xr, xl, p, pair, lane);
+    } else {
+      load_x_pair(xr, p, pair, lane);
+    }
+    // Tickets of the blobs flushed so far are taken in batches of up to 32 (one atomic per lane, one
+    // round trip per batch): batch_tile is the row tile of the batch's first blob, batch_n its size.
+    uint32_t batch_tile = tile, batch_n = 0, flushed = 0;
+    auto commit_batch = [&]() {
+      __syncwarp();
+      uint32_t done = 0, my_tile = 0;
+      if ((uint32_t)lane < batch_n) {
+        my_tile = (batch_tile + lane) % nt;
+        done = atom_add_acq_rel(p.counters + CNT_TICKET0 + my_tile, 1u) + 1u == p.tile_target ? 1u : 0u;
+      }
+      const uint32_t mask = __ballot_sync(0xffffffffu, done != 0);
+      if (mask) {
+        if (done) finish_row_tile(p, my_tile);
+        uint32_t last = 0;
+        if (lane == 0) last = atom_add_acq_rel(p.counters + CNT_TILES_DONE, (uint32_t)__popc(mask)) + __popc(mask) == p.w_nt ? 1u : 0u;
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {                               // the whole layer is done: nobody reads t any more
+          for (int i = lane; i < 8 * p.r_pad / 4; i += 32) st_zero4(p.d_t + 4 * i);
+          if (lane == 0) { p.counters[CNT_A_DONE] = 0u; p.counters[CNT_TILES_DONE] = 0u; }
+        }
+      }
+      batch_n = 0;
+    };
+    while (n > 0) {
+      const uint32_t cn = n < per_copy ? n : per_copy;
+      if (!mbar_wait_warp(r.bars + r.slot, r.parity, p.dev_status, lane)) return false;
+      const uint8_t* src = r.slots + r.slot * kSlotBytes;
+#pragma unroll 1
+      for (uint32_t j = 0; j < cn; ++j) {
+        float tot[4];
+        blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot);
+        if constexpr (OUT == OUT_T) {
+          flush_sums(p.d_t, p.r_pad, tile, tot, p.m, lane);
+          ++flushed;
+        } else {
+          if (batch_n == 0) batch_tile = tile;
+          flush_sums(p.y_ws, p.n_pad, tile, tot, p.m, lane);
+          if (++batch_n == 32) commit_batch();
+        }
+        if (++tile == nt) {
+          tile = 0;
+          ++pair;
+          if (j + 1 < cn || n > cn) {
+            if constexpr (HILO) load_t_pair(xr, xl, p, pair, lane);
+            else load_x_pair(xr, p, pair, lane);
+          }
+        }
+      }
+      __syncwarp();                               // every lane is done with the slot
+      ring_issue(r, r.slot, lane);
+      if (++r.slot == kRing) { r.slot = 0; r.parity ^= 1u; }
+      n -= cn;
+    }
+    if constexpr (OUT == OUT_T) {
+      __syncwarp();
+      if (lane == 0) red_add_release(p.counters + CNT_A_DONE, flushed);
+    } else {
+      if (batch_n) commit_batch();
+    }
+    return true;
   }
 }
 
-// Issue the bulk copies of one slice (quanta [q0, q0 + nq) of row tile `tile`) in kChunks pieces,
-// plus (with the first piece) the scales and zero-points of the groups the slice touches.
-// Returns the tile offset of the slice start inside its first group.
-__device__ __forceinline__ int issue_slice(const WMat& m, int tile, int q0, int nq, int qt, int cq, uint8_t* wbuf,
-                                           uint32_t* sc_s, uint16_t* zz_s, uint64_t* bars) {
-  const int tb = tile_bytes(m.fmt);
-  const uint8_t* src = m.q + ((int64_t)tile * m.kc + (int64_t)q0 * qt) * tb;
-  const bool quant = m.fmt == FMT_Q4 || m.fmt == FMT_Q3 || m.fmt == FMT_Q8;
-  const int gt = m.group / 64;
-  const int g0 = (q0 * qt) / gt;
-  for (int c = 0; c < kChunks; ++c) {
-    int qa = c * cq, qb = (c + 1) * cq < nq ? (c + 1) * cq : nq;
-    uint32_t bytes = qb > qa ? (uint32_t)(qb - qa) * qt * tb : 0u;
-    uint32_t extra_sc = 0, extra_zz = 0;
-    if (c == 0 && quant) {
-      const int g1 = ((q0 + nq) * qt + gt - 1) / gt;
-      extra_sc = (uint32_t)(g1 - g0) * 32u;
-      extra_zz = (uint32_t)(g1 - g0) * 16u;
-    }
-    mbar_expect_tx(bars + c, bytes + extra_sc + extra_zz);
-    if (bytes) bulk_g2s(wbuf + (size_t)qa * qt * tb, src + (size_t)qa * qt * tb, bytes, bars + c);
-    if (extra_sc) {
-      bulk_g2s(sc_s, m.sc + ((int64_t)tile * m.ng + g0) * 8, extra_sc, bars + c);
-      bulk_g2s(zz_s, m.zz + ((int64_t)tile * m.ng + g0) * 8, extra_zz, bars + c);
-    }
-  }
-  return q0 * qt - g0 * gt;
-}
-
-template <int WF, int ABF, int MT>
-__global__ void __launch_bounds__(kThreads, MT == 1 ? 3 : (MT == 2 ? 2 : 1)) k_decode(const DecodeArgs p) {
+template <int WF, int ABF>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_constant__ DecodeArgs p) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) uint64_t bars[2 * kChunks];
-  __shared__ uint32_t s_flag;
-
-  asm volatile("griddepcontrol.launch_dependents;");
-  EORA_TRACE(0);
-
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int unit = blockIdx.x;
-  const bool is_a = unit < p.a_units;
-  int tile, slice, split;
-  if (is_a) { tile = unit / p.a_split; slice = unit % p.a_split; split = p.a_split; }
-  else { int u = unit - p.a_units; tile = u / p.w_split; slice = u % p.w_split; split = p.w_split; }
-  const WMat& mat = is_a ? p.a : p.w;
-  const int qt = is_a ? p.qt_a : p.qt_w;
-  const int nq_all = mat.kc / qt;                   // quanta per row tile
-  const int q0 = (int)((int64_t)nq_all * slice / split), q1 = (int)((int64_t)nq_all * (slice + 1) / split);
-  const int nq = q1 - q0;
-  const int cq = (nq + kChunks - 1) / kChunks;
-  const int k_base = q0 * qt * 64, k_len = nq * qt * 64;
-  const int xrow = k_len + kXPad;
-  const bool owns_b = !is_a && slice == split - 1 && p.a_units > 0;
-  const int nqb = owns_b ? p.b.kc / p.qt_b : 0;
-  const int cqb = owns_b ? (nqb + kChunks - 1) / kChunks : 1;
+  const uint32_t gw = blockIdx.x * kWarps + warp;
+  asm volatile("griddepcontrol.launch_dependents;");
+  unsigned long long* tr = p.trace ? p.trace + (size_t)gw * 4 : nullptr;
+  if (tr && lane == 0) tr[0] = globaltimer_ns();
 
-  uint8_t* wbuf = smem;
-  uint32_t* sc_s = reinterpret_cast<uint32_t*>(smem + p.off_sc);
-  uint16_t* zz_s = reinterpret_cast<uint16_t*>(smem + p.off_zz);
-  uint8_t* bbuf = smem + p.off_b;
-  uint32_t* bsc_s = reinterpret_cast<uint32_t*>(smem + p.off_bsc);
-  uint16_t* bzz_s = reinterpret_cast<uint16_t*>(smem + p.off_bzz);
-  __half* xs = reinterpret_cast<__half*>(smem + p.off_x);
-  float* red = reinterpret_cast<float*>(smem + p.off_red);
-
-  // the slice start inside its first quantisation group, in tiles (same formula as issue_slice)
-  const int gofs = q0 * qt - ((q0 * qt) / (mat.group / 64)) * (mat.group / 64);
-
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < 2 * kChunks; ++i) mbar_init(bars + i, 1);
+  Ring r;
+  r.slots = smem + warp * (kRing * kSlotBytes);
+  r.bars = reinterpret_cast<uint64_t*>(smem + kWarps * kRing * kSlotBytes) + warp * kRing;
+  r.slot = 0; r.parity = 0; r.pseg = 0;
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < kRing; ++i) mbar_init(r.bars + i, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    // weights are immutable: their copies may start before the previous kernel has finished
-    issue_slice(mat, tile, q0, nq, qt, cq, wbuf, sc_s, zz_s, bars);
-    if (owns_b) issue_slice(p.b, tile, 0, nqb, p.qt_b, cqb, bbuf, bsc_s, bzz_s, bars + kChunks);
   }
-  EORA_TRACE(1);
+  __syncwarp();
+
+  // this warp's three runs: A, W, B (one of A / B is empty)
+  const bool a_owner = gw < p.n_a;
+  uint32_t a0 = 0, an = 0, w0, wn, bb0 = 0, bn = 0;
+  if (a_owner) {
+    a0 = share_lo(p.sh_a, gw); an = share_n(p.sh_a, gw);
+    w0 = share_lo(p.sh_w1, gw); wn = share_n(p.sh_w1, gw);
+  } else {
+    const uint32_t i = gw - p.n_a;
+    w0 = p.w1_blobs + share_lo(p.sh_w2, i); wn = share_n(p.sh_w2, i);
+    bb0 = share_lo(p.sh_b, i); bn = share_n(p.sh_b, i);
+  }
+  const uint32_t blob_a = blob_bytes(ABF, p.a_sz2), blob_w = blob_bytes(WF, p.w_sz2), blob_b = blob_bytes(ABF, p.b_sz2);
+  r.ptr[0] = p.a_q + (size_t)a0 * blob_a; r.rem[0] = an; r.blob[0] = blob_a; r.per[0] = p.a_per_copy;
+  r.ptr[1] = p.w_q + (size_t)w0 * blob_w; r.rem[1] = wn; r.blob[1] = blob_w; r.per[1] = p.w_per_copy;
+  r.ptr[2] = p.b_q + (size_t)bb0 * blob_b; r.rem[2] = bn; r.blob[2] = blob_b; r.per[2] = p.b_per_copy;
+
+#pragma unroll
+  for (int i = 0; i < kRing; ++i) ring_issue(r, i, lane);
+
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  EORA_TRACE(2);
-  stage_x(xs, xrow, p.x, p.x_dtype, p.m, p.d_in, k_base, k_len);
-  __syncthreads();      // barriers initialised, X staged
-  EORA_TRACE(3);
+  if (tr && lane == 0) tr[1] = globaltimer_ns();
 
-  float acc[MT][4];
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
-
-  SliceView sv;
-  sv.wbuf = wbuf; sv.sc = sc_s; sv.zz = zz_s; sv.bars = bars; sv.nq = nq; sv.qt = qt; sv.cq = cq;
-  sv.group_tiles = mat.group / 64; sv.gofs = gofs;
-  if (is_a) {
-    if constexpr (ABF != FMT_NONE) run_slice<ABF, MT, 1>(sv, warp, lane, xs, xrow, 0, p.m, p.dev_status, acc);
-  } else {
-    run_slice<WF, MT, 1>(sv, warp, lane, xs, xrow, 0, p.m, p.dev_status, acc);
-  }
-
-  EORA_TRACE(4);
-  // ---- B extension: the last slice of a backbone row tile adds (X.A).B for its 16 output columns
-  if constexpr (ABF != FMT_NONE) {
-    if (owns_b) {
-      __syncthreads();                                   // everyone is done reading the staged X
-      if (threadIdx.x == 0) {
-        counter_wait(p.counters + CNT_T_DONE, (uint32_t)p.a_units, p.dev_status);
-      }
-      __syncthreads();
-      EORA_TRACE(5);
-      // t -> fp16 hi + lo in shared memory (two sources), rows padded like X
-      const int trow = p.r_pad + kXPad;
-      __half* ts = xs;
-      for (int row = 0; row < p.m; ++row) {
-        for (int j = threadIdx.x; j < p.r_pad; j += kThreads) {
-          float v = ld_cg(p.t_ws + (int64_t)row * p.r_pad + j);
-          __half hi = __float2half_rn(v);
-          __half lo = __float2half_rn(v - __half2float(hi));
-          ts[row * trow + j] = hi;
-          ts[(p.m + row) * trow + j] = lo;
-        }
-      }
-      __syncthreads();
-      // all reads of t by this CTA are done: the last consumer returns t_ws and the counters to zero
-      if (threadIdx.x == 0) {
-        __threadfence();
-        uint32_t c = atomicAdd(p.counters + CNT_T_CONSUMED, 1u);
-        s_flag = (c == (uint32_t)p.w.nt - 1) ? 1u : 0u;
-      }
-      __syncthreads();
-      if (s_flag) {
-        for (int i = threadIdx.x; i < p.m * p.r_pad; i += kThreads) p.t_ws[i] = 0.f;
-        if (threadIdx.x == 0) { p.counters[CNT_T_DONE] = 0; p.counters[CNT_T_CONSUMED] = 0; }
-      }
-      EORA_TRACE(6);
-      SliceView sb;
-      sb.wbuf = bbuf; sb.sc = bsc_s; sb.zz = bzz_s; sb.bars = bars + kChunks; sb.nq = nqb; sb.qt = p.qt_b; sb.cq = cqb;
-      sb.group_tiles = p.b.group / 64; sb.gofs = 0;
-      run_slice<ABF, MT, 2>(sb, warp, lane, ts, trow, p.m * trow, p.m, p.dev_status, acc);
-    }
-  }
-
-  EORA_TRACE(7);
-  // ---- sum the 8 warps
-#pragma unroll
-  for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-    for (int c = 0; c < 4; ++c) red[warp * (MT * 128) + (mt * 4 + c) * 32 + lane] = acc[mt][c];
-  __syncthreads();
-  EORA_TRACE(8);
-
-  // outputs of this unit: 16 rows x 8*MT tokens; element idx of the warp sums is
-  // (mt, c, lane) = (idx >> 7, (idx >> 5) & 3, idx & 31)
-  auto out_pos = [&](int idx, int& token, int& row) {
-    const int l = idx & 31, c = (idx >> 5) & 3, mt = idx >> 7;
-    token = mt * 8 + 2 * (l & 3) + (c & 1);
-    row = tile * 16 + (l >> 2) + 8 * (c >> 1);
-  };
-  auto warp_sum = [&](int idx) {
-    float v = 0.f;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) v += red[w * (MT * 128) + idx];
-    return v;
-  };
-
-  if (is_a) {
-    for (int idx = threadIdx.x; idx < MT * 128; idx += kThreads) {
-      int token, row;
-      out_pos(idx, token, row);
-      if (token < p.m) red_add(p.t_ws + (int64_t)token * p.r_pad + row, warp_sum(idx));
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) atomicAdd(p.counters + CNT_T_DONE, 1u);
-    EORA_TRACE(9);
-    return;
-  }
-  if (split == 1) {
-    for (int idx = threadIdx.x; idx < MT * 128; idx += kThreads) {
-      int token, row;
-      out_pos(idx, token, row);
-      if (token < p.m) store_y(p.y, p.y_dtype, (int64_t)token * p.d_out + row, warp_sum(idx));
-    }
-    EORA_TRACE(9);
-    return;
-  }
-  for (int idx = threadIdx.x; idx < MT * 128; idx += kThreads) {
-    int token, row;
-    out_pos(idx, token, row);
-    if (token < p.m) red_add(p.y_ws + (int64_t)token * p.d_out + row, warp_sum(idx));
-  }
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t c = atomicAdd(p.counters + CNT_TILE0 + tile, 1u);
-    s_flag = (c == (uint32_t)split - 1) ? 1u : 0u;
-  }
-  __syncthreads();
-  if (s_flag) {
-    __threadfence();
-    for (int idx = threadIdx.x; idx < MT * 128; idx += kThreads) {
-      int token, row;
-      out_pos(idx, token, row);
-      if (token < p.m) {
-        float* src = p.y_ws + (int64_t)token * p.d_out + row;
-        store_y(p.y, p.y_dtype, (int64_t)token * p.d_out + row, ld_cg(src));
-        *src = 0.f;
-      }
-    }
-    if (threadIdx.x == 0) p.counters[CNT_TILE0 + tile] = 0;
-  }
-  EORA_TRACE(9);
-}
-
-// ------------------------------------------------------------------------------------------ host
-struct Plan {
-  int a_units, a_split, w_split, smem;
-  int off_sc, off_zz, off_b, off_bsc, off_bzz, off_x, off_red;
-};
-
-inline int align_up_i(int v, int a) { return (v + a - 1) / a * a; }
-
-Plan make_plan(const Handle* h, int m) {
-  Plan pl = {};
-  const int slots = 3 * h->sm_count;
-  const int mt = m <= 8 ? 1 : m <= 16 ? 2 : m <= 32 ? 4 : 8;
-  const int max_slice_k_x = (kXSmemBudget / (2 * m)) & ~127;          // activations staged per CTA
-  auto max_slice_k = [&](const WMat& mat) {
-    int by_bytes = ((kUnitBytes / tile_bytes(mat.fmt)) * 64) & ~127;
-    return by_bytes < max_slice_k_x ? by_bytes : max_slice_k_x;
-  };
-  auto split_for = [&](const WMat& mat, int want) {
-    int qt = quantum_tiles(mat), nq = mat.kc / qt;
-    int msk = max_slice_k(mat);
-    int min_split = (mat.k_red + msk - 1) / msk;
-    int s = want > min_split ? want : min_split;
-    if (s > nq) s = nq;
-    if (s < 1) s = 1;
-    return s;
-  };
-  auto slice_len = [&](const WMat& mat, int split) {      // longest slice in reduction elements
-    int qt = quantum_tiles(mat), nq = mat.kc / qt, best = 0;
-    for (int s = 0; s < split; ++s) {
-      int l = (int)(((int64_t)nq * (s + 1) / split) - ((int64_t)nq * s / split)) * qt * 64;
-      if (l > best) best = l;
-    }
-    return best;
-  };
-  int want_w = (h->w.nt * 4 >= slots * 3) ? 1 : (slots + h->w.nt - 1) / h->w.nt;
-  pl.w_split = split_for(h->w, want_w);
-  const bool ab = h->cfg.rank > 0;
-  if (ab) {
-    // size A units like backbone units (in bytes streamed)
-    int64_t w_unit_bytes = wmat_q_bytes(h->w.fmt, 1, h->w.kc) / pl.w_split;
-    if (w_unit_bytes < 8192) w_unit_bytes = 8192;
-    int64_t a_tile_bytes = wmat_q_bytes(h->a.fmt, 1, h->a.kc);
-    pl.a_split = split_for(h->a, (int)((a_tile_bytes + w_unit_bytes - 1) / w_unit_bytes));
-    pl.a_units = h->a.nt * pl.a_split;
-  } else {
-    pl.a_split = 1;
-  }
-  int lw = slice_len(h->w, pl.w_split), la = ab ? slice_len(h->a, pl.a_split) : 0;
-  int wbytes = lw / 64 * tile_bytes(h->w.fmt);
-  if (ab && la / 64 * tile_bytes(h->a.fmt) > wbytes) wbytes = la / 64 * tile_bytes(h->a.fmt);
-  int max_k = lw > la ? lw : la;
-  int groups_w = lw / h->w.group + 2;
-  int groups_a = ab ? la / h->a.group + 2 : 0;
-  int groups = groups_w > groups_a ? groups_w : groups_a;
-  int off = align_up_i(wbytes, 128);
-  pl.off_sc = off; off += align_up_i(groups * 32, 128);
-  pl.off_zz = off; off += align_up_i(groups * 16, 128);
-  pl.off_b = off; off += ab ? align_up_i(h->b.kc * tile_bytes(h->b.fmt), 128) : 0;
-  pl.off_bsc = off; off += ab ? align_up_i((h->b.ng + 1) * 32, 128) : 0;
-  pl.off_bzz = off; off += ab ? align_up_i((h->b.ng + 1) * 16, 128) : 0;
-  pl.off_x = off;
-  int xb = m * (max_k + kXPad) * 2;
-  int tb = ab ? 2 * m * (h->r_pad + kXPad) * 2 : 0;
-  off += align_up_i(xb > tb ? xb : tb, 128);
-  pl.off_red = off; off += kWarps * mt * 128 * 4;
-  pl.smem = off;
-  return pl;
+  bool ok = run_segment<ABF, false, OUT_T>(p, r, a0, an, p.a_nt, blob_a, p.a_per_copy, p.a_sz2, lane);
+  if (ok) ok = run_segment<WF, false, OUT_Y>(p, r, w0, wn, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+  if (tr && lane == 0) tr[2] = globaltimer_ns();
+  if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
+  if (tr && lane == 0) tr[3] = globaltimer_ns();
 }
 
 template <auto KERNEL>
 cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const DecodeArgs& args) {
   static bool attr_set = false;   // one per kernel (KERNEL is a template argument)
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   return cudaLaunchKernelEx(&cfg, KERNEL, args);
 }
 
-template <int WF, int ABF>
-cudaError_t launch_mt(const DecodeArgs& args, int mt, int grid, int smem, cudaStream_t st) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  switch (mt) {
-    case 1: return launch_kernel<k_decode<WF, ABF, 1>>(cfg, args);
-    case 2: return launch_kernel<k_decode<WF, ABF, 2>>(cfg, args);
-    case 4: return launch_kernel<k_decode<WF, ABF, 4>>(cfg, args);
-    default: return launch_kernel<k_decode<WF, ABF, 8>>(cfg, args);
+template <int WF>
+cudaError_t launch_ab(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf) {
+  switch (abf) {
+    case FMT_F16: return launch_kernel<k_decode<WF, FMT_F16>>(cfg, args);
+    case FMT_Q4: return launch_kernel<k_decode<WF, FMT_Q4>>(cfg, args);
+    case FMT_Q8: return launch_kernel<k_decode<WF, FMT_Q8>>(cfg, args);
+    default: return launch_kernel<k_decode<WF, FMT_NONE>>(cfg, args);
   }
 }
 
-template <int WF>
-cudaError_t launch_ab(const DecodeArgs& args, int abf, int mt, int grid, int smem, cudaStream_t st) {
-  switch (abf) {
-    case FMT_F16: return launch_mt<WF, FMT_F16>(args, mt, grid, smem, st);
-    case FMT_Q4: return launch_mt<WF, FMT_Q4>(args, mt, grid, smem, st);
-    case FMT_Q8: return launch_mt<WF, FMT_Q8>(args, mt, grid, smem, st);
-    default: return launch_mt<WF, FMT_NONE>(args, mt, grid, smem, st);
+// Relative cost of one blob (time a warp spends on it); only the ratios matter.
+double blob_cost(int fmt, bool hilo) {
+  switch (fmt) {
+    case FMT_Q3: return 1.00;
+    case FMT_Q4: return 1.05;
+    case FMT_Q8: return 1.40;
+    case FMT_F16: return hilo ? 1.30 : 1.10;
+    default: return 0.0;
   }
+}
+
+Share make_share(uint32_t total, uint32_t n) {
+  Share s;
+  s.per = n ? total / n : 0;
+  s.rem = n ? total % n : 0;
+  return s;
+}
+
+uint32_t blobs_per_copy(const WMat& m) {
+  int n = kSlotBytes / m.blob;
+  return (uint32_t)(n < 1 ? 1 : n);
 }
 
 }  // namespace
@@ -482,42 +434,86 @@ cudaError_t launch_ab(const DecodeArgs& args, int abf, int mt, int grid, int sme
 bool decode_supported(const Handle* h, int m) {
   if (m < 1 || m > 64) return false;
   if (h->w.fmt != FMT_Q4 && h->w.fmt != FMT_Q3) return false;
-  if (h->w.group % 64) return false;
-  Plan pl = make_plan(h, m);
-  return pl.smem <= kMaxSmem;
+  if (h->w.blob > kSlotBytes) return false;
+  if (h->cfg.rank > 0 && (h->a.blob > kSlotBytes || h->b.blob > kSlotBytes)) return false;
+  return true;
 }
 
-void decode_make_plan(Handle* h) { h->plan = DecodePlan(); }
+int decode_launch_count(const Handle*, int m) { return (m + 7) / 8; }
 
-int decode_launch_count(const Handle*, int) { return 1; }
-
-int decode_grid(const Handle* h, int m) {
-  if (decode_stream_supported(h, m)) return decode_stream_grid(h, m);
-  Plan pl = make_plan(h, m);
-  return pl.a_units + h->w.nt * pl.w_split;
-}
+int decode_grid(const Handle* h, int) { return h->sm_count * kCtasPerSm; }
 
 cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st) {
-  if (decode_stream_supported(h, m)) return launch_decode_stream(h, x, m, y, st);
-  Plan pl = make_plan(h, m);
-  DecodeArgs a;
-  a.w = h->w; a.a = h->a; a.b = h->b;
-  a.x = x; a.y = y;
-  a.t_ws = h->t_ws; a.y_ws = h->y_ws; a.counters = h->counters; a.dev_status = h->dev_status;
-  a.m = m; a.d_in = h->cfg.d_in; a.d_out = h->cfg.d_out; a.r_pad = h->r_pad;
+  const bool ab = h->cfg.rank > 0;
+  DecodeArgs a = {};
+  a.w_q = h->w.q; a.w_nt = h->w.nt; a.w_sz2 = h->w.sz2; a.w_per_copy = blobs_per_copy(h->w);
+  const uint32_t w_blobs = (uint32_t)h->w.np * h->w.nt;
+  uint32_t b_blobs = 0;
+  if (ab) {
+    a.a_q = h->a.q; a.a_nt = h->a.nt; a.a_sz2 = h->a.sz2; a.a_per_copy = blobs_per_copy(h->a);
+    a.b_q = h->b.q; a.b_sz2 = h->b.sz2; a.b_per_copy = blobs_per_copy(h->b);
+    a.a_blobs = (uint32_t)h->a.np * h->a.nt;
+    b_blobs = (uint32_t)h->b.np * h->b.nt;
+  } else {
+    a.a_nt = 1; a.a_per_copy = 1; a.b_per_copy = 1;
+  }
+  const int grid = decode_grid(h, m);
+  const uint32_t nw = (uint32_t)grid * kWarps;
+  // Deal the blobs so that every warp gets the same estimated time: A owners take A plus a part of W,
+  // the others the rest of W plus B.
+  if (ab) {
+    const double ca = a.a_blobs * blob_cost(h->a.fmt, false), cb = b_blobs * blob_cost(h->b.fmt, true);
+    const double cw1 = blob_cost(h->w.fmt, false), cw = w_blobs * cw1;
+    const double tau = (ca + cw + cb) / nw;
+    uint32_t lo = (uint32_t)(ca / tau) + 1, hi = nw - ((uint32_t)(cb / tau) + 1);
+    uint32_t n_a = nw / 2;
+    if (n_a < lo) n_a = lo;
+    if (n_a > hi) n_a = hi;
+    if (n_a < 1) n_a = 1;
+    if (n_a > nw - 1) n_a = nw - 1;
+    double w1 = (n_a * tau - ca) / cw1;
+    if (w1 < 0) w1 = 0;
+    if (w1 > w_blobs) w1 = w_blobs;
+    a.n_a = n_a;
+    a.w1_blobs = (uint32_t)w1;
+    a.sh_a = make_share(a.a_blobs, n_a);
+    a.sh_w1 = make_share(a.w1_blobs, n_a);
+    a.sh_w2 = make_share(w_blobs - a.w1_blobs, nw - n_a);
+    a.sh_b = make_share(b_blobs, nw - n_a);
+  } else {
+    a.n_a = nw;
+    a.w1_blobs = w_blobs;
+    a.sh_a = make_share(0, nw);
+    a.sh_w1 = make_share(w_blobs, nw);
+    a.sh_w2 = make_share(0, 0);
+    a.sh_b = make_share(0, 0);
+  }
+  a.tile_target = (uint32_t)h->w.np + (ab ? (uint32_t)h->b.np : 0u);
+  a.d_t = h->d_t; a.y_ws = h->y_ws; a.counters = h->counters; a.dev_status = h->dev_status;
+  a.d_in = h->cfg.d_in; a.d_out = h->cfg.d_out; a.r_pad = h->r_pad > 0 ? h->r_pad : 128; a.n_pad = h->w.n_rows;
   a.x_dtype = h->cfg.x_dtype; a.y_dtype = h->cfg.y_dtype;
-  a.a_units = pl.a_units; a.a_split = pl.a_split; a.w_split = pl.w_split;
-  a.qt_w = quantum_tiles(h->w);
-  a.qt_a = h->cfg.rank > 0 ? quantum_tiles(h->a) : 1;
-  a.qt_b = h->cfg.rank > 0 ? quantum_tiles(h->b) : 1;
-  a.off_sc = pl.off_sc; a.off_zz = pl.off_zz; a.off_b = pl.off_b; a.off_bsc = pl.off_bsc; a.off_bzz = pl.off_bzz;
-  a.off_x = pl.off_x; a.off_red = pl.off_red;
   a.trace = reinterpret_cast<unsigned long long*>(h->trace);
-  int grid = pl.a_units + h->w.nt * pl.w_split;
-  int mt = m <= 8 ? 1 : m <= 16 ? 2 : m <= 32 ? 4 : 8;
-  int abf = h->cfg.rank > 0 ? h->a.fmt : FMT_NONE;
-  if (h->w.fmt == FMT_Q4) return launch_ab<FMT_Q4>(a, abf, mt, grid, pl.smem, st);
-  return launch_ab<FMT_Q3>(a, abf, mt, grid, pl.smem, st);
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const int abf = ab ? h->a.fmt : FMT_NONE;
+  const size_t ybytes = h->cfg.y_dtype == EORA_Y_F32 ? 4 : 2;
+  for (int m0 = 0; m0 < m; m0 += 8) {             // eight tokens per pass (the n8 side of the mma)
+    a.m = m - m0 < 8 ? m - m0 : 8;
+    a.x = reinterpret_cast<const uint8_t*>(x) + (size_t)m0 * h->cfg.d_in * 2;
+    a.y = reinterpret_cast<uint8_t*>(y) + (size_t)m0 * h->cfg.d_out * ybytes;
+    cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf) : launch_ab<FMT_Q3>(cfg, a, abf);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace eora

@@ -6,8 +6,6 @@
 namespace eora {
 namespace dec {
 
-enum { CNT_T_DONE = 0, CNT_T_CONSUMED = 1, CNT_TILE0 = 2 };
-
 // ------------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -212,12 +210,6 @@ __device__ __forceinline__ void store_y(void* y, int dtype, int64_t i, float v) 
   if (dtype == EORA_Y_F16) reinterpret_cast<__half*>(y)[i] = __float2half_rn(v);
   else if (dtype == EORA_Y_BF16) reinterpret_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
   else reinterpret_cast<float*>(y)[i] = v;
-}
-
-// tiles per quantum: the unit of work that shares one scale / zero-point (at most 128 elements)
-inline int quantum_tiles(const WMat& m) {
-  if (m.fmt == FMT_F16) return 1;
-  return (m.group % 128 == 0) ? 2 : 1;
 }
 
 }  // namespace dec

@@ -28,22 +28,20 @@ struct Carve {
 void wmat_shape(WMat& m, int fmt, int rows, int k_red, int group) {
   m.fmt = fmt;
   m.n_rows = (int)align_up(rows, 16);
-  m.k_red = (int)align_up(k_red, 64);
+  m.k_red = (int)align_up(k_red, 128);
   m.group = group > 0 ? group : m.k_red;
   if (m.group > m.k_red) m.group = m.k_red;
   m.nt = m.n_rows / 16;
   m.kc = m.k_red / 64;
-  m.ng = m.k_red / m.group;
-  m.q = nullptr; m.sc = nullptr; m.zz = nullptr;
+  m.np = m.k_red / 128;
+  m.sz2 = (m.group % 128) ? 1 : 0;
+  m.blob = blob_bytes(fmt, m.sz2);
+  m.q = nullptr;
 }
 
 void wmat_carve(WMat& m, Carve& c) {
   if (m.fmt == FMT_NONE) return;
-  m.q = c.take<uint8_t>(wmat_q_bytes(m.fmt, m.nt, m.kc));
-  if (m.fmt == FMT_Q4 || m.fmt == FMT_Q3 || m.fmt == FMT_Q8) {
-    m.sc = c.take<uint32_t>((int64_t)m.nt * m.ng * 8 * 4);
-    m.zz = c.take<uint16_t>((int64_t)m.nt * m.ng * 8 * 2);
-  }
+  m.q = c.take<uint8_t>(wmat_q_bytes(m));
 }
 
 int check_config(const eora_linear_config& c) {
@@ -131,13 +129,13 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
   if (cudaGetDevice(&h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
 
-  h->r_pad = (int)align_up(c.rank, 64);
+  h->r_pad = (int)align_up(c.rank, 128);
   int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : FMT_Q8;
   wmat_shape(h->w, quant_w ? (c.w_bits == 4 ? FMT_Q4 : FMT_Q3) : FMT_SP24, c.d_out, c.d_in, quant_w ? c.w_group : 0);
   if (c.rank > 0) {
     int ga = c.ab_format == EORA_AB_Q4 ? c.ab_group : 0;
     int gb = c.ab_format == EORA_AB_Q4 ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 0;
-    wmat_shape(h->a, ab_fmt, h->r_pad, c.d_in, ga);
+    wmat_shape(h->a, ab_fmt, c.rank, c.d_in, ga);
     wmat_shape(h->b, ab_fmt, c.d_out, h->r_pad, gb);
   } else {
     wmat_shape(h->a, FMT_NONE, 0, 0, 0);
@@ -153,16 +151,15 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
   wmat_carve(h->w, wc); wmat_carve(h->a, wc); wmat_carve(h->b, wc);
 
   // ---- scratch: one allocation, zero-initialised
-  decode_make_plan(h);
-  int m_dec = c.max_m < 64 ? c.max_m : 64;
-  int64_t n_counters = h->w.nt + h->a.nt + 64;
+  const int64_t rp = h->r_pad > 0 ? h->r_pad : 128;
   for (int pass = 0; pass < 2; ++pass) {
     Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
-    h->t_ws = sc.take<float>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 4);
-    h->y_ws = sc.take<float>((int64_t)m_dec * c.d_out * 4);
-    h->t_gen = sc.take<float>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 4);
-    h->t16 = sc.take<__half>((int64_t)c.max_m * (h->r_pad > 0 ? h->r_pad : 64) * 2);
-    h->counters = sc.take<uint32_t>(n_counters * 4);
+    h->t_ws = sc.take<float>((int64_t)c.max_m * rp * 4);
+    h->t_gen = sc.take<float>((int64_t)c.max_m * rp * 4);
+    h->t16 = sc.take<__half>((int64_t)c.max_m * rp * 2);
+    h->d_t = sc.take<float>(8 * rp * 4);
+    h->y_ws = sc.take<float>((int64_t)8 * h->w.n_rows * 4);
+    h->counters = sc.take<uint32_t>((int64_t)(h->w.nt + 2) * 4);
     h->dev_status = sc.take<int>(256);
     h->x_stage = sc.take<void>((int64_t)c.max_m * c.d_in * 2);
     h->y_stage = sc.take<void>((int64_t)c.max_m * c.d_out * y_elem_bytes(c.y_dtype));

@@ -21,11 +21,17 @@ namespace eora {
 //     part 0 = (n_a, ka)   part 1 = (n_b, ka)   part 2 = (n_a, kb)   part 3 = (n_b, kb)
 // of 8 consecutive reduction elements each.  Eight consecutive elements of one row are also one
 // 16-byte chunk of a K-major tensor-core operand, so the same layout feeds the prefill kernel.
-// Tiles of one row-tile are contiguous along the reduction axis: index = tile * kc + c.
 //
-// Every tile is one contiguous blob of tile_bytes(fmt) bytes, so the tiles a CTA needs are one
-// contiguous byte range that a single bulk copy can bring into shared memory.
-// Per format, the payload of lane L inside the blob of tile (tile, c):
+// Blobs.  Two tiles that are neighbours along the reduction axis (k-tiles 2p and 2p+1, "pair" p: 128
+// reduction elements) plus the scales and zero-points they need form one contiguous blob, and the
+// blobs are ordered pair-major:  blob (p, tile) sits at  q + (p * nt + tile) * blob.  A run of consecutive
+// blobs is therefore a set of row tiles that all multiply the same 128 activations, and it is one
+// contiguous byte range that a single bulk copy brings into shared memory, scales included.
+//   blob = [tile 2p][tile 2p+1][sz entry 0][sz entry 1 (only if sz2)]
+//   sz entry (48 B) = 8 x half2 scales (s[n_a], s[n_b]) indexed by g, then 8 x u8x2 zero-points (z[n_a] | z[n_b] << 8).
+//   If the group size is a multiple of 128 the pair has one entry (its group), otherwise (64, 192, ...)
+//   one per tile (sz2).  Unquantised formats have no entries.
+// Per format, the payload of lane L inside the tile:
 //   Q4  : 512 B: one uint4 per lane; word `part` holds the 8 codes of that part, element e in nibble
 //         (e & 1) * 4 + (e >> 1)   (so that (w & 0x000f000f) is the pair (e0, e1), ...).
 //   Q3  : 384 B: three words; w0, w1 as a uint2 per lane in bytes [0, 256), w2 as one word per lane
@@ -40,35 +46,43 @@ namespace eora {
 //   SP24: 1152 B: values in two planes of one uint4 per lane (plane = part/2), the half (part%2) holds
 //         the 4 kept fp16 values of the part's two quads; then one word per lane in bytes [1024, 1152),
 //         byte `part` = nibble(quad0) | nibble(quad1)<<4.
-// Scales / zero-points (Q4, Q3, Q8): sc[(tile*G + grp)*8 + g] = half2(s[n_a], s[n_b]),
-//   zz[(tile*G + grp)*8 + g] = z[n_a] | z[n_b] << 8, with grp = k / group.
 // ---------------------------------------------------------------------------------------------
 enum Fmt : int { FMT_NONE = 0, FMT_Q4 = 1, FMT_Q3 = 2, FMT_Q8 = 3, FMT_F16 = 4, FMT_SP24 = 5 };
 
 struct WMat {
   int fmt;
   int n_rows;      // padded to a multiple of 16
-  int k_red;       // padded to a multiple of 64
+  int k_red;       // padded to a multiple of 128
   int group;       // quantisation group along the reduction axis (multiple of 64)
   int nt;          // n_rows / 16
   int kc;          // k_red / 64
-  int ng;          // k_red / group
-  const uint8_t* q;      // tile blobs
-  const uint32_t* sc;    // half2 scales
-  const uint16_t* zz;    // u8x2 zero-points
+  int np;          // k_red / 128: pairs of k-tiles
+  int sz2;         // 1: one scale entry per tile, 0: one per pair
+  int blob;        // bytes of one blob
+  const uint8_t* q;      // blobs
 };
 
-__host__ __device__ inline int tile_bytes(int fmt) {
-  switch (fmt) {
-    case FMT_Q4: return 512;
-    case FMT_Q3: return 384;
-    case FMT_Q8: return 1024;
-    case FMT_F16: return 2048;
-    case FMT_SP24: return 1152;
-    default: return 0;
-  }
+constexpr int kSzEntryBytes = 48;
+
+__host__ __device__ constexpr int tile_bytes(int fmt) {
+  return fmt == FMT_Q4 ? 512 : fmt == FMT_Q3 ? 384 : fmt == FMT_Q8 ? 1024 : fmt == FMT_F16 ? 2048 : fmt == FMT_SP24 ? 1152 : 0;
 }
-__host__ __device__ inline int64_t wmat_q_bytes(int fmt, int nt, int kc) { return (int64_t)nt * kc * tile_bytes(fmt); }
+__host__ __device__ constexpr bool fmt_quantised(int fmt) { return fmt == FMT_Q4 || fmt == FMT_Q3 || fmt == FMT_Q8; }
+__host__ __device__ constexpr int blob_bytes(int fmt, int sz2) {
+  return 2 * tile_bytes(fmt) + (fmt_quantised(fmt) ? (sz2 ? 2 : 1) * kSzEntryBytes : 0);
+}
+__host__ __device__ inline int64_t wmat_q_bytes(const WMat& w) { return (int64_t)w.np * w.nt * w.blob; }
+
+// tile (row tile `tile`, k-tile c) and the scale entry that covers it
+__host__ __device__ inline const uint8_t* wmat_blob(const WMat& w, int tile, int pair) {
+  return w.q + ((int64_t)pair * w.nt + tile) * w.blob;
+}
+__host__ __device__ inline const uint8_t* wmat_tile(const WMat& w, int tile, int c) {
+  return wmat_blob(w, tile, c >> 1) + (c & 1) * tile_bytes(w.fmt);
+}
+__host__ __device__ inline const uint8_t* wmat_sz(const WMat& w, int tile, int c) {
+  return wmat_blob(w, tile, c >> 1) + 2 * tile_bytes(w.fmt) + (w.sz2 ? (c & 1) * kSzEntryBytes : 0);
+}
 
 // nibble / byte positions (shared by the repack kernels and the accessors below)
 __host__ __device__ inline int q4_nibble(int e) { return (e & 1) * 4 + (e >> 1); }
@@ -79,7 +93,7 @@ __device__ inline int wmat_code(const WMat& w, int k, int n) {
   int tile = n >> 4, g = n & 7, half = (n >> 3) & 1;
   int c = k >> 6, blk = (k >> 5) & 1, t = (k >> 3) & 3, e = k & 7;
   int lane = g * 4 + t, part = blk * 2 + half;
-  const uint32_t* blob = reinterpret_cast<const uint32_t*>(w.q + ((int64_t)tile * w.kc + c) * tile_bytes(w.fmt));
+  const uint32_t* blob = reinterpret_cast<const uint32_t*>(wmat_tile(w, tile, c));
   if (w.fmt == FMT_Q4) {
     return (blob[lane * 4 + part] >> (4 * q4_nibble(e))) & 15;
   } else if (w.fmt == FMT_Q3) {
@@ -99,16 +113,16 @@ __device__ inline float wmat_elem(const WMat& w, int k, int n) {
   int tile = n >> 4, g = n & 7, half = (n >> 3) & 1;
   if (w.fmt == FMT_Q4 || w.fmt == FMT_Q3 || w.fmt == FMT_Q8) {
     int q = wmat_code(w, k, n);
-    int64_t si = ((int64_t)tile * w.ng + k / w.group) * 8 + g;
-    uint32_t s2 = w.sc[si];
-    uint32_t z2 = w.zz[si];
+    const uint8_t* sz = wmat_sz(w, tile, k >> 6);
+    uint32_t s2 = reinterpret_cast<const uint32_t*>(sz)[g];
+    uint32_t z2 = reinterpret_cast<const uint16_t*>(sz + 32)[g];
     float s = __half2float(__ushort_as_half((unsigned short)(half ? (s2 >> 16) : (s2 & 0xffff))));
     int z = half ? (int)(z2 >> 8) : (int)(z2 & 255);
     return (float)(q - z) * s;
   }
   int c = k >> 6, blk = (k >> 5) & 1, t = (k >> 3) & 3, e = k & 7;
   int lane = g * 4 + t, part = blk * 2 + half;
-  const uint8_t* blob = w.q + ((int64_t)tile * w.kc + c) * tile_bytes(w.fmt);
+  const uint8_t* blob = wmat_tile(w, tile, c);
   if (w.fmt == FMT_F16) {
     const __half* p = reinterpret_cast<const __half*>(blob) + (part * 32 + lane) * 8;
     return __half2float(p[e]);
@@ -127,33 +141,27 @@ __device__ inline float wmat_elem(const WMat& w, int k, int n) {
 // ---------------------------------------------------------------------------------------------
 // Handle
 // ---------------------------------------------------------------------------------------------
-struct DecodePlan {      // launch shape of the decode kernel for this layer
-  int a_split;           // A units: a.nt row-tiles x a_split reduction slices
-  int w_split;           // backbone units: w.nt row-tiles x w_split reduction slices
-  int a_units, w_units;
-};
-
 struct Handle {
   eora_linear_config cfg;
   int device;
-  int r_pad;             // rank padded to a multiple of 64
-  WMat w, a, b;          // b: rows = d_out, reduction = r_pad
+  int r_pad;             // rank padded to a multiple of 128 (reduction length of B, row stride of t)
+  WMat w, a, b;          // a: rows = rank (padded to 16); b: rows = d_out, reduction = r_pad
   void* weight_mem;      // one allocation holding all re-tiled payloads
   int64_t weight_bytes;
   void* scratch_mem;     // one allocation: t, split-K sums, counters, staging
   int64_t scratch_bytes;
-  float* t_ws;           // [max_m][r_pad] fp32 sums of the fast kernels; zero between calls
+  float* t_ws;           // [max_m][r_pad] fp32 split-K sums of t (prefill); zero between calls
   float* t_gen;          // [max_m][r_pad] fp32, simple kernels only
-  float* y_ws;           // [min(max_m,64)][d_out] fp32 split-K sums (decode)
   __half* t16;           // [max_m][r_pad] fp16 (prefill)
-  uint32_t* counters;    // see decode.cu
+  float* d_t;            // [8][r_pad] fp32 sums of t (decode); zero between calls
+  float* y_ws;           // [8][d_out] fp32 sums of y (decode); zero between calls
+  uint32_t* counters;    // decode: [0] blobs of A done, [1] row tiles finished, [2 + tile] blobs of that row tile done
   int* dev_status;       // latched device status
   void* x_stage;         // [max_m][d_in] staging for forward_host
   void* y_stage;         // [max_m][d_out]
-  DecodePlan plan;
   int sm_count;
   void* prefill_state;   // owned by prefill.cu (tensor maps), may be NULL
-  void* trace;           // optional caller-owned timestamp buffer (decode kernel), may be NULL
+  void* trace;           // optional caller-owned timestamp buffer, may be NULL
 };
 
 // kernels / launchers implemented in the other translation units ------------------------------
@@ -169,13 +177,9 @@ cudaError_t launch_generic_forward(const Handle* h, const void* x, int m, void* 
 int generic_launch_count(const Handle* h);
 
 bool decode_supported(const Handle* h, int m);
-void decode_make_plan(Handle* h);
 cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
 int decode_launch_count(const Handle* h, int m);
 int decode_grid(const Handle* h, int m);
-bool decode_stream_supported(const Handle* h, int m);
-int decode_stream_grid(const Handle* h, int m);
-cudaError_t launch_decode_stream(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
 
 bool prefill_supported(const Handle* h, int m);
 cudaError_t prefill_init(Handle* h);

@@ -23,7 +23,8 @@ __global__ void k_generic_t(WMat a, const void* x, int x_dtype, int m, int d_in,
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     int j = (int)(idx % r_pad), mm = (int)(idx / r_pad);
     float acc = 0.f;
-    for (int k = 0; k < d_in; ++k) acc = fmaf(load_x(x, x_dtype, (int64_t)mm * d_in + k), wmat_elem(a, k, j), acc);
+    if (j < a.n_rows)
+      for (int k = 0; k < d_in; ++k) acc = fmaf(load_x(x, x_dtype, (int64_t)mm * d_in + k), wmat_elem(a, k, j), acc);
     t[idx] = acc;
   }
 }

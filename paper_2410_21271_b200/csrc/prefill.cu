@@ -243,11 +243,12 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
     uint32_t scq[PF], zzq[PF];
     auto issue = [&](int kb, int slot) {
       if (!active || kb >= kb_hi) return;
-      load_packed<FMT>(pk[slot], mat.q + ((int64_t)rt * mat.kc + kb) * tb, lane);
+      const uint8_t* blob = mat.q + ((int64_t)(kb >> 1) * mat.nt + rt) * mat.blob;
+      load_packed<FMT>(pk[slot], blob + (kb & 1) * tb, lane);
       if constexpr (quant) {
-        const int64_t si = ((int64_t)rt * mat.ng + kb / gt) * 8 + g;
-        scq[slot] = __ldg(mat.sc + si);
-        zzq[slot] = __ldg(mat.zz + si);
+        const uint8_t* sz = blob + 2 * tb + (mat.sz2 ? (kb & 1) * kSzEntryBytes : 0);
+        scq[slot] = __ldg(reinterpret_cast<const uint32_t*>(sz) + g);
+        zzq[slot] = __ldg(reinterpret_cast<const uint16_t*>(sz + 32) + g);
       }
     };
 #pragma unroll

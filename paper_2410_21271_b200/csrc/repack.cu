@@ -54,7 +54,7 @@ __global__ void k_repack_q4(WMat d, const uint32_t* codes, const uint32_t* zeros
         w |= padded_code(codes, zeros, 4, k0 + e, n, rows_src, k_src, d.group, ldz) << (4 * q4_nibble(e));
       out[part] = w;
     }
-    reinterpret_cast<uint4*>(const_cast<uint8_t*>(d.q))[idx] = make_uint4(out[0], out[1], out[2], out[3]);
+    reinterpret_cast<uint4*>(const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c)))[p.lane] = make_uint4(out[0], out[1], out[2], out[3]);
   }
 }
 
@@ -76,7 +76,7 @@ __global__ void k_repack_q3(WMat d, const uint32_t* codes, const uint32_t* zeros
         }
       }
     }
-    uint32_t* blob = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(d.q) + (idx >> 5) * 384);
+    uint32_t* blob = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c)));
     blob[p.lane * 2] = wd[0];
     blob[p.lane * 2 + 1] = wd[1];
     blob[64 + p.lane] = wd[2];
@@ -87,7 +87,7 @@ __global__ void k_repack_q8(WMat d, const uint8_t* codes, const uint8_t* zeros, 
   int64_t total = (int64_t)d.nt * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
-    int64_t ti = idx >> 5;
+    uint8_t* tb = const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c));
     for (int part = 0; part < 4; ++part) {
       int n = p.tile * 16 + p.g + 8 * (part & 1);
       int k0 = p.c * 64 + (part >> 1) * 32 + 8 * p.t;
@@ -97,7 +97,7 @@ __global__ void k_repack_q8(WMat d, const uint8_t* codes, const uint8_t* zeros, 
         if (n < rows_src) q = (k0 + e < k_src) ? codes[(int64_t)(k0 + e) * rows_src + n] : zeros[n];
         w2[e >> 2] |= q << (8 * q8_byte(e & 3));
       }
-      uint32_t* dst = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(d.q)) + ((ti * 2 + (part >> 1)) * 32 + p.lane) * 4;
+      uint32_t* dst = reinterpret_cast<uint32_t*>(tb) + ((part >> 1) * 32 + p.lane) * 4;
       dst[2 * (part & 1)] = w2[0];
       dst[2 * (part & 1) + 1] = w2[1];
     }
@@ -109,11 +109,11 @@ __global__ void k_repack_f16(WMat d, const __half* src, int rows_src, int k_src)
   int64_t total = (int64_t)d.nt * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
-    int64_t ti = idx >> 5;
+    uint8_t* tb = const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c));
     for (int part = 0; part < 4; ++part) {
       int n = p.tile * 16 + p.g + 8 * (part & 1);
       int k0 = p.c * 64 + (part >> 1) * 32 + 8 * p.t;
-      __half* dst = reinterpret_cast<__half*>(const_cast<uint8_t*>(d.q)) + ((ti * 4 + part) * 32 + p.lane) * 8;
+      __half* dst = reinterpret_cast<__half*>(tb) + (part * 32 + p.lane) * 8;
       for (int e = 0; e < 8; ++e) {
         int k = k0 + e;
         dst[e] = (n < rows_src && k < k_src) ? src[(int64_t)k * rows_src + n] : __float2half(0.f);
@@ -126,13 +126,13 @@ __global__ void k_repack_sp24(WMat d, const __half* values, const uint32_t* meta
   int64_t total = (int64_t)d.nt * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
-    int64_t ti = idx >> 5;
+    uint8_t* tb = const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c));
     uint32_t m = 0;
     for (int part = 0; part < 4; ++part) {
       int n = p.tile * 16 + p.g + 8 * (part & 1);
       int k0 = p.c * 64 + (part >> 1) * 32 + 8 * p.t;
       int j0 = k0 >> 2;   // first of the part's two quads
-      __half* dst = reinterpret_cast<__half*>(const_cast<uint8_t*>(d.q) + ti * 1152) + ((part >> 1) * 32 + p.lane) * 8 + 4 * (part & 1);
+      __half* dst = reinterpret_cast<__half*>(tb) + ((part >> 1) * 32 + p.lane) * 8 + 4 * (part & 1);
       uint32_t mb = 0x44;  // positions (0,1) with zero values outside the source
       if (n < rows_src && k0 < k_src) {
         for (int i = 0; i < 4; ++i) dst[i] = values[(int64_t)n * (k_src / 2) + 2 * j0 + i];
@@ -142,16 +142,19 @@ __global__ void k_repack_sp24(WMat d, const __half* values, const uint32_t* meta
       }
       m |= mb << (8 * part);
     }
-    reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(d.q) + ti * 1152 + 1024)[p.lane] = m;
+    reinterpret_cast<uint32_t*>(tb + 1024)[p.lane] = m;
   }
 }
 
-// scales fp16 [G][rows_src]; zeros packed stream.  One thread per (tile, grp, g).
+// Scale entries.  scales fp16 [G][rows_src]; zeros packed stream.  One thread per (k-tile c, row tile, g);
+// the entry of k-tile c is written once per blob (by the even tile when the pair shares one entry).
 __global__ void k_repack_sz(WMat d, const __half* scales, const uint32_t* zeros, int bits, int rows_src, int ldz,
                             int ng_src) {
-  int total = d.nt * d.ng * 8;
+  int total = d.nt * d.kc * 8;
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-    int g = idx & 7, grp = (idx >> 3) % d.ng, tile = (idx >> 3) / d.ng;
+    int g = idx & 7, c = (idx >> 3) % d.kc, tile = (idx >> 3) / d.kc;
+    if (!d.sz2 && (c & 1)) continue;
+    int grp = (c * 64) / d.group;
     uint32_t s2 = 0, z2 = 0;
     for (int half = 0; half < 2; ++half) {
       int n = tile * 16 + g + 8 * half;
@@ -164,15 +167,17 @@ __global__ void k_repack_sz(WMat d, const __half* scales, const uint32_t* zeros,
       s2 |= sb << (16 * half);
       z2 |= zb << (8 * half);
     }
-    const_cast<uint32_t*>(d.sc)[idx] = s2;
-    const_cast<uint16_t*>(d.zz)[idx] = (uint16_t)z2;
+    uint8_t* sz = const_cast<uint8_t*>(wmat_sz(d, tile, c));
+    reinterpret_cast<uint32_t*>(sz)[g] = s2;
+    reinterpret_cast<uint16_t*>(sz + 32)[g] = (uint16_t)z2;
   }
 }
 
 __global__ void k_repack_sz_q8(WMat d, const __half* scales, const uint8_t* zeros, int rows_src) {
-  int total = d.nt * 8;   // one group
+  int total = d.nt * d.kc * 8;   // one group: every pair carries a copy
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-    int g = idx & 7, tile = idx >> 3;
+    int g = idx & 7, c = (idx >> 3) % d.kc, tile = (idx >> 3) / d.kc;
+    if (!d.sz2 && (c & 1)) continue;
     uint32_t s2 = 0, z2 = 0;
     for (int half = 0; half < 2; ++half) {
       int n = tile * 16 + g + 8 * half;
@@ -181,8 +186,9 @@ __global__ void k_repack_sz_q8(WMat d, const __half* scales, const uint8_t* zero
         z2 |= (uint32_t)zeros[n] << (8 * half);
       }
     }
-    const_cast<uint32_t*>(d.sc)[idx] = s2;
-    const_cast<uint16_t*>(d.zz)[idx] = (uint16_t)z2;
+    uint8_t* sz = const_cast<uint8_t*>(wmat_sz(d, tile, c));
+    reinterpret_cast<uint32_t*>(sz)[g] = s2;
+    reinterpret_cast<uint16_t*>(sz + 32)[g] = (uint16_t)z2;
   }
 }
 
@@ -204,7 +210,7 @@ cudaError_t launch_repack_quant(const WMat& d, const void* codes, const void* sc
     k_repack_q4<<<grid_for(total, 256), 256, 0, st>>>(d, (const uint32_t*)codes, (const uint32_t*)zeros, rows_src, k_src, ldz);
   else
     k_repack_q3<<<grid_for(total, 256), 256, 0, st>>>(d, (const uint32_t*)codes, (const uint32_t*)zeros, rows_src, k_src, ldz);
-  k_repack_sz<<<grid_for((int64_t)d.nt * d.ng * 8, 256), 256, 0, st>>>(d, (const __half*)scales, (const uint32_t*)zeros, bits,
+  k_repack_sz<<<grid_for((int64_t)d.nt * d.kc * 8, 256), 256, 0, st>>>(d, (const __half*)scales, (const uint32_t*)zeros, bits,
                                                                      rows_src, ldz, ng_src);
   return cudaGetLastError();
 }
@@ -213,7 +219,7 @@ cudaError_t launch_repack_q8(const WMat& d, const void* codes, const void* scale
                              int k_src, cudaStream_t st) {
   int64_t total = (int64_t)d.nt * d.kc * 32;
   k_repack_q8<<<grid_for(total, 256), 256, 0, st>>>(d, (const uint8_t*)codes, (const uint8_t*)zeros, rows_src, k_src);
-  k_repack_sz_q8<<<grid_for((int64_t)d.nt * 8, 256), 256, 0, st>>>(d, (const __half*)scales, (const uint8_t*)zeros, rows_src);
+  k_repack_sz_q8<<<grid_for((int64_t)d.nt * d.kc * 8, 256), 256, 0, st>>>(d, (const __half*)scales, (const uint8_t*)zeros, rows_src);
   return cudaGetLastError();
 }
 
