@@ -26,6 +26,7 @@
 // griddepcontrol.wait, i.e. while the previous kernel in the stream is still draining; activations
 // and scratch are only touched after it.
 #include "decode_common.cuh"
+#include <cstdlib>   // PROBE
 
 namespace eora {
 namespace {
@@ -110,48 +111,6 @@ __device__ __forceinline__ void load_t_pair(uint32_t (&xh)[16], uint32_t (&xl)[1
       }
     }
   }
-}
-
-// One blob: 16 rows x 128 reduction elements times the activation fragments -> tot (this lane's four
-// entries of the 16 x 8 result: rows g / g + 8, tokens 2t / 2t + 1).
-template <int FMT, bool HILO>
-__device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint32_t sz2, const uint32_t (&xr)[16],
-                                             const uint32_t (&xl)[16], float (&tot)[4]) {
-  constexpr int tb = tile_bytes(FMT);
-  constexpr bool quant = fmt_quantised(FMT);
-  const int g = lane >> 2;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  tot[0] = tot[1] = tot[2] = tot[3] = 0.f;
-  ZC zc;
-  float s_a = 0.f, s_b = 0.f;
-#pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    if constexpr (quant) {
-      if (c == 0 || sz2) {
-        const uint8_t* sz = blob + 2 * tb + c * kSzEntryBytes;      // c != 0 only with two entries
-        const uint32_t s2 = reinterpret_cast<const uint32_t*>(sz)[g];
-        const uint32_t z2 = reinterpret_cast<const uint16_t*>(sz + 32)[g];
-        make_zc<FMT>(zc, z2);
-        s_a = __half2float(__ushort_as_half((unsigned short)(s2 & 0xffffu)));
-        s_b = __half2float(__ushort_as_half((unsigned short)(s2 >> 16)));
-      }
-    }
-    uint32_t a[4][4];
-    tile_frags<FMT>(blob + c * tb, lane, zc, a);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      mma16816(acc, a[i], xr[8 * c + 2 * i], xr[8 * c + 2 * i + 1]);
-      if constexpr (HILO) mma16816(acc, a[i], xl[8 * c + 2 * i], xl[8 * c + 2 * i + 1]);
-    }
-    if constexpr (quant) {
-      if (c == 1 || sz2) {
-        tot[0] = fmaf(acc[0], s_a, tot[0]); tot[1] = fmaf(acc[1], s_a, tot[1]);
-        tot[2] = fmaf(acc[2], s_b, tot[2]); tot[3] = fmaf(acc[3], s_b, tot[3]);
-        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
-      }
-    }
-  }
-  if constexpr (!quant) { tot[0] = acc[0]; tot[1] = acc[1]; tot[2] = acc[2]; tot[3] = acc[3]; }
 }
 
 // tot -> sums[token][ld] for rows 16 * tile + {g, g + 8}
@@ -368,9 +327,19 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
     bb0 = share_lo(p.sh_b, i); bn = share_n(p.sh_b, i);
   }
   const uint32_t blob_a = blob_bytes(ABF, p.a_sz2), blob_w = blob_bytes(WF, p.w_sz2), blob_b = blob_bytes(ABF, p.b_sz2);
-  r.ptr[0] = p.a_q + (size_t)a0 * blob_a; r.rem[0] = an; r.blob[0] = blob_a; r.per[0] = p.a_per_copy;
-  r.ptr[1] = p.w_q + (size_t)w0 * blob_w; r.rem[1] = wn; r.blob[1] = blob_w; r.per[1] = p.w_per_copy;
-  r.ptr[2] = p.b_q + (size_t)bb0 * blob_b; r.rem[2] = bn; r.blob[2] = blob_b; r.per[2] = p.b_per_copy;
+  // Order of the runs.  A owners: A, then W.  The others: the first copy's worth of W, then B, then the
+  // rest of W: by then t is complete, and the round trips of the B share (reading t back, its tickets)
+  // are hidden behind the other warps' W work instead of sitting at the end of the kernel.
+  const uint32_t wf = a_owner ? wn : (wn < p.w_per_copy ? wn : p.w_per_copy);
+  if (a_owner) {
+    r.ptr[0] = p.a_q + (size_t)a0 * blob_a; r.rem[0] = an; r.blob[0] = blob_a; r.per[0] = p.a_per_copy;
+    r.ptr[1] = p.w_q + (size_t)w0 * blob_w; r.rem[1] = wn; r.blob[1] = blob_w; r.per[1] = p.w_per_copy;
+    r.ptr[2] = p.w_q; r.rem[2] = 0; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
+  } else {
+    r.ptr[0] = p.w_q + (size_t)w0 * blob_w; r.rem[0] = wf; r.blob[0] = blob_w; r.per[0] = p.w_per_copy;
+    r.ptr[1] = p.b_q + (size_t)bb0 * blob_b; r.rem[1] = bn; r.blob[1] = blob_b; r.per[1] = p.b_per_copy;
+    r.ptr[2] = p.w_q + (size_t)(w0 + wf) * blob_w; r.rem[2] = wn - wf; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
+  }
 
 #pragma unroll
   for (int i = 0; i < kRing; ++i) ring_issue(r, i, lane);
@@ -378,10 +347,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tr && lane == 0) tr[1] = globaltimer_ns();
 
-  bool ok = run_segment<ABF, false, OUT_T>(p, r, a0, an, p.a_nt, blob_a, p.a_per_copy, p.a_sz2, lane);
-  if (ok) ok = run_segment<WF, false, OUT_Y>(p, r, w0, wn, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+  bool ok = true;
+  if (a_owner) ok = run_segment<ABF, false, OUT_T>(p, r, a0, an, p.a_nt, blob_a, p.a_per_copy, p.a_sz2, lane);
+  if (ok) ok = run_segment<WF, false, OUT_Y>(p, r, w0, wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
   if (tr && lane == 0) tr[2] = globaltimer_ns();
-  if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
+  if (!a_owner) {
+    if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
+    if (ok) ok = run_segment<WF, false, OUT_Y>(p, r, w0 + wf, wn - wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+  }
   if (tr && lane == 0) tr[3] = globaltimer_ns();
 }
 
@@ -464,14 +437,23 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y
   if (ab) {
     const double ca = a.a_blobs * blob_cost(h->a.fmt, false), cb = b_blobs * blob_cost(h->b.fmt, true);
     const double cw1 = blob_cost(h->w.fmt, false), cw = w_blobs * cw1;
+    // Besides the per-blob cost each kind of warp has a fixed one (in units of one backbone blob): the B
+    // share starts with a read-back of t and ends with its own round of tickets, which is latency that
+    // the warp cannot hide from itself.
+    double fixed_a = 0.5, fixed_b = 6.0;
+    if (const char* e = getenv("EORA_FB")) fixed_b = atof(e);   // PROBE
+    if (const char* e = getenv("EORA_FA")) fixed_a = atof(e);   // PROBE
     const double tau = (ca + cw + cb) / nw;
     uint32_t lo = (uint32_t)(ca / tau) + 1, hi = nw - ((uint32_t)(cb / tau) + 1);
     uint32_t n_a = nw / 2;
+    if (b_blobs < nw - n_a) n_a = nw - b_blobs;          // no B owner without a blob of B
     if (n_a < lo) n_a = lo;
     if (n_a > hi) n_a = hi;
     if (n_a < 1) n_a = 1;
     if (n_a > nw - 1) n_a = nw - 1;
-    double w1 = (n_a * tau - ca) / cw1;
+    const double n_b = nw - n_a;
+    // equal finishing time:  fixed_a + (ca + w1 cw1) / n_a  =  fixed_b + (cb + (W - w1) cw1) / n_b
+    double w1 = ((fixed_b - fixed_a) + cb / n_b + cw / n_b - ca / n_a) / (cw1 * (1.0 / n_a + 1.0 / n_b));
     if (w1 < 0) w1 = 0;
     if (w1 > w_blobs) w1 = w_blobs;
     a.n_a = n_a;

@@ -206,6 +206,49 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
 }
 
 
+// One blob: 16 rows x 128 reduction elements times the activation fragments -> tot (this lane's four
+// entries of the 16 x 8 result: rows g / g + 8, tokens 2t / 2t + 1).
+template <int FMT, bool HILO>
+__device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint32_t sz2, const uint32_t (&xr)[16],
+                                             const uint32_t (&xl)[16], float (&tot)[4]) {
+  constexpr int tb = tile_bytes(FMT);
+  constexpr bool quant = fmt_quantised(FMT);
+  const int g = lane >> 2;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  tot[0] = tot[1] = tot[2] = tot[3] = 0.f;
+  ZC zc;
+  float s_a = 0.f, s_b = 0.f;
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    if constexpr (quant) {
+      if (c == 0 || sz2) {
+        const uint8_t* sz = blob + 2 * tb + c * kSzEntryBytes;      // c != 0 only with two entries
+        const uint32_t s2 = reinterpret_cast<const uint32_t*>(sz)[g];
+        const uint32_t z2 = reinterpret_cast<const uint16_t*>(sz + 32)[g];
+        make_zc<FMT>(zc, z2);
+        s_a = __half2float(__ushort_as_half((unsigned short)(s2 & 0xffffu)));
+        s_b = __half2float(__ushort_as_half((unsigned short)(s2 >> 16)));
+      }
+    }
+    uint32_t a[4][4];
+    tile_frags<FMT>(blob + c * tb, lane, zc, a);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      mma16816(acc, a[i], xr[8 * c + 2 * i], xr[8 * c + 2 * i + 1]);
+      if constexpr (HILO) mma16816(acc, a[i], xl[8 * c + 2 * i], xl[8 * c + 2 * i + 1]);
+    }
+    if constexpr (quant) {
+      if (c == 1 || sz2) {
+        tot[0] = fmaf(acc[0], s_a, tot[0]); tot[1] = fmaf(acc[1], s_a, tot[1]);
+        tot[2] = fmaf(acc[2], s_b, tot[2]); tot[3] = fmaf(acc[3], s_b, tot[3]);
+        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+      }
+    }
+  }
+  if constexpr (!quant) { tot[0] = acc[0]; tot[1] = acc[1]; tot[2] = acc[2]; tot[3] = acc[3]; }
+}
+
+
 __device__ __forceinline__ void store_y(void* y, int dtype, int64_t i, float v) {
   if (dtype == EORA_Y_F16) reinterpret_cast<__half*>(y)[i] = __float2half_rn(v);
   else if (dtype == EORA_Y_BF16) reinterpret_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
