@@ -26,7 +26,6 @@
 // griddepcontrol.wait, i.e. while the previous kernel in the stream is still draining; activations
 // and scratch are only touched after it.
 #include "decode_common.cuh"
-#include <cstdlib>   // PROBE
 
 namespace eora {
 namespace {
@@ -243,9 +242,12 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
       }
       const uint32_t mask = __ballot_sync(0xffffffffu, done != 0);
       if (mask) {
-        if (done) finish_row_tile(p, my_tile);
+        // With an adapter the finished row tiles are counted (the count is taken before the tiles are
+        // written out, so that the two round trips overlap): the last one restores t and the counters.
         uint32_t last = 0;
-        if (lane == 0) last = atom_add_acq_rel(p.counters + CNT_TILES_DONE, (uint32_t)__popc(mask)) + __popc(mask) == p.w_nt ? 1u : 0u;
+        if (p.a_blobs && lane == 0)
+          last = atom_add_acq_rel(p.counters + CNT_TILES_DONE, (uint32_t)__popc(mask)) + __popc(mask) == p.w_nt ? 1u : 0u;
+        if (done) finish_row_tile(p, my_tile);
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {                               // the whole layer is done: nobody reads t any more
           for (int i = lane; i < 8 * p.r_pad / 4; i += 32) st_zero4(p.d_t + 4 * i);
@@ -440,9 +442,7 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y
     // Besides the per-blob cost each kind of warp has a fixed one (in units of one backbone blob): the B
     // share starts with a read-back of t and ends with its own round of tickets, which is latency that
     // the warp cannot hide from itself.
-    double fixed_a = 0.5, fixed_b = 6.0;
-    if (const char* e = getenv("EORA_FB")) fixed_b = atof(e);   // PROBE
-    if (const char* e = getenv("EORA_FA")) fixed_a = atof(e);   // PROBE
+    const double fixed_a = 0.5, fixed_b = 9.0;
     const double tau = (ca + cw + cb) / nw;
     uint32_t lo = (uint32_t)(ca / tau) + 1, hi = nw - ((uint32_t)(cb / tau) + 1);
     uint32_t n_a = nw / 2;
