@@ -238,6 +238,13 @@ def time_prefill(device: str, steps: int = 10, warmup: int = 3):
             "path": {0: "generic", 1: "decode", 2: "prefill"}[path], "l2": "flushed between iterations"}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of k_decode, mean over the seven layers of a block,
+# from the ncu capture summarised in profiles/k_decode_llama3-8b-w3g128-r128-M1.md (traffic grows with the
+# number of blocks in proportion, every block being the same seven launches).  Set to None when the kernel
+# changes until the capture is redone.
+DRAM_BYTES_PER_LAUNCH = 15.52e6
+
+
 def cpu_oracle_sample(blocks_sample: int = 1):
     """The CPU oracle, as it stands, on `blocks_sample` block(s) of the decode workload."""
     from oracle import eora_oracle as orc
@@ -300,6 +307,7 @@ def main():
     ap.add_argument("--blocks", type=int, default=gen.LLAMA3_8B_BLOCKS, help=argparse.SUPPRESS)
     ap.add_argument("--no-extras", action="store_true", help="skip the prefill / e2e / cpu legs")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--only-prefill", action="store_true", help="run the prefill leg alone (for profiling) and print its result")
     ap.add_argument("--single-stream", action="store_true", help="launch all layers of a block in stream order")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -338,6 +346,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(device))
         _DIST["on"] = True
 
+    if args.only_prefill:
+        if rank == 0:
+            print(json.dumps({"prefill": time_prefill(device)}))
+        return
     layers, xs, ys = build_layer_set(args.blocks, device)
     n_launch_step = sum(L.launches(M_DECODE) for _, _, _, L in layers)
     ms_local, clocks, graphed = time_decode(layers, xs, ys, args.steps, args.warmup, local_rank, not args.no_graph,
@@ -348,7 +360,8 @@ def main():
     achieved = bytes_step / (ms_local / 1e3) / 1e9
     roofline = {"bound": "hbm", "kernel": "k_decode", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
-                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": None,
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "traffic": DRAM_BYTES_PER_LAUNCH if args.blocks == gen.LLAMA3_8B_BLOCKS else None,
                 "bytes_per_launch": bytes_step / n_launch_step, "us_per_launch": ms_local * 1e3 / n_launch_step}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
