@@ -154,12 +154,15 @@ int eora_linear_dump(eora_linear_t h, int32_t what, void* out, void* stream);
 int eora_linear_last_device_status(eora_linear_t h);
 
 /*
- * Diagnostics of the decode kernel.  eora_linear_decode_grid: how many CTAs forward(m) launches
- * (0 if m is not served by the decode family).  eora_linear_set_trace: give the handle a device
- * buffer of 16 x uint64 per CTA (or NULL to switch tracing off); every decode forward then
- * records, per CTA, %globaltimer nanoseconds at fixed points of the kernel (0 start, 1 weight
- * copies issued, 2 dependency wait over, 3 X staged, 4 own slice done, 5 t available, 6 t staged,
- * 7 B extension done, 8 warps summed, 9 end).  The buffer is caller-owned.
+ * Diagnostics.  eora_linear_decode_grid: how many CTAs a decode forward(m) launches (0 if m is
+ * not served by the decode family); each CTA has four warps.  eora_linear_set_trace: give the
+ * handle a caller-owned device buffer (or NULL to switch tracing off).  A decode forward then
+ * records four %globaltimer values (nanoseconds) per warp, at uint64 index
+ * 4 * (4 * cta + warp) + k:  k = 0 kernel entry, 1 dependency wait over, 2 first share of the
+ * backbone done, 3 all work of the warp done; the buffer must hold 16 * grid values.  A prefill
+ * forward records, for CTA (0, 0) only, four clock64 values per 64-element k-block
+ * (producer / dequantisation / MMA issue / MMA complete) at index 4 * k_block + k; the buffer
+ * must hold 4 * (d_in + rank + 128) / 64 values.  Tracing costs time; leave it off in production.
  */
 int eora_linear_decode_grid(eora_linear_t h, int32_t m);
 int eora_linear_set_trace(eora_linear_t h, void* trace_buf);
