@@ -135,6 +135,15 @@ __device__ __forceinline__ void make_zc(ZC& zc, uint32_t zz) {
 
 constexpr uint32_t kMagic = 0x64006400u;   // fp16x2 (1024, 1024)
 
+// (a & mask) | c in ONE instruction.  Written as `(a & mask) | kMagic` with two immediates the compiler
+// emits two logic instructions (an instruction holds only one 32-bit immediate), and those run on the
+// half-rate integer pipe that bounds the decode kernel; with the constant in a register it is one LOP3.
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(c));
+  return d;
+}
+
 template <int FMT> constexpr bool is_quant() { return FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8; }
 
 // Build the A-operand registers of the four mma of one tile from its blob in shared memory.
@@ -148,8 +157,8 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
     for (int part = 0; part < 4; ++part) {
       const int hf = part & 1, blk = part >> 1;
       uint32_t lo = w[part], hi = w[part] >> 8;
-      uint32_t h0 = (lo & 0x000f000fu) | kMagic, h1 = (lo & 0x00f000f0u) | kMagic;
-      uint32_t h2 = (hi & 0x000f000fu) | kMagic, h3 = (hi & 0x00f000f0u) | kMagic;
+      uint32_t h0 = and_or(lo, 0x000f000fu, kMagic), h1 = and_or(lo, 0x00f000f0u, kMagic);
+      uint32_t h2 = and_or(hi, 0x000f000fu, kMagic), h3 = and_or(hi, 0x00f000f0u, kMagic);
       a[blk * 2 + 0][hf] = h2sub(h0, zc.c[hf][0]);
       a[blk * 2 + 0][hf + 2] = h2fma(h1, 0x2C002C00u, zc.c[hf][1]);   // * 1/16
       a[blk * 2 + 1][hf] = h2sub(h2, zc.c[hf][0]);
@@ -167,14 +176,14 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
       if (p < 15) {
         const int wi = p / 5, f = p % 5, ff = f >= 3 ? f - 3 : f;
         const uint32_t src = f >= 3 ? ws[wi] : w[wi];
-        const uint32_t h = (src & (0x00070007u << (3 * ff))) | kMagic;
+        const uint32_t h = and_or(src, 0x00070007u << (3 * ff), kMagic);
         if (ff == 0) v = h2sub(h, zc.c[hf][0]);
         else if (ff == 1) v = h2fma(h, 0x30003000u, zc.c[hf][1]);   // * 1/8
         else v = h2fma(h, 0x24002400u, zc.c[hf][2]);                // * 1/64
       } else {
-        uint32_t h = ((w[0] >> 15) & 0x00010001u) | kMagic;
-        h |= (w[1] >> 14) & 0x00020002u;
-        h |= (w[2] >> 13) & 0x00040004u;
+        uint32_t h = and_or(w[0] >> 15, 0x00010001u, kMagic);
+        h = and_or(w[1] >> 14, 0x00020002u, h);
+        h = and_or(w[2] >> 13, 0x00040004u, h);
         v = h2sub(h, zc.c[hf][0]);
       }
       a[blk * 2 + (j >> 1)][hf + 2 * (j & 1)] = v;
@@ -186,10 +195,10 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
         const uint32_t w0 = hf ? u.z : u.x, w1 = hf ? u.w : u.y;
-        a[pl * 2 + 0][hf] = h2sub((w0 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[pl * 2 + 0][hf + 2] = h2sub(((w0 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[pl * 2 + 1][hf] = h2sub((w1 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[pl * 2 + 1][hf + 2] = h2sub(((w1 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[pl * 2 + 0][hf] = h2sub(and_or(w0, 0x00ff00ffu, kMagic), zc.c[hf][0]);
+        a[pl * 2 + 0][hf + 2] = h2sub(and_or(w0 >> 8, 0x00ff00ffu, kMagic), zc.c[hf][0]);
+        a[pl * 2 + 1][hf] = h2sub(and_or(w1, 0x00ff00ffu, kMagic), zc.c[hf][0]);
+        a[pl * 2 + 1][hf + 2] = h2sub(and_or(w1 >> 8, 0x00ff00ffu, kMagic), zc.c[hf][0]);
       }
     }
   } else if constexpr (FMT == FMT_F16) {
@@ -214,8 +223,12 @@ __device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint
   constexpr int tb = tile_bytes(FMT);
   constexpr bool quant = fmt_quantised(FMT);
   const int g = lane >> 2;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  tot[0] = tot[1] = tot[2] = tot[3] = 0.f;
+  // Two independent accumulator chains per tile: the four mma of a tile would otherwise wait for one
+  // another (an mma takes ~30 cycles to deliver its accumulator), and with four warps per scheduler that
+  // latency is not hidden.
+  float acc[2][4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) { acc[0][k] = 0.f; acc[1][k] = 0.f; tot[k] = 0.f; }
   ZC zc;
   float s_a = 0.f, s_b = 0.f;
 #pragma unroll
@@ -234,18 +247,22 @@ __device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint
     tile_frags<FMT>(blob + c * tb, lane, zc, a);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      mma16816(acc, a[i], xr[8 * c + 2 * i], xr[8 * c + 2 * i + 1]);
-      if constexpr (HILO) mma16816(acc, a[i], xl[8 * c + 2 * i], xl[8 * c + 2 * i + 1]);
+      mma16816(acc[i & 1], a[i], xr[8 * c + 2 * i], xr[8 * c + 2 * i + 1]);
+      if constexpr (HILO) mma16816(acc[i & 1], a[i], xl[8 * c + 2 * i], xl[8 * c + 2 * i + 1]);
     }
     if constexpr (quant) {
       if (c == 1 || sz2) {
-        tot[0] = fmaf(acc[0], s_a, tot[0]); tot[1] = fmaf(acc[1], s_a, tot[1]);
-        tot[2] = fmaf(acc[2], s_b, tot[2]); tot[3] = fmaf(acc[3], s_b, tot[3]);
-        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+        tot[0] = fmaf(acc[0][0] + acc[1][0], s_a, tot[0]); tot[1] = fmaf(acc[0][1] + acc[1][1], s_a, tot[1]);
+        tot[2] = fmaf(acc[0][2] + acc[1][2], s_b, tot[2]); tot[3] = fmaf(acc[0][3] + acc[1][3], s_b, tot[3]);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { acc[0][k] = 0.f; acc[1][k] = 0.f; }
       }
     }
   }
-  if constexpr (!quant) { tot[0] = acc[0]; tot[1] = acc[1]; tot[2] = acc[2]; tot[3] = acc[3]; }
+  if constexpr (!quant) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) tot[k] = acc[0][k] + acc[1][k];
+  }
 }
 
 
