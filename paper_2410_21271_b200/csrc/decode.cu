@@ -140,6 +140,7 @@ struct Ring {
   // consumer side
   int slot;
   uint32_t parity;
+  int deferred;             // slots [kRing - deferred, kRing) have not had their first copy requested yet
 };
 
 __device__ __forceinline__ void ring_issue(Ring& r, int slot, int lane) {
@@ -230,6 +231,9 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     } else {
       load_x_pair(xr, p, pair, lane);
     }
+    // The first copies that were held back (see the kernel) go out behind the loads of the activations,
+    // not in front of them.
+    for (; r.deferred > 0; --r.deferred) ring_issue(r, kRing - r.deferred, lane);
     // Tickets of the blobs flushed so far are taken in batches of up to 32 (one atomic per lane, one
     // round trip per batch): batch_tile is the row tile of the batch's first blob, batch_n its size.
     uint32_t batch_tile = tile, batch_n = 0, flushed = 0;
@@ -260,7 +264,7 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
       const uint32_t cn = n < per_copy ? n : per_copy;
       if (!mbar_wait_warp(r.bars + r.slot, r.parity, p.dev_status, lane)) return false;
       const uint8_t* src = r.slots + r.slot * kSlotBytes;
-#pragma unroll 1
+#pragma unroll 2
       for (uint32_t j = 0; j < cn; ++j) {
         float tot[4];
         blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot);
@@ -343,8 +347,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
     r.ptr[2] = p.w_q + (size_t)(w0 + wf) * blob_w; r.rem[2] = wn - wf; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
   }
 
-#pragma unroll
-  for (int i = 0; i < kRing; ++i) ring_issue(r, i, lane);
+  // Before the dependency resolves only two of the three first copies per warp are requested:
+  // the activations are read right after the wait, and their loads would otherwise queue behind 29 MB of
+  // weight requests.
+  ring_issue(r, 0, lane);
+  ring_issue(r, 1, lane);
+  r.deferred = kRing - 2;
 
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tr && lane == 0) tr[1] = globaltimer_ns();

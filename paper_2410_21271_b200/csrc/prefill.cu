@@ -161,10 +161,10 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
       for (int part = 0; part < 4; ++part) {
         const int hf = part & 1;
         uint32_t lo = w[part], hi = w[part] >> 8;
-        a[part][0] = h2sub((lo & 0x000f000fu) | kMagic, zc.c[hf][0]);
-        a[part][1] = h2fma((lo & 0x00f000f0u) | kMagic, 0x2C002C00u, zc.c[hf][1]);
-        a[part][2] = h2sub((hi & 0x000f000fu) | kMagic, zc.c[hf][0]);
-        a[part][3] = h2fma((hi & 0x00f000f0u) | kMagic, 0x2C002C00u, zc.c[hf][1]);
+        a[part][0] = h2sub(and_or(lo, 0x000f000fu, kMagic), zc.c[hf][0]);
+        a[part][1] = h2fma(and_or(lo, 0x00f000f0u, kMagic), 0x2C002C00u, zc.c[hf][1]);
+        a[part][2] = h2sub(and_or(hi, 0x000f000fu, kMagic), zc.c[hf][0]);
+        a[part][3] = h2fma(and_or(hi, 0x00f000f0u, kMagic), 0x2C002C00u, zc.c[hf][1]);
       }
     } else if constexpr (FMT == FMT_Q3) {
       const uint32_t w[3] = {r.v.x, r.v.y, r.w2};
@@ -176,14 +176,14 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
         if (p < 15) {
           const int wi = p / 5, f = p % 5, ff = f >= 3 ? f - 3 : f;
           const uint32_t src = f >= 3 ? ws[wi] : w[wi];
-          const uint32_t h = (src & (0x00070007u << (3 * ff))) | kMagic;
+          const uint32_t h = and_or(src, 0x00070007u << (3 * ff), kMagic);
           if (ff == 0) v = h2sub(h, zc.c[hf][0]);
           else if (ff == 1) v = h2fma(h, 0x30003000u, zc.c[hf][1]);
           else v = h2fma(h, 0x24002400u, zc.c[hf][2]);
         } else {
-          uint32_t h = ((w[0] >> 15) & 0x00010001u) | kMagic;
-          h |= (w[1] >> 14) & 0x00020002u;
-          h |= (w[2] >> 13) & 0x00040004u;
+          uint32_t h = and_or(w[0] >> 15, 0x00010001u, kMagic);
+          h = and_or(w[1] >> 14, 0x00020002u, h);
+          h = and_or(w[2] >> 13, 0x00040004u, h);
           v = h2sub(h, zc.c[hf][0]);
         }
         a[part][j] = v;
@@ -194,10 +194,10 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
         const int hf = part & 1;
         const uint4 u = r.v[part >> 1];
         const uint32_t w0 = hf ? u.z : u.x, w1 = hf ? u.w : u.y;
-        a[part][0] = h2sub((w0 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[part][1] = h2sub(((w0 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[part][2] = h2sub((w1 & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
-        a[part][3] = h2sub(((w1 >> 8) & 0x00ff00ffu) | kMagic, zc.c[hf][0]);
+        a[part][0] = h2sub(and_or(w0, 0x00ff00ffu, kMagic), zc.c[hf][0]);
+        a[part][1] = h2sub(and_or(w0 >> 8, 0x00ff00ffu, kMagic), zc.c[hf][0]);
+        a[part][2] = h2sub(and_or(w1, 0x00ff00ffu, kMagic), zc.c[hf][0]);
+        a[part][3] = h2sub(and_or(w1 >> 8, 0x00ff00ffu, kMagic), zc.c[hf][0]);
       }
     }
     const uint32_t s_a = (sc2 & 0xffffu) * 0x00010001u, s_b = (sc2 >> 16) * 0x00010001u;
