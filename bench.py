@@ -44,8 +44,17 @@ def measured_peaks() -> tuple[dict, str]:
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
 
 
-def step_bytes(blocks: int) -> int:
-    return blocks * sum(traffic.forward_bytes(W_FMT, AB_FMT, K, N, RANK, M_DECODE) for _, (K, N) in LAYERS)
+# Layers of a block that read the same activations are fused into one launch (q|k|v and gate|up).
+FUSE_GROUPS = (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))
+
+
+def step_bytes(blocks: int, fused: bool = True) -> int:
+    """Algorithmic bytes of a step; a fused group reads its X once."""
+    shapes = dict(LAYERS)
+    per_block = sum(traffic.forward_bytes(W_FMT, AB_FMT, K, N, RANK, M_DECODE) for _, (K, N) in LAYERS)
+    if fused:
+        per_block -= sum((len(g) - 1) * 2 * M_DECODE * shapes[g[0]][0] for g in FUSE_GROUPS)
+    return blocks * per_block
 
 
 # --------------------------------------------------------------------------------------------
@@ -96,51 +105,75 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------------
-def build_layer_set(blocks: int, device: str, seed0: int = 1000):
-    """blocks x 7 layers with distinct seeded weights; returns (layers, x buffers, y buffers)."""
+def build_layer_set(blocks: int, device: str, seed0: int = 1000, fused: bool = True):
+    """blocks x 7 layers with distinct seeded weights as launch units (names, K, Ns, object): with `fused` the
+    layers of a block that share their input sit behind one handle (one launch), otherwise every layer has
+    its own.  Returns (units, x buffers, y buffers)."""
     import torch
     import paper_2410_21271_b200 as eora
-    layers = []
+    shapes = dict(LAYERS)
+    index = {name: li for li, (name, _) in enumerate(LAYERS)}
+    groups = FUSE_GROUPS if fused else tuple((name,) for name, _ in LAYERS)
+    units = []
     for b in range(blocks):
-        for li, (name, (K, N)) in enumerate(LAYERS):
-            seed = seed0 + 16 * b + li
-            wf = gen.make_backbone_quant(seed, K, N, 3 if W_FMT == "q3" else 4, 128)
-            af, bf = gen.make_ab_f16(seed, K, N, RANK)
-            layers.append((name, K, N, eora.Layer(wf, af, bf, max_m=M_DECODE, device=device)))
+        for names in groups:
+            parts = []
+            for name in names:
+                K, N = shapes[name]
+                seed = seed0 + 16 * b + index[name]
+                wf = gen.make_backbone_quant(seed, K, N, 3 if W_FMT == "q3" else 4, 128)
+                af, bf = gen.make_ab_f16(seed, K, N, RANK)
+                parts.append((wf, af, bf))
+            K = shapes[names[0]][0]
+            Ns = tuple(shapes[n][1] for n in names)
+            if len(names) == 1:
+                obj = eora.Layer(*parts[0], max_m=M_DECODE, device=device)
+            else:
+                obj = eora.FusedLayers(parts, max_m=M_DECODE, device=device)
+            units.append((names, K, Ns, obj))
     xs, ys = {}, {}
     for name, (K, N) in LAYERS:
         xs[name] = torch.from_numpy(gen.make_x(7, M_DECODE, K)).to(device)
         ys[name] = torch.empty((M_DECODE, N), dtype=torch.float16, device=device)
-    return layers, xs, ys
+    return units, xs, ys
 
 
-# Inside a transformer block q, k, v read the same hidden state and gate, up the same one, so those launches
-# do not depend on each other: they go to side streams and join before o / down.  Everything else is in
-# stream order (each layer's input is the previous layer's output in the real model).
+# Inside a transformer block q, k, v read the same hidden state and gate, up the same one, so (when they are
+# not fused into one launch) those launches do not depend on each other: they go to side streams and join
+# before o / down.  Everything else is in stream order (each layer's input is the previous layer's output in
+# the real model).
 CONCURRENT_WITH_PREVIOUS = {"k", "v", "up"}
 
 
-def run_step(layers, xs, ys, side=None):
-    import torch
+def launch_unit(unit, xs, ys, stream):
     import paper_2410_21271_b200 as eora
+    names, K, Ns, obj = unit
+    if len(names) == 1:
+        eora.eora_linear_forward(obj.handle, xs[names[0]], M_DECODE, ys[names[0]], stream)
+    else:
+        eora.eora_linear_forward_fused(obj.handle, xs[names[0]], M_DECODE, [ys[n] for n in names], stream)
+
+
+def run_step(units, xs, ys, side=None):
+    import torch
     main = torch.cuda.current_stream()
     pending = []
     i = 0
-    while i < len(layers):
-        group = [layers[i]]
-        while i + len(group) < len(layers) and layers[i + len(group)][0] in CONCURRENT_WITH_PREVIOUS:
-            group.append(layers[i + len(group)])
+    while i < len(units):
+        group = [units[i]]
+        while i + len(group) < len(units) and units[i + len(group)][0][0] in CONCURRENT_WITH_PREVIOUS:
+            group.append(units[i + len(group)])
         i += len(group)
         if side is None or len(group) == 1:
-            for name, K, N, L in group:
-                eora.eora_linear_forward(L.handle, xs[name], M_DECODE, ys[name], main)
+            for u in group:
+                launch_unit(u, xs, ys, main)
             continue
         fork = main.record_event()
-        for j, (name, K, N, L) in enumerate(group):
+        for j, u in enumerate(group):
             st = main if j == 0 else side[(j - 1) % len(side)]
             if j:
                 st.wait_event(fork)
-            eora.eora_linear_forward(L.handle, xs[name], M_DECODE, ys[name], st)
+            launch_unit(u, xs, ys, st)
             if j:
                 pending.append(st.record_event())
         for ev in pending:
@@ -181,8 +214,8 @@ def time_decode(layers, xs, ys, steps: int, warmup: int, device_index: int, use_
             torch.cuda.synchronize()
         barrier()
         ms = e0.elapsed_time(e1) / steps
-    for _, _, _, L in layers:
-        assert L.device_status() == 0, "a device-side wait ran out"
+    for _, _, _, obj in layers:
+        assert obj.device_status() == 0, "a device-side wait ran out"
     return ms, cs.summary(), graph is not None
 
 
@@ -192,8 +225,11 @@ def time_e2e(layers, steps: int, warmup: int):
     hx = {name: torch.from_numpy(gen.make_x(7, M_DECODE, K)).pin_memory() for name, (K, N) in LAYERS}
     hy = {name: torch.empty((M_DECODE, N), dtype=torch.float16).pin_memory() for name, (K, N) in LAYERS}
     def step():
-        for name, K, N, L in layers:
-            L.forward_host(hx[name], hy[name])
+        for names, K, Ns, obj in layers:
+            if len(names) == 1:
+                obj.forward_host(hx[names[0]], hy[names[0]])
+            else:
+                obj.forward_host(hx[names[0]], [hy[n] for n in names])
     for _ in range(max(1, warmup)):
         step()
     torch.cuda.synchronize()
@@ -202,8 +238,8 @@ def time_e2e(layers, steps: int, warmup: int):
         step()
     torch.cuda.synchronize()
     sec = (time.perf_counter() - t0) / steps
-    h2d = sum(2 * M_DECODE * K for _, K, N, _ in layers)
-    d2h = sum(2 * M_DECODE * N for _, K, N, _ in layers)
+    h2d = sum(2 * M_DECODE * K for _, K, Ns, _ in layers)
+    d2h = sum(2 * M_DECODE * N for _, K, Ns, _ in layers for N in Ns)
     return sec, h2d, d2h
 
 
@@ -238,11 +274,11 @@ def time_prefill(device: str, steps: int = 10, warmup: int = 3):
             "path": {0: "generic", 1: "decode", 2: "prefill"}[path], "l2": "flushed between iterations"}
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of k_decode, mean over the seven layers of a block,
-# from the ncu capture summarised in profiles/k_decode_llama3-8b-w3g128-r128-M1.md (traffic grows with the
-# number of blocks in proportion, every block being the same seven launches).  Set to None when the kernel
-# changes until the capture is redone.
-DRAM_BYTES_PER_LAUNCH = 15.52e6
+# dram__bytes_read.sum + dram__bytes_write.sum of k_decode over the seven layers of one block, from the ncu
+# capture summarised in profiles/k_decode_llama3-8b-w3g128-r128-M1.md (traffic grows with the number of
+# blocks in proportion; fusing layers changes the number of launches, not the bytes).  Set to None when the
+# kernel's memory behaviour changes until the capture is redone.
+DRAM_BYTES_PER_BLOCK = 108.64e6
 
 
 def cpu_oracle_sample(blocks_sample: int = 1):
@@ -307,6 +343,7 @@ def main():
     ap.add_argument("--blocks", type=int, default=gen.LLAMA3_8B_BLOCKS, help=argparse.SUPPRESS)
     ap.add_argument("--no-extras", action="store_true", help="skip the prefill / e2e / cpu legs")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--unfused", action="store_true", help="one launch per layer (224 per token) instead of fusing q|k|v and gate|up")
     ap.add_argument("--only-prefill", action="store_true", help="run the prefill leg alone (for profiling) and print its result")
     ap.add_argument("--single-stream", action="store_true", help="launch all layers of a block in stream order")
     args = ap.parse_args()
@@ -315,7 +352,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     config = {"workload": WORKLOAD, "blocks": args.blocks, "layers_per_block": 7, "M": M_DECODE,
               "l2": "weights of one step (3.4 GB) exceed L2, no flush needed", "parallelism": f"replicas x{world}",
-              "streams": ("stream order" if args.single_stream else
+              "launches_per_token": 224 if args.unfused else 128,
+              "fusion": ("none: one launch per layer" if args.unfused else
+                         "q|k|v and gate|up of a block share their input and run as one launch each"),
+              "streams": ("stream order" if (args.single_stream or not args.unfused) else
                           "q,k,v and gate,up of a block are independent and run on 3 / 2 streams; the rest in stream order")}
 
     if args.impl == "reference":
@@ -350,18 +390,19 @@ def main():
         if rank == 0:
             print(json.dumps({"prefill": time_prefill(device)}))
         return
-    layers, xs, ys = build_layer_set(args.blocks, device)
-    n_launch_step = sum(L.launches(M_DECODE) for _, _, _, L in layers)
+    fused = not args.unfused
+    layers, xs, ys = build_layer_set(args.blocks, device, fused=fused)
+    n_launch_step = sum(obj.launches(M_DECODE) for _, _, _, obj in layers)
     ms_local, clocks, graphed = time_decode(layers, xs, ys, args.steps, args.warmup, local_rank, not args.no_graph,
                                              not args.single_stream)
     value, ms = aggregate(ms_local, M_DECODE, world)
     peaks, peak_kind = measured_peaks()
-    bytes_step = step_bytes(args.blocks)
+    bytes_step = step_bytes(args.blocks, fused)
     achieved = bytes_step / (ms_local / 1e3) / 1e9
     roofline = {"bound": "hbm", "kernel": "k_decode", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": DRAM_BYTES_PER_LAUNCH if args.blocks == gen.LLAMA3_8B_BLOCKS else None,
+                "traffic": DRAM_BYTES_PER_BLOCK * args.blocks / n_launch_step,
                 "bytes_per_launch": bytes_step / n_launch_step, "us_per_launch": ms_local * 1e3 / n_launch_step}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -373,9 +414,9 @@ def main():
         sec, h2d, d2h = time_e2e(layers, max(2, min(args.steps, 10)), 1)
         sec = max_over_ranks(sec)
         line["e2e"] = {"value": world * M_DECODE / sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                       "note": "per layer: pinned host X -> device, fused layer, Y -> host, stream sync"}
-    for _, _, _, L in layers:
-        L.close()
+                       "note": "per launch unit: pinned host X -> device, the layer(s), Y -> host, stream sync"}
+    for _, _, _, obj in layers:
+        obj.close()
     if not args.no_extras and rank == 0:
         if world == 1:
             line["cpu_baseline"] = cpu_oracle_sample(8)[0]

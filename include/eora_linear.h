@@ -123,6 +123,26 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
 int eora_linear_forward(eora_linear_t h, const void* x, int32_t m, void* y, void* stream);
 
 /*
+ * Fused layers.  The compensation of Eq. 4 is applied to every compressed linear layer of a model
+ * (Section 3), and several of them read the same activations: q/k/v of an attention block, gate/up
+ * of an MLP.  eora_linear_create_fused builds ONE handle for n_layers (2..4) such layers, given as
+ * arrays of configs and weights; they must agree in everything but d_out (same d_in, rank, formats,
+ * groups, dtypes, max_m <= 64, policy AUTO, quantised backbone).  eora_linear_forward_fused computes
+ *     ys[i][M][d_out_i] = X . deq(Wq_i) + (X . A_i) . B_i      for every layer i
+ * with ONE kernel launch per eight tokens: X is read once, and the launch latency is paid once.
+ * ys: host array of n_layers device pointers (16-byte aligned, caller-owned).  The handle serves
+ * the decode family only (M <= 64); eora_linear_forward / _forward_host on it return
+ * EORA_ERR_UNSUPPORTED, everything else (destroy, launches, last_device_status, dump of the
+ * stacked matrices) works as for a plain handle.  Errors as for create / forward.
+ */
+int eora_linear_create_fused(const eora_linear_config* cfgs, const eora_linear_weights* weights, int32_t n_layers,
+                             void* stream, eora_linear_t* out);
+int eora_linear_forward_fused(eora_linear_t h, const void* x, int32_t m, void* const* ys, void* stream);
+/* The fused forward for activations in HOST memory (see eora_linear_forward_host): ys_host is a host array
+ * of n_layers host pointers; synchronises `stream` before returning. */
+int eora_linear_forward_fused_host(eora_linear_t h, const void* x_host, int32_t m, void* const* ys_host, void* stream);
+
+/*
  * The same forward for callers whose activations live in HOST memory: copies x_host (pinned or
  * pageable, [m][d_in]) to a library-owned device staging buffer, runs the forward, copies the
  * result back to y_host ([m][d_out]) and synchronises `stream` before returning.

@@ -60,6 +60,12 @@ def lib() -> ctypes.CDLL:
         L.eora_linear_forward.restype = c_int
         L.eora_linear_forward_host.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
         L.eora_linear_forward_host.restype = c_int
+        L.eora_linear_create_fused.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_create_fused.restype = c_int
+        L.eora_linear_forward_fused.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_forward_fused.restype = c_int
+        L.eora_linear_forward_fused_host.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_forward_fused_host.restype = c_int
         L.eora_linear_destroy.argtypes = [c_void_p]
         L.eora_linear_destroy.restype = c_int
         L.eora_linear_path.argtypes = [c_void_p, c_int32]
@@ -148,6 +154,39 @@ def eora_linear_forward_host(handle: int, x_host, m: int, y_host, stream=None, c
     return st
 
 
+def eora_linear_create_fused(cfgs, weights, stream=None, check: bool = True):
+    """cfgs / weights: sequences of eora_linear_config / eora_linear_weights (one per fused layer).
+    Returns the handle, or (with check=False) the status."""
+    n = len(cfgs)
+    carr = (eora_linear_config * n)(*cfgs)
+    warr = (eora_linear_weights * n)(*weights)
+    out = c_void_p()
+    st = lib().eora_linear_create_fused(carr, warr, n, _stream(stream), byref(out))
+    if not check:
+        if st == EORA_OK:
+            lib().eora_linear_destroy(out)
+        return st
+    if st != EORA_OK:
+        raise EoraError(st, "eora_linear_create_fused")
+    return out.value
+
+
+def eora_linear_forward_fused(handle: int, x, m: int, ys, stream=None, check: bool = True) -> int:
+    arr = (c_void_p * len(ys))(*[_ptr(y) for y in ys])
+    st = lib().eora_linear_forward_fused(handle, _ptr(x), int(m), arr, _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward_fused")
+    return st
+
+
+def eora_linear_forward_fused_host(handle: int, x_host, m: int, ys_host, stream=None, check: bool = True) -> int:
+    arr = (c_void_p * len(ys_host))(*[_ptr(y) for y in ys_host])
+    st = lib().eora_linear_forward_fused_host(handle, _ptr(x_host), int(m), arr, _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward_fused_host")
+    return st
+
+
 def eora_linear_destroy(handle: int) -> int:
     return lib().eora_linear_destroy(handle)
 
@@ -214,6 +253,46 @@ def _dev(arr, device):
     return torch.from_numpy(a).to(device)
 
 
+def _marshal(w_fmt: dict, a_fmt, b_fmt, *, max_m: int, x_dtype: str, y_dtype: str, kernel_policy: int, device):
+    """Upload one layer's interchange buffers and fill the two C structs.  Returns (cfg, weights, buffers);
+    the buffers must stay alive until create has returned."""
+    cfg = eora_linear_config()
+    wts = eora_linear_weights()
+    keep = []
+    cfg.d_in, cfg.d_out = w_fmt["rows"], w_fmt["cols"]
+    if w_fmt["kind"] == "quant":
+        cfg.w_format, cfg.w_bits, cfg.w_group = EORA_W_QUANT, w_fmt["bits"], w_fmt["group"]
+        bufs = [_dev(w_fmt["codes"], device), _dev(w_fmt["scales"], device), _dev(w_fmt["zeros"], device)]
+    elif w_fmt["kind"] == "sparse24":
+        cfg.w_format = EORA_W_SPARSE24
+        bufs = [_dev(w_fmt["values"], device), None, _dev(w_fmt["meta"], device)]
+    else:
+        raise ValueError(w_fmt["kind"])
+    keep += bufs
+    wts.w_codes, wts.w_scales, wts.w_zeros = [_ptr(b) for b in bufs]
+    cfg.rank = 0
+    cfg.ab_format, cfg.ab_group = EORA_AB_F16, 128
+    if a_fmt is not None and b_fmt is not None:
+        kind = a_fmt["kind"]
+        if kind == "f16":
+            cfg.rank = a_fmt["data"].shape[1]
+            ab = [_dev(a_fmt["data"], device), None, None, _dev(b_fmt["data"], device), None, None]
+        elif kind == "quant":
+            cfg.rank, cfg.ab_format, cfg.ab_group = a_fmt["cols"], EORA_AB_Q4, a_fmt["group"]
+            ab = [_dev(f[k], device) for f in (a_fmt, b_fmt) for k in ("codes", "scales", "zeros")]
+        elif kind == "q8":
+            cfg.rank, cfg.ab_format = a_fmt["cols"], EORA_AB_Q8
+            ab = [_dev(f[k], device) for f in (a_fmt, b_fmt) for k in ("codes", "scales", "zeros")]
+        else:
+            raise ValueError(kind)
+        keep += ab
+        (wts.a, wts.a_scales, wts.a_zeros, wts.b, wts.b_scales, wts.b_zeros) = [_ptr(b) for b in ab]
+    cfg.x_dtype = {"f16": EORA_X_F16, "bf16": EORA_X_BF16}[x_dtype]
+    cfg.y_dtype = {"f16": EORA_Y_F16, "bf16": EORA_Y_BF16, "f32": EORA_Y_F32}[y_dtype]
+    cfg.max_m, cfg.kernel_policy = max_m, kernel_policy
+    return cfg, wts, keep
+
+
 class Layer:
     """Owns a library handle plus nothing else (the uploaded interchange buffers are dropped after
     create).  Methods only marshal arguments."""
@@ -221,40 +300,8 @@ class Layer:
     def __init__(self, w_fmt: dict, a_fmt: dict | None, b_fmt: dict | None, *, max_m: int, x_dtype: str = "f16",
                  y_dtype: str = "f16", kernel_policy: int = EORA_POLICY_AUTO, device="cuda:0"):
         import torch
-        cfg = eora_linear_config()
-        wts = eora_linear_weights()
-        keep = []
-        cfg.d_in, cfg.d_out = w_fmt["rows"], w_fmt["cols"]
-        if w_fmt["kind"] == "quant":
-            cfg.w_format, cfg.w_bits, cfg.w_group = EORA_W_QUANT, w_fmt["bits"], w_fmt["group"]
-            bufs = [_dev(w_fmt["codes"], device), _dev(w_fmt["scales"], device), _dev(w_fmt["zeros"], device)]
-        elif w_fmt["kind"] == "sparse24":
-            cfg.w_format = EORA_W_SPARSE24
-            bufs = [_dev(w_fmt["values"], device), None, _dev(w_fmt["meta"], device)]
-        else:
-            raise ValueError(w_fmt["kind"])
-        keep += bufs
-        wts.w_codes, wts.w_scales, wts.w_zeros = [_ptr(b) for b in bufs]
-        cfg.rank = 0
-        cfg.ab_format, cfg.ab_group = EORA_AB_F16, 128
-        if a_fmt is not None and b_fmt is not None:
-            kind = a_fmt["kind"]
-            if kind == "f16":
-                cfg.rank = a_fmt["data"].shape[1]
-                ab = [_dev(a_fmt["data"], device), None, None, _dev(b_fmt["data"], device), None, None]
-            elif kind == "quant":
-                cfg.rank, cfg.ab_format, cfg.ab_group = a_fmt["cols"], EORA_AB_Q4, a_fmt["group"]
-                ab = [_dev(f[k], device) for f in (a_fmt, b_fmt) for k in ("codes", "scales", "zeros")]
-            elif kind == "q8":
-                cfg.rank, cfg.ab_format = a_fmt["cols"], EORA_AB_Q8
-                ab = [_dev(f[k], device) for f in (a_fmt, b_fmt) for k in ("codes", "scales", "zeros")]
-            else:
-                raise ValueError(kind)
-            keep += ab
-            (wts.a, wts.a_scales, wts.a_zeros, wts.b, wts.b_scales, wts.b_zeros) = [_ptr(b) for b in ab]
-        cfg.x_dtype = {"f16": EORA_X_F16, "bf16": EORA_X_BF16}[x_dtype]
-        cfg.y_dtype = {"f16": EORA_Y_F16, "bf16": EORA_Y_BF16, "f32": EORA_Y_F32}[y_dtype]
-        cfg.max_m, cfg.kernel_policy = max_m, kernel_policy
+        cfg, wts, keep = _marshal(w_fmt, a_fmt, b_fmt, max_m=max_m, x_dtype=x_dtype, y_dtype=y_dtype,
+                                  kernel_policy=kernel_policy, device=device)
         self.cfg = cfg
         self.device = torch.device(device)
         self.y_torch_dtype = {"f16": torch.float16, "bf16": torch.bfloat16, "f32": torch.float32}[y_dtype]
@@ -288,6 +335,54 @@ class Layer:
         out = torch.empty(shape, dtype=dt, device=self.device)
         eora_linear_dump(self.handle, what, out)
         return out
+
+    def device_status(self) -> int:
+        return eora_linear_last_device_status(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            eora_linear_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class FusedLayers:
+    """Several layers that read the same X (q/k/v, gate/up) behind ONE handle and one launch per forward.
+    Decode only (max_m <= 64).  Methods only marshal arguments."""
+
+    def __init__(self, layers, *, max_m: int, x_dtype: str = "f16", y_dtype: str = "f16", device="cuda:0"):
+        import torch
+        cfgs, wtss, keep = [], [], []
+        for (w_fmt, a_fmt, b_fmt) in layers:
+            cfg, wts, k = _marshal(w_fmt, a_fmt, b_fmt, max_m=max_m, x_dtype=x_dtype, y_dtype=y_dtype,
+                                   kernel_policy=EORA_POLICY_AUTO, device=device)
+            cfgs.append(cfg); wtss.append(wts); keep.append(k)
+        self.cfgs = cfgs
+        self.device = torch.device(device)
+        self.y_torch_dtype = {"f16": torch.float16, "bf16": torch.bfloat16, "f32": torch.float32}[y_dtype]
+        with torch.cuda.device(self.device):
+            self.handle = eora_linear_create_fused(cfgs, wtss)
+        del keep
+
+    def forward(self, x, ys=None, stream=None):
+        import torch
+        m = x.shape[0]
+        if ys is None:
+            ys = [torch.empty((m, c.d_out), dtype=self.y_torch_dtype, device=x.device) for c in self.cfgs]
+        eora_linear_forward_fused(self.handle, x, m, ys, stream)
+        return ys
+
+    def forward_host(self, x_host, ys_host, stream=None):
+        eora_linear_forward_fused_host(self.handle, x_host, x_host.shape[0], ys_host, stream)
+        return ys_host
+
+    def launches(self, m: int) -> int:
+        return eora_linear_launches(self.handle, m)
 
     def device_status(self) -> int:
         return eora_linear_last_device_status(self.handle)

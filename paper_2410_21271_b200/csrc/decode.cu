@@ -51,9 +51,15 @@ struct DecodeArgs {
   uint32_t n_a;                           // number of A-owner warps
   Share sh_a, sh_w1, sh_w2, sh_b;
   uint32_t tile_target;                   // blobs per output row tile: pairs of W + pairs of B
-  const void* x; void* y;
+  const void* x;
+  void* ys[4];                            // outputs of the fused layers (one for a plain layer)
+  uint32_t sub_tile0[5];                  // layer i owns row tiles [sub_tile0[i], sub_tile0[i+1])
+  int sub_dout[4];
+  int n_sub;
+  uint32_t b_np;                          // pairs of B per layer: the activations of B's blob (pair, tile) are
+                                          // pair (layer(tile) * b_np + pair) of t
   float* d_t; float* y_ws; uint32_t* counters; int* dev_status;
-  int m, d_in, d_out, r_pad, n_pad, x_dtype, y_dtype;
+  int m, d_in, r_pad, n_pad, x_dtype, y_dtype;   // r_pad: columns of t (all fused layers)
   unsigned long long* trace;
 };
 
@@ -175,6 +181,12 @@ __device__ __forceinline__ void st_zero4(float* p) {
 // it converts the tile's 16 x m sums, stores them and puts the scratch back to zero.  Several lanes of a
 // warp may each be finishing a tile of their own at the same time.
 __device__ __forceinline__ void finish_row_tile(const DecodeArgs& p, uint32_t tile) {
+  void* y = p.ys[0];
+  uint32_t tile0 = 0;
+  int dout = p.sub_dout[0];
+#pragma unroll
+  for (int i = 1; i < 4; ++i)
+    if (i < p.n_sub && tile >= p.sub_tile0[i]) { y = p.ys[i]; tile0 = p.sub_tile0[i]; dout = p.sub_dout[i]; }
   for (int token = 0; token < p.m; ++token) {
     float* s = p.y_ws + (size_t)token * p.n_pad + tile * 16;
     uint4 u[4];
@@ -186,9 +198,9 @@ __device__ __forceinline__ void finish_row_tile(const DecodeArgs& p, uint32_t ti
                          __uint_as_float(u[1].x), __uint_as_float(u[1].y), __uint_as_float(u[1].z), __uint_as_float(u[1].w),
                          __uint_as_float(u[2].x), __uint_as_float(u[2].y), __uint_as_float(u[2].z), __uint_as_float(u[2].w),
                          __uint_as_float(u[3].x), __uint_as_float(u[3].y), __uint_as_float(u[3].z), __uint_as_float(u[3].w)};
-    const int64_t o = (int64_t)token * p.d_out + tile * 16;       // d_out is a multiple of 32: the 16 outputs exist
+    const int64_t o = (int64_t)token * dout + (tile - tile0) * 16;   // d_out is a multiple of 32: the 16 outputs exist
     if (p.y_dtype == EORA_Y_F32) {
-      float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.y) + o);
+      float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(y) + o);
 #pragma unroll
       for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
     } else {
@@ -202,7 +214,7 @@ __device__ __forceinline__ void finish_row_tile(const DecodeArgs& p, uint32_t ti
           h[i] = *reinterpret_cast<const uint32_t*>(&b);
         }
       }
-      uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(p.y) + o);
+      uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(y) + o);
       dst[0] = make_uint4(h[0], h[1], h[2], h[3]);
       dst[1] = make_uint4(h[4], h[5], h[6], h[7]);
     }
@@ -220,6 +232,7 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     if (n == 0) return true;
     uint32_t pair = b0 / nt, tile = b0 - pair * nt;
     uint32_t xr[16], xl[16];
+    uint32_t sub = 0, sub_end = nt;
     if constexpr (HILO) {
       // all of A must be in t
       int ok = 1;
@@ -227,7 +240,13 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) return false;
       __syncwarp();
-      load_t_pair(xr, xl, p, pair, lane);
+      // the activations of B's blob (pair, tile) belong to the layer that owns the row tile
+      sub = 0;
+#pragma unroll
+      for (int i = 1; i < 4; ++i)
+        if (i < p.n_sub && tile >= p.sub_tile0[i]) sub = i;
+      sub_end = p.sub_tile0[sub + 1];
+      load_t_pair(xr, xl, p, sub * p.b_np + pair, lane);
     } else {
       load_x_pair(xr, p, pair, lane);
     }
@@ -280,8 +299,18 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
           tile = 0;
           ++pair;
           if (j + 1 < cn || n > cn) {
-            if constexpr (HILO) load_t_pair(xr, xl, p, pair, lane);
-            else load_x_pair(xr, p, pair, lane);
+            if constexpr (HILO) {
+              sub = 0; sub_end = p.sub_tile0[1];
+              load_t_pair(xr, xl, p, pair, lane);
+            } else {
+              load_x_pair(xr, p, pair, lane);
+            }
+          }
+        } else if constexpr (HILO) {
+          if (tile == sub_end && (j + 1 < cn || n > cn)) {      // the next row tile belongs to the next fused layer
+            ++sub;
+            sub_end = p.sub_tile0[sub + 1];
+            load_t_pair(xr, xl, p, sub * p.b_np + pair, lane);
           }
         }
       }
@@ -426,7 +455,7 @@ int decode_launch_count(const Handle*, int m) { return (m + 7) / 8; }
 
 int decode_grid(const Handle* h, int) { return h->sm_count * kCtasPerSm; }
 
-cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st) {
+cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st) {
   const bool ab = h->cfg.rank > 0;
   DecodeArgs a = {};
   a.w_q = h->w.q; a.w_nt = h->w.nt; a.w_sz2 = h->w.sz2; a.w_per_copy = blobs_per_copy(h->w);
@@ -480,7 +509,12 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y
   }
   a.tile_target = (uint32_t)h->w.np + (ab ? (uint32_t)h->b.np : 0u);
   a.d_t = h->d_t; a.y_ws = h->y_ws; a.counters = h->counters; a.dev_status = h->dev_status;
-  a.d_in = h->cfg.d_in; a.d_out = h->cfg.d_out; a.r_pad = h->r_pad > 0 ? h->r_pad : 128; a.n_pad = h->w.n_rows;
+  a.d_in = h->cfg.d_in; a.r_pad = h->t_cols; a.n_pad = h->w.n_rows;
+  a.n_sub = h->n_sub;
+  a.b_np = ab ? (uint32_t)h->b.np : 0u;
+  for (int i = 0; i <= h->n_sub; ++i) a.sub_tile0[i] = (uint32_t)h->sub_tile0[i];
+  for (int i = h->n_sub + 1; i < 5; ++i) a.sub_tile0[i] = (uint32_t)h->w.nt;
+  for (int i = 0; i < 4; ++i) a.sub_dout[i] = i < h->n_sub ? h->sub_dout[i] : 0;
   a.x_dtype = h->cfg.x_dtype; a.y_dtype = h->cfg.y_dtype;
   a.trace = reinterpret_cast<unsigned long long*>(h->trace);
 
@@ -499,7 +533,7 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y
   for (int m0 = 0; m0 < m; m0 += 8) {             // eight tokens per pass (the n8 side of the mma)
     a.m = m - m0 < 8 ? m - m0 : 8;
     a.x = reinterpret_cast<const uint8_t*>(x) + (size_t)m0 * h->cfg.d_in * 2;
-    a.y = reinterpret_cast<uint8_t*>(y) + (size_t)m0 * h->cfg.d_out * ybytes;
+    for (int i = 0; i < h->n_sub; ++i) a.ys[i] = reinterpret_cast<uint8_t*>(ys[i]) + (size_t)m0 * h->sub_dout[i] * ybytes;
     cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf) : launch_ab<FMT_Q3>(cfg, a, abf);
     if (e != cudaSuccess) return e;
   }

@@ -94,24 +94,56 @@ const char* eora_status_string(int s) {
   }
 }
 
-int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights* wts, void* stream, eora_linear_t* out) {
-  if (out) *out = nullptr;
-  if (!cfg || !wts || !out) return EORA_ERR_NULL_ARG;
-  int st = check_config(*cfg);
-  if (st != EORA_OK) return st;
-  const eora_linear_config& c = *cfg;
-  bool quant_w = c.w_format == EORA_W_QUANT;
-  if (!wts->w_codes || !wts->w_zeros || (quant_w && !wts->w_scales)) return EORA_ERR_NULL_ARG;
-  if (!aligned16(wts->w_codes) || !aligned16(wts->w_zeros) || !aligned16(wts->w_scales)) return EORA_ERR_MISALIGNED;
+}  // extern "C"
+
+namespace {
+
+int check_weights(const eora_linear_config& c, const eora_linear_weights& w) {
+  const bool quant_w = c.w_format == EORA_W_QUANT;
+  if (!w.w_codes || !w.w_zeros || (quant_w && !w.w_scales)) return EORA_ERR_NULL_ARG;
+  if (!aligned16(w.w_codes) || !aligned16(w.w_zeros) || !aligned16(w.w_scales)) return EORA_ERR_MISALIGNED;
   if (c.rank > 0) {
-    if (!wts->a || !wts->b) return EORA_ERR_NULL_ARG;
-    if (!aligned16(wts->a) || !aligned16(wts->b)) return EORA_ERR_MISALIGNED;
+    if (!w.a || !w.b) return EORA_ERR_NULL_ARG;
+    if (!aligned16(w.a) || !aligned16(w.b)) return EORA_ERR_MISALIGNED;
     if (c.ab_format != EORA_AB_F16) {
-      if (!wts->a_scales || !wts->a_zeros || !wts->b_scales || !wts->b_zeros) return EORA_ERR_NULL_ARG;
-      if (!aligned16(wts->a_scales) || !aligned16(wts->a_zeros) || !aligned16(wts->b_scales) || !aligned16(wts->b_zeros))
+      if (!w.a_scales || !w.a_zeros || !w.b_scales || !w.b_zeros) return EORA_ERR_NULL_ARG;
+      if (!aligned16(w.a_scales) || !aligned16(w.a_zeros) || !aligned16(w.b_scales) || !aligned16(w.b_zeros))
         return EORA_ERR_MISALIGNED;
     }
   }
+  return EORA_OK;
+}
+
+// A view of `m` that starts at row tile t0 (see launch_repack_*).
+WMat tile_view(const WMat& m, int t0) {
+  WMat v = m;
+  v.q = m.q + (int64_t)t0 * m.blob;
+  return v;
+}
+
+// One layer (n == 1) or n layers that share X, stacked along the output axis (fused, decode only).
+int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, int n, void* stream, eora_linear_t* out) {
+  if (out) *out = nullptr;
+  if (!cfgs || !wts || !out) return EORA_ERR_NULL_ARG;
+  if (n < 1 || n > 4) return EORA_ERR_BAD_SHAPE;
+  eora_linear_config c = cfgs[0];
+  int d_out_total = 0;
+  for (int i = 0; i < n; ++i) {
+    int st = check_config(cfgs[i]);
+    if (st != EORA_OK) return st;
+    st = check_weights(cfgs[i], wts[i]);
+    if (st != EORA_OK) return st;
+    const eora_linear_config& ci = cfgs[i];
+    if (ci.d_in != c.d_in || ci.rank != c.rank || ci.w_format != c.w_format || ci.w_bits != c.w_bits || ci.w_group != c.w_group ||
+        ci.ab_format != c.ab_format || ci.ab_group != c.ab_group || ci.x_dtype != c.x_dtype || ci.y_dtype != c.y_dtype ||
+        ci.max_m != c.max_m || ci.kernel_policy != c.kernel_policy)
+      return EORA_ERR_BAD_SHAPE;
+    d_out_total += ci.d_out;
+  }
+  const bool fused = n > 1;
+  if (fused && (c.w_format != EORA_W_QUANT || c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO)) return EORA_ERR_UNSUPPORTED;
+  c.d_out = d_out_total;
+  const bool quant_w = c.w_format == EORA_W_QUANT;
 
   eora_linear* obj = new (std::nothrow) eora_linear();
   if (!obj) return EORA_ERR_CUDA;
@@ -130,12 +162,20 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
   if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
 
   h->r_pad = (int)align_up(c.rank, 128);
+  h->n_sub = n;
+  h->t_cols = n * (h->r_pad > 0 ? h->r_pad : 128);
+  h->sub_tile0[0] = 0;
+  for (int i = 0; i < n; ++i) {
+    h->sub_dout[i] = cfgs[i].d_out;
+    h->sub_tile0[i + 1] = h->sub_tile0[i] + cfgs[i].d_out / 16;
+  }
+  for (int i = n + 1; i < 5; ++i) h->sub_tile0[i] = h->sub_tile0[n];
   int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : FMT_Q8;
   wmat_shape(h->w, quant_w ? (c.w_bits == 4 ? FMT_Q4 : FMT_Q3) : FMT_SP24, c.d_out, c.d_in, quant_w ? c.w_group : 0);
   if (c.rank > 0) {
     int ga = c.ab_format == EORA_AB_Q4 ? c.ab_group : 0;
     int gb = c.ab_format == EORA_AB_Q4 ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 0;
-    wmat_shape(h->a, ab_fmt, c.rank, c.d_in, ga);
+    wmat_shape(h->a, ab_fmt, fused ? n * h->r_pad : c.rank, c.d_in, ga);   // fused: layer i owns rows [i r_pad, (i+1) r_pad)
     wmat_shape(h->b, ab_fmt, c.d_out, h->r_pad, gb);
   } else {
     wmat_shape(h->a, FMT_NONE, 0, 0, 0);
@@ -151,7 +191,7 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
   wmat_carve(h->w, wc); wmat_carve(h->a, wc); wmat_carve(h->b, wc);
 
   // ---- scratch: one allocation, zero-initialised
-  const int64_t rp = h->r_pad > 0 ? h->r_pad : 128;
+  const int64_t rp = h->t_cols;
   for (int pass = 0; pass < 2; ++pass) {
     Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
     h->t_ws = sc.take<float>((int64_t)c.max_m * rp * 4);
@@ -170,26 +210,89 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
   }
   if (cudaMemsetAsync(h->scratch_mem, 0, (size_t)h->scratch_bytes, s) != cudaSuccess) return fail(EORA_ERR_CUDA);
 
-  // ---- re-tile
+  // ---- re-tile, layer by layer into its range of row tiles
   cudaError_t e = cudaSuccess;
-  if (quant_w) e = launch_repack_quant(h->w, wts->w_codes, wts->w_scales, wts->w_zeros, c.w_bits, c.d_out, c.d_in, s);
-  else e = launch_repack_sp24(h->w, wts->w_codes, wts->w_zeros, c.d_out, c.d_in, s);
-  if (e == cudaSuccess && c.rank > 0) {
+  for (int i = 0; i < n && e == cudaSuccess; ++i) {
+    const eora_linear_weights& w = wts[i];
+    const int d_out_i = cfgs[i].d_out, nt_i = d_out_i / 16;
+    const WMat wv = tile_view(h->w, h->sub_tile0[i]);
+    if (quant_w) e = launch_repack_quant(wv, w.w_codes, w.w_scales, w.w_zeros, c.w_bits, d_out_i, c.d_in, s, fused ? nt_i : -1);
+    else e = launch_repack_sp24(wv, w.w_codes, w.w_zeros, d_out_i, c.d_in, s, -1);
+    if (e != cudaSuccess || c.rank == 0) continue;
+    const WMat av = tile_view(h->a, fused ? i * h->r_pad / 16 : 0);
+    const WMat bv = tile_view(h->b, h->sub_tile0[i]);
+    const int a_nt = fused ? h->r_pad / 16 : -1, b_nt = fused ? nt_i : -1;
     if (c.ab_format == EORA_AB_F16) {
-      e = launch_repack_f16(h->a, wts->a, c.rank, c.d_in, s);
-      if (e == cudaSuccess) e = launch_repack_f16(h->b, wts->b, c.d_out, c.rank, s);
+      e = launch_repack_f16(av, w.a, c.rank, c.d_in, s, a_nt);
+      if (e == cudaSuccess) e = launch_repack_f16(bv, w.b, d_out_i, c.rank, s, b_nt);
     } else if (c.ab_format == EORA_AB_Q4) {
-      e = launch_repack_quant(h->a, wts->a, wts->a_scales, wts->a_zeros, 4, c.rank, c.d_in, s);
-      if (e == cudaSuccess) e = launch_repack_quant(h->b, wts->b, wts->b_scales, wts->b_zeros, 4, c.d_out, c.rank, s);
+      e = launch_repack_quant(av, w.a, w.a_scales, w.a_zeros, 4, c.rank, c.d_in, s, a_nt);
+      if (e == cudaSuccess) e = launch_repack_quant(bv, w.b, w.b_scales, w.b_zeros, 4, d_out_i, c.rank, s, b_nt);
     } else {
-      e = launch_repack_q8(h->a, wts->a, wts->a_scales, wts->a_zeros, c.rank, c.d_in, s);
-      if (e == cudaSuccess) e = launch_repack_q8(h->b, wts->b, wts->b_scales, wts->b_zeros, c.d_out, c.rank, s);
+      e = launch_repack_q8(av, w.a, w.a_scales, w.a_zeros, c.rank, c.d_in, s, a_nt);
+      if (e == cudaSuccess) e = launch_repack_q8(bv, w.b, w.b_scales, w.b_zeros, d_out_i, c.rank, s, b_nt);
     }
   }
   if (e != cudaSuccess) return fail(EORA_ERR_CUDA);
-  if (prefill_init(h) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (!fused && prefill_init(h) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (fused && !decode_supported(h, 1)) return fail(EORA_ERR_UNSUPPORTED);
   if (cudaStreamSynchronize(s) != cudaSuccess) return fail(EORA_ERR_CUDA);
   *out = obj;
+  return EORA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights* wts, void* stream, eora_linear_t* out) {
+  return create_impl(cfg, wts, 1, stream, out);
+}
+
+int eora_linear_create_fused(const eora_linear_config* cfgs, const eora_linear_weights* wts, int32_t n_layers, void* stream,
+                             eora_linear_t* out) {
+  return create_impl(cfgs, wts, n_layers, stream, out);
+}
+
+int eora_linear_forward_fused(eora_linear_t obj, const void* x, int32_t m, void* const* ys, void* stream) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (m == 0) return EORA_OK;
+  if (m < 0) return EORA_ERR_BAD_SHAPE;
+  if (!x || !ys) return EORA_ERR_NULL_ARG;
+  Handle* h = &obj->h;
+  if (!aligned16(x)) return EORA_ERR_MISALIGNED;
+  for (int i = 0; i < h->n_sub; ++i) {
+    if (!ys[i]) return EORA_ERR_NULL_ARG;
+    if (!aligned16(ys[i])) return EORA_ERR_MISALIGNED;
+  }
+  if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  if (!decode_supported(h, m)) return EORA_ERR_UNSUPPORTED;
+  return launch_decode_forward(h, x, m, ys, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
+}
+
+int eora_linear_forward_fused_host(eora_linear_t obj, const void* x_host, int32_t m, void* const* ys_host, void* stream) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (m == 0) return EORA_OK;
+  if (m < 0) return EORA_ERR_BAD_SHAPE;
+  if (!x_host || !ys_host) return EORA_ERR_NULL_ARG;
+  Handle* h = &obj->h;
+  for (int i = 0; i < h->n_sub; ++i)
+    if (!ys_host[i]) return EORA_ERR_NULL_ARG;
+  if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const size_t eb = y_elem_bytes(h->cfg.y_dtype);
+  if (cudaMemcpyAsync(h->x_stage, x_host, (size_t)m * h->cfg.d_in * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return EORA_ERR_CUDA;
+  void* ys[4] = {nullptr, nullptr, nullptr, nullptr};
+  size_t off = 0;
+  for (int i = 0; i < h->n_sub; ++i) {          // outputs side by side in the staging buffer ([m][d_out_i] each)
+    ys[i] = reinterpret_cast<char*>(h->y_stage) + off;
+    off += (size_t)m * h->sub_dout[i] * eb;
+  }
+  int rc = eora_linear_forward_fused(obj, h->x_stage, m, ys, stream);
+  if (rc != EORA_OK) return rc;
+  for (int i = 0; i < h->n_sub; ++i)
+    if (cudaMemcpyAsync(ys_host[i], ys[i], (size_t)m * h->sub_dout[i] * eb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EORA_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return EORA_ERR_CUDA;
   return EORA_OK;
 }
 
@@ -226,11 +329,13 @@ int eora_linear_forward(eora_linear_t obj, const void* x, int32_t m, void* y, vo
   if (!x || !y) return EORA_ERR_NULL_ARG;
   if (!aligned16(x) || !aligned16(y)) return EORA_ERR_MISALIGNED;
   Handle* h = &obj->h;
+  if (h->n_sub != 1) return EORA_ERR_UNSUPPORTED;             // fused layers have several outputs: forward_fused
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   int p = pick_path(h, m);
   cudaError_t e;
-  if (p == EORA_PATH_DECODE) e = launch_decode_forward(h, x, m, y, s);
+  void* ys[1] = {y};
+  if (p == EORA_PATH_DECODE) e = launch_decode_forward(h, x, m, ys, s);
   else if (p == EORA_PATH_PREFILL) e = launch_prefill_forward(h, x, m, y, s);
   else e = launch_generic_forward(h, x, m, y, s);
   return e == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;

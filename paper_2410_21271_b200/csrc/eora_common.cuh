@@ -153,31 +153,38 @@ struct Handle {
   float* t_ws;           // [max_m][r_pad] fp32 split-K sums of t (prefill); zero between calls
   float* t_gen;          // [max_m][r_pad] fp32, simple kernels only
   __half* t16;           // [max_m][r_pad] fp16 (prefill)
-  float* d_t;            // [8][r_pad] fp32 sums of t (decode); zero between calls
+  float* d_t;            // [8][t_cols] fp32 sums of t (decode); zero between calls
   float* y_ws;           // [8][d_out] fp32 sums of y (decode); zero between calls
   uint32_t* counters;    // decode: [0] blobs of A done, [1] row tiles finished, [2 + tile] blobs of that row tile done
   int* dev_status;       // latched device status
   void* x_stage;         // [max_m][d_in] staging for forward_host
   void* y_stage;         // [max_m][d_out]
   int sm_count;
+  // Fused layers (several layers that read the same X, e.g. q/k/v): their backbones and B's are stacked
+  // along the output axis (sub i owns row tiles [sub_tile0[i], sub_tile0[i+1])), their A's along the rank
+  // axis (sub i owns columns [i * r_pad, (i+1) * r_pad) of t).  n_sub == 1 for a plain layer.
+  int n_sub;
+  int sub_tile0[5];
+  int sub_dout[4];
+  int t_cols;            // columns of t: n_sub * r_pad
   void* prefill_state;   // owned by prefill.cu (tensor maps), may be NULL
   void* trace;           // optional caller-owned timestamp buffer, may be NULL
 };
 
 // kernels / launchers implemented in the other translation units ------------------------------
 cudaError_t launch_repack_quant(const WMat& dst, const void* codes, const void* scales, const void* zeros,
-                                int bits, int rows_src, int k_src, cudaStream_t st);
+                                int bits, int rows_src, int k_src, cudaStream_t st, int nt_sub = -1);
 cudaError_t launch_repack_q8(const WMat& dst, const void* codes, const void* scales, const void* zeros,
-                             int rows_src, int k_src, cudaStream_t st);
-cudaError_t launch_repack_f16(const WMat& dst, const void* src, int rows_src, int k_src, cudaStream_t st);
+                             int rows_src, int k_src, cudaStream_t st, int nt_sub = -1);
+cudaError_t launch_repack_f16(const WMat& dst, const void* src, int rows_src, int k_src, cudaStream_t st, int nt_sub = -1);
 cudaError_t launch_repack_sp24(const WMat& dst, const void* values, const void* meta, int rows_src, int k_src,
-                               cudaStream_t st);
+                               cudaStream_t st, int nt_sub = -1);
 cudaError_t launch_dump(const Handle* h, int what, void* out, cudaStream_t st);
 cudaError_t launch_generic_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
 int generic_launch_count(const Handle* h);
 
 bool decode_supported(const Handle* h, int m);
-cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
+cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st);
 int decode_launch_count(const Handle* h, int m);
 int decode_grid(const Handle* h, int m);
 

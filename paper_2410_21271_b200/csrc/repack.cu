@@ -41,8 +41,8 @@ __device__ inline uint32_t padded_code(const uint32_t* codes, const uint32_t* ze
   return src_code(codes, bits, k, n, rows_src);
 }
 
-__global__ void k_repack_q4(WMat d, const uint32_t* codes, const uint32_t* zeros, int rows_src, int k_src, int ldz) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
+__global__ void k_repack_q4(WMat d, int nt_sub, const uint32_t* codes, const uint32_t* zeros, int rows_src, int k_src, int ldz) {
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
     uint32_t out[4];
@@ -58,8 +58,8 @@ __global__ void k_repack_q4(WMat d, const uint32_t* codes, const uint32_t* zeros
   }
 }
 
-__global__ void k_repack_q3(WMat d, const uint32_t* codes, const uint32_t* zeros, int rows_src, int k_src, int ldz) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
+__global__ void k_repack_q3(WMat d, int nt_sub, const uint32_t* codes, const uint32_t* zeros, int rows_src, int k_src, int ldz) {
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
     uint32_t wd[3] = {0, 0, 0};
@@ -83,8 +83,8 @@ __global__ void k_repack_q3(WMat d, const uint32_t* codes, const uint32_t* zeros
   }
 }
 
-__global__ void k_repack_q8(WMat d, const uint8_t* codes, const uint8_t* zeros, int rows_src, int k_src) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
+__global__ void k_repack_q8(WMat d, int nt_sub, const uint8_t* codes, const uint8_t* zeros, int rows_src, int k_src) {
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
     uint8_t* tb = const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c));
@@ -105,8 +105,8 @@ __global__ void k_repack_q8(WMat d, const uint8_t* codes, const uint8_t* zeros, 
 }
 
 // src element (k, n) at src[k * rows_src + n]  ([reduction][rows] row-major, as A [K][r] and B [r][N])
-__global__ void k_repack_f16(WMat d, const __half* src, int rows_src, int k_src) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
+__global__ void k_repack_f16(WMat d, int nt_sub, const __half* src, int rows_src, int k_src) {
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
     uint8_t* tb = const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c));
@@ -122,8 +122,8 @@ __global__ void k_repack_f16(WMat d, const __half* src, int rows_src, int k_src)
   }
 }
 
-__global__ void k_repack_sp24(WMat d, const __half* values, const uint32_t* meta, int rows_src, int k_src) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
+__global__ void k_repack_sp24(WMat d, int nt_sub, const __half* values, const uint32_t* meta, int rows_src, int k_src) {
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
   for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
     Pos p = pos_of(idx, d.kc);
     uint8_t* tb = const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c));
@@ -148,9 +148,9 @@ __global__ void k_repack_sp24(WMat d, const __half* values, const uint32_t* meta
 
 // Scale entries.  scales fp16 [G][rows_src]; zeros packed stream.  One thread per (k-tile c, row tile, g);
 // the entry of k-tile c is written once per blob (by the even tile when the pair shares one entry).
-__global__ void k_repack_sz(WMat d, const __half* scales, const uint32_t* zeros, int bits, int rows_src, int ldz,
+__global__ void k_repack_sz(WMat d, int nt_sub, const __half* scales, const uint32_t* zeros, int bits, int rows_src, int ldz,
                             int ng_src) {
-  int total = d.nt * d.kc * 8;
+  int total = nt_sub * d.kc * 8;
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
     int g = idx & 7, c = (idx >> 3) % d.kc, tile = (idx >> 3) / d.kc;
     if (!d.sz2 && (c & 1)) continue;
@@ -173,8 +173,8 @@ __global__ void k_repack_sz(WMat d, const __half* scales, const uint32_t* zeros,
   }
 }
 
-__global__ void k_repack_sz_q8(WMat d, const __half* scales, const uint8_t* zeros, int rows_src) {
-  int total = d.nt * d.kc * 8;   // one group: every pair carries a copy
+__global__ void k_repack_sz_q8(WMat d, int nt_sub, const __half* scales, const uint8_t* zeros, int rows_src) {
+  int total = nt_sub * d.kc * 8;   // one group: every pair carries a copy
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
     int g = idx & 7, c = (idx >> 3) % d.kc, tile = (idx >> 3) / d.kc;
     if (!d.sz2 && (c & 1)) continue;
@@ -201,38 +201,45 @@ inline int grid_for(int64_t total, int block) {
 
 }  // namespace
 
+// All launchers fill the first nt_sub row tiles of `d` (nt_sub < 0: all of them).  To fill row tiles
+// [t0, t0 + n) of a larger matrix pass a copy of its WMat whose q points at row tile t0 and nt_sub = n.
 cudaError_t launch_repack_quant(const WMat& d, const void* codes, const void* scales, const void* zeros, int bits,
-                                int rows_src, int k_src, cudaStream_t st) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
+                                int rows_src, int k_src, cudaStream_t st, int nt_sub) {
+  if (nt_sub < 0) nt_sub = d.nt;
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
   int ldz = bits * rows_src / 32;
   int ng_src = k_src / d.group;
+  if (ng_src < 1) ng_src = 1;
   if (bits == 4)
-    k_repack_q4<<<grid_for(total, 256), 256, 0, st>>>(d, (const uint32_t*)codes, (const uint32_t*)zeros, rows_src, k_src, ldz);
+    k_repack_q4<<<grid_for(total, 256), 256, 0, st>>>(d, nt_sub, (const uint32_t*)codes, (const uint32_t*)zeros, rows_src, k_src, ldz);
   else
-    k_repack_q3<<<grid_for(total, 256), 256, 0, st>>>(d, (const uint32_t*)codes, (const uint32_t*)zeros, rows_src, k_src, ldz);
-  k_repack_sz<<<grid_for((int64_t)d.nt * d.kc * 8, 256), 256, 0, st>>>(d, (const __half*)scales, (const uint32_t*)zeros, bits,
-                                                                     rows_src, ldz, ng_src);
+    k_repack_q3<<<grid_for(total, 256), 256, 0, st>>>(d, nt_sub, (const uint32_t*)codes, (const uint32_t*)zeros, rows_src, k_src, ldz);
+  k_repack_sz<<<grid_for((int64_t)nt_sub * d.kc * 8, 256), 256, 0, st>>>(d, nt_sub, (const __half*)scales, (const uint32_t*)zeros, bits,
+                                                                        rows_src, ldz, ng_src);
   return cudaGetLastError();
 }
 
 cudaError_t launch_repack_q8(const WMat& d, const void* codes, const void* scales, const void* zeros, int rows_src,
-                             int k_src, cudaStream_t st) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
-  k_repack_q8<<<grid_for(total, 256), 256, 0, st>>>(d, (const uint8_t*)codes, (const uint8_t*)zeros, rows_src, k_src);
-  k_repack_sz_q8<<<grid_for((int64_t)d.nt * d.kc * 8, 256), 256, 0, st>>>(d, (const __half*)scales, (const uint8_t*)zeros, rows_src);
+                             int k_src, cudaStream_t st, int nt_sub) {
+  if (nt_sub < 0) nt_sub = d.nt;
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
+  k_repack_q8<<<grid_for(total, 256), 256, 0, st>>>(d, nt_sub, (const uint8_t*)codes, (const uint8_t*)zeros, rows_src, k_src);
+  k_repack_sz_q8<<<grid_for((int64_t)nt_sub * d.kc * 8, 256), 256, 0, st>>>(d, nt_sub, (const __half*)scales, (const uint8_t*)zeros, rows_src);
   return cudaGetLastError();
 }
 
-cudaError_t launch_repack_f16(const WMat& d, const void* src, int rows_src, int k_src, cudaStream_t st) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
-  k_repack_f16<<<grid_for(total, 256), 256, 0, st>>>(d, (const __half*)src, rows_src, k_src);
+cudaError_t launch_repack_f16(const WMat& d, const void* src, int rows_src, int k_src, cudaStream_t st, int nt_sub) {
+  if (nt_sub < 0) nt_sub = d.nt;
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
+  k_repack_f16<<<grid_for(total, 256), 256, 0, st>>>(d, nt_sub, (const __half*)src, rows_src, k_src);
   return cudaGetLastError();
 }
 
 cudaError_t launch_repack_sp24(const WMat& d, const void* values, const void* meta, int rows_src, int k_src,
-                               cudaStream_t st) {
-  int64_t total = (int64_t)d.nt * d.kc * 32;
-  k_repack_sp24<<<grid_for(total, 256), 256, 0, st>>>(d, (const __half*)values, (const uint32_t*)meta, rows_src, k_src);
+                               cudaStream_t st, int nt_sub) {
+  if (nt_sub < 0) nt_sub = d.nt;
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
+  k_repack_sp24<<<grid_for(total, 256), 256, 0, st>>>(d, nt_sub, (const __half*)values, (const uint32_t*)meta, rows_src, k_src);
   return cudaGetLastError();
 }
 

@@ -1,0 +1,86 @@
+"""GPU parity of the fused-layer entry points (several layers that read the same X behind one handle and one
+launch): every output is compared with the CPU oracle's forward of its own layer, and with the plain
+per-layer handle.  Tolerances as in the other parity tests."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+from oracle import eora_oracle as orc
+import eora_inputs as gen
+import paper_2410_21271_b200 as eora
+from helpers import make_case, check_parity, x_to_torch
+
+SHAPES = gen.LLAMA3_8B_SHAPES
+
+
+def run_fused(F, x, xd):
+    import torch
+    ys = F.forward(x_to_torch(x, xd))
+    torch.cuda.synchronize()
+    assert F.device_status() == 0
+    return [y.float().cpu().numpy().astype(np.float64) for y in ys]
+
+
+CASES = [
+    # w, ab, K, [N...], r, M, x dtype
+    ("q4", "f16", 256, [64, 32], 64, 1, "f16"),
+    ("q3", "f16", 512, [96, 32, 64], 128, 3, "f16"),
+    ("q4", "q4", 512, [96, 160], 128, 8, "f16"),
+    ("q4", "q8", 384, [64, 64, 32, 96], 40, 5, "bf16"),
+    ("q3", "f16", 1024, [224, 96], 0, 2, "f16"),
+    ("q3", "f16", 640, [160, 352], 256, 19, "f16"),          # three passes of eight tokens
+]
+
+
+@pytest.mark.parametrize("w,ab,K,Ns,r,M,xd", CASES)
+def test_fused_matches_oracle_small(w, ab, K, Ns, r, M, xd):
+    layers = [make_case(50 + i, K, N, r, w=w, ab=ab) for i, N in enumerate(Ns)]
+    x = gen.make_x(51, M, K, xd)
+    F = eora.FusedLayers(layers, max_m=M, x_dtype=xd)
+    assert F.launches(M) == (M + 7) // 8
+    for rep in range(2):                                   # second call: the scratch was restored
+        ys = run_fused(F, x, xd)
+        for i, (wf, af, bf) in enumerate(layers):
+            check_parity(ys[i], orc.forward(x, xd, wf, af, bf), f"layer {i} call {rep}")
+    F.close()
+
+
+@pytest.mark.parametrize("names,w", [(("q", "k", "v"), "q3"), (("gate", "up"), "q3"), (("q", "k", "v"), "q4")])
+def test_fused_fullsize(names, w):
+    K = SHAPES[names[0]][0]
+    layers = [make_case(60 + i, K, SHAPES[nm][1], 128, w=w) for i, nm in enumerate(names)]
+    x = gen.make_x(61, 1, K)
+    F = eora.FusedLayers(layers, max_m=1)
+    ys = run_fused(F, x, "f16")
+    for i, (wf, af, bf) in enumerate(layers):
+        rel, _ = check_parity(ys[i], orc.forward(x, "f16", wf, af, bf), names[i])
+        assert 5e-5 < rel < 1e-3
+    F.close()
+
+
+def test_fused_argument_errors():
+    import torch
+    K = 256
+    la = make_case(70, K, 64, 64)
+    lb = make_case(71, K, 32, 64)
+    lc = make_case(72, K, 32, 128)                         # other rank
+    ld = make_case(73, 512, 32, 64)                        # other d_in
+    m = dict(max_m=4, x_dtype="f16", y_dtype="f16", kernel_policy=eora.EORA_POLICY_AUTO, device="cuda:0")
+    def status(ls, **kw):
+        mm = dict(m); mm.update(kw)
+        parts = [eora._marshal(*l, **mm) for l in ls]
+        return eora.eora_linear_create_fused([p[0] for p in parts], [p[1] for p in parts], check=False)
+    assert status([la, lb]) == eora.EORA_OK
+    assert status([la, lc]) == eora.EORA_ERR_BAD_SHAPE
+    assert status([la, ld]) == eora.EORA_ERR_BAD_SHAPE
+    assert status([la, lb], max_m=65) == eora.EORA_ERR_UNSUPPORTED
+    assert status([la] * 5) == eora.EORA_ERR_BAD_SHAPE
+    F = eora.FusedLayers([la, lb], max_m=4)
+    x = torch.zeros((4, K), dtype=torch.float16, device="cuda:0")
+    y = torch.zeros((4, 96), dtype=torch.float16, device="cuda:0")
+    assert eora.eora_linear_forward(F.handle, x, 1, y, check=False) == eora.EORA_ERR_UNSUPPORTED
+    assert eora.eora_linear_forward_fused(F.handle, x, 5, [y, y], check=False) == eora.EORA_ERR_M_TOO_LARGE
+    assert eora.eora_linear_forward_fused(F.handle, x, 1, [y, None], check=False) == eora.EORA_ERR_NULL_ARG
+    torch.cuda.synchronize()
+    F.close()
