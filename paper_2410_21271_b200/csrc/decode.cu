@@ -36,7 +36,8 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kCtasPerSm = 4;
 constexpr int kRing = 3;                  // bulk copies in flight per warp
 constexpr int kSlotBytes = 4352;          // one ring slot = one bulk copy (a run of whole blobs)
-constexpr int kSmemBytes = kWarps * kRing * kSlotBytes + kWarps * kRing * 8;
+constexpr int kBarBytes = 128;            // kWarps * kRing mbarriers
+constexpr int kSmemBytes = kWarps * kRing * kSlotBytes + kBarBytes + kSp24LutBytes;
 
 enum { CNT_A_DONE = 0, CNT_TILES_DONE = 1, CNT_TICKET0 = 2 };
 
@@ -147,6 +148,7 @@ struct Ring {
   int slot;
   uint32_t parity;
   int deferred;             // slots [kRing - deferred, kRing) have not had their first copy requested yet
+  uint32_t aux;             // shared-memory address of the 2:4 expansion table (2:4 backbone only)
 };
 
 __device__ __forceinline__ void ring_issue(Ring& r, int slot, int lane) {
@@ -286,7 +288,7 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
 #pragma unroll 2
       for (uint32_t j = 0; j < cn; ++j) {
         float tot[4];
-        blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot);
+        blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
         if constexpr (OUT == OUT_T) {
           flush_sums(p.d_t, p.r_pad, tile, tot, p.m, lane);
           ++flushed;
@@ -342,6 +344,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   r.slots = smem + warp * (kRing * kSlotBytes);
   r.bars = reinterpret_cast<uint64_t*>(smem + kWarps * kRing * kSlotBytes) + warp * kRing;
   r.slot = 0; r.parity = 0; r.pseg = 0;
+  r.aux = 0;
+  if constexpr (WF == FMT_SP24) {
+    // every warp writes the same 16 values, so no CTA-wide barrier is needed before a warp reads them
+    uint32_t* lut = reinterpret_cast<uint32_t*>(smem + kWarps * kRing * kSlotBytes + kBarBytes);
+    if (lane < 16) lut[lane] = sp24_selectors((uint32_t)lane);
+    r.aux = smem_u32(lut);
+  }
   if (lane == 0) {
 #pragma unroll
     for (int i = 0; i < kRing; ++i) mbar_init(r.bars + i, 1);
@@ -425,6 +434,7 @@ double blob_cost(int fmt, bool hilo) {
     case FMT_Q4: return 1.05;
     case FMT_Q8: return 1.40;
     case FMT_F16: return hilo ? 1.30 : 1.10;
+    case FMT_SP24: return 1.60;
     default: return 0.0;
   }
 }
@@ -445,7 +455,7 @@ uint32_t blobs_per_copy(const WMat& m) {
 
 bool decode_supported(const Handle* h, int m) {
   if (m < 1 || m > 64) return false;
-  if (h->w.fmt != FMT_Q4 && h->w.fmt != FMT_Q3) return false;
+  if (h->w.fmt != FMT_Q4 && h->w.fmt != FMT_Q3 && h->w.fmt != FMT_SP24) return false;
   if (h->w.blob > kSlotBytes) return false;
   if (h->cfg.rank > 0 && (h->a.blob > kSlotBytes || h->b.blob > kSlotBytes)) return false;
   return true;
@@ -534,7 +544,8 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
     a.m = m - m0 < 8 ? m - m0 : 8;
     a.x = reinterpret_cast<const uint8_t*>(x) + (size_t)m0 * h->cfg.d_in * 2;
     for (int i = 0; i < h->n_sub; ++i) a.ys[i] = reinterpret_cast<uint8_t*>(ys[i]) + (size_t)m0 * h->sub_dout[i] * ybytes;
-    cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf) : launch_ab<FMT_Q3>(cfg, a, abf);
+    cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf)
+                  : h->w.fmt == FMT_Q3 ? launch_ab<FMT_Q3>(cfg, a, abf) : launch_ab<FMT_SP24>(cfg, a, abf);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

@@ -148,8 +148,30 @@ template <int FMT> constexpr bool is_quant() { return FMT == FMT_Q4 || FMT == FM
 
 // Build the A-operand registers of the four mma of one tile from its blob in shared memory.
 // a[i][*]: mma i = 2*blk + sub; entries are fp16x2.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+
+// 2:4 expansion table: for the position nibble p0 | p1 << 2 of a quad, the two byte-permute selectors that
+// spread the quad's two kept fp16 values (one register) over its four positions (two registers), zero
+// elsewhere.  Low half: selector of positions (0, 1), high half: of positions (2, 3).  Selector bytes: 0x10 =
+// first value, 0x32 = second value, 0x44 = zero (the permute's other operand).
+__host__ __device__ constexpr uint32_t sp24_selectors(uint32_t nib) {
+  const uint32_t p0 = nib & 3u, p1 = nib >> 2;
+  uint32_t r = 0;
+  for (uint32_t e = 0; e < 4; ++e) {
+    const uint32_t sel = e == p0 ? 0x10u : e == p1 ? 0x32u : 0x44u;
+    r |= sel << (8 * e);
+  }
+  return r;
+}
+constexpr int kSp24LutBytes = 64;       // 16 entries; every entry in its own shared-memory bank
+
+// `aux`: shared-memory address (32-bit, shared window) of the 2:4 expansion table; unused by other formats.
 template <int FMT>
-__device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const ZC& zc, uint32_t (&a)[4][4]) {
+__device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const ZC& zc, uint32_t (&a)[4][4], uint32_t aux = 0) {
   if constexpr (FMT == FMT_Q4) {
     const uint4 v = *reinterpret_cast<const uint4*>(blob + lane * 16);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -211,6 +233,24 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
       a[blk * 2 + 1][hf] = u.z;
       a[blk * 2 + 1][hf + 2] = u.w;
     }
+  } else if constexpr (FMT == FMT_SP24) {
+    const uint32_t meta = *reinterpret_cast<const uint32_t*>(blob + 1024 + lane * 4);
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+      const uint4 u = *reinterpret_cast<const uint4*>(blob + blk * 512 + lane * 16);
+      const uint32_t vv[2][2] = {{u.x, u.y}, {u.z, u.w}};       // [hf][quad]: the quad's two kept values
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+        for (int quad = 0; quad < 2; ++quad) {
+          const uint32_t nib = (meta >> (8 * (blk * 2 + hf) + 4 * quad)) & 15u;
+          uint32_t sel;
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(sel) : "r"(aux + nib * 4));
+          a[blk * 2 + quad][hf] = prmt(vv[hf][quad], 0u, sel);
+          a[blk * 2 + quad][hf + 2] = prmt(vv[hf][quad], 0u, sel >> 16);
+        }
+      }
+    }
   }
 }
 
@@ -219,7 +259,7 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
 // entries of the 16 x 8 result: rows g / g + 8, tokens 2t / 2t + 1).
 template <int FMT, bool HILO>
 __device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint32_t sz2, const uint32_t (&xr)[16],
-                                             const uint32_t (&xl)[16], float (&tot)[4]) {
+                                             const uint32_t (&xl)[16], float (&tot)[4], uint32_t aux = 0) {
   constexpr int tb = tile_bytes(FMT);
   constexpr bool quant = fmt_quantised(FMT);
   const int g = lane >> 2;
@@ -244,7 +284,7 @@ __device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint
       }
     }
     uint32_t a[4][4];
-    tile_frags<FMT>(blob + c * tb, lane, zc, a);
+    tile_frags<FMT>(blob + c * tb, lane, zc, a, aux);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       mma16816(acc[i & 1], a[i], xr[8 * c + 2 * i], xr[8 * c + 2 * i + 1]);

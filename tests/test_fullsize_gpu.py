@@ -106,6 +106,7 @@ def test_sparse24_fullsize(name, M):
     x = gen.make_x(42, M, K)
     L = eora.Layer(wf, af, bf, max_m=M)
     if M == 1:
+        assert L.path(M) == eora.EORA_PATH_DECODE
         check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} sp24 M1")
     else:
         assert L.path(M) == eora.EORA_PATH_PREFILL

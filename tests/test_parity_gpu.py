@@ -40,6 +40,21 @@ def test_adapter_storage_bit_exact(ab, r):
     L.close()
 
 
+def test_sparse24_one_hot_rows_through_the_fast_path():
+    """X = e_k, rank 0, fp32 output: the decode kernel's own expansion of the 2:4 tiles, bit for bit."""
+    K, N = 512, 96
+    wf, _, _ = make_case(14, K, N, 0, w="sp24")
+    ks = [0, 1, 2, 3, 5, 63, 64, 130, 257, 511]
+    x = np.zeros((len(ks), K), dtype=np.float16)
+    for i, k in enumerate(ks):
+        x[i, k] = 1.0
+    L = eora.Layer(wf, None, None, max_m=len(ks), y_dtype="f32")
+    assert L.path(len(ks)) == eora.EORA_PATH_DECODE
+    y = run_layer(L, x, "f16")
+    assert np.array_equal(y, orc.dequant_matrix(wf)[ks])
+    L.close()
+
+
 def test_sparse24_expansion_bit_exact():
     K, N = 256, 64
     wf, _, _ = make_case(13, K, N, 0, w="sp24")
@@ -63,6 +78,9 @@ SMALL = [
     ("q4", "q8", 256, 64, 40, 2, "f16"),
     ("sp24", "f16", 512, 96, 128, 1, "f16"),
     ("sp24", "f16", 256, 64, 64, 9, "bf16"),
+    ("sp24", "q4", 512, 160, 128, 8, "f16"),
+    ("sp24", "q8", 384, 96, 40, 3, "f16"),
+    ("sp24", "f16", 1024, 352, 0, 1, "f16"),
     ("q4", "f16", 1152, 352, 128, 63, "f16"),
     ("q3", "f16", 1152, 352, 128, 65, "f16"),
     ("q4", "f16", 640, 160, 64, 200, "f16"),
