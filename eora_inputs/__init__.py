@@ -122,14 +122,18 @@ def rtn_quantize(mat: np.ndarray, bits: int, group: int) -> dict:
     return {"q": q.reshape(rows, cols).astype(np.int64), "scales": s, "z": z.astype(np.int64)}
 
 
-def quantize_matrix_4bit(mat: np.ndarray, group: int) -> dict:
-    """fp16 [rows][cols] -> 4-bit group-wise interchange format (groups along rows)."""
+def quantize_matrix_bits(mat: np.ndarray, bits: int, group: int) -> dict:
+    """fp16 [rows][cols] -> b-bit (3 or 4) group-wise interchange format (groups along rows)."""
     rows, cols = mat.shape
     g = min(group, rows)
-    r = rtn_quantize(mat, 4, g)
-    return {"kind": "quant", "bits": 4, "group": g, "rows": rows, "cols": cols,
-            "codes": pack_stream(r["q"], 4), "scales": r["scales"],
-            "zeros": np.ascontiguousarray(pack_stream(np.ascontiguousarray(r["z"].T), 4).T)}
+    r = rtn_quantize(mat, bits, g)
+    return {"kind": "quant", "bits": bits, "group": g, "rows": rows, "cols": cols,
+            "codes": pack_stream(r["q"], bits), "scales": r["scales"],
+            "zeros": np.ascontiguousarray(pack_stream(np.ascontiguousarray(r["z"].T), bits).T)}
+
+
+def quantize_matrix_4bit(mat: np.ndarray, group: int) -> dict:
+    return quantize_matrix_bits(mat, 4, group)
 
 
 def quantize_matrix_8bit(mat: np.ndarray) -> dict:
@@ -141,10 +145,12 @@ def quantize_matrix_8bit(mat: np.ndarray) -> dict:
 
 
 def make_ab_quant(seed: int, K: int, N: int, r: int, ab_format: str, group: int = 128) -> tuple[dict, dict]:
-    """Quantised adapter derived from the seeded fp16 one.  ab_format: 'q4' or 'q8'."""
+    """Quantised adapter derived from the seeded fp16 one.  ab_format: 'q4', 'q3' (group-wise) or 'q8'."""
     a16, b16 = make_ab_f16(seed, K, N, r)
     if ab_format == "q4":
         return quantize_matrix_4bit(a16["data"], group), quantize_matrix_4bit(b16["data"], group)
+    if ab_format == "q3":
+        return quantize_matrix_bits(a16["data"], 3, group), quantize_matrix_bits(b16["data"], 3, group)
     if ab_format == "q8":
         return quantize_matrix_8bit(a16["data"]), quantize_matrix_8bit(b16["data"])
     raise ValueError(ab_format)

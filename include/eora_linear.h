@@ -63,7 +63,7 @@ enum {
 };
 
 enum { EORA_W_QUANT = 0, EORA_W_SPARSE24 = 1 };
-enum { EORA_AB_F16 = 0, EORA_AB_Q4 = 1, EORA_AB_Q8 = 2 };
+enum { EORA_AB_F16 = 0, EORA_AB_Q4 = 1, EORA_AB_Q8 = 2, EORA_AB_Q3 = 3 };
 enum { EORA_X_F16 = 0, EORA_X_BF16 = 1 };
 enum { EORA_Y_F16 = 0, EORA_Y_BF16 = 1, EORA_Y_F32 = 2 };
 /* kernel families reported by eora_linear_path */
@@ -79,8 +79,8 @@ typedef struct {
   int32_t w_format;    /* EORA_W_QUANT or EORA_W_SPARSE24 */
   int32_t w_bits;      /* 3 or 4 (EORA_W_QUANT) */
   int32_t w_group;     /* group size along d_in: multiple of 64 dividing d_in (d_in = channel-wise) */
-  int32_t ab_format;   /* EORA_AB_F16 / EORA_AB_Q4 / EORA_AB_Q8 */
-  int32_t ab_group;    /* group size for EORA_AB_Q4 (128); B uses min(ab_group, rank) */
+  int32_t ab_format;   /* EORA_AB_F16 / EORA_AB_Q4 / EORA_AB_Q8 / EORA_AB_Q3 */
+  int32_t ab_group;    /* group size for EORA_AB_Q4 / _Q3 (128); B uses min(ab_group, rank) */
   int32_t x_dtype;     /* EORA_X_F16 or EORA_X_BF16 */
   int32_t y_dtype;     /* EORA_Y_F16, EORA_Y_BF16 or EORA_Y_F32 */
   int32_t max_m;       /* largest M forward will be called with (sizes the scratch memory) */

@@ -19,7 +19,7 @@ EORA_OK = 0
 EORA_ERR_NULL_ARG, EORA_ERR_BAD_SHAPE, EORA_ERR_UNSUPPORTED, EORA_ERR_MISALIGNED = -1, -2, -3, -4
 EORA_ERR_M_TOO_LARGE, EORA_ERR_CUDA, EORA_ERR_DEVICE_TIMEOUT = -5, -6, -7
 EORA_W_QUANT, EORA_W_SPARSE24 = 0, 1
-EORA_AB_F16, EORA_AB_Q4, EORA_AB_Q8 = 0, 1, 2
+EORA_AB_F16, EORA_AB_Q4, EORA_AB_Q8, EORA_AB_Q3 = 0, 1, 2, 3
 EORA_X_F16, EORA_X_BF16 = 0, 1
 EORA_Y_F16, EORA_Y_BF16, EORA_Y_F32 = 0, 1, 2
 EORA_PATH_GENERIC, EORA_PATH_DECODE, EORA_PATH_PREFILL = 0, 1, 2
@@ -278,7 +278,7 @@ def _marshal(w_fmt: dict, a_fmt, b_fmt, *, max_m: int, x_dtype: str, y_dtype: st
             cfg.rank = a_fmt["data"].shape[1]
             ab = [_dev(a_fmt["data"], device), None, None, _dev(b_fmt["data"], device), None, None]
         elif kind == "quant":
-            cfg.rank, cfg.ab_format, cfg.ab_group = a_fmt["cols"], EORA_AB_Q4, a_fmt["group"]
+            cfg.rank, cfg.ab_format, cfg.ab_group = a_fmt["cols"], {4: EORA_AB_Q4, 3: EORA_AB_Q3}[a_fmt["bits"]], a_fmt["group"]
             ab = [_dev(f[k], device) for f in (a_fmt, b_fmt) for k in ("codes", "scales", "zeros")]
         elif kind == "q8":
             cfg.rank, cfg.ab_format = a_fmt["cols"], EORA_AB_Q8

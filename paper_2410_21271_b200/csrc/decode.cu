@@ -423,6 +423,7 @@ cudaError_t launch_ab(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int
     case FMT_F16: return launch_kernel<k_decode<WF, FMT_F16>>(cfg, args);
     case FMT_Q4: return launch_kernel<k_decode<WF, FMT_Q4>>(cfg, args);
     case FMT_Q8: return launch_kernel<k_decode<WF, FMT_Q8>>(cfg, args);
+    case FMT_Q3: return launch_kernel<k_decode<WF, FMT_Q3>>(cfg, args);
     default: return launch_kernel<k_decode<WF, FMT_NONE>>(cfg, args);
   }
 }

@@ -53,8 +53,9 @@ int check_config(const eora_linear_config& c) {
   } else if (c.w_format != EORA_W_SPARSE24) {
     return EORA_ERR_UNSUPPORTED;
   }
-  if (c.ab_format != EORA_AB_F16 && c.ab_format != EORA_AB_Q4 && c.ab_format != EORA_AB_Q8) return EORA_ERR_UNSUPPORTED;
-  if (c.rank > 0 && c.ab_format == EORA_AB_Q4) {
+  if (c.ab_format != EORA_AB_F16 && c.ab_format != EORA_AB_Q4 && c.ab_format != EORA_AB_Q8 && c.ab_format != EORA_AB_Q3)
+    return EORA_ERR_UNSUPPORTED;
+  if (c.rank > 0 && (c.ab_format == EORA_AB_Q4 || c.ab_format == EORA_AB_Q3)) {
     if (c.rank % 64 || c.ab_group <= 0 || c.ab_group % 64 || c.d_in % c.ab_group) return EORA_ERR_BAD_SHAPE;
     int gb = c.ab_group < c.rank ? c.ab_group : c.rank;
     if (c.rank % gb) return EORA_ERR_BAD_SHAPE;
@@ -170,11 +171,12 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     h->sub_tile0[i + 1] = h->sub_tile0[i] + cfgs[i].d_out / 16;
   }
   for (int i = n + 1; i < 5; ++i) h->sub_tile0[i] = h->sub_tile0[n];
-  int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : FMT_Q8;
+  const bool ab_grouped = c.ab_format == EORA_AB_Q4 || c.ab_format == EORA_AB_Q3;
+  int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : c.ab_format == EORA_AB_Q3 ? FMT_Q3 : FMT_Q8;
   wmat_shape(h->w, quant_w ? (c.w_bits == 4 ? FMT_Q4 : FMT_Q3) : FMT_SP24, c.d_out, c.d_in, quant_w ? c.w_group : 0);
   if (c.rank > 0) {
-    int ga = c.ab_format == EORA_AB_Q4 ? c.ab_group : 0;
-    int gb = c.ab_format == EORA_AB_Q4 ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 0;
+    int ga = ab_grouped ? c.ab_group : 0;
+    int gb = ab_grouped ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 0;
     wmat_shape(h->a, ab_fmt, fused ? n * h->r_pad : c.rank, c.d_in, ga);   // fused: layer i owns rows [i r_pad, (i+1) r_pad)
     wmat_shape(h->b, ab_fmt, c.d_out, h->r_pad, gb);
   } else {
@@ -225,9 +227,10 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     if (c.ab_format == EORA_AB_F16) {
       e = launch_repack_f16(av, w.a, c.rank, c.d_in, s, a_nt);
       if (e == cudaSuccess) e = launch_repack_f16(bv, w.b, d_out_i, c.rank, s, b_nt);
-    } else if (c.ab_format == EORA_AB_Q4) {
-      e = launch_repack_quant(av, w.a, w.a_scales, w.a_zeros, 4, c.rank, c.d_in, s, a_nt);
-      if (e == cudaSuccess) e = launch_repack_quant(bv, w.b, w.b_scales, w.b_zeros, 4, d_out_i, c.rank, s, b_nt);
+    } else if (ab_grouped) {
+      const int bits = c.ab_format == EORA_AB_Q4 ? 4 : 3;
+      e = launch_repack_quant(av, w.a, w.a_scales, w.a_zeros, bits, c.rank, c.d_in, s, a_nt);
+      if (e == cudaSuccess) e = launch_repack_quant(bv, w.b, w.b_scales, w.b_zeros, bits, d_out_i, c.rank, s, b_nt);
     } else {
       e = launch_repack_q8(av, w.a, w.a_scales, w.a_zeros, c.rank, c.d_in, s, a_nt);
       if (e == cudaSuccess) e = launch_repack_q8(bv, w.b, w.b_scales, w.b_zeros, d_out_i, c.rank, s, b_nt);

@@ -491,6 +491,7 @@ cudaError_t launch_bf(int bf, dim3 grid, int smem, cudaStream_t st, const CUtens
     case FMT_F16: return launch_p<k_prefill<WF, FMT_F16>>(grid, smem, st, tx, tt, a);
     case FMT_Q4: return launch_p<k_prefill<WF, FMT_Q4>>(grid, smem, st, tx, tt, a);
     case FMT_Q8: return launch_p<k_prefill<WF, FMT_Q8>>(grid, smem, st, tx, tt, a);
+    case FMT_Q3: return launch_p<k_prefill<WF, FMT_Q3>>(grid, smem, st, tx, tt, a);
     default: return launch_p<k_prefill<WF, FMT_NONE>>(grid, smem, st, tx, tt, a);
   }
 }

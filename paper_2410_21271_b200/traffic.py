@@ -25,13 +25,14 @@ def matrix_bytes(kind: str, rows: int, cols: int, *, bits: int = 4, group: int =
 
 
 def adapter_bytes(ab: str, K: int, N: int, r: int, group: int = 128) -> int:
-    """Bytes of A [K][r] plus B [r][N].  ab: 'f16' | 'q4' | 'q8'."""
+    """Bytes of A [K][r] plus B [r][N].  ab: 'f16' | 'q4' | 'q3' | 'q8'."""
     if r == 0:
         return 0
     if ab == "f16":
         return matrix_bytes("f16", K, r) + matrix_bytes("f16", r, N)
-    if ab == "q4":
-        return matrix_bytes("quant", K, r, bits=4, group=group) + matrix_bytes("quant", r, N, bits=4, group=group)
+    if ab in ("q4", "q3"):
+        b = 4 if ab == "q4" else 3
+        return matrix_bytes("quant", K, r, bits=b, group=group) + matrix_bytes("quant", r, N, bits=b, group=group)
     if ab == "q8":
         return matrix_bytes("q8", K, r) + matrix_bytes("q8", r, N)
     raise ValueError(ab)

@@ -300,7 +300,7 @@ def test_3bit_equals_4bit_on_codes_below_8():
     assert np.array_equal(orc.forward(x, "f16", fmts[0], None, None), orc.forward(x, "f16", fmts[1], None, None))
 
 
-@pytest.mark.parametrize("abf", ["q4", "q8"])
+@pytest.mark.parametrize("abf", ["q4", "q3", "q8"])
 def test_quantised_adapter_equals_dense_adapter(abf):
     K, N, r = 256, 64, 128
     wf = gen.make_backbone_quant(31, K, N, 4, 128)
@@ -308,8 +308,9 @@ def test_quantised_adapter_equals_dense_adapter(abf):
     x = gen.make_x(33, 3, K)
     # dense adapter rebuilt element by element from the integer codes of the quantiser itself
     a16, b16 = gen.make_ab_f16(32, K, N, r)
-    if abf == "q4":
-        ra, rb = gen.rtn_quantize(a16["data"], 4, 128), gen.rtn_quantize(b16["data"], 4, 128)
+    if abf in ("q4", "q3"):
+        bits = 4 if abf == "q4" else 3
+        ra, rb = gen.rtn_quantize(a16["data"], bits, 128), gen.rtn_quantize(b16["data"], bits, 128)
         ga, gb = 128, 128
     else:
         ra, rb = gen.rtn_quantize(a16["data"], 8, K), gen.rtn_quantize(b16["data"], 8, r)

@@ -28,7 +28,7 @@ def test_unpack_and_dequant_bit_exact(w, K, N, group):
     L.close()
 
 
-@pytest.mark.parametrize("ab,r", [("f16", 64), ("f16", 24), ("q4", 64), ("q4", 256), ("q8", 64), ("q8", 40)])
+@pytest.mark.parametrize("ab,r", [("f16", 64), ("f16", 24), ("q4", 64), ("q4", 256), ("q8", 64), ("q8", 40), ("q3", 64), ("q3", 256)])
 def test_adapter_storage_bit_exact(ab, r):
     K, N = 256, 96
     wf, af, bf = make_case(12, K, N, r, ab=ab)
@@ -78,6 +78,9 @@ SMALL = [
     ("q4", "q8", 256, 64, 40, 2, "f16"),
     ("sp24", "f16", 512, 96, 128, 1, "f16"),
     ("sp24", "f16", 256, 64, 64, 9, "bf16"),
+    ("q4", "q3", 512, 96, 128, 1, "f16"),
+    ("q3", "q3", 1024, 224, 256, 16, "f16"),
+    ("q4", "q3", 640, 160, 64, 100, "bf16"),
     ("sp24", "q4", 512, 160, 128, 8, "f16"),
     ("sp24", "q8", 384, 96, 40, 3, "f16"),
     ("sp24", "f16", 1024, 352, 0, 1, "f16"),
@@ -100,6 +103,19 @@ def test_forward_matches_oracle_small(policy, w, ab, K, N, r, M, xd):
     # second call on the same handle: scratch state must have been restored
     y2 = run_layer(L, x, xd)
     check_parity(y2, y_ref, "second call")
+    L.close()
+
+
+@pytest.mark.parametrize("w,M", [("q4", 1), ("q3", 5), ("q4", 130)])
+def test_channel_wise_backbone(w, M):
+    """One (scale, zero) per output channel: the group spans the whole reduction axis (the setting of the
+    paper's main tables, Section 4.1)."""
+    K, N, r = 512, 96, 64
+    wf, af, bf = make_case(31, K, N, r, w=w, group=K)
+    x = gen.make_x(32, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    assert L.path(M) != eora.EORA_PATH_GENERIC
+    check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"channel-wise {w} M{M}")
     L.close()
 
 
