@@ -119,12 +119,31 @@ __device__ __forceinline__ void load_t_pair(uint32_t (&xh)[16], uint32_t (&xl)[1
   }
 }
 
-// tot -> sums[token][ld] for rows 16 * tile + {g, g + 8}
-__device__ __forceinline__ void flush_sums(float* sums, int ld, uint32_t tile, const float (&tot)[4], int m, int lane) {
+// red.add under a predicate (no branch: with one token only a quarter of the lanes has something to add,
+// and a divergent branch per blob costs more than the adds).
+__device__ __forceinline__ void red_add_if(float* p, float v, uint32_t pred) {
+  asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q red.global.add.f32 [%0], %1;\n\t}" ::"l"(p), "f"(v), "r"(pred) : "memory");
+}
+
+// Where a lane's partial sums go: sums[token][ld] for rows 16 * tile + {g, g + 8} and tokens {2t, 2t + 1}.
+struct Flush {
+  float* base;              // sums + 2t * ld + g
+  uint32_t ld;
+  uint32_t has0, has1;      // token 2t / 2t + 1 exists
+};
+__device__ __forceinline__ Flush make_flush(float* sums, int ld, int m, int lane) {
   const int g = lane >> 2, t = lane & 3;
-  float* base = sums + (size_t)(2 * t) * ld + tile * 16 + g;
-  if (2 * t < m) { red_add(base, tot[0]); red_add(base + 8, tot[2]); }
-  if (2 * t + 1 < m) { red_add(base + ld, tot[1]); red_add(base + ld + 8, tot[3]); }
+  Flush f;
+  f.base = sums + (size_t)(2 * t) * ld + g;
+  f.ld = (uint32_t)ld;
+  f.has0 = 2 * t < m ? 1u : 0u;
+  f.has1 = 2 * t + 1 < m ? 1u : 0u;
+  return f;
+}
+__device__ __forceinline__ void flush_sums(const Flush& f, uint32_t tile, const float (&tot)[4]) {
+  float* b = f.base + tile * 16;
+  red_add_if(b, tot[0], f.has0); red_add_if(b + 8, tot[2], f.has0);
+  red_add_if(b + f.ld, tot[1], f.has1); red_add_if(b + f.ld + 8, tot[3], f.has1);
 }
 
 __device__ __forceinline__ uint32_t atom_add_acq_rel(uint32_t* p, uint32_t v) {
@@ -235,6 +254,7 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     uint32_t pair = b0 / nt, tile = b0 - pair * nt;
     uint32_t xr[16], xl[16];
     uint32_t sub = 0, sub_end = nt;
+    const Flush fl = OUT == OUT_T ? make_flush(p.d_t, p.r_pad, p.m, lane) : make_flush(p.y_ws, p.n_pad, p.m, lane);
     if constexpr (HILO) {
       // all of A must be in t
       int ok = 1;
@@ -290,11 +310,11 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
         float tot[4];
         blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
         if constexpr (OUT == OUT_T) {
-          flush_sums(p.d_t, p.r_pad, tile, tot, p.m, lane);
+          flush_sums(fl, tile, tot);
           ++flushed;
         } else {
           if (batch_n == 0) batch_tile = tile;
-          flush_sums(p.y_ws, p.n_pad, tile, tot, p.m, lane);
+          flush_sums(fl, tile, tot);
           if (++batch_n == 32) commit_batch();
         }
         if (++tile == nt) {
