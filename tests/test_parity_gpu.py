@@ -106,6 +106,30 @@ def test_forward_matches_oracle_small(policy, w, ab, K, N, r, M, xd):
     L.close()
 
 
+@pytest.mark.parametrize("w,K,group,M", [("q4", 512, 64, 1), ("q3", 512, 64, 9), ("q4", 384, 192, 3), ("q3", 768, 256, 2),
+                                         ("q3", 384, 192, 70), ("q4", 512, 64, 200)])
+def test_group_sizes_other_than_128(w, K, group, M):
+    """Groups of 64 or 192 put two scale entries into a 128-element blob, 256 and more repeat one entry."""
+    N, r = 96, 64
+    wf, af, bf = make_case(33, K, N, r, w=w, group=group)
+    x = gen.make_x(34, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    assert L.path(M) != eora.EORA_PATH_GENERIC
+    check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{w} g{group} M{M}")
+    L.close()
+
+
+def test_large_output_dimension():
+    """A vocabulary-sized layer (d_out = 32064) at M = 1: many row tiles per warp, fp32 output."""
+    K, N, r = 256, 32064, 64
+    wf, af, bf = make_case(35, K, N, r, w="q4")
+    x = gen.make_x(36, 1, K)
+    L = eora.Layer(wf, af, bf, max_m=1, y_dtype="f32")
+    assert L.path(1) == eora.EORA_PATH_DECODE
+    check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), "large N")
+    L.close()
+
+
 @pytest.mark.parametrize("w,M", [("q4", 1), ("q3", 5), ("q4", 130)])
 def test_channel_wise_backbone(w, M):
     """One (scale, zero) per output channel: the group spans the whole reduction axis (the setting of the
