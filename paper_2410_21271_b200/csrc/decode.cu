@@ -244,7 +244,8 @@ __device__ __forceinline__ void finish_row_tile(const DecodeArgs& p, uint32_t ti
 }
 
 // One segment: `n` consecutive blobs of one matrix starting at blob index b0.
-template <int FMT, bool HILO, int OUT>
+// I8: single-token integer inner product (backbone blobs only), see blob_product_i8.
+template <int FMT, bool HILO, int OUT, bool I8 = false>
 __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32_t b0, uint32_t n, uint32_t nt, uint32_t blob_b,
                                             uint32_t per_copy, uint32_t sz2, int lane) {
   if constexpr (FMT == FMT_NONE) {
@@ -253,6 +254,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     if (n == 0) return true;
     uint32_t pair = b0 / nt, tile = b0 - pair * nt;
     uint32_t xr[16], xl[16];
+    XI8 xi;
+    const bool x_bf16 = p.x_dtype == EORA_X_BF16;
     uint32_t sub = 0, sub_end = nt;
     const Flush fl = OUT == OUT_T ? make_flush(p.d_t, p.r_pad, p.m, lane) : make_flush(p.y_ws, p.n_pad, p.m, lane);
     if constexpr (HILO) {
@@ -269,6 +272,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
         if (i < p.n_sub && tile >= p.sub_tile0[i]) sub = i;
       sub_end = p.sub_tile0[sub + 1];
       load_t_pair(xr, xl, p, sub * p.b_np + pair, lane);
+    } else if constexpr (I8) {
+      load_x_i8<FMT>(xi, p.x, x_bf16, pair, lane);
     } else {
       load_x_pair(xr, p, pair, lane);
     }
@@ -308,7 +313,13 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
 #pragma unroll 2
       for (uint32_t j = 0; j < cn; ++j) {
         float tot[4];
-        blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
+        if constexpr (I8) {
+          float t2[2];
+          blob_product_i8<FMT>(src + j * blob_b, lane, sz2, xi, t2);
+          tot[0] = t2[0]; tot[2] = t2[1]; tot[1] = 0.f; tot[3] = 0.f;     // token 0 only; lanes t != 0 do not flush
+        } else {
+          blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
+        }
         if constexpr (OUT == OUT_T) {
           flush_sums(fl, tile, tot);
           ++flushed;
@@ -324,6 +335,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
             if constexpr (HILO) {
               sub = 0; sub_end = p.sub_tile0[1];
               load_t_pair(xr, xl, p, pair, lane);
+            } else if constexpr (I8) {
+              load_x_i8<FMT>(xi, p.x, x_bf16, pair, lane);
             } else {
               load_x_pair(xr, p, pair, lane);
             }
@@ -351,7 +364,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
   }
 }
 
-template <int WF, int ABF>
+// I8: the launch has one token and the backbone goes through the integer inner product.
+template <int WF, int ABF, bool I8>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_constant__ DecodeArgs p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -417,11 +431,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
 
   bool ok = true;
   if (a_owner) ok = run_segment<ABF, false, OUT_T>(p, r, a0, an, p.a_nt, blob_a, p.a_per_copy, p.a_sz2, lane);
-  if (ok) ok = run_segment<WF, false, OUT_Y>(p, r, w0, wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+  if (ok) ok = run_segment<WF, false, OUT_Y, I8>(p, r, w0, wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
   if (tr && lane == 0) tr[2] = globaltimer_ns();
   if (!a_owner) {
     if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
-    if (ok) ok = run_segment<WF, false, OUT_Y>(p, r, w0 + wf, wn - wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+    if (ok) ok = run_segment<WF, false, OUT_Y, I8>(p, r, w0 + wf, wn - wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
   }
   if (tr && lane == 0) tr[3] = globaltimer_ns();
 }
@@ -437,15 +451,25 @@ cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const DecodeArgs& args)
   return cudaLaunchKernelEx(&cfg, KERNEL, args);
 }
 
+// Formats whose backbone blobs have an integer inner product.
+constexpr bool has_i8(int fmt) { return fmt == FMT_Q4 || fmt == FMT_Q3; }
+
+template <int WF, bool I8>
+cudaError_t launch_ab2(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf) {
+  switch (abf) {
+    case FMT_F16: return launch_kernel<k_decode<WF, FMT_F16, I8>>(cfg, args);
+    case FMT_Q4: return launch_kernel<k_decode<WF, FMT_Q4, I8>>(cfg, args);
+    case FMT_Q8: return launch_kernel<k_decode<WF, FMT_Q8, I8>>(cfg, args);
+    case FMT_Q3: return launch_kernel<k_decode<WF, FMT_Q3, I8>>(cfg, args);
+    default: return launch_kernel<k_decode<WF, FMT_NONE, I8>>(cfg, args);
+  }
+}
 template <int WF>
 cudaError_t launch_ab(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf) {
-  switch (abf) {
-    case FMT_F16: return launch_kernel<k_decode<WF, FMT_F16>>(cfg, args);
-    case FMT_Q4: return launch_kernel<k_decode<WF, FMT_Q4>>(cfg, args);
-    case FMT_Q8: return launch_kernel<k_decode<WF, FMT_Q8>>(cfg, args);
-    case FMT_Q3: return launch_kernel<k_decode<WF, FMT_Q3>>(cfg, args);
-    default: return launch_kernel<k_decode<WF, FMT_NONE>>(cfg, args);
+  if constexpr (has_i8(WF)) {
+    if (args.m == 1) return launch_ab2<WF, true>(cfg, args, abf);
   }
+  return launch_ab2<WF, false>(cfg, args, abf);
 }
 
 // Relative cost of one blob (time a warp spends on it); only the ratios matter.

@@ -126,10 +126,6 @@ __device__ __forceinline__ void make_zc(ZC& zc, uint32_t zz) {
     uint32_t z = (zz >> (8 * hf)) & 255u;
     zc.c[hf][0] = (0x6400u | z) * 0x00010001u;                                      //  1024 + z
     if constexpr (FMT == FMT_Q4) zc.c[hf][1] = (0xD400u | (z << 4)) * 0x00010001u;   // -(64 + z)
-    if constexpr (FMT == FMT_Q3) {
-      zc.c[hf][1] = (0xD800u | (z << 3)) * 0x00010001u;                              // -(128 + z)
-      zc.c[hf][2] = (0xCC00u | (z << 6)) * 0x00010001u;                              // -(16 + z)
-    }
   }
 }
 
@@ -169,6 +165,22 @@ __host__ __device__ constexpr uint32_t sp24_selectors(uint32_t nib) {
 }
 constexpr int kSp24LutBytes = 64;       // 16 entries; every entry in its own shared-memory bank
 
+// The eight byte quads (one code per byte) of a lane's 32 codes of a 3-bit tile: q[part][quad].
+__device__ __forceinline__ void q3_quads(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t (&q)[4][2]) {
+  const uint32_t w[3] = {w0, w1, w2};
+#pragma unroll
+  for (int p = 0; p < 3; ++p) {
+    q[p][0] = w[p] & 0x07070707u;
+    q[p][1] = (w[p] >> 3) & 0x07070707u;
+  }
+  q[3][0] = and_or(w2 >> 4, 0x04040404u, (w0 >> 6) & 0x03030303u);
+  q[3][1] = and_or(w2 >> 5, 0x04040404u, (w1 >> 6) & 0x03030303u);
+}
+// Two neighbouring codes of a byte quad as fp16x2 (1024 + c0, 1024 + c1): which = 0: bytes 0, 1; 1: bytes 2, 3.
+__device__ __forceinline__ uint32_t quad_pair(uint32_t quad, int which) {
+  return prmt(quad, 0x64646464u, which ? 0x4342u : 0x4140u);
+}
+
 // `aux`: shared-memory address (32-bit, shared window) of the 2:4 expansion table; unused by other formats.
 template <int FMT>
 __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const ZC& zc, uint32_t (&a)[4][4], uint32_t aux = 0) {
@@ -189,26 +201,16 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
   } else if constexpr (FMT == FMT_Q3) {
     const uint2 v01 = *reinterpret_cast<const uint2*>(blob + lane * 8);
     const uint32_t v2 = *reinterpret_cast<const uint32_t*>(blob + 256 + lane * 4);
-    const uint32_t w[3] = {v01.x, v01.y, v2};
-    const uint32_t ws[3] = {v01.x >> 9, v01.y >> 9, v2 >> 9};
+    uint32_t q[4][2];
+    q3_quads(v01.x, v01.y, v2, q);
 #pragma unroll
-    for (int p = 0; p < 16; ++p) {
-      const int part = p >> 2, j = p & 3, hf = part & 1, blk = part >> 1;
-      uint32_t v;
-      if (p < 15) {
-        const int wi = p / 5, f = p % 5, ff = f >= 3 ? f - 3 : f;
-        const uint32_t src = f >= 3 ? ws[wi] : w[wi];
-        const uint32_t h = and_or(src, 0x00070007u << (3 * ff), kMagic);
-        if (ff == 0) v = h2sub(h, zc.c[hf][0]);
-        else if (ff == 1) v = h2fma(h, 0x30003000u, zc.c[hf][1]);   // * 1/8
-        else v = h2fma(h, 0x24002400u, zc.c[hf][2]);                // * 1/64
-      } else {
-        uint32_t h = and_or(w[0] >> 15, 0x00010001u, kMagic);
-        h = and_or(w[1] >> 14, 0x00020002u, h);
-        h = and_or(w[2] >> 13, 0x00040004u, h);
-        v = h2sub(h, zc.c[hf][0]);
+    for (int part = 0; part < 4; ++part) {
+      const int hf = part & 1, blk = part >> 1;
+#pragma unroll
+      for (int quad = 0; quad < 2; ++quad) {          // quad = which of the part's two mma
+        a[blk * 2 + quad][hf] = h2sub(quad_pair(q[part][quad], 0), zc.c[hf][0]);
+        a[blk * 2 + quad][hf + 2] = h2sub(quad_pair(q[part][quad], 1), zc.c[hf][0]);
       }
-      a[blk * 2 + (j >> 1)][hf + 2 * (j & 1)] = v;
     }
   } else if constexpr (FMT == FMT_Q8) {
 #pragma unroll
@@ -305,6 +307,164 @@ __device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint
   }
 }
 
+
+// ------------------------------------------------------------------------------------------ integer path (M = 1)
+// With a single token the tensor core is mostly idle (one of eight columns) and its instructions are what
+// the inner loop waits for.  For M = 1 the backbone product is therefore done with integer dot products: the
+// codes stay bytes (one and-or extracts four of them), the 128 activations of a pair are turned once into a
+// 16-bit fixed-point number relative to their largest magnitude (error <= 2^-16 of that magnitude, far
+// inside the fp16 rounding of the inputs themselves), split into a signed high and an unsigned low byte
+// plane, and  sum_k q_k X_k = 256 * dp4a(q, Xh) + dp4a(q, Xl)  is exact in int32.  Zero-point and scales
+// follow per group:  y += s * sx * (sum q X - z * sum X).
+struct XI8 {
+  uint32_t h[8], l[8];      // byte planes of this lane's 32 activations: index 2 * (2 * c + blk) + quad
+  int sum[2];               // sum of X over the 64 activations of tile c (all lanes of the warp hold it)
+  float scale;              // activation = X * scale
+};
+
+__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {
+  int d;
+  asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {
+  int d;
+  asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
+// Order of the eight elements of a part inside its two byte quads (quad 0 | quad 1), per format: the order in
+// which one and-or delivers the codes.
+template <int FMT> __device__ __forceinline__ constexpr int i8_elem(int quad, int byte) {
+  if constexpr (FMT == FMT_Q4) return quad == 0 ? (byte == 0 ? 0 : byte == 1 ? 4 : byte == 2 ? 1 : 5)
+                                                : (byte == 0 ? 2 : byte == 1 ? 6 : byte == 2 ? 3 : 7);
+  return 4 * quad + byte;
+}
+
+// x: token 0's activations (fp16 or bf16 bits), pair: which 128 of them.
+template <int FMT>
+__device__ __forceinline__ void load_x_i8(XI8& xi, const void* x, bool bf16, uint32_t pair, int lane) {
+  const int t = lane & 3;
+  const uint16_t* src = reinterpret_cast<const uint16_t*>(x) + pair * 128 + 8 * t;
+  float v[4][8];
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {                       // i = 2 * c + blk
+    uint4 u;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "l"(src + 32 * i) : "memory");
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float lo, hi;
+      if (bf16) {
+        lo = __uint_as_float(w[j] << 16); hi = __uint_as_float(w[j] & 0xffff0000u);
+      } else {
+        const __half2 h2 = *reinterpret_cast<const __half2*>(&w[j]);
+        lo = __low2float(h2); hi = __high2float(h2);
+      }
+      v[i][2 * j] = lo; v[i][2 * j + 1] = hi;
+      amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+    }
+  }
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+  const float scale = amax > 0.f ? amax * (1.f / 32767.f) : 1.f;
+  const float inv = 1.f / scale;
+  xi.scale = scale;
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    int s = 0;
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+      const int i = 2 * c + blk;
+      int X[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { X[e] = __float2int_rn(v[i][e] * inv); s += X[e]; }
+#pragma unroll
+      for (int quad = 0; quad < 2; ++quad) {
+        uint32_t h = 0, l = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int Xe = X[i8_elem<FMT>(quad, b)];
+          h |= ((uint32_t)(Xe >> 8) & 255u) << (8 * b);
+          l |= ((uint32_t)Xe & 255u) << (8 * b);
+        }
+        xi.h[2 * i + quad] = h;
+        xi.l[2 * i + quad] = l;
+      }
+    }
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s += __shfl_xor_sync(0xffffffffu, s, 2);
+    xi.sum[c] = s;
+  }
+}
+
+// Byte quads of one part (8 codes of one row): qa, qb in the element order of i8_elem.
+template <int FMT>
+__device__ __forceinline__ void tile_quads(const uint8_t* blob, int lane, uint32_t (&q)[4][2]) {
+  if constexpr (FMT == FMT_Q4) {
+    const uint4 v = *reinterpret_cast<const uint4*>(blob + lane * 16);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int part = 0; part < 4; ++part) {
+      q[part][0] = w[part] & 0x0f0f0f0fu;
+      q[part][1] = (w[part] >> 4) & 0x0f0f0f0fu;
+    }
+  } else if constexpr (FMT == FMT_Q3) {
+    const uint2 v01 = *reinterpret_cast<const uint2*>(blob + lane * 8);
+    const uint32_t v2 = *reinterpret_cast<const uint32_t*>(blob + 256 + lane * 4);
+    q3_quads(v01.x, v01.y, v2, q);
+  }
+}
+
+// One blob times the byte planes: tot[0] / tot[1] = this blob's contribution to rows g / g + 8 (token 0),
+// complete (summed over the four lanes that share a row) in every lane.
+template <int FMT>
+__device__ __forceinline__ void blob_product_i8(const uint8_t* blob, int lane, uint32_t sz2, const XI8& xi, float (&tot)[2]) {
+  constexpr int tb = tile_bytes(FMT);
+  const int g = lane >> 2;
+  int acc[2] = {0, 0};
+  tot[0] = tot[1] = 0.f;
+  int z_a = 0, z_b = 0;
+  float s_a = 0.f, s_b = 0.f;
+  int zsum_a = 0, zsum_b = 0;          // z * sum X over the tiles of the current scale entry
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    if (c == 0 || sz2) {
+      const uint8_t* sz = blob + 2 * tb + c * kSzEntryBytes;
+      const uint32_t s2 = reinterpret_cast<const uint32_t*>(sz)[g];
+      const uint32_t z2 = reinterpret_cast<const uint16_t*>(sz + 32)[g];
+      z_a = (int)(z2 & 255u); z_b = (int)(z2 >> 8);
+      s_a = __half2float(__ushort_as_half((unsigned short)(s2 & 0xffffu))) * xi.scale;
+      s_b = __half2float(__ushort_as_half((unsigned short)(s2 >> 16))) * xi.scale;
+      zsum_a = 0; zsum_b = 0;
+    }
+    zsum_a += z_a * xi.sum[c];
+    zsum_b += z_b * xi.sum[c];
+    uint32_t q[4][2];
+    tile_quads<FMT>(blob + c * tb, lane, q);
+    int sh[2] = {0, 0}, sl[2] = {0, 0};
+#pragma unroll
+    for (int part = 0; part < 4; ++part) {
+      const int hf = part & 1, i = 2 * c + (part >> 1);
+#pragma unroll
+      for (int quad = 0; quad < 2; ++quad) {
+        sh[hf] = dp4a_us(q[part][quad], xi.h[2 * i + quad], sh[hf]);
+        sl[hf] = dp4a_uu(q[part][quad], xi.l[2 * i + quad], sl[hf]);
+      }
+    }
+    acc[0] += sh[0] * 256 + sl[0];
+    acc[1] += sh[1] * 256 + sl[1];
+    if (c == 1 || sz2) {
+      int ra = acc[0], rb = acc[1];
+      ra += __shfl_xor_sync(0xffffffffu, ra, 1); rb += __shfl_xor_sync(0xffffffffu, rb, 1);
+      ra += __shfl_xor_sync(0xffffffffu, ra, 2); rb += __shfl_xor_sync(0xffffffffu, rb, 2);
+      tot[0] = fmaf((float)(ra - zsum_a), s_a, tot[0]);
+      tot[1] = fmaf((float)(rb - zsum_b), s_b, tot[1]);
+      acc[0] = acc[1] = 0;
+    }
+  }
+}
 
 __device__ __forceinline__ void store_y(void* y, int dtype, int64_t i, float v) {
   if (dtype == EORA_Y_F16) reinterpret_cast<__half*>(y)[i] = __float2half_rn(v);

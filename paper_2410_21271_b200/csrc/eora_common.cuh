@@ -35,11 +35,11 @@ namespace eora {
 //   Q4  : 512 B: one uint4 per lane; word `part` holds the 8 codes of that part, element e in nibble
 //         (e & 1) * 4 + (e >> 1)   (so that (w & 0x000f000f) is the pair (e0, e1), ...).
 //   Q3  : 384 B: three words; w0, w1 as a uint2 per lane in bytes [0, 256), w2 as one word per lane
-//         in bytes [256, 384).  The 32 codes form 16 pairs,
-//         pair p = part*4 + e/2; for p < 15 the pair lives in word p/5, field f = p%5: the even
-//         element in bits [3f, 3f+3), the odd one in bits [16+3f, 16+3f+3).  Pair 15 is spread
-//         over the spare bits: bit i of the even element is bit 15 of word i, bit i of the odd
-//         element is bit 31 of word i.
+//         in bytes [256, 384).  Byte-planar: for part p < 3, byte b of word p holds element b in bits
+//         [0, 3) and element 4 + b in bits [3, 6), so that (w & 0x07070707) and ((w >> 3) & 0x07070707)
+//         are the part's two quads of codes, one code per byte.  Part 3 lives in the spare bits: element
+//         4*quad + b has its low two bits in bits [6, 8) of byte b of word `quad`, its high bit in bit
+//         6 + quad of byte b of w2.
 //   Q8  : 1024 B: two planes of one uint4 per lane (plane = part/2); words 2*(part%2) and 2*(part%2)+1
 //         hold elements 0..3 and 4..7; inside a word element i sits in byte {0, 2, 1, 3}[i].
 //   F16 : 2048 B: four planes of one uint4 per lane (plane = part), 8 fp16 in natural order.
@@ -88,6 +88,23 @@ __host__ __device__ inline const uint8_t* wmat_sz(const WMat& w, int tile, int c
 __host__ __device__ inline int q4_nibble(int e) { return (e & 1) * 4 + (e >> 1); }
 __host__ __device__ inline int q8_byte(int i) { return (i == 1) ? 2 : (i == 2) ? 1 : i; }
 
+// 3-bit code of element e of part `part` from the three words of a lane (see the Q3 layout above)
+__host__ __device__ inline int q3_code(const uint32_t (&wd)[3], int part, int e) {
+  const int quad = e >> 2, b = e & 3;
+  if (part < 3) return (wd[part] >> (8 * b + 3 * quad)) & 7;
+  return ((wd[quad] >> (8 * b + 6)) & 3) | (((wd[2] >> (8 * b + 6 + quad)) & 1) << 2);
+}
+// and the inverse: put code q there
+__host__ __device__ inline void q3_put(uint32_t (&wd)[3], int part, int e, uint32_t q) {
+  const int quad = e >> 2, b = e & 3;
+  if (part < 3) {
+    wd[part] |= q << (8 * b + 3 * quad);
+  } else {
+    wd[quad] |= (q & 3u) << (8 * b + 6);
+    wd[2] |= ((q >> 2) & 1u) << (8 * b + 6 + quad);
+  }
+}
+
 // Integer code of element (k, n) of a quantised WMat.
 __device__ inline int wmat_code(const WMat& w, int k, int n) {
   int tile = n >> 4, g = n & 7, half = (n >> 3) & 1;
@@ -98,10 +115,7 @@ __device__ inline int wmat_code(const WMat& w, int k, int n) {
     return (blob[lane * 4 + part] >> (4 * q4_nibble(e))) & 15;
   } else if (w.fmt == FMT_Q3) {
     uint32_t wd[3] = {blob[lane * 2], blob[lane * 2 + 1], blob[64 + lane]};
-    int pr = part * 4 + (e >> 1), hi = (e & 1) * 16;
-    if (pr < 15) return (wd[pr / 5] >> (3 * (pr % 5) + hi)) & 7;
-    int b = 15 + hi;
-    return ((wd[0] >> b) & 1) | (((wd[1] >> b) & 1) << 1) | (((wd[2] >> b) & 1) << 2);
+    return q3_code(wd, part, e);
   } else {  // FMT_Q8
     uint32_t wd = blob[(part >> 1) * 128 + lane * 4 + 2 * (part & 1) + (e >> 2)];
     return (wd >> (8 * q8_byte(e & 3))) & 255;

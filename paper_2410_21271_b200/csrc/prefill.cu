@@ -167,26 +167,13 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
         a[part][3] = h2fma(and_or(hi, 0x00f000f0u, kMagic), 0x2C002C00u, zc.c[hf][1]);
       }
     } else if constexpr (FMT == FMT_Q3) {
-      const uint32_t w[3] = {r.v.x, r.v.y, r.w2};
-      const uint32_t ws[3] = {r.v.x >> 9, r.v.y >> 9, r.w2 >> 9};
+      uint32_t q[4][2];
+      q3_quads(r.v.x, r.v.y, r.w2, q);
 #pragma unroll
-      for (int p = 0; p < 16; ++p) {
-        const int part = p >> 2, j = p & 3, hf = part & 1;
-        uint32_t v;
-        if (p < 15) {
-          const int wi = p / 5, f = p % 5, ff = f >= 3 ? f - 3 : f;
-          const uint32_t src = f >= 3 ? ws[wi] : w[wi];
-          const uint32_t h = and_or(src, 0x00070007u << (3 * ff), kMagic);
-          if (ff == 0) v = h2sub(h, zc.c[hf][0]);
-          else if (ff == 1) v = h2fma(h, 0x30003000u, zc.c[hf][1]);
-          else v = h2fma(h, 0x24002400u, zc.c[hf][2]);
-        } else {
-          uint32_t h = and_or(w[0] >> 15, 0x00010001u, kMagic);
-          h = and_or(w[1] >> 14, 0x00020002u, h);
-          h = and_or(w[2] >> 13, 0x00040004u, h);
-          v = h2sub(h, zc.c[hf][0]);
-        }
-        a[part][j] = v;
+      for (int part = 0; part < 4; ++part) {
+        const int hf = part & 1;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) a[part][j] = h2sub(quad_pair(q[part][j >> 1], j & 1), zc.c[hf][0]);
       }
     } else {   // FMT_Q8
 #pragma unroll

@@ -68,12 +68,7 @@ __global__ void k_repack_q3(WMat d, int nt_sub, const uint32_t* codes, const uin
       int k0 = p.c * 64 + (part >> 1) * 32 + 8 * p.t;
       for (int e = 0; e < 8; ++e) {
         uint32_t q = padded_code(codes, zeros, 3, k0 + e, n, rows_src, k_src, d.group, ldz);
-        int pr = part * 4 + (e >> 1), hi = (e & 1) * 16;
-        if (pr < 15) {
-          wd[pr / 5] |= q << (3 * (pr % 5) + hi);
-        } else {
-          for (int i = 0; i < 3; ++i) wd[i] |= ((q >> i) & 1u) << (15 + hi);
-        }
+        q3_put(wd, part, e, q);
       }
     }
     uint32_t* blob = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c)));
