@@ -257,7 +257,11 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     XI8 xi;
     const bool x_bf16 = p.x_dtype == EORA_X_BF16;
     uint32_t sub = 0, sub_end = nt;
-    const Flush fl = OUT == OUT_T ? make_flush(p.d_t, p.r_pad, p.m, lane) : make_flush(p.y_ws, p.n_pad, p.m, lane);
+    Flush fl = OUT == OUT_T ? make_flush(p.d_t, p.r_pad, p.m, lane) : make_flush(p.y_ws, p.n_pad, p.m, lane);
+    if constexpr (I8) {       // all four lanes of a row add to token 0
+      fl.base = p.y_ws + (lane >> 2);
+      fl.has0 = 1u; fl.has1 = 0u;
+    }
     if constexpr (HILO) {
       // all of A must be in t
       int ok = 1;
@@ -316,7 +320,7 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
         if constexpr (I8) {
           float t2[2];
           blob_product_i8<FMT>(src + j * blob_b, lane, sz2, xi, t2);
-          tot[0] = t2[0]; tot[2] = t2[1]; tot[1] = 0.f; tot[3] = 0.f;     // token 0 only; lanes t != 0 do not flush
+          tot[0] = t2[0]; tot[2] = t2[1]; tot[1] = 0.f; tot[3] = 0.f;     // token 0 only, every lane its own share
         } else {
           blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
         }

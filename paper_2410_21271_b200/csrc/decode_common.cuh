@@ -318,7 +318,7 @@ __device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint
 // follow per group:  y += s * sx * (sum q X - z * sum X).
 struct XI8 {
   uint32_t h[8], l[8];      // byte planes of this lane's 32 activations: index 2 * (2 * c + blk) + quad
-  int sum[2];               // sum of X over the 64 activations of tile c (all lanes of the warp hold it)
+  int sum[2];               // sum of X over this lane's 16 activations of tile c
   float scale;              // activation = X * scale
 };
 
@@ -393,8 +393,6 @@ __device__ __forceinline__ void load_x_i8(XI8& xi, const void* x, bool bf16, uin
         xi.l[2 * i + quad] = l;
       }
     }
-    s += __shfl_xor_sync(0xffffffffu, s, 1);
-    s += __shfl_xor_sync(0xffffffffu, s, 2);
     xi.sum[c] = s;
   }
 }
@@ -417,8 +415,9 @@ __device__ __forceinline__ void tile_quads(const uint8_t* blob, int lane, uint32
   }
 }
 
-// One blob times the byte planes: tot[0] / tot[1] = this blob's contribution to rows g / g + 8 (token 0),
-// complete (summed over the four lanes that share a row) in every lane.
+// One blob times the byte planes: tot[0] / tot[1] = this LANE's share of the blob's contribution to rows g /
+// g + 8 (token 0): the four lanes that share a row each add their own share to the row's sum (a reduction
+// over those lanes first would put two dependent shuffle round trips into every blob).
 template <int FMT>
 __device__ __forceinline__ void blob_product_i8(const uint8_t* blob, int lane, uint32_t sz2, const XI8& xi, float (&tot)[2]) {
   constexpr int tb = tile_bytes(FMT);
@@ -456,11 +455,8 @@ __device__ __forceinline__ void blob_product_i8(const uint8_t* blob, int lane, u
     acc[0] += sh[0] * 256 + sl[0];
     acc[1] += sh[1] * 256 + sl[1];
     if (c == 1 || sz2) {
-      int ra = acc[0], rb = acc[1];
-      ra += __shfl_xor_sync(0xffffffffu, ra, 1); rb += __shfl_xor_sync(0xffffffffu, rb, 1);
-      ra += __shfl_xor_sync(0xffffffffu, ra, 2); rb += __shfl_xor_sync(0xffffffffu, rb, 2);
-      tot[0] = fmaf((float)(ra - zsum_a), s_a, tot[0]);
-      tot[1] = fmaf((float)(rb - zsum_b), s_b, tot[1]);
+      tot[0] = fmaf((float)(acc[0] - zsum_a), s_a, tot[0]);
+      tot[1] = fmaf((float)(acc[1] - zsum_b), s_b, tot[1]);
       acc[0] = acc[1] = 0;
     }
   }
