@@ -341,33 +341,26 @@ template <int FMT> __device__ __forceinline__ constexpr int i8_elem(int quad, in
   return 4 * quad + byte;
 }
 
-// x: token 0's activations (fp16 or bf16 bits), pair: which 128 of them.
+// x: token 0's activations (fp16 or bf16 bits), pair: which 128 of them.  Every lane converts its own 32
+// activations with a scale of its own (its largest magnitude / 32767): lanes never exchange anything.
 template <int FMT>
 __device__ __forceinline__ void load_x_i8(XI8& xi, const void* x, bool bf16, uint32_t pair, int lane) {
   const int t = lane & 3;
   const uint16_t* src = reinterpret_cast<const uint16_t*>(x) + pair * 128 + 8 * t;
-  float v[4][8];
+  float2 v[4][4];                                     // [2 * c + blk][pair of elements]
   float amax = 0.f;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {                       // i = 2 * c + blk
+  for (int i = 0; i < 4; ++i) {
     uint4 u;
     asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "l"(src + 32 * i) : "memory");
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      float lo, hi;
-      if (bf16) {
-        lo = __uint_as_float(w[j] << 16); hi = __uint_as_float(w[j] & 0xffff0000u);
-      } else {
-        const __half2 h2 = *reinterpret_cast<const __half2*>(&w[j]);
-        lo = __low2float(h2); hi = __high2float(h2);
-      }
-      v[i][2 * j] = lo; v[i][2 * j + 1] = hi;
-      amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+      if (bf16) v[i][j] = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xffff0000u));
+      else v[i][j] = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
+      amax = fmaxf(amax, fmaxf(fabsf(v[i][j].x), fabsf(v[i][j].y)));
     }
   }
-  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
   const float scale = amax > 0.f ? amax * (1.f / 32767.f) : 1.f;
   const float inv = 1.f / scale;
   xi.scale = scale;
@@ -377,20 +370,20 @@ __device__ __forceinline__ void load_x_i8(XI8& xi, const void* x, bool bf16, uin
 #pragma unroll
     for (int blk = 0; blk < 2; ++blk) {
       const int i = 2 * c + blk;
-      int X[8];
+      uint32_t P[4];                                  // (X[2j], X[2j+1]) as two 16-bit halves
 #pragma unroll
-      for (int e = 0; e < 8; ++e) { X[e] = __float2int_rn(v[i][e] * inv); s += X[e]; }
-#pragma unroll
-      for (int quad = 0; quad < 2; ++quad) {
-        uint32_t h = 0, l = 0;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-          const int Xe = X[i8_elem<FMT>(quad, b)];
-          h |= ((uint32_t)(Xe >> 8) & 255u) << (8 * b);
-          l |= ((uint32_t)Xe & 255u) << (8 * b);
-        }
-        xi.h[2 * i + quad] = h;
-        xi.l[2 * i + quad] = l;
+      for (int j = 0; j < 4; ++j) {
+        const int x0 = __float2int_rn(v[i][j].x * inv), x1 = __float2int_rn(v[i][j].y * inv);
+        s += x0 + x1;
+        P[j] = prmt((uint32_t)x0, (uint32_t)x1, 0x5410u);
+      }
+      // byte planes in the element order of i8_elem<FMT>: low bytes / high bytes of four 16-bit values
+      if constexpr (FMT == FMT_Q4) {                  // quads (0, 4, 1, 5) and (2, 6, 3, 7)
+        xi.l[2 * i] = prmt(P[0], P[2], 0x6240u); xi.h[2 * i] = prmt(P[0], P[2], 0x7351u);
+        xi.l[2 * i + 1] = prmt(P[1], P[3], 0x6240u); xi.h[2 * i + 1] = prmt(P[1], P[3], 0x7351u);
+      } else {                                        // quads (0, 1, 2, 3) and (4, 5, 6, 7)
+        xi.l[2 * i] = prmt(P[0], P[1], 0x6420u); xi.h[2 * i] = prmt(P[0], P[1], 0x7531u);
+        xi.l[2 * i + 1] = prmt(P[2], P[3], 0x6420u); xi.h[2 * i + 1] = prmt(P[2], P[3], 0x7531u);
       }
     }
     xi.sum[c] = s;
