@@ -329,7 +329,12 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
           ++flushed;
         } else {
           if (batch_n == 0) batch_tile = tile;
-          flush_sums(fl, tile, tot);
+          if constexpr (I8) {                     // one token, every lane adds: two unconditional adds
+            float* b = fl.base + tile * 16;
+            red_add(b, tot[0]); red_add(b + 8, tot[2]);
+          } else {
+            flush_sums(fl, tile, tot);
+          }
           if (++batch_n == 32) commit_batch();
         }
         if (++tile == nt) {
