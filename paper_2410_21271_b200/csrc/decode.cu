@@ -539,7 +539,9 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
   // the others the rest of W plus B.
   if (ab) {
     const double ca = a.a_blobs * blob_cost(h->a.fmt, false), cb = b_blobs * blob_cost(h->b.fmt, true);
-    const double cw1 = blob_cost(h->w.fmt, false), cw = w_blobs * cw1;
+    // with one token the backbone blobs go through the integer inner product, which is cheaper
+    const bool i8 = m == 1 && (h->w.fmt == FMT_Q4 || h->w.fmt == FMT_Q3);
+    const double cw1 = blob_cost(h->w.fmt, false) * (i8 ? 0.75 : 1.0), cw = w_blobs * cw1;
     // Besides the per-blob cost each kind of warp has a fixed one (in units of one backbone blob): the B
     // share starts with a read-back of t and ends with its own round of tickets, which is latency that
     // the warp cannot hide from itself.
