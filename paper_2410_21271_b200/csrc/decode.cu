@@ -10,9 +10,11 @@
 // contiguous run of blobs of up to three matrices, fetches it with its own bulk copies into its own
 // shared-memory ring and never synchronises with another warp of its CTA.
 //
-//   * warps [0, n_a) ("A owners") take A first (t += X . A, sums in d_t) and then a share of W,
-//   * the other warps take their share of W first and then a share of B, for which the activations are
-//     t (read back as fp32 and split into an fp16 high and low part, so that t keeps fp32-like accuracy).
+//   * the first warps ("A owners") take the blobs of A first (t += X . A, sums in d_t) and then a share of W,
+//   * the last warps ("B owners") take one copy of W, then their blobs of B, for which the activations are t
+//     (read back as fp32 and split into an fp16 high and low part, so that t keeps fp32-like accuracy),
+//     then the rest of their share of W,
+//   * the warps in between take backbone blobs only.
 // The only wait in the kernel is the one before the B share: all of A must have been added to t.  A
 // owners never wait, and they sit in the CTAs with the lowest indices, which are dispatched first, so a
 // waiting warp never holds the slot of a CTA it is waiting for.  The wait is bounded like every other.
@@ -46,11 +48,14 @@ struct Share { uint32_t per, rem; };      // blobs of a matrix dealt to n warps:
 struct DecodeArgs {
   const uint8_t* a_q; const uint8_t* w_q; const uint8_t* b_q;
   uint32_t a_nt, w_nt;                    // row tiles of A and of W (= of B)
-  uint32_t a_blobs, w1_blobs;             // all of A; the part of W that the A owners take
+  uint32_t a_blobs;                       // all of A
   uint32_t a_per_copy, w_per_copy, b_per_copy;   // blobs per bulk copy
   uint32_t a_sz2, w_sz2, b_sz2;
-  uint32_t n_a;                           // number of A-owner warps
-  Share sh_a, sh_w1, sh_w2, sh_b;
+  // Three groups of warps: [0, n1) hold the blobs of A ("A owners"), [n1, n12) only backbone blobs,
+  // [n12, all) the blobs of B.  Every group has its own share of the backbone, starting at w_base[group].
+  uint32_t n1, n12;
+  Share sh_a, sh_b, sh_w[3];
+  uint32_t w_base[3];
   uint32_t tile_target;                   // blobs per output row tile: pairs of W + pairs of B
   const void* x;
   void* ys[4];                            // outputs of the fused layers (one for a plain layer)
@@ -403,22 +408,25 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   __syncwarp();
 
   // this warp's three runs: A, W, B (one of A / B is empty)
-  const bool a_owner = gw < p.n_a;
+  const bool a_owner = gw < p.n1, b_owner = gw >= p.n12;
   uint32_t a0 = 0, an = 0, w0, wn, bb0 = 0, bn = 0;
   if (a_owner) {
     a0 = share_lo(p.sh_a, gw); an = share_n(p.sh_a, gw);
-    w0 = share_lo(p.sh_w1, gw); wn = share_n(p.sh_w1, gw);
+    w0 = p.w_base[0] + share_lo(p.sh_w[0], gw); wn = share_n(p.sh_w[0], gw);
+  } else if (!b_owner) {
+    const uint32_t i = gw - p.n1;
+    w0 = p.w_base[1] + share_lo(p.sh_w[1], i); wn = share_n(p.sh_w[1], i);
   } else {
-    const uint32_t i = gw - p.n_a;
-    w0 = p.w1_blobs + share_lo(p.sh_w2, i); wn = share_n(p.sh_w2, i);
+    const uint32_t i = gw - p.n12;
+    w0 = p.w_base[2] + share_lo(p.sh_w[2], i); wn = share_n(p.sh_w[2], i);
     bb0 = share_lo(p.sh_b, i); bn = share_n(p.sh_b, i);
   }
   const uint32_t blob_a = blob_bytes(ABF, p.a_sz2), blob_w = blob_bytes(WF, p.w_sz2), blob_b = blob_bytes(ABF, p.b_sz2);
   // Order of the runs.  A owners: A, then W.  The others: the first copy's worth of W, then B, then the
   // rest of W: by then t is complete, and the round trips of the B share (reading t back, its tickets)
   // are hidden behind the other warps' W work instead of sitting at the end of the kernel.
-  const uint32_t wf = a_owner ? wn : (wn < p.w_per_copy ? wn : p.w_per_copy);
-  if (a_owner) {
+  const uint32_t wf = !b_owner ? wn : (wn < p.w_per_copy ? wn : p.w_per_copy);
+  if (!b_owner) {
     r.ptr[0] = p.a_q + (size_t)a0 * blob_a; r.rem[0] = an; r.blob[0] = blob_a; r.per[0] = p.a_per_copy;
     r.ptr[1] = p.w_q + (size_t)w0 * blob_w; r.rem[1] = wn; r.blob[1] = blob_w; r.per[1] = p.w_per_copy;
     r.ptr[2] = p.w_q; r.rem[2] = 0; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
@@ -442,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   if (a_owner) ok = run_segment<ABF, false, OUT_T>(p, r, a0, an, p.a_nt, blob_a, p.a_per_copy, p.a_sz2, lane);
   if (ok) ok = run_segment<WF, false, OUT_Y, I8>(p, r, w0, wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
   if (tr && lane == 0) tr[2] = globaltimer_ns();
-  if (!a_owner) {
+  if (b_owner) {
     if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
     if (ok) ok = run_segment<WF, false, OUT_Y, I8>(p, r, w0 + wf, wn - wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
   }
@@ -535,43 +543,37 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
   }
   const int grid = decode_grid(h, m);
   const uint32_t nw = (uint32_t)grid * kWarps;
-  // Deal the blobs so that every warp gets the same estimated time: A owners take A plus a part of W,
-  // the others the rest of W plus B.
+  // Deal the blobs so that every warp gets the same estimated time.  Costs are in units of one backbone
+  // blob on the tensor-core path.  Besides its blobs of A or B a warp of the first or third group has a
+  // fixed extra cost: the A owners fetch a second set of activations, the B owners read t back and end
+  // with their own round of tickets, which is latency that a warp cannot hide from itself.
   if (ab) {
-    const double ca = a.a_blobs * blob_cost(h->a.fmt, false), cb = b_blobs * blob_cost(h->b.fmt, true);
     // with one token the backbone blobs go through the integer inner product, which is cheaper
     const bool i8 = m == 1 && (h->w.fmt == FMT_Q4 || h->w.fmt == FMT_Q3);
-    const double cw1 = blob_cost(h->w.fmt, false) * (i8 ? 0.75 : 1.0), cw = w_blobs * cw1;
-    // Besides the per-blob cost each kind of warp has a fixed one (in units of one backbone blob): the B
-    // share starts with a read-back of t and ends with its own round of tickets, which is latency that
-    // the warp cannot hide from itself.
-    const double fixed_a = 0.5, fixed_b = 9.0;
-    const double tau = (ca + cw + cb) / nw;
-    uint32_t lo = (uint32_t)(ca / tau) + 1, hi = nw - ((uint32_t)(cb / tau) + 1);
-    uint32_t n_a = nw / 2;
-    if (b_blobs < nw - n_a) n_a = nw - b_blobs;          // no B owner without a blob of B
-    if (n_a < lo) n_a = lo;
-    if (n_a > hi) n_a = hi;
-    if (n_a < 1) n_a = 1;
-    if (n_a > nw - 1) n_a = nw - 1;
-    const double n_b = nw - n_a;
-    // equal finishing time:  fixed_a + (ca + w1 cw1) / n_a  =  fixed_b + (cb + (W - w1) cw1) / n_b
-    double w1 = ((fixed_b - fixed_a) + cb / n_b + cw / n_b - ca / n_a) / (cw1 * (1.0 / n_a + 1.0 / n_b));
-    if (w1 < 0) w1 = 0;
-    if (w1 > w_blobs) w1 = w_blobs;
-    a.n_a = n_a;
-    a.w1_blobs = (uint32_t)w1;
-    a.sh_a = make_share(a.a_blobs, n_a);
-    a.sh_w1 = make_share(a.w1_blobs, n_a);
-    a.sh_w2 = make_share(w_blobs - a.w1_blobs, nw - n_a);
-    a.sh_b = make_share(b_blobs, nw - n_a);
+    const double cw1 = blob_cost(h->w.fmt, false) * (i8 ? 0.75 : 1.0);
+    const double fixed_a = i8 ? 4.0 : 2.0, fixed_b = 9.0;
+    uint32_t n1 = a.a_blobs < nw / 3 ? a.a_blobs : nw / 3;
+    uint32_t n3 = b_blobs < nw / 3 ? b_blobs : nw / 3;
+    if (n1 < 1) n1 = 1;
+    if (n3 < 1) n3 = 1;
+    const uint32_t n2 = nw - n1 - n3;
+    const double e1 = fixed_a + (double)a.a_blobs / n1 * blob_cost(h->a.fmt, false);
+    const double e3 = fixed_b + (double)b_blobs / n3 * blob_cost(h->b.fmt, true);
+    const double T = (w_blobs * cw1 + n1 * e1 + n3 * e3) / nw;      // finishing time of every warp
+    double W1 = T > e1 ? n1 * (T - e1) / cw1 : 0.0, W3 = T > e3 ? n3 * (T - e3) / cw1 : 0.0;
+    if (W1 + W3 > w_blobs) { const double f = w_blobs / (W1 + W3); W1 *= f; W3 *= f; }
+    const uint32_t w1 = (uint32_t)W1, w3 = (uint32_t)W3, w2 = w_blobs - w1 - w3;
+    a.n1 = n1; a.n12 = n1 + n2;
+    a.sh_a = make_share(a.a_blobs, n1);
+    a.sh_b = make_share(b_blobs, n3);
+    a.sh_w[0] = make_share(w1, n1); a.sh_w[1] = make_share(w2, n2); a.sh_w[2] = make_share(w3, n3);
+    a.w_base[0] = 0; a.w_base[1] = w1; a.w_base[2] = w1 + w2;
   } else {
-    a.n_a = nw;
-    a.w1_blobs = w_blobs;
-    a.sh_a = make_share(0, nw);
-    a.sh_w1 = make_share(w_blobs, nw);
-    a.sh_w2 = make_share(0, 0);
+    a.n1 = 0; a.n12 = nw;
+    a.sh_a = make_share(0, 0);
     a.sh_b = make_share(0, 0);
+    a.sh_w[0] = make_share(0, 0); a.sh_w[1] = make_share(w_blobs, nw); a.sh_w[2] = make_share(0, 0);
+    a.w_base[0] = 0; a.w_base[1] = 0; a.w_base[2] = w_blobs;
   }
   a.tile_target = (uint32_t)h->w.np + (ab ? (uint32_t)h->b.np : 0u);
   a.d_t = h->d_t; a.y_ws = h->y_ws; a.counters = h->counters; a.dev_status = h->dev_status;
