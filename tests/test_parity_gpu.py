@@ -78,6 +78,8 @@ SMALL = [
     ("q4", "q8", 256, 64, 40, 2, "f16"),
     ("sp24", "f16", 512, 96, 128, 1, "f16"),
     ("sp24", "f16", 256, 64, 64, 9, "bf16"),
+    ("q3", "f16", 1024, 224, 128, 1, "bf16"),
+    ("q4", "q4", 512, 96, 128, 1, "bf16"),
     ("q4", "q3", 512, 96, 128, 1, "f16"),
     ("q3", "q3", 1024, 224, 256, 16, "f16"),
     ("q4", "q3", 640, 160, 64, 100, "bf16"),
@@ -171,6 +173,28 @@ def test_one_hot_rows_read_back_exact_weights(w):
     q = orc.unpack_codes(wf["codes"], wf["bits"], K); z = orc.unpack_zeros(wf["zeros"], wf["bits"], N)
     W = orc.deq_fp32(q, z, wf["scales"], 128).astype(np.float64)
     assert np.array_equal(y, W[ks])
+    L.close()
+
+
+@pytest.mark.parametrize("w", ["q4", "q3"])
+def test_single_token_extreme_activations(w):
+    """The single-token path turns the activations into fixed point relative to their largest magnitude:
+    all-zero input, one huge value among tiny ones, and a wide dynamic range must stay inside the tolerance."""
+    K, N, r = 512, 96, 64
+    wf, af, bf = make_case(37, K, N, r, w=w)
+    L = eora.Layer(wf, af, bf, max_m=1)
+    rng = np.random.default_rng(38)
+    xs = [np.zeros((1, K), dtype=np.float16)]
+    x = (rng.standard_normal((1, K)) * 1e-3).astype(np.float16); x[0, 17] = 3000.0; xs.append(x)
+    x = (rng.standard_normal((1, K)) * np.exp(rng.uniform(-6, 3, (1, K)))).astype(np.float16); xs.append(x)
+    x = (rng.standard_normal((1, K)) * 200).astype(np.float16); xs.append(x)
+    for i, x in enumerate(xs):
+        y = run_layer(L, x, "f16")
+        ref = orc.forward(x, "f16", wf, af, bf)
+        if not ref.any():
+            assert not y.any()
+        else:
+            check_parity(y, ref, f"extreme activations case {i}")
     L.close()
 
 
