@@ -138,6 +138,23 @@ int eora_linear_forward(eora_linear_t h, const void* x, int32_t m, void* y, void
 int eora_linear_create_fused(const eora_linear_config* cfgs, const eora_linear_weights* weights, int32_t n_layers,
                              void* stream, eora_linear_t* out);
 int eora_linear_forward_fused(eora_linear_t h, const void* x, int32_t m, void* const* ys, void* stream);
+/*
+ * Several adapters on one backbone.  The paper stores the compensation apart from the compressed
+ * weights so that task-specific low-rank modules can be switched on and off (Sections 1 and 3); a
+ * server decoding several requests at once needs a different module per token.
+ * eora_linear_create_multi builds one handle from the layer's config and n_adapters (1..8) weight
+ * structs: the backbone is taken from weights[0], adapter j (A_j, B_j and their scales / zeros) from
+ * weights[j]; all adapters have the config's rank and format.  eora_linear_forward_multi computes
+ *     y[i] = x[i] . deq(Wq) + (x[i] . A_j) . B_j   with j = adapter_ids[i],   or without the second
+ * term if adapter_ids[i] is negative (or not below n_adapters),
+ * for M <= max_m <= 64 tokens in one launch per eight tokens.  adapter_ids: HOST array of m int32,
+ * read before the call returns.  Decode family only; eora_linear_forward on such a handle returns
+ * EORA_ERR_UNSUPPORTED.  Cost: every adapter's A and B are streamed once per launch whatever the ids.
+ */
+int eora_linear_create_multi(const eora_linear_config* cfg, const eora_linear_weights* weights, int32_t n_adapters,
+                             void* stream, eora_linear_t* out);
+int eora_linear_forward_multi(eora_linear_t h, const void* x, int32_t m, const int32_t* adapter_ids, void* y, void* stream);
+
 /* The fused forward for activations in HOST memory (see eora_linear_forward_host): ys_host is a host array
  * of n_layers host pointers; synchronises `stream` before returning. */
 int eora_linear_forward_fused_host(eora_linear_t h, const void* x_host, int32_t m, void* const* ys_host, void* stream);

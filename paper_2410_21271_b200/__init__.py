@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
         L.eora_linear_forward_fused.restype = c_int
         L.eora_linear_forward_fused_host.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
         L.eora_linear_forward_fused_host.restype = c_int
+        L.eora_linear_create_multi.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_create_multi.restype = c_int
+        L.eora_linear_forward_multi.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p]
+        L.eora_linear_forward_multi.restype = c_int
         L.eora_linear_destroy.argtypes = [c_void_p]
         L.eora_linear_destroy.restype = c_int
         L.eora_linear_path.argtypes = [c_void_p, c_int32]
@@ -184,6 +188,30 @@ def eora_linear_forward_fused_host(handle: int, x_host, m: int, ys_host, stream=
     st = lib().eora_linear_forward_fused_host(handle, _ptr(x_host), int(m), arr, _stream(stream))
     if check and st != EORA_OK:
         raise EoraError(st, "eora_linear_forward_fused_host")
+    return st
+
+
+def eora_linear_create_multi(cfg, weights, stream=None, check: bool = True):
+    """cfg: the layer's eora_linear_config; weights: one eora_linear_weights per adapter (backbone from the
+    first).  Returns the handle, or (with check=False) the status."""
+    n = len(weights)
+    warr = (eora_linear_weights * n)(*weights)
+    out = c_void_p()
+    st = lib().eora_linear_create_multi(byref(cfg), warr, n, _stream(stream), byref(out))
+    if not check:
+        if st == EORA_OK:
+            lib().eora_linear_destroy(out)
+        return st
+    if st != EORA_OK:
+        raise EoraError(st, "eora_linear_create_multi")
+    return out.value
+
+
+def eora_linear_forward_multi(handle: int, x, m: int, adapter_ids, y, stream=None, check: bool = True) -> int:
+    ids = (c_int32 * int(m))(*[int(i) for i in adapter_ids])
+    st = lib().eora_linear_forward_multi(handle, _ptr(x), int(m), ids, _ptr(y), _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward_multi")
     return st
 
 
@@ -383,6 +411,48 @@ class FusedLayers:
 
     def launches(self, m: int) -> int:
         return eora_linear_launches(self.handle, m)
+
+    def device_status(self) -> int:
+        return eora_linear_last_device_status(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            eora_linear_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class MultiAdapterLayer:
+    """One backbone with several adapters; every token of a forward names the adapter it uses (-1: none).
+    Decode only (max_m <= 64).  Methods only marshal arguments."""
+
+    def __init__(self, w_fmt: dict, adapters, *, max_m: int, x_dtype: str = "f16", y_dtype: str = "f16", device="cuda:0"):
+        import torch
+        cfg, wtss, keep = None, [], []
+        for (a_fmt, b_fmt) in adapters:
+            c, wts, k = _marshal(w_fmt, a_fmt, b_fmt, max_m=max_m, x_dtype=x_dtype, y_dtype=y_dtype,
+                                 kernel_policy=EORA_POLICY_AUTO, device=device)
+            cfg = cfg or c
+            wtss.append(wts); keep.append(k)
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.y_torch_dtype = {"f16": torch.float16, "bf16": torch.bfloat16, "f32": torch.float32}[y_dtype]
+        with torch.cuda.device(self.device):
+            self.handle = eora_linear_create_multi(cfg, wtss)
+        del keep
+
+    def forward(self, x, adapter_ids, y=None, stream=None):
+        import torch
+        m = x.shape[0]
+        if y is None:
+            y = torch.empty((m, self.cfg.d_out), dtype=self.y_torch_dtype, device=x.device)
+        eora_linear_forward_multi(self.handle, x, m, adapter_ids, y, stream)
+        return y
 
     def device_status(self) -> int:
         return eora_linear_last_device_status(self.handle)

@@ -64,8 +64,12 @@ struct DecodeArgs {
   int n_sub;
   uint32_t b_np;                          // pairs of B per layer: the activations of B's blob (pair, tile) are
                                           // pair (layer(tile) * b_np + pair) of t
+  // Several adapters on one backbone: pair p of B belongs to adapter p / adp_pairs, and token i uses adapter
+  // adp[i] (-1: none).  adp_pairs == 0: one adapter for all tokens.
+  uint32_t adp_pairs;
+  int adp[8];
   float* d_t; float* y_ws; uint32_t* counters; int* dev_status;
-  int m, d_in, r_pad, n_pad, x_dtype, y_dtype;   // r_pad: columns of t (all fused layers)
+  int m, d_in, r_pad, n_pad, x_dtype, y_dtype;   // r_pad: columns of t (all fused layers / adapters)
   unsigned long long* trace;
 };
 
@@ -106,6 +110,16 @@ __device__ __forceinline__ void load_x_pair(uint32_t (&xr)[16], const DecodeArgs
 // The same for t (fp32 sums in d_t [8][r_pad]), split into high and low fp16 parts.
 __device__ __forceinline__ void load_t_pair(uint32_t (&xh)[16], uint32_t (&xl)[16], const DecodeArgs& p, uint32_t pair, int lane) {
   const int g = lane >> 2, t = lane & 3;
+  if (p.adp_pairs) {                      // the token takes part only in its own adapter's pairs
+    int mine = p.adp[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) if (g == i) mine = p.adp[i];
+    if (mine < 0 || (uint32_t)mine != pair / p.adp_pairs) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) { xh[i] = 0u; xl[i] = 0u; }
+      return;
+    }
+  }
   const float* src = p.d_t + (size_t)g * p.r_pad + pair * 128 + 8 * t;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -527,7 +541,8 @@ int decode_launch_count(const Handle*, int m) { return (m + 7) / 8; }
 
 int decode_grid(const Handle* h, int) { return h->sm_count * kCtasPerSm; }
 
-cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st) {
+cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st,
+                                  const int32_t* adapter_ids) {
   const bool ab = h->cfg.rank > 0;
   DecodeArgs a = {};
   a.w_q = h->w.q; a.w_nt = h->w.nt; a.w_sz2 = h->w.sz2; a.w_per_copy = blobs_per_copy(h->w);
@@ -602,6 +617,14 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
     a.m = m - m0 < 8 ? m - m0 : 8;
     a.x = reinterpret_cast<const uint8_t*>(x) + (size_t)m0 * h->cfg.d_in * 2;
     for (int i = 0; i < h->n_sub; ++i) a.ys[i] = reinterpret_cast<uint8_t*>(ys[i]) + (size_t)m0 * h->sub_dout[i] * ybytes;
+    a.adp_pairs = 0;
+    if (h->multi) {
+      a.adp_pairs = (uint32_t)h->r_pad / 128;
+      for (int i = 0; i < 8; ++i) {
+        const int id = (adapter_ids && m0 + i < m) ? adapter_ids[m0 + i] : -1;
+        a.adp[i] = (id >= 0 && id < h->n_adapters) ? id : -1;
+      }
+    }
     cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf)
                   : h->w.fmt == FMT_Q3 ? launch_ab<FMT_Q3>(cfg, a, abf) : launch_ab<FMT_SP24>(cfg, a, abf);
     if (e != cudaSuccess) return e;

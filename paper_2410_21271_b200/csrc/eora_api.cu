@@ -122,6 +122,18 @@ WMat tile_view(const WMat& m, int t0) {
   return v;
 }
 
+// A view of `m` that starts at pair p0 of the reduction axis and is n_pairs long.
+WMat pair_view(const WMat& m, int p0, int n_pairs) {
+  WMat v = m;
+  v.q = m.q + (int64_t)p0 * m.nt * m.blob;
+  v.np = n_pairs; v.kc = 2 * n_pairs; v.k_red = 128 * n_pairs;
+  return v;
+}
+
+// One backbone with n adapters (decode only): cfg is the layer's, wts[j] carries adapter j (the backbone
+// pointers are taken from wts[0]).
+int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* wts, int n, void* stream, eora_linear_t* out);
+
 // One layer (n == 1) or n layers that share X, stacked along the output axis (fused, decode only).
 int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, int n, void* stream, eora_linear_t* out) {
   if (out) *out = nullptr;
@@ -164,6 +176,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
 
   h->r_pad = (int)align_up(c.rank, 128);
   h->n_sub = n;
+  h->n_adapters = 1;
   h->t_cols = n * (h->r_pad > 0 ? h->r_pad : 128);
   h->sub_tile0[0] = 0;
   for (int i = 0; i < n; ++i) {
@@ -244,6 +257,106 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   return EORA_OK;
 }
 
+int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* wts, int n, void* stream, eora_linear_t* out) {
+  if (out) *out = nullptr;
+  if (!cfg || !wts || !out) return EORA_ERR_NULL_ARG;
+  if (n < 1 || n > 8) return EORA_ERR_BAD_SHAPE;
+  const eora_linear_config c = *cfg;
+  int st = check_config(c);
+  if (st != EORA_OK) return st;
+  if (c.rank == 0) return EORA_ERR_BAD_SHAPE;
+  if (c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO) return EORA_ERR_UNSUPPORTED;
+  for (int j = 0; j < n; ++j) {
+    eora_linear_weights w = wts[j];
+    w.w_codes = wts[0].w_codes; w.w_scales = wts[0].w_scales; w.w_zeros = wts[0].w_zeros;
+    st = check_weights(c, w);
+    if (st != EORA_OK) return st;
+  }
+  const bool quant_w = c.w_format == EORA_W_QUANT;
+
+  eora_linear* obj = new (std::nothrow) eora_linear();
+  if (!obj) return EORA_ERR_CUDA;
+  Handle* h = &obj->h;
+  *h = Handle();
+  h->cfg = c;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  auto fail = [&](int code) {
+    if (h->weight_mem) cudaFree(h->weight_mem);
+    if (h->scratch_mem) cudaFree(h->scratch_mem);
+    delete obj;
+    return code;
+  };
+  if (cudaGetDevice(&h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  h->r_pad = (int)align_up(c.rank, 128);
+  h->n_sub = 1;
+  h->n_adapters = n;
+  h->multi = 1;
+  h->t_cols = n * h->r_pad;
+  h->sub_tile0[0] = 0;
+  for (int i = 1; i < 5; ++i) h->sub_tile0[i] = c.d_out / 16;
+  h->sub_dout[0] = c.d_out;
+  const bool ab_grouped = c.ab_format == EORA_AB_Q4 || c.ab_format == EORA_AB_Q3;
+  const int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : c.ab_format == EORA_AB_Q3 ? FMT_Q3 : FMT_Q8;
+  wmat_shape(h->w, quant_w ? (c.w_bits == 4 ? FMT_Q4 : FMT_Q3) : FMT_SP24, c.d_out, c.d_in, quant_w ? c.w_group : 0);
+  const int ga = ab_grouped ? c.ab_group : 0;
+  const int gb = ab_grouped ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 128;   // per-channel: one entry per pair
+  wmat_shape(h->a, ab_fmt, n * h->r_pad, c.d_in, ga);
+  wmat_shape(h->b, ab_fmt, c.d_out, n * h->r_pad, gb);
+
+  Carve sizing{nullptr, 0};
+  { WMat tw = h->w, ta = h->a, tb = h->b; wmat_carve(tw, sizing); wmat_carve(ta, sizing); wmat_carve(tb, sizing); }
+  h->weight_bytes = sizing.off;
+  if (cudaMalloc(&h->weight_mem, (size_t)h->weight_bytes) != cudaSuccess) { h->weight_mem = nullptr; return fail(EORA_ERR_CUDA); }
+  Carve wc{reinterpret_cast<char*>(h->weight_mem), 0};
+  wmat_carve(h->w, wc); wmat_carve(h->a, wc); wmat_carve(h->b, wc);
+
+  const int64_t rp = h->t_cols;
+  for (int pass = 0; pass < 2; ++pass) {
+    Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
+    h->t_ws = sc.take<float>(256);            // prefill scratch is not used by this kind of handle
+    h->t_gen = sc.take<float>(256);
+    h->t16 = sc.take<__half>(256);
+    h->d_t = sc.take<float>(8 * rp * 4);
+    h->y_ws = sc.take<float>((int64_t)8 * h->w.n_rows * 4);
+    h->counters = sc.take<uint32_t>((int64_t)(h->w.nt + 2) * 4);
+    h->dev_status = sc.take<int>(256);
+    h->x_stage = sc.take<void>((int64_t)c.max_m * c.d_in * 2);
+    h->y_stage = sc.take<void>((int64_t)c.max_m * c.d_out * y_elem_bytes(c.y_dtype));
+    if (pass == 0) {
+      h->scratch_bytes = sc.off;
+      if (cudaMalloc(&h->scratch_mem, (size_t)h->scratch_bytes) != cudaSuccess) { h->scratch_mem = nullptr; return fail(EORA_ERR_CUDA); }
+    }
+  }
+  if (cudaMemsetAsync(h->scratch_mem, 0, (size_t)h->scratch_bytes, s) != cudaSuccess) return fail(EORA_ERR_CUDA);
+
+  cudaError_t e;
+  if (quant_w) e = launch_repack_quant(h->w, wts[0].w_codes, wts[0].w_scales, wts[0].w_zeros, c.w_bits, c.d_out, c.d_in, s);
+  else e = launch_repack_sp24(h->w, wts[0].w_codes, wts[0].w_zeros, c.d_out, c.d_in, s);
+  for (int j = 0; j < n && e == cudaSuccess; ++j) {
+    const eora_linear_weights& w = wts[j];
+    const WMat av = tile_view(h->a, j * h->r_pad / 16);
+    const WMat bv = pair_view(h->b, j * h->r_pad / 128, h->r_pad / 128);
+    const int a_nt = h->r_pad / 16;
+    if (c.ab_format == EORA_AB_F16) {
+      e = launch_repack_f16(av, w.a, c.rank, c.d_in, s, a_nt);
+      if (e == cudaSuccess) e = launch_repack_f16(bv, w.b, c.d_out, c.rank, s);
+    } else if (ab_grouped) {
+      const int bits = c.ab_format == EORA_AB_Q4 ? 4 : 3;
+      e = launch_repack_quant(av, w.a, w.a_scales, w.a_zeros, bits, c.rank, c.d_in, s, a_nt);
+      if (e == cudaSuccess) e = launch_repack_quant(bv, w.b, w.b_scales, w.b_zeros, bits, c.d_out, c.rank, s);
+    } else {
+      e = launch_repack_q8(av, w.a, w.a_scales, w.a_zeros, c.rank, c.d_in, s, a_nt);
+      if (e == cudaSuccess) e = launch_repack_q8(bv, w.b, w.b_scales, w.b_zeros, c.d_out, c.rank, s);
+    }
+  }
+  if (e != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (!decode_supported(h, 1)) return fail(EORA_ERR_UNSUPPORTED);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  *out = obj;
+  return EORA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -255,6 +368,25 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
 int eora_linear_create_fused(const eora_linear_config* cfgs, const eora_linear_weights* wts, int32_t n_layers, void* stream,
                              eora_linear_t* out) {
   return create_impl(cfgs, wts, n_layers, stream, out);
+}
+
+int eora_linear_create_multi(const eora_linear_config* cfg, const eora_linear_weights* wts, int32_t n_adapters, void* stream,
+                             eora_linear_t* out) {
+  return create_multi_impl(cfg, wts, n_adapters, stream, out);
+}
+
+int eora_linear_forward_multi(eora_linear_t obj, const void* x, int32_t m, const int32_t* adapter_ids, void* y, void* stream) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (m == 0) return EORA_OK;
+  if (m < 0) return EORA_ERR_BAD_SHAPE;
+  if (!x || !y || !adapter_ids) return EORA_ERR_NULL_ARG;
+  if (!aligned16(x) || !aligned16(y)) return EORA_ERR_MISALIGNED;
+  Handle* h = &obj->h;
+  if (!h->multi) return EORA_ERR_UNSUPPORTED;
+  if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  if (!decode_supported(h, m)) return EORA_ERR_UNSUPPORTED;
+  void* ys[1] = {y};
+  return launch_decode_forward(h, x, m, ys, reinterpret_cast<cudaStream_t>(stream), adapter_ids) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
 }
 
 int eora_linear_forward_fused(eora_linear_t obj, const void* x, int32_t m, void* const* ys, void* stream) {
@@ -333,6 +465,7 @@ int eora_linear_forward(eora_linear_t obj, const void* x, int32_t m, void* y, vo
   if (!aligned16(x) || !aligned16(y)) return EORA_ERR_MISALIGNED;
   Handle* h = &obj->h;
   if (h->n_sub != 1) return EORA_ERR_UNSUPPORTED;             // fused layers have several outputs: forward_fused
+  if (h->multi) return EORA_ERR_UNSUPPORTED;                  // several adapters: forward_multi says which
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   int p = pick_path(h, m);

@@ -180,7 +180,11 @@ struct Handle {
   int n_sub;
   int sub_tile0[5];
   int sub_dout[4];
-  int t_cols;            // columns of t: n_sub * r_pad
+  int t_cols;            // columns of t: n_sub * r_pad (or n_adapters * r_pad)
+  // Several adapters for one backbone: their A's are stacked along the rank axis like those of fused layers,
+  // their B's along the reduction axis (adapter j owns pairs [j * r_pad / 128, (j + 1) * r_pad / 128) of B).
+  int n_adapters;        // 1 for a plain layer
+  int multi;             // 1: created with per-token adapter selection (eora_linear_create_multi)
   void* prefill_state;   // owned by prefill.cu (tensor maps), may be NULL
   void* trace;           // optional caller-owned timestamp buffer, may be NULL
 };
@@ -198,7 +202,8 @@ cudaError_t launch_generic_forward(const Handle* h, const void* x, int m, void* 
 int generic_launch_count(const Handle* h);
 
 bool decode_supported(const Handle* h, int m);
-cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st);
+cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st,
+                                  const int32_t* adapter_ids = nullptr);
 int decode_launch_count(const Handle* h, int m);
 int decode_grid(const Handle* h, int m);
 
