@@ -275,6 +275,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_x[kMaxXStages], empty_x[kMaxXStages], full_w[kMaxWStages], empty_w[kMaxWStages], acc_full;
   __shared__ uint32_t tmem_base_s;
+  __shared__ int fail_s;                 // set by an epilogue warp whose bounded wait ran out
   // 1024-byte alignment of the operand tiles (the swizzle pattern is anchored at 1 KB)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -288,6 +289,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   const uint32_t xbytes = (uint32_t)p.bt * 128;
 
   if (threadIdx.x == 0) {
+    fail_s = 0;
     for (int i = 0; i < p.sx; ++i) { mbar_init(full_x + i, 1); mbar_init(empty_x + i, 1); }
     for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8 * nh); mbar_init(empty_w + i, 1); }
     mbar_init(&acc_full, 1);
@@ -355,6 +357,10 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       // Epilogue (4 warps).  Warp dw owns accumulator rows (= weight rows n) 32*dw .. 32*dw+31 of each half,
       // its TMEM lanes; columns are tokens.
       if (ok) ok = mbar_wait_warp(&acc_full, 0, p.dev_status, lane);
+      // the four epilogue warps meet at barriers below: they must all take the same way
+      if (!ok) *reinterpret_cast<volatile int*>(&fail_s) = 1;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      ok = *reinterpret_cast<volatile int*>(&fail_s) == 0;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int nl = dw * 32 + lane;                     // local weight row inside the half
       if (p.out_dtype == 3) {
