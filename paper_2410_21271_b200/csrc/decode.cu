@@ -95,9 +95,12 @@ __device__ __forceinline__ void load_x_pair(uint32_t (&xr)[16], const DecodeArgs
   const int g = lane >> 2, t = lane & 3;
   if (g < p.m) {
     const uint16_t* src = reinterpret_cast<const uint16_t*>(p.x) + (size_t)g * p.d_in + pair * 128 + 8 * t;
+    uint4 u[4];                            // all loads first: a use in between would serialise the round trips
+#pragma unroll
+    for (int i = 0; i < 4; ++i) u[i] = ld_cg_u4(src + 32 * i);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      uint4 v = ld_cg_u4(src + 32 * i);
+      uint4 v = u[i];
       if (p.x_dtype == EORA_X_BF16) { v.x = bf2_to_h2(v.x); v.y = bf2_to_h2(v.y); v.z = bf2_to_h2(v.z); v.w = bf2_to_h2(v.w); }
       xr[4 * i] = v.x; xr[4 * i + 1] = v.y; xr[4 * i + 2] = v.z; xr[4 * i + 3] = v.w;
     }
@@ -121,11 +124,14 @@ __device__ __forceinline__ void load_t_pair(uint32_t (&xh)[16], uint32_t (&xl)[1
     }
   }
   const float* src = p.d_t + (size_t)g * p.r_pad + pair * 128 + 8 * t;
+  uint4 ua[8];                             // all loads first: a use in between would serialise the round trips
+#pragma unroll
+  for (int i = 0; i < 8; ++i) ua[i] = ld_cg_u4(src + 32 * (i >> 1) + 4 * (i & 1));
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
 #pragma unroll
     for (int hq = 0; hq < 2; ++hq) {
-      const uint4 u = ld_cg_u4(src + 32 * i + 4 * hq);
+      const uint4 u = ua[2 * i + hq];
       const float f[4] = {__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w)};
 #pragma unroll
       for (int j = 0; j < 2; ++j) {

@@ -349,10 +349,13 @@ __device__ __forceinline__ void load_x_i8(XI8& xi, const void* x, bool bf16, uin
   const uint16_t* src = reinterpret_cast<const uint16_t*>(x) + pair * 128 + 8 * t;
   float2 v[4][4];                                     // [2 * c + blk][pair of elements]
   float amax = 0.f;
+  uint4 ua[4];                                        // all loads first: a use in between would serialise the round trips
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(ua[i].x), "=r"(ua[i].y), "=r"(ua[i].z), "=r"(ua[i].w) : "l"(src + 32 * i) : "memory");
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    uint4 u;
-    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "l"(src + 32 * i) : "memory");
+    const uint4 u = ua[i];
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
