@@ -162,7 +162,10 @@ int eora_linear_forward_fused_host(eora_linear_t h, const void* x_host, int32_t 
 /*
  * The same forward for callers whose activations live in HOST memory: copies x_host (pinned or
  * pageable, [m][d_in]) to a library-owned device staging buffer, runs the forward, copies the
- * result back to y_host ([m][d_out]) and synchronises `stream` before returning.
+ * result back to y_host ([m][d_out]) and synchronises `stream` before returning.  When y_host is
+ * page-locked memory mapped into the device's address space (cudaHostAlloc / cudaHostRegister) and
+ * m <= 64, the kernel stores the result there itself and the copy back is skipped; the bytes
+ * crossing the link are the same.
  */
 int eora_linear_forward_host(eora_linear_t h, const void* x_host, int32_t m, void* y_host, void* stream);
 

@@ -405,6 +405,15 @@ int eora_linear_forward_fused(eora_linear_t obj, const void* x, int32_t m, void*
   return launch_decode_forward(h, x, m, ys, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
 }
 
+// Device-side alias of a host result buffer the GPU can store to directly (page-locked and mapped), else nullptr. Small
+// results are then written by the kernel itself, which saves the copy engine's round trip per output.
+static void* mapped_alias(void* host, int32_t m) {
+  if (m > 64) return nullptr;                    // large results: the copy engine moves them at full link rate
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 int eora_linear_forward_fused_host(eora_linear_t obj, const void* x_host, int32_t m, void* const* ys_host, void* stream) {
   if (!obj) return EORA_ERR_NULL_ARG;
   if (m == 0) return EORA_OK;
@@ -419,14 +428,18 @@ int eora_linear_forward_fused_host(eora_linear_t obj, const void* x_host, int32_
   if (cudaMemcpyAsync(h->x_stage, x_host, (size_t)m * h->cfg.d_in * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return EORA_ERR_CUDA;
   void* ys[4] = {nullptr, nullptr, nullptr, nullptr};
   size_t off = 0;
-  for (int i = 0; i < h->n_sub; ++i) {          // outputs side by side in the staging buffer ([m][d_out_i] each)
+  bool staged[4] = {false, false, false, false};
+  for (int i = 0; i < h->n_sub; ++i) {          // staged outputs side by side in the staging buffer ([m][d_out_i] each)
+    ys[i] = mapped_alias(ys_host[i], m);
+    if (ys[i]) continue;
+    staged[i] = true;
     ys[i] = reinterpret_cast<char*>(h->y_stage) + off;
     off += (size_t)m * h->sub_dout[i] * eb;
   }
   int rc = eora_linear_forward_fused(obj, h->x_stage, m, ys, stream);
   if (rc != EORA_OK) return rc;
   for (int i = 0; i < h->n_sub; ++i)
-    if (cudaMemcpyAsync(ys_host[i], ys[i], (size_t)m * h->sub_dout[i] * eb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EORA_ERR_CUDA;
+    if (staged[i] && cudaMemcpyAsync(ys_host[i], ys[i], (size_t)m * h->sub_dout[i] * eb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EORA_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return EORA_ERR_CUDA;
   return EORA_OK;
 }
@@ -487,9 +500,10 @@ int eora_linear_forward_host(eora_linear_t obj, const void* x_host, int32_t m, v
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   size_t xb = (size_t)m * h->cfg.d_in * 2, yb = (size_t)m * h->cfg.d_out * y_elem_bytes(h->cfg.y_dtype);
   if (cudaMemcpyAsync(h->x_stage, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EORA_ERR_CUDA;
-  int rc = eora_linear_forward(obj, h->x_stage, m, h->y_stage, stream);
+  void* y_dev = mapped_alias(y_host, m);
+  int rc = eora_linear_forward(obj, h->x_stage, m, y_dev ? y_dev : h->y_stage, stream);
   if (rc != EORA_OK) return rc;
-  if (cudaMemcpyAsync(y_host, h->y_stage, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EORA_ERR_CUDA;
+  if (!y_dev && cudaMemcpyAsync(y_host, h->y_stage, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EORA_ERR_CUDA;
   if (cudaStreamSynchronize(s) != cudaSuccess) return EORA_ERR_CUDA;
   return EORA_OK;
 }

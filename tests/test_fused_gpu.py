@@ -59,6 +59,27 @@ def test_fused_fullsize(names, w):
     F.close()
 
 
+@pytest.mark.parametrize("pinned", [(True, True), (True, False), (False, False)])
+def test_fused_forward_host(pinned):
+    """The host entry point: every combination of page-locked (written by the kernel) and pageable (staged) results."""
+    import torch
+    K, Ns, r, M = 512, [96, 160], 128, 5
+    layers = [make_case(80 + i, K, N, r, w="q3") for i, N in enumerate(Ns)]
+    x = gen.make_x(81, M, K)
+    F = eora.FusedLayers(layers, max_m=M)
+    xh = torch.from_numpy(x.copy()).pin_memory()
+    yh = [torch.full((M, N), float("nan"), dtype=torch.float16) for N in Ns]
+    yh = [y.pin_memory() if p else y for y, p in zip(yh, pinned)]
+    for rep in range(2):
+        for y in yh:
+            y.fill_(float("nan"))
+        F.forward_host(xh, yh)
+        assert F.device_status() == 0
+        for i, (wf, af, bf) in enumerate(layers):
+            check_parity(yh[i].float().numpy().astype(np.float64), orc.forward(x, "f16", wf, af, bf), f"layer {i} call {rep}")
+    F.close()
+
+
 def test_fused_argument_errors():
     import torch
     K = 256
