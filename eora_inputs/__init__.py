@@ -169,3 +169,15 @@ def make_sparse24(seed: int, K: int, N: int) -> dict:
     for i in range(8):
         meta |= nib[:, :, i] << np.uint32(4 * i)
     return {"kind": "sparse24", "rows": K, "cols": N, "values": values, "meta": meta}
+
+
+def make_sparse24_quant(seed: int, K: int, N: int, bits: int = 4, group: int = 128) -> dict:
+    """2:4 structured-sparse backbone whose kept values are quantised group-wise: the seeded 2:4 matrix,
+    its [K/2][N] kept values rounded to `bits` with groups of `group` original k (group/2 kept values)."""
+    sp = make_sparse24(seed, K, N)
+    g = min(group, K)
+    assert g % 2 == 0 and K % g == 0
+    kept = np.ascontiguousarray(sp["values"].T)                 # [K/2][N]
+    qz = quantize_matrix_bits(kept, bits, g // 2)
+    return {"kind": "sparse24q", "rows": K, "cols": N, "bits": bits, "group": g, "codes": qz["codes"],
+            "scales": qz["scales"], "zeros": qz["zeros"], "meta": sp["meta"]}

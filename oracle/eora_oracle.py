@@ -33,6 +33,13 @@ the bit layouts below are this library's interchange format):
   consecutive k, in increasing-k order) and uint32 meta [N][K/32]; quad j owns
   nibble (meta[n][j/8] >> 4*(j%8)) & 0xF = p0 | p1 << 2 with 0 <= p0 < p1 <= 3,
   and w[4j+p0][n] = values[n][2j], w[4j+p1][n] = values[n][2j+1], others 0.
+* 2:4 sparse AND 4-bit (the appendix on sparsity & quantisation error compensation;
+  the paper prunes to 2:4 and quantises to 4 bits without fixing a storage):
+  the K/2 kept values of a column are a group-wise asymmetric 4-bit matrix
+  [K/2][N] in the layout above (codes uint32 [K/16][N]); a group covers `group`
+  consecutive k of the ORIGINAL axis, i.e. group/2 kept values, so scales are
+  fp16 [K/group][N] and zeros [K/group][N/8]; meta as for 2:4.
+  w[4j+p0][n] = (q[2j][n] - z) * s, w[4j+p1][n] = (q[2j+1][n] - z) * s, others 0.
 
 All floating point is float64; inputs are converted exactly from their storage
 types.  No blocking, no fusion: unpack, dequantise, two matrix products.
@@ -133,6 +140,8 @@ def dequant_matrix(fmt: dict) -> np.ndarray:
       'quant'  : b-bit group-wise asymmetric: 'codes', 'scales', 'zeros', 'bits', 'group', 'rows', 'cols'
       'q8'     : 8-bit per-channel: 'codes' uint8 [rows][cols], 'scales' fp16 [cols], 'zeros' uint8 [cols]
       'sparse24': 'values' fp16 [cols][rows/2], 'meta' uint32 [cols][rows/32], 'rows', 'cols'
+      'sparse24q': 2:4 + 4-bit: 'codes', 'scales', 'zeros' of the kept values ([rows/2][cols], groups of
+                 group/2), 'meta' uint32 [cols][rows/32], 'bits' (4), 'group', 'rows', 'cols'
     rows is the reduction axis of the product the matrix is used in.
     """
     kind = fmt["kind"]
@@ -151,6 +160,9 @@ def dequant_matrix(fmt: dict) -> np.ndarray:
         return (q - z[None, :]).astype(np.float64) * s[None, :]
     if kind == "sparse24":
         return expand_sparse24(fmt["values"], fmt["meta"], fmt["rows"], fmt["cols"])
+    if kind == "sparse24q":
+        return expand_sparse24_quant(fmt["codes"], fmt["scales"], fmt["zeros"], fmt["meta"], fmt["bits"],
+                                     fmt["group"], fmt["rows"], fmt["cols"])
     raise ValueError(kind)
 
 
@@ -172,7 +184,22 @@ def deq_fp16(q: np.ndarray, z: np.ndarray, s_f16: np.ndarray, group: int) -> np.
 # ----------------------------------------------------------------------------
 def expand_sparse24(values: np.ndarray, meta: np.ndarray, K: int, N: int) -> np.ndarray:
     """Dense float64 [K][N] from compressed 2:4 storage (see module docstring)."""
-    vals = to_f64(values, "f16")
+    return scatter24(to_f64(values, "f16"), meta, K, N)
+
+
+def expand_sparse24_quant(codes, scales, zeros, meta, bits: int, group: int, K: int, N: int) -> np.ndarray:
+    """Dense float64 [K][N] of a backbone that is 2:4 sparse with its kept values quantised (appendix on
+    sparsity & quantisation error compensation): dequantise the K/2 kept values of every column (a group
+    of `group` original k holds group/2 of them), then put them where the metadata says."""
+    assert group % 2 == 0 and K % group == 0
+    q = unpack_codes(codes, bits, K // 2)
+    z = unpack_zeros(zeros, bits, N)
+    kept = dequant_groupwise(q, z, scales, group // 2)          # [K/2][N]
+    return scatter24(np.ascontiguousarray(kept.T), meta, K, N)
+
+
+def scatter24(vals: np.ndarray, meta: np.ndarray, K: int, N: int) -> np.ndarray:
+    """vals float64 [N][K/2] (kept values in increasing-k order) -> dense [K][N] by the position nibbles."""
     meta = np.asarray(meta)
     assert vals.shape == (N, K // 2) and meta.shape == (N, K // 32) and meta.dtype == np.uint32
     w = np.zeros((K, N), dtype=np.float64)

@@ -359,6 +359,61 @@ def test_sparse24_hand_packed():
     assert W[:8].tolist() == [0.0, 2.0, 0.0, -4.0, 1.0, 0.0, 3.0, 0.0]
 
 
+def test_sparse24_quant_scalar_expansion():
+    """2:4 + 4-bit (appendix on sparsity & quantisation compensation): bit-by-bit scalar unpack of every stored
+    field, independent of the oracle's vectorised helpers."""
+    K, N, group = 256, 16, 128
+    sq = gen.make_sparse24_quant(44, K, N, 4, group)
+    codes, scales, zeros, meta = sq["codes"], sq["scales"], sq["zeros"], sq["meta"]
+    assert codes.shape == (K // 16, N) and scales.shape == (K // group, N) and zeros.shape == (K // group, N // 8)
+    Wd = np.zeros((K, N))
+    for n in range(N):
+        for j in range(K // 4):
+            nib = (int(meta[n][j // 8]) >> (4 * (j % 8))) & 0xF
+            pos = (nib & 3, nib >> 2)
+            for i in range(2):
+                c = 2 * j + i                                       # index among the kept values
+                q = (int(codes[c // 8][n]) >> (4 * (c % 8))) & 0xF
+                g = (4 * j) // group                                # group of the ORIGINAL k
+                z = (int(zeros[g][n // 8]) >> (4 * (n % 8))) & 0xF
+                Wd[4 * j + pos[i], n] = (q - z) * float(scales[g][n])
+    assert np.array_equal(orc.dequant_matrix(sq), Wd)
+    # the zero pattern is the 2:4 one, and the forward equals the dense forward on the expanded matrix
+    assert np.all((Wd.reshape(K // 4, 4, N) != 0).sum(axis=1) <= 2)
+    af, bf = gen.make_ab_f16(45, K, N, 32)
+    x = gen.make_x(46, 3, K)
+    assert np.array_equal(orc.forward(x, "f16", sq, af, bf), orc.forward(x, "f16", {"kind": "f64", "data": Wd}, af, bf))
+
+
+def test_sparse24_quant_hand_packed():
+    # K = 32, one column, group 32 (16 kept values): scale 0.5, zero 3; quad 0 keeps positions (1, 3) with codes
+    # (7, 0), quad 1 positions (0, 2) with codes (3, 15); the other quads positions (0, 1) with code 3 (-> 0)
+    codes = np.zeros((2, 1), dtype=np.uint32)
+    codes[0, 0] = 7 | 0 << 4 | 3 << 8 | 15 << 12 | 0x33330000
+    codes[1, 0] = 0x33333333
+    scales = np.array([[0.5]], dtype=np.float16)
+    zeros = np.array([[3]], dtype=np.uint32)
+    meta = np.array([[0xD | (0x8 << 4) | 0x44444400]], dtype=np.uint32)
+    W = orc.expand_sparse24_quant(codes, scales, zeros, meta, 4, 32, 32, 1)[:, 0]
+    assert W[:8].tolist() == [0.0, 2.0, 0.0, -1.5, 0.0, 0.0, 6.0, 0.0]
+    assert not W[8:].any()
+
+
+def test_sparse24_quant_tracks_the_sparse_matrix():
+    """The generator quantises the kept values of the seeded 2:4 matrix: same pattern, error within half a step."""
+    K, N, group = 512, 32, 128
+    sp, sq = gen.make_sparse24(47, K, N), gen.make_sparse24_quant(47, K, N, 4, group)
+    assert np.array_equal(sp["meta"], sq["meta"])
+    Ws, Wq = orc.dequant_matrix(sp), orc.dequant_matrix(sq)
+    step = np.repeat(sq["scales"].astype(np.float64), group, axis=0)       # [K][N]
+    assert np.all(np.abs(Ws - Wq) <= 0.5 * step * (1 + 1e-3) + 1e-12)
+    assert np.all(Wq[Ws == 0] == 0)
+    # group-size-K (channel-wise) and a group of 64 go through the same code
+    for g in (64, K):
+        Wg = orc.dequant_matrix(gen.make_sparse24_quant(47, K, N, 4, g))
+        assert np.all(Wg[Ws == 0] == 0) and np.abs(Wg - Ws).max() < 0.02
+
+
 # --------------------------------------------------------------------------- generator properties
 @pytest.mark.parametrize("bits,group", [(4, 128), (8, 256)])
 def test_rtn_quantiser_error_bound_and_idempotence(bits, group):
