@@ -39,6 +39,12 @@
  *       quad of consecutive k in increasing-k order), w_zeros = uint32 meta [d_out][d_in/32]:
  *       quad j owns nibble (meta[n][j/8] >> 4*(j%8)) & 0xF = p0 | p1<<2, 0 <= p0 < p1 <= 3;
  *       w_scales is unused (may be NULL).
+ *   2:4 + 4-bit backbone (w_format 2; the appendix on sparsity & quantisation error compensation prunes to 2:4
+ *       and quantises to 4 bits): the d_in/2 kept values of every column are a 4-bit group-wise matrix
+ *       [d_in/2][d_out] in the code layout above (w_codes uint32 [d_in/16][d_out]); w_group counts ORIGINAL
+ *       reduction elements, so a group holds w_group/2 kept values: w_scales fp16 [d_in/w_group][d_out],
+ *       w_zeros uint32 [d_in/w_group][d_out/8]; w_meta = the 2:4 position words uint32 [d_out][d_in/32] as
+ *       for w_format 1.  w[4j+p0][n] = (q[2j][n] - z) * s, w[4j+p1][n] = (q[2j+1][n] - z) * s, others 0.
  */
 #ifndef EORA_LINEAR_H_
 #define EORA_LINEAR_H_
@@ -62,7 +68,7 @@ enum {
   EORA_ERR_DEVICE_TIMEOUT = -7
 };
 
-enum { EORA_W_QUANT = 0, EORA_W_SPARSE24 = 1 };
+enum { EORA_W_QUANT = 0, EORA_W_SPARSE24 = 1, EORA_W_SPARSE24_Q4 = 2 };
 enum { EORA_AB_F16 = 0, EORA_AB_Q4 = 1, EORA_AB_Q8 = 2, EORA_AB_Q3 = 3 };
 enum { EORA_X_F16 = 0, EORA_X_BF16 = 1 };
 enum { EORA_Y_F16 = 0, EORA_Y_BF16 = 1, EORA_Y_F32 = 2 };
@@ -76,8 +82,8 @@ typedef struct {
   int32_t d_in;        /* K; multiple of 128 */
   int32_t d_out;       /* N; multiple of 32 */
   int32_t rank;        /* r >= 0, multiple of 8 (0 = no adapter: the plain compressed layer) */
-  int32_t w_format;    /* EORA_W_QUANT or EORA_W_SPARSE24 */
-  int32_t w_bits;      /* 3 or 4 (EORA_W_QUANT) */
+  int32_t w_format;    /* EORA_W_QUANT, EORA_W_SPARSE24 or EORA_W_SPARSE24_Q4 */
+  int32_t w_bits;      /* 3 or 4 (EORA_W_QUANT); 4 (EORA_W_SPARSE24_Q4) */
   int32_t w_group;     /* group size along d_in: multiple of 64 dividing d_in (d_in = channel-wise) */
   int32_t ab_format;   /* EORA_AB_F16 / EORA_AB_Q4 / EORA_AB_Q8 / EORA_AB_Q3 */
   int32_t ab_group;    /* group size for EORA_AB_Q4 / _Q3 (128); B uses min(ab_group, rank) */
@@ -98,6 +104,7 @@ typedef struct {
   const void* b;
   const void* b_scales;
   const void* b_zeros;
+  const void* w_meta;    /* 2:4 position words of EORA_W_SPARSE24_Q4; unused (may be NULL) otherwise */
 } eora_linear_weights;
 
 /*

@@ -18,7 +18,7 @@ HEADER_PATH = os.path.join(os.path.dirname(_HERE), "include", "eora_linear.h")
 EORA_OK = 0
 EORA_ERR_NULL_ARG, EORA_ERR_BAD_SHAPE, EORA_ERR_UNSUPPORTED, EORA_ERR_MISALIGNED = -1, -2, -3, -4
 EORA_ERR_M_TOO_LARGE, EORA_ERR_CUDA, EORA_ERR_DEVICE_TIMEOUT = -5, -6, -7
-EORA_W_QUANT, EORA_W_SPARSE24 = 0, 1
+EORA_W_QUANT, EORA_W_SPARSE24, EORA_W_SPARSE24_Q4 = 0, 1, 2
 EORA_AB_F16, EORA_AB_Q4, EORA_AB_Q8, EORA_AB_Q3 = 0, 1, 2, 3
 EORA_X_F16, EORA_X_BF16 = 0, 1
 EORA_Y_F16, EORA_Y_BF16, EORA_Y_F32 = 0, 1, 2
@@ -33,7 +33,7 @@ class eora_linear_config(Structure):
 
 class eora_linear_weights(Structure):
     _fields_ = [(n, c_void_p) for n in ("w_codes", "w_scales", "w_zeros", "a", "a_scales", "a_zeros",
-                                        "b", "b_scales", "b_zeros")]
+                                        "b", "b_scales", "b_zeros", "w_meta")]
 
 
 class EoraError(RuntimeError):
@@ -294,6 +294,12 @@ def _marshal(w_fmt: dict, a_fmt, b_fmt, *, max_m: int, x_dtype: str, y_dtype: st
     elif w_fmt["kind"] == "sparse24":
         cfg.w_format = EORA_W_SPARSE24
         bufs = [_dev(w_fmt["values"], device), None, _dev(w_fmt["meta"], device)]
+    elif w_fmt["kind"] == "sparse24q":
+        cfg.w_format, cfg.w_bits, cfg.w_group = EORA_W_SPARSE24_Q4, w_fmt["bits"], w_fmt["group"]
+        bufs = [_dev(w_fmt["codes"], device), _dev(w_fmt["scales"], device), _dev(w_fmt["zeros"], device)]
+        meta = _dev(w_fmt["meta"], device)
+        keep.append(meta)
+        wts.w_meta = _ptr(meta)
     else:
         raise ValueError(w_fmt["kind"])
     keep += bufs

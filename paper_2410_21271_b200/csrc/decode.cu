@@ -413,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   r.bars = reinterpret_cast<uint64_t*>(smem + kWarps * kRing * kSlotBytes) + warp * kRing;
   r.slot = 0; r.parity = 0; r.pseg = 0;
   r.aux = 0;
-  if constexpr (WF == FMT_SP24) {
+  if constexpr (WF == FMT_SP24 || WF == FMT_SQ4) {
     // every warp writes the same 16 values, so no CTA-wide barrier is needed before a warp reads them
     uint32_t* lut = reinterpret_cast<uint32_t*>(smem + kWarps * kRing * kSlotBytes + kBarBytes);
     if (lane < 16) lut[lane] = sp24_selectors((uint32_t)lane);
@@ -517,6 +517,7 @@ double blob_cost(int fmt, bool hilo) {
     case FMT_Q8: return 1.40;
     case FMT_F16: return hilo ? 1.30 : 1.10;
     case FMT_SP24: return 1.60;
+    case FMT_SQ4: return 1.10;
     default: return 0.0;
   }
 }
@@ -537,7 +538,7 @@ uint32_t blobs_per_copy(const WMat& m) {
 
 bool decode_supported(const Handle* h, int m) {
   if (m < 1 || m > 64) return false;
-  if (h->w.fmt != FMT_Q4 && h->w.fmt != FMT_Q3 && h->w.fmt != FMT_SP24) return false;
+  if (h->w.fmt != FMT_Q4 && h->w.fmt != FMT_Q3 && h->w.fmt != FMT_SP24 && h->w.fmt != FMT_SQ4) return false;
   if (h->w.blob > kSlotBytes) return false;
   if (h->cfg.rank > 0 && (h->a.blob > kSlotBytes || h->b.blob > kSlotBytes)) return false;
   return true;
@@ -632,7 +633,8 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
       }
     }
     cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf)
-                  : h->w.fmt == FMT_Q3 ? launch_ab<FMT_Q3>(cfg, a, abf) : launch_ab<FMT_SP24>(cfg, a, abf);
+                  : h->w.fmt == FMT_Q3 ? launch_ab<FMT_Q3>(cfg, a, abf)
+                  : h->w.fmt == FMT_SQ4 ? launch_ab<FMT_SQ4>(cfg, a, abf) : launch_ab<FMT_SP24>(cfg, a, abf);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

@@ -140,7 +140,7 @@ __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t c
   return d;
 }
 
-template <int FMT> constexpr bool is_quant() { return FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8; }
+template <int FMT> constexpr bool is_quant() { return fmt_quantised(FMT); }
 
 // Build the A-operand registers of the four mma of one tile from its blob in shared memory.
 // a[i][*]: mma i = 2*blk + sub; entries are fp16x2.
@@ -250,6 +250,26 @@ __device__ __forceinline__ void tile_frags(const uint8_t* blob, int lane, const 
           asm volatile("ld.shared.u32 %0, [%1];" : "=r"(sel) : "r"(aux + nib * 4));
           a[blk * 2 + quad][hf] = prmt(vv[hf][quad], 0u, sel);
           a[blk * 2 + quad][hf + 2] = prmt(vv[hf][quad], 0u, sel >> 16);
+        }
+      }
+    }
+  } else if constexpr (FMT == FMT_SQ4) {
+    // 2:4 pattern with 4-bit kept values: the quad's two codes -> exact fp16 (q - z), then spread like SP24
+    const uint2 v = *reinterpret_cast<const uint2*>(blob + lane * 8);
+    const uint32_t meta = *reinterpret_cast<const uint32_t*>(blob + 256 + lane * 4);
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+      const uint32_t w = blk ? v.y : v.x;
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+        for (int quad = 0; quad < 2; ++quad) {
+          const uint32_t kept = h2sub(and_or(w >> (8 * hf + 4 * quad), 0x000f000fu, kMagic), zc.c[hf][0]);
+          const uint32_t nib = (meta >> (8 * (blk * 2 + hf) + 4 * quad)) & 15u;
+          uint32_t sel;
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(sel) : "r"(aux + nib * 4));
+          a[blk * 2 + quad][hf] = prmt(kept, 0u, sel);
+          a[blk * 2 + quad][hf + 2] = prmt(kept, 0u, sel >> 16);
         }
       }
     }

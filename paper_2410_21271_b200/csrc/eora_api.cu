@@ -50,6 +50,9 @@ int check_config(const eora_linear_config& c) {
   if (c.w_format == EORA_W_QUANT) {
     if (c.w_bits != 3 && c.w_bits != 4) return EORA_ERR_UNSUPPORTED;
     if (c.w_group <= 0 || c.w_group % 64 || c.d_in % c.w_group) return EORA_ERR_BAD_SHAPE;
+  } else if (c.w_format == EORA_W_SPARSE24_Q4) {
+    if (c.w_bits != 4) return EORA_ERR_UNSUPPORTED;
+    if (c.w_group <= 0 || c.w_group % 64 || c.d_in % c.w_group) return EORA_ERR_BAD_SHAPE;
   } else if (c.w_format != EORA_W_SPARSE24) {
     return EORA_ERR_UNSUPPORTED;
   }
@@ -100,9 +103,10 @@ const char* eora_status_string(int s) {
 namespace {
 
 int check_weights(const eora_linear_config& c, const eora_linear_weights& w) {
-  const bool quant_w = c.w_format == EORA_W_QUANT;
-  if (!w.w_codes || !w.w_zeros || (quant_w && !w.w_scales)) return EORA_ERR_NULL_ARG;
-  if (!aligned16(w.w_codes) || !aligned16(w.w_zeros) || !aligned16(w.w_scales)) return EORA_ERR_MISALIGNED;
+  const bool scaled_w = c.w_format != EORA_W_SPARSE24, meta_w = c.w_format == EORA_W_SPARSE24_Q4;
+  if (!w.w_codes || !w.w_zeros || (scaled_w && !w.w_scales) || (meta_w && !w.w_meta)) return EORA_ERR_NULL_ARG;
+  if (!aligned16(w.w_codes) || !aligned16(w.w_zeros) || !aligned16(w.w_scales) || (meta_w && !aligned16(w.w_meta)))
+    return EORA_ERR_MISALIGNED;
   if (c.rank > 0) {
     if (!w.a || !w.b) return EORA_ERR_NULL_ARG;
     if (!aligned16(w.a) || !aligned16(w.b)) return EORA_ERR_MISALIGNED;
@@ -113,6 +117,21 @@ int check_weights(const eora_linear_config& c, const eora_linear_weights& w) {
     }
   }
   return EORA_OK;
+}
+
+// Internal format and group of the backbone.
+int backbone_fmt(const eora_linear_config& c) {
+  if (c.w_format == EORA_W_SPARSE24) return FMT_SP24;
+  if (c.w_format == EORA_W_SPARSE24_Q4) return FMT_SQ4;
+  return c.w_bits == 4 ? FMT_Q4 : FMT_Q3;
+}
+int backbone_group(const eora_linear_config& c) { return c.w_format == EORA_W_SPARSE24 ? 0 : c.w_group; }
+
+cudaError_t repack_backbone(const WMat& dst, const eora_linear_config& c, const eora_linear_weights& w, int d_out, cudaStream_t s,
+                            int nt_sub) {
+  if (c.w_format == EORA_W_QUANT) return launch_repack_quant(dst, w.w_codes, w.w_scales, w.w_zeros, c.w_bits, d_out, c.d_in, s, nt_sub);
+  if (c.w_format == EORA_W_SPARSE24_Q4) return launch_repack_sq4(dst, w.w_codes, w.w_scales, w.w_zeros, w.w_meta, d_out, c.d_in, s, nt_sub);
+  return launch_repack_sp24(dst, w.w_codes, w.w_zeros, d_out, c.d_in, s, nt_sub);
 }
 
 // A view of `m` that starts at row tile t0 (see launch_repack_*).
@@ -156,7 +175,6 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   const bool fused = n > 1;
   if (fused && (c.w_format != EORA_W_QUANT || c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO)) return EORA_ERR_UNSUPPORTED;
   c.d_out = d_out_total;
-  const bool quant_w = c.w_format == EORA_W_QUANT;
 
   eora_linear* obj = new (std::nothrow) eora_linear();
   if (!obj) return EORA_ERR_CUDA;
@@ -186,7 +204,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   for (int i = n + 1; i < 5; ++i) h->sub_tile0[i] = h->sub_tile0[n];
   const bool ab_grouped = c.ab_format == EORA_AB_Q4 || c.ab_format == EORA_AB_Q3;
   int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : c.ab_format == EORA_AB_Q3 ? FMT_Q3 : FMT_Q8;
-  wmat_shape(h->w, quant_w ? (c.w_bits == 4 ? FMT_Q4 : FMT_Q3) : FMT_SP24, c.d_out, c.d_in, quant_w ? c.w_group : 0);
+  wmat_shape(h->w, backbone_fmt(c), c.d_out, c.d_in, backbone_group(c));
   if (c.rank > 0) {
     int ga = ab_grouped ? c.ab_group : 0;
     int gb = ab_grouped ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 0;
@@ -231,8 +249,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     const eora_linear_weights& w = wts[i];
     const int d_out_i = cfgs[i].d_out, nt_i = d_out_i / 16;
     const WMat wv = tile_view(h->w, h->sub_tile0[i]);
-    if (quant_w) e = launch_repack_quant(wv, w.w_codes, w.w_scales, w.w_zeros, c.w_bits, d_out_i, c.d_in, s, fused ? nt_i : -1);
-    else e = launch_repack_sp24(wv, w.w_codes, w.w_zeros, d_out_i, c.d_in, s, -1);
+    e = repack_backbone(wv, c, w, d_out_i, s, fused ? nt_i : -1);
     if (e != cudaSuccess || c.rank == 0) continue;
     const WMat av = tile_view(h->a, fused ? i * h->r_pad / 16 : 0);
     const WMat bv = tile_view(h->b, h->sub_tile0[i]);
@@ -268,11 +285,10 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
   if (c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO) return EORA_ERR_UNSUPPORTED;
   for (int j = 0; j < n; ++j) {
     eora_linear_weights w = wts[j];
-    w.w_codes = wts[0].w_codes; w.w_scales = wts[0].w_scales; w.w_zeros = wts[0].w_zeros;
+    w.w_codes = wts[0].w_codes; w.w_scales = wts[0].w_scales; w.w_zeros = wts[0].w_zeros; w.w_meta = wts[0].w_meta;
     st = check_weights(c, w);
     if (st != EORA_OK) return st;
   }
-  const bool quant_w = c.w_format == EORA_W_QUANT;
 
   eora_linear* obj = new (std::nothrow) eora_linear();
   if (!obj) return EORA_ERR_CUDA;
@@ -298,7 +314,7 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
   h->sub_dout[0] = c.d_out;
   const bool ab_grouped = c.ab_format == EORA_AB_Q4 || c.ab_format == EORA_AB_Q3;
   const int ab_fmt = c.ab_format == EORA_AB_F16 ? FMT_F16 : c.ab_format == EORA_AB_Q4 ? FMT_Q4 : c.ab_format == EORA_AB_Q3 ? FMT_Q3 : FMT_Q8;
-  wmat_shape(h->w, quant_w ? (c.w_bits == 4 ? FMT_Q4 : FMT_Q3) : FMT_SP24, c.d_out, c.d_in, quant_w ? c.w_group : 0);
+  wmat_shape(h->w, backbone_fmt(c), c.d_out, c.d_in, backbone_group(c));
   const int ga = ab_grouped ? c.ab_group : 0;
   const int gb = ab_grouped ? (c.ab_group < c.rank ? c.ab_group : c.rank) : 128;   // per-channel: one entry per pair
   wmat_shape(h->a, ab_fmt, n * h->r_pad, c.d_in, ga);
@@ -330,9 +346,7 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
   }
   if (cudaMemsetAsync(h->scratch_mem, 0, (size_t)h->scratch_bytes, s) != cudaSuccess) return fail(EORA_ERR_CUDA);
 
-  cudaError_t e;
-  if (quant_w) e = launch_repack_quant(h->w, wts[0].w_codes, wts[0].w_scales, wts[0].w_zeros, c.w_bits, c.d_out, c.d_in, s);
-  else e = launch_repack_sp24(h->w, wts[0].w_codes, wts[0].w_zeros, c.d_out, c.d_in, s);
+  cudaError_t e = repack_backbone(h->w, c, wts[0], c.d_out, s, -1);
   for (int j = 0; j < n && e == cudaSuccess; ++j) {
     const eora_linear_weights& w = wts[j];
     const WMat av = tile_view(h->a, j * h->r_pad / 16);

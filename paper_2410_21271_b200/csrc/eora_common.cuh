@@ -46,8 +46,14 @@ namespace eora {
 //   SP24: 1152 B: values in two planes of one uint4 per lane (plane = part/2), the half (part%2) holds
 //         the 4 kept fp16 values of the part's two quads; then one word per lane in bytes [1024, 1152),
 //         byte `part` = nibble(quad0) | nibble(quad1)<<4.
+//   SQ4 : 384 B (2:4 pattern, kept values as 4-bit codes): one uint2 per lane in bytes [0, 256): word blk
+//         (= part/2) holds the 8 kept codes of parts 2*blk and 2*blk+1; kept value i (0..3: two per quad) of
+//         the part with half = part%2 sits in nibble q4_nibble(4*half + i), so that (w >> 8*half) & 0x000f000f
+//         is the pair kept by the part's first quad and the same with >> 4 more its second quad's.  Then the
+//         position word of SP24 in bytes [256, 384).  Scale entries as for the quantised formats; a group
+//         is counted along the original reduction axis.
 // ---------------------------------------------------------------------------------------------
-enum Fmt : int { FMT_NONE = 0, FMT_Q4 = 1, FMT_Q3 = 2, FMT_Q8 = 3, FMT_F16 = 4, FMT_SP24 = 5 };
+enum Fmt : int { FMT_NONE = 0, FMT_Q4 = 1, FMT_Q3 = 2, FMT_Q8 = 3, FMT_F16 = 4, FMT_SP24 = 5, FMT_SQ4 = 6 };
 
 struct WMat {
   int fmt;
@@ -65,9 +71,11 @@ struct WMat {
 constexpr int kSzEntryBytes = 48;
 
 __host__ __device__ constexpr int tile_bytes(int fmt) {
-  return fmt == FMT_Q4 ? 512 : fmt == FMT_Q3 ? 384 : fmt == FMT_Q8 ? 1024 : fmt == FMT_F16 ? 2048 : fmt == FMT_SP24 ? 1152 : 0;
+  return fmt == FMT_Q4 ? 512 : fmt == FMT_Q3 ? 384 : fmt == FMT_Q8 ? 1024 : fmt == FMT_F16 ? 2048 : fmt == FMT_SP24 ? 1152
+       : fmt == FMT_SQ4 ? 384 : 0;
 }
-__host__ __device__ constexpr bool fmt_quantised(int fmt) { return fmt == FMT_Q4 || fmt == FMT_Q3 || fmt == FMT_Q8; }
+// formats whose blobs carry scale / zero-point entries
+__host__ __device__ constexpr bool fmt_quantised(int fmt) { return fmt == FMT_Q4 || fmt == FMT_Q3 || fmt == FMT_Q8 || fmt == FMT_SQ4; }
 __host__ __device__ constexpr int blob_bytes(int fmt, int sz2) {
   return 2 * tile_bytes(fmt) + (fmt_quantised(fmt) ? (sz2 ? 2 : 1) * kSzEntryBytes : 0);
 }
@@ -122,11 +130,29 @@ __device__ inline int wmat_code(const WMat& w, int k, int n) {
   }
 }
 
+// Kept value of a 2:4 quad that element e (0..7) of a part refers to: 2*quad + {0, 1}, or -1 if the position is pruned.
+__host__ __device__ inline int sp24_kept(uint32_t meta_byte, int e) {
+  const int quad = e >> 2, pos = e & 3;
+  const uint32_t nib = (meta_byte >> (4 * quad)) & 15u;
+  if (pos == (int)(nib & 3u)) return 2 * quad;
+  if (pos == (int)(nib >> 2)) return 2 * quad + 1;
+  return -1;
+}
+
 // Dequantised element (k, n) as fp32: exactly (float)(q - z) * (float)s for the quantised formats.
 __device__ inline float wmat_elem(const WMat& w, int k, int n) {
   int tile = n >> 4, g = n & 7, half = (n >> 3) & 1;
-  if (w.fmt == FMT_Q4 || w.fmt == FMT_Q3 || w.fmt == FMT_Q8) {
-    int q = wmat_code(w, k, n);
+  if (w.fmt == FMT_Q4 || w.fmt == FMT_Q3 || w.fmt == FMT_Q8 || w.fmt == FMT_SQ4) {
+    int q;
+    if (w.fmt == FMT_SQ4) {
+      const int c = k >> 6, blk = (k >> 5) & 1, t = (k >> 3) & 3, lane = g * 4 + t, part = blk * 2 + half;
+      const uint32_t* tb = reinterpret_cast<const uint32_t*>(wmat_tile(w, tile, c));
+      const int i = sp24_kept((tb[64 + lane] >> (8 * part)) & 255u, k & 7);
+      if (i < 0) return 0.f;
+      q = (tb[lane * 2 + blk] >> (4 * q4_nibble(4 * half + i))) & 15;
+    } else {
+      q = wmat_code(w, k, n);
+    }
     const uint8_t* sz = wmat_sz(w, tile, k >> 6);
     uint32_t s2 = reinterpret_cast<const uint32_t*>(sz)[g];
     uint32_t z2 = reinterpret_cast<const uint16_t*>(sz + 32)[g];
@@ -197,6 +223,8 @@ cudaError_t launch_repack_q8(const WMat& dst, const void* codes, const void* sca
 cudaError_t launch_repack_f16(const WMat& dst, const void* src, int rows_src, int k_src, cudaStream_t st, int nt_sub = -1);
 cudaError_t launch_repack_sp24(const WMat& dst, const void* values, const void* meta, int rows_src, int k_src,
                                cudaStream_t st, int nt_sub = -1);
+cudaError_t launch_repack_sq4(const WMat& dst, const void* codes, const void* scales, const void* zeros, const void* meta,
+                              int rows_src, int k_src, cudaStream_t st, int nt_sub = -1);
 cudaError_t launch_dump(const Handle* h, int what, void* out, cudaStream_t st);
 cudaError_t launch_generic_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
 int generic_launch_count(const Handle* h);

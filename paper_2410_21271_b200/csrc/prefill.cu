@@ -97,6 +97,7 @@ template <> struct Packed<FMT_Q3> { uint2 v; uint32_t w2; };
 template <> struct Packed<FMT_Q8> { uint4 v[2]; };
 template <> struct Packed<FMT_F16> { uint4 v[4]; };
 template <> struct Packed<FMT_SP24> { uint4 v[2]; uint32_t meta; };
+template <> struct Packed<FMT_SQ4> { uint2 v; uint32_t meta; };
 
 template <int FMT>
 __device__ __forceinline__ void load_packed(Packed<FMT>& r, const uint8_t* blob, int lane) {
@@ -110,6 +111,9 @@ __device__ __forceinline__ void load_packed(Packed<FMT>& r, const uint8_t* blob,
   } else if constexpr (FMT == FMT_F16) {
 #pragma unroll
     for (int p = 0; p < 4; ++p) r.v[p] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * p) + lane);
+  } else if constexpr (FMT == FMT_SQ4) {
+    r.v = __ldg(reinterpret_cast<const uint2*>(blob) + lane);
+    r.meta = __ldg(reinterpret_cast<const uint32_t*>(blob + 256) + lane);
   } else {
     r.v[0] = __ldg(reinterpret_cast<const uint4*>(blob) + lane);
     r.v[1] = __ldg(reinterpret_cast<const uint4*>(blob + 512) + lane);
@@ -133,11 +137,22 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
   if constexpr (FMT == FMT_F16) {
 #pragma unroll
     for (int p = 0; p < 4; ++p) { out[p][0] = r.v[p].x; out[p][1] = r.v[p].y; out[p][2] = r.v[p].z; out[p][3] = r.v[p].w; }
-  } else if constexpr (FMT == FMT_SP24) {
+  } else if constexpr (FMT == FMT_SP24 || FMT == FMT_SQ4) {
+    [[maybe_unused]] ZC zc;
+    if constexpr (FMT == FMT_SQ4) make_zc<FMT>(zc, zz2);
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
-      const uint4 u = r.v[p >> 1];
-      const uint32_t v01 = (p & 1) ? u.z : u.x, v23 = (p & 1) ? u.w : u.y;   // (val0,val1) of quad 0, of quad 1
+      uint32_t v01, v23;                                                      // (val0,val1) of quad 0, of quad 1
+      if constexpr (FMT == FMT_SP24) {
+        const uint4 u = r.v[p >> 1];
+        v01 = (p & 1) ? u.z : u.x; v23 = (p & 1) ? u.w : u.y;
+      } else {                                                                // kept codes -> RN((q - z) * s)
+        const int hf = p & 1;
+        const uint32_t w = (p >> 1) ? r.v.y : r.v.x;
+        const uint32_t s2 = (hf ? (sc2 >> 16) : (sc2 & 0xffffu)) * 0x00010001u;
+        v01 = h2mul(h2sub(and_or(w >> (8 * hf), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
+        v23 = h2mul(h2sub(and_or(w >> (8 * hf + 4), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
+      }
       const uint32_t mb = (r.meta >> (8 * p)) & 255u;
 #pragma unroll
       for (int quad = 0; quad < 2; ++quad) {
@@ -220,7 +235,7 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
     return true;
   } else {
     constexpr int PF = FMT == FMT_F16 ? 2 : kPrefetch;
-    constexpr bool quant = FMT == FMT_Q4 || FMT == FMT_Q3 || FMT == FMT_Q8;
+    constexpr bool quant = fmt_quantised(FMT);
     const int rt = (n0 >> 4) + tile;                     // this warp's row tile of the matrix
     const bool active = rt < mat.nt;
     const int g = lane >> 2;
@@ -495,6 +510,7 @@ cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, con
     case FMT_Q4: return launch_bf<FMT_Q4>(bf, grid, smem, st, tx, tt, a);
     case FMT_Q3: return launch_bf<FMT_Q3>(bf, grid, smem, st, tx, tt, a);
     case FMT_SP24: return launch_bf<FMT_SP24>(bf, grid, smem, st, tx, tt, a);
+    case FMT_SQ4: return launch_bf<FMT_SQ4>(bf, grid, smem, st, tx, tt, a);
     // A as the weight of the first launch (t = X.A): no K-extension there
     case FMT_F16: return launch_p<k_prefill<FMT_F16, FMT_NONE>>(grid, smem, st, tx, tt, a);
     case FMT_Q8: return launch_p<k_prefill<FMT_Q8, FMT_NONE>>(grid, smem, st, tx, tt, a);

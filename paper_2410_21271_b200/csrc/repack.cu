@@ -141,6 +141,31 @@ __global__ void k_repack_sp24(WMat d, int nt_sub, const __half* values, const ui
   }
 }
 
+// 2:4 pattern with 4-bit kept values: `codes` is the 4-bit stream of the [k_src/2][rows_src] matrix of kept values.
+__global__ void k_repack_sq4(WMat d, int nt_sub, const uint32_t* codes, const uint32_t* meta, int rows_src, int k_src) {
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
+  for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    Pos p = pos_of(idx, d.kc);
+    uint32_t* tb = reinterpret_cast<uint32_t*>(const_cast<uint8_t*>(wmat_tile(d, p.tile, p.c)));
+    uint32_t m = 0, wd[2] = {0, 0};
+    for (int part = 0; part < 4; ++part) {
+      int n = p.tile * 16 + p.g + 8 * (part & 1);
+      int k0 = p.c * 64 + (part >> 1) * 32 + 8 * p.t;
+      int j0 = k0 >> 2;   // first of the part's two quads
+      uint32_t mb = 0x44;  // rows past the source: positions (0,1); their scale entry is zero
+      if (n < rows_src && k0 < k_src) {
+        for (int i = 0; i < 4; ++i)
+          wd[part >> 1] |= src_code(codes, 4, 2 * j0 + i, n, rows_src) << (4 * q4_nibble(4 * (part & 1) + i));
+        mb = (meta[(int64_t)n * (k_src / 32) + (j0 >> 3)] >> (4 * (j0 & 7))) & 255u;
+      }
+      m |= mb << (8 * part);
+    }
+    tb[p.lane * 2] = wd[0];
+    tb[p.lane * 2 + 1] = wd[1];
+    tb[64 + p.lane] = m;
+  }
+}
+
 // Scale entries.  scales fp16 [G][rows_src]; zeros packed stream.  One thread per (k-tile c, row tile, g);
 // the entry of k-tile c is written once per blob (by the even tile when the pair shares one entry).
 __global__ void k_repack_sz(WMat d, int nt_sub, const __half* scales, const uint32_t* zeros, int bits, int rows_src, int ldz,
@@ -235,6 +260,19 @@ cudaError_t launch_repack_sp24(const WMat& d, const void* values, const void* me
   if (nt_sub < 0) nt_sub = d.nt;
   int64_t total = (int64_t)nt_sub * d.kc * 32;
   k_repack_sp24<<<grid_for(total, 256), 256, 0, st>>>(d, nt_sub, (const __half*)values, (const uint32_t*)meta, rows_src, k_src);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_repack_sq4(const WMat& d, const void* codes, const void* scales, const void* zeros, const void* meta,
+                              int rows_src, int k_src, cudaStream_t st, int nt_sub) {
+  if (nt_sub < 0) nt_sub = d.nt;
+  int64_t total = (int64_t)nt_sub * d.kc * 32;
+  int ldz = 4 * rows_src / 32;
+  int ng_src = k_src / d.group;
+  if (ng_src < 1) ng_src = 1;
+  k_repack_sq4<<<grid_for(total, 256), 256, 0, st>>>(d, nt_sub, (const uint32_t*)codes, (const uint32_t*)meta, rows_src, k_src);
+  k_repack_sz<<<grid_for((int64_t)nt_sub * d.kc * 8, 256), 256, 0, st>>>(d, nt_sub, (const __half*)scales, (const uint32_t*)zeros, 4,
+                                                                        rows_src, ldz, ng_src);
   return cudaGetLastError();
 }
 

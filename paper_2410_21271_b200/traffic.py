@@ -10,7 +10,8 @@ def matrix_bytes(kind: str, rows: int, cols: int, *, bits: int = 4, group: int =
     """Bytes of a stored [rows (reduction)][cols] matrix.
     kind: 'f16' | 'quant' (b-bit codes + fp16 scale + b-bit zero per group and column)
           | 'q8' (uint8 codes + fp16 scale + uint8 zero per column) | 'sparse24' (fp16 values for half
-          the entries + 2 bits of position per kept value)."""
+          the entries + 2 bits of position per kept value) | 'sparse24q' (b-bit codes for half the entries
+          + 2 bits of position per kept value + fp16 scale and b-bit zero per group of `group` original rows)."""
     if kind == "f16":
         return 2 * rows * cols
     if kind == "quant":
@@ -21,6 +22,10 @@ def matrix_bytes(kind: str, rows: int, cols: int, *, bits: int = 4, group: int =
         return rows * cols + cols * 2 + cols
     if kind == "sparse24":
         return (rows // 2) * cols * 2 + (rows // 4) * cols * 4 // 8
+    if kind == "sparse24q":
+        g = min(group, rows)
+        groups = rows // g
+        return (rows // 2) * cols * bits // 8 + (rows // 4) * cols * 4 // 8 + groups * cols * 2 + groups * cols * bits // 8
     raise ValueError(kind)
 
 
@@ -39,13 +44,15 @@ def adapter_bytes(ab: str, K: int, N: int, r: int, group: int = 128) -> int:
 
 
 def backbone_bytes(w: str, K: int, N: int, group: int = 128) -> int:
-    """w: 'q4' | 'q3' | 'sp24'."""
+    """w: 'q4' | 'q3' | 'sp24' | 'sq4' (2:4 with 4-bit kept values)."""
     if w == "q4":
         return matrix_bytes("quant", K, N, bits=4, group=group)
     if w == "q3":
         return matrix_bytes("quant", K, N, bits=3, group=group)
     if w == "sp24":
         return matrix_bytes("sparse24", K, N)
+    if w == "sq4":
+        return matrix_bytes("sparse24q", K, N, bits=4, group=group)
     raise ValueError(w)
 
 

@@ -14,6 +14,8 @@ def make_case(seed, K, N, r, *, w="q4", ab="f16", group=128):
         wf = gen.make_backbone_quant(seed, K, N, 4 if w == "q4" else 3, group)
     elif w == "sp24":
         wf = gen.make_sparse24(seed, K, N)
+    elif w == "sq4":
+        wf = gen.make_sparse24_quant(seed, K, N, 4, group)
     else:
         raise ValueError(w)
     if r == 0:

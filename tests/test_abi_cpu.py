@@ -33,7 +33,12 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_struct_layout_matches_header():
     assert ctypes.sizeof(eora.eora_linear_config) == 12 * 4
-    assert ctypes.sizeof(eora.eora_linear_weights) == 9 * ctypes.sizeof(ctypes.c_void_p)
+    assert ctypes.sizeof(eora.eora_linear_weights) == 10 * ctypes.sizeof(ctypes.c_void_p)
+    # field order as declared in the header
+    hdr = open(os.path.join(os.path.dirname(__file__), "..", "include", "eora_linear.h")).read()
+    body = hdr[hdr.index("typedef struct {", hdr.index("} eora_linear_config;")):hdr.index("} eora_linear_weights;")]
+    names = re.findall(r"const void\* (\w+);", body)
+    assert names == [f[0] for f in eora.eora_linear_weights._fields_]
 
 
 def test_status_strings(lib):
@@ -77,6 +82,14 @@ def test_create_rejects_bad_arguments_without_a_device(lib):
     w.a = w.b = 4096
     w.w_codes = 4100
     assert eora.eora_linear_create_status(good_cfg(), w) == eora.EORA_ERR_MISALIGNED
+    # 2:4 + 4-bit backbone: 4 bits only, a group like the quantised backbone, and the position words
+    w.w_codes = 4096
+    sq = dict(w_format=eora.EORA_W_SPARSE24_Q4)
+    assert eora.eora_linear_create_status(good_cfg(w_bits=3, **sq), w) == eora.EORA_ERR_UNSUPPORTED
+    assert eora.eora_linear_create_status(good_cfg(w_group=96, **sq), w) == eora.EORA_ERR_BAD_SHAPE
+    assert eora.eora_linear_create_status(good_cfg(**sq), w) == eora.EORA_ERR_NULL_ARG  # w_meta missing
+    w.w_meta = 4104
+    assert eora.eora_linear_create_status(good_cfg(**sq), w) == eora.EORA_ERR_MISALIGNED
 
 
 def test_calls_on_null_handle(lib):

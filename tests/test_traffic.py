@@ -29,5 +29,7 @@ def test_forward_bytes_hand_arithmetic():
     assert traffic.forward_bytes("q4", "f16", 4096, 4096, 128, 1) == 8388608 + 327680 + 2097152 + 16384
     assert traffic.forward_bytes("q3", "f16", 4096, 4096, 0, 1) == 6291456 + 32 * 4096 * 2 + 32 * 4096 * 3 // 8 + 16384
     assert traffic.backbone_bytes("sp24", 4096, 4096) == 4096 * 2048 * 2 + 4096 * 1024 // 2
+    # 2:4 + 4-bit: half a byte per kept value, half a byte of positions per quad, scale + zero per group of 128 k
+    assert traffic.backbone_bytes("sq4", 4096, 4096) == 4096 * 2048 // 2 + 4096 * 1024 // 2 + 32 * 4096 * 2 + 32 * 4096 // 2
     assert traffic.matrix_bytes("q8", 4096, 128) == 4096 * 128 + 3 * 128
     assert traffic.forward_flops(4096, 4096, 128, 2048) == 2 * 2048 * (4096 * 4096 + 128 * 8192)
