@@ -134,7 +134,7 @@ int eora_linear_forward(eora_linear_t h, const void* x, int32_t m, void* y, void
  * (Section 3), and several of them read the same activations: q/k/v of an attention block, gate/up
  * of an MLP.  eora_linear_create_fused builds ONE handle for n_layers (2..4) such layers, given as
  * arrays of configs and weights; they must agree in everything but d_out (same d_in, rank, formats,
- * groups, dtypes, max_m <= 64, policy AUTO, quantised backbone).  eora_linear_forward_fused computes
+ * groups, dtypes, max_m <= 64, policy AUTO; any backbone format).  eora_linear_forward_fused computes
  *     ys[i][M][d_out_i] = X . deq(Wq_i) + (X . A_i) . B_i      for every layer i
  * with ONE kernel launch per eight tokens: X is read once, and the launch latency is paid once.
  * ys: host array of n_layers device pointers (16-byte aligned, caller-owned).  The handle serves

@@ -173,7 +173,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     d_out_total += ci.d_out;
   }
   const bool fused = n > 1;
-  if (fused && (c.w_format != EORA_W_QUANT || c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO)) return EORA_ERR_UNSUPPORTED;
+  if (fused && (c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO)) return EORA_ERR_UNSUPPORTED;
   c.d_out = d_out_total;
 
   eora_linear* obj = new (std::nothrow) eora_linear();

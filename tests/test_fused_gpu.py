@@ -30,6 +30,8 @@ CASES = [
     ("q4", "q8", 384, [64, 64, 32, 96], 40, 5, "bf16"),
     ("q3", "f16", 1024, [224, 96], 0, 2, "f16"),
     ("q3", "f16", 640, [160, 352], 256, 19, "f16"),          # three passes of eight tokens
+    ("sp24", "f16", 512, [96, 64], 64, 2, "f16"),            # 2:4 backbones
+    ("sq4", "q4", 512, [64, 160, 32], 128, 9, "f16"),        # 2:4 with 4-bit kept values
 ]
 
 

@@ -38,6 +38,7 @@ CASES = [
     ("q3", "q8", 384, 96, 40, 2, [1, -1, 0], "bf16"),
     ("q4", "q3", 640, 96, 64, 3, list(range(-1, 3)) * 5, "f16"),          # 20 tokens: three passes
     ("sp24", "f16", 512, 96, 64, 2, [1, 0, 0], "f16"),
+    ("sq4", "f16", 512, 96, 64, 3, [2, -1, 0, 1, 1], "f16"),
     ("q4", "f16", 256, 64, 64, 1, [0, -1], "f16"),                         # a single adapter that can be off
     ("q3", "f16", 4096, 1024, 128, 8, [7], "f16"),                         # k-shaped layer, full size
 ]
