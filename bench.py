@@ -278,7 +278,7 @@ def time_prefill(device: str, steps: int = 10, warmup: int = 3):
 # capture summarised in profiles/k_decode_llama3-8b-w3g128-r128-M1.md (traffic grows with the number of
 # blocks in proportion; fusing layers changes the number of launches, not the bytes).  Set to None when the
 # kernel's memory behaviour changes until the capture is redone.
-DRAM_BYTES_PER_BLOCK = 108.54e6
+DRAM_BYTES_PER_BLOCK = 108.52e6
 
 
 def cpu_oracle_sample(blocks_sample: int = 1):
