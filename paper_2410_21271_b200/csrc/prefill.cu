@@ -62,9 +62,6 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, in
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(smem_u32(dst)), "l"(tm), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
 __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
@@ -99,26 +96,41 @@ template <> struct Packed<FMT_F16> { uint4 v[4]; };
 template <> struct Packed<FMT_SP24> { uint4 v[2]; uint32_t meta; };
 template <> struct Packed<FMT_SQ4> { uint2 v; uint32_t meta; };
 
+// Lanes with an odd row index g store the two 32-element halves of their rows in the opposite order
+// (see dequant_store), so they take them in the opposite order too: where a half is a separate piece of
+// the tile the swap is done here, by address (sw = 1 for such lanes); otherwise swap_halves does it on
+// the loaded words, at the time they are used.
 template <int FMT>
-__device__ __forceinline__ void load_packed(Packed<FMT>& r, const uint8_t* blob, int lane) {
+__device__ __forceinline__ void load_packed(Packed<FMT>& r, const uint8_t* blob, int lane, int sw) {
   if constexpr (FMT == FMT_Q4) r.v = __ldg(reinterpret_cast<const uint4*>(blob) + lane);
   else if constexpr (FMT == FMT_Q3) {
     r.v = __ldg(reinterpret_cast<const uint2*>(blob) + lane);
     r.w2 = __ldg(reinterpret_cast<const uint32_t*>(blob + 256) + lane);
   } else if constexpr (FMT == FMT_Q8) {
-    r.v[0] = __ldg(reinterpret_cast<const uint4*>(blob) + lane);
-    r.v[1] = __ldg(reinterpret_cast<const uint4*>(blob + 512) + lane);
+    r.v[0] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * sw) + lane);
+    r.v[1] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * (sw ^ 1)) + lane);
   } else if constexpr (FMT == FMT_F16) {
 #pragma unroll
-    for (int p = 0; p < 4; ++p) r.v[p] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * p) + lane);
+    for (int p = 0; p < 4; ++p) r.v[p] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * (p ^ (2 * sw))) + lane);
   } else if constexpr (FMT == FMT_SQ4) {
     r.v = __ldg(reinterpret_cast<const uint2*>(blob) + lane);
     r.meta = __ldg(reinterpret_cast<const uint32_t*>(blob + 256) + lane);
   } else {
-    r.v[0] = __ldg(reinterpret_cast<const uint4*>(blob) + lane);
-    r.v[1] = __ldg(reinterpret_cast<const uint4*>(blob + 512) + lane);
+    r.v[0] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * sw) + lane);
+    r.v[1] = __ldg(reinterpret_cast<const uint4*>(blob + 512 * (sw ^ 1)) + lane);
     r.meta = __ldg(reinterpret_cast<const uint32_t*>(blob + 1024) + lane);
   }
+}
+__device__ __forceinline__ void cswap(uint32_t& a, uint32_t& b, bool sw) {
+  const uint32_t x = sw ? b : a, y = sw ? a : b;
+  a = x; b = y;
+}
+// The value-level part of the swap (formats whose halves share a load; the position bytes of the 2:4 formats).
+template <int FMT>
+__device__ __forceinline__ void swap_halves(Packed<FMT>& r, bool sw) {
+  if constexpr (FMT == FMT_Q4) { cswap(r.v.x, r.v.z, sw); cswap(r.v.y, r.v.w, sw); }
+  else if constexpr (FMT == FMT_SQ4) { cswap(r.v.x, r.v.y, sw); r.meta = __funnelshift_l(r.meta, r.meta, sw ? 16 : 0); }
+  else if constexpr (FMT == FMT_SP24) r.meta = __funnelshift_l(r.meta, r.meta, sw ? 16 : 0);
 }
 
 __device__ __forceinline__ uint32_t h2mul(uint32_t a, uint32_t b) {
@@ -127,19 +139,50 @@ __device__ __forceinline__ uint32_t h2mul(uint32_t a, uint32_t b) {
   return d;
 }
 
-// Dequantise one 16 x 64 tile to fp16 RN((q - z) * s) and store this lane's four 16-byte chunks
-// (8 consecutive reduction elements of one row each) into the swizzled B operand.
-// btile: start of the stage's B operand; row0: first row of the tile inside the operand.
-template <int FMT>
-__device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2, uint32_t zz2, uint8_t* btile, int row0, int lane) {
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// Byte offsets, inside one stage of the weight ring, of the four 16-byte chunks (8 consecutive reduction
+// elements of one row each) that a lane stores per tile.  Store k holds row g + 8 * (k & 1) and the half
+// (k >> 1) ^ (g & 1) of the 64 reduction elements: in step k lanes with even g write one half and lanes
+// with odd g the other, so that the 8 lanes of a quarter warp (two rows) hit 8 different 16-byte columns
+// of the 128-byte swizzle.
+__device__ __forceinline__ void store_offsets(uint32_t (&off)[4], int tile, int lane) {
   const int g = lane >> 2, t = lane & 3;
-  uint32_t out[4][4];     // [part][pair]
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int row = tile * 16 + g + 8 * (k & 1);
+    const int chunk = (((k >> 1) ^ (g & 1)) << 2) + t;          // 16-byte chunk index along K inside the 128-byte row
+    off[k] = (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
+  }
+}
+
+// Per-tile constants (1024 + z), -(64 + z) as fp16x2 for the two rows of a lane, one byte permute each.
+template <int FMT>
+__device__ __forceinline__ void make_zc_p(ZC& zc, uint32_t zz) {
+  zc.c[0][0] = prmt(zz, 0x64646464u, 0x4040u);
+  zc.c[1][0] = prmt(zz, 0x64646464u, 0x4141u);
+  if constexpr (FMT == FMT_Q4) {
+    const uint32_t z4 = zz << 4;                                  // bytes: z_a << 4, z_b << 4 (zero-points < 16)
+    zc.c[0][1] = prmt(z4, 0xD4D4D4D4u, 0x4040u);
+    zc.c[1][1] = prmt(z4, 0xD4D4D4D4u, 0x4141u);
+  }
+}
+
+// Dequantise one 16 x 64 tile to fp16 RN((q - z) * s) and store this lane's four chunks into the swizzled
+// operand of the stage at shared address `stage`.  The lane's words arrive with their halves in storage
+// order; `odd` (= g & 1) says that this lane stores them in the opposite order (store_offsets).
+template <int FMT>
+__device__ __forceinline__ void dequant_store(Packed<FMT> r, uint32_t sc2, uint32_t zz2, uint32_t stage, const uint32_t (&off)[4], bool odd) {
+  swap_halves<FMT>(r, odd);
+  uint32_t out[4][4];     // [part][pair]; part = 2 * (half as stored by this lane) + (row g or g + 8)
   if constexpr (FMT == FMT_F16) {
 #pragma unroll
     for (int p = 0; p < 4; ++p) { out[p][0] = r.v[p].x; out[p][1] = r.v[p].y; out[p][2] = r.v[p].z; out[p][3] = r.v[p].w; }
   } else if constexpr (FMT == FMT_SP24 || FMT == FMT_SQ4) {
     [[maybe_unused]] ZC zc;
-    if constexpr (FMT == FMT_SQ4) make_zc<FMT>(zc, zz2);
+    if constexpr (FMT == FMT_SQ4) make_zc_p<FMT>(zc, zz2);
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
       uint32_t v01, v23;                                                      // (val0,val1) of quad 0, of quad 1
@@ -149,7 +192,7 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
       } else {                                                                // kept codes -> RN((q - z) * s)
         const int hf = p & 1;
         const uint32_t w = (p >> 1) ? r.v.y : r.v.x;
-        const uint32_t s2 = (hf ? (sc2 >> 16) : (sc2 & 0xffffu)) * 0x00010001u;
+        const uint32_t s2 = prmt(sc2, 0u, hf ? 0x3232u : 0x1010u);
         v01 = h2mul(h2sub(and_or(w >> (8 * hf), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
         v23 = h2mul(h2sub(and_or(w >> (8 * hf + 4), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
       }
@@ -168,7 +211,7 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
     }
   } else {
     ZC zc;
-    make_zc<FMT>(zc, zz2);
+    make_zc_p<FMT>(zc, zz2);
     uint32_t a[4][4];
     if constexpr (FMT == FMT_Q4) {
       const uint32_t w[4] = {r.v.x, r.v.y, r.v.z, r.v.w};
@@ -184,6 +227,8 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
     } else if constexpr (FMT == FMT_Q3) {
       uint32_t q[4][2];
       q3_quads(r.v.x, r.v.y, r.w2, q);
+#pragma unroll
+      for (int j = 0; j < 2; ++j) { cswap(q[0][j], q[2][j], odd); cswap(q[1][j], q[3][j], odd); }
 #pragma unroll
       for (int part = 0; part < 4; ++part) {
         const int hf = part & 1;
@@ -202,32 +247,31 @@ __device__ __forceinline__ void dequant_store(const Packed<FMT>& r, uint32_t sc2
         a[part][3] = h2sub(and_or(w1 >> 8, 0x00ff00ffu, kMagic), zc.c[hf][0]);
       }
     }
-    const uint32_t s_a = (sc2 & 0xffffu) * 0x00010001u, s_b = (sc2 >> 16) * 0x00010001u;
+    const uint32_t s_a = prmt(sc2, 0u, 0x1010u), s_b = prmt(sc2, 0u, 0x3232u);
 #pragma unroll
     for (int part = 0; part < 4; ++part)
 #pragma unroll
       for (int j = 0; j < 4; ++j) out[part][j] = h2mul(a[part][j], (part & 1) ? s_b : s_a);
   }
-  // Store order: in step k lanes with even g write their blk = k/2 part and lanes with odd g the other
-  // one, so that the 8 lanes of a quarter warp (two rows) hit 8 different 16-byte columns of the swizzle.
-  const int odd = g & 1;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    const int hf = k & 1, blk_even = k >> 1;
-    const int blk = blk_even ^ odd;
-    const int pe = blk_even * 2 + hf, po = (blk_even ^ 1) * 2 + hf;
-    const uint4 v = odd ? make_uint4(out[po][0], out[po][1], out[po][2], out[po][3])
-                        : make_uint4(out[pe][0], out[pe][1], out[pe][2], out[pe][3]);
-    const int row = row0 + g + 8 * hf;
-    const int chunk = blk * 4 + t;                              // 16-byte chunk index along K inside the 128-byte row
-    uint8_t* dst = btile + row * 128 + ((chunk ^ (row & 7)) << 4);
-    *reinterpret_cast<uint4*>(dst) = v;
+    const int part = (k >> 1) * 2 + (k & 1);
+    st_shared_v4(stage + off[k], out[part][0], out[part][1], out[part][2], out[part][3]);
   }
+}
+
+__device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar_addr, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar_addr), "r"(parity) : "memory");
+  return ok != 0;
 }
 
 // One part (W or the K-extension B) of a dequant warp's work.  The warp owns row tile `tile` (0..15) of
 // the CTA's 256 weight rows; k-blocks [kb_lo, kb_hi) of `mat` land in pipeline iterations it0, it0 + 1, ...
-// Packed weights, scales and zero-points are loaded PF k-blocks ahead.
+// Packed weights, scales and zero-points are loaded PF k-blocks ahead.  The loop is what bounds the
+// kernel (four of these warps share a scheduler), so everything that does not change per k-block is
+// computed once: the store offsets, the ring position as a running (slot, wrap) pair, shared addresses.
 template <int FMT>
 __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo, int kb_hi, int it0, int tile, int lane,
                                              uint8_t* smem, const PrefillArgs& p, uint64_t* full_w, uint64_t* empty_w) {
@@ -236,47 +280,55 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
   } else {
     constexpr int PF = FMT == FMT_F16 ? 2 : kPrefetch;
     constexpr bool quant = fmt_quantised(FMT);
+    constexpr int tb = tile_bytes(FMT);
     const int rt = (n0 >> 4) + tile;                     // this warp's row tile of the matrix
     const bool active = rt < mat.nt;
     const int g = lane >> 2;
-    const int tb = tile_bytes(FMT);
-    const int gt = mat.group / 64;
+    const int odd = g & 1;
+    uint32_t off[4];
+    store_offsets(off, tile, lane);
+    const uint8_t* base = mat.q + (int64_t)rt * mat.blob;                 // this row tile's blob of pair 0
+    const int64_t pair_stride = (int64_t)mat.nt * mat.blob;
+    const int sz_step = mat.sz2 ? kSzEntryBytes : 0;
+    const uint32_t ring = smem_u32(smem + p.w_off), full0 = smem_u32(full_w), empty0 = smem_u32(empty_w);
     Packed<FMT> pk[PF];
     uint32_t scq[PF], zzq[PF];
     auto issue = [&](int kb, int slot) {
       if (!active || kb >= kb_hi) return;
-      const uint8_t* blob = mat.q + ((int64_t)(kb >> 1) * mat.nt + rt) * mat.blob;
-      load_packed<FMT>(pk[slot], blob + (kb & 1) * tb, lane);
+      const uint8_t* blob = base + (kb >> 1) * pair_stride;
+      load_packed<FMT>(pk[slot], blob + (kb & 1) * tb, lane, odd);
       if constexpr (quant) {
-        const uint8_t* sz = blob + 2 * tb + (mat.sz2 ? (kb & 1) * kSzEntryBytes : 0);
+        const uint8_t* sz = blob + 2 * tb + (kb & 1) * sz_step;
         scq[slot] = __ldg(reinterpret_cast<const uint32_t*>(sz) + g);
         zzq[slot] = __ldg(reinterpret_cast<const uint16_t*>(sz + 32) + g);
       }
     };
 #pragma unroll
     for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(kb_lo + j, j); }
+    int s = it0 % p.sw, wrap = it0 / p.sw, it = it0;     // ring slot of iteration `it`, and how often it has been used before
     for (int kbb = kb_lo; kbb < kb_hi; kbb += PF) {
 #pragma unroll
       for (int j = 0; j < PF; ++j) {
         const int kb = kbb + j;
         if (kb < kb_hi) {
-          const int it = it0 + (kb - kb_lo), s = it % p.sw;
-          if (it >= p.sw && !mbar_wait_warp(empty_w + s, ((it / p.sw) - 1) & 1, p.dev_status, lane)) return false;
-          uint8_t* wt = smem + p.w_off + (size_t)s * (2 * BN_W * 128);
+          if (wrap > 0 && !mbar_try_wait_a(empty0 + 8 * s, (wrap - 1) & 1) &&
+              !mbar_wait_warp(empty_w + s, (wrap - 1) & 1, p.dev_status, lane)) return false;
+          const uint32_t stage = ring + (uint32_t)s * (2 * BN_W * 128);
           if (active) {
-            dequant_store<FMT>(pk[j], scq[j], zzq[j], wt, tile * 16, lane);
+            dequant_store<FMT>(pk[j], scq[j], zzq[j], stage, off, odd != 0);
           } else {                                        // rows past the matrix: keep the operand finite
-            const int gg = lane >> 2, tt = lane & 3;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const int row = tile * 16 + gg + 8 * (k & 1), chunk = (k >> 1) * 4 + tt;
-              *reinterpret_cast<uint4*>(wt + row * 128 + ((chunk ^ (row & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-            }
+            for (int k = 0; k < 4; ++k) st_shared_v4(stage + off[k], 0u, 0u, 0u, 0u);
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy stores -> visible to the MMA
           __syncwarp();
-          if (lane == 0) { mbar_arrive(full_w + s); if (tile == 0) PTRACE(it, 1); }
+          if (lane == 0) {
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full0 + 8 * s) : "memory");
+            if (tile == 0) PTRACE(it, 1);
+          }
           issue(kb + PF, j);
+          ++it;
+          if (++s == p.sw) { s = 0; ++wrap; }
         }
       }
     }
@@ -323,14 +375,15 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (token tiles)
     if (lane == 0) {
+      int s = 0, wrap = 0;                          // ring slot of iteration `it`, and how often it has been used before
       for (int it = 0; it < nkb; ++it) {
-        const int s = it % p.sx;
-        if (it >= p.sx && !mbar_wait(empty_x + s, ((it / p.sx) - 1) & 1, p.dev_status)) break;
+        if (wrap > 0 && !mbar_wait(empty_x + s, (wrap - 1) & 1, p.dev_status)) break;
         PTRACE(it, 0);
         mbar_expect_tx(full_x + s, xbytes);
         uint8_t* xt = smem + (size_t)s * xbytes;
         if (it < nkw) tma_load_2d(xt, &tm_x, (kw_lo + it) * BK, m0, full_x + s);
         else tma_load_2d(xt, &tm_t, (it - nkw) * BK, m0, full_x + s);
+        if (++s == p.sx) { s = 0; ++wrap; }
       }
     }
   } else if (warp == 1) {
@@ -339,12 +392,13 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       // instruction descriptor: fp32 accumulate, fp16 x fp16, both operands K-major, M = 128 weight rows, N = bt tokens
       const uint32_t idesc = (1u << 4) | ((uint32_t)(p.bt >> 3) << 17) | ((uint32_t)(BN_W >> 4) << 24);
       bool ok = true;
+      int sx = 0, sw = 0;                           // ring slots of iteration `it` and their phases
+      uint32_t px = 0, pw = 0;
       for (int it = 0; it < nkb && ok; ++it) {
-        const int sx = it % p.sx, sw = it % p.sw;
-        ok = mbar_wait(full_x + sx, (it / p.sx) & 1, p.dev_status);
+        ok = mbar_wait(full_x + sx, px, p.dev_status);
         if (!ok) break;
         PTRACE(it, 2);
-        ok = mbar_wait(full_w + sw, (it / p.sw) & 1, p.dev_status);
+        ok = mbar_wait(full_w + sw, pw, p.dev_status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint64_t bdesc = make_desc(smem + (size_t)sx * xbytes);
@@ -357,6 +411,8 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
         umma_commit(empty_x + sx);                  // both arrive when these MMAs have finished reading their operands
         umma_commit(empty_w + sw);
         PTRACE(it, 3);
+        if (++sx == p.sx) { sx = 0; px ^= 1u; }
+        if (++sw == p.sw) { sw = 0; pw ^= 1u; }
       }
       umma_commit(&acc_full);                       // arrives when every MMA above has completed
     }
