@@ -207,9 +207,11 @@ int eora_linear_last_device_status(eora_linear_t h);
  * records four %globaltimer values (nanoseconds) per warp, at uint64 index
  * 4 * (4 * cta + warp) + k:  k = 0 kernel entry, 1 dependency wait over, 2 first share of the
  * backbone done, 3 all work of the warp done; the buffer must hold 16 * grid values.  A prefill
- * forward records, for CTA (0, 0) only, four clock64 values per 64-element k-block
- * (producer / dequantisation / MMA issue / MMA complete) at index 4 * k_block + k; the buffer
- * must hold 4 * (d_in + rank + 128) / 64 values.  Tracing costs time; leave it off in production.
+ * forward records, for CTA (0, 0) only, four clock64 values per 64-element k-block (token tile
+ * requested / first weight tile dequantised / token tile seen by the MMA warp / MMAs issued) at
+ * index 4 * k_block + k, k_block < nkb = d_in / 64 + (rank padded to 128) / 64, and one more row at
+ * k_block = nkb: kernel entry / set-up done / accumulators complete / epilogue done; the buffer
+ * must hold 4 * ((d_in + rank) / 64 + 4) values.  Tracing costs time; leave it off in production.
  */
 int eora_linear_decode_grid(eora_linear_t h, int32_t m);
 int eora_linear_set_trace(eora_linear_t h, void* trace_buf);

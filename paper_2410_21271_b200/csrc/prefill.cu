@@ -48,7 +48,8 @@ struct PrefillArgs {
   int split_k;       // gridDim.z: each z handles a slice of the k-blocks and adds into a fp32 `out` (out_dtype 3)
   int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
   int* dev_status;
-  long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (dequant start, W ready, X ready, MMA issued)
+  long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (token copy requested, W ready, X ready, MMA issued),
+                     // then one more row: kernel entry, set-up done, accumulators complete, epilogue done
 };
 
 #define PTRACE(it, slot) do { if (p.trace && blockIdx.x == 0 && blockIdx.y == 0) p.trace[(it) * 4 + (slot)] = clock64(); } while (0)
@@ -356,6 +357,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   const uint32_t xbytes = (uint32_t)p.bt * 128;
 
   if (threadIdx.x == 0) {
+    PTRACE(nkb, 0);
     fail_s = 0;
     for (int i = 0; i < p.sx; ++i) { mbar_init(full_x + i, 1); mbar_init(empty_x + i, 1); }
     for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8 * nh); mbar_init(empty_w + i, 1); }
@@ -371,6 +373,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_d = tmem_base_s;
+  if (threadIdx.x == 0) PTRACE(nkb, 1);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (token tiles)
@@ -424,23 +427,30 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       ok = dequant_part<WF>(p.w, n0, kw_lo, kw_hi, 0, dw, lane, smem, p, full_w, empty_w);
       if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, 0, p.nkb_b, nkw, dw, lane, smem, p, full_w, empty_w);
     }
-    if (dw < 4) {
-      // Epilogue (4 warps).  Warp dw owns accumulator rows (= weight rows n) 32*dw .. 32*dw+31 of each half,
-      // its TMEM lanes; columns are tokens.
+    {
+      // Epilogue: all sixteen warps, as four groups of four.  A warp can read the quarter of the TMEM lanes
+      // that its index selects (warp % 4 == dw % 4), i.e. accumulator rows (= weight rows n) 32 * (dw % 4) ...
+      // of each half; columns are tokens.  The chunks of 32 tokens are dealt to the groups round-robin.
       if (ok) ok = mbar_wait_warp(&acc_full, 0, p.dev_status, lane);
-      // the four epilogue warps meet at barriers below: they must all take the same way
+      // the warps meet at barriers below: they must all take the same way
       if (!ok) *reinterpret_cast<volatile int*>(&fail_s) = 1;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 512;" ::: "memory");
       ok = *reinterpret_cast<volatile int*>(&fail_s) == 0;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int nl = dw * 32 + lane;                     // local weight row inside the half
+      if (dw == 0 && lane == 0) PTRACE(nkb, 2);
+      const int grp = dw >> 2, lq = dw & 3;
+      const int nl = lq * 32 + lane;                     // local weight row inside the half = thread index inside the group
+      const int nchunk = (p.bt + 31) >> 5;
+      const uint32_t lane_base = tmem_d + ((uint32_t)(lq * 32) << 16);
       if (p.out_dtype == 3) {
         // split-K partial: add fp32 into out[token][n]; lanes hold consecutive n, so each red is a 128-byte row piece
         for (int hh = 0; hh < nh && ok; ++hh) {
           const int col = n0 + hh * BN_W + nl;
-          for (int c0 = 0; c0 < p.bt; c0 += 32) {
+          for (int cc = 0; cc < nchunk; ++cc) {
+            if (((hh * nchunk + cc) & 3) != grp) continue;
+            const int c0 = cc * 32;
             uint32_t v[32];
-            tmem_ld32(tmem_d + hh * 256 + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
+            tmem_ld32(lane_base + hh * 256 + (uint32_t)c0, v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             if (col < p.n_valid) {
 #pragma unroll
@@ -452,15 +462,22 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
           }
         }
       } else {
-        // Chunks of 32 tokens go through shared memory as [token][128 n] so that the global stores are 16-byte
-        // pieces of rows of Y.  The token ring is free by now (every MMA has completed).
+        // A chunk goes through shared memory as [32 tokens][128 n] so that the global stores are 16-byte
+        // pieces of rows of Y.  The rings are free by now (every MMA has completed).  Each group has two
+        // buffers and alternates: a buffer is rewritten two chunks later, after a barrier that every thread of
+        // the group passes only when it has read the buffer out, so one barrier per chunk is enough.
         const int esz = p.out_dtype == EORA_Y_F32 ? 4 : 2;
-        uint8_t* tbuf = smem;                            // 32 tokens x 128 n x esz bytes (<= 16 KB)
-        const int et = threadIdx.x - 128;                // 0..127 among the epilogue threads
+        const int row_sh = esz == 4 ? 5 : 4;             // log2 of the 16-byte pieces per token row (128 n)
+        uint8_t* gbuf = smem + grp * 32768;              // 2 x (32 tokens x 128 n x esz bytes <= 16 KB)
+        int flip = 0;
         for (int hh = 0; hh < nh && ok; ++hh) {
-          for (int c0 = 0; c0 < p.bt; c0 += 32) {
+          for (int cc = 0; cc < nchunk; ++cc) {
+            if (((hh * nchunk + cc) & 3) != grp) continue;
+            const int c0 = cc * 32;
+            uint8_t* tbuf = gbuf + flip * 16384;
+            flip ^= 1;
             uint32_t v[32];
-            tmem_ld32(tmem_d + hh * 256 + ((uint32_t)(dw * 32) << 16) + (uint32_t)c0, v);
+            tmem_ld32(lane_base + hh * 256 + (uint32_t)c0, v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -469,20 +486,20 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
               else if (p.out_dtype == EORA_Y_F16) reinterpret_cast<__half*>(tbuf)[j * BN_W + nl] = __float2half_rn(f);
               else reinterpret_cast<__nv_bfloat16*>(tbuf)[j * BN_W + nl] = __float2bfloat16_rn(f);
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            const int per_row = BN_W * esz / 16;         // 16 or 32 pieces per token row
-            for (int i = et; i < 32 * per_row; i += 128) {
-              const int tok = i / per_row, piece = i - tok * per_row;
+            asm volatile("bar.sync %0, 128;" ::"r"(2 + grp) : "memory");
+            const int pieces = 32 << row_sh;
+            for (int i = nl; i < pieces; i += 128) {
+              const int tok = i >> row_sh, piece = i & ((1 << row_sh) - 1);
               const int row = m0 + c0 + tok, col = n0 + hh * BN_W + piece * (16 / esz);
               if (row < p.m && col < p.n_valid) {
                 const uint4 val = *reinterpret_cast<const uint4*>(tbuf + (size_t)tok * BN_W * esz + piece * 16);
                 *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + ((int64_t)row * p.ld_out + col) * esz) = val;
               }
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
           }
         }
       }
+      if (dw == 0 && lane == 0) PTRACE(nkb, 3);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
