@@ -227,7 +227,6 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   const int64_t rp = h->t_cols;
   for (int pass = 0; pass < 2; ++pass) {
     Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
-    h->t_ws = sc.take<float>((int64_t)c.max_m * rp * 4);
     h->t_gen = sc.take<float>((int64_t)c.max_m * rp * 4);
     h->t16 = sc.take<__half>((int64_t)c.max_m * rp * 2);
     h->d_t = sc.take<float>(8 * rp * 4);
@@ -330,8 +329,7 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
   const int64_t rp = h->t_cols;
   for (int pass = 0; pass < 2; ++pass) {
     Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
-    h->t_ws = sc.take<float>(256);            // prefill scratch is not used by this kind of handle
-    h->t_gen = sc.take<float>(256);
+    h->t_gen = sc.take<float>(256);            // prefill scratch is not used by this kind of handle
     h->t16 = sc.take<__half>(256);
     h->d_t = sc.take<float>(8 * rp * 4);
     h->y_ws = sc.take<float>((int64_t)8 * h->w.n_rows * 4);

@@ -188,9 +188,8 @@ struct Handle {
   WMat w, a, b;          // a: rows = rank (padded to 16); b: rows = d_out, reduction = r_pad
   void* weight_mem;      // one allocation holding all re-tiled payloads
   int64_t weight_bytes;
-  void* scratch_mem;     // one allocation: t, split-K sums, counters, staging
+  void* scratch_mem;     // one allocation: t, partial sums, counters, staging
   int64_t scratch_bytes;
-  float* t_ws;           // [max_m][r_pad] fp32 split-K sums of t (prefill); zero between calls
   float* t_gen;          // [max_m][r_pad] fp32, simple kernels only
   __half* t16;           // [max_m][r_pad] fp16 (prefill)
   float* d_t;            // [8][t_cols] fp32 sums of t (decode); zero between calls

@@ -14,9 +14,10 @@
 //     memory; tcgen05.commit releases the ring slots when the MMAs have drained;
 //   * the low-rank term is a K-extension: after the d_in/64 backbone k-blocks come r/64 k-blocks whose
 //     token operand is t = X.A (fp16, from a first launch of the same kernel with A as the weight) and
-//     whose weight operand is B, so (X.A).B lands in the same accumulator;
-//   * epilogue: tcgen05.ld -> fp16/bf16/fp32 -> transpose through shared memory -> 16-byte row stores,
-//     so Y is written once.
+//     whose weight operand is B, so (X.A).B lands in the same accumulator.  The two launches overlap:
+//     the main one is a programmatic dependent launch that waits for t only in front of the K-extension;
+//   * epilogue (all sixteen dequant warps): tcgen05.ld -> fp16/bf16/fp32 -> transpose through shared
+//     memory -> 16-byte row stores, so Y is written once.
 // Launches per forward: 1 (rank 0) or 2 (t = X.A, then the main product), plus a conversion launch
 // when X is bf16 (the f16 MMA kind needs both operands in fp16; weights are kept fp16 because
 // bf16 weights alone cost 1.7e-3 of the 2e-3 error budget).
@@ -45,7 +46,6 @@ struct PrefillArgs {
   int bt;            // token tile (the MMA N): multiple of 16, at most 256
   int nkb_w, nkb_b;  // k-blocks of each part
   int sx, sw;        // stages of the token ring / of the weight ring
-  int split_k;       // gridDim.z: each z handles a slice of the k-blocks and adds into a fp32 `out` (out_dtype 3)
   int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
   int* dev_status;
   long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (token copy requested, W ready, X ready, MMA issued),
@@ -347,12 +347,14 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   // 1024-byte alignment of the operand tiles (the swizzle pattern is anchored at 1 KB)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
+  // Programmatic dependent launch: a kernel launched behind this one with the serialisation attribute may
+  // start at once (the main product behind the launch that computes t; see launch_prefill_forward).
+  asm volatile("griddepcontrol.launch_dependents;");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * (2 * BN_W), m0 = blockIdx.y * p.bt;
   const int nh = (p.n_valid - n0 > BN_W) ? 2 : 1;          // 128-row halves of this CTA that hold real rows
-  // this CTA's slice of the k-blocks (split-K over gridDim.z; the K-extension only exists without split)
-  const int kw_lo = (int)((int64_t)p.nkb_w * blockIdx.z / p.split_k), kw_hi = (int)((int64_t)p.nkb_w * (blockIdx.z + 1) / p.split_k);
-  const int nkw = kw_hi - kw_lo;
+  const int kw_lo = 0, kw_hi = p.nkb_w;
+  const int nkw = p.nkb_w;
   const int nkb = nkw + p.nkb_b;
   const uint32_t xbytes = (uint32_t)p.bt * 128;
 
@@ -384,8 +386,13 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
         PTRACE(it, 0);
         mbar_expect_tx(full_x + s, xbytes);
         uint8_t* xt = smem + (size_t)s * xbytes;
-        if (it < nkw) tma_load_2d(xt, &tm_x, (kw_lo + it) * BK, m0, full_x + s);
-        else tma_load_2d(xt, &tm_t, (it - nkw) * BK, m0, full_x + s);
+        if (it < nkw) {
+          tma_load_2d(xt, &tm_x, (kw_lo + it) * BK, m0, full_x + s);
+        } else {
+          // t comes from the previous launch, which may still be running: everything up to here overlapped with it
+          if (it == nkw) asm volatile("griddepcontrol.wait;" ::: "memory");
+          tma_load_2d(xt, &tm_t, (it - nkw) * BK, m0, full_x + s);
+        }
         if (++s == p.sx) { s = 0; ++wrap; }
       }
     }
@@ -442,26 +449,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       const int nl = lq * 32 + lane;                     // local weight row inside the half = thread index inside the group
       const int nchunk = (p.bt + 31) >> 5;
       const uint32_t lane_base = tmem_d + ((uint32_t)(lq * 32) << 16);
-      if (p.out_dtype == 3) {
-        // split-K partial: add fp32 into out[token][n]; lanes hold consecutive n, so each red is a 128-byte row piece
-        for (int hh = 0; hh < nh && ok; ++hh) {
-          const int col = n0 + hh * BN_W + nl;
-          for (int cc = 0; cc < nchunk; ++cc) {
-            if (((hh * nchunk + cc) & 3) != grp) continue;
-            const int c0 = cc * 32;
-            uint32_t v[32];
-            tmem_ld32(lane_base + hh * 256 + (uint32_t)c0, v);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (col < p.n_valid) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const int row = m0 + c0 + j;
-                if (row < p.m) red_add(reinterpret_cast<float*>(p.out) + (int64_t)row * p.ld_out + col, __uint_as_float(v[j]));
-              }
-            }
-          }
-        }
-      } else {
+      {
         // A chunk goes through shared memory as [32 tokens][128 n] so that the global stores are 16-byte
         // pieces of rows of Y.  The rings are free by now (every MMA has completed).  Each group has two
         // buffers and alternates: a buffer is rewritten two chunks later, after a barrier that every thread of
@@ -507,14 +495,6 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(512u) : "memory");
 }
 
-// t (fp32 split-K sums) -> fp16 operand of the K-extension; the sums are returned to zero for the next call
-__global__ void k_t32_to_f16(float* t32, __half* t16, int64_t n) {
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-    t16[i] = __float2half_rn(t32[i]);
-    t32[i] = 0.f;
-  }
-}
-
 __global__ void k_bf16_to_f16(const __nv_bfloat16* in, __half* out, int64_t n) {
   for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 2; i < n; i += (int64_t)gridDim.x * blockDim.x * 2) {
     float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(in + i));
@@ -553,40 +533,52 @@ bool make_map(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int
 
 constexpr int kSmemP = 225 * 1024;
 
+// pdl: the launch may begin while the previous kernel of the stream is still running (it waits, on the
+// device, before it touches what that kernel writes).
 template <auto KERNEL>
-cudaError_t launch_p(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt, const PrefillArgs& a) {
+cudaError_t launch_p(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt, const PrefillArgs& a,
+                     bool pdl) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  KERNEL<<<grid, kThreadsP, smem, st>>>(tx, tt, a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreadsP);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, KERNEL, tx, tt, a);
 }
 
 template <int WF>
 cudaError_t launch_bf(int bf, dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt,
-                      const PrefillArgs& a) {
+                      const PrefillArgs& a, bool pdl) {
   switch (bf) {
-    case FMT_F16: return launch_p<k_prefill<WF, FMT_F16>>(grid, smem, st, tx, tt, a);
-    case FMT_Q4: return launch_p<k_prefill<WF, FMT_Q4>>(grid, smem, st, tx, tt, a);
-    case FMT_Q8: return launch_p<k_prefill<WF, FMT_Q8>>(grid, smem, st, tx, tt, a);
-    case FMT_Q3: return launch_p<k_prefill<WF, FMT_Q3>>(grid, smem, st, tx, tt, a);
-    default: return launch_p<k_prefill<WF, FMT_NONE>>(grid, smem, st, tx, tt, a);
+    case FMT_F16: return launch_p<k_prefill<WF, FMT_F16>>(grid, smem, st, tx, tt, a, pdl);
+    case FMT_Q4: return launch_p<k_prefill<WF, FMT_Q4>>(grid, smem, st, tx, tt, a, pdl);
+    case FMT_Q8: return launch_p<k_prefill<WF, FMT_Q8>>(grid, smem, st, tx, tt, a, pdl);
+    case FMT_Q3: return launch_p<k_prefill<WF, FMT_Q3>>(grid, smem, st, tx, tt, a, pdl);
+    default: return launch_p<k_prefill<WF, FMT_NONE>>(grid, smem, st, tx, tt, a, pdl);
   }
 }
 
 cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt,
-                       const PrefillArgs& a) {
+                       const PrefillArgs& a, bool pdl) {
   switch (wf) {
-    case FMT_Q4: return launch_bf<FMT_Q4>(bf, grid, smem, st, tx, tt, a);
-    case FMT_Q3: return launch_bf<FMT_Q3>(bf, grid, smem, st, tx, tt, a);
-    case FMT_SP24: return launch_bf<FMT_SP24>(bf, grid, smem, st, tx, tt, a);
-    case FMT_SQ4: return launch_bf<FMT_SQ4>(bf, grid, smem, st, tx, tt, a);
+    case FMT_Q4: return launch_bf<FMT_Q4>(bf, grid, smem, st, tx, tt, a, pdl);
+    case FMT_Q3: return launch_bf<FMT_Q3>(bf, grid, smem, st, tx, tt, a, pdl);
+    case FMT_SP24: return launch_bf<FMT_SP24>(bf, grid, smem, st, tx, tt, a, pdl);
+    case FMT_SQ4: return launch_bf<FMT_SQ4>(bf, grid, smem, st, tx, tt, a, pdl);
     // A as the weight of the first launch (t = X.A): no K-extension there
-    case FMT_F16: return launch_p<k_prefill<FMT_F16, FMT_NONE>>(grid, smem, st, tx, tt, a);
-    case FMT_Q8: return launch_p<k_prefill<FMT_Q8, FMT_NONE>>(grid, smem, st, tx, tt, a);
+    case FMT_F16: return launch_p<k_prefill<FMT_F16, FMT_NONE>>(grid, smem, st, tx, tt, a, pdl);
+    case FMT_Q8: return launch_p<k_prefill<FMT_Q8, FMT_NONE>>(grid, smem, st, tx, tt, a, pdl);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -614,7 +606,7 @@ bool prefill_supported(const Handle* h, int m) {
 }
 
 int prefill_launch_count(const Handle* h, int) {
-  return (h->cfg.rank > 0 ? 3 : 1) + (h->cfg.x_dtype == EORA_X_BF16 ? 1 : 0);
+  return (h->cfg.rank > 0 ? 2 : 1) + (h->cfg.x_dtype == EORA_X_BF16 ? 1 : 0);
 }
 
 cudaError_t prefill_init(Handle* h) {
@@ -653,23 +645,21 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   const bool ab = c.rank > 0;
   if (ab) {
     if (!make_map(&tm_t, h->t16, m, h->r_pad, h->r_pad, bt)) return cudaErrorInvalidValue;
-    // launch 1: t = X.A with A as the weight (rows = r_pad), split over K so that the small product fills the
-    // GPU; partial sums are added into the fp32 buffer t_ws (zero between calls); launch 2 rounds them to fp16.
+    // launch 1: t = X.A with A as the weight (rows = r_pad), written as fp16.  It is a small product (a few
+    // CTAs with token tiles of 128), and the main launch behind it starts at once (programmatic dependent
+    // launch) on the other SMs: the main product needs t only for its last k-blocks and waits for this
+    // launch there, so the two overlap.
+    const int bt_t = m >= 128 ? 128 : bt;
+    CUtensorMap tm_xt;
+    if (!make_map(&tm_xt, x16, m, c.d_in, c.d_in, bt_t)) return cudaErrorInvalidValue;
     PrefillArgs a = {};
     a.w = h->a; a.b = WMat(); a.b.fmt = FMT_NONE;
-    a.out = h->t_ws; a.out_dtype = 3; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt;
+    a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt_t;
     a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status; a.trace = nullptr;
     const int smem_t = fill_stages(a);
-    const int tiles = ((h->r_pad + 2 * BN_W - 1) / (2 * BN_W)) * ((m + bt - 1) / bt);
-    int split = h->sm_count / tiles;
-    if (split > a.nkb_w / 2) split = a.nkb_w / 2;
-    if (split < 1) split = 1;
-    a.split_k = split;
-    dim3 grid((h->r_pad + 2 * BN_W - 1) / (2 * BN_W), (m + bt - 1) / bt, split);
-    cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_x, tm_x, a);
+    dim3 grid((h->r_pad + 2 * BN_W - 1) / (2 * BN_W), (m + bt_t - 1) / bt_t, 1);
+    cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_xt, tm_xt, a, false);
     if (e != cudaSuccess) return e;
-    const int64_t nt = (int64_t)m * h->r_pad;
-    k_t32_to_f16<<<(int)((nt + 255) / 256 > 1184 ? 1184 : (nt + 255) / 256), 256, 0, st>>>(h->t_ws, h->t16, nt);
   } else {
     tm_t = tm_x;
   }
@@ -679,10 +669,9 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m; a.bt = bt;
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
   a.trace = reinterpret_cast<long long*>(h->trace);
-  a.split_k = 1;
   const int smem_y = fill_stages(a);
   dim3 grid((c.d_out + 2 * BN_W - 1) / (2 * BN_W), (m + bt - 1) / bt, 1);
-  return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, a);
+  return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, a, ab);
 }
 
 }  // namespace eora
