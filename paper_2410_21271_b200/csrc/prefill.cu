@@ -44,6 +44,7 @@ struct PrefillArgs {
   int n_valid;       // columns of out to write
   int m;
   int bt;            // token tile (the MMA N): multiple of 16, at most 256
+  int rows;          // weight rows per CTA: 256 (two MMA halves) or 128 (small matrices: more CTAs, half the dequant work each)
   int nkb_w, nkb_b;  // k-blocks of each part
   int sx, sw;        // stages of the token ring / of the weight ring
   int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
@@ -269,13 +270,16 @@ __device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar_addr, uint32_t pari
 }
 
 // One part (W or the K-extension B) of a dequant warp's work.  The warp owns row tile `tile` (0..15) of
-// the CTA's 256 weight rows; k-blocks [kb_lo, kb_hi) of `mat` land in pipeline iterations it0, it0 + 1, ...
-// Packed weights, scales and zero-points are loaded PF k-blocks ahead.  The loop is what bounds the
+// the CTA's 256 weight rows; k-blocks [kb_lo, kb_hi) of `mat` land in pipeline iterations it0, it0 + 1, ...,
+// and the warp takes those with index kb_lo + kphase + i * kstep (kstep = 2 when two warps share a row
+// tile, which is how a CTA with 128 rows keeps all sixteen warps and twice the loads in flight).
+// Packed weights, scales and zero-points are loaded PF of the warp's k-blocks ahead.  The loop is what bounds the
 // kernel (four of these warps share a scheduler), so everything that does not change per k-block is
 // computed once: the store offsets, the ring position as a running (slot, wrap) pair, shared addresses.
 template <int FMT>
-__device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo, int kb_hi, int it0, int tile, int lane,
-                                             uint8_t* smem, const PrefillArgs& p, uint64_t* full_w, uint64_t* empty_w) {
+__device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo, int kb_hi, int it0, int tile, int kphase,
+                                             int kstep, int lane, uint8_t* smem, const PrefillArgs& p, uint64_t* full_w,
+                                             uint64_t* empty_w) {
   if constexpr (FMT == FMT_NONE) {
     return true;
   } else {
@@ -305,12 +309,13 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
       }
     };
 #pragma unroll
-    for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(kb_lo + j, j); }
-    int s = it0 % p.sw, wrap = it0 / p.sw, it = it0;     // ring slot of iteration `it`, and how often it has been used before
-    for (int kbb = kb_lo; kbb < kb_hi; kbb += PF) {
+    for (int j = 0; j < PF; ++j) { scq[j] = 0; zzq[j] = 0; issue(kb_lo + kphase + j * kstep, j); }
+    int it = it0 + kphase;
+    int s = it % p.sw, wrap = it / p.sw;                 // ring slot of iteration `it`, and how often it has been used before
+    for (int kbb = kb_lo + kphase; kbb < kb_hi; kbb += PF * kstep) {
 #pragma unroll
       for (int j = 0; j < PF; ++j) {
-        const int kb = kbb + j;
+        const int kb = kbb + j * kstep;
         if (kb < kb_hi) {
           if (wrap > 0 && !mbar_try_wait_a(empty0 + 8 * s, (wrap - 1) & 1) &&
               !mbar_wait_warp(empty_w + s, (wrap - 1) & 1, p.dev_status, lane)) return false;
@@ -327,9 +332,10 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full0 + 8 * s) : "memory");
             if (tile == 0) PTRACE(it, 1);
           }
-          issue(kb + PF, j);
-          ++it;
-          if (++s == p.sw) { s = 0; ++wrap; }
+          issue(kb + PF * kstep, j);
+          it += kstep;
+          s += kstep;
+          if (s >= p.sw) { s -= p.sw; ++wrap; }             // kstep <= 2 <= stages
         }
       }
     }
@@ -351,8 +357,8 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   // start at once (the main product behind the launch that computes t; see launch_prefill_forward).
   asm volatile("griddepcontrol.launch_dependents;");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * (2 * BN_W), m0 = blockIdx.y * p.bt;
-  const int nh = (p.n_valid - n0 > BN_W) ? 2 : 1;          // 128-row halves of this CTA that hold real rows
+  const int n0 = blockIdx.x * p.rows, m0 = blockIdx.y * p.bt;
+  const int nh = (p.rows > BN_W && p.n_valid - n0 > BN_W) ? 2 : 1;   // 128-row halves of this CTA that hold real rows
   const int kw_lo = 0, kw_hi = p.nkb_w;
   const int nkw = p.nkb_w;
   const int nkb = nkw + p.nkb_b;
@@ -430,9 +436,11 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
     // ------------------------------------------------------------------ dequant warps, then epilogue
     const int dw = warp - 4;
     bool ok = true;
-    if (dw < 8 * nh) {
-      ok = dequant_part<WF>(p.w, n0, kw_lo, kw_hi, 0, dw, lane, smem, p, full_w, empty_w);
-      if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, 0, p.nkb_b, nkw, dw, lane, smem, p, full_w, empty_w);
+    {
+      // two halves: one row tile per warp; one half: two warps per row tile, alternating k-blocks
+      const int kstep = 3 - nh, tile = nh == 2 ? dw : (dw & 7), kphase = nh == 2 ? 0 : (dw >> 3);
+      ok = dequant_part<WF>(p.w, n0, kw_lo, kw_hi, 0, tile, kphase, kstep, lane, smem, p, full_w, empty_w);
+      if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, 0, p.nkb_b, nkw, tile, kphase, kstep, lane, smem, p, full_w, empty_w);
     }
     {
       // Epilogue: all sixteen warps, as four groups of four.  A warp can read the quarter of the TMEM lanes
@@ -592,6 +600,13 @@ int fill_stages(PrefillArgs& a) {      // returns the dynamic shared memory to r
   return a.w_off + w_bytes + 1024;
 }
 
+// Weight rows per CTA: 256, or 128 when 256-row tiles would leave more than half of the SMs without a CTA
+// (the dequantisation of a CTA's rows is what bounds its k-block period, so halving the rows halves its time).
+int cta_rows(int n_rows, int m, int bt, int sm_count) {
+  const int tiles = ((n_rows + 2 * BN_W - 1) / (2 * BN_W)) * ((m + bt - 1) / bt);
+  return (n_rows > BN_W && 2 * tiles <= sm_count) ? BN_W : 2 * BN_W;
+}
+
 int token_tile(int m) {                // the MMA N: a multiple of 16 up to 256
   if (m >= 256) return 256;
   return (m + 15) / 16 * 16;
@@ -656,8 +671,9 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     a.w = h->a; a.b = WMat(); a.b.fmt = FMT_NONE;
     a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt_t;
     a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status; a.trace = nullptr;
+    a.rows = cta_rows(h->r_pad, m, bt_t, h->sm_count);
     const int smem_t = fill_stages(a);
-    dim3 grid((h->r_pad + 2 * BN_W - 1) / (2 * BN_W), (m + bt_t - 1) / bt_t, 1);
+    dim3 grid((h->r_pad + a.rows - 1) / a.rows, (m + bt_t - 1) / bt_t, 1);
     cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_xt, tm_xt, a, false);
     if (e != cudaSuccess) return e;
   } else {
@@ -669,8 +685,9 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m; a.bt = bt;
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
   a.trace = reinterpret_cast<long long*>(h->trace);
+  a.rows = cta_rows(c.d_out, m, bt, h->sm_count);
   const int smem_y = fill_stages(a);
-  dim3 grid((c.d_out + 2 * BN_W - 1) / (2 * BN_W), (m + bt - 1) / bt, 1);
+  dim3 grid((c.d_out + a.rows - 1) / a.rows, (m + bt - 1) / bt, 1);
   return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, a, ab);
 }
 
