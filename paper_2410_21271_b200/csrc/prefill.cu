@@ -176,39 +176,40 @@ __device__ __forceinline__ void make_zc_p(ZC& zc, uint32_t zz) {
 // operand of the stage at shared address `stage`.  The lane's words arrive with their halves in storage
 // order; `odd` (= g & 1) says that this lane stores them in the opposite order (store_offsets).
 template <int FMT>
-__device__ __forceinline__ void dequant_store(Packed<FMT> r, uint32_t sc2, uint32_t zz2, uint32_t stage, const uint32_t (&off)[4], bool odd) {
+__device__ __forceinline__ void dequant_store(Packed<FMT> r, uint32_t sc2, uint32_t zz2, uint32_t stage, const uint32_t (&off)[4], bool odd,
+                                              uint32_t lut) {
   swap_halves<FMT>(r, odd);
   uint32_t out[4][4];     // [part][pair]; part = 2 * (half as stored by this lane) + (row g or g + 8)
   if constexpr (FMT == FMT_F16) {
 #pragma unroll
     for (int p = 0; p < 4; ++p) { out[p][0] = r.v[p].x; out[p][1] = r.v[p].y; out[p][2] = r.v[p].z; out[p][3] = r.v[p].w; }
   } else if constexpr (FMT == FMT_SP24 || FMT == FMT_SQ4) {
+    // A quad's two kept values (one register) are spread over its four positions (two registers) with two
+    // byte permutes whose selectors come from a 16-entry table in shared memory indexed by the quad's
+    // position nibble (sp24_selectors).
     [[maybe_unused]] ZC zc;
     if constexpr (FMT == FMT_SQ4) make_zc_p<FMT>(zc, zz2);
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
-      uint32_t v01, v23;                                                      // (val0,val1) of quad 0, of quad 1
+      uint32_t vq[2];                                                         // (val0,val1) of quad 0, of quad 1
       if constexpr (FMT == FMT_SP24) {
         const uint4 u = r.v[p >> 1];
-        v01 = (p & 1) ? u.z : u.x; v23 = (p & 1) ? u.w : u.y;
+        vq[0] = (p & 1) ? u.z : u.x; vq[1] = (p & 1) ? u.w : u.y;
       } else {                                                                // kept codes -> RN((q - z) * s)
         const int hf = p & 1;
         const uint32_t w = (p >> 1) ? r.v.y : r.v.x;
         const uint32_t s2 = prmt(sc2, 0u, hf ? 0x3232u : 0x1010u);
-        v01 = h2mul(h2sub(and_or(w >> (8 * hf), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
-        v23 = h2mul(h2sub(and_or(w >> (8 * hf + 4), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
+        vq[0] = h2mul(h2sub(and_or(w >> (8 * hf), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
+        vq[1] = h2mul(h2sub(and_or(w >> (8 * hf + 4), 0x000f000fu, kMagic), zc.c[hf][0]), s2);
       }
-      const uint32_t mb = (r.meta >> (8 * p)) & 255u;
 #pragma unroll
       for (int quad = 0; quad < 2; ++quad) {
-        const uint32_t vv = quad ? v23 : v01;
-        const uint32_t nib = (mb >> (4 * quad)) & 15u, p0 = nib & 3u, p1 = nib >> 2;
-        const uint32_t v0 = vv & 0xffffu, v1 = vv >> 16;
-        uint32_t e[4];
-#pragma unroll
-        for (uint32_t pos = 0; pos < 4; ++pos) e[pos] = (pos == p0) ? v0 : (pos == p1) ? v1 : 0u;
-        out[p][2 * quad] = e[0] | (e[1] << 16);
-        out[p][2 * quad + 1] = e[2] | (e[3] << 16);
+        const int sh = 8 * p + 4 * quad - 2;                                  // nibble * 4 = byte offset into the table
+        const uint32_t offb = (sh < 0 ? (r.meta << 2) : (r.meta >> (sh < 0 ? 0 : sh))) & 0x3Cu;
+        uint32_t sel;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(sel) : "r"(lut + offb));
+        out[p][2 * quad] = prmt(vq[quad], 0u, sel);
+        out[p][2 * quad + 1] = prmt(vq[quad], 0u, sel >> 16);
       }
     }
   } else {
@@ -279,7 +280,7 @@ __device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar_addr, uint32_t pari
 template <int FMT>
 __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo, int kb_hi, int it0, int tile, int kphase,
                                              int kstep, int lane, uint8_t* smem, const PrefillArgs& p, uint64_t* full_w,
-                                             uint64_t* empty_w) {
+                                             uint64_t* empty_w, uint32_t lut) {
   if constexpr (FMT == FMT_NONE) {
     return true;
   } else {
@@ -321,7 +322,7 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
               !mbar_wait_warp(empty_w + s, (wrap - 1) & 1, p.dev_status, lane)) return false;
           const uint32_t stage = ring + (uint32_t)s * (2 * BN_W * 128);
           if (active) {
-            dequant_store<FMT>(pk[j], scq[j], zzq[j], stage, off, odd != 0);
+            dequant_store<FMT>(pk[j], scq[j], zzq[j], stage, off, odd != 0, lut);
           } else {                                        // rows past the matrix: keep the operand finite
 #pragma unroll
             for (int k = 0; k < 4; ++k) st_shared_v4(stage + off[k], 0u, 0u, 0u, 0u);
@@ -349,6 +350,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_x[kMaxXStages], empty_x[kMaxXStages], full_w[kMaxWStages], empty_w[kMaxWStages], acc_full;
   __shared__ uint32_t tmem_base_s;
+  __shared__ uint32_t sp_lut[16];        // 2:4 expansion selectors (2:4 backbones only)
   __shared__ int fail_s;                 // set by an epilogue warp whose bounded wait ran out
   // 1024-byte alignment of the operand tiles (the swizzle pattern is anchored at 1 KB)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -364,6 +366,10 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   const int nkb = nkw + p.nkb_b;
   const uint32_t xbytes = (uint32_t)p.bt * 128;
 
+  if constexpr (WF == FMT_SP24 || WF == FMT_SQ4) {
+    if (threadIdx.x >= 32 && threadIdx.x < 48) sp_lut[threadIdx.x - 32] = sp24_selectors(threadIdx.x - 32);
+  }
+  const uint32_t lut = smem_u32(sp_lut);
   if (threadIdx.x == 0) {
     PTRACE(nkb, 0);
     fail_s = 0;
@@ -439,8 +445,8 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
     {
       // two halves: one row tile per warp; one half: two warps per row tile, alternating k-blocks
       const int kstep = 3 - nh, tile = nh == 2 ? dw : (dw & 7), kphase = nh == 2 ? 0 : (dw >> 3);
-      ok = dequant_part<WF>(p.w, n0, kw_lo, kw_hi, 0, tile, kphase, kstep, lane, smem, p, full_w, empty_w);
-      if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, 0, p.nkb_b, nkw, tile, kphase, kstep, lane, smem, p, full_w, empty_w);
+      ok = dequant_part<WF>(p.w, n0, kw_lo, kw_hi, 0, tile, kphase, kstep, lane, smem, p, full_w, empty_w, lut);
+      if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, 0, p.nkb_b, nkw, tile, kphase, kstep, lane, smem, p, full_w, empty_w, lut);
     }
     {
       // Epilogue: all sixteen warps, as four groups of four.  A warp can read the quarter of the TMEM lanes
@@ -503,10 +509,18 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(512u) : "memory");
 }
 
+// n is a multiple of 8 (d_in is a multiple of 128): 16 bytes in, 16 bytes out per step
 __global__ void k_bf16_to_f16(const __nv_bfloat16* in, __half* out, int64_t n) {
-  for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 2; i < n; i += (int64_t)gridDim.x * blockDim.x * 2) {
-    float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(in + i));
-    *reinterpret_cast<__half2*>(out + i) = __floats2half2_rn(f.x, f.y);
+  for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 8; i < n; i += (int64_t)gridDim.x * blockDim.x * 8) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(in + i));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const __half2 h = __floats2half2_rn(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xffff0000u));
+      o[j] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(out + i) = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
 
@@ -649,8 +663,8 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     PrefillState* ps = reinterpret_cast<PrefillState*>(h->prefill_state);
     if (!ps) return cudaErrorInvalidValue;
     int64_t n = (int64_t)m * c.d_in;
-    int64_t blocks = (n / 2 + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    int64_t blocks = (n / 8 + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
     k_bf16_to_f16<<<(int)blocks, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), ps->x16, n);
     x16 = ps->x16;
   }
@@ -664,7 +678,14 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     // CTAs with token tiles of 128), and the main launch behind it starts at once (programmatic dependent
     // launch) on the other SMs: the main product needs t only for its last k-blocks and waits for this
     // launch there, so the two overlap.
-    const int bt_t = m >= 128 ? 128 : bt;
+    // Token tiles of 128 give it more CTAs and a shorter chain, unless those CTAs would push CTAs of a main
+    // launch that fits into one wave off the SMs (a CTA of either launch needs an SM of its own).
+    int bt_t = m >= 128 ? 128 : bt;
+    {
+      const int t_rows = (h->r_pad + 2 * BN_W - 1) / (2 * BN_W);
+      const int main_tiles = ((c.d_out + 2 * BN_W - 1) / (2 * BN_W)) * ((m + bt - 1) / bt);
+      if (main_tiles <= h->sm_count && main_tiles + t_rows * ((m + bt_t - 1) / bt_t) > h->sm_count) bt_t = bt;
+    }
     CUtensorMap tm_xt;
     if (!make_map(&tm_xt, x16, m, c.d_in, c.d_in, bt_t)) return cudaErrorInvalidValue;
     PrefillArgs a = {};
