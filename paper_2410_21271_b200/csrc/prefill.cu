@@ -284,7 +284,7 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
   if constexpr (FMT == FMT_NONE) {
     return true;
   } else {
-    constexpr int PF = FMT == FMT_F16 ? 2 : kPrefetch;
+    constexpr int PF = FMT == FMT_F16 ? 3 : kPrefetch;
     constexpr bool quant = fmt_quantised(FMT);
     constexpr int tb = tile_bytes(FMT);
     const int rt = (n0 >> 4) + tile;                     // this warp's row tile of the matrix
@@ -678,13 +678,21 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     // CTAs with token tiles of 128), and the main launch behind it starts at once (programmatic dependent
     // launch) on the other SMs: the main product needs t only for its last k-blocks and waits for this
     // launch there, so the two overlap.
-    // Token tiles of 128 give it more CTAs and a shorter chain, unless those CTAs would push CTAs of a main
-    // launch that fits into one wave off the SMs (a CTA of either launch needs an SM of its own).
-    int bt_t = m >= 128 ? 128 : bt;
+    // Its tile: 128 rows and 128 tokens per CTA give the shortest chain of k-blocks, but a CTA of either
+    // launch needs an SM of its own, so when the main launch fits into one wave the first shape whose CTAs
+    // fit beside it is taken (more rows, then more tokens per CTA: fewer CTAs, longer chain).
+    const int rows_m = cta_rows(c.d_out, m, bt, h->sm_count);
+    const int main_tiles = ((c.d_out + rows_m - 1) / rows_m) * ((m + bt - 1) / bt);
+    const int room = main_tiles <= h->sm_count ? h->sm_count - main_tiles : h->sm_count;
+    int rows_t = 2 * BN_W, bt_t = bt;
     {
-      const int t_rows = (h->r_pad + 2 * BN_W - 1) / (2 * BN_W);
-      const int main_tiles = ((c.d_out + 2 * BN_W - 1) / (2 * BN_W)) * ((m + bt - 1) / bt);
-      if (main_tiles <= h->sm_count && main_tiles + t_rows * ((m + bt_t - 1) / bt_t) > h->sm_count) bt_t = bt;
+      const int cand[4][2] = {{BN_W, 128}, {2 * BN_W, 128}, {BN_W, 256}, {2 * BN_W, 256}};
+      for (int i = 0; i < 4; ++i) {
+        const int rr = h->r_pad > BN_W ? cand[i][0] : 2 * BN_W;     // one half of rows at most: the tile height does not matter
+        const int tt = cand[i][1] < bt ? cand[i][1] : bt;
+        rows_t = rr; bt_t = tt;
+        if (((h->r_pad + rr - 1) / rr) * ((m + tt - 1) / tt) <= room) break;
+      }
     }
     CUtensorMap tm_xt;
     if (!make_map(&tm_xt, x16, m, c.d_in, c.d_in, bt_t)) return cudaErrorInvalidValue;
@@ -692,7 +700,7 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     a.w = h->a; a.b = WMat(); a.b.fmt = FMT_NONE;
     a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt_t;
     a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status; a.trace = nullptr;
-    a.rows = cta_rows(h->r_pad, m, bt_t, h->sm_count);
+    a.rows = rows_t;
     const int smem_t = fill_stages(a);
     dim3 grid((h->r_pad + a.rows - 1) / a.rows, (m + bt_t - 1) / bt_t, 1);
     cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_xt, tm_xt, a, false);
