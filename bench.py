@@ -243,19 +243,15 @@ def time_e2e(layers, steps: int, warmup: int):
     return sec, h2d, d2h
 
 
-def time_prefill(device: str, steps: int = 10, warmup: int = 3):
-    """Extra: tensor-core prefill, q-shaped layer, 4-bit g128, fp16 r=128, M=2048."""
+def _time_prefill_layer(device: str, K: int, N: int, r: int, M: int, steps: int, warmup: int, flush):
     import torch
     import paper_2410_21271_b200 as eora
-    K = N = 4096
-    M, r = 2048, 128
     wf = gen.make_backbone_quant(5, K, N, 4, 128)
     af, bf = gen.make_ab_f16(5, K, N, r)
     L = eora.Layer(wf, af, bf, max_m=M, device=device)
     path = L.path(M)
     x = torch.from_numpy(gen.make_x(6, M, K)).to(device)
     y = torch.empty((M, N), dtype=torch.float16, device=device)
-    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device)
     if path == eora.EORA_PATH_GENERIC:
         steps, warmup = 2, 1
     for _ in range(warmup):
@@ -267,11 +263,33 @@ def time_prefill(device: str, steps: int = 10, warmup: int = 3):
         e0.record(); L.forward(x, y); e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
-    ms = float(np.median(times))
-    fl = traffic.forward_flops(K, N, r, M)
     L.close()
-    return {"workload": "q 4096x4096/w4-g128/eora-fp16-r128/M2048", "ms": ms, "tflops": fl / ms / 1e9,
-            "path": {0: "generic", 1: "decode", 2: "prefill"}[path], "l2": "flushed between iterations"}
+    return float(np.median(times)), path
+
+
+def time_prefill(device: str, steps: int = 10, warmup: int = 3, layer_set: bool = False):
+    """Extra: tensor-core prefill, 4-bit g128, fp16 r=128, M=2048: the q-shaped layer (the workload of the
+    committed profile) and, with layer_set, every distinct shape of the LLaMA3-8B block."""
+    import torch
+    K = N = 4096
+    M, r = 2048, 128
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device)
+    ms, path = _time_prefill_layer(device, K, N, r, M, steps, warmup, flush)
+    fl = traffic.forward_flops(K, N, r, M)
+    out = {"workload": "q 4096x4096/w4-g128/eora-fp16-r128/M2048", "ms": ms, "tflops": fl / ms / 1e9,
+           "path": {0: "generic", 1: "decode", 2: "prefill"}[path], "l2": "flushed between iterations"}
+    if layer_set:
+        shapes = {"q,o": (4096, 4096, 2), "k,v": (4096, 1024, 2), "gate,up": (4096, 14336, 2), "down": (14336, 4096, 1)}
+        per, tot_ms, tot_fl = {}, 0.0, 0.0
+        for name, (k, n, count) in shapes.items():
+            ms_s = ms if (k, n) == (K, N) else _time_prefill_layer(device, k, n, r, M, 6, warmup, flush)[0]
+            fl_s = traffic.forward_flops(k, n, r, M)
+            per[name] = {"ms": ms_s, "tflops": fl_s / ms_s / 1e9}
+            tot_ms += count * ms_s
+            tot_fl += count * fl_s
+        out["layer_set"] = {"per_shape": per, "ms_block": tot_ms, "tflops": tot_fl / tot_ms / 1e9,
+                            "note": "seven layers of a block, one launch unit per layer, times summed"}
+    return out
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of k_decode over the seven layers of one block, from the ncu
@@ -421,8 +439,9 @@ def main():
         if world == 1:
             line["cpu_baseline"] = cpu_oracle_sample(8)[0]
         try:
-            line["prefill"] = time_prefill(device)
+            line["prefill"] = time_prefill(device, layer_set=True)
             line["prefill"]["frac_of_measured_bf16_burst"] = line["prefill"]["tflops"] / peaks["bf16_tflops"]
+            line["prefill"]["layer_set"]["frac_of_measured_bf16_burst"] = line["prefill"]["layer_set"]["tflops"] / peaks["bf16_tflops"]
         except Exception as e:  # the decode line must still be printed
             line["prefill"] = {"error": repr(e)}
     if rank == 0:
