@@ -122,8 +122,10 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
 /*
  * Y[M][d_out] = X[M][d_in] . deq(Wq) + (X . A) . B   (Eq. 4), enqueued on `stream`.
  * x, y: device pointers, row-major, 16-byte aligned, caller-owned; 1 <= m <= max_m; m == 0 is a
- * no-op returning EORA_OK.  Never synchronises and never allocates.  M <= 64 runs the decode
- * kernel family, larger M the tensor-core (tcgen05) prefill family.  Asynchronous device-side
+ * no-op returning EORA_OK.  Never synchronises and never allocates.  M <= 16 runs the decode
+ * kernel family (one streaming pass over the weights per eight tokens), M > 64 the tensor-core
+ * (tcgen05) prefill family, and in between whichever is cheaper for the layer: the prefill family
+ * once ceil(M / 8) * 30 exceeds d_in / 64 (eora_linear_path reports the choice).  Asynchronous device-side
  * problems (a bounded wait that ran out) are latched in a status word readable with
  * eora_linear_last_device_status after the caller has synchronised.
  */

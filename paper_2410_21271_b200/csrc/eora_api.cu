@@ -73,8 +73,13 @@ int y_elem_bytes(int y_dtype) { return y_dtype == EORA_Y_F32 ? 4 : 2; }
 
 int pick_path(const Handle* h, int m) {
   if (h->cfg.kernel_policy == EORA_POLICY_GENERIC) return EORA_PATH_GENERIC;
-  if (m <= 64 && decode_supported(h, m)) return EORA_PATH_DECODE;
-  if (m > 64 && prefill_supported(h, m)) return EORA_PATH_PREFILL;
+  // The decode family streams the weights once per eight tokens, the tensor-core family walks the d_in / 64
+  // k-blocks of the layer once whatever m is: measured, a decode pass costs about as much as 30 k-blocks, so
+  // from three passes on (m > 16 with d_in = 4096, m > 56 with d_in = 14336) the tensor-core family is faster.
+  const bool dec = m <= 64 && decode_supported(h, m), pre = prefill_supported(h, m);
+  if (dec && pre) return ((m + 7) / 8) * 30 > h->cfg.d_in / 64 ? EORA_PATH_PREFILL : EORA_PATH_DECODE;
+  if (dec) return EORA_PATH_DECODE;
+  if (pre) return EORA_PATH_PREFILL;
   return EORA_PATH_GENERIC;
 }
 

@@ -1,4 +1,5 @@
-// Prefill kernel family (M > 64): Y = X.deq(Wq) + (X.A).B  (paper Eq. 4) as a tcgen05 GEMM.
+// Prefill kernel family (M > 64, and 16 < M <= 64 where it beats the decode passes): Y = X.deq(Wq) + (X.A).B
+// (paper Eq. 4) as a tcgen05 GEMM.
 //
 // The paper measures only batch-1 decoding (Section 4.5); for many tokens the layer is a dense
 // contraction, so it runs on the 5th-generation tensor cores.  The product is computed transposed,
@@ -629,7 +630,8 @@ int token_tile(int m) {                // the MMA N: a multiple of 16 up to 256
 }  // namespace
 
 bool prefill_supported(const Handle* h, int m) {
-  if (m <= 64) return false;
+  if (m <= 16) return false;             // up to two decode passes are always cheaper
+  if (h->n_sub > 1 || h->multi) return false;   // fused layers and per-token adapters: decode family only
   if (h->w.group % 64) return false;
   return encode_fn() != nullptr;
 }
@@ -640,7 +642,7 @@ int prefill_launch_count(const Handle* h, int) {
 
 cudaError_t prefill_init(Handle* h) {
   h->prefill_state = nullptr;
-  if (h->cfg.max_m <= 64 || h->cfg.x_dtype != EORA_X_BF16) return cudaSuccess;
+  if (h->cfg.max_m <= 16 || h->cfg.x_dtype != EORA_X_BF16) return cudaSuccess;
   PrefillState* ps = new PrefillState();
   cudaError_t e = cudaMalloc(&ps->x16, (size_t)h->cfg.max_m * h->cfg.d_in * 2);
   if (e != cudaSuccess) { delete ps; return e; }

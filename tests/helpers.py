@@ -49,3 +49,12 @@ def check_parity(y, y_ref, what=""):
     assert rel <= REL_FRO_TOL, f"{what}: rel Frobenius {rel:.3e}"
     assert mabs <= MAX_ABS_TOL, f"{what}: max abs {mabs:.3e}"
     return rel, mabs
+
+
+def expected_family(M, K):
+    """The kernel family a plain layer takes under EORA_POLICY_AUTO when both families support it (the rule in
+    include/eora_linear.h): decode up to 16 tokens, tensor-core beyond 64, in between whichever is cheaper."""
+    import paper_2410_21271_b200 as eora
+    if M > 64 or (M > 16 and ((M + 7) // 8) * 30 > K // 64):
+        return eora.EORA_PATH_PREFILL
+    return eora.EORA_PATH_DECODE

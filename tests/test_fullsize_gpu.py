@@ -55,7 +55,8 @@ def test_decode_quantised_adapter_fullsize(name, ab, r, M):
     wf, af, bf = make_case(33, K, N, r, w="q4", ab=ab)
     x = gen.make_x(34, M, K)
     L = eora.Layer(wf, af, bf, max_m=M)
-    assert L.path(M) == eora.EORA_PATH_DECODE
+    # eight decode passes (M = 64) cost more than one walk over the k-blocks with the tensor-core family
+    assert L.path(M) == (eora.EORA_PATH_PREFILL if M == 64 else eora.EORA_PATH_DECODE)
     check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} {ab} r{r} M{M}")
     L.close()
 
@@ -128,4 +129,18 @@ def test_prefill_small_formats():
         y2 = run_layer(L, x, "f16")           # scratch (the split-K sums of t) must have been restored
         rel2, mabs2 = orc.parity_errors(y2, orc.forward(x, "f16", wf, af, bf))
         assert rel2 <= 2e-3 and mabs2 <= 1e-2, (w, ab, rel2, mabs2)
+        L.close()
+
+
+def test_mid_size_m_takes_the_cheaper_family():
+    """Between 17 and 64 tokens the library weighs ceil(M / 8) decode passes against one walk over the k-blocks."""
+    for name, expect in [("q", {8: "d", 16: "d", 17: "p", 24: "p", 64: "p"}), ("down", {16: "d", 48: "d", 56: "d", 57: "p", 64: "p"})]:
+        K, N = SHAPES[name]
+        wf, af, bf = make_case(45, K, N, 128, w="q4")
+        L = eora.Layer(wf, af, bf, max_m=64)
+        for M, fam in expect.items():
+            assert L.path(M) == (eora.EORA_PATH_DECODE if fam == "d" else eora.EORA_PATH_PREFILL), (name, M)
+        M = 24 if name == "q" else 57
+        x = gen.make_x(46, M, K)
+        check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} q4 M{M} tensor-core family")
         L.close()

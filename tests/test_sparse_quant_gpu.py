@@ -9,7 +9,7 @@ pytestmark = pytest.mark.gpu
 from oracle import eora_oracle as orc
 import eora_inputs as gen
 import paper_2410_21271_b200 as eora
-from helpers import make_case, run_layer, check_parity
+from helpers import make_case, run_layer, check_parity, expected_family
 
 SHAPES = gen.LLAMA3_8B_SHAPES
 
@@ -66,7 +66,7 @@ def test_forward_matches_oracle(policy, ab, K, N, r, M, xd, group):
     x = gen.make_x(93, M, K, xd)
     L = eora.Layer(wf, af, bf, max_m=M, x_dtype=xd, kernel_policy=policy)
     if policy == eora.EORA_POLICY_AUTO:
-        assert L.path(M) == (eora.EORA_PATH_DECODE if M <= 64 else eora.EORA_PATH_PREFILL)
+        assert L.path(M) == expected_family(M, K)
     y_ref = orc.forward(x, xd, wf, af, bf)
     for rep in range(2):                                # second call: the scratch was restored
         check_parity(run_layer(L, x, xd), y_ref, f"sq4/{ab} K{K} N{N} r{r} M{M} g{group} path{L.path(M)} call {rep}")
