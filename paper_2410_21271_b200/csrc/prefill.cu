@@ -34,6 +34,7 @@ constexpr int kDqWarps = 16;                    // dequant warps (warps 4..19): 
 constexpr int kThreadsP = (4 + kDqWarps) * 32;  // warp 0: TMA, warp 1: MMA, warp 2: TMEM alloc, warp 3: idle
 constexpr int kMaxXStages = 8;                  // ring of token tiles (TMA latency is long: deep)
 constexpr int kMaxWStages = 4;                  // ring of dequantised weight tiles (produced on chip: shallow)
+constexpr int kSmallTile = 128;                // rows and tokens of the small tiles that fill a launch's last wave
 constexpr int kPrefetch = 4;                    // k-blocks of packed weights held in registers ahead of use (2 for fp16)
 
 struct PrefillArgs {
@@ -46,6 +47,10 @@ struct PrefillArgs {
   int m;
   int bt;            // token tile (the MMA N): multiple of 16, at most 256
   int rows;          // weight rows per CTA: 256 (two MMA halves) or 128 (small matrices: more CTAs, half the dequant work each)
+  // The grid is one-dimensional.  CTAs [0, n_small) take tiles of 128 rows x 128 tokens of the weight rows
+  // [n_split, n_valid) (small_x row tiles per token tile); the others take tiles of rows x bt of the weight rows
+  // [0, n_split) (big_x row tiles per token tile).  Without small tiles n_small = 0 and n_split = n_valid.
+  int n_small, small_x, n_split, big_x;
   int nkb_w, nkb_b;  // k-blocks of each part
   int sx, sw;        // stages of the token ring / of the weight ring
   int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
@@ -347,7 +352,9 @@ __device__ __forceinline__ bool dequant_part(const WMat& mat, int n0, int kb_lo,
 
 template <int WF, int BF>
 __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant__ CUtensorMap tm_x,
-                                                          const __grid_constant__ CUtensorMap tm_t, const PrefillArgs p) {
+                                                          const __grid_constant__ CUtensorMap tm_t,
+                                                          const __grid_constant__ CUtensorMap tm_x_small,
+                                                          const __grid_constant__ CUtensorMap tm_t_small, const PrefillArgs p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_x[kMaxXStages], empty_x[kMaxXStages], full_w[kMaxWStages], empty_w[kMaxWStages], acc_full;
   __shared__ uint32_t tmem_base_s;
@@ -360,12 +367,21 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   // start at once (the main product behind the launch that computes t; see launch_prefill_forward).
   asm volatile("griddepcontrol.launch_dependents;");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * p.rows, m0 = blockIdx.y * p.bt;
-  const int nh = (p.rows > BN_W && p.n_valid - n0 > BN_W) ? 2 : 1;   // 128-row halves of this CTA that hold real rows
+  const bool small = (int)blockIdx.x < p.n_small;
+  const int big_id = (int)blockIdx.x - p.n_small;
+  const int bt = small ? kSmallTile : p.bt;                 // tokens of this CTA's tile (the MMA N)
+  const int rows = small ? kSmallTile : p.rows;
+  const int n0 = small ? p.n_split + ((int)blockIdx.x % p.small_x) * kSmallTile : (big_id % p.big_x) * rows;
+  const int m0 = small ? ((int)blockIdx.x / p.small_x) * kSmallTile : (big_id / p.big_x) * bt;
+  const int n_end = small ? p.n_valid : p.n_split;          // this CTA writes columns n0 .. n_end - 1 at most
+  const int nh = (rows > BN_W && n_end - n0 > BN_W) ? 2 : 1;   // 128-row halves of this CTA that hold real rows
+  const CUtensorMap* map_x = small ? &tm_x_small : &tm_x;
+  const CUtensorMap* map_t = small ? &tm_t_small : &tm_t;
   const int kw_lo = 0, kw_hi = p.nkb_w;
   const int nkw = p.nkb_w;
   const int nkb = nkw + p.nkb_b;
-  const uint32_t xbytes = (uint32_t)p.bt * 128;
+  const uint32_t xbytes = (uint32_t)bt * 128;               // bytes of a token tile; the ring's slots are p.bt * 128 apart
+  const uint32_t xslot = (uint32_t)p.bt * 128;
 
   if constexpr (WF == FMT_SP24 || WF == FMT_SQ4) {
     if (threadIdx.x >= 32 && threadIdx.x < 48) sp_lut[threadIdx.x - 32] = sp24_selectors(threadIdx.x - 32);
@@ -398,13 +414,13 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
         if (wrap > 0 && !mbar_wait(empty_x + s, (wrap - 1) & 1, p.dev_status)) break;
         PTRACE(it, 0);
         mbar_expect_tx(full_x + s, xbytes);
-        uint8_t* xt = smem + (size_t)s * xbytes;
+        uint8_t* xt = smem + (size_t)s * xslot;
         if (it < nkw) {
-          tma_load_2d(xt, &tm_x, (kw_lo + it) * BK, m0, full_x + s);
+          tma_load_2d(xt, map_x, (kw_lo + it) * BK, m0, full_x + s);
         } else {
           // t comes from the previous launch, which may still be running: everything up to here overlapped with it
           if (it == nkw) asm volatile("griddepcontrol.wait;" ::: "memory");
-          tma_load_2d(xt, &tm_t, (it - nkw) * BK, m0, full_x + s);
+          tma_load_2d(xt, map_t, (it - nkw) * BK, m0, full_x + s);
         }
         if (++s == p.sx) { s = 0; ++wrap; }
       }
@@ -413,7 +429,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       // instruction descriptor: fp32 accumulate, fp16 x fp16, both operands K-major, M = 128 weight rows, N = bt tokens
-      const uint32_t idesc = (1u << 4) | ((uint32_t)(p.bt >> 3) << 17) | ((uint32_t)(BN_W >> 4) << 24);
+      const uint32_t idesc = (1u << 4) | ((uint32_t)(bt >> 3) << 17) | ((uint32_t)(BN_W >> 4) << 24);
       bool ok = true;
       int sx = 0, sw = 0;                           // ring slots of iteration `it` and their phases
       uint32_t px = 0, pw = 0;
@@ -424,7 +440,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
         ok = mbar_wait(full_w + sw, pw, p.dev_status);
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t bdesc = make_desc(smem + (size_t)sx * xbytes);
+        const uint64_t bdesc = make_desc(smem + (size_t)sx * xslot);
         for (int hh = 0; hh < nh; ++hh) {
           const uint64_t adesc = make_desc(smem + p.w_off + (size_t)sw * (2 * BN_W * 128) + hh * (BN_W * 128));
 #pragma unroll
@@ -462,7 +478,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       if (dw == 0 && lane == 0) PTRACE(nkb, 2);
       const int grp = dw >> 2, lq = dw & 3;
       const int nl = lq * 32 + lane;                     // local weight row inside the half = thread index inside the group
-      const int nchunk = (p.bt + 31) >> 5;
+      const int nchunk = (bt + 31) >> 5;
       const uint32_t lane_base = tmem_d + ((uint32_t)(lq * 32) << 16);
       {
         // A chunk goes through shared memory as [32 tokens][128 n] so that the global stores are 16-byte
@@ -494,7 +510,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
             for (int i = nl; i < pieces; i += 128) {
               const int tok = i >> row_sh, piece = i & ((1 << row_sh) - 1);
               const int row = m0 + c0 + tok, col = n0 + hh * BN_W + piece * (16 / esz);
-              if (row < p.m && col < p.n_valid) {
+              if (row < p.m && col < n_end) {
                 const uint4 val = *reinterpret_cast<const uint4*>(tbuf + (size_t)tok * BN_W * esz + piece * 16);
                 *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + ((int64_t)row * p.ld_out + col) * esz) = val;
               }
@@ -559,8 +575,8 @@ constexpr int kSmemP = 225 * 1024;
 // pdl: the launch may begin while the previous kernel of the stream is still running (it waits, on the
 // device, before it touches what that kernel writes).
 template <auto KERNEL>
-cudaError_t launch_p(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt, const PrefillArgs& a,
-                     bool pdl) {
+cudaError_t launch_p(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt, const CUtensorMap& txs,
+                     const CUtensorMap& tts, const PrefillArgs& a, bool pdl) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
@@ -577,31 +593,31 @@ cudaError_t launch_p(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, KERNEL, tx, tt, a);
+  return cudaLaunchKernelEx(&cfg, KERNEL, tx, tt, txs, tts, a);
 }
 
 template <int WF>
 cudaError_t launch_bf(int bf, dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt,
-                      const PrefillArgs& a, bool pdl) {
+                      const CUtensorMap& txs, const CUtensorMap& tts, const PrefillArgs& a, bool pdl) {
   switch (bf) {
-    case FMT_F16: return launch_p<k_prefill<WF, FMT_F16>>(grid, smem, st, tx, tt, a, pdl);
-    case FMT_Q4: return launch_p<k_prefill<WF, FMT_Q4>>(grid, smem, st, tx, tt, a, pdl);
-    case FMT_Q8: return launch_p<k_prefill<WF, FMT_Q8>>(grid, smem, st, tx, tt, a, pdl);
-    case FMT_Q3: return launch_p<k_prefill<WF, FMT_Q3>>(grid, smem, st, tx, tt, a, pdl);
-    default: return launch_p<k_prefill<WF, FMT_NONE>>(grid, smem, st, tx, tt, a, pdl);
+    case FMT_F16: return launch_p<k_prefill<WF, FMT_F16>>(grid, smem, st, tx, tt, txs, tts, a, pdl);
+    case FMT_Q4: return launch_p<k_prefill<WF, FMT_Q4>>(grid, smem, st, tx, tt, txs, tts, a, pdl);
+    case FMT_Q8: return launch_p<k_prefill<WF, FMT_Q8>>(grid, smem, st, tx, tt, txs, tts, a, pdl);
+    case FMT_Q3: return launch_p<k_prefill<WF, FMT_Q3>>(grid, smem, st, tx, tt, txs, tts, a, pdl);
+    default: return launch_p<k_prefill<WF, FMT_NONE>>(grid, smem, st, tx, tt, txs, tts, a, pdl);
   }
 }
 
 cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt,
-                       const PrefillArgs& a, bool pdl) {
+                       const CUtensorMap& txs, const CUtensorMap& tts, const PrefillArgs& a, bool pdl) {
   switch (wf) {
-    case FMT_Q4: return launch_bf<FMT_Q4>(bf, grid, smem, st, tx, tt, a, pdl);
-    case FMT_Q3: return launch_bf<FMT_Q3>(bf, grid, smem, st, tx, tt, a, pdl);
-    case FMT_SP24: return launch_bf<FMT_SP24>(bf, grid, smem, st, tx, tt, a, pdl);
-    case FMT_SQ4: return launch_bf<FMT_SQ4>(bf, grid, smem, st, tx, tt, a, pdl);
+    case FMT_Q4: return launch_bf<FMT_Q4>(bf, grid, smem, st, tx, tt, txs, tts, a, pdl);
+    case FMT_Q3: return launch_bf<FMT_Q3>(bf, grid, smem, st, tx, tt, txs, tts, a, pdl);
+    case FMT_SP24: return launch_bf<FMT_SP24>(bf, grid, smem, st, tx, tt, txs, tts, a, pdl);
+    case FMT_SQ4: return launch_bf<FMT_SQ4>(bf, grid, smem, st, tx, tt, txs, tts, a, pdl);
     // A as the weight of the first launch (t = X.A): no K-extension there
-    case FMT_F16: return launch_p<k_prefill<FMT_F16, FMT_NONE>>(grid, smem, st, tx, tt, a, pdl);
-    case FMT_Q8: return launch_p<k_prefill<FMT_Q8, FMT_NONE>>(grid, smem, st, tx, tt, a, pdl);
+    case FMT_F16: return launch_p<k_prefill<FMT_F16, FMT_NONE>>(grid, smem, st, tx, tt, txs, tts, a, pdl);
+    case FMT_Q8: return launch_p<k_prefill<FMT_Q8, FMT_NONE>>(grid, smem, st, tx, tt, txs, tts, a, pdl);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -703,9 +719,10 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt_t;
     a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status; a.trace = nullptr;
     a.rows = rows_t;
+    a.n_small = 0; a.small_x = 1; a.n_split = a.n_valid; a.big_x = (h->r_pad + a.rows - 1) / a.rows;
     const int smem_t = fill_stages(a);
-    dim3 grid((h->r_pad + a.rows - 1) / a.rows, (m + bt_t - 1) / bt_t, 1);
-    cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_xt, tm_xt, a, false);
+    dim3 grid(a.big_x * ((m + bt_t - 1) / bt_t), 1, 1);
+    cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_xt, tm_xt, tm_xt, tm_xt, a, false);
     if (e != cudaSuccess) return e;
   } else {
     tm_t = tm_x;
@@ -717,9 +734,29 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
   a.trace = reinterpret_cast<long long*>(h->trace);
   a.rows = cta_rows(c.d_out, m, bt, h->sm_count);
+  a.n_small = 0; a.small_x = 1; a.n_split = c.d_out; a.big_x = (c.d_out + a.rows - 1) / a.rows;
+  const int big_y = (m + bt - 1) / bt;
+  // Wave quantisation: a CTA needs an SM of its own, so a few tiles more than a whole number of waves cost a whole
+  // wave (gate / up at M = 2048: 448 tiles on 148 SMs).  Then the last row tiles are taken out of the big grid until
+  // it fits, and their rows are covered by small tiles (128 x 128, about half the time of a big one each) that are
+  // dispatched first and share the launch's first wave with the big tiles.
+  CUtensorMap tm_xs = tm_x, tm_ts = tm_t;
+  const int tiles = a.big_x * big_y, over = tiles % h->sm_count;
+  if (a.rows == 2 * BN_W && bt == 256 && tiles > h->sm_count && over > 0 && 4 * over <= h->sm_count) {
+    const int peel = (over + big_y - 1) / big_y;                 // row tiles to take out
+    if (peel < a.big_x) {
+      a.big_x -= peel;
+      a.n_split = a.big_x * a.rows;
+      a.small_x = (c.d_out - a.n_split + kSmallTile - 1) / kSmallTile;
+      a.n_small = a.small_x * ((m + kSmallTile - 1) / kSmallTile);
+      if (!make_map(&tm_xs, x16, m, c.d_in, c.d_in, kSmallTile)) return cudaErrorInvalidValue;
+      if (ab && !make_map(&tm_ts, h->t16, m, h->r_pad, h->r_pad, kSmallTile)) return cudaErrorInvalidValue;
+      if (!ab) tm_ts = tm_xs;
+    }
+  }
   const int smem_y = fill_stages(a);
-  dim3 grid((c.d_out + a.rows - 1) / a.rows, (m + bt - 1) / bt, 1);
-  return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, a, ab);
+  dim3 grid(a.n_small + a.big_x * big_y, 1, 1);
+  return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, tm_xs, tm_ts, a, ab);
 }
 
 }  // namespace eora

@@ -24,6 +24,10 @@ def sampled_check(L, wf, af, bf, x, xd, n_samples=96, seed=0):
     mi = rng.integers(0, M, n_samples)
     ni = rng.integers(0, N, n_samples)
     mi[:4] = [0, M - 1, 0, M - 1]; ni[:4] = [0, 0, N - 1, N - 1]          # corners: first / last tile edges
+    # the last output columns (a launch may cover them with tiles of another size) and both sides of tile borders
+    ni[4:20] = N - 1 - rng.integers(0, min(N, 512), 16)
+    ni[20:28] = np.clip(128 * rng.integers(1, max(2, N // 128), 8) - rng.integers(0, 2, 8), 0, N - 1)
+    mi[28:36] = np.clip(128 * rng.integers(1, max(2, M // 128), 8) - rng.integers(0, 2, 8), 0, M - 1)
     ref = orc.forward_at(x, xd, wf, af, bf, mi, ni)
     got = y[mi, ni]
     d = got - ref
