@@ -32,8 +32,7 @@ namespace {
 constexpr int BN_W = 128, BK = 64;               // weight rows per MMA (its M), k-block; a CTA owns up to two such halves
 constexpr int kDqWarps = 16;                    // dequant warps (warps 4..19): one 16-row tile of the 256 weight rows each
 constexpr int kThreadsP = (4 + kDqWarps) * 32;  // warp 0: TMA, warp 1: MMA, warp 2: TMEM alloc, warp 3: idle
-constexpr int kMaxXStages = 8;                  // ring of token tiles (TMA latency is long: deep)
-constexpr int kMaxWStages = 4;                  // ring of dequantised weight tiles (produced on chip: shallow)
+constexpr int kMaxWStages = 4;                  // ring of k-block stages (token tile + dequantised weight tile)
 constexpr int kSmallTile = 128;                // rows and tokens of the small tiles that fill a launch's last wave
 constexpr int kPrefetch = 4;                    // k-blocks of packed weights held in registers ahead of use (2 for fp16)
 
@@ -52,7 +51,7 @@ struct PrefillArgs {
   // [0, n_split) (big_x row tiles per token tile).  Without small tiles n_small = 0 and n_split = n_valid.
   int n_small, small_x, n_split, big_x;
   int nkb_w, nkb_b;  // k-blocks of each part
-  int sx, sw;        // stages of the token ring / of the weight ring
+  int sx, sw;        // stages of the ring (sx == sw: token tiles first, weight tiles from w_off on)
   int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
   int* dev_status;
   long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (token copy requested, W ready, X ready, MMA issued),
@@ -356,7 +355,11 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
                                                           const __grid_constant__ CUtensorMap tm_x_small,
                                                           const __grid_constant__ CUtensorMap tm_t_small, const PrefillArgs p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_x[kMaxXStages], empty_x[kMaxXStages], full_w[kMaxWStages], empty_w[kMaxWStages], acc_full;
+  // One ring for both operands: stage s holds the token tile and the dequantised weight tile of a k-block, full_w[s]
+  // collects the copy's bytes and the dequant warps' arrivals, empty_w[s] one commit.  The thread that issues the MMAs
+  // is what bounds a k-block (every MMA blocks it for the ~130 cycles its 128-row operand takes to load), so it gets
+  // one wait and one commit per k-block instead of two of each.
+  __shared__ __align__(8) uint64_t full_w[kMaxWStages], empty_w[kMaxWStages], acc_full;
   __shared__ uint32_t tmem_base_s;
   __shared__ uint32_t sp_lut[16];        // 2:4 expansion selectors (2:4 backbones only)
   __shared__ int fail_s;                 // set by an epilogue warp whose bounded wait ran out
@@ -390,8 +393,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   if (threadIdx.x == 0) {
     PTRACE(nkb, 0);
     fail_s = 0;
-    for (int i = 0; i < p.sx; ++i) { mbar_init(full_x + i, 1); mbar_init(empty_x + i, 1); }
-    for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8 * nh); mbar_init(empty_w + i, 1); }
+    for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8 * nh + 1); mbar_init(empty_w + i, 1); }
     mbar_init(&acc_full, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -411,18 +413,18 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
     if (lane == 0) {
       int s = 0, wrap = 0;                          // ring slot of iteration `it`, and how often it has been used before
       for (int it = 0; it < nkb; ++it) {
-        if (wrap > 0 && !mbar_wait(empty_x + s, (wrap - 1) & 1, p.dev_status)) break;
+        if (wrap > 0 && !mbar_wait(empty_w + s, (wrap - 1) & 1, p.dev_status)) break;
         PTRACE(it, 0);
-        mbar_expect_tx(full_x + s, xbytes);
+        mbar_expect_tx(full_w + s, xbytes);
         uint8_t* xt = smem + (size_t)s * xslot;
         if (it < nkw) {
-          tma_load_2d(xt, map_x, (kw_lo + it) * BK, m0, full_x + s);
+          tma_load_2d(xt, map_x, (kw_lo + it) * BK, m0, full_w + s);
         } else {
           // t comes from the previous launch, which may still be running: everything up to here overlapped with it
           if (it == nkw) asm volatile("griddepcontrol.wait;" ::: "memory");
-          tma_load_2d(xt, map_t, (it - nkw) * BK, m0, full_x + s);
+          tma_load_2d(xt, map_t, (it - nkw) * BK, m0, full_w + s);
         }
-        if (++s == p.sx) { s = 0; ++wrap; }
+        if (++s == p.sw) { s = 0; ++wrap; }
       }
     }
   } else if (warp == 1) {
@@ -431,26 +433,25 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       // instruction descriptor: fp32 accumulate, fp16 x fp16, both operands K-major, M = 128 weight rows, N = bt tokens
       const uint32_t idesc = (1u << 4) | ((uint32_t)(bt >> 3) << 17) | ((uint32_t)(BN_W >> 4) << 24);
       bool ok = true;
-      int sx = 0, sw = 0;                           // ring slots of iteration `it` and their phases
-      uint32_t px = 0, pw = 0;
+      int sw = 0;                                   // ring slot of iteration `it` and its phase
+      uint32_t pw = 0;
       for (int it = 0; it < nkb && ok; ++it) {
-        ok = mbar_wait(full_x + sx, px, p.dev_status);
+        ok = mbar_wait(full_w + sw, pw, p.dev_status);   // token tile copied and weight tile dequantised
         if (!ok) break;
         PTRACE(it, 2);
-        ok = mbar_wait(full_w + sw, pw, p.dev_status);
-        if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t bdesc = make_desc(smem + (size_t)sx * xslot);
-        for (int hh = 0; hh < nh; ++hh) {
-          const uint64_t adesc = make_desc(smem + p.w_off + (size_t)sw * (2 * BN_W * 128) + hh * (BN_W * 128));
+        const uint64_t bdesc = make_desc(smem + (size_t)sw * xslot);
+        const uint64_t adesc = make_desc(smem + p.w_off + (size_t)sw * (2 * BN_W * 128));
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)        // 32 bytes (16 fp16) further along K per step: +2 in the address field
-            umma_f16(tmem_d + hh * 256, adesc + 2 * k, bdesc + 2 * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+        for (int j = 0; j < 8; ++j) {
+          // half j / 4 of the weight rows is 128 rows = 16 KB further (+1024 in the address field), each K step of
+          // 16 fp16 is 32 bytes further (+2)
+          if (j < 4 * nh)
+            umma_f16(tmem_d + (j >> 2) * 256, adesc + (uint64_t)((j >> 2) * ((BN_W * 128) >> 4) + 2 * (j & 3)), bdesc + 2 * (j & 3),
+                     idesc, (it > 0 || (j & 3) > 0) ? 1u : 0u);
         }
-        umma_commit(empty_x + sx);                  // both arrive when these MMAs have finished reading their operands
-        umma_commit(empty_w + sw);
+        umma_commit(empty_w + sw);                  // arrives when these MMAs have finished reading their operands
         PTRACE(it, 3);
-        if (++sx == p.sx) { sx = 0; px ^= 1u; }
         if (++sw == p.sw) { sw = 0; pw ^= 1u; }
       }
       umma_commit(&acc_full);                       // arrives when every MMA above has completed
@@ -623,12 +624,12 @@ cudaError_t launch_any(int wf, int bf, dim3 grid, int smem, cudaStream_t st, con
 }
 
 int fill_stages(PrefillArgs& a) {      // returns the dynamic shared memory to request
-  a.sw = 3;
-  const int w_bytes = a.sw * 2 * BN_W * 128;
-  a.sx = (kSmemP - 1024 - w_bytes) / (a.bt * 128);
-  if (a.sx > kMaxXStages) a.sx = kMaxXStages;
+  const int stage = a.bt * 128 + 2 * BN_W * 128;       // token tile + weight tile of one k-block
+  a.sw = (kSmemP - 1024) / stage;
+  if (a.sw > kMaxWStages) a.sw = kMaxWStages;
+  a.sx = a.sw;
   a.w_off = a.sx * a.bt * 128;
-  return a.w_off + w_bytes + 1024;
+  return a.w_off + a.sw * 2 * BN_W * 128 + 1024;
 }
 
 // Weight rows per CTA: 256, or 128 when 256-row tiles would leave more than half of the SMs without a CTA
