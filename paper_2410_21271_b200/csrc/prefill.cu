@@ -9,8 +9,8 @@
 //     warp), turn them into fp16 RN((q - z) * s) in registers and store them as a K-major,
 //     128-byte-swizzled operand tile (bank-conflict-free stores);
 //   * MMA "B" operand (up to 256 rows): a tile of tokens of X, K-major, brought in by TMA
-//     (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a deep ring, because TMA latency is
-//     several k-blocks long;
+//     (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into the same ring of k-block stages as
+//     the dequantised weight tile;
 //   * one thread issues tcgen05.mma (M = 128, N = tokens, K = 16) with the fp32 accumulator in tensor
 //     memory; tcgen05.commit releases the ring slots when the MMAs have drained;
 //   * the low-rank term is a K-extension: after the d_in/64 backbone k-blocks come r/64 k-blocks whose
