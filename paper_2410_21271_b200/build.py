@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libeora_linear.so")
-SOURCES = ["eora_api.cu", "repack.cu", "generic.cu", "decode.cu", "prefill.cu", "noalloc.cu"]
+SOURCES = ["eora_api.cu", "repack.cu", "generic.cu", "decode.cu", "decode_tc.cu", "tmat.cu", "prefill.cu", "noalloc.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

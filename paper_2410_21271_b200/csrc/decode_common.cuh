@@ -64,6 +64,25 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, i
   if (ok) { while (!mbar_try_wait(bar, parity)) {} }
   return ok != 0;
 }
+// The same without the back-off, for hand-overs that are short and sit on the critical path of a pipeline (a sleeping
+// poll adds up to its period to every hand-over).  try_wait itself suspends the thread for a while, so this is no hot spin.
+__device__ __forceinline__ bool mbar_wait_warp_fast(uint64_t* bar, uint32_t parity, int* dev_status, int lane) {
+  if (mbar_try_wait(bar, parity)) return true;
+  int ok = 1;
+  if (lane == 0) {
+    const unsigned long long t0 = globaltimer_ns();
+    ok = 0;
+    for (;;) {
+#pragma unroll 1
+      for (int it = 0; it < 256 && !ok; ++it) ok = mbar_try_wait(bar, parity) ? 1 : 0;
+      if (ok || globaltimer_ns() - t0 > kWaitLimitNs) break;
+    }
+    if (!ok) atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
+  }
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  if (ok) { while (!mbar_try_wait(bar, parity)) {} }
+  return ok != 0;
+}
 
 // Bounded spin on a global counter reaching `target`.
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p);

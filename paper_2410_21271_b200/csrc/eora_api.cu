@@ -76,6 +76,7 @@ int pick_path(const Handle* h, int m) {
   // The decode family streams the weights once per eight tokens, the tensor-core family walks the d_in / 64
   // k-blocks of the layer once whatever m is: measured, a decode pass costs about as much as 30 k-blocks, so
   // from three passes on (m > 16 with d_in = 4096, m > 56 with d_in = 14336) the tensor-core family is faster.
+  if (decode_tc_supported(h, m)) return EORA_PATH_DECODE;   // one pass over the weights per sixteen tokens
   const bool dec = m <= 64 && decode_supported(h, m), pre = prefill_supported(h, m);
   if (dec && pre) return ((m + 7) / 8) * 30 > h->cfg.d_in / 64 ? EORA_PATH_PREFILL : EORA_PATH_DECODE;
   if (dec) return EORA_PATH_DECODE;
@@ -189,6 +190,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   auto fail = [&](int code) {
     if (h->prefill_state) prefill_free(h);
+    if (h->tc_state) decode_tc_free(h);
     if (h->weight_mem) cudaFree(h->weight_mem);
     if (h->scratch_mem) cudaFree(h->scratch_mem);
     delete obj;
@@ -272,7 +274,8 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   }
   if (e != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (!fused && prefill_init(h) != cudaSuccess) return fail(EORA_ERR_CUDA);
-  if (fused && !decode_supported(h, 1)) return fail(EORA_ERR_UNSUPPORTED);
+  if (decode_tc_init(h, s) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (fused && !decode_supported(h, 1) && !decode_tc_supported(h, 1)) return fail(EORA_ERR_UNSUPPORTED);
   if (cudaStreamSynchronize(s) != cudaSuccess) return fail(EORA_ERR_CUDA);
   *out = obj;
   return EORA_OK;
@@ -417,9 +420,12 @@ int eora_linear_forward_fused(eora_linear_t obj, const void* x, int32_t m, void*
     if (!ys[i]) return EORA_ERR_NULL_ARG;
     if (!aligned16(ys[i])) return EORA_ERR_MISALIGNED;
   }
+  if (h->multi) return EORA_ERR_UNSUPPORTED;                  // several adapters: forward_multi says which
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (decode_tc_supported(h, m)) return launch_decode_tc_forward(h, x, m, ys, s) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
   if (!decode_supported(h, m)) return EORA_ERR_UNSUPPORTED;
-  return launch_decode_forward(h, x, m, ys, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
+  return launch_decode_forward(h, x, m, ys, s) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
 }
 
 // Device-side alias of a host result buffer the GPU can store to directly (page-locked and mapped), else nullptr. Small
@@ -466,6 +472,7 @@ int eora_linear_destroy(eora_linear_t obj) {
   Handle* h = &obj->h;
   int rc = EORA_OK;
   if (h->prefill_state) prefill_free(h);
+  if (h->tc_state) decode_tc_free(h);
   if (h->weight_mem && cudaFree(h->weight_mem) != cudaSuccess) rc = EORA_ERR_CUDA;
   if (h->scratch_mem && cudaFree(h->scratch_mem) != cudaSuccess) rc = EORA_ERR_CUDA;
   delete obj;
@@ -482,7 +489,7 @@ int eora_linear_path(eora_linear_t obj, int32_t m) {
 int eora_linear_launches(eora_linear_t obj, int32_t m) {
   int p = eora_linear_path(obj, m);
   if (p < 0) return p;
-  if (p == EORA_PATH_DECODE) return decode_launch_count(&obj->h, m);
+  if (p == EORA_PATH_DECODE) return decode_tc_supported(&obj->h, m) ? decode_tc_launch_count(&obj->h, m) : decode_launch_count(&obj->h, m);
   if (p == EORA_PATH_PREFILL) return prefill_launch_count(&obj->h, m);
   return generic_launch_count(&obj->h);
 }
@@ -501,7 +508,7 @@ int eora_linear_forward(eora_linear_t obj, const void* x, int32_t m, void* y, vo
   int p = pick_path(h, m);
   cudaError_t e;
   void* ys[1] = {y};
-  if (p == EORA_PATH_DECODE) e = launch_decode_forward(h, x, m, ys, s);
+  if (p == EORA_PATH_DECODE) e = decode_tc_supported(h, m) ? launch_decode_tc_forward(h, x, m, ys, s) : launch_decode_forward(h, x, m, ys, s);
   else if (p == EORA_PATH_PREFILL) e = launch_prefill_forward(h, x, m, y, s);
   else e = launch_generic_forward(h, x, m, y, s);
   return e == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
@@ -536,11 +543,16 @@ int eora_linear_dump(eora_linear_t obj, int32_t what, void* outp, void* stream) 
 
 int eora_linear_last_device_status(eora_linear_t obj) {
   if (!obj) return EORA_ERR_NULL_ARG;
+  Handle* h = &obj->h;
   int v = 0;
-  if (cudaMemcpy(&v, obj->h.dev_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EORA_ERR_CUDA;
+  if (cudaMemcpy(&v, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EORA_ERR_CUDA;
   if (v != 0) {
-    int z = 0;
-    if (cudaMemcpy(obj->h.dev_status, &z, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return EORA_ERR_CUDA;
+    // A kernel whose wait ran out returned early and left partial sums, tickets and counters behind: put all
+    // scratch that must be zero between launches (status word included) back, so that the handle stays usable.
+    char* lo = reinterpret_cast<char*>(h->d_t);
+    char* hi = reinterpret_cast<char*>(h->dev_status) + 256;
+    if (cudaMemset(lo, 0, (size_t)(hi - lo)) != cudaSuccess) return EORA_ERR_CUDA;
+    if (decode_tc_reset(h, nullptr) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return EORA_ERR_CUDA;
   }
   return v;
 }
@@ -555,10 +567,11 @@ int eora_linear_decode_grid(eora_linear_t obj, int32_t m) {
   if (!obj) return EORA_ERR_NULL_ARG;
   if (m < 1 || m > 64) return EORA_ERR_BAD_SHAPE;
   if (pick_path(&obj->h, m) != EORA_PATH_DECODE) return 0;
+  if (decode_tc_supported(&obj->h, m)) return decode_tc_grid(&obj->h);
   return decode_grid(&obj->h, m);
 }
 
-int64_t eora_linear_weight_bytes(eora_linear_t obj) { return obj ? obj->h.weight_bytes : 0; }
-int64_t eora_linear_scratch_bytes(eora_linear_t obj) { return obj ? obj->h.scratch_bytes : 0; }
+int64_t eora_linear_weight_bytes(eora_linear_t obj) { return obj ? obj->h.weight_bytes + decode_tc_weight_bytes(&obj->h) : 0; }
+int64_t eora_linear_scratch_bytes(eora_linear_t obj) { return obj ? obj->h.scratch_bytes + decode_tc_scratch_bytes(&obj->h) : 0; }
 
 }  // extern "C"

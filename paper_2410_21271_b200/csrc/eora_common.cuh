@@ -211,6 +211,7 @@ struct Handle {
   int n_adapters;        // 1 for a plain layer
   int multi;             // 1: created with per-token adapter selection (eora_linear_create_multi)
   void* prefill_state;   // owned by prefill.cu (tensor maps), may be NULL
+  void* tc_state;        // owned by decode_tc.cu (its copy of the weights, scratch, work split), NULL if that family does not serve the handle
   void* trace;           // optional caller-owned timestamp buffer, may be NULL
 };
 
@@ -233,6 +234,17 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
                                   const int32_t* adapter_ids = nullptr);
 int decode_launch_count(const Handle* h, int m);
 int decode_grid(const Handle* h, int m);
+
+// tensor-memory decode family (decode_tc.cu)
+cudaError_t decode_tc_init(Handle* h, cudaStream_t st);
+void decode_tc_free(Handle* h);
+bool decode_tc_supported(const Handle* h, int m);
+cudaError_t launch_decode_tc_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st);
+int decode_tc_launch_count(const Handle* h, int m);
+int decode_tc_grid(const Handle* h);
+int64_t decode_tc_weight_bytes(const Handle* h);
+int64_t decode_tc_scratch_bytes(const Handle* h);
+cudaError_t decode_tc_reset(const Handle* h, cudaStream_t st);
 
 bool prefill_supported(const Handle* h, int m);
 cudaError_t prefill_init(Handle* h);
