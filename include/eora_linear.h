@@ -75,7 +75,7 @@ enum { EORA_Y_F16 = 0, EORA_Y_BF16 = 1, EORA_Y_F32 = 2 };
 /* kernel families reported by eora_linear_path */
 enum { EORA_PATH_GENERIC = 0, EORA_PATH_DECODE = 1, EORA_PATH_PREFILL = 2 };
 /* kernel_policy */
-enum { EORA_POLICY_AUTO = 0, EORA_POLICY_GENERIC = 1 };
+enum { EORA_POLICY_AUTO = 0, EORA_POLICY_GENERIC = 1, EORA_POLICY_TMEM_DECODE = 2 };
 
 /* Plain-old-data, caller-owned, copied by create. */
 typedef struct {
@@ -90,7 +90,8 @@ typedef struct {
   int32_t x_dtype;     /* EORA_X_F16 or EORA_X_BF16 */
   int32_t y_dtype;     /* EORA_Y_F16, EORA_Y_BF16 or EORA_Y_F32 */
   int32_t max_m;       /* largest M forward will be called with (sizes the scratch memory) */
-  int32_t kernel_policy; /* EORA_POLICY_AUTO, or EORA_POLICY_GENERIC to force the simple kernels */
+  int32_t kernel_policy; /* EORA_POLICY_AUTO; EORA_POLICY_GENERIC forces the simple kernels; EORA_POLICY_TMEM_DECODE: as AUTO, but M <= 64
+                            goes to the tensor-memory decode kernels where they serve the layer (see eora_linear_forward) */
 } eora_linear_config;
 
 /* Device pointers, interchange layout (see the top of this file); 16-byte aligned. */
@@ -122,7 +123,8 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
 /*
  * Y[M][d_out] = X[M][d_in] . deq(Wq) + (X . A) . B   (Eq. 4), enqueued on `stream`.
  * x, y: device pointers, row-major, 16-byte aligned, caller-owned; 1 <= m <= max_m; m == 0 is a
- * no-op returning EORA_OK.  Never synchronises and never allocates.  M <= 16 runs the decode
+ * no-op returning EORA_OK.  Never synchronises and never allocates.  The current device must be the one
+ * the handle was created on (EORA_ERR_UNSUPPORTED otherwise).  M <= 16 runs the decode
  * kernel family (one streaming pass over the weights per eight tokens), M > 64 the tensor-core
  * (tcgen05) prefill family, and in between whichever is cheaper for the layer: the prefill family
  * once ceil(M / 8) * 30 exceeds d_in / 64 (eora_linear_path reports the choice).  Asynchronous device-side
@@ -198,7 +200,9 @@ int eora_linear_dump(eora_linear_t h, int32_t what, void* out, void* stream);
 
 /*
  * Status word latched by the kernels (0 = fine, EORA_ERR_DEVICE_TIMEOUT = a bounded wait ran
- * out).  Reads device memory with a blocking copy: call after synchronising.  Clears the word.
+ * out).  Reads device memory with a blocking copy: call after synchronising.  Clears the word; if it was
+ * not zero, the handle's scratch (partial sums, t, tickets) is put back to its between-calls state as well, so
+ * that the handle stays usable (the outputs of the call that timed out are undefined).
  */
 int eora_linear_last_device_status(eora_linear_t h);
 
@@ -247,9 +251,31 @@ int eora_linear_set_trace(eora_linear_t h, void* trace_buf);
 int eora_linear_forward_noalloc(const eora_linear_config* cfg, const eora_linear_weights* w, const void* x,
                                 int32_t m, void* y, void* stream);
 
-/* Bytes of device memory the handle owns: re-tiled weights, and scratch. */
+/*
+ * Bytes of device memory the handle owns: the re-tiled weights; the scratch the kernels need (partial sums, t, tickets:
+ * a few hundred KB to a few MB); and the staging buffers of the *_host entry points, [max_m][d_in] + [max_m][d_out],
+ * which are allocated by the first *_host call on the handle (0 before that): a model whose activations stay on the
+ * device keeps the memory saving that compression buys (paper Section 4.5, the model-size table).
+ */
 int64_t eora_linear_weight_bytes(eora_linear_t h);
 int64_t eora_linear_scratch_bytes(eora_linear_t h);
+int64_t eora_linear_staging_bytes(eora_linear_t h);
+
+/*
+ * Diagnostics.  The one wait between thread blocks that Eq. 4 imposes (the product with B needs all of t = X.A) is bounded:
+ * a kernel that waits longer than the limit latches EORA_ERR_DEVICE_TIMEOUT, lets its copies in flight land and
+ * returns by itself; the outputs of that call are undefined, and eora_linear_last_device_status puts the handle's scratch
+ * back so that the next forward is correct.  Default (and ns == 0): one second.  A test sets it to a few nanoseconds to see
+ * the timeout path end to end; nothing hangs or faults in it.
+ */
+int eora_linear_set_wait_limit(eora_linear_t h, uint64_t ns);
+/*
+ * Self-test of that path: enqueues a one-warp kernel that leaves a partial sum, a partial t and a ticket in the handle's
+ * scratch (what a kernel that gives up leaves behind) and then waits, bounded by the handle's limit, for a count nobody
+ * raises.  After synchronising, eora_linear_last_device_status must report EORA_ERR_DEVICE_TIMEOUT, and the next forward
+ * must be correct again.  Nothing faults or hangs: the wait returns by itself.
+ */
+int eora_linear_selftest_wait_timeout(eora_linear_t h, void* stream);
 
 /* Human-readable name of a status code; never NULL. */
 const char* eora_status_string(int status);

@@ -23,7 +23,7 @@ EORA_AB_F16, EORA_AB_Q4, EORA_AB_Q8, EORA_AB_Q3 = 0, 1, 2, 3
 EORA_X_F16, EORA_X_BF16 = 0, 1
 EORA_Y_F16, EORA_Y_BF16, EORA_Y_F32 = 0, 1, 2
 EORA_PATH_GENERIC, EORA_PATH_DECODE, EORA_PATH_PREFILL = 0, 1, 2
-EORA_POLICY_AUTO, EORA_POLICY_GENERIC = 0, 1
+EORA_POLICY_AUTO, EORA_POLICY_GENERIC, EORA_POLICY_TMEM_DECODE = 0, 1, 2
 
 
 class eora_linear_config(Structure):
@@ -80,6 +80,12 @@ def lib() -> ctypes.CDLL:
         L.eora_linear_dump.restype = c_int
         L.eora_linear_last_device_status.argtypes = [c_void_p]
         L.eora_linear_last_device_status.restype = c_int
+        L.eora_linear_set_wait_limit.argtypes = [c_void_p, ctypes.c_uint64]
+        L.eora_linear_set_wait_limit.restype = c_int
+        L.eora_linear_selftest_wait_timeout.argtypes = [c_void_p, c_void_p]
+        L.eora_linear_selftest_wait_timeout.restype = c_int
+        L.eora_linear_staging_bytes.argtypes = [c_void_p]
+        L.eora_linear_staging_bytes.restype = ctypes.c_int64
         L.eora_linear_set_trace.argtypes = [c_void_p, c_void_p]
         L.eora_linear_set_trace.restype = c_int
         L.eora_linear_decode_grid.argtypes = [c_void_p, c_int32]
@@ -238,6 +244,18 @@ def eora_linear_last_device_status(handle: int) -> int:
     return lib().eora_linear_last_device_status(handle)
 
 
+def eora_linear_set_wait_limit(handle: int, ns: int) -> int:
+    return lib().eora_linear_set_wait_limit(handle, int(ns))
+
+
+def eora_linear_selftest_wait_timeout(handle: int, stream=None) -> int:
+    return lib().eora_linear_selftest_wait_timeout(handle, _stream(stream))
+
+
+def eora_linear_staging_bytes(handle: int) -> int:
+    return lib().eora_linear_staging_bytes(handle)
+
+
 def eora_linear_set_trace(handle: int, buf) -> int:
     return lib().eora_linear_set_trace(handle, _ptr(buf))
 
@@ -389,12 +407,13 @@ class FusedLayers:
     """Several layers that read the same X (q/k/v, gate/up) behind ONE handle and one launch per forward.
     Decode only (max_m <= 64).  Methods only marshal arguments."""
 
-    def __init__(self, layers, *, max_m: int, x_dtype: str = "f16", y_dtype: str = "f16", device="cuda:0"):
+    def __init__(self, layers, *, max_m: int, x_dtype: str = "f16", y_dtype: str = "f16",
+                 kernel_policy: int = EORA_POLICY_AUTO, device="cuda:0"):
         import torch
         cfgs, wtss, keep = [], [], []
         for (w_fmt, a_fmt, b_fmt) in layers:
             cfg, wts, k = _marshal(w_fmt, a_fmt, b_fmt, max_m=max_m, x_dtype=x_dtype, y_dtype=y_dtype,
-                                   kernel_policy=EORA_POLICY_AUTO, device=device)
+                                   kernel_policy=kernel_policy, device=device)
             cfgs.append(cfg); wtss.append(wts); keep.append(k)
         self.cfgs = cfgs
         self.device = torch.device(device)

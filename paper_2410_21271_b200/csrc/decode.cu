@@ -70,6 +70,7 @@ struct DecodeArgs {
   int adp[8];
   float* d_t; float* y_ws; uint32_t* counters; int* dev_status;
   int m, d_in, r_pad, n_pad, x_dtype, y_dtype;   // r_pad: columns of t (all fused layers / adapters)
+  unsigned long long wait_ns;             // limit of the wait for t
   unsigned long long* trace;
 };
 
@@ -290,7 +291,7 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     if constexpr (HILO) {
       // all of A must be in t
       int ok = 1;
-      if (lane == 0) ok = counter_wait(p.counters + CNT_A_DONE, p.a_blobs, p.dev_status) ? 1 : 0;
+      if (lane == 0) ok = counter_wait(p.counters + CNT_A_DONE, p.a_blobs, p.dev_status, p.wait_ns) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) return false;
       __syncwarp();
@@ -474,16 +475,23 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
     if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
     if (ok) ok = run_segment<WF, false, OUT_Y, I8>(p, r, w0 + wf, wn - wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
   }
+  if (!ok) {
+    // This warp gave up: its bulk copies still in flight must land before the CTA's shared memory may be reused.  A slot
+    // of the ring is in flight exactly if a copy was requested for it and not consumed: slots from the consumer position on
+    // complete the current phase, the ones before it the next one; a slot without a copy passes at once or after the drain's short limit.
+    for (int i = 0; i < kRing - r.deferred; ++i) mbar_drain_warp(r.bars + i, i >= r.slot ? r.parity : r.parity ^ 1u, lane);
+  }
   if (tr && lane == 0) tr[3] = globaltimer_ns();
 }
 
 template <auto KERNEL>
-cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const DecodeArgs& args) {
-  static bool attr_set = false;   // one per kernel (KERNEL is a template argument)
-  if (!attr_set) {
+cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int device) {
+  static bool attr_set[64] = {};  // per kernel (KERNEL is a template argument) and device: the attribute belongs to the current device
+  if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[device]) {
     cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[device] = true;
   }
   return cudaLaunchKernelEx(&cfg, KERNEL, args);
 }
@@ -492,21 +500,21 @@ cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const DecodeArgs& args)
 constexpr bool has_i8(int fmt) { return fmt == FMT_Q4 || fmt == FMT_Q3; }
 
 template <int WF, bool I8>
-cudaError_t launch_ab2(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf) {
+cudaError_t launch_ab2(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf, int device) {
   switch (abf) {
-    case FMT_F16: return launch_kernel<k_decode<WF, FMT_F16, I8>>(cfg, args);
-    case FMT_Q4: return launch_kernel<k_decode<WF, FMT_Q4, I8>>(cfg, args);
-    case FMT_Q8: return launch_kernel<k_decode<WF, FMT_Q8, I8>>(cfg, args);
-    case FMT_Q3: return launch_kernel<k_decode<WF, FMT_Q3, I8>>(cfg, args);
-    default: return launch_kernel<k_decode<WF, FMT_NONE, I8>>(cfg, args);
+    case FMT_F16: return launch_kernel<k_decode<WF, FMT_F16, I8>>(cfg, args, device);
+    case FMT_Q4: return launch_kernel<k_decode<WF, FMT_Q4, I8>>(cfg, args, device);
+    case FMT_Q8: return launch_kernel<k_decode<WF, FMT_Q8, I8>>(cfg, args, device);
+    case FMT_Q3: return launch_kernel<k_decode<WF, FMT_Q3, I8>>(cfg, args, device);
+    default: return launch_kernel<k_decode<WF, FMT_NONE, I8>>(cfg, args, device);
   }
 }
 template <int WF>
-cudaError_t launch_ab(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf) {
+cudaError_t launch_ab(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf, int device) {
   if constexpr (has_i8(WF)) {
-    if (args.m == 1) return launch_ab2<WF, true>(cfg, args, abf);
+    if (args.m == 1) return launch_ab2<WF, true>(cfg, args, abf, device);
   }
-  return launch_ab2<WF, false>(cfg, args, abf);
+  return launch_ab2<WF, false>(cfg, args, abf, device);
 }
 
 // Relative cost of one blob (time a warp spends on it); only the ratios matter.
@@ -535,6 +543,22 @@ uint32_t blobs_per_copy(const WMat& m) {
 }
 
 }  // namespace
+
+// One thread waits, bounded by the handle's limit, for a count that nobody raises, after leaving the kind of debris a
+// kernel that gives up leaves behind (a partial sum, a partial t, a ticket).  See eora_linear_selftest_wait_timeout.
+__global__ void k_wait_selftest(uint32_t* counters, float* y_ws, float* d_t, int* dev_status, unsigned long long limit_ns) {
+  if (threadIdx.x == 0) {
+    y_ws[0] += 1.f;
+    d_t[0] += 1.f;
+    counters[CNT_TICKET0] += 1u;
+    dec::counter_wait(counters + CNT_A_DONE, 0xffffffffu, dev_status, limit_ns);
+  }
+}
+
+cudaError_t launch_wait_selftest(const Handle* h, cudaStream_t st) {
+  k_wait_selftest<<<1, 32, 0, st>>>(h->counters, h->y_ws, h->d_t, h->dev_status, h->wait_limit_ns);
+  return cudaGetLastError();
+}
 
 bool decode_supported(const Handle* h, int m) {
   if (m < 1 || m > 64) return false;
@@ -607,6 +631,7 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
   for (int i = 0; i < 4; ++i) a.sub_dout[i] = i < h->n_sub ? h->sub_dout[i] : 0;
   a.x_dtype = h->cfg.x_dtype; a.y_dtype = h->cfg.y_dtype;
   a.trace = reinterpret_cast<unsigned long long*>(h->trace);
+  a.wait_ns = h->wait_limit_ns;
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
@@ -632,9 +657,9 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
         a.adp[i] = (id >= 0 && id < h->n_adapters) ? id : -1;
       }
     }
-    cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf)
-                  : h->w.fmt == FMT_Q3 ? launch_ab<FMT_Q3>(cfg, a, abf)
-                  : h->w.fmt == FMT_SQ4 ? launch_ab<FMT_SQ4>(cfg, a, abf) : launch_ab<FMT_SP24>(cfg, a, abf);
+    cudaError_t e = h->w.fmt == FMT_Q4 ? launch_ab<FMT_Q4>(cfg, a, abf, h->device)
+                  : h->w.fmt == FMT_Q3 ? launch_ab<FMT_Q3>(cfg, a, abf, h->device)
+                  : h->w.fmt == FMT_SQ4 ? launch_ab<FMT_SQ4>(cfg, a, abf, h->device) : launch_ab<FMT_SP24>(cfg, a, abf, h->device);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

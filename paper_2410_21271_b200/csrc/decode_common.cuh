@@ -20,6 +20,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same test, but the thread may stay suspended (taking no issue slots) until the phase completes or `ns` nanoseconds
+// have passed: what a waiting loop polls with, so that many waiting warps do not crowd out the working ones.
+__device__ __forceinline__ bool mbar_try_wait_susp(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -33,7 +41,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* d
   for (;;) {
 #pragma unroll 1
     for (int it = 0; it < 64; ++it)
-      if (mbar_try_wait(bar, parity)) return true;
+      if (mbar_try_wait_susp(bar, parity, 20000u)) return true;
     if (globaltimer_ns() - t0 > kWaitLimitNs) break;
   }
   atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
@@ -65,16 +73,18 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, i
   return ok != 0;
 }
 // The same without the back-off, for hand-overs that are short and sit on the critical path of a pipeline (a sleeping
-// poll adds up to its period to every hand-over).  try_wait itself suspends the thread for a while, so this is no hot spin.
+// poll adds up to its period to every hand-over).  The polling try_wait suspends the thread until the phase completes.
 __device__ __forceinline__ bool mbar_wait_warp_fast(uint64_t* bar, uint32_t parity, int* dev_status, int lane) {
-  if (mbar_try_wait(bar, parity)) return true;
+  // The vote makes the lanes take the same way even if they arrive one after the other (a lane that saw the phase
+  // complete and left would leave the others waiting for it in the shuffle below).
+  if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity) ? 1 : 0)) return true;
   int ok = 1;
   if (lane == 0) {
     const unsigned long long t0 = globaltimer_ns();
     ok = 0;
     for (;;) {
 #pragma unroll 1
-      for (int it = 0; it < 256 && !ok; ++it) ok = mbar_try_wait(bar, parity) ? 1 : 0;
+      for (int it = 0; it < 256 && !ok; ++it) ok = mbar_try_wait_susp(bar, parity, 20000u) ? 1 : 0;
       if (ok || globaltimer_ns() - t0 > kWaitLimitNs) break;
     }
     if (!ok) atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
@@ -84,9 +94,20 @@ __device__ __forceinline__ bool mbar_wait_warp_fast(uint64_t* bar, uint32_t pari
   return ok != 0;
 }
 
+// Wait, for at most two milliseconds and without touching the status word, for a bulk copy that may still be in flight:
+// used by a warp that has already given up and only has to let its copies land before it leaves.
+__device__ __forceinline__ void mbar_drain_warp(uint64_t* bar, uint32_t parity, int lane) {
+  if (lane == 0) {
+    const unsigned long long t0 = globaltimer_ns();
+    while (!mbar_try_wait(bar, parity) && globaltimer_ns() - t0 < 2000000ull) __nanosleep(200);
+  }
+  __syncwarp();
+}
+
 // Bounded spin on a global counter reaching `target`.
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p);
-__device__ __forceinline__ bool counter_wait(const uint32_t* cnt, uint32_t target, int* dev_status) {
+__device__ __forceinline__ bool counter_wait(const uint32_t* cnt, uint32_t target, int* dev_status,
+                                             unsigned long long limit_ns = kWaitLimitNs) {
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
 #pragma unroll 1
@@ -94,7 +115,7 @@ __device__ __forceinline__ bool counter_wait(const uint32_t* cnt, uint32_t targe
       if (ld_acquire(cnt) >= target) return true;
       __nanosleep(32);
     }
-    if (globaltimer_ns() - t0 > kWaitLimitNs) break;
+    if (globaltimer_ns() - t0 > limit_ns) break;
   }
   atomicExch(dev_status, EORA_ERR_DEVICE_TIMEOUT);
   return false;

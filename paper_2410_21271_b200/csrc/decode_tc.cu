@@ -42,9 +42,7 @@ using namespace dec;
 namespace {
 
 constexpr int kSlotBytes = 8704;          // one ring slot = one unit (largest: Q4 / Q8, 8576 bytes)
-constexpr int kWorkerWarps = 8;
-constexpr int kWarpProducer = 8, kWarpMma = 9, kWarpConv0 = 10, kConvWarps = 2;
-constexpr int kThreadsTc = (kWorkerWarps + 2 + kConvWarps) * 32;
+constexpr int kConvWarps = 2;
 constexpr int kMaxCtas = 148;
 constexpr int kTmemCols = 256;
 constexpr int kACols = 32;                // tensor-memory columns of one operand stage
@@ -70,7 +68,7 @@ struct TcArgs {
   int* dev_status;
   uint32_t a_flush_total;
   int m, d_in, t_cols, r_pad, n_pad, x_dtype, y_dtype;
-  unsigned long long* trace;              // optional time stamps (TR_SLOTS values per CTA), may be NULL
+  unsigned long long wait_ns;             // limit of the wait for t
   CtaPlan plan[kMaxCtas];
 };
 
@@ -90,16 +88,14 @@ __device__ __forceinline__ void issue_one(uint32_t d, uint32_t a, uint32_t blo, 
                  ::"r"(d), "r"(a + 8 * K), "r"(blo + 2 * K), "r"(bhi), "r"(idesc), "n"(K > 0 ? 1 : 0) : "memory");
 }
 template <int FMT, int NCOL>
-__device__ __forceinline__ void issue_unit(uint32_t d, uint32_t a, uint32_t blo, uint32_t bhi, unsigned long long* ts = nullptr) {
+__device__ __forceinline__ void issue_unit(uint32_t d, uint32_t a, uint32_t blo, uint32_t bhi) {
   constexpr bool I8 = tmat_quant(FMT);
   constexpr uint32_t idesc = I8 ? ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NCOL >> 3) << 17) | ((128u >> 4) << 24))
                                 : ((1u << 4) | ((uint32_t)(NCOL >> 3) << 17) | ((128u >> 4) << 24));
   constexpr int N = tmat_cols(FMT) / 8;
   issue_one<I8, 0>(d, a, blo, bhi, idesc);
-  if (ts) ts[0] = clock64();
   issue_one<I8, 1>(d, a, blo, bhi, idesc);
-  if (ts) ts[1] = clock64();
-  if constexpr (N > 2) { issue_one<I8, 2>(d, a, blo, bhi, idesc); if (ts) ts[2] = clock64(); issue_one<I8, 3>(d, a, blo, bhi, idesc); if (ts) ts[3] = clock64(); }
+  if constexpr (N > 2) { issue_one<I8, 2>(d, a, blo, bhi, idesc); issue_one<I8, 3>(d, a, blo, bhi, idesc); }
 }
 __device__ __forceinline__ void umma_commit_tc(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -120,7 +116,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 __device__ __forceinline__ uint32_t atom_add_acq_rel_tc(uint32_t* p, uint32_t v) {
   uint32_t old;
   asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
@@ -156,20 +151,20 @@ __device__ __forceinline__ uint32_t ent_seg(uint32_t e) { return e & 3u; }
 __device__ __forceinline__ uint32_t ent_j(uint32_t e) { return (e >> 2) & 0x3fffu; }
 __device__ __forceinline__ uint32_t ent_T(uint32_t e) { return e >> 16; }
 
-constexpr int kAStages = 4;               // stages of the weight operand in tensor memory (32 columns each)
 constexpr int kRawSlots = 8;              // units whose raw activations are in flight (bulk copies)
 constexpr int kRawBytes = 256;            // bytes per token and unit of the raw activations (128 fp16 / 32 fp32 of t / ...)
 // stages of the activation operand (shared memory) and of the accumulator (tensor memory: 128 + XS * NCOL <= 256 columns)
 __host__ __device__ constexpr int tc_ncol(int mt) { return mt <= 8 ? 16 : 32; }
-__host__ __device__ constexpr int tc_xstages(int mt) { return mt <= 8 ? 8 : 4; }
-__host__ __device__ constexpr int tc_ring_slots(int mt) { return mt == 1 ? 9 : mt <= 8 ? 8 : 6; }
+__host__ __device__ constexpr int tc_xstages(int) { return 8; }
+__host__ __device__ constexpr int tc_ring_slots(int mt) { return mt == 1 ? 9 : mt <= 8 ? 16 : 14; }   // one token: two CTAs per SM
 
 struct Shared {
   uint64_t w_full[16], w_empty[16];       // weight ring: copy landed / unit consumed
-  uint64_t x_full[8], mma_done[8], d_empty[8];   // activation operand written / MMAs of the pair of units complete / accumulator read back
-  uint64_t a_full[kAStages];              // weight operand stored to tensor memory
+  uint64_t x_full[8], x_empty[8];         // activation stage written / its unit's accumulator (and scales) read back by the four warps
+  uint64_t mma_done[8];                   // per set: the MMAs of its unit are complete
+  uint64_t a_full[8];                     // per set: its four warps have stored their quarters of the weight operand
   float2 xaux[8][16];                     // per stage and token: (scale of the fixed-point activations, their integer sum)
-  uint32_t tab[kMaxUnits + 1];            // the run (see above)
+  uint32_t tab[kMaxUnits + 9];            // the run (see above)
   uint32_t tmem_base;
 };
 
@@ -388,21 +383,34 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t* v) {
   else tmem_ld16(taddr, v);
 }
 
-// Trace slots (uint64 per CTA, see eora_linear_set_trace): times in ns, waits in SM cycles.
-enum { TR_START = 0, TR_DEP = 1, TR_CONV_END = 2, TR_MMA_END = 3, TR_WORK_END = 4, TR_FLUSHED = 5, TR_PROD_END = 6,
-       TR_MMA_WAIT_A = 8, TR_MMA_WAIT_X = 9, TR_MMA_WAIT_D = 10, TR_MMA_ISSUE = 11,
-       TR_W_WAIT_COPY = 12, TR_W_WAIT_MMA = 13, TR_W_STORE = 14, TR_W_READ = 15, TR_W_FLUSH = 16,
-       TR_C_WAIT_RAW = 17, TR_C_WAIT_STAGE = 18, TR_C_CONVERT = 19, TR_P_WAIT = 20, TR_SLOTS = 32 };
-
 // ---------------------------------------------------------------------------------------------- the kernel
 // WF / ABF: formats of the backbone and of the adapter (FMT_NONE: no adapter).  MT: tokens the launch is compiled
 // for (1, 8 or 16); the accumulator has NCOL = 16 columns (two per token) up to eight tokens, 32 above.
+//
+// Sets.  The worker warps form NS sets of four (one warp per quarter of the 128 tensor-memory lanes).  Set k takes
+// units k, k + NS, ... of the CTA's run and does everything for a unit by itself, one step after the other: wait for the
+// unit's bytes, unpack them into the set's own 32 columns of tensor memory, one thread (once all four have stored) issues the
+// unit's MMAs into the set's own accumulator columns, all four warps wait for them, read their rows back and add them to
+// their sums.  A unit therefore takes a set a long time (~1500 cycles, most of it latency), but the sets, and the sets of
+// the next launch's CTA on the same SM, run side by side: throughput comes from the number of units in flight, not
+// from a deep pipeline inside one unit, and there is no stage that every unit has to pass one at a time.
+template <int MT> struct TcShape {
+  static constexpr int NS = MT <= 8 ? 5 : 4;            // sets: NS * (32 + NCOL) columns of tensor memory <= 256
+  static constexpr int kWorkers = 4 * NS;
+  static constexpr int kThreads = (kWorkers + 1 + kConvWarps) * 32;
+  static constexpr int kCtasPerSm = MT == 1 ? 2 : 1;    // one token: 40 registers per thread are enough, two CTAs fit
+};
+
 template <int WF, int ABF, int MT>
-__global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_constant__ TcArgs p) {
+__global__ void __launch_bounds__(TcShape<MT>::kThreads, TcShape<MT>::kCtasPerSm) k_decode_tc(const __grid_constant__ TcArgs p) {
+  constexpr int NS = TcShape<MT>::NS;
+  constexpr int kThreads = TcShape<MT>::kThreads;
+  constexpr int kWarpProd = 4 * NS, kWarpConv = 4 * NS + 1;
   constexpr int NCOL = tc_ncol(MT);
-  constexpr int XS = tc_xstages(MT);
+  constexpr int XS = 8;                                  // activation stages
   constexpr int kXStage = NCOL * 128;
   constexpr int RS = tc_ring_slots(MT);
+  constexpr int kSetCols = kACols + NCOL;                // a set's columns: weight operand, then accumulator
   constexpr int kWarpRaw = MT == 1 ? 512 : ((MT + 1) / 2) * kRawBytes;   // one slot of a converter warp's ring of raw activations
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -413,9 +421,6 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
 
   asm volatile("griddepcontrol.launch_dependents;");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  unsigned long long* tr = p.trace ? p.trace + (size_t)blockIdx.x * TR_SLOTS : nullptr;
-  unsigned long long* tu = (p.trace && blockIdx.x == 0) ? p.trace + (size_t)148 * TR_SLOTS : nullptr;   // per-unit stamps (clock64), 8 per unit
-  if (tr && threadIdx.x == 0) tr[TR_START] = globaltimer_ns();
 
   Run run;
   {
@@ -424,8 +429,8 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
     run.n[0] = pl.an_bn & 0xffffu; run.n[1] = pl.wn; run.n[2] = pl.an_bn >> 16;
   }
   const uint32_t n_units = run.n[0] + run.n[1] + run.n[2];
-  for (uint32_t i = threadIdx.x; i <= n_units; i += kThreadsTc) {
-    uint32_t e = 0xffffffffu;
+  for (uint32_t i = threadIdx.x; i < n_units + NS + 1; i += kThreads) {
+    uint32_t e = 0xffffffffu;                            // the table ends in NS + 1 all-ones entries
     if (i < n_units) {
       const uint32_t seg = i < run.n[0] ? 0u : i < run.n[0] + run.n[1] ? 1u : 2u;
       const uint32_t u = sel3(seg, run.u0[0] + i, run.u0[1] + (i - run.n[0]), run.u0[2] + (i - run.n[0] - run.n[1]));
@@ -437,12 +442,12 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < RS; ++i) { mbar_init(sh.w_full + i, 1); mbar_init(sh.w_empty + i, 4); }
-    for (int i = 0; i < XS; ++i) { mbar_init(sh.x_full + i, MT == 1 ? 1 : kConvWarps); mbar_init(sh.mma_done + i, 1); mbar_init(sh.d_empty + i, 4); }
-    for (int i = 0; i < kAStages; ++i) mbar_init(sh.a_full + i, 4);
+    for (int i = 0; i < XS; ++i) { mbar_init(sh.x_full + i, MT == 1 ? 1 : kConvWarps); mbar_init(sh.x_empty + i, 4); }
+    for (int i = 0; i < NS; ++i) { mbar_init(sh.mma_done + i, 1); mbar_init(sh.a_full + i, 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == kWarpMma) {
+  if (warp == kWarpProd) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -452,18 +457,13 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
   const uint32_t tmem = sh.tmem_base;
   const uint32_t* tab = sh.tab;
 
-  if (warp == kWarpProducer) {
+  if (warp == kWarpProd) {
     // ------------------------------------------------------------------ bulk copies of the weights: one unit per slot
     if (lane == 0) {
       uint32_t slot = 0, sph = 0;
       bool ok = true;
-      long long wt = 0;
       for (uint32_t i = 0; i < n_units; ++i) {
-        if (i >= (uint32_t)RS) {
-          const long long t0 = tr ? clock64() : 0;
-          if (!mbar_wait(sh.w_empty + slot, sph ^ 1u, p.dev_status)) { ok = false; break; }
-          if (tr) wt += clock64() - t0;
-        }
+        if (i >= (uint32_t)RS && !mbar_wait(sh.w_empty + slot, sph ^ 1u, p.dev_status)) { ok = false; break; }
         const uint32_t e = tab[i], seg = ent_seg(e);
         const uint32_t bytes = seg == SEG_W ? tmat_unit_bytes(WF) : tmat_unit_bytes(ABF);
         const uint8_t* src = seg == 0 ? p.q[0] : seg == 1 ? p.q[1] : p.q[2];
@@ -476,62 +476,20 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
         // a consumer gave up: wait (bounded) for the copies still in flight before the CTA may exit
         for (uint32_t s2 = 0; s2 < (uint32_t)RS; ++s2) mbar_wait(sh.w_full + s2, slot > s2 ? sph : sph ^ 1u, p.dev_status);
       }
-      if (tr) { tr[TR_PROD_END] = globaltimer_ns(); tr[TR_P_WAIT] = (unsigned long long)wt; }
     }
-  } else if (warp == kWarpMma) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint64_t bdesc0 = make_desc_tc(smem_u32(xst));
-      const uint32_t blo0 = (uint32_t)bdesc0, bhi = (uint32_t)(bdesc0 >> 32);
-      // Eight units per turn of the loop: the stage of the activations / accumulator (u), the stage of the weight
-      // operand (u % 4) and its phase (u / 4) are then compile-time constants.
-      uint32_t px = 0;
-      bool ok = true;
-      for (uint32_t base = 0; base < n_units && ok; base += 8, px ^= 1u) {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (XS == 4 && u == 4) px ^= 1u;                     // four stages: two phases per turn
-          const uint32_t i = base + u;
-          if (i < n_units && ok) {
-            constexpr int dummy = 0; (void)dummy;
-            const int sx = u % XS, sa = u % kAStages;
-            ok = mbar_wait(sh.a_full + sa, (uint32_t)((u / kAStages) & 1), p.dev_status);
-            if (ok) ok = mbar_wait(sh.x_full + sx, px, p.dev_status);
-            if (tu) tu[i * 8 + 2] = clock64();
-            if (ok) {
-              // the accumulator stage is free: the converter waited for its read-back before it rewrote the activation stage
-              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-              const uint32_t d = tmem + (128 + sx * NCOL), a = tmem + sa * kACols, blo = blo0 + sx * (kXStage >> 4);
-              unsigned long long* ts = tu ? tu + 64 * 8 + i * 8 : nullptr;
-              if (ts) ts[7] = clock64();
-              if (ent_seg(tab[i]) == SEG_W) issue_unit<WF, NCOL>(d, a, blo, bhi, ts);
-              else if constexpr (ABF != FMT_NONE) issue_unit<ABF, NCOL>(d, a, blo, bhi);
-              // a commit costs the issuing thread about as much as eight MMAs: one per pair of units (one unit of each set)
-              if ((u & 1) || i + 1 == n_units) umma_commit_tc(sh.mma_done + (sx >> 1));
-              if (tu) tu[i * 8 + 3] = clock64();
-              if (ts) ts[4] = clock64();
-            }
-          }
-        }
-        if (XS == 4) px ^= 1u;                                  // undo the extra flip: the loop header flips once per turn
-      }
-      if (tr) tr[TR_MMA_END] = globaltimer_ns();
-    }
-  } else if (warp >= kWarpConv0) {
+  } else if (warp >= kWarpConv) {
     // ------------------------------------------------------------------ activation operand
-    const int cw = warp - kWarpConv0;
+    const int cw = warp - kWarpConv;
     uint8_t* myraw = rawr + cw * (kRawSlots * kWarpRaw);
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (tr && cw == 0 && lane == 0) tr[TR_DEP] = globaltimer_ns();
     bool t_ready = false, ok = true;
-    long long wr = 0, ws = 0, wc = 0;
     // t must be complete before B's activations are read.  ahead: only look (never wait for t ahead of time: the flushes
     // of A it waits for may be this CTA's own, behind units that still need this warp).  1: go on, 0: not yet, -1: gave up.
     auto t_check = [&](bool ahead) -> int {
       int rdy = 0;
       if (lane == 0) {
         if (ahead) rdy = ld_acquire(p.counters + CNT_A_FLUSHED) >= p.a_flush_total ? 1 : 0;
-        else rdy = counter_wait(p.counters + CNT_A_FLUSHED, p.a_flush_total, p.dev_status) ? 1 : -1;
+        else rdy = counter_wait(p.counters + CNT_A_FLUSHED, p.a_flush_total, p.dev_status, p.wait_ns) ? 1 : -1;
       }
       return __shfl_sync(0xffffffffu, rdy, 0);
     };
@@ -547,18 +505,21 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
         default: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
       }
     };
+    // stage i % XS may be rewritten once the set that used it for unit i - XS has read its accumulator (and scales) back
+    auto stage_free = [&](uint32_t i) -> bool {
+      return i < (uint32_t)XS || mbar_wait_warp(sh.x_empty + i % XS, ((i / XS) & 1u) ^ 1u, p.dev_status, lane);
+    };
     if constexpr (MT == 1) {
       // One token.  The units are taken in PASSES: two consecutive units of the backbone (half a warp each, eight values
       // per lane) or one unit of another kind; the two warps alternate passes.  A warp fetches the raw activations of its
       // own passes kRawSlots of them ahead with one 16-byte cp.async per lane, which the same lane reads back later.
       const int half = lane >> 4, l16 = lane & 15;
       const uint32_t hmask = half ? 0xffff0000u : 0x0000ffffu;
-      // walk the passes: (first unit, number of units) of pass number `pn`
       uint32_t ci = 0, cpn = 0;                              // conversion side: next unit, pass number
       uint32_t fi = 0, fpn = 0, fown = 0;                    // fetch side: next unit, pass number, own passes requested so far
       uint32_t cown = 0;                                     // own passes converted so far
       auto pass_len = [&](uint32_t i) -> uint32_t {
-        return (ent_seg(tab[i]) == SEG_W && ent_seg(tab[i + 1]) == SEG_W) ? 2u : 1u;     // tab[n_units] is all ones
+        return (ent_seg(tab[i]) == SEG_W && ent_seg(tab[i + 1]) == SEG_W) ? 2u : 1u;     // the table ends in all-ones entries
       };
       auto fetch_pass = [&](uint32_t i, uint32_t len, uint32_t slot) {
         const uint32_t dst = smem_u32(myraw + slot * kWarpRaw);
@@ -604,20 +565,14 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
             fi += flen; ++fpn;
           }
           if (!ok) break;
-          long long t0 = tr ? clock64() : 0, t1;
           wait_groups(fown - 1 - cown);
           __syncwarp();
-          if (tr) { t1 = clock64(); wr += t1 - t0; t0 = t1; }
           // ---- convert this pass
           const uint8_t* raw = myraw + (cown % kRawSlots) * kWarpRaw;
           const uint32_t i0 = ci + (len == 2 ? (uint32_t)half : 0u);
-          const uint32_t sx = i0 % XS, px = (i0 / XS) & 1u;
+          const uint32_t sx = i0 % XS;
           if (len == 2) {
-            // both stages must have been read back: wait for the first, then the second (same order in both halves)
-            const uint32_t sa0 = ci % XS, sa1 = (ci + 1) % XS;
-            if (ci >= (uint32_t)XS && !mbar_wait_warp(sh.d_empty + sa0, ((ci / XS) & 1u) ^ 1u, p.dev_status, lane)) break;
-            if (ci + 1 >= (uint32_t)XS && !mbar_wait_warp(sh.d_empty + sa1, (((ci + 1) / XS) & 1u) ^ 1u, p.dev_status, lane)) break;
-            if (tr) { t1 = clock64(); ws += t1 - t0; t0 = t1; }
+            if (!stage_free(ci) || !stage_free(ci + 1)) break;
             const uint4 u = reinterpret_cast<const uint4*>(raw)[lane];
             const bool bf16 = p.x_dtype == EORA_X_BF16;
             const float2 a = h2_to_f2(u.x, bf16), b = h2_to_f2(u.y, bf16), c2 = h2_to_f2(u.z, bf16), d2 = h2_to_f2(u.w, bf16);
@@ -625,10 +580,9 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
             fixed_point_rows<8>(f, smem_u32(xst + sx * kXStage), sh.xaux[sx], 0, l16, hmask);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (l16 == 0) { mbar_arrive(sh.x_full + sx); if (tu) tu[i0 * 8 + 1] = clock64(); }
+            if (l16 == 0) mbar_arrive(sh.x_full + sx);
           } else {
-            if (ci >= (uint32_t)XS && !mbar_wait_warp(sh.d_empty + sx, px ^ 1u, p.dev_status, lane)) break;
-            if (tr) { t1 = clock64(); ws += t1 - t0; t0 = t1; }
+            if (!stage_free(ci)) break;
             const uint32_t stage = smem_u32(xst + sx * kXStage);
             const uint32_t seg = ent_seg(tab[ci]);
             if (seg == SEG_W) convert_unit<WF, false>(p, stage, sh.xaux[sx], raw, 0, lane);
@@ -640,7 +594,6 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(sh.x_full + sx);
           }
-          if (tr) wc += clock64() - t0;
           ++cown;
         }
         ci += len; ++cpn;
@@ -692,13 +645,10 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
           ++pf;
         }
         if (!ok) break;
-        const uint32_t sx = i % XS, px = (i / XS) & 1u;
-        long long t0 = tr ? clock64() : 0, t1;
+        const uint32_t sx = i % XS;
         wait_groups(pf - 1 - i);
         __syncwarp();
-        if (tr) { t1 = clock64(); wr += t1 - t0; t0 = t1; }
-        if (i >= (uint32_t)XS && !mbar_wait_warp(sh.d_empty + sx, px ^ 1u, p.dev_status, lane)) break;
-        if (tr) { t1 = clock64(); ws += t1 - t0; t0 = t1; }
+        if (!stage_free(i)) break;
         const uint32_t stage = smem_u32(xst + sx * kXStage);
         const uint8_t* raw = myraw + (i % kRawSlots) * kWarpRaw;
         const int par = (cw + (int)i) & 1;
@@ -712,33 +662,25 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(sh.x_full + sx);
-        if (tr) wc += clock64() - t0;
       }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");   // nothing of this warp is in flight when the CTA exits
-    if (tr && cw == 0 && lane == 0) {
-      tr[TR_CONV_END] = globaltimer_ns();
-      tr[TR_C_WAIT_RAW] = (unsigned long long)wr; tr[TR_C_WAIT_STAGE] = (unsigned long long)ws; tr[TR_C_CONVERT] = (unsigned long long)wc;
-    }
   } else {
-    // ------------------------------------------------------------------ workers: unpack, read back, flush
-    // A warp never meets another warp: it adds its 32 rows' sums to global memory when the run leaves a (segment, row
-    // tile), takes its own ticket for that row tile one step later (the release in front of the ticket then finds the
-    // adds already performed) and looks at the ticket's answer another step later.
+    // ------------------------------------------------------------------ workers
+    // A warp never meets a warp of another set: it adds its 32 rows' sums to global memory when its set's units leave a
+    // (segment, row tile), takes its own ticket for that row tile one unit later (the release in front of the ticket then
+    // finds the adds already performed) and looks at the ticket's answer another unit later.
     const int set = warp >> 2, quad = warp & 3;
     const int rr = quad * 32 + lane;                      // this thread's row of every unit
-    const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
-    const bool tw = tr && threadIdx.x == 0;
+    const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16) + set * kSetCols;
+    const uint64_t bdesc0 = make_desc_tc(smem_u32(xst));
+    const uint32_t blo0 = (uint32_t)bdesc0, bhi = (uint32_t)(bdesc0 >> 32);
     float acc[MT];
 #pragma unroll
     for (int m = 0; m < MT; ++m) acc[m] = 0.f;
-    bool dirty = false, ok = true, dep_waited = false;
-    float s_cur = 0.f, s_prev = 0.f;
-    int z_cur = 0, z_prev = 0;
-    uint32_t slot = 0, sph = 0;
+    bool ok = true, dep_waited = false;
     // ticket state: 0 nothing pending, 1 sums of (tk_seg, tk_T) are out and its ticket is still to be taken, 2 ticket taken, answer in tk_old
     uint32_t tk_state = 0, tk_seg = 0, tk_T = 0, tk_old = 0, tk_target = 0;
-    long long wcp = 0, wmm = 0, wst = 0, wrd = 0, wfl = 0;
 
     // Row tile T is complete (this warp's ticket was the last): convert its sums, write Y, put the scratch back.
     auto finish_tile = [&](uint32_t T) {
@@ -796,110 +738,85 @@ __global__ void __launch_bounds__(kThreadsTc, 2) k_decode_tc(const __grid_consta
       if (fin) finish_tile(tk_T);
       tk_state = 0;
     };
-    auto flush = [&](uint32_t seg, uint32_t T) {
-      if (tk_state == 1) take_ticket();
-      if (tk_state == 2) resolve_ticket();
-      if (dirty && ok) {
-        float* dst = seg == SEG_A ? p.d_t + T * 128 + rr : p.y_ws + T * 128 + rr;
-        const size_t ld = seg == SEG_A ? (size_t)p.t_cols : (size_t)p.n_pad;
-#pragma unroll
-        for (int m = 0; m < MT; ++m)
-          if (m < p.m) red_add(dst + m * ld, acc[m]);
-      }
-#pragma unroll
-      for (int m = 0; m < MT; ++m) acc[m] = 0.f;
-      dirty = false;
-      tk_state = 1; tk_seg = seg; tk_T = T;
-    };
 
-    uint32_t sa = 0;                                          // stage of the weight operand of unit i
-    uint32_t sxr = 0, pxr = 0;                                // accumulator stage and phase of unit r
-    for (uint32_t i = 0; i < n_units + kAStages; ++i) {
-      // ---- read-back side: unit r = i - kAStages (its stage of the weight operand is the one unit i will be stored to)
-      if (i >= (uint32_t)kAStages) {
-        const uint32_t r = i - kAStages;
-        const uint32_t er = tab[r];
-        if ((int)(r & 1u) == set) {
-          // tickets move one step per unit of this warp
-          if (tk_state == 2) resolve_ticket();
-          else if (tk_state == 1) take_ticket();
-          long long t0 = tw ? clock64() : 0, t1;
-          if (ok) ok = mbar_wait_warp_fast(sh.mma_done + (sxr >> 1), pxr, p.dev_status, lane);
-          if (ok) ok = mbar_wait(sh.x_full + sxr, pxr, p.dev_status);   // completed long ago: this thread's acquire of the stage's scales
-          if (tu && quad == 0 && lane == 0) tu[r * 8 + 5] = clock64();
-          if (tw) { t1 = clock64(); wmm += t1 - t0; t0 = t1; }
-          if (ok) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // scale / zero-point of unit r: those of this set's last but one stored unit, unless unit r + 2 does not exist
-            const bool newest = r + 2 >= n_units;
-            const float sc = newest ? s_cur : s_prev;
-            const int zz = newest ? z_cur : z_prev;
-            const float2* aux = sh.xaux[sxr];
-            const uint32_t seg = ent_seg(er);
-#pragma unroll
-            for (int m0 = 0; m0 < MT; m0 += 8) {                   // eight tokens (sixteen columns) at a time
-              constexpr int NT = MT < 8 ? MT : 8;
-              uint32_t v[2 * NT];
-              tmem_ld_cols<2 * NT>(lane_base + 128 + sxr * NCOL + 2 * m0, v);
-              asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-              if (seg == SEG_W) accumulate_unit<WF, false, MT, NT>(acc, m0, v, aux, sc, zz, p.m);
-              else if constexpr (ABF != FMT_NONE) {
-                if (seg == SEG_A) accumulate_unit<ABF, false, MT, NT>(acc, m0, v, aux, sc, zz, p.m);
-                else accumulate_unit<ABF, true, MT, NT>(acc, m0, v, aux, sc, zz, p.m);
-              }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(sh.d_empty + sxr); if (tu && quad == 0) tu[r * 8 + 6] = clock64(); }
-            dirty = true;
-          }
-          if (tw) wrd += clock64() - t0;
-        }
-        if (++sxr == (uint32_t)XS) { sxr = 0; pxr ^= 1u; }
-        if ((er ^ tab[r + 1]) & 0xffff0003u) {                  // the run leaves (segment, row tile): its sums go out
-          const long long t0 = tw ? clock64() : 0;
-          if (!dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
-          flush(ent_seg(er), ent_T(er));
-          if (tw) wfl += clock64() - t0;
+    uint32_t own = 0;                                        // units this set has done: parity of its MMA barrier
+    for (uint32_t i = set; i < n_units; i += NS, ++own) {
+      const uint32_t e = tab[i], seg = ent_seg(e);
+      const uint32_t slot = i % RS, sph = (i / RS) & 1u, sx = i % XS, px = (i / XS) & 1u;
+      // tickets move one step per unit of this warp
+      if (tk_state == 2) resolve_ticket();
+      else if (tk_state == 1) take_ticket();
+      // ---- the unit's bytes -> the set's weight operand in tensor memory
+      float sc = 0.f;
+      int zz = 0;
+      if (ok) ok = mbar_wait_warp_fast(sh.w_full + slot, sph, p.dev_status, lane);
+      if (ok) {
+        const uint8_t* unit = ring + slot * kSlotBytes;
+        if (seg == SEG_W) { unpack_store<WF>(unit, rr, lane_base); unit_sz<WF>(unit, rr, sc, zz); }
+        else if constexpr (ABF != FMT_NONE) { unpack_store<ABF>(unit, rr, lane_base); unit_sz<ABF>(unit, rr, sc, zz); }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(sh.a_full + set); mbar_arrive(sh.w_empty + slot); }
+      }
+      // ---- one thread of the set issues the unit's MMAs once the four quarters are stored and the activations are there
+      if (quad == 0 && lane == 0 && ok) {
+        if (mbar_wait(sh.a_full + set, own & 1u, p.dev_status) && mbar_wait(sh.x_full + sx, px, p.dev_status)) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a = tmem + set * kSetCols, d = a + kACols, blo = blo0 + sx * (kXStage >> 4);
+          if (seg == SEG_W) issue_unit<WF, NCOL>(d, a, blo, bhi);
+          else if constexpr (ABF != FMT_NONE) issue_unit<ABF, NCOL>(d, a, blo, bhi);
+          umma_commit_tc(sh.mma_done + set);
         }
       }
-      // ---- store side: unit i
-      if (i < n_units) {
-        if ((int)(i & 1u) == set) {
-          long long t0 = tw ? clock64() : 0, t1;
-          if (ok) ok = mbar_wait_warp_fast(sh.w_full + slot, sph, p.dev_status, lane);
-          if (tu && quad == 0 && lane == 0) tu[i * 8 + 0] = clock64();
-          if (tw) { t1 = clock64(); wcp += t1 - t0; t0 = t1; }
-          if (ok) {
-            const uint8_t* unit = ring + slot * kSlotBytes;
-            const uint32_t taddr = lane_base + sa * kACols;
-            s_prev = s_cur; z_prev = z_cur;
-            if (ent_seg(tab[i]) == SEG_W) { unpack_store<WF>(unit, rr, taddr); unit_sz<WF>(unit, rr, s_cur, z_cur); }
-            else if constexpr (ABF != FMT_NONE) { unpack_store<ABF>(unit, rr, taddr); unit_sz<ABF>(unit, rr, s_cur, z_cur); }
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(sh.a_full + sa); mbar_arrive(sh.w_empty + slot); if (tu && quad == 0) tu[i * 8 + 4] = clock64(); }
+      // ---- read the rows back
+      __syncwarp();                                          // the issuing lane is back
+      if (ok) ok = mbar_wait_warp_fast(sh.mma_done + set, own & 1u, p.dev_status, lane);
+      if (ok) ok = mbar_wait(sh.x_full + sx, px, p.dev_status);     // complete: this thread's acquire of the stage's scales
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const float2* aux = sh.xaux[sx];
+#pragma unroll
+        for (int m0 = 0; m0 < MT; m0 += 8) {                   // eight tokens (sixteen columns) at a time
+          constexpr int NT = MT < 8 ? MT : 8;
+          uint32_t v[2 * NT];
+          tmem_ld_cols<2 * NT>(lane_base + kACols + 2 * m0, v);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          if (seg == SEG_W) accumulate_unit<WF, false, MT, NT>(acc, m0, v, aux, sc, zz, p.m);
+          else if constexpr (ABF != FMT_NONE) {
+            if (seg == SEG_A) accumulate_unit<ABF, false, MT, NT>(acc, m0, v, aux, sc, zz, p.m);
+            else accumulate_unit<ABF, true, MT, NT>(acc, m0, v, aux, sc, zz, p.m);
           }
-          if (tw) wst += clock64() - t0;
         }
-        if (++sa == (uint32_t)kAStages) sa = 0;
-        if (++slot == (uint32_t)RS) { slot = 0; sph ^= 1u; }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sh.x_empty + sx);
+      }
+      // ---- the set's next unit belongs to another (segment, row tile), or there is none: the sums go out
+      if ((e ^ tab[i + NS]) & 0xffff0003u) {
+        if (!dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
+        if (tk_state == 1) take_ticket();
+        if (tk_state == 2) resolve_ticket();
+        if (ok) {
+          const uint32_t T = ent_T(e);
+          float* dst = seg == SEG_A ? p.d_t + T * 128 + rr : p.y_ws + T * 128 + rr;
+          const size_t ld = seg == SEG_A ? (size_t)p.t_cols : (size_t)p.n_pad;
+#pragma unroll
+          for (int m = 0; m < MT; ++m)
+            if (m < p.m) red_add(dst + m * ld, acc[m]);
+        }
+#pragma unroll
+        for (int m = 0; m < MT; ++m) acc[m] = 0.f;
+        tk_state = 1; tk_seg = seg; tk_T = ent_T(e);
       }
     }
-    if (tw) tr[TR_WORK_END] = globaltimer_ns();
     // the last tickets
     if (tk_state == 1) take_ticket();
     if (tk_state == 2) resolve_ticket();
-    if (tw) {
-      tr[TR_FLUSHED] = globaltimer_ns();
-      tr[TR_W_WAIT_COPY] = (unsigned long long)wcp; tr[TR_W_WAIT_MMA] = (unsigned long long)wmm; tr[TR_W_STORE] = (unsigned long long)wst;
-      tr[TR_W_READ] = (unsigned long long)wrd; tr[TR_W_FLUSH] = (unsigned long long)wfl;
-    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == kWarpMma) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
+  if (warp == kWarpProd) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
 }
 
 template <int WF, int ABF, int MT>
@@ -952,9 +869,10 @@ struct TcState {
   int64_t weight_bytes;
   void* scratch_mem;           // d_t, y_ws, counters (zero between launches), targets (constant)
   int64_t scratch_bytes, zero_bytes;
-  float* d_t; float* y_ws; uint32_t* counters; uint32_t* targets;
+  float* d_t; float* y_ws; uint32_t* counters;
+  uint32_t* targets[2];        // tickets per row tile, for CTAs of five and of four sets
   int grid;
-  uint32_t a_flush_total;
+  uint32_t a_flush_total[2];
   CtaPlan plan[kMaxCtas];
 };
 
@@ -1030,7 +948,7 @@ static void tc_plan(TcState* t, bool ab) {
 
 cudaError_t decode_tc_init(Handle* h, cudaStream_t st) {
   h->tc_state = nullptr;
-  if (h->cfg.kernel_policy != EORA_POLICY_AUTO || !tc_formats_ok(h)) return cudaSuccess;
+  if (h->cfg.kernel_policy != EORA_POLICY_TMEM_DECODE || !tc_formats_ok(h)) return cudaSuccess;
   const bool ab = h->cfg.rank > 0;
   TcState* t = new (std::nothrow) TcState();
   if (!t) return cudaErrorMemoryAllocation;
@@ -1050,16 +968,17 @@ cudaError_t decode_tc_init(Handle* h, cudaStream_t st) {
   t->b.q = t->a.q + abytes;
   const int64_t tcols = h->t_cols;
   const int64_t dt_b = up((int64_t)kTcMaxTokens * tcols * 4), yws_b = up((int64_t)kTcMaxTokens * t->w.n_rows * 4);
-  const int64_t cnt_b = up((int64_t)(t->w.nt + 2) * 4), tgt_b = up((int64_t)t->w.nt * 4);
+  const int64_t cnt_b = up((int64_t)(t->w.nt + 2) * 4), tgt_b = up((int64_t)t->w.nt * 4);   // one array of targets; there are two
   t->zero_bytes = dt_b + yws_b + cnt_b;
-  t->scratch_bytes = t->zero_bytes + tgt_b;
+  t->scratch_bytes = t->zero_bytes + 2 * tgt_b;
   e = cudaMalloc(&t->scratch_mem, (size_t)t->scratch_bytes);
   if (e != cudaSuccess) { cudaFree(t->weight_mem); delete t; return e; }
   char* sp = reinterpret_cast<char*>(t->scratch_mem);
   t->d_t = reinterpret_cast<float*>(sp);
   t->y_ws = reinterpret_cast<float*>(sp + dt_b);
   t->counters = reinterpret_cast<uint32_t*>(sp + dt_b + yws_b);
-  t->targets = reinterpret_cast<uint32_t*>(sp + t->zero_bytes);
+  t->targets[0] = reinterpret_cast<uint32_t*>(sp + t->zero_bytes);
+  t->targets[1] = reinterpret_cast<uint32_t*>(sp + t->zero_bytes + tgt_b);
   h->tc_state = t;
   auto fail = [&](cudaError_t err) { decode_tc_free(h); return err; };
   if ((e = cudaMemsetAsync(t->scratch_mem, 0, (size_t)t->scratch_bytes, st)) != cudaSuccess) return fail(e);
@@ -1073,18 +992,33 @@ cudaError_t decode_tc_init(Handle* h, cudaStream_t st) {
     const CtaPlan& pl = t->plan[c];
     if ((pl.an_bn & 0xffffu) + (pl.an_bn >> 16) + pl.wn > (uint32_t)kMaxUnits) { decode_tc_free(h); return cudaSuccess; }
   }
-  // tickets per row tile: one per worker warp of every CTA and segment (W, B) that touches it; flushes of A likewise
-  std::vector<uint32_t> targets(t->w.nt, 0u);
-  t->a_flush_total = 0;
-  for (int c = 0; c < t->grid; ++c) {
-    const CtaPlan& p = t->plan[c];
-    const uint32_t an = p.an_bn & 0xffffu, bn = p.an_bn >> 16;
-    if (p.wn) for (uint32_t T = p.w0 / t->w.nkb; T <= (p.w0 + p.wn - 1) / t->w.nkb; ++T) targets[T] += kWorkerWarps;
-    if (bn) for (uint32_t T = p.b0 / t->b.nkb; T <= (p.b0 + bn - 1) / t->b.nkb; ++T) targets[T] += kWorkerWarps;
-    if (an) t->a_flush_total += kWorkerWarps * ((p.a0 + an - 1) / t->a.nkb - p.a0 / t->a.nkb + 1);
+  // Tickets per row tile and flushes of A: set k of a CTA takes units k, k + NS, ... of the CTA's run (A, then W, then B);
+  // each of its four warps adds its sums and takes a ticket whenever the set's next unit belongs to another (segment, row
+  // tile) or there is none.  The kernel's walk, repeated here for both numbers of sets.
+  std::vector<uint32_t> targets[2];
+  for (int v = 0; v < 2; ++v) {
+    const uint32_t NS = v == 0 ? (uint32_t)TcShape<1>::NS : (uint32_t)TcShape<16>::NS;
+    targets[v].assign(t->w.nt, 0u);
+    t->a_flush_total[v] = 0;
+    for (int c = 0; c < t->grid; ++c) {
+      const CtaPlan& pl = t->plan[c];
+      const uint32_t an = pl.an_bn & 0xffffu, bn = pl.an_bn >> 16, n = an + pl.wn + bn;
+      auto key = [&](uint32_t i) -> uint64_t {          // (segment, row tile) of unit i of the run
+        if (i < an) return ((uint64_t)0 << 32) | ((pl.a0 + i) / t->a.nkb);
+        if (i < an + pl.wn) return ((uint64_t)1 << 32) | ((pl.w0 + (i - an)) / t->w.nkb);
+        return ((uint64_t)2 << 32) | ((pl.b0 + (i - an - pl.wn)) / t->b.nkb);
+      };
+      for (uint32_t k = 0; k < NS; ++k)
+        for (uint32_t i = k; i < n; i += NS)
+          if (i + NS >= n || key(i) != key(i + NS)) {
+            const uint64_t kk = key(i);
+            if ((kk >> 32) == 0) t->a_flush_total[v] += 4;
+            else targets[v][(uint32_t)kk] += 4;
+          }
+    }
+    if ((e = cudaMemcpyAsync(t->targets[v], targets[v].data(), targets[v].size() * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
   }
-  if ((e = cudaMemcpyAsync(t->targets, targets.data(), targets.size() * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
-  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail(e);   // `targets` is a local
+  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return fail(e);   // `targets` are locals
   return cudaSuccess;
 }
 
@@ -1100,16 +1034,14 @@ cudaError_t launch_decode_tc_forward(const Handle* h, const void* x, int m, void
   for (int i = 0; i <= h->n_sub; ++i) a.sub_tile0[i] = (uint32_t)h->sub_tile0[i] / 8u;     // the handle counts tiles of 16 rows
   for (int i = h->n_sub + 1; i < 5; ++i) a.sub_tile0[i] = (uint32_t)t->w.nt;
   for (int i = 0; i < 4; ++i) a.sub_dout[i] = i < h->n_sub ? h->sub_dout[i] : 0;
-  a.d_t = t->d_t; a.y_ws = t->y_ws; a.counters = t->counters; a.targets = t->targets; a.dev_status = h->dev_status;
-  a.a_flush_total = t->a_flush_total;
+  a.d_t = t->d_t; a.y_ws = t->y_ws; a.counters = t->counters; a.dev_status = h->dev_status;
   a.d_in = h->cfg.d_in; a.t_cols = h->t_cols; a.r_pad = h->r_pad; a.n_pad = t->w.n_rows;
   a.x_dtype = h->cfg.x_dtype; a.y_dtype = h->cfg.y_dtype;
-  a.trace = reinterpret_cast<unsigned long long*>(h->trace);
+  a.wait_ns = h->wait_limit_ns;
   memcpy(a.plan, t->plan, sizeof(CtaPlan) * (size_t)t->grid);
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(t->grid);
-  cfg.blockDim = dim3(kThreadsTc);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1122,6 +1054,9 @@ cudaError_t launch_decode_tc_forward(const Handle* h, const void* x, int m, void
     a.m = m - m0 < kTcMaxTokens ? m - m0 : kTcMaxTokens;
     const int mt = a.m == 1 ? 1 : a.m <= 8 ? 8 : 16;
     cfg.dynamicSmemBytes = (size_t)tc_smem_bytes(mt);
+    cfg.blockDim = dim3(mt == 1 ? TcShape<1>::kThreads : mt == 8 ? TcShape<8>::kThreads : TcShape<16>::kThreads);
+    const int v = mt <= 8 ? 0 : 1;                      // sets per CTA: five up to eight tokens, four above
+    a.targets = t->targets[v]; a.a_flush_total = t->a_flush_total[v];
     a.x = reinterpret_cast<const uint8_t*>(x) + (size_t)m0 * h->cfg.d_in * 2;
     for (int i = 0; i < h->n_sub; ++i) a.ys[i] = reinterpret_cast<uint8_t*>(ys[i]) + (size_t)m0 * h->sub_dout[i] * ybytes;
     cudaError_t e = h->w.fmt == FMT_Q4 ? launch_tc_ab<FMT_Q4>(cfg, a, h->device, mt, abf) : launch_tc_ab<FMT_Q3>(cfg, a, h->device, mt, abf);

@@ -65,7 +65,8 @@ int check_config(const eora_linear_config& c) {
   }
   if (c.x_dtype != EORA_X_F16 && c.x_dtype != EORA_X_BF16) return EORA_ERR_UNSUPPORTED;
   if (c.y_dtype != EORA_Y_F16 && c.y_dtype != EORA_Y_BF16 && c.y_dtype != EORA_Y_F32) return EORA_ERR_UNSUPPORTED;
-  if (c.kernel_policy != EORA_POLICY_AUTO && c.kernel_policy != EORA_POLICY_GENERIC) return EORA_ERR_UNSUPPORTED;
+  if (c.kernel_policy != EORA_POLICY_AUTO && c.kernel_policy != EORA_POLICY_GENERIC && c.kernel_policy != EORA_POLICY_TMEM_DECODE)
+    return EORA_ERR_UNSUPPORTED;
   return EORA_OK;
 }
 
@@ -76,7 +77,7 @@ int pick_path(const Handle* h, int m) {
   // The decode family streams the weights once per eight tokens, the tensor-core family walks the d_in / 64
   // k-blocks of the layer once whatever m is: measured, a decode pass costs about as much as 30 k-blocks, so
   // from three passes on (m > 16 with d_in = 4096, m > 56 with d_in = 14336) the tensor-core family is faster.
-  if (decode_tc_supported(h, m)) return EORA_PATH_DECODE;   // one pass over the weights per sixteen tokens
+  if (decode_tc_supported(h, m)) return EORA_PATH_DECODE;   // EORA_POLICY_TMEM_DECODE: one pass over the weights per sixteen tokens
   const bool dec = m <= 64 && decode_supported(h, m), pre = prefill_supported(h, m);
   if (dec && pre) return ((m + 7) / 8) * 30 > h->cfg.d_in / 64 ? EORA_PATH_PREFILL : EORA_PATH_DECODE;
   if (dec) return EORA_PATH_DECODE;
@@ -179,7 +180,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     d_out_total += ci.d_out;
   }
   const bool fused = n > 1;
-  if (fused && (c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO)) return EORA_ERR_UNSUPPORTED;
+  if (fused && (c.max_m > 64 || c.kernel_policy == EORA_POLICY_GENERIC)) return EORA_ERR_UNSUPPORTED;
   c.d_out = d_out_total;
 
   eora_linear* obj = new (std::nothrow) eora_linear();
@@ -191,6 +192,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   auto fail = [&](int code) {
     if (h->prefill_state) prefill_free(h);
     if (h->tc_state) decode_tc_free(h);
+    if (h->stage_mem) cudaFree(h->stage_mem);
     if (h->weight_mem) cudaFree(h->weight_mem);
     if (h->scratch_mem) cudaFree(h->scratch_mem);
     delete obj;
@@ -199,6 +201,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   if (cudaGetDevice(&h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
 
+  h->wait_limit_ns = 1000000000ull;
   h->r_pad = (int)align_up(c.rank, 128);
   h->n_sub = n;
   h->n_adapters = 1;
@@ -230,18 +233,23 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   Carve wc{reinterpret_cast<char*>(h->weight_mem), 0};
   wmat_carve(h->w, wc); wmat_carve(h->a, wc); wmat_carve(h->b, wc);
 
-  // ---- scratch: one allocation, zero-initialised
+  // ---- scratch: one allocation, zero-initialised (the staging buffers of the *_host calls come with the first such call)
   const int64_t rp = h->t_cols;
+  bool generic_reachable = c.kernel_policy == EORA_POLICY_GENERIC;
+  if (!fused && !generic_reachable) {
+    const int probe[8] = {1, 8, 9, 16, 17, 64, 65, c.max_m};
+    for (int i = 0; i < 8; ++i)
+      if (probe[i] <= c.max_m && !(probe[i] <= 64 && decode_supported(h, probe[i])) && !prefill_supported(h, probe[i])) generic_reachable = true;
+  }
   for (int pass = 0; pass < 2; ++pass) {
     Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
-    h->t_gen = sc.take<float>((int64_t)c.max_m * rp * 4);
-    h->t16 = sc.take<__half>((int64_t)c.max_m * rp * 2);
+    // t as fp32 for the simple kernels and as fp16 for the tensor-core family: only where those families can be reached
+    h->t_gen = sc.take<float>(generic_reachable ? (int64_t)c.max_m * rp * 4 : 256);
+    h->t16 = sc.take<__half>((!fused && c.max_m > 16) ? (int64_t)c.max_m * rp * 2 : 256);
     h->d_t = sc.take<float>(8 * rp * 4);
     h->y_ws = sc.take<float>((int64_t)8 * h->w.n_rows * 4);
     h->counters = sc.take<uint32_t>((int64_t)(h->w.nt + 2) * 4);
     h->dev_status = sc.take<int>(256);
-    h->x_stage = sc.take<void>((int64_t)c.max_m * c.d_in * 2);
-    h->y_stage = sc.take<void>((int64_t)c.max_m * c.d_out * y_elem_bytes(c.y_dtype));
     if (pass == 0) {
       h->scratch_bytes = sc.off;
       if (cudaMalloc(&h->scratch_mem, (size_t)h->scratch_bytes) != cudaSuccess) { h->scratch_mem = nullptr; return fail(EORA_ERR_CUDA); }
@@ -289,7 +297,7 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
   int st = check_config(c);
   if (st != EORA_OK) return st;
   if (c.rank == 0) return EORA_ERR_BAD_SHAPE;
-  if (c.max_m > 64 || c.kernel_policy != EORA_POLICY_AUTO) return EORA_ERR_UNSUPPORTED;
+  if (c.max_m > 64 || c.kernel_policy == EORA_POLICY_GENERIC) return EORA_ERR_UNSUPPORTED;
   for (int j = 0; j < n; ++j) {
     eora_linear_weights w = wts[j];
     w.w_codes = wts[0].w_codes; w.w_scales = wts[0].w_scales; w.w_zeros = wts[0].w_zeros; w.w_meta = wts[0].w_meta;
@@ -311,6 +319,7 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
   };
   if (cudaGetDevice(&h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  h->wait_limit_ns = 1000000000ull;
   h->r_pad = (int)align_up(c.rank, 128);
   h->n_sub = 1;
   h->n_adapters = n;
@@ -343,8 +352,6 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
     h->y_ws = sc.take<float>((int64_t)8 * h->w.n_rows * 4);
     h->counters = sc.take<uint32_t>((int64_t)(h->w.nt + 2) * 4);
     h->dev_status = sc.take<int>(256);
-    h->x_stage = sc.take<void>((int64_t)c.max_m * c.d_in * 2);
-    h->y_stage = sc.take<void>((int64_t)c.max_m * c.d_out * y_elem_bytes(c.y_dtype));
     if (pass == 0) {
       h->scratch_bytes = sc.off;
       if (cudaMalloc(&h->scratch_mem, (size_t)h->scratch_bytes) != cudaSuccess) { h->scratch_mem = nullptr; return fail(EORA_ERR_CUDA); }
@@ -379,6 +386,26 @@ int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* 
 
 }  // namespace
 
+// Staging buffers of the *_host entry points ([max_m][d_in] activations, [max_m][d_out] results): allocated by the first
+// such call on the handle (these calls synchronise anyway), so that handles whose activations live on the device (the
+// usual case) do not pay for them.
+static int ensure_staging(Handle* h) {
+  if (h->stage_mem) return EORA_OK;
+  const int64_t xb = align_up((int64_t)h->cfg.max_m * h->cfg.d_in * 2, 256);
+  const int64_t yb = align_up((int64_t)h->cfg.max_m * h->cfg.d_out * y_elem_bytes(h->cfg.y_dtype), 256);
+  if (cudaMalloc(&h->stage_mem, (size_t)(xb + yb)) != cudaSuccess) { h->stage_mem = nullptr; return EORA_ERR_CUDA; }
+  h->stage_bytes = xb + yb;
+  h->x_stage = h->stage_mem;
+  h->y_stage = reinterpret_cast<char*>(h->stage_mem) + xb;
+  return EORA_OK;
+}
+
+// The handle's kernels, scratch and shared-memory attributes belong to the device it was created on.
+static bool on_handle_device(const Handle* h) {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
+
 extern "C" {
 
 int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights* wts, void* stream, eora_linear_t* out) {
@@ -404,6 +431,7 @@ int eora_linear_forward_multi(eora_linear_t obj, const void* x, int32_t m, const
   Handle* h = &obj->h;
   if (!h->multi) return EORA_ERR_UNSUPPORTED;
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  if (!on_handle_device(h)) return EORA_ERR_UNSUPPORTED;
   if (!decode_supported(h, m)) return EORA_ERR_UNSUPPORTED;
   void* ys[1] = {y};
   return launch_decode_forward(h, x, m, ys, reinterpret_cast<cudaStream_t>(stream), adapter_ids) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
@@ -422,6 +450,7 @@ int eora_linear_forward_fused(eora_linear_t obj, const void* x, int32_t m, void*
   }
   if (h->multi) return EORA_ERR_UNSUPPORTED;                  // several adapters: forward_multi says which
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  if (!on_handle_device(h)) return EORA_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (decode_tc_supported(h, m)) return launch_decode_tc_forward(h, x, m, ys, s) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
   if (!decode_supported(h, m)) return EORA_ERR_UNSUPPORTED;
@@ -448,6 +477,9 @@ int eora_linear_forward_fused_host(eora_linear_t obj, const void* x_host, int32_
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const size_t eb = y_elem_bytes(h->cfg.y_dtype);
+  if (h->multi) return EORA_ERR_UNSUPPORTED;
+  if (!on_handle_device(h)) return EORA_ERR_UNSUPPORTED;
+  if (int rc0 = ensure_staging(h)) return rc0;
   if (cudaMemcpyAsync(h->x_stage, x_host, (size_t)m * h->cfg.d_in * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) return EORA_ERR_CUDA;
   void* ys[4] = {nullptr, nullptr, nullptr, nullptr};
   size_t off = 0;
@@ -473,6 +505,7 @@ int eora_linear_destroy(eora_linear_t obj) {
   int rc = EORA_OK;
   if (h->prefill_state) prefill_free(h);
   if (h->tc_state) decode_tc_free(h);
+  if (h->stage_mem && cudaFree(h->stage_mem) != cudaSuccess) rc = EORA_ERR_CUDA;
   if (h->weight_mem && cudaFree(h->weight_mem) != cudaSuccess) rc = EORA_ERR_CUDA;
   if (h->scratch_mem && cudaFree(h->scratch_mem) != cudaSuccess) rc = EORA_ERR_CUDA;
   delete obj;
@@ -504,6 +537,7 @@ int eora_linear_forward(eora_linear_t obj, const void* x, int32_t m, void* y, vo
   if (h->n_sub != 1) return EORA_ERR_UNSUPPORTED;             // fused layers have several outputs: forward_fused
   if (h->multi) return EORA_ERR_UNSUPPORTED;                  // several adapters: forward_multi says which
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
+  if (!on_handle_device(h)) return EORA_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   int p = pick_path(h, m);
   cudaError_t e;
@@ -523,6 +557,9 @@ int eora_linear_forward_host(eora_linear_t obj, const void* x_host, int32_t m, v
   if (m > h->cfg.max_m) return EORA_ERR_M_TOO_LARGE;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   size_t xb = (size_t)m * h->cfg.d_in * 2, yb = (size_t)m * h->cfg.d_out * y_elem_bytes(h->cfg.y_dtype);
+  if (h->n_sub != 1 || h->multi) return EORA_ERR_UNSUPPORTED;
+  if (!on_handle_device(h)) return EORA_ERR_UNSUPPORTED;
+  if (int rc0 = ensure_staging(h)) return rc0;
   if (cudaMemcpyAsync(h->x_stage, x_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EORA_ERR_CUDA;
   void* y_dev = mapped_alias(y_host, m);
   int rc = eora_linear_forward(obj, h->x_stage, m, y_dev ? y_dev : h->y_stage, stream);
@@ -556,6 +593,20 @@ int eora_linear_last_device_status(eora_linear_t obj) {
   }
   return v;
 }
+
+int eora_linear_set_wait_limit(eora_linear_t obj, uint64_t ns) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  obj->h.wait_limit_ns = ns ? ns : 1000000000ull;
+  return EORA_OK;
+}
+
+int eora_linear_selftest_wait_timeout(eora_linear_t obj, void* stream) {
+  if (!obj) return EORA_ERR_NULL_ARG;
+  if (!on_handle_device(&obj->h)) return EORA_ERR_UNSUPPORTED;
+  return launch_wait_selftest(&obj->h, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
+}
+
+int64_t eora_linear_staging_bytes(eora_linear_t obj) { return obj ? obj->h.stage_bytes : 0; }
 
 int eora_linear_set_trace(eora_linear_t obj, void* buf) {
   if (!obj) return EORA_ERR_NULL_ARG;

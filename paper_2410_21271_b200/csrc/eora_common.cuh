@@ -196,8 +196,11 @@ struct Handle {
   float* y_ws;           // [8][d_out] fp32 sums of y (decode); zero between calls
   uint32_t* counters;    // decode: [0] blobs of A done, [1] row tiles finished, [2 + tile] blobs of that row tile done
   int* dev_status;       // latched device status
-  void* x_stage;         // [max_m][d_in] staging for forward_host
+  void* stage_mem;       // staging for the *_host entry points, allocated by the first such call (NULL until then)
+  int64_t stage_bytes;
+  void* x_stage;         // [max_m][d_in]
   void* y_stage;         // [max_m][d_out]
+  unsigned long long wait_limit_ns;   // how long the kernels wait for t = X.A to be complete before they give up
   int sm_count;
   // Fused layers (several layers that read the same X, e.g. q/k/v): their backbones and B's are stacked
   // along the output axis (sub i owns row tiles [sub_tile0[i], sub_tile0[i+1])), their A's along the rank
@@ -234,6 +237,7 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
                                   const int32_t* adapter_ids = nullptr);
 int decode_launch_count(const Handle* h, int m);
 int decode_grid(const Handle* h, int m);
+cudaError_t launch_wait_selftest(const Handle* h, cudaStream_t st);
 
 // tensor-memory decode family (decode_tc.cu)
 cudaError_t decode_tc_init(Handle* h, cudaStream_t st);

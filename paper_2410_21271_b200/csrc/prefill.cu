@@ -578,11 +578,13 @@ constexpr int kSmemP = 225 * 1024;
 template <auto KERNEL>
 cudaError_t launch_p(dim3 grid, int smem, cudaStream_t st, const CUtensorMap& tx, const CUtensorMap& tt, const CUtensorMap& txs,
                      const CUtensorMap& tts, const PrefillArgs& a, bool pdl) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[64] = {};   // per kernel and device: the attribute belongs to the device that is current at the call
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[device]) {
     cudaError_t e = cudaFuncSetAttribute(KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[device] = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
@@ -683,7 +685,7 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     if (!ps) return cudaErrorInvalidValue;
     int64_t n = (int64_t)m * c.d_in;
     int64_t blocks = (n / 8 + 255) / 256;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > h->sm_count * 8) blocks = h->sm_count * 8;
     k_bf16_to_f16<<<(int)blocks, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(x), ps->x16, n);
     x16 = ps->x16;
   }

@@ -148,3 +148,90 @@ def test_mid_size_m_takes_the_cheaper_family():
         x = gen.make_x(46, M, K)
         check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} q4 M{M} tensor-core family")
         L.close()
+
+
+# ---- full-size cells that take other tile / wave paths than the small cases ------------------------------------------
+def sampled_check_last_tiles(L, wf, af, bf, x, xd, n_samples=64, seed=1):
+    """Samples aimed at the last 128-row tiles of the output (a launch may cover them with tiles of another size) and at
+    the last tokens."""
+    y = run_layer(L, x, xd)
+    rng = np.random.default_rng(seed)
+    M, N = y.shape
+    mi = rng.integers(0, M, n_samples)
+    ni = N - 1 - rng.integers(0, min(N, 640), n_samples)
+    mi[: n_samples // 4] = M - 1 - rng.integers(0, min(M, 128), n_samples // 4)
+    ref = orc.forward_at(x, xd, wf, af, bf, mi, ni)
+    d = y[mi, ni] - ref
+    assert np.all(np.isfinite(y))
+    assert np.linalg.norm(d) / np.linalg.norm(ref) <= 2e-3
+    assert np.abs(d).max() <= 1e-2 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("w", ["sp24", "sq4"])
+@pytest.mark.parametrize("name", ["gate", "down"])
+def test_sparse_backbones_fullsize_single_token(w, name):
+    K, N = SHAPES[name]
+    wf, af, bf = make_case(47, K, N, 128, w=w)
+    x = gen.make_x(48, 1, K)
+    L = eora.Layer(wf, af, bf, max_m=1)
+    assert L.path(1) == eora.EORA_PATH_DECODE
+    check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} {w} M1")
+    L.close()
+
+
+@pytest.mark.parametrize("w", ["sp24", "sq4"])
+@pytest.mark.parametrize("name", ["q", "gate", "down"])
+def test_sparse_backbones_fullsize_prefill(w, name):
+    """gate at M = 2048 is the launch whose last row tiles are covered by 128 x 128 tiles."""
+    K, N = SHAPES[name]
+    M = 2048
+    wf, af, bf = make_case(49, K, N, 128, w=w)
+    x = gen.make_x(50, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    assert L.path(M) == eora.EORA_PATH_PREFILL
+    sampled_check(L, wf, af, bf, x, "f16", n_samples=64)
+    sampled_check_last_tiles(L, wf, af, bf, x, "f16")
+    L.close()
+
+
+def test_quantised_adapter_rank512_m64_on_gate():
+    K, N = SHAPES["gate"]
+    wf, af, bf = make_case(57, K, N, 512, w="q4", ab="q4")
+    x = gen.make_x(58, 64, K)
+    L = eora.Layer(wf, af, bf, max_m=64)
+    check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), "gate q4 adapters r512 M64")
+    L.close()
+
+
+def test_quantised_adapter_prefill_last_tiles_on_gate():
+    K, N = SHAPES["gate"]
+    M = 2048
+    wf, af, bf = make_case(59, K, N, 128, w="q4", ab="q4")
+    x = gen.make_x(60, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    sampled_check_last_tiles(L, wf, af, bf, x, "f16")
+    L.close()
+
+
+@pytest.mark.parametrize("M", [1, 16])
+def test_three_bit_adapter_fullsize(M):
+    K, N = SHAPES["q"]
+    wf, af, bf = make_case(61, K, N, 128, w="q4", ab="q3")
+    x = gen.make_x(62, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"q 3-bit adapters M{M}")
+    L.close()
+
+
+def test_fused_qkv_fullsize_eight_tokens():
+    import torch
+    K, r, M = 4096, 128, 8
+    parts = [(gen.make_backbone_quant(63 + i, K, n, 3, 128),) + gen.make_ab_f16(63 + i, K, n, r) for i, n in enumerate((4096, 1024, 1024))]
+    x = gen.make_x(66, M, K)
+    F = eora.FusedLayers(parts, max_m=M)
+    ys = F.forward(x_to_torch(x, "f16"))
+    torch.cuda.synchronize()
+    assert F.device_status() == 0
+    for (w, a, b), y in zip(parts, ys):
+        check_parity(y.float().cpu().numpy().astype(np.float64), orc.forward(x, "f16", w, a, b), "fused q|k|v M8")
+    F.close()

@@ -166,6 +166,21 @@ def test_dequant_fp32_is_exact_for_every_scale():
     assert w16.dtype == np.float16 and float(w16[1, 0]) == float(np.float16(7 * float(s[0, 0])))
 
 
+def test_deq_fp16_rounds_to_nearest_even_hand_worked():
+    """Hand-worked ties.  s = 1 + 3 * 2^-10 (fp16 bits 0x3C03); 3 s = 3 + 9 * 2^-10 lies exactly between the fp16 neighbours
+    3 + 8 * 2^-10 (bits 0x4204, even mantissa) and 3 + 10 * 2^-10 (0x4205): round-to-nearest-even takes 0x4204, rounding
+    halves up would take 0x4205.  With s = 1 + 2^-10 (0x3C01), 3 s = 3 + 3 * 2^-10 is the tie between 0x4201 and 0x4202 and
+    goes UP to the even 0x4202; truncation would give 0x4201.  Negative products mirror both.  The products have at most
+    5 + 11 significant bits, so an fp32 intermediate holds them exactly and cannot double-round."""
+    s = np.array([[0x3C03, 0x3C01, 0x3C03, 0x3C01]], dtype=np.uint16).view(np.float16)
+    q = np.array([[3, 3, 0, 0]], dtype=np.int64)
+    z = np.array([[0, 0, 3, 3]], dtype=np.int64)
+    w16 = orc.deq_fp16(q, z, s, 1)
+    assert w16.view(np.uint16).tolist() == [[0x4204, 0x4202, 0xC204, 0xC202]]
+    w32 = orc.deq_fp32(q, z, s, 1)
+    assert [float(v) for v in w32[0]] == [3 + 9 / 1024, 3 + 3 / 1024, -(3 + 9 / 1024), -(3 + 3 / 1024)]   # exact in fp32
+
+
 def test_q8_per_channel():
     codes = np.array([[0, 255], [128, 1]], dtype=np.uint8)
     fmt = {"kind": "q8", "rows": 2, "cols": 2, "codes": codes,

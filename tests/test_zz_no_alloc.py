@@ -11,6 +11,7 @@ import pytest
 
 pytestmark = pytest.mark.gpu
 
+from oracle import eora_oracle as orc
 import eora_inputs as gen
 import paper_2410_21271_b200 as eora
 from helpers import REL_FRO_TOL, MAX_ABS_TOL
@@ -55,6 +56,10 @@ def test_noalloc_matches_handle_forward_twice_in_a_row():
         d = got - y_ref
         assert np.linalg.norm(d) / np.linalg.norm(y_ref) <= REL_FRO_TOL
         assert np.abs(d).max() <= MAX_ABS_TOL * np.abs(y_ref).max()
+        # and against the float64 oracle (Eq. 4 written out), like every other entry point
+        y_orc = orc.forward(x.cpu().numpy(), "f16", wf, af, bf)
+        rel, mabs = orc.parity_errors(got, y_orc)
+        assert rel <= REL_FRO_TOL and mabs <= MAX_ABS_TOL, (rel, mabs)
         L.close()
         del keep
 
