@@ -292,11 +292,25 @@ def time_prefill(device: str, steps: int = 10, warmup: int = 3, layer_set: bool 
     return out
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of k_decode over the seven layers of one block, from the ncu
-# capture summarised in profiles/k_decode_llama3-8b-w3g128-r128-M1.md (traffic grows with the number of
-# blocks in proportion; fusing layers changes the number of launches, not the bytes).  Set to None when the
-# kernel's memory behaviour changes until the capture is redone.
-DRAM_BYTES_PER_BLOCK = 108.52e6
+def kernel_sources_sha() -> str:
+    """Hash of the decode kernel's sources: the DRAM traffic taken with ncu is only valid for the code it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("decode.cu", "decode_common.cuh", "eora_common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2410_21271_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def measured_dram_bytes_per_block():
+    """dram__bytes_read.sum + dram__bytes_write.sum of k_decode over the seven layers of one block, from the ncu capture
+    recorded in profiles/k_decode_traffic.json (traffic grows with the number of blocks in proportion; fusing layers
+    changes the number of launches, not the bytes).  None once the kernel's sources differ from the captured ones."""
+    p = os.path.join(ROOT, "profiles", "k_decode_traffic.json")
+    try:
+        rec = json.load(open(p))
+    except (OSError, ValueError):
+        return None
+    return rec["dram_bytes_per_block"] if rec.get("sources_sha") == kernel_sources_sha() else None
 
 
 def cpu_oracle_sample(blocks_sample: int = 1):
@@ -322,6 +336,262 @@ def cpu_oracle_sample(blocks_sample: int = 1):
     return {"value": 1.0 / sec_per_token, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{blocks_sample} of {gen.LLAMA3_8B_BLOCKS} blocks (7 layers each) of the same workload, "
                       f"{sec:.1f} s of CPU work, scaled to a whole token"}, sec
+
+
+# -------------------------------------------------------------------------------------------- all configurations
+def _host_block(w: str, ab: str, r: int, seed0: int = 2000):
+    """Seeded host data of the seven layers of one block: (name, K, N, wf, af, bf)."""
+    out = []
+    for li, (name, (K, N)) in enumerate(LAYERS):
+        seed = seed0 + li
+        if w in ("q3", "q4"):
+            wf = gen.make_backbone_quant(seed, K, N, 3 if w == "q3" else 4, 128)
+        elif w == "sp24":
+            wf = gen.make_sparse24(seed, K, N)
+        else:
+            raise ValueError(w)
+        if r == 0:
+            af = bf = None
+        elif ab == "f16":
+            af, bf = gen.make_ab_f16(seed, K, N, r)
+        else:
+            af, bf = gen.make_ab_quant(seed, K, N, r, ab)
+        out.append((name, K, N, wf, af, bf))
+    return out
+
+
+def block_bytes(w: str, ab: str, r: int, M: int, fused: bool) -> int:
+    shapes = dict(LAYERS)
+    b = sum(traffic.forward_bytes(w, ab, K, N, r, M) for _, (K, N) in LAYERS)
+    if fused:
+        b -= sum((len(g) - 1) * 2 * M * shapes[g[0]][0] for g in FUSE_GROUPS)
+    return b
+
+
+def time_decode_config(device: str, w: str, ab: str, r: int, Ms, copies: int = 4, iters: int = 20, policy: int = 0):
+    """One block's seven layers (q|k|v and gate|up fused), `copies` device copies of it (distinct handles and memory:
+    4 x 107..266 MB is far more than L2, so every launch streams from HBM), replayed as one CUDA graph.  Returns
+    {M: (ms per block, launches per block)}."""
+    import torch
+    import paper_2410_21271_b200 as eora
+    host = {name: (K, N, wf, af, bf) for name, K, N, wf, af, bf in _host_block(w, ab, r)}
+    max_m = max(Ms)
+    rings = []
+    for _ in range(copies):
+        units = []
+        for names in FUSE_GROUPS:
+            parts = [host[n][2:] for n in names]
+            if len(names) == 1:
+                obj = eora.Layer(*parts[0], max_m=max_m, device=device, kernel_policy=policy)
+            else:
+                obj = eora.FusedLayers(parts, max_m=max_m, device=device, kernel_policy=policy)
+            units.append((names, host[names[0]][0], tuple(host[n][1] for n in names), obj))
+        rings.append(units)
+    out = {}
+    stream = torch.cuda.Stream()
+    for M in Ms:
+        xs = {name: torch.from_numpy(gen.make_x(7, M, K)).to(device) for name, (K, N) in LAYERS}
+        ys = {name: torch.empty((M, N), dtype=torch.float16, device=device) for name, (K, N) in LAYERS}
+
+        def step():
+            for units in rings:
+                for names, K, Ns, obj in units:
+                    if len(names) == 1:
+                        eora.eora_linear_forward(obj.handle, xs[names[0]], M, ys[names[0]], stream)
+                    else:
+                        eora.eora_linear_forward_fused(obj.handle, xs[names[0]], M, [ys[n] for n in names], stream)
+        with torch.cuda.stream(stream):
+            step(); torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step()
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(iters):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        launches = sum(obj.launches(M) for _, _, _, obj in rings[0])
+        out[M] = (e0.elapsed_time(e1) / (iters * copies), launches)
+    for units in rings:
+        for _, _, _, obj in units:
+            assert obj.device_status() == 0, "a device-side wait ran out"
+            obj.close()
+    return out
+
+
+def time_single_layer(device: str, K: int, N: int, w: str, r: int, M: int, copies: int = 48, iters: int = 20):
+    """Config 1: one layer; `copies` device copies (48 x 10.8 MB = 4 x L2) replayed as one CUDA graph."""
+    import torch
+    import paper_2410_21271_b200 as eora
+    wf = gen.make_backbone_quant(3000, K, N, 4 if w == "q4" else 3, 128)
+    af, bf = gen.make_ab_f16(3000, K, N, r)
+    Ls = [eora.Layer(wf, af, bf, max_m=M, device=device) for _ in range(copies)]
+    x = torch.from_numpy(gen.make_x(7, M, K)).to(device)
+    y = torch.empty((M, N), dtype=torch.float16, device=device)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for L in Ls:
+            L.forward(x, y)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for L in Ls:
+                eora.eora_linear_forward(L.handle, x, M, y, stream)
+        for _ in range(3):
+            g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(iters):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    for L in Ls:
+        L.close()
+    return e0.elapsed_time(e1) / (iters * copies)
+
+
+PREFILL_SHAPES = {"q,o": (4096, 4096, 2), "k,v": (4096, 1024, 2), "gate,up": (4096, 14336, 2), "down": (14336, 4096, 1)}
+
+
+def time_prefill_config(device: str, w: str, r: int, xd: str, M: int = 2048, iters: int = 200, copies: int = 4,
+                        sustain_s: float = 0.0, device_index: int = 0):
+    """Per distinct shape of the block: `copies` device copies of the layer with their own X and Y (42..105 MB per copy:
+    more than L2 together), `iters` forwards in stream order inside one event pair.  With sustain_s > 0 the whole block
+    (seven layers) is then looped for that many seconds with the SM clock sampled, for the number against the sustained peak."""
+    import torch
+    import paper_2410_21271_b200 as eora
+    per, tot_ms, tot_fl = {}, 0.0, 0.0
+    keep = []
+    for name, (K, N, count) in PREFILL_SHAPES.items():
+        if w == "sp24":
+            wf = gen.make_sparse24(5, K, N)
+        else:
+            wf = gen.make_backbone_quant(5, K, N, 4 if w == "q4" else 3, 128)
+        af, bf = gen.make_ab_f16(5, K, N, r)
+        Ls = [eora.Layer(wf, af, bf, max_m=M, x_dtype=xd, device=device) for _ in range(copies)]
+        xh = gen.make_x(6, M, K, xd)
+        xs = [(torch.from_numpy(xh).to(device) if xd == "f16" else torch.from_numpy(xh.view(np.int16)).to(device).view(torch.bfloat16))
+              for _ in range(copies)]
+        ys = [torch.empty((M, N), dtype=torch.float16, device=device) for _ in range(copies)]
+        for L, x, y in zip(Ls, xs, ys):
+            L.forward(x, y)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            Ls[i % copies].forward(xs[i % copies], ys[i % copies])
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        fl = traffic.forward_flops(K, N, r, M)
+        per[name] = {"ms": ms, "tflops": fl / ms / 1e9, "path": {0: "generic", 1: "decode", 2: "prefill"}[Ls[0].path(M)]}
+        tot_ms += count * ms
+        tot_fl += count * fl
+        keep.append((count, Ls, xs, ys))
+    out = {"per_shape": per, "ms_block": tot_ms, "tflops_block": tot_fl / tot_ms / 1e9}
+    if sustain_s > 0:
+        def block(i):
+            for count, Ls, xs, ys in keep:
+                for c in range(count):
+                    j = (i + c) % copies
+                    Ls[j].forward(xs[j], ys[j])
+        n = max(8, int(sustain_s * 1e3 / tot_ms))
+        block(0); torch.cuda.synchronize()
+        with ClockSampler(device_index) as cs:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(n):
+                block(i)
+            e1.record()
+            torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / n
+        out["sustained"] = {"seconds": e0.elapsed_time(e1) / 1e3, "blocks": n, "ms_block": ms, "tflops_block": tot_fl / ms / 1e9,
+                            "clocks": cs.summary()}
+    for _, Ls, _, _ in keep:
+        for L in Ls:
+            L.close()
+    return out
+
+
+def all_configs(device: str, device_index: int, peaks: dict) -> list:
+    """Every configuration of the benchmark definition that the headline does not cover, device-timed."""
+    import paper_2410_21271_b200 as eora
+    hbm, burst, sust = peaks["hbm_gbs"], peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    out = []
+
+    def dec_entry(cfg, w, ab, r, M, ms, launches, note=""):
+        by = block_bytes(w, ab, r, M, True)
+        gbs = by / ms / 1e6
+        e = {"config": cfg, "workload": f"llama3-8b-block/{w}-g128/eora-{ab}-r{r}/M{M}", "kind": "decode", "ms_per_block": ms,
+             "launches_per_block": launches, "bytes_per_block": by, "GB/s": gbs, "frac_of_measured_hbm": gbs / hbm,
+             "tokens_per_s_32_blocks": M / (ms * 32 / 1e3)}
+        if note:
+            e["note"] = note
+        out.append(e)
+
+    # config 1: single 4096 x 4096 4-bit layer, fp16 r = 128, M = 1
+    ms = time_single_layer(device, 4096, 4096, "q4", 128, 1)
+    by = traffic.forward_bytes("q4", "f16", 4096, 4096, 128, 1)
+    out.append({"config": 1, "workload": "single 4096x4096/q4-g128/eora-f16-r128/M1", "kind": "decode", "ms": ms, "bytes": by,
+                "GB/s": by / ms / 1e6, "frac_of_measured_hbm": by / ms / 1e6 / hbm})
+    # config 2 at M = 8, 16 (M = 1 is the headline)
+    for M, (ms, nl) in time_decode_config(device, "q3", "f16", 128, (1, 8, 16)).items():
+        dec_entry(2, "q3", "f16", 128, M, ms, nl, "4-copy ring of one block; the headline runs all 32 blocks" if M == 1 else "")
+    # the same through the tensor-memory decode family (tcgen05 kind::i8, opt-in policy)
+    for M, (ms, nl) in time_decode_config(device, "q3", "f16", 128, (1, 16), policy=eora.EORA_POLICY_TMEM_DECODE).items():
+        dec_entry(2, "q3", "f16", 128, M, ms, nl, "kernel_policy = EORA_POLICY_TMEM_DECODE")
+    # config 3: quantised adapters
+    for ab in ("q4", "q8"):
+        for r in (128, 512):
+            for M, (ms, nl) in time_decode_config(device, "q4", ab, r, (1, 16, 64)).items():
+                dec_entry(3, "q4", ab, r, M, ms, nl)
+    # config 5 at M = 1
+    for M, (ms, nl) in time_decode_config(device, "sp24", "f16", 128, (1,)).items():
+        dec_entry(5, "sp24", "f16", 128, M, ms, nl)
+    # config 4: prefill, 4-bit, M = 2048
+    for r, xd, sustain in ((128, "f16", 2.0), (64, "f16", 0.0), (512, "f16", 0.0), (128, "bf16", 0.0)):
+        res = time_prefill_config(device, "q4", r, xd, sustain_s=sustain, device_index=device_index)
+        e = {"config": 4, "workload": f"llama3-8b-block/q4-g128/eora-f16-r{r}/X-{xd}/M2048", "kind": "prefill", **res,
+             "frac_of_measured_bf16_burst": res["tflops_block"] / burst}
+        for v in e["per_shape"].values():
+            v["frac_of_measured_bf16_burst"] = v["tflops"] / burst
+        if "sustained" in res:
+            e["sustained"]["frac_of_measured_bf16_sustained"] = res["sustained"]["tflops_block"] / sust
+        out.append(e)
+    # config 5 at M = 2048: dense-equivalent flops against 1x and 2x the dense peak (a sparse tensor path could reach 2x)
+    res = time_prefill_config(device, "sp24", 128, "f16")
+    out.append({"config": 5, "workload": "llama3-8b-block/sp24/eora-f16-r128/M2048", "kind": "prefill", **res,
+                "frac_of_measured_bf16_burst": res["tflops_block"] / burst, "frac_of_2x_burst": res["tflops_block"] / (2 * burst),
+                "note": "dense-equivalent flops; the kernel expands the 2:4 tiles on chip and issues dense MMAs"})
+    return out
+
+
+def cpu_oracle_more():
+    """The oracle, as it stands, on the other workloads: config 1, the 4-bit set with 4-bit adapters and the 2:4 set at
+    M = 1 (one block each, scaled to 32), and the q-shaped layer at M = 64."""
+    from oracle import eora_oracle as orc
+    res = []
+
+    def run(label, layers, M, scale):
+        xs = {K: gen.make_x(7, M, K) for (_, K, N, *_r) in layers}
+        t0 = time.perf_counter()
+        for (_, K, N, wf, af, bf) in layers:
+            orc.forward(xs[K], "f16", wf, af, bf)
+        sec = time.perf_counter() - t0
+        res.append({"workload": label, "seconds": sec, "value": M / (sec * scale), "unit": UNIT if scale > 1 else "tokens/s (this layer only)",
+                    "kind": "oracle", "sample": f"measured once, {sec:.1f} s of CPU work" + (f", scaled x{scale} to a whole token" if scale > 1 else "")})
+    wf = gen.make_backbone_quant(3000, 4096, 4096, 4, 128)
+    af, bf = gen.make_ab_f16(3000, 4096, 4096, 128)
+    run("config 1: single 4096x4096/q4-g128/eora-f16-r128/M1", [("q", 4096, 4096, wf, af, bf)], 1, 1)
+    run("config 3: llama3-8b-block/q4-g128/eora-q4-r128/M1", _host_block("q4", "q4", 128), 1, gen.LLAMA3_8B_BLOCKS)
+    run("config 5: llama3-8b-block/sp24/eora-f16-r128/M1", _host_block("sp24", "f16", 128), 1, gen.LLAMA3_8B_BLOCKS)
+    run("config 3: q 4096x4096/q4-g128/eora-q4-r128/M64 (one layer)", _host_block("q4", "q4", 128)[:1], 64, 1)
+    return res
 
 
 # --------------------------------------------------------------------------------------------
@@ -420,7 +690,7 @@ def main():
     roofline = {"bound": "hbm", "kernel": "k_decode", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": DRAM_BYTES_PER_BLOCK * args.blocks / n_launch_step,
+                "traffic": (lambda t: t * args.blocks / n_launch_step if t is not None else None)(measured_dram_bytes_per_block()),
                 "bytes_per_launch": bytes_step / n_launch_step, "us_per_launch": ms_local * 1e3 / n_launch_step}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -438,12 +708,14 @@ def main():
     if not args.no_extras and rank == 0:
         if world == 1:
             line["cpu_baseline"] = cpu_oracle_sample(8)[0]
+            try:
+                line["cpu_baseline"]["other_workloads"] = cpu_oracle_more()
+            except Exception as e:
+                line["cpu_baseline"]["other_workloads"] = {"error": repr(e)}
         try:
-            line["prefill"] = time_prefill(device, layer_set=True)
-            line["prefill"]["frac_of_measured_bf16_burst"] = line["prefill"]["tflops"] / peaks["bf16_tflops"]
-            line["prefill"]["layer_set"]["frac_of_measured_bf16_burst"] = line["prefill"]["layer_set"]["tflops"] / peaks["bf16_tflops"]
+            line["configs"] = all_configs(device, local_rank, peaks)
         except Exception as e:  # the decode line must still be printed
-            line["prefill"] = {"error": repr(e)}
+            line["configs"] = {"error": repr(e)}
     if rank == 0:
         print(json.dumps(line))
     if _DIST["on"]:
