@@ -36,7 +36,8 @@ using namespace dec;
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kCtasPerSm = 4;
-constexpr int kRing = 3;                  // bulk copies in flight per warp
+constexpr int kCtasPerSmI8 = 4;            // the single-token integer kernels need fewer registers
+constexpr int kRing = 2;                  // bulk copies in flight per warp
 constexpr int kSlotBytes = 4352;          // one ring slot = one bulk copy (a run of whole blobs)
 constexpr int kBarBytes = 128;            // kWarps * kRing mbarriers
 constexpr int kSmemBytes = kWarps * kRing * kSlotBytes + kBarBytes + kSp24LutBytes;
@@ -191,10 +192,17 @@ struct Ring {
   int pseg;
   // consumer side
   int slot;
-  uint32_t parity;
+  uint32_t phase;           // bit i: parity of the phase that the next copy into slot i completes
   int deferred;             // slots [kRing - deferred, kRing) have not had their first copy requested yet
   uint32_t aux;             // shared-memory address of the 2:4 expansion table (2:4 backbone only)
 };
+
+constexpr uint32_t kNone = 0xffffffffu;
+__device__ __forceinline__ uint32_t slot_parity(const Ring& r) { return (r.phase >> r.slot) & 1u; }
+__device__ __forceinline__ void slot_consumed(Ring& r) {
+  r.phase ^= 1u << r.slot;
+  if (++r.slot == kRing) r.slot = 0;
+}
 
 __device__ __forceinline__ void ring_issue(Ring& r, int slot, int lane) {
   if (r.pseg == 0 && r.rem[0] == 0) r.pseg = 1;
@@ -270,8 +278,7 @@ __device__ __forceinline__ void finish_row_tile(const DecodeArgs& p, uint32_t ti
 }
 
 // One segment: `n` consecutive blobs of one matrix starting at blob index b0.
-// I8: single-token integer inner product (backbone blobs only), see blob_product_i8.
-template <int FMT, bool HILO, int OUT, bool I8 = false>
+template <int FMT, bool HILO, int OUT>
 __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32_t b0, uint32_t n, uint32_t nt, uint32_t blob_b,
                                             uint32_t per_copy, uint32_t sz2, int lane) {
   if constexpr (FMT == FMT_NONE) {
@@ -280,14 +287,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     if (n == 0) return true;
     uint32_t pair = b0 / nt, tile = b0 - pair * nt;
     uint32_t xr[16], xl[16];
-    XI8 xi;
-    const bool x_bf16 = p.x_dtype == EORA_X_BF16;
     uint32_t sub = 0, sub_end = nt;
     Flush fl = OUT == OUT_T ? make_flush(p.d_t, p.r_pad, p.m, lane) : make_flush(p.y_ws, p.n_pad, p.m, lane);
-    if constexpr (I8) {       // all four lanes of a row add to token 0
-      fl.base = p.y_ws + (lane >> 2);
-      fl.has0 = 1u; fl.has1 = 0u;
-    }
     if constexpr (HILO) {
       // all of A must be in t
       int ok = 1;
@@ -302,8 +303,6 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
         if (i < p.n_sub && tile >= p.sub_tile0[i]) sub = i;
       sub_end = p.sub_tile0[sub + 1];
       load_t_pair(xr, xl, p, sub * p.b_np + pair, lane);
-    } else if constexpr (I8) {
-      load_x_i8<FMT>(xi, p.x, x_bf16, pair, lane);
     } else {
       load_x_pair(xr, p, pair, lane);
     }
@@ -338,29 +337,18 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     };
     while (n > 0) {
       const uint32_t cn = n < per_copy ? n : per_copy;
-      if (!mbar_wait_warp(r.bars + r.slot, r.parity, p.dev_status, lane)) return false;
+      if (!mbar_wait_warp(r.bars + r.slot, slot_parity(r), p.dev_status, lane)) return false;
       const uint8_t* src = r.slots + r.slot * kSlotBytes;
 #pragma unroll 2
       for (uint32_t j = 0; j < cn; ++j) {
         float tot[4];
-        if constexpr (I8) {
-          float t2[2];
-          blob_product_i8<FMT>(src + j * blob_b, lane, sz2, xi, t2);
-          tot[0] = t2[0]; tot[2] = t2[1]; tot[1] = 0.f; tot[3] = 0.f;     // token 0 only, every lane its own share
-        } else {
-          blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
-        }
+        blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
         if constexpr (OUT == OUT_T) {
           flush_sums(fl, tile, tot);
           ++flushed;
         } else {
           if (batch_n == 0) batch_tile = tile;
-          if constexpr (I8) {                     // one token, every lane adds: two unconditional adds
-            float* b = fl.base + tile * 16;
-            red_add(b, tot[0]); red_add(b + 8, tot[2]);
-          } else {
-            flush_sums(fl, tile, tot);
-          }
+          flush_sums(fl, tile, tot);
           if (++batch_n == 32) commit_batch();
         }
         if (++tile == nt) {
@@ -370,8 +358,6 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
             if constexpr (HILO) {
               sub = 0; sub_end = p.sub_tile0[1];
               load_t_pair(xr, xl, p, pair, lane);
-            } else if constexpr (I8) {
-              load_x_i8<FMT>(xi, p.x, x_bf16, pair, lane);
             } else {
               load_x_pair(xr, p, pair, lane);
             }
@@ -386,7 +372,7 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
       }
       __syncwarp();                               // every lane is done with the slot
       ring_issue(r, r.slot, lane);
-      if (++r.slot == kRing) { r.slot = 0; r.parity ^= 1u; }
+      slot_consumed(r);
       n -= cn;
     }
     if constexpr (OUT == OUT_T) {
@@ -399,9 +385,127 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
   }
 }
 
+// The backbone share of a single-token launch (integer inner product): the same walk as run_segment, written for
+// instruction count -- this loop is what bounds the kernel (a warp retires an instruction every ~10 cycles, and every
+// instruction around the product of a blob costs as much as one inside it): running addresses instead of index
+// arithmetic, the group layout as a compile-time constant, runs of blobs without a branch in between.
+struct WalkI8 {
+  XI8 xi;
+  uint32_t pair, tile;          // the next blob; pair == kNone: no activations loaded yet
+  uint32_t next_b;              // its index (to tell whether the next run continues this one)
+  float* yb;
+  uint32_t batch_n, my_tile;    // blobs added but without a ticket yet; lane i < batch_n: the row tile of the i-th
+  uint32_t tk_old, tk_tile, tk_n;   // tickets asked for (lane i: the one of the batch's blob i), not looked at yet
+};
+
+// The tickets asked for last time: whoever holds a row tile's last one finishes the tile.
+__device__ __forceinline__ void tickets_resolve(const DecodeArgs& p, WalkI8& w, int lane) {
+  if (w.tk_n == 0) return;
+  const uint32_t done = ((uint32_t)lane < w.tk_n && w.tk_old + 1u == p.tile_target) ? 1u : 0u;
+  const uint32_t mask = __ballot_sync(0xffffffffu, done != 0);
+  if (mask) {
+    // With an adapter the finished row tiles are counted (before they are written out, so that the two round
+    // trips overlap): the last one restores t and the counters.
+    uint32_t last = 0;
+    if (p.a_blobs && lane == 0)
+      last = atom_add_acq_rel(p.counters + CNT_TILES_DONE, (uint32_t)__popc(mask)) + __popc(mask) == p.w_nt ? 1u : 0u;
+    if (done) finish_row_tile(p, w.tk_tile);
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (last) {
+      for (int i = lane; i < 8 * p.r_pad / 4; i += 32) st_zero4(p.d_t + 4 * i);
+      if (lane == 0) { p.counters[CNT_A_DONE] = 0u; p.counters[CNT_TILES_DONE] = 0u; }
+    }
+  }
+  w.tk_n = 0;
+}
+// Tickets for the blobs added since the last batch (the release in front of them waits for the warp's additions
+// to arrive, which is why they are not taken more often than every 32 blobs).  The answers are looked at one batch later: nothing waits for
+// the round trip.
+__device__ __forceinline__ void tickets_take(const DecodeArgs& p, WalkI8& w, int lane) {
+  tickets_resolve(p, w, lane);
+  if (w.batch_n == 0) return;
+  __syncwarp();
+  if ((uint32_t)lane < w.batch_n) {
+    w.tk_tile = w.my_tile;
+    w.tk_old = atom_add_acq_rel(p.counters + CNT_TICKET0 + w.my_tile, 1u);
+  }
+  w.tk_n = w.batch_n;
+  w.batch_n = 0;
+}
+
+// The next blobs are b0, b0 + 1, ...
+template <int FMT>
+__device__ __forceinline__ void walk_seek(const DecodeArgs& p, WalkI8& w, uint32_t b0, int lane) {
+  if (b0 == w.next_b && w.pair != kNone) return;
+  const uint32_t pair = b0 / p.w_nt;
+  w.tile = b0 - pair * p.w_nt;
+  w.next_b = b0;
+  w.yb = p.y_ws + (lane >> 2) + w.tile * 16;
+  if (pair != w.pair) load_x_i8<FMT>(w.xi, p.x, p.x_dtype == EORA_X_BF16, pair, lane);
+  w.pair = pair;
+}
+
+// cn blobs in shared memory at bp; more: blobs follow after these (then the activations of the next pair are
+// fetched when these end a pair).
+template <int FMT, bool SZ2>
+__device__ __forceinline__ void walk_blobs(const DecodeArgs& p, WalkI8& w, const uint8_t* bp, uint32_t cn, bool more, int lane) {
+  constexpr uint32_t blob_b = blob_bytes(FMT, SZ2 ? 1 : 0);
+  const uint32_t nt = p.w_nt;
+  const uint32_t owner = (lane & 3) == 0 ? 1u : 0u;
+  const uint8_t* bl = bp + (FMT == FMT_Q4 ? 16 : 8) * lane;
+  const uint8_t* bg = bp + 4 * (lane >> 2);
+  w.next_b += cn;
+  for (uint32_t left = cn; left > 0;) {
+    // a run of blobs without a change of pair and without a ticket batch filling up: nothing but products and adds
+    uint32_t run = min(left, min(nt - w.tile, 32u - w.batch_n));
+    if ((uint32_t)lane - w.batch_n < run) w.my_tile = w.tile + ((uint32_t)lane - w.batch_n);
+    left -= run; w.tile += run; w.batch_n += run;
+#pragma unroll 4
+    for (; run > 0; --run, bl += blob_b, bg += blob_b, w.yb += 16) {
+      float t2[2];
+      blob_product_i8<FMT, SZ2>(bl, bg, lane, w.xi, t2);
+      red_add_if(w.yb, t2[0], owner);
+      red_add_if(w.yb + 8, t2[1], owner);
+    }
+    if (w.tile == nt) {                                 // next pair of reduction elements: other activations
+      w.tile = 0; ++w.pair; w.yb = p.y_ws + (lane >> 2);
+      if (left > 0 || more) load_x_i8<FMT>(w.xi, p.x, p.x_dtype == EORA_X_BF16, w.pair, lane);
+      else w.pair = kNone;
+    }
+    if (w.batch_n == 32) tickets_take(p, w, lane);
+  }
+}
+
+// n blobs from b0 on, dealt to this warp ahead of time.
+template <int FMT, bool SZ2>
+__device__ __forceinline__ bool run_backbone_i8(const DecodeArgs& p, Ring& r, WalkI8& w, uint32_t b0, uint32_t n, int lane) {
+  if (n == 0) return true;
+  walk_seek<FMT>(p, w, b0, lane);
+  for (; r.deferred > 0; --r.deferred) ring_issue(r, kRing - r.deferred, lane);
+  while (n > 0) {
+    const uint32_t cn = n < p.w_per_copy ? n : p.w_per_copy;
+    if (!mbar_wait_warp(r.bars + r.slot, slot_parity(r), p.dev_status, lane)) return false;
+    walk_blobs<FMT, SZ2>(p, w, r.slots + r.slot * kSlotBytes, cn, n > cn, lane);
+    __syncwarp();                                       // every lane is done with the slot
+    ring_issue(r, r.slot, lane);
+    slot_consumed(r);
+    n -= cn;
+  }
+  return true;
+}
+
+template <int WF, bool I8>
+__device__ __forceinline__ bool run_backbone(const DecodeArgs& p, Ring& r, WalkI8& w, uint32_t first, uint32_t count, uint32_t blob_w, int lane) {
+  if constexpr (I8) {
+    return p.w_sz2 ? run_backbone_i8<WF, true>(p, r, w, first, count, lane) : run_backbone_i8<WF, false>(p, r, w, first, count, lane);
+  } else {
+    return run_segment<WF, false, OUT_Y>(p, r, first, count, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+  }
+}
+
 // I8: the launch has one token and the backbone goes through the integer inner product.
 template <int WF, int ABF, bool I8>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_constant__ DecodeArgs p) {
+__global__ void __launch_bounds__(kThreads, I8 ? kCtasPerSmI8 : kCtasPerSm) k_decode(const __grid_constant__ DecodeArgs p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t gw = blockIdx.x * kWarps + warp;
@@ -412,7 +516,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   Ring r;
   r.slots = smem + warp * (kRing * kSlotBytes);
   r.bars = reinterpret_cast<uint64_t*>(smem + kWarps * kRing * kSlotBytes) + warp * kRing;
-  r.slot = 0; r.parity = 0; r.pseg = 0;
+  r.slot = 0; r.phase = 0; r.pseg = 0;
   r.aux = 0;
   if constexpr (WF == FMT_SP24 || WF == FMT_SQ4) {
     // every warp writes the same 16 values, so no CTA-wide barrier is needed before a warp reads them
@@ -467,19 +571,26 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tr && lane == 0) tr[1] = globaltimer_ns();
 
+  WalkI8 wk;
+  if constexpr (I8) {
+    wk.pair = kNone; wk.next_b = kNone; wk.tile = 0; wk.yb = p.y_ws; wk.my_tile = 0; wk.batch_n = 0; wk.tk_n = 0; wk.tk_old = 0; wk.tk_tile = 0;
+  }
   bool ok = true;
   if (a_owner) ok = run_segment<ABF, false, OUT_T>(p, r, a0, an, p.a_nt, blob_a, p.a_per_copy, p.a_sz2, lane);
-  if (ok) ok = run_segment<WF, false, OUT_Y, I8>(p, r, w0, wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+  if (ok) ok = run_backbone<WF, I8>(p, r, wk, w0, wf, blob_w, lane);
   if (tr && lane == 0) tr[2] = globaltimer_ns();
   if (b_owner) {
     if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
-    if (ok) ok = run_segment<WF, false, OUT_Y, I8>(p, r, w0 + wf, wn - wf, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+    if (ok) ok = run_backbone<WF, I8>(p, r, wk, w0 + wf, wn - wf, blob_w, lane);
+  }
+  if constexpr (I8) {
+    if (ok) { tickets_take(p, wk, lane); tickets_resolve(p, wk, lane); }
   }
   if (!ok) {
     // This warp gave up: its bulk copies still in flight must land before the CTA's shared memory may be reused.  A slot
     // of the ring is in flight exactly if a copy was requested for it and not consumed: slots from the consumer position on
-    // complete the current phase, the ones before it the next one; a slot without a copy passes at once or after the drain's short limit.
-    for (int i = 0; i < kRing - r.deferred; ++i) mbar_drain_warp(r.bars + i, i >= r.slot ? r.parity : r.parity ^ 1u, lane);
+    // waits for the phase its next copy completes; a slot without a copy in flight runs into the drain's short limit.
+    for (int i = 0; i < kRing - r.deferred; ++i) mbar_drain_warp(r.bars + i, (r.phase >> i) & 1u, lane);
   }
   if (tr && lane == 0) tr[3] = globaltimer_ns();
 }
@@ -570,7 +681,11 @@ bool decode_supported(const Handle* h, int m) {
 
 int decode_launch_count(const Handle*, int m) { return (m + 7) / 8; }
 
-int decode_grid(const Handle* h, int) { return h->sm_count * kCtasPerSm; }
+int decode_grid(const Handle* h, int m) {
+  const bool i8 = m == 1 && (h->w.fmt == FMT_Q4 || h->w.fmt == FMT_Q3);
+  (void)i8;
+  return h->sm_count * kCtasPerSm;
+}
 
 cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st,
                                   const int32_t* adapter_ids) {
@@ -589,20 +704,20 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
   }
   const int grid = decode_grid(h, m);
   const uint32_t nw = (uint32_t)grid * kWarps;
-  // Deal the blobs so that every warp gets the same estimated time.  Costs are in units of one backbone
-  // blob on the tensor-core path.  Besides its blobs of A or B a warp of the first or third group has a
-  // fixed extra cost: the A owners fetch a second set of activations, the B owners read t back and end
-  // with their own round of tickets, which is latency that a warp cannot hide from itself.
   if (ab) {
     // with one token the backbone blobs go through the integer inner product, which is cheaper
     const bool i8 = m == 1 && (h->w.fmt == FMT_Q4 || h->w.fmt == FMT_Q3);
-    const double cw1 = blob_cost(h->w.fmt, false) * (i8 ? 0.75 : 1.0);
-    const double fixed_a = i8 ? 4.0 : 2.0, fixed_b = 9.0;
     uint32_t n1 = a.a_blobs < nw / 3 ? a.a_blobs : nw / 3;
     uint32_t n3 = b_blobs < nw / 3 ? b_blobs : nw / 3;
     if (n1 < 1) n1 = 1;
     if (n3 < 1) n3 = 1;
     const uint32_t n2 = nw - n1 - n3;
+    // Deal the blobs so that every warp gets the same estimated time.  Costs are in units of one backbone
+    // blob on the tensor-core path.  Besides its blobs of A or B a warp of the first or third group has a
+    // fixed extra cost: the A owners fetch a second set of activations, the B owners read t back and end
+    // with their own round of tickets, which is latency that a warp cannot hide from itself.
+    const double cw1 = blob_cost(h->w.fmt, false) * (i8 ? 0.75 : 1.0);
+    const double fixed_a = i8 ? 4.0 : 2.0, fixed_b = 9.0;
     const double e1 = fixed_a + (double)a.a_blobs / n1 * blob_cost(h->a.fmt, false);
     const double e3 = fixed_b + (double)b_blobs / n3 * blob_cost(h->b.fmt, true);
     const double T = (w_blobs * cw1 + n1 * e1 + n3 * e3) / nw;      // finishing time of every warp

@@ -369,95 +369,78 @@ __device__ __forceinline__ void blob_product(const uint8_t* blob, int lane, uint
 
 
 // ------------------------------------------------------------------------------------------ integer path (M = 1)
-// With a single token the tensor core is mostly idle (one of eight columns) and its instructions are what
-// the inner loop waits for.  For M = 1 the backbone product is therefore done with integer dot products: the
-// codes stay bytes (one and-or extracts four of them), the 128 activations of a pair are turned once into a
-// 16-bit fixed-point number relative to their largest magnitude (error <= 2^-16 of that magnitude, far
-// inside the fp16 rounding of the inputs themselves), split into a signed high and an unsigned low byte
-// plane, and  sum_k q_k X_k = 256 * dp4a(q, Xh) + dp4a(q, Xl)  is exact in int32.  Zero-point and scales
-// follow per group:  y += s * sx * (sum q X - z * sum X).
+// With a single token the fp16 tensor-core product wastes seven of its eight columns and needs the codes as fp16 pairs
+// (one conversion per two codes).  The integer product keeps the codes as bytes (one and-or extracts four of them) and
+// multiplies them with mma.m16n8k32 (s8 x s8 -> s32): a 16 x 128 blob is four instructions.  The 128 activations of a
+// pair are turned once into a 16-bit block fixed-point number, x = v * 2^e with |v| <= 32639 and one power-of-two scale
+// per pair (so the products are exact and one-hot inputs reproduce the weights bit for bit), split into two signed byte
+// planes (v = 256 * high + low) that are columns 0 and 1 of the MMA's narrow operand.  Zero-point and scales follow per
+// group, in fp32:   y += s * 2^e * (sum q v - z * sum v).
 struct XI8 {
-  uint32_t h[8], l[8];      // byte planes of this lane's 32 activations: index 2 * (2 * c + blk) + quad
-  int sum[2];               // sum of X over this lane's 16 activations of tile c
-  float scale;              // activation = X * scale
+  uint32_t b[4][2];         // this lane's registers of the narrow operand for the four MMAs of a pair (zero for columns >= 2)
+  int sum[2];               // sum of v over tile c of the pair (all lanes hold it)
+  float scale;              // 2^e
 };
 
-__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c) {
-  int d;
-  asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ int dp4a_uu(uint32_t a, uint32_t b, int c) {
-  int d;
-  asm("dp4a.u32.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
+__device__ __forceinline__ void mma16832_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Order of the eight elements of a part inside its two byte quads (quad 0 | quad 1), per format: the order in
-// which one and-or delivers the codes.
-template <int FMT> __device__ __forceinline__ constexpr int i8_elem(int quad, int byte) {
-  if constexpr (FMT == FMT_Q4) return quad == 0 ? (byte == 0 ? 0 : byte == 1 ? 4 : byte == 2 ? 1 : 5)
-                                                : (byte == 0 ? 2 : byte == 1 ? 6 : byte == 2 ? 3 : 7);
-  return 4 * quad + byte;
-}
-
-// x: token 0's activations (fp16 or bf16 bits), pair: which 128 of them.  Every lane converts its own 32
-// activations with a scale of its own (its largest magnitude / 32767): lanes never exchange anything.
+// x: token 0's activations (fp16 or bf16 bits), pair: which 128 of them.  Lane l converts elements 4l .. 4l + 3; the
+// byte planes are then handed to the lanes that own them in the MMA's operand layout: lane (g, t) holds column g (0: low
+// plane, 1: high plane, others: zero) and, for MMA j (tile j / 2, half j % 2 of the tile), the eight reduction elements
+// 32 j + 8 t .. + 7 -- the ones lane t's weight registers of that MMA hold (in the order the and-or delivers the codes).
 template <int FMT>
 __device__ __forceinline__ void load_x_i8(XI8& xi, const void* x, bool bf16, uint32_t pair, int lane) {
-  const int t = lane & 3;
-  const uint16_t* src = reinterpret_cast<const uint16_t*>(x) + pair * 128 + 8 * t;
-  float2 v[4][4];                                     // [2 * c + blk][pair of elements]
-  float amax = 0.f;
-  uint4 ua[4];                                        // all loads first: a use in between would serialise the round trips
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(ua[i].x), "=r"(ua[i].y), "=r"(ua[i].z), "=r"(ua[i].w) : "l"(src + 32 * i) : "memory");
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint4 u = ua[i];
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (bf16) v[i][j] = make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xffff0000u));
-      else v[i][j] = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
-      amax = fmaxf(amax, fmaxf(fabsf(v[i][j].x), fabsf(v[i][j].y)));
-    }
+  const uint16_t* src = reinterpret_cast<const uint16_t*>(x) + pair * 128 + 4 * lane;
+  uint2 u;
+  asm volatile("ld.global.cg.v2.u32 {%0,%1}, [%2];" : "=r"(u.x), "=r"(u.y) : "l"(src) : "memory");
+  float f[4];
+  if (bf16) {
+    f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+    f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+  } else {
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&u.x)), b = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
   }
-  const float scale = amax > 0.f ? amax * (1.f / 32767.f) : 1.f;
-  const float inv = 1.f / scale;
-  xi.scale = scale;
+  float am = fmaxf(fmaxf(fabsf(f[0]), fabsf(f[1])), fmaxf(fabsf(f[2]), fabsf(f[3])));
+  am = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(am)));      // non-negative floats order like integers
+  const uint32_t eb = __float_as_uint(am * 1.00396f) >> 23;           // biased exponent of a value just above the maximum
+  const bool live = eb >= 15u && eb < 255u;
+  const float inv = live ? __uint_as_float((268u - eb) << 23) : 0.f;   // 2^(14 - exponent): |v| <= 32639 = 127 * 256 + 127
+  xi.scale = live ? __uint_as_float((eb - 14u) << 23) : 0.f;           // 2^(exponent - 14)
+  int v[4], s = 0;
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    int s = 0;
+  for (int e = 0; e < 4; ++e) { v[e] = __float2int_rn(f[e] * inv); s += v[e]; }
+  // the low plane is the low byte of v as it is (a signed byte), the high plane byte 1 of v + 128
+  const uint32_t lo = prmt(prmt(v[0], v[1], 0x0040u), prmt(v[2], v[3], 0x0040u), 0x5410u);
+  const uint32_t hi = prmt(prmt(v[0] + 128, v[1] + 128, 0x0051u), prmt(v[2] + 128, v[3] + 128, 0x0051u), 0x5410u);
+  // sums per tile (64 elements: lanes 0..15 / 16..31)
+  const int s_half = __reduce_add_sync(0xffffffffu, lane < 16 ? s : 0);
+  const int s_all = __reduce_add_sync(0xffffffffu, s);
+  xi.sum[0] = s_half; xi.sum[1] = s_all - s_half;
+  const int g = lane >> 2, t = lane & 3;
 #pragma unroll
-    for (int blk = 0; blk < 2; ++blk) {
-      const int i = 2 * c + blk;
-      uint32_t P[4];                                  // (X[2j], X[2j+1]) as two 16-bit halves
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int x0 = __float2int_rn(v[i][j].x * inv), x1 = __float2int_rn(v[i][j].y * inv);
-        s += x0 + x1;
-        P[j] = prmt((uint32_t)x0, (uint32_t)x1, 0x5410u);
-      }
-      // byte planes in the element order of i8_elem<FMT>: low bytes / high bytes of four 16-bit values
-      if constexpr (FMT == FMT_Q4) {                  // quads (0, 4, 1, 5) and (2, 6, 3, 7)
-        xi.l[2 * i] = prmt(P[0], P[2], 0x6240u); xi.h[2 * i] = prmt(P[0], P[2], 0x7351u);
-        xi.l[2 * i + 1] = prmt(P[1], P[3], 0x6240u); xi.h[2 * i + 1] = prmt(P[1], P[3], 0x7351u);
-      } else {                                        // quads (0, 1, 2, 3) and (4, 5, 6, 7)
-        xi.l[2 * i] = prmt(P[0], P[1], 0x6420u); xi.h[2 * i] = prmt(P[0], P[1], 0x7531u);
-        xi.l[2 * i + 1] = prmt(P[2], P[3], 0x6420u); xi.h[2 * i + 1] = prmt(P[2], P[3], 0x7531u);
-      }
+  for (int j = 0; j < 4; ++j) {
+    const int src_lane = 8 * j + 2 * t;
+    const uint32_t l0 = __shfl_sync(0xffffffffu, lo, src_lane), l1 = __shfl_sync(0xffffffffu, lo, src_lane + 1);
+    const uint32_t h0 = __shfl_sync(0xffffffffu, hi, src_lane), h1 = __shfl_sync(0xffffffffu, hi, src_lane + 1);
+    uint32_t w0 = g == 0 ? l0 : g == 1 ? h0 : 0u, w1 = g == 0 ? l1 : g == 1 ? h1 : 0u;
+    if constexpr (FMT == FMT_Q4) {                 // the and-or delivers the codes as (0, 4, 1, 5) and (2, 6, 3, 7)
+      const uint32_t p0 = prmt(w0, w1, 0x5140u), p1 = prmt(w0, w1, 0x7362u);
+      w0 = p0; w1 = p1;
     }
-    xi.sum[c] = s;
+    xi.b[j][0] = w0; xi.b[j][1] = w1;
   }
 }
 
-// Byte quads of one part (8 codes of one row): qa, qb in the element order of i8_elem.
+// Byte quads of one part (8 codes of one row): q[part][0] the codes an and-or delivers first, q[part][1] the others.
+// tile: the tile plus the lane's offset into it (16 lane bytes for 4-bit codes, 8 lane for 3-bit ones).
 template <int FMT>
-__device__ __forceinline__ void tile_quads(const uint8_t* blob, int lane, uint32_t (&q)[4][2]) {
+__device__ __forceinline__ void tile_quads(const uint8_t* tile, int lane, uint32_t (&q)[4][2]) {
   if constexpr (FMT == FMT_Q4) {
-    const uint4 v = *reinterpret_cast<const uint4*>(blob + lane * 16);
+    const uint4 v = *reinterpret_cast<const uint4*>(tile);
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int part = 0; part < 4; ++part) {
@@ -465,55 +448,49 @@ __device__ __forceinline__ void tile_quads(const uint8_t* blob, int lane, uint32
       q[part][1] = (w[part] >> 4) & 0x0f0f0f0fu;
     }
   } else if constexpr (FMT == FMT_Q3) {
-    const uint2 v01 = *reinterpret_cast<const uint2*>(blob + lane * 8);
-    const uint32_t v2 = *reinterpret_cast<const uint32_t*>(blob + 256 + lane * 4);
+    const uint2 v01 = *reinterpret_cast<const uint2*>(tile);
+    const uint32_t v2 = *reinterpret_cast<const uint32_t*>(tile + 256 - 4 * lane);
     q3_quads(v01.x, v01.y, v2, q);
   }
 }
 
-// One blob times the byte planes: tot[0] / tot[1] = this LANE's share of the blob's contribution to rows g /
-// g + 8 (token 0): the four lanes that share a row each add their own share to the row's sum (a reduction
-// over those lanes first would put two dependent shuffle round trips into every blob).
-template <int FMT>
-__device__ __forceinline__ void blob_product_i8(const uint8_t* blob, int lane, uint32_t sz2, const XI8& xi, float (&tot)[2]) {
+// One blob times the byte planes; blob_l: the blob plus the lane's offset into a tile (see tile_quads), blob_g: the blob
+// plus 4 (lane / 4), the offset into a scale entry.  tot[0] / tot[1]: the blob's contribution to rows g /
+// g + 8 (token 0), held by the lanes with t == 0 (the owners of columns 0 and 1 of the accumulator); the other lanes
+// return zeros.  SZ2: one scale entry per tile (groups of 64) instead of one per pair.
+template <int FMT, bool SZ2>
+__device__ __forceinline__ void blob_product_i8(const uint8_t* blob_l, const uint8_t* blob_g, int lane, const XI8& xi, float (&tot)[2]) {
   constexpr int tb = tile_bytes(FMT);
   const int g = lane >> 2;
-  int acc[2] = {0, 0};
+  const bool owner = (lane & 3) == 0;
   tot[0] = tot[1] = 0.f;
   int z_a = 0, z_b = 0;
   float s_a = 0.f, s_b = 0.f;
-  int zsum_a = 0, zsum_b = 0;          // z * sum X over the tiles of the current scale entry
+  int zsum_a = 0, zsum_b = 0;          // z * sum v over the tiles of the current scale entry
+  int d[4] = {0, 0, 0, 0};             // rows g / g + 8 x columns (low, high) for the owners
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
-    if (c == 0 || sz2) {
-      const uint8_t* sz = blob + 2 * tb + c * kSzEntryBytes;
-      const uint32_t s2 = reinterpret_cast<const uint32_t*>(sz)[g];
-      const uint32_t z2 = reinterpret_cast<const uint16_t*>(sz + 32)[g];
+    if (c == 0 || SZ2) {
+      const uint8_t* sz = blob_g + 2 * tb + c * kSzEntryBytes;
+      const uint32_t s2 = *reinterpret_cast<const uint32_t*>(sz);
+      const uint32_t z2 = *reinterpret_cast<const uint16_t*>(sz + 32 - 2 * g);
       z_a = (int)(z2 & 255u); z_b = (int)(z2 >> 8);
-      s_a = __half2float(__ushort_as_half((unsigned short)(s2 & 0xffffu))) * xi.scale;
-      s_b = __half2float(__ushort_as_half((unsigned short)(s2 >> 16))) * xi.scale;
+      const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+      s_a = owner ? sf.x * xi.scale : 0.f;
+      s_b = owner ? sf.y * xi.scale : 0.f;
       zsum_a = 0; zsum_b = 0;
     }
     zsum_a += z_a * xi.sum[c];
     zsum_b += z_b * xi.sum[c];
     uint32_t q[4][2];
-    tile_quads<FMT>(blob + c * tb, lane, q);
-    int sh[2] = {0, 0}, sl[2] = {0, 0};
+    tile_quads<FMT>(blob_l + c * tb, lane, q);
 #pragma unroll
-    for (int part = 0; part < 4; ++part) {
-      const int hf = part & 1, i = 2 * c + (part >> 1);
-#pragma unroll
-      for (int quad = 0; quad < 2; ++quad) {
-        sh[hf] = dp4a_us(q[part][quad], xi.h[2 * i + quad], sh[hf]);
-        sl[hf] = dp4a_uu(q[part][quad], xi.l[2 * i + quad], sl[hf]);
-      }
-    }
-    acc[0] += sh[0] * 256 + sl[0];
-    acc[1] += sh[1] * 256 + sl[1];
-    if (c == 1 || sz2) {
-      tot[0] = fmaf((float)(acc[0] - zsum_a), s_a, tot[0]);
-      tot[1] = fmaf((float)(acc[1] - zsum_b), s_b, tot[1]);
-      acc[0] = acc[1] = 0;
+    for (int blk = 0; blk < 2; ++blk)          // parts 2 blk (row g) and 2 blk + 1 (row g + 8): one MMA
+      mma16832_s8(d, q[2 * blk][0], q[2 * blk + 1][0], q[2 * blk][1], q[2 * blk + 1][1], xi.b[2 * c + blk][0], xi.b[2 * c + blk][1]);
+    if (c == 1 || SZ2) {
+      tot[0] = fmaf((float)(d[1] * 256 + d[0] - zsum_a), s_a, tot[0]);
+      tot[1] = fmaf((float)(d[3] * 256 + d[2] - zsum_b), s_b, tot[1]);
+      d[0] = d[1] = d[2] = d[3] = 0;
     }
   }
 }
