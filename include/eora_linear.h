@@ -208,11 +208,11 @@ int eora_linear_last_device_status(eora_linear_t h);
 
 /*
  * Diagnostics.  eora_linear_decode_grid: how many CTAs a decode forward(m) launches (0 if m is
- * not served by the decode family); each CTA has four warps.  eora_linear_set_trace: give the
+ * not served by the decode family); each CTA has sixteen warps.  eora_linear_set_trace: give the
  * handle a caller-owned device buffer (or NULL to switch tracing off).  A decode forward then
  * records four %globaltimer values (nanoseconds) per warp, at uint64 index
- * 4 * (4 * cta + warp) + k:  k = 0 kernel entry, 1 dependency wait over, 2 first share of the
- * backbone done, 3 all work of the warp done; the buffer must hold 16 * grid values.  A prefill
+ * 4 * (16 * cta + warp) + k:  k = 0 kernel entry, 1 dependency wait over, 2 first share of the
+ * backbone done, 3 all work of the warp done; the buffer must hold 64 * grid values.  A prefill
  * forward records, for CTA (0, 0) only, four clock64 values per 64-element k-block (token tile
  * requested / first weight tile dequantised / token tile seen by the MMA warp / MMAs issued) at
  * index 4 * k_block + k, k_block < nkb = d_in / 64 + (rank padded to 128) / 64, and one more row at

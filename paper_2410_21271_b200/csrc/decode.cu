@@ -16,8 +16,8 @@
 //     then the rest of their share of W,
 //   * the warps in between take backbone blobs only.
 // The only wait in the kernel is the one before the B share: all of A must have been added to t.  A
-// owners never wait, and they sit in the CTAs with the lowest indices, which are dispatched first, so a
-// waiting warp never holds the slot of a CTA it is waiting for.  The wait is bounded like every other.
+// owners never wait, and they sit in the first half of the CTAs, which are dispatched first and hold no B
+// owner, so a waiting warp never holds the place of a CTA it is waiting for.  The wait is bounded like every other.
 //
 // Completion.  Every blob of W or B that has been added to y_ws bumps the ticket of its row tile; the
 // warp that brings a ticket to its final count converts the 16 x m sums to the output type, writes Y and
@@ -33,13 +33,14 @@ namespace eora {
 namespace {
 using namespace dec;
 
-constexpr int kWarps = 4;
+// One CTA of sixteen warps per SM.  The warps of a CTA start together; with several smaller CTAs per SM the ones that
+// are placed last ran a fifth slower than the first (the scheduler prefers the older warps) and ended the kernel late.
+constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
-constexpr int kCtasPerSm = 4;
-constexpr int kCtasPerSmI8 = 4;            // the single-token integer kernels need fewer registers
+constexpr int kCtasPerSm = 1;
 constexpr int kRing = 2;                  // bulk copies in flight per warp
 constexpr int kSlotBytes = 4352;          // one ring slot = one bulk copy (a run of whole blobs)
-constexpr int kBarBytes = 128;            // kWarps * kRing mbarriers
+constexpr int kBarBytes = 512;            // kWarps * kRing mbarriers
 constexpr int kSmemBytes = kWarps * kRing * kSlotBytes + kBarBytes + kSp24LutBytes;
 
 enum { CNT_A_DONE = 0, CNT_TILES_DONE = 1, CNT_TICKET0 = 2 };
@@ -505,12 +506,26 @@ __device__ __forceinline__ bool run_backbone(const DecodeArgs& p, Ring& r, WalkI
 
 // I8: the launch has one token and the backbone goes through the integer inner product.
 template <int WF, int ABF, bool I8>
-__global__ void __launch_bounds__(kThreads, I8 ? kCtasPerSmI8 : kCtasPerSm) k_decode(const __grid_constant__ DecodeArgs p) {
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_constant__ DecodeArgs p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t gw = blockIdx.x * kWarps + warp;
+  // Position in the deal.  Neighbours in the deal sit on different SMs, so that the few warps that hold A (whose sums
+  // everybody's B share waits for) work in parallel on many SMs: the A owners are dealt warp by warp over the first
+  // half of the CTAs, the B owners over the second half, and the warps left over are numbered after them.  No CTA
+  // holds both kinds: the CTAs with A owners are dispatched first and never wait, so a waiting warp never holds the
+  // place of a CTA that it is waiting for.
+  uint32_t gw;
+  {
+    const uint32_t ca = gridDim.x / 2, cb = gridDim.x - ca, n3 = gridDim.x * kWarps - p.n12;
+    if (blockIdx.x < ca) {
+      gw = warp * ca + blockIdx.x;                                    // < n1: an A owner
+    } else {
+      const uint32_t rid = warp * cb + (blockIdx.x - ca);
+      gw = rid < n3 ? p.n12 + rid : p.n1 + (kWarps * ca - p.n1) + (rid - n3);
+    }
+  }
   asm volatile("griddepcontrol.launch_dependents;");
-  unsigned long long* tr = p.trace ? p.trace + (size_t)gw * 4 : nullptr;
+  unsigned long long* tr = p.trace ? p.trace + (size_t)(blockIdx.x * kWarps + warp) * 4 : nullptr;
   if (tr && lane == 0) tr[0] = globaltimer_ns();
 
   Ring r;
@@ -673,6 +688,7 @@ cudaError_t launch_wait_selftest(const Handle* h, cudaStream_t st) {
 
 bool decode_supported(const Handle* h, int m) {
   if (m < 1 || m > 64) return false;
+  if (h->sm_count < 2) return false;
   if (h->w.fmt != FMT_Q4 && h->w.fmt != FMT_Q3 && h->w.fmt != FMT_SP24 && h->w.fmt != FMT_SQ4) return false;
   if (h->w.blob > kSlotBytes) return false;
   if (h->cfg.rank > 0 && (h->a.blob > kSlotBytes || h->b.blob > kSlotBytes)) return false;
@@ -711,6 +727,9 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
     uint32_t n3 = b_blobs < nw / 3 ? b_blobs : nw / 3;
     if (n1 < 1) n1 = 1;
     if (n3 < 1) n3 = 1;
+    // the A owners sit in the first half of the CTAs, the B owners in the second (see the kernel)
+    if (n1 > (uint32_t)(grid / 2) * kWarps) n1 = (uint32_t)(grid / 2) * kWarps;
+    if (n3 > (uint32_t)(grid - grid / 2) * kWarps) n3 = (uint32_t)(grid - grid / 2) * kWarps;
     const uint32_t n2 = nw - n1 - n3;
     // Deal the blobs so that every warp gets the same estimated time.  Costs are in units of one backbone
     // blob on the tensor-core path.  Besides its blobs of A or B a warp of the first or third group has a

@@ -511,7 +511,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
             for (int i = nl; i < pieces; i += 128) {
               const int tok = i >> row_sh, piece = i & ((1 << row_sh) - 1);
               const int row = m0 + c0 + tok, col = n0 + hh * BN_W + piece * (16 / esz);
-              if (row < p.m && col < n_end) {
+              if (c0 + tok < bt && row < p.m && col < n_end) {     // a chunk may reach past the tile's tokens
                 const uint4 val = *reinterpret_cast<const uint4*>(tbuf + (size_t)tok * BN_W * esz + piece * 16);
                 *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + ((int64_t)row * p.ld_out + col) * esz) = val;
               }
