@@ -461,7 +461,7 @@ __device__ __forceinline__ void walk_blobs(const DecodeArgs& p, WalkI8& w, const
     uint32_t run = min(left, min(nt - w.tile, 32u - w.batch_n));
     if ((uint32_t)lane - w.batch_n < run) w.my_tile = w.tile + ((uint32_t)lane - w.batch_n);
     left -= run; w.tile += run; w.batch_n += run;
-#pragma unroll 4
+#pragma unroll 2
     for (; run > 0; --run, bl += blob_b, bg += blob_b, w.yb += 16) {
       float t2[2];
       blob_product_i8<FMT, SZ2>(bl, bg, lane, w.xi, t2);
