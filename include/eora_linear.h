@@ -124,10 +124,12 @@ int eora_linear_create(const eora_linear_config* cfg, const eora_linear_weights*
  * Y[M][d_out] = X[M][d_in] . deq(Wq) + (X . A) . B   (Eq. 4), enqueued on `stream`.
  * x, y: device pointers, row-major, 16-byte aligned, caller-owned; 1 <= m <= max_m; m == 0 is a
  * no-op returning EORA_OK.  Never synchronises and never allocates.  The current device must be the one
- * the handle was created on (EORA_ERR_UNSUPPORTED otherwise).  M <= 16 runs the decode
- * kernel family (one streaming pass over the weights per eight tokens), M > 64 the tensor-core
- * (tcgen05) prefill family, and in between whichever is cheaper for the layer: the prefill family
- * once ceil(M / 8) * 30 exceeds d_in / 64 (eora_linear_path reports the choice).  Asynchronous device-side
+ * the handle was created on (EORA_ERR_UNSUPPORTED otherwise).  M <= 8 runs the decode
+ * kernel family (one streaming pass over the weights), M > 8 the tensor-core (tcgen05) family, which
+ * for up to 64 tokens splits the reduction axis of a tile over several thread blocks (fp32 sums in the
+ * handle's scratch, restored by the block that completes a tile); handles that the tensor-core family
+ * does not serve run ceil(M / 8) decode passes up to M = 64 (eora_linear_path reports the choice).
+ * Asynchronous device-side
  * problems (a bounded wait that ran out) are latched in a status word readable with
  * eora_linear_last_device_status after the caller has synchronised.
  */
@@ -140,9 +142,11 @@ int eora_linear_forward(eora_linear_t h, const void* x, int32_t m, void* y, void
  * arrays of configs and weights; they must agree in everything but d_out (same d_in, rank, formats,
  * groups, dtypes, max_m <= 64, policy AUTO; any backbone format).  eora_linear_forward_fused computes
  *     ys[i][M][d_out_i] = X . deq(Wq_i) + (X . A_i) . B_i      for every layer i
- * with ONE kernel launch per eight tokens: X is read once, and the launch latency is paid once.
+ * with ONE kernel launch for up to eight tokens: X is read once, and the launch latency is paid once.
  * ys: host array of n_layers device pointers (16-byte aligned, caller-owned).  The handle serves
- * the decode family only (M <= 64); eora_linear_forward / _forward_host on it return
+ * M <= 64: the decode family, and for 9..64 tokens the tensor-core family (two launches, the first for
+ * t = X . A of all layers) if every d_out_i is a multiple of 128, else ceil(M / 8) decode passes;
+ * eora_linear_forward / _forward_host on it return
  * EORA_ERR_UNSUPPORTED, everything else (destroy, launches, last_device_status, dump of the
  * stacked matrices) works as for a plain handle.  Errors as for create / forward.
  */

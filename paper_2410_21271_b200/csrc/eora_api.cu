@@ -74,12 +74,12 @@ int y_elem_bytes(int y_dtype) { return y_dtype == EORA_Y_F32 ? 4 : 2; }
 
 int pick_path(const Handle* h, int m) {
   if (h->cfg.kernel_policy == EORA_POLICY_GENERIC) return EORA_PATH_GENERIC;
-  // The decode family streams the weights once per eight tokens, the tensor-core family walks the d_in / 64
-  // k-blocks of the layer once whatever m is: measured, a decode pass costs about as much as 30 k-blocks, so
-  // from three passes on (m > 16 with d_in = 4096, m > 56 with d_in = 14336) the tensor-core family is faster.
+  // The decode family streams the weights once per eight tokens.  From two passes on (m > 8) one launch of the
+  // tensor-core family is cheaper: for up to 64 tokens it splits the reduction axis over several CTAs per tile, so it
+  // is no longer a chain over all of d_in (measured, 4-bit q-shaped layer, 16 tokens: 23.6 us in two passes, 17 us so).
   if (decode_tc_supported(h, m)) return EORA_PATH_DECODE;   // EORA_POLICY_TMEM_DECODE: one pass over the weights per sixteen tokens
   const bool dec = m <= 64 && decode_supported(h, m), pre = prefill_supported(h, m);
-  if (dec && pre) return ((m + 7) / 8) * 30 > h->cfg.d_in / 64 ? EORA_PATH_PREFILL : EORA_PATH_DECODE;
+  if (dec && pre) return EORA_PATH_PREFILL;
   if (dec) return EORA_PATH_DECODE;
   if (pre) return EORA_PATH_PREFILL;
   return EORA_PATH_GENERIC;
@@ -245,7 +245,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     Carve sc{reinterpret_cast<char*>(h->scratch_mem), 0};
     // t as fp32 for the simple kernels and as fp16 for the tensor-core family: only where those families can be reached
     h->t_gen = sc.take<float>(generic_reachable ? (int64_t)c.max_m * rp * 4 : 256);
-    h->t16 = sc.take<__half>((!fused && c.max_m > 16) ? (int64_t)c.max_m * rp * 2 : 256);
+    h->t16 = sc.take<__half>(c.max_m > 8 ? (int64_t)c.max_m * rp * 2 : 256);
     h->d_t = sc.take<float>(8 * rp * 4);
     h->y_ws = sc.take<float>((int64_t)8 * h->w.n_rows * 4);
     h->counters = sc.take<uint32_t>((int64_t)(h->w.nt + 2) * 4);
@@ -281,7 +281,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     }
   }
   if (e != cudaSuccess) return fail(EORA_ERR_CUDA);
-  if (!fused && prefill_init(h) != cudaSuccess) return fail(EORA_ERR_CUDA);
+  if (prefill_init(h) != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (decode_tc_init(h, s) != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (fused && !decode_supported(h, 1) && !decode_tc_supported(h, 1)) return fail(EORA_ERR_UNSUPPORTED);
   if (cudaStreamSynchronize(s) != cudaSuccess) return fail(EORA_ERR_CUDA);
@@ -453,6 +453,7 @@ int eora_linear_forward_fused(eora_linear_t obj, const void* x, int32_t m, void*
   if (!on_handle_device(h)) return EORA_ERR_UNSUPPORTED;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   if (decode_tc_supported(h, m)) return launch_decode_tc_forward(h, x, m, ys, s) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
+  if (pick_path(h, m) == EORA_PATH_PREFILL) return launch_prefill_forward(h, x, m, ys, s) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
   if (!decode_supported(h, m)) return EORA_ERR_UNSUPPORTED;
   return launch_decode_forward(h, x, m, ys, s) == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
 }
@@ -543,7 +544,7 @@ int eora_linear_forward(eora_linear_t obj, const void* x, int32_t m, void* y, vo
   cudaError_t e;
   void* ys[1] = {y};
   if (p == EORA_PATH_DECODE) e = decode_tc_supported(h, m) ? launch_decode_tc_forward(h, x, m, ys, s) : launch_decode_forward(h, x, m, ys, s);
-  else if (p == EORA_PATH_PREFILL) e = launch_prefill_forward(h, x, m, y, s);
+  else if (p == EORA_PATH_PREFILL) e = launch_prefill_forward(h, x, m, ys, s);
   else e = launch_generic_forward(h, x, m, y, s);
   return e == cudaSuccess ? EORA_OK : EORA_ERR_CUDA;
 }
@@ -589,7 +590,7 @@ int eora_linear_last_device_status(eora_linear_t obj) {
     char* lo = reinterpret_cast<char*>(h->d_t);
     char* hi = reinterpret_cast<char*>(h->dev_status) + 256;
     if (cudaMemset(lo, 0, (size_t)(hi - lo)) != cudaSuccess) return EORA_ERR_CUDA;
-    if (decode_tc_reset(h, nullptr) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return EORA_ERR_CUDA;
+    if (decode_tc_reset(h, nullptr) != cudaSuccess || prefill_reset(h, nullptr) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return EORA_ERR_CUDA;
   }
   return v;
 }

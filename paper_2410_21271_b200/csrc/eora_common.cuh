@@ -253,7 +253,8 @@ cudaError_t decode_tc_reset(const Handle* h, cudaStream_t st);
 bool prefill_supported(const Handle* h, int m);
 cudaError_t prefill_init(Handle* h);
 void prefill_free(Handle* h);
-cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st);
+cudaError_t prefill_reset(Handle* h, cudaStream_t st);   // after a launch that gave up: split-K sums and tickets back to zero
+cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st);
 int prefill_launch_count(const Handle* h, int m);
 
 }  // namespace eora

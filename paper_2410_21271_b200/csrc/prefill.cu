@@ -53,16 +53,41 @@ struct PrefillArgs {
   int nkb_w, nkb_b;  // k-blocks of each part
   int sx, sw;        // stages of the ring (sx == sw: token tiles first, weight tiles from w_off on)
   int w_off;         // byte offset of the weight ring (after sx token tiles of bt*128 bytes)
+  // Few tokens (one token tile): the reduction axis is split over ksplit CTAs per tile (kchunk k-blocks each; the
+  // first one also takes the K-extension).  Each adds its accumulator to ws (fp32, [tokens][ld_ws], zero between
+  // launches) and takes a ticket of its tile; the CTA that takes the last one converts the sums to `out` and puts
+  // ws and the ticket back to zero.  ksplit == 1: the accumulator goes straight to `out`.
+  // Fused layers (stacked along the weight rows, few tokens only): layer i owns rows [sub_row0[i], sub_row0[i + 1]),
+  // writes to outs[i] (leading dimension sub_ld[i]) and takes columns [i * t_sub, (i + 1) * t_sub) of t in the
+  // K-extension.  A plain layer: n_sub = 1, sub_row0 = {0, n_valid}, outs[0] = out.
+  int n_sub;
+  int sub_row0[5];
+  void* outs[4];
+  int sub_ld[4];
+  int t_sub;
+  int ksplit, kchunk;
+  float* ws;
+  int ld_ws;
+  uint32_t* tickets;
   int* dev_status;
   long long* trace;  // optional: for CTA (0,0), 4 clock64() stamps per k-block (token copy requested, W ready, X ready, MMA issued),
                      // then one more row: kernel entry, set-up done, accumulators complete, epilogue done
 };
 
+#define CTRACE(slot) do { if (p.trace) p.trace[1024 + 4 * blockIdx.x + (slot)] = (long long)globaltimer_ns(); } while (0)
 #define PTRACE(it, slot) do { if (p.trace && blockIdx.x == 0 && blockIdx.y == 0) p.trace[(it) * 4 + (slot)] = clock64(); } while (0)
 
 struct PrefillState {
-  __half* x16;       // fp16 copy of a bf16 X, [max_m][d_in]
+  __half* x16;       // fp16 copy of a bf16 X, [max_m][d_in] (bf16 handles only)
+  // split-K workspace of launches with few tokens (see PrefillArgs::ksplit): sums and tickets of the main product
+  // and of t = X.A; one allocation, zero between launches
+  void* split_mem;
+  size_t split_bytes;
+  float* ws_y; float* ws_t;
+  uint32_t* tk_y; uint32_t* tk_t;
 };
+
+constexpr int kThinTokens = 64;        // launches of up to this many tokens may split the reduction axis
 
 // ---------------------------------------------------------------------------------------------- PTX
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int c0, int c1, uint64_t* bar) {
@@ -363,6 +388,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   __shared__ uint32_t tmem_base_s;
   __shared__ uint32_t sp_lut[16];        // 2:4 expansion selectors (2:4 backbones only)
   __shared__ int fail_s;                 // set by an epilogue warp whose bounded wait ran out
+  __shared__ int last_s;                 // split-K: this CTA took its tile's last ticket
   // 1024-byte alignment of the operand tiles (the swizzle pattern is anchored at 1 KB)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
@@ -374,15 +400,24 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   const int big_id = (int)blockIdx.x - p.n_small;
   const int bt = small ? kSmallTile : p.bt;                 // tokens of this CTA's tile (the MMA N)
   const int rows = small ? kSmallTile : p.rows;
-  const int n0 = small ? p.n_split + ((int)blockIdx.x % p.small_x) * kSmallTile : (big_id % p.big_x) * rows;
-  const int m0 = small ? ((int)blockIdx.x / p.small_x) * kSmallTile : (big_id / p.big_x) * bt;
-  const int n_end = small ? p.n_valid : p.n_split;          // this CTA writes columns n0 .. n_end - 1 at most
+  // big tiles: row tile fastest, then the split of the reduction axis, then the token tile
+  const int tile_x = big_id % p.big_x, split = small ? 0 : (big_id / p.big_x) % p.ksplit, tile_y = big_id / (p.big_x * p.ksplit);
+  const int n0 = small ? p.n_split + ((int)blockIdx.x % p.small_x) * kSmallTile : tile_x * rows;
+  const int m0 = small ? ((int)blockIdx.x / p.small_x) * kSmallTile : tile_y * bt;
+  int sub = 0;                                              // fused layers: whose rows these are (tiles never straddle)
+#pragma unroll
+  for (int i = 1; i < 4; ++i)
+    if (i < p.n_sub && n0 >= p.sub_row0[i]) sub = i;
+  const int n_end = min(small ? p.n_valid : p.n_split, p.sub_row0[sub + 1]);   // this CTA writes columns n0 .. n_end - 1 at most
+  void* const out_p = p.outs[sub];
+  const int ld_o = p.sub_ld[sub], col0 = p.sub_row0[sub];   // output column of weight row n: n - col0
   const int nh = (rows > BN_W && n_end - n0 > BN_W) ? 2 : 1;   // 128-row halves of this CTA that hold real rows
   const CUtensorMap* map_x = small ? &tm_x_small : &tm_x;
   const CUtensorMap* map_t = small ? &tm_t_small : &tm_t;
-  const int kw_lo = 0, kw_hi = p.nkb_w;
-  const int nkw = p.nkb_w;
-  const int nkb = nkw + p.nkb_b;
+  const int kw_lo = split * p.kchunk, kw_hi = min(p.nkb_w, kw_lo + p.kchunk);
+  const int nkw = kw_hi - kw_lo;
+  const int nkb_ext = split == 0 ? p.nkb_b : 0;             // the K-extension goes with the first split
+  const int nkb = nkw + nkb_ext;
   const uint32_t xbytes = (uint32_t)bt * 128;               // bytes of a token tile; the ring's slots are p.bt * 128 apart
   const uint32_t xslot = (uint32_t)p.bt * 128;
 
@@ -392,6 +427,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
   const uint32_t lut = smem_u32(sp_lut);
   if (threadIdx.x == 0) {
     PTRACE(nkb, 0);
+    CTRACE(0);
     fail_s = 0;
     for (int i = 0; i < p.sw; ++i) { mbar_init(full_w + i, 8 * nh + 1); mbar_init(empty_w + i, 1); }
     mbar_init(&acc_full, 1);
@@ -422,7 +458,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
         } else {
           // t comes from the previous launch, which may still be running: everything up to here overlapped with it
           if (it == nkw) asm volatile("griddepcontrol.wait;" ::: "memory");
-          tma_load_2d(xt, map_t, (it - nkw) * BK, m0, full_w + s);
+          tma_load_2d(xt, map_t, (it - nkw) * BK + sub * p.t_sub, m0, full_w + s);
         }
         if (++s == p.sw) { s = 0; ++wrap; }
       }
@@ -464,7 +500,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       // two halves: one row tile per warp; one half: two warps per row tile, alternating k-blocks
       const int kstep = 3 - nh, tile = nh == 2 ? dw : (dw & 7), kphase = nh == 2 ? 0 : (dw >> 3);
       ok = dequant_part<WF>(p.w, n0, kw_lo, kw_hi, 0, tile, kphase, kstep, lane, smem, p, full_w, empty_w, lut);
-      if (ok && p.nkb_b > 0) ok = dequant_part<BF>(p.b, n0, 0, p.nkb_b, nkw, tile, kphase, kstep, lane, smem, p, full_w, empty_w, lut);
+      if (ok && nkb_ext > 0) ok = dequant_part<BF>(p.b, n0, 0, nkb_ext, nkw, tile, kphase, kstep, lane, smem, p, full_w, empty_w, lut);
     }
     {
       // Epilogue: all sixteen warps, as four groups of four.  A warp can read the quarter of the TMEM lanes
@@ -476,12 +512,79 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
       asm volatile("bar.sync 1, 512;" ::: "memory");
       ok = *reinterpret_cast<volatile int*>(&fail_s) == 0;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      if (dw == 0 && lane == 0) PTRACE(nkb, 2);
+      if (dw == 0 && lane == 0) { PTRACE(nkb, 2); CTRACE(1); }
       const int grp = dw >> 2, lq = dw & 3;
       const int nl = lq * 32 + lane;                     // local weight row inside the half = thread index inside the group
       const int nchunk = (bt + 31) >> 5;
       const uint32_t lane_base = tmem_d + ((uint32_t)(lq * 32) << 16);
-      {
+      if (p.ksplit > 1) {
+        // Split reduction axis: add this CTA's share to the fp32 sums (a thread holds one column n for the 32 tokens of a
+        // chunk; a warp's 32 lanes add 128 contiguous bytes per token), then one ticket per CTA.
+        const int tok_valid = min(bt, p.m - m0);
+        if (ok) {
+          float* wsb = p.ws + (int64_t)m0 * p.ld_ws;
+          for (int hh = 0; hh < nh; ++hh) {
+            const int col = n0 + hh * BN_W + nl;
+            for (int cc = 0; cc < nchunk; ++cc) {
+              if (((hh * nchunk + cc) & 3) != grp) continue;
+              const int c0 = cc * 32;
+              uint32_t v[32];
+              tmem_ld32(lane_base + hh * 256 + (uint32_t)c0, v);
+              asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+              if (col < n_end) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (c0 + j < tok_valid)
+                    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(wsb + (int64_t)(c0 + j) * p.ld_ws + col), "f"(__uint_as_float(v[j])) : "memory");
+              }
+            }
+          }
+          __threadfence();
+        }
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        if (dw == 0 && lane == 0) {
+          uint32_t old = 0;
+          uint32_t* tk = p.tickets + tile_y * p.big_x + tile_x;
+          if (ok) asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(tk), "r"(1u) : "memory");
+          last_s = (ok && old + 1u == (uint32_t)p.ksplit) ? 1 : 0;
+          if (last_s) *tk = 0u;                          // nobody else touches the ticket any more
+        }
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        if (*reinterpret_cast<volatile int*>(&last_s)) {
+          __threadfence();
+          // every share is in: sums -> output type, one token row per warp and step, 32 columns per instruction
+          // (all loads of a warp's share first: one round trip to L2, not one per row)
+          const int ncols = min(rows, n_end - n0);
+          const int esz = p.out_dtype == EORA_Y_F32 ? 4 : 2;
+          constexpr int kTok = (kThinTokens + kDqWarps - 1) / kDqWarps, kCol = 2 * BN_W / 32;
+          float f[kTok][kCol];
+#pragma unroll
+          for (int i = 0; i < kTok; ++i) {
+            const int tok = dw + i * kDqWarps;
+#pragma unroll
+            for (int k = 0; k < kCol; ++k) {
+              const int c = lane + 32 * k;
+              f[i][k] = (tok < tok_valid && c < ncols) ? __ldcg(p.ws + (int64_t)(m0 + tok) * p.ld_ws + n0 + c) : 0.f;
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < kTok; ++i) {
+            const int tok = dw + i * kDqWarps;
+            if (tok >= tok_valid) continue;
+            float* src = p.ws + (int64_t)(m0 + tok) * p.ld_ws + n0;
+            uint8_t* dst = reinterpret_cast<uint8_t*>(out_p) + ((int64_t)(m0 + tok) * ld_o + n0 - col0) * esz;
+#pragma unroll
+            for (int k = 0; k < kCol; ++k) {
+              const int c = lane + 32 * k;
+              if (c >= ncols) continue;
+              src[c] = 0.f;
+              if (p.out_dtype == EORA_Y_F32) reinterpret_cast<float*>(dst)[c] = f[i][k];
+              else if (p.out_dtype == EORA_Y_F16) reinterpret_cast<__half*>(dst)[c] = __float2half_rn(f[i][k]);
+              else reinterpret_cast<__nv_bfloat16*>(dst)[c] = __float2bfloat16_rn(f[i][k]);
+            }
+          }
+        }
+      } else {
         // A chunk goes through shared memory as [32 tokens][128 n] so that the global stores are 16-byte
         // pieces of rows of Y.  The rings are free by now (every MMA has completed).  Each group has two
         // buffers and alternates: a buffer is rewritten two chunks later, after a barrier that every thread of
@@ -513,13 +616,13 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_prefill(const __grid_constant_
               const int row = m0 + c0 + tok, col = n0 + hh * BN_W + piece * (16 / esz);
               if (c0 + tok < bt && row < p.m && col < n_end) {     // a chunk may reach past the tile's tokens
                 const uint4 val = *reinterpret_cast<const uint4*>(tbuf + (size_t)tok * BN_W * esz + piece * 16);
-                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.out) + ((int64_t)row * p.ld_out + col) * esz) = val;
+                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(out_p) + ((int64_t)row * ld_o + col - col0) * esz) = val;
               }
             }
           }
         }
       }
-      if (dw == 0 && lane == 0) PTRACE(nkb, 3);
+      if (dw == 0 && lane == 0) { PTRACE(nkb, 3); CTRACE(2); }
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -649,8 +752,13 @@ int token_tile(int m) {                // the MMA N: a multiple of 16 up to 256
 }  // namespace
 
 bool prefill_supported(const Handle* h, int m) {
-  if (m <= 16) return false;             // up to two decode passes are always cheaper
-  if (h->n_sub > 1 || h->multi) return false;   // fused layers and per-token adapters: decode family only
+  if (m <= 8) return false;              // one decode pass is always cheaper
+  if (h->multi) return false;            // per-token adapters: decode family only
+  if (h->n_sub > 1) {                    // fused layers: launches of few tokens only, tiles of 128 rows must not straddle two layers
+    if (m > kThinTokens) return false;
+    for (int i = 0; i < h->n_sub; ++i)
+      if (h->sub_dout[i] % BN_W) return false;
+  }
   if (h->w.group % 64) return false;
   return encode_fn() != nullptr;
 }
@@ -661,11 +769,31 @@ int prefill_launch_count(const Handle* h, int) {
 
 cudaError_t prefill_init(Handle* h) {
   h->prefill_state = nullptr;
-  if (h->cfg.max_m <= 16 || h->cfg.x_dtype != EORA_X_BF16) return cudaSuccess;
+  if (h->cfg.max_m <= 8) return cudaSuccess;
   PrefillState* ps = new PrefillState();
-  cudaError_t e = cudaMalloc(&ps->x16, (size_t)h->cfg.max_m * h->cfg.d_in * 2);
-  if (e != cudaSuccess) { delete ps; return e; }
+  *ps = PrefillState();
+  cudaError_t e = cudaSuccess;
+  if (h->cfg.x_dtype == EORA_X_BF16) e = cudaMalloc(&ps->x16, (size_t)h->cfg.max_m * h->cfg.d_in * 2);
+  if (e == cudaSuccess) {
+    // split-K sums and tickets for launches of up to kThinTokens tokens
+    const size_t tok = (size_t)(h->cfg.max_m < kThinTokens ? h->cfg.max_m : kThinTokens);
+    const size_t rp = (size_t)(h->cfg.rank > 0 ? h->t_cols : 0);
+    const size_t n_all = (size_t)(h->n_sub > 1 ? 16 * h->sub_tile0[h->n_sub] : h->cfg.d_out);
+    const size_t y_b = tok * n_all * 4, t_b = tok * rp * 4;
+    const size_t tky_b = ((n_all + BN_W - 1) / BN_W) * 4, tkt_b = ((rp + BN_W - 1) / BN_W) * 4;
+    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
+    ps->split_bytes = up(y_b) + up(t_b) + up(tky_b) + up(tkt_b) + 256;
+    e = cudaMalloc(&ps->split_mem, ps->split_bytes);
+    if (e == cudaSuccess) e = cudaMemset(ps->split_mem, 0, ps->split_bytes);
+    char* q = reinterpret_cast<char*>(ps->split_mem);
+    ps->ws_y = reinterpret_cast<float*>(q); q += up(y_b);
+    ps->ws_t = reinterpret_cast<float*>(q); q += up(t_b);
+    ps->tk_y = reinterpret_cast<uint32_t*>(q); q += up(tky_b);
+    ps->tk_t = reinterpret_cast<uint32_t*>(q);
+  }
+  if (e != cudaSuccess) { cudaFree(ps->x16); cudaFree(ps->split_mem); delete ps; return e; }
   h->prefill_state = ps;
+  h->scratch_bytes += (int64_t)ps->split_bytes;
   return cudaSuccess;
 }
 
@@ -673,16 +801,33 @@ void prefill_free(Handle* h) {
   PrefillState* ps = reinterpret_cast<PrefillState*>(h->prefill_state);
   if (!ps) return;
   cudaFree(ps->x16);
+  cudaFree(ps->split_mem);
   delete ps;
   h->prefill_state = nullptr;
 }
 
-cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* y, cudaStream_t st) {
+// After a launch that gave up: sums and tickets back to zero.
+cudaError_t prefill_reset(Handle* h, cudaStream_t st) {
+  PrefillState* ps = reinterpret_cast<PrefillState*>(h->prefill_state);
+  if (!ps || !ps->split_mem) return cudaSuccess;
+  return cudaMemsetAsync(ps->split_mem, 0, ps->split_bytes, st);
+}
+
+// How many CTAs share a tile's reduction axis in a launch of few tokens: as many as there are SMs for, each with at
+// least min_kb k-blocks (a CTA's set-up and epilogue are worth about eight of them).
+int pick_ksplit(int tiles, int nkb, int sm_count, int min_kb, int cap) {
+  int s = sm_count / (tiles > 0 ? tiles : 1);
+  if (s > nkb / min_kb) s = nkb / min_kb;
+  if (s > cap) s = cap;
+  return s < 1 ? 1 : s;
+}
+
+cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* const* ys, cudaStream_t st) {
   const eora_linear_config& c = h->cfg;
   const void* x16 = x;
   if (c.x_dtype == EORA_X_BF16) {
     PrefillState* ps = reinterpret_cast<PrefillState*>(h->prefill_state);
-    if (!ps) return cudaErrorInvalidValue;
+    if (!ps || !ps->x16) return cudaErrorInvalidValue;
     int64_t n = (int64_t)m * c.d_in;
     int64_t blocks = (n / 8 + 255) / 256;
     if (blocks > h->sm_count * 8) blocks = h->sm_count * 8;
@@ -690,11 +835,13 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     x16 = ps->x16;
   }
   const int bt = token_tile(m);
+  PrefillState* pst = reinterpret_cast<PrefillState*>(h->prefill_state);
+  const bool thin = m <= kThinTokens && pst && pst->split_mem;      // one token tile: split the reduction axis instead
   CUtensorMap tm_x, tm_t;
   if (!make_map(&tm_x, x16, m, c.d_in, c.d_in, bt)) return cudaErrorInvalidValue;
   const bool ab = c.rank > 0;
   if (ab) {
-    if (!make_map(&tm_t, h->t16, m, h->r_pad, h->r_pad, bt)) return cudaErrorInvalidValue;
+    if (!make_map(&tm_t, h->t16, m, h->t_cols, h->t_cols, bt)) return cudaErrorInvalidValue;
     // launch 1: t = X.A with A as the weight (rows = r_pad), written as fp16.  It is a small product (a few
     // CTAs with token tiles of 128), and the main launch behind it starts at once (programmatic dependent
     // launch) on the other SMs: the main product needs t only for its last k-blocks and waits for this
@@ -702,29 +849,42 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     // Its tile: 128 rows and 128 tokens per CTA give the shortest chain of k-blocks, but a CTA of either
     // launch needs an SM of its own, so when the main launch fits into one wave the first shape whose CTAs
     // fit beside it is taken (more rows, then more tokens per CTA: fewer CTAs, longer chain).
-    const int rows_m = cta_rows(c.d_out, m, bt, h->sm_count);
-    const int main_tiles = ((c.d_out + rows_m - 1) / rows_m) * ((m + bt - 1) / bt);
+    const int n_rows_all = h->n_sub > 1 ? 16 * h->sub_tile0[h->n_sub] : c.d_out;
+    const int rows_m = thin ? BN_W : cta_rows(n_rows_all, m, bt, h->sm_count);
+    const int main_tiles = ((n_rows_all + rows_m - 1) / rows_m) * ((m + bt - 1) / bt);
     const int room = main_tiles <= h->sm_count ? h->sm_count - main_tiles : h->sm_count;
     int rows_t = 2 * BN_W, bt_t = bt;
     {
       const int cand[4][2] = {{BN_W, 128}, {2 * BN_W, 128}, {BN_W, 256}, {2 * BN_W, 256}};
       for (int i = 0; i < 4; ++i) {
-        const int rr = h->r_pad > BN_W ? cand[i][0] : 2 * BN_W;     // one half of rows at most: the tile height does not matter
+        const int rr = h->t_cols > BN_W ? cand[i][0] : 2 * BN_W;    // one half of rows at most: the tile height does not matter
         const int tt = cand[i][1] < bt ? cand[i][1] : bt;
         rows_t = rr; bt_t = tt;
-        if (((h->r_pad + rr - 1) / rr) * ((m + tt - 1) / tt) <= room) break;
+        if (((h->t_cols + rr - 1) / rr) * ((m + tt - 1) / tt) <= room) break;
       }
     }
     CUtensorMap tm_xt;
     if (!make_map(&tm_xt, x16, m, c.d_in, c.d_in, bt_t)) return cudaErrorInvalidValue;
     PrefillArgs a = {};
     a.w = h->a; a.b = WMat(); a.b.fmt = FMT_NONE;
-    a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->r_pad; a.n_valid = h->r_pad; a.m = m; a.bt = bt_t;
+    a.out = h->t16; a.out_dtype = EORA_Y_F16; a.ld_out = h->t_cols; a.n_valid = h->t_cols; a.m = m; a.bt = bt_t;
     a.nkb_w = c.d_in / BK; a.nkb_b = 0; a.dev_status = h->dev_status; a.trace = nullptr;
     a.rows = rows_t;
-    a.n_small = 0; a.small_x = 1; a.n_split = a.n_valid; a.big_x = (h->r_pad + a.rows - 1) / a.rows;
+    a.n_small = 0; a.small_x = 1; a.n_split = a.n_valid; a.big_x = (h->t_cols + a.rows - 1) / a.rows;
+    a.n_sub = 1; a.sub_row0[0] = 0; a.outs[0] = a.out; a.sub_ld[0] = a.ld_out; a.t_sub = 0;
+    for (int i = 1; i < 5; ++i) a.sub_row0[i] = a.n_valid;
+    a.ksplit = 1; a.kchunk = a.nkb_w; a.ws = nullptr; a.ld_ws = 0; a.tickets = nullptr;
+    if (thin) {
+      // t is the head of the chain (the main product waits for it in front of its K-extension): as short as possible
+      a.rows = h->t_cols > BN_W ? BN_W : a.rows;
+      a.big_x = (h->t_cols + a.rows - 1) / a.rows;
+      a.ksplit = pick_ksplit(a.big_x, a.nkb_w, h->sm_count / 4, 4, 16);
+      a.kchunk = (a.nkb_w + a.ksplit - 1) / a.ksplit;
+      a.ksplit = (a.nkb_w + a.kchunk - 1) / a.kchunk;
+      a.ws = pst->ws_t; a.ld_ws = h->t_cols; a.tickets = pst->tk_t;
+    }
     const int smem_t = fill_stages(a);
-    dim3 grid(a.big_x * ((m + bt_t - 1) / bt_t), 1, 1);
+    dim3 grid(a.big_x * a.ksplit * ((m + bt_t - 1) / bt_t), 1, 1);
     cudaError_t e = launch_any(h->a.fmt, FMT_NONE, grid, smem_t, st, tm_xt, tm_xt, tm_xt, tm_xt, a, false);
     if (e != cudaSuccess) return e;
   } else {
@@ -733,11 +893,35 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   PrefillArgs a = {};
   a.w = h->w; a.b = h->b;
   if (!ab) a.b.fmt = FMT_NONE;
-  a.out = y; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = c.d_out; a.m = m; a.bt = bt;
+  // fused layers: the stacked rows; a plain layer has one part
+  const int n_all = h->w.n_rows < 16 * h->sub_tile0[h->n_sub] ? h->w.n_rows : 16 * h->sub_tile0[h->n_sub];
+  const int n_valid = h->n_sub > 1 ? n_all : c.d_out;
+  a.out = ys[0]; a.out_dtype = c.y_dtype; a.ld_out = c.d_out; a.n_valid = n_valid; a.m = m; a.bt = bt;
+  a.n_sub = h->n_sub; a.t_sub = h->n_sub > 1 ? h->r_pad : 0;
+  for (int i = 0; i < 5; ++i) a.sub_row0[i] = n_valid;
+  for (int i = 0; i < h->n_sub; ++i) {
+    a.sub_row0[i] = h->n_sub > 1 ? 16 * h->sub_tile0[i] : 0;
+    a.outs[i] = ys[i];
+    a.sub_ld[i] = h->n_sub > 1 ? h->sub_dout[i] : c.d_out;
+  }
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
   a.trace = reinterpret_cast<long long*>(h->trace);
-  a.rows = cta_rows(c.d_out, m, bt, h->sm_count);
-  a.n_small = 0; a.small_x = 1; a.n_split = c.d_out; a.big_x = (c.d_out + a.rows - 1) / a.rows;
+  a.rows = cta_rows(n_valid, m, bt, h->sm_count);
+  a.n_small = 0; a.small_x = 1; a.n_split = n_valid; a.big_x = (n_valid + a.rows - 1) / a.rows;
+  a.ksplit = 1; a.kchunk = a.nkb_w; a.ws = nullptr; a.ld_ws = 0; a.tickets = nullptr;
+  if (thin) {
+    // tiles of 128 rows, unless those need a second wave and tiles of 256 rows do not (fused layers: every layer a whole
+    // number of tiles)
+    bool r256 = (n_valid + BN_W - 1) / BN_W > h->sm_count && (n_valid + 2 * BN_W - 1) / (2 * BN_W) <= h->sm_count;
+    for (int i = 0; i < h->n_sub && h->n_sub > 1; ++i) r256 = r256 && h->sub_dout[i] % (2 * BN_W) == 0;
+    a.rows = n_valid > BN_W && !r256 ? BN_W : 2 * BN_W;
+    a.big_x = (n_valid + a.rows - 1) / a.rows;
+    const int t_ctas = ab ? 16 : 0;                         // leave room for the CTAs of the t launch
+    a.ksplit = pick_ksplit(a.big_x, a.nkb_w, h->sm_count - t_ctas, 8, 16);
+    a.kchunk = (a.nkb_w + a.ksplit - 1) / a.ksplit;
+    a.ksplit = (a.nkb_w + a.kchunk - 1) / a.kchunk;
+    a.ws = pst->ws_y; a.ld_ws = n_valid; a.tickets = pst->tk_y;
+  }
   const int big_y = (m + bt - 1) / bt;
   // Wave quantisation: a CTA needs an SM of its own, so a few tiles more than a whole number of waves cost a whole
   // wave (gate / up at M = 2048: 448 tiles on 148 SMs).  Then the last row tiles are taken out of the big grid until
@@ -750,7 +934,7 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     if (peel < a.big_x) {
       a.big_x -= peel;
       a.n_split = a.big_x * a.rows;
-      a.small_x = (c.d_out - a.n_split + kSmallTile - 1) / kSmallTile;
+      a.small_x = (n_valid - a.n_split + kSmallTile - 1) / kSmallTile;
       a.n_small = a.small_x * ((m + kSmallTile - 1) / kSmallTile);
       if (!make_map(&tm_xs, x16, m, c.d_in, c.d_in, kSmallTile)) return cudaErrorInvalidValue;
       if (ab && !make_map(&tm_ts, h->t16, m, h->r_pad, h->r_pad, kSmallTile)) return cudaErrorInvalidValue;
@@ -758,7 +942,7 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
     }
   }
   const int smem_y = fill_stages(a);
-  dim3 grid(a.n_small + a.big_x * big_y, 1, 1);
+  dim3 grid(a.n_small + a.big_x * a.ksplit * big_y, 1, 1);
   return launch_any(h->w.fmt, ab ? h->b.fmt : FMT_NONE, grid, smem_y, st, tm_x, tm_t, tm_xs, tm_ts, a, ab);
 }
 

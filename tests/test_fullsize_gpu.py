@@ -44,7 +44,7 @@ def test_decode_fullsize(name, w, M):
     wf, af, bf = make_case(31, K, N, 128, w=w)
     x = gen.make_x(32, M, K)
     L = eora.Layer(wf, af, bf, max_m=M)
-    assert L.path(M) == eora.EORA_PATH_DECODE
+    assert L.path(M) == (eora.EORA_PATH_DECODE if M <= 8 else eora.EORA_PATH_PREFILL)
     y = run_layer(L, x, "f16")
     rel, _ = check_parity(y, orc.forward(x, "f16", wf, af, bf), f"{name} {w} M{M}")
     assert 5e-5 < rel < 1e-3          # fp16 output rounding alone is ~2e-4: far off means a harness bug
@@ -60,7 +60,7 @@ def test_decode_quantised_adapter_fullsize(name, ab, r, M):
     x = gen.make_x(34, M, K)
     L = eora.Layer(wf, af, bf, max_m=M)
     # eight decode passes (M = 64) cost more than one walk over the k-blocks with the tensor-core family
-    assert L.path(M) == (eora.EORA_PATH_PREFILL if M == 64 else eora.EORA_PATH_DECODE)
+    assert L.path(M) == (eora.EORA_PATH_PREFILL if M > 8 else eora.EORA_PATH_DECODE)
     check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} {ab} r{r} M{M}")
     L.close()
 
@@ -136,18 +136,47 @@ def test_prefill_small_formats():
         L.close()
 
 
-def test_mid_size_m_takes_the_cheaper_family():
-    """Between 17 and 64 tokens the library weighs ceil(M / 8) decode passes against one walk over the k-blocks."""
-    for name, expect in [("q", {8: "d", 16: "d", 17: "p", 24: "p", 64: "p"}), ("down", {16: "d", 48: "d", 56: "d", 57: "p", 64: "p"})]:
+def test_mid_size_m_takes_the_tensor_core_family():
+    """Up to 8 tokens: one decode pass; from 9 on one launch of the tensor-core family, which for up to 64 tokens splits
+    the reduction axis over several CTAs per tile (sums in fp32 scratch, tickets, restored by the last CTA)."""
+    for name, Ms in [("q", (9, 24, 64)), ("down", (16, 57)), ("k", (33,))]:
         K, N = SHAPES[name]
         wf, af, bf = make_case(45, K, N, 128, w="q4")
         L = eora.Layer(wf, af, bf, max_m=64)
-        for M, fam in expect.items():
-            assert L.path(M) == (eora.EORA_PATH_DECODE if fam == "d" else eora.EORA_PATH_PREFILL), (name, M)
-        M = 24 if name == "q" else 57
-        x = gen.make_x(46, M, K)
-        check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} q4 M{M} tensor-core family")
+        for M in (1, 8):
+            assert L.path(M) == eora.EORA_PATH_DECODE, (name, M)
+        for M in (9, 16, 17, 24, 48, 64):
+            assert L.path(M) == eora.EORA_PATH_PREFILL, (name, M)
+        for M in Ms:
+            x = gen.make_x(46, M, K)
+            for rep in range(2):               # second call: sums and tickets were restored
+                check_parity(run_layer(L, x, "f16"), orc.forward(x, "f16", wf, af, bf), f"{name} q4 M{M} call {rep}")
         L.close()
+
+
+@pytest.mark.parametrize("w,ab,K,N,r,M,xd,yd", [
+    ("q4", "f16", 2048, 384, 128, 17, "f16", "f16"),      # 32 k-blocks: four CTAs per tile
+    ("q3", "q4", 1152, 160, 64, 40, "f16", "f32"),        # 18 k-blocks in two uneven shares, rows past the matrix
+    ("q4", "q8", 4096, 96, 512, 64, "bf16", "bf16"),      # rank 512: t has four row tiles
+    ("sp24", "f16", 2048, 256, 0, 33, "f16", "f16"),      # no adapter
+    ("sq4", "q3", 1024, 128, 128, 64, "f16", "f16"),
+    ("q3", "f16", 640, 224, 32, 20, "f16", "f16"),        # too few k-blocks to split: one CTA per tile
+])
+def test_few_tokens_split_reduction(w, ab, K, N, r, M, xd, yd):
+    wf, af, bf = make_case(47, K, N, r, w=w, ab=ab)
+    x = gen.make_x(48, M, K, xd)
+    L = eora.Layer(wf, af, bf, max_m=64, x_dtype=xd, y_dtype=yd)
+    assert L.path(M) == eora.EORA_PATH_PREFILL
+    ref = orc.forward(x, xd, wf, af, bf)
+    for rep in range(3):
+        y = run_layer(L, x, xd)
+        rel, mabs = orc.parity_errors(y, ref)
+        assert rel <= 2e-3 and mabs <= 1e-2, (rep, rel, mabs)
+    x1 = gen.make_x(49, 1, K, xd)              # the decode family on the same handle afterwards
+    y1 = run_layer(L, x1, xd)
+    rel, mabs = orc.parity_errors(y1, orc.forward(x1, xd, wf, af, bf))
+    assert rel <= 2e-3 and mabs <= 1e-2, ("M=1 after split launches", rel, mabs)
+    L.close()
 
 
 # ---- full-size cells that take other tile / wave paths than the small cases ------------------------------------------

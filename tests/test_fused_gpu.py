@@ -48,6 +48,42 @@ def test_fused_matches_oracle_small(w, ab, K, Ns, r, M, xd):
     F.close()
 
 
+@pytest.mark.parametrize("w,ab,K,Ns,r,M,xd", [
+    ("q4", "f16", 2048, [256, 128], 128, 17, "f16"),
+    ("q3", "q4", 1024, [128, 128, 384], 64, 64, "f16"),
+    ("q4", "q8", 2048, [128, 256], 256, 40, "bf16"),
+    ("q3", "f16", 1536, [384, 128], 0, 33, "f16"),
+])
+def test_fused_few_tokens_tensor_core_family(w, ab, K, Ns, r, M, xd):
+    """17 to 64 tokens on a fused handle whose layers are whole tiles of 128 rows: one launch of the tensor-core family
+    (plus the one for t), every layer with its own slice of t and its own output."""
+    layers = [make_case(70 + i, K, N, r, w=w, ab=ab) for i, N in enumerate(Ns)]
+    x = gen.make_x(71, M, K, xd)
+    F = eora.FusedLayers(layers, max_m=64, x_dtype=xd)
+    assert F.launches(M) <= 3
+    for rep in range(2):
+        ys = run_fused(F, x, xd)
+        for i, (wf, af, bf) in enumerate(layers):
+            check_parity(ys[i], orc.forward(x, xd, wf, af, bf), f"layer {i} call {rep}")
+    x8 = gen.make_x(72, 8, K, xd)              # and the decode family on the same handle
+    ys = run_fused(F, x8, xd)
+    for i, (wf, af, bf) in enumerate(layers):
+        check_parity(ys[i], orc.forward(x8, xd, wf, af, bf), f"layer {i} M=8")
+    F.close()
+
+
+def test_fused_fullsize_64_tokens():
+    names = ("q", "k", "v")
+    K = SHAPES[names[0]][0]
+    layers = [make_case(80 + i, K, SHAPES[nm][1], 128, w="q4", ab="q4") for i, nm in enumerate(names)]
+    x = gen.make_x(81, 64, K)
+    F = eora.FusedLayers(layers, max_m=64)
+    ys = run_fused(F, x, "f16")
+    for i, (wf, af, bf) in enumerate(layers):
+        check_parity(ys[i], orc.forward(x, "f16", wf, af, bf), names[i])
+    F.close()
+
+
 @pytest.mark.parametrize("names,w", [(("q", "k", "v"), "q3"), (("gate", "up"), "q3"), (("q", "k", "v"), "q4")])
 def test_fused_fullsize(names, w):
     K = SHAPES[names[0]][0]
