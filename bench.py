@@ -634,6 +634,8 @@ def main():
     ap.add_argument("--unfused", action="store_true", help="one launch per layer (224 per token) instead of fusing q|k|v and gate|up")
     ap.add_argument("--only-prefill", action="store_true", help="run the prefill leg alone (for profiling) and print its result")
     ap.add_argument("--single-stream", action="store_true", help="launch all layers of a block in stream order")
+    ap.add_argument("--only-few-tokens", action="store_true",
+                    help="run the 64-token q-shaped layer alone (for profiling the split-reduction launches) and print its time")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -674,6 +676,11 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(device))
         _DIST["on"] = True
 
+    if args.only_few_tokens:
+        if rank == 0:
+            ms = time_single_layer(device, 4096, 4096, "q4", RANK, 64, copies=8, iters=5)
+            print(json.dumps({"few_tokens": {"workload": "q 4096x4096/w4-g128/eora-fp16-r128/M64", "ms": ms}}))
+        return
     if args.only_prefill:
         if rank == 0:
             print(json.dumps({"prefill": time_prefill(device)}))
