@@ -181,3 +181,31 @@ def make_sparse24_quant(seed: int, K: int, N: int, bits: int = 4, group: int = 1
     qz = quantize_matrix_bits(kept, bits, g // 2)
     return {"kind": "sparse24q", "rows": K, "cols": N, "bits": bits, "group": g, "codes": qz["codes"],
             "scales": qz["scales"], "zeros": qz["zeros"], "meta": sp["meta"]}
+
+
+# ----------------------------------------------------------------------------
+# inputs of the offline solve (Algorithm 1): a weight, its compressed version and calibration activations
+# ----------------------------------------------------------------------------
+def make_solve_case(seed: int, d: int, k: int, n: int, bits: int = 3, kind: str = "rtn", rank_signal: int = 0):
+    """W [d][k] ~ N(0, 0.02^2); W^ = W rounded to a per-row uniform grid of 2^bits levels (a stand-in for the
+    compressed checkpoint: the error is bounded, zero-mean noise like that of a round-to-nearest quantiser);
+    X~ [k][n]: Gaussian columns with log-normal per-channel scales and a few strong channels, the shape of LLM
+    activations (the paper's calibration activations need the real model).  kind == "gap": the error is a rank
+    `rank_signal` matrix plus noise 100 times smaller, so the top singular subspace of the projected error is
+    well separated (for element-wise comparisons)."""
+    rng = _rng(seed, 0x501E, d, k, n)
+    w = (rng.standard_normal((d, k)) * 0.02).astype(np.float32)
+    if kind == "gap":
+        u = rng.standard_normal((d, rank_signal)); v = rng.standard_normal((rank_signal, k))
+        s = np.geomspace(1.0, 0.2, rank_signal)
+        dw = (u * s[None, :]) @ v / np.sqrt(d * k) + rng.standard_normal((d, k)) * 1e-5
+        w_hat = (w.astype(np.float64) - dw).astype(np.float32)
+    else:
+        amax = np.abs(w).max(axis=1, keepdims=True)
+        step = 2.0 * amax / (2 ** bits - 1)
+        w_hat = (np.round(w / step) * step).astype(np.float32)
+    scale = np.exp(rng.standard_normal(k) * 0.8)
+    strong = rng.choice(k, size=max(1, k // 64), replace=False)
+    scale[strong] *= 12.0
+    x = (rng.standard_normal((k, n)) * scale[:, None]).astype(np.float32)
+    return w, w_hat, x
