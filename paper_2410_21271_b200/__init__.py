@@ -36,6 +36,10 @@ class eora_linear_weights(Structure):
                                         "b", "b_scales", "b_zeros", "w_meta")]
 
 
+class eora_solve_config(Structure):
+    _fields_ = [("d", c_int32), ("k", c_int32), ("n", c_int32), ("rank", c_int32), ("oversample", c_int32), ("iters", c_int32)]
+
+
 class EoraError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -97,6 +101,14 @@ def lib() -> ctypes.CDLL:
         L.eora_linear_weight_bytes.restype = c_int64
         L.eora_linear_scratch_bytes.argtypes = [c_void_p]
         L.eora_linear_scratch_bytes.restype = c_int64
+        L.eora_solve_workspace_bytes.argtypes = [POINTER(eora_solve_config)]
+        L.eora_solve_workspace_bytes.restype = ctypes.c_size_t
+        L.eora_solve.argtypes = [POINTER(eora_solve_config), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                 c_void_p, ctypes.c_size_t, c_void_p]
+        L.eora_solve.restype = c_int
+        L.eora_solve_loss.argtypes = [POINTER(eora_solve_config), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                      c_void_p, ctypes.c_size_t, c_void_p]
+        L.eora_solve_loss.restype = c_int
         L.eora_status_string.argtypes = [c_int]
         L.eora_status_string.restype = c_char_p
         L.eora_version.argtypes = []
@@ -492,3 +504,55 @@ class MultiAdapterLayer:
             self.close()
         except Exception:
             pass
+
+
+# ---- offline solve (Algorithm 1 steps 1-6), include/eora_solve.h -------------------------------------------------
+def eora_solve_workspace_bytes(cfg: eora_solve_config) -> int:
+    return int(lib().eora_solve_workspace_bytes(ctypes.byref(cfg)))
+
+
+def eora_solve(cfg: eora_solve_config, w, w_hat, x_tilde, b_prime, a, sigma, workspace, stream=None, check: bool = True) -> int:
+    """Device tensors in, device tensors out (fp32, row-major); `workspace`: a device byte tensor."""
+    rc = lib().eora_solve(ctypes.byref(cfg), _ptr(w), _ptr(w_hat), _ptr(x_tilde), _ptr(b_prime), _ptr(a), _ptr(sigma),
+                          _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    if check and rc != EORA_OK:
+        raise EoraError(rc, "eora_solve")
+    return rc
+
+
+def eora_solve_loss(cfg: eora_solve_config, w, w_hat, x_tilde, b_prime, a, loss_sq, workspace, stream=None, check: bool = True) -> int:
+    rc = lib().eora_solve_loss(ctypes.byref(cfg), _ptr(w), _ptr(w_hat), _ptr(x_tilde), _ptr(b_prime), _ptr(a), _ptr(loss_sq),
+                               _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    if check and rc != EORA_OK:
+        raise EoraError(rc, "eora_solve_loss")
+    return rc
+
+
+def solve(w, w_hat, x_tilde, rank: int, oversample: int = 0, iters: int = 0, stream=None):
+    """Convenience wrapper: device fp32 tensors W, W^ [d][k] and X~ [k][n] in, (B' [d][r], A [r][k], sigma [r]) out.
+    Allocates the outputs and the workspace with torch; every step of the computation runs in the library."""
+    import torch
+    d, k = w.shape
+    n = x_tilde.shape[1]
+    cfg = eora_solve_config(d, k, n, rank, oversample, iters)
+    nbytes = eora_solve_workspace_bytes(cfg)
+    if nbytes == 0:
+        raise EoraError(EORA_ERR_BAD_SHAPE, "eora_solve_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=w.device)
+    b = torch.empty((d, rank), dtype=torch.float32, device=w.device)
+    a = torch.empty((rank, k), dtype=torch.float32, device=w.device)
+    sigma = torch.empty(rank, dtype=torch.float32, device=w.device)
+    eora_solve(cfg, w.contiguous(), w_hat.contiguous(), x_tilde.contiguous(), b, a, sigma, ws, stream)
+    return b, a, sigma
+
+
+def solve_loss(w, w_hat, x_tilde, b_prime, a, stream=None) -> float:
+    """|| (dW - B'A) X~ ||_F computed on the device (synchronises to return the value)."""
+    import torch
+    d, k = w.shape
+    cfg = eora_solve_config(d, k, x_tilde.shape[1], b_prime.shape[1], 0, 0)
+    ws = torch.empty(eora_solve_workspace_bytes(cfg), dtype=torch.uint8, device=w.device)
+    out = torch.zeros(1, dtype=torch.float64, device=w.device)
+    eora_solve_loss(cfg, w.contiguous(), w_hat.contiguous(), x_tilde.contiguous(), b_prime.contiguous(), a.contiguous(), out, ws, stream)
+    torch.cuda.synchronize()
+    return float(out.item()) ** 0.5

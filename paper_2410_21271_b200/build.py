@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libeora_linear.so")
-SOURCES = ["eora_api.cu", "repack.cu", "generic.cu", "decode.cu", "decode_tc.cu", "tmat.cu", "prefill.cu", "noalloc.cu"]
+SOURCES = ["eora_api.cu", "repack.cu", "generic.cu", "decode.cu", "decode_tc.cu", "tmat.cu", "prefill.cu", "noalloc.cu", "solve.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
@@ -27,6 +27,7 @@ def needs_build() -> bool:
     t = os.path.getmtime(LIB)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "eora_linear.h"))
+    deps.append(os.path.join(os.path.dirname(HERE), "include", "eora_solve.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 

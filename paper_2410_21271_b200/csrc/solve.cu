@@ -1,0 +1,404 @@
+// Offline EoRA solve (Algorithm 1, steps 1-6) on the GPU; the interface and the mathematics are in eora_solve.h.
+//
+//   1.  dW = W - W^                                                    (k_sub)
+//   2-4 the paper projects dW into the eigenspace of X~ X~^T, dW' = dW Q sqrt(L).  Only dW' dW'^T is needed here:
+//       G = X~ X~^T  (k x k),  T = dW G,  Mm = T dW^T = dW' dW'^T  (d x d)   (three fp32 contractions)
+//   5.  top-r eigenpairs (U', S'^2) of Mm by subspace iteration on m = r + oversample vectors:
+//         Y = Mm Q;  Q = orth(Y)  by Cholesky-QR (Gram matrix and factor in fp64);  repeated `iters` times, then a
+//         Rayleigh-Ritz step:  H = Q^T Mm Q  (m x m, fp64),  H = V diag(lam) V^T  by one-sided Jacobi in one CTA,
+//         U' = Q V[:, top r],  S' = sqrt(lam)
+//   6.  B' = U' S',  A = S'^{-1} U'^T dW
+//
+// Every kernel here is plain fp32 / fp64 CUDA-core arithmetic: the large contractions are tiled SGEMMs
+// (128 x 128 x 16 tiles through shared memory, 8 x 8 outputs per thread); fp32 because the quality of the
+// eigenvectors near the cut depends on the small differences between neighbouring eigenvalues of Mm.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "../../include/eora_linear.h"
+#include "../../include/eora_solve.h"
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------ SGEMM
+constexpr int BM = 128, BN = 128, BKS = 16, PAD = 4;
+
+// C[M][N] (ldc) = sum_p opA[m][p] opB[p][n];  opA[m][p] = ta ? A[p * lda + m] : A[m * lda + p];
+// opB[p][n] = tb ? B[n * ldb + p] : B[p * ldb + n].  Out-of-range elements read as zero.
+__global__ void __launch_bounds__(256) k_sgemm(int M, int N, int P, const float* __restrict__ A, int lda, int ta,
+                                               const float* __restrict__ B, int ldb, int tb, float* __restrict__ C, int ldc) {
+  __shared__ float As[BKS][BM + PAD];
+  __shared__ float Bs[BKS][BN + PAD];
+  const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+  for (int p0 = 0; p0 < P; p0 += BKS) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int e = t + 256 * i;
+      {
+        const int m = ta ? (e & (BM - 1)) : (e >> 4), p = ta ? (e >> 7) : (e & 15);
+        const int gm = m0 + m, gp = p0 + p;
+        float v = 0.f;
+        if (gm < M && gp < P) v = ta ? A[(int64_t)gp * lda + gm] : A[(int64_t)gm * lda + gp];
+        As[p][m] = v;
+      }
+      {
+        const int n = tb ? (e >> 4) : (e & (BN - 1)), p = tb ? (e & 15) : (e >> 7);
+        const int gn = n0 + n, gp = p0 + p;
+        float v = 0.f;
+        if (gn < N && gp < P) v = tb ? B[(int64_t)gn * ldb + gp] : B[(int64_t)gp * ldb + gn];
+        Bs[p][n] = v;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int p = 0; p < BKS; ++p) {
+      float a[8], b[8];
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[p][ty * 4]), a1 = *reinterpret_cast<const float4*>(&As[p][64 + ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[p][tx * 4]), b1 = *reinterpret_cast<const float4*>(&Bs[p][64 + tx * 4]);
+      a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w; a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
+      b[0] = b0.x; b[1] = b0.y; b[2] = b0.z; b[3] = b0.w; b[4] = b1.x; b[5] = b1.y; b[6] = b1.z; b[7] = b1.w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int gm = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + i - 4);
+    if (gm >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int gn = n0 + (j < 4 ? tx * 4 + j : 64 + tx * 4 + j - 4);
+      if (gn < N) C[(int64_t)gm * ldc + gn] = acc[i][j];
+    }
+  }
+}
+
+cudaError_t sgemm(cudaStream_t st, int M, int N, int P, const float* A, int lda, bool ta, const float* B, int ldb, bool tb, float* C, int ldc) {
+  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
+  k_sgemm<<<grid, 256, 0, st>>>(M, N, P, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------ small pieces
+__global__ void k_sub(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ c, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) c[i] = a[i] - b[i];
+}
+
+// A fixed start for the iteration: values in (-1, 1) from a counter hash (any full-rank start converges).
+__global__ void k_init(float* y, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    uint64_t z = (uint64_t)i * 0x9E3779B97F4A7C15ull + 0xD1B54A32D192ED03ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    y[i] = (float)((double)(z >> 11) * (2.0 / 9007199254740992.0) - 1.0);
+  }
+}
+
+// S[i][j] = sum_row A[row][i] B[row][j]  for two [rows][m] fp32 matrices, products and sums in fp64.
+// One CTA per 16 x 16 block of S; its 256 threads stride over the rows and meet in a shared-memory reduction.
+__global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, const float* __restrict__ B, int rows, int m, double* __restrict__ S) {
+  __shared__ float sa[16][17], sb[16][17];
+  const int i0 = blockIdx.y * 16, j0 = blockIdx.x * 16, t = threadIdx.x, ti = t >> 4, tj = t & 15;
+  double acc = 0.0;
+  for (int r0 = 0; r0 < rows; r0 += 16) {
+    {
+      const int rr = r0 + ti;
+      sa[ti][tj] = (rr < rows && i0 + tj < m) ? A[(int64_t)rr * m + i0 + tj] : 0.f;
+      sb[ti][tj] = (rr < rows && j0 + tj < m) ? B[(int64_t)rr * m + j0 + tj] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc += (double)sa[r][ti] * (double)sb[r][tj];
+    __syncthreads();
+  }
+  if (i0 + ti < m && j0 + tj < m) S[(int64_t)(i0 + ti) * m + j0 + tj] = acc;
+}
+
+// In-place Cholesky S = L L^T (lower triangle, fp64) of an m x m matrix in global memory by one CTA.
+// A small multiple of the trace is added to the diagonal first, so that a rank-deficient iterate still factors.
+__global__ void __launch_bounds__(1024) k_chol64(double* S, int m) {
+  __shared__ double shift_s;
+  const int t = threadIdx.x, nt = blockDim.x;
+  if (t == 0) {
+    double tr = 0.0;
+    for (int i = 0; i < m; ++i) tr += S[(int64_t)i * m + i];
+    shift_s = 1e-13 * tr + 1e-300;
+  }
+  __syncthreads();
+  for (int i = t; i < m; i += nt) S[(int64_t)i * m + i] += shift_s;
+  __syncthreads();
+  for (int j = 0; j < m; ++j) {
+    if (t == 0) {
+      const double v = S[(int64_t)j * m + j];
+      S[(int64_t)j * m + j] = sqrt(v > shift_s * 1e-3 ? v : shift_s * 1e-3);
+    }
+    __syncthreads();
+    const double ljj = S[(int64_t)j * m + j];
+    for (int i = j + 1 + t; i < m; i += nt) S[(int64_t)i * m + j] /= ljj;
+    __syncthreads();
+    // trailing update of the lower triangle: S[i][c] -= L[i][j] L[c][j] for j < c <= i
+    const int rem = m - j - 1;
+    for (int e = t; e < rem * rem; e += nt) {
+      const int i = j + 1 + e / rem, c = j + 1 + e % rem;
+      if (c <= i) S[(int64_t)i * m + c] -= S[(int64_t)i * m + j] * S[(int64_t)c * m + j];
+    }
+    __syncthreads();
+  }
+}
+
+// Q = Y L^{-T}: every row q of Q solves q L^T = y by forward substitution (one thread per row; L is read by all).
+__global__ void k_trsm_rows(const float* __restrict__ Y, const double* __restrict__ L, int rows, int m, float* __restrict__ Q) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  const float* y = Y + (int64_t)row * m;
+  float* q = Q + (int64_t)row * m;
+  for (int j = 0; j < m; ++j) {
+    double v = (double)y[j];
+    for (int i = 0; i < j; ++i) v -= (double)q[i] * L[(int64_t)j * m + i];
+    q[j] = (float)(v / L[(int64_t)j * m + j]);
+  }
+}
+
+// Symmetric positive semi-definite eigenproblem H = V diag(lam) V^T, m x m, fp64, by one-sided (Hestenes) Jacobi in one
+// CTA: pairs of columns of H are rotated until they are orthogonal; then lam_i = ||h_i|| and V holds the rotations.
+// Pairs follow the round-robin tournament (m' / 2 disjoint pairs per step, m' - 1 steps per sweep); a warp takes a pair.
+// Output: eigenvalues in descending order (lam) and the matching eigenvectors as fp32 columns of Vf ([m][m] row-major).
+__global__ void __launch_bounds__(1024) k_jacobi64(double* H, double* V, int m, double* lam, float* Vf, int max_sweeps) {
+  __shared__ int moved_s;
+  __shared__ int rank_s[512];
+  const int t = threadIdx.x, nt = blockDim.x, warp = t >> 5, lane = t & 31, nwarp = nt >> 5;
+  for (int e = t; e < m * m; e += nt) V[e] = (e / m == e % m) ? 1.0 : 0.0;
+  __syncthreads();
+  const int mp = (m + 1) & ~1;                       // players of the tournament (one bye if m is odd)
+  for (int sweep = 0; sweep < max_sweeps; ++sweep) {
+    if (t == 0) moved_s = 0;
+    __syncthreads();
+    for (int step = 0; step < mp - 1; ++step) {
+      for (int pr = warp; pr < mp / 2; pr += nwarp) {
+        // circle method: player mp - 1 is fixed, the others rotate
+        int p = pr == 0 ? mp - 1 : (step + pr) % (mp - 1);
+        int q = (step + mp - 1 - pr) % (mp - 1);
+        if (p > q) { const int x = p; p = q; q = x; }
+        if (q >= m) continue;                        // the bye
+        // columns p and q of H (column c of the symmetric start is stored as row c: H[c * m + i])
+        double* hp = H + (int64_t)p * m; double* hq = H + (int64_t)q * m;
+        double al = 0.0, be = 0.0, ga = 0.0;
+        for (int i = lane; i < m; i += 32) { const double a = hp[i], b = hq[i]; al += a * a; be += b * b; ga += a * b; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          al += __shfl_xor_sync(0xffffffffu, al, o); be += __shfl_xor_sync(0xffffffffu, be, o); ga += __shfl_xor_sync(0xffffffffu, ga, o);
+        }
+        if (fabs(ga) <= 1e-15 * sqrt(al * be) || ga == 0.0) continue;
+        const double zeta = (be - al) / (2.0 * ga);
+        const double tt = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+        const double c = 1.0 / sqrt(1.0 + tt * tt), s = c * tt;
+        for (int i = lane; i < m; i += 32) {
+          const double a = hp[i], b = hq[i];
+          hp[i] = c * a - s * b; hq[i] = s * a + c * b;
+        }
+        double* vp = V + (int64_t)p * m; double* vq = V + (int64_t)q * m;
+        for (int i = lane; i < m; i += 32) {
+          const double a = vp[i], b = vq[i];
+          vp[i] = c * a - s * b; vq[i] = s * a + c * b;
+        }
+        if (lane == 0 && fabs(ga) > 1e-13 * sqrt(al * be)) moved_s = 1;
+      }
+      __syncthreads();
+    }
+    const int moved = moved_s;
+    __syncthreads();
+    if (!moved) break;
+  }
+  // eigenvalues = column norms; order them (descending; ties by index)
+  for (int c = warp; c < m; c += nwarp) {
+    double al = 0.0;
+    for (int i = lane; i < m; i += 32) { const double a = H[(int64_t)c * m + i]; al += a * a; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) al += __shfl_xor_sync(0xffffffffu, al, o);
+    if (lane == 0) lam[m + c] = sqrt(al);            // unsorted, behind the sorted ones
+  }
+  __syncthreads();
+  for (int c = t; c < m; c += nt) {
+    int rk = 0;
+    const double mine = lam[m + c];
+    for (int o = 0; o < m; ++o) { const double v = lam[m + o]; rk += (v > mine || (v == mine && o < c)) ? 1 : 0; }
+    rank_s[c] = rk;
+  }
+  __syncthreads();
+  for (int c = t; c < m; c += nt) lam[rank_s[c]] = lam[m + c];
+  for (int e = t; e < m * m; e += nt) {
+    const int c = e / m, i = e % m;                  // eigenvector c, component i  ->  Vf[i][rank of c]
+    Vf[(int64_t)i * m + rank_s[c]] = (float)V[e];
+  }
+}
+
+// sigma_i = sqrt(lam_i);  B'[row][i] = U[row][i] sigma_i  (U: [d][r])
+__global__ void k_finish_b(const float* __restrict__ U, const double* __restrict__ lam, int d, int r, float* __restrict__ Bp, float* __restrict__ sigma) {
+  const int64_t n = (int64_t)d * r;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+    const int i = (int)(e % r);
+    const float s = (float)sqrt(fmax(lam[i], 0.0));
+    Bp[e] = U[e] * s;
+    if (e < r) sigma[e] = (float)sqrt(fmax(lam[e], 0.0));
+  }
+}
+// A[i][:] /= sigma_i  (A: [r][k] holding U^T dW)
+__global__ void k_finish_a(float* __restrict__ A, const double* __restrict__ lam, int r, int k) {
+  const int64_t n = (int64_t)r * k;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+    const double s = sqrt(fmax(lam[e / k], 0.0));
+    A[e] = s > 0.0 ? (float)((double)A[e] / s) : 0.f;
+  }
+}
+// sum of squares of a matrix, fp64, into *out (zeroed by the caller)
+__global__ void k_sumsq(const float* __restrict__ a, int64_t n, double* out) {
+  double acc = 0.0;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) acc += (double)a[i] * (double)a[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) atomicAdd(out, acc);
+}
+__global__ void k_axpy_neg(float* __restrict__ c, const float* __restrict__ a, int64_t n) {      // c = a - c
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) c[i] = a[i] - c[i];
+}
+
+// ------------------------------------------------------------------------------------------------ workspace
+struct Plan {
+  int d, k, n, r, m, iters;
+  size_t off_dw, off_g, off_t, off_m, off_y, off_q, off_z, off_u, off_s, off_h, off_v, off_lam, off_vf, total;
+};
+size_t up256(size_t v) { return (v + 255) & ~size_t(255); }
+bool make_plan(const eora_solve_config* c, Plan& p) {
+  if (!c || c->d < 1 || c->k < 1 || c->n < 1 || c->rank < 1) return false;
+  p.d = c->d; p.k = c->k; p.n = c->n; p.r = c->rank;
+  int over = c->oversample > 0 ? c->oversample : 32;
+  p.m = p.r + over;
+  if (p.m > p.d) p.m = p.d;
+  if (p.r > p.m || p.m > 512) return false;
+  p.iters = c->iters > 0 ? c->iters : 24;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o += up256(bytes); return at; };
+  p.off_dw = take((size_t)p.d * p.k * 4);
+  p.off_g = take((size_t)p.k * p.k * 4);
+  p.off_t = take((size_t)p.d * (p.k > p.n ? p.k : p.n) * 4);      // T = dW G; the loss check keeps dW X~ here
+  p.off_m = take((size_t)p.d * p.d * 4);
+  p.off_y = take((size_t)p.d * p.m * 4);
+  p.off_q = take((size_t)p.d * p.m * 4);
+  p.off_z = take((size_t)p.d * p.m * 4);
+  p.off_u = take((size_t)p.d * p.r * 4);
+  p.off_s = take((size_t)p.m * p.m * 8);
+  p.off_h = take((size_t)p.m * p.m * 8);
+  p.off_v = take((size_t)p.m * p.m * 8);
+  p.off_lam = take((size_t)2 * p.m * 8);
+  p.off_vf = take((size_t)p.m * p.m * 4);
+  p.total = o;
+  return true;
+}
+inline bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; }
+
+#define CK(x) do { cudaError_t e__ = (x); if (e__ != cudaSuccess) return EORA_ERR_CUDA; } while (0)
+
+// Q = orth(Y) by Cholesky-QR, Gram matrix and factor in fp64.
+int orthonormalise(cudaStream_t st, const Plan& p, const float* Y, float* Q, double* S) {
+  dim3 g((p.m + 15) / 16, (p.m + 15) / 16);
+  k_gram64<<<g, 256, 0, st>>>(Y, Y, p.d, p.m, S);
+  k_chol64<<<1, 1024, 0, st>>>(S, p.m);
+  k_trsm_rows<<<(p.d + 127) / 128, 128, 0, st>>>(Y, S, p.d, p.m, Q);
+  CK(cudaGetLastError());
+  return EORA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t eora_solve_workspace_bytes(const eora_solve_config* cfg) {
+  Plan p;
+  return make_plan(cfg, p) ? p.total : 0;
+}
+
+int eora_solve(const eora_solve_config* cfg, const float* w, const float* w_hat, const float* x_tilde, float* b_prime, float* a,
+               float* sigma, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!cfg || !w || !w_hat || !x_tilde || !b_prime || !a || !sigma || !workspace) return EORA_ERR_NULL_ARG;
+  Plan p;
+  if (!make_plan(cfg, p) || workspace_bytes < p.total) return EORA_ERR_BAD_SHAPE;
+  if (!aligned16(w) || !aligned16(w_hat) || !aligned16(x_tilde) || !aligned16(b_prime) || !aligned16(a) || !aligned16(workspace)) return EORA_ERR_MISALIGNED;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+  float* dW = reinterpret_cast<float*>(ws + p.off_dw);
+  float* G = reinterpret_cast<float*>(ws + p.off_g);
+  float* T = reinterpret_cast<float*>(ws + p.off_t);
+  float* Mm = reinterpret_cast<float*>(ws + p.off_m);
+  float* Y = reinterpret_cast<float*>(ws + p.off_y);
+  float* Q = reinterpret_cast<float*>(ws + p.off_q);
+  float* Z = reinterpret_cast<float*>(ws + p.off_z);
+  float* U = reinterpret_cast<float*>(ws + p.off_u);
+  double* S = reinterpret_cast<double*>(ws + p.off_s);
+  double* H = reinterpret_cast<double*>(ws + p.off_h);
+  double* V = reinterpret_cast<double*>(ws + p.off_v);
+  double* lam = reinterpret_cast<double*>(ws + p.off_lam);
+  float* Vf = reinterpret_cast<float*>(ws + p.off_vf);
+  const int d = p.d, k = p.k, n = p.n, r = p.r, m = p.m;
+
+  // step 1
+  k_sub<<<592, 256, 0, st>>>(w, w_hat, dW, (int64_t)d * k);
+  // steps 2-4, as the d x d matrix dW' dW'^T = dW (X~ X~^T) dW^T
+  CK(sgemm(st, k, k, n, x_tilde, n, false, x_tilde, n, true, G, k));          // G = X~ X~^T
+  CK(sgemm(st, d, k, k, dW, k, false, G, k, false, T, k));                    // T = dW G
+  CK(sgemm(st, d, d, k, T, k, false, dW, k, true, Mm, d));                    // Mm = T dW^T
+  // step 5: subspace iteration
+  k_init<<<592, 256, 0, st>>>(Y, (int64_t)d * m);
+  if (int rc = orthonormalise(st, p, Y, Q, S)) return rc;
+  for (int it = 0; it < p.iters; ++it) {
+    CK(sgemm(st, d, m, d, Mm, d, false, Q, m, false, Y, m));                  // Y = Mm Q
+    if (int rc = orthonormalise(st, p, Y, Q, S)) return rc;
+  }
+  if (int rc = orthonormalise(st, p, Q, Y, S)) return rc;                     // second pass: orthogonal to fp32 rounding
+  // Rayleigh-Ritz on span(Y)
+  CK(sgemm(st, d, m, d, Mm, d, false, Y, m, false, Z, m));                    // Z = Mm Y
+  {
+    dim3 g((m + 15) / 16, (m + 15) / 16);
+    k_gram64<<<g, 256, 0, st>>>(Y, Z, d, m, H);                               // H = Y^T Mm Y
+  }
+  k_jacobi64<<<1, 1024, 0, st>>>(H, V, m, lam, Vf, 40);
+  CK(cudaGetLastError());
+  CK(sgemm(st, d, r, m, Y, m, false, Vf, m, false, U, r));                    // U' = Y V[:, :r]
+  // step 6
+  k_finish_b<<<296, 256, 0, st>>>(U, lam, d, r, b_prime, sigma);
+  CK(sgemm(st, r, k, d, U, r, true, dW, k, false, a, k));                     // U'^T dW
+  k_finish_a<<<296, 256, 0, st>>>(a, lam, r, k);
+  CK(cudaGetLastError());
+  return EORA_OK;
+}
+
+int eora_solve_loss(const eora_solve_config* cfg, const float* w, const float* w_hat, const float* x_tilde, const float* b_prime,
+                    const float* a, double* loss_sq, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!cfg || !w || !w_hat || !x_tilde || !b_prime || !a || !loss_sq || !workspace) return EORA_ERR_NULL_ARG;
+  Plan p;
+  if (!make_plan(cfg, p) || workspace_bytes < p.total) return EORA_ERR_BAD_SHAPE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  char* ws = reinterpret_cast<char*>(workspace);
+  float* dW = reinterpret_cast<float*>(ws + p.off_dw);
+  float* R = reinterpret_cast<float*>(ws + p.off_g);       // B'A, then the residual (d x k fits: the slot holds k x k ... see below)
+  float* E = reinterpret_cast<float*>(ws + p.off_t);       // (dW - B'A) X~  (d x n)
+  if ((size_t)p.d * p.k > (size_t)p.k * p.k) R = reinterpret_cast<float*>(ws + p.off_m);   // d > k: use the d x d slot
+  k_sub<<<592, 256, 0, st>>>(w, w_hat, dW, (int64_t)p.d * p.k);
+  CK(sgemm(st, p.d, p.k, p.r, b_prime, p.r, false, a, p.k, false, R, p.k));    // B' A
+  k_axpy_neg<<<592, 256, 0, st>>>(R, dW, (int64_t)p.d * p.k);                  // dW - B'A
+  CK(sgemm(st, p.d, p.n, p.k, R, p.k, false, x_tilde, p.n, false, E, p.n));
+  CK(cudaMemsetAsync(loss_sq, 0, sizeof(double), st));
+  k_sumsq<<<592, 256, 0, st>>>(E, (int64_t)p.d * p.n, loss_sq);
+  CK(cudaGetLastError());
+  return EORA_OK;
+}
+
+}  // extern "C"
