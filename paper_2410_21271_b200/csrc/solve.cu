@@ -81,9 +81,98 @@ __global__ void __launch_bounds__(256) k_sgemm(int M, int N, int P, const float*
   }
 }
 
+// The same product for whole tiles (M, N multiples of 128, P of 16, rows 16-byte aligned): 16-byte global loads, the
+// next k-slice fetched into registers while the current one is multiplied.
+template <bool TA, bool TB>
+__global__ void __launch_bounds__(256) k_sgemm_full(int P, const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
+                                                    float* __restrict__ C, int ldc) {
+  __shared__ __align__(16) float As[2][BKS][BM + PAD];
+  __shared__ __align__(16) float Bs[2][BKS][BN + PAD];
+  const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  // this thread's two 16-byte pieces of each operand tile
+  // A not transposed: tile rows m (128) x 16 p: piece = (row, p4), 4 pieces per row;  transposed: A[p][m]: (p, m4), 32 per p
+  int a_r[2], a_c[2], b_r[2], b_c[2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int e = t + 256 * i;
+    if (TA) { a_r[i] = e >> 5; a_c[i] = (e & 31) * 4; } else { a_r[i] = e >> 2; a_c[i] = (e & 3) * 4; }
+    if (TB) { b_r[i] = e >> 2; b_c[i] = (e & 3) * 4; } else { b_r[i] = e >> 5; b_c[i] = (e & 31) * 4; }
+  }
+  auto load_a = [&](int p0, int i) -> float4 {
+    return TA ? *reinterpret_cast<const float4*>(A + (int64_t)(p0 + a_r[i]) * lda + m0 + a_c[i])
+              : *reinterpret_cast<const float4*>(A + (int64_t)(m0 + a_r[i]) * lda + p0 + a_c[i]);
+  };
+  auto load_b = [&](int p0, int i) -> float4 {
+    return TB ? *reinterpret_cast<const float4*>(B + (int64_t)(n0 + b_r[i]) * ldb + p0 + b_c[i])
+              : *reinterpret_cast<const float4*>(B + (int64_t)(p0 + b_r[i]) * ldb + n0 + b_c[i]);
+  };
+  auto store_a = [&](int buf, int i, const float4& v) {
+    if (TA) *reinterpret_cast<float4*>(&As[buf][a_r[i]][a_c[i]]) = v;
+    else { As[buf][a_c[i]][a_r[i]] = v.x; As[buf][a_c[i] + 1][a_r[i]] = v.y; As[buf][a_c[i] + 2][a_r[i]] = v.z; As[buf][a_c[i] + 3][a_r[i]] = v.w; }
+  };
+  auto store_b = [&](int buf, int i, const float4& v) {
+    if (TB) { Bs[buf][b_c[i]][b_r[i]] = v.x; Bs[buf][b_c[i] + 1][b_r[i]] = v.y; Bs[buf][b_c[i] + 2][b_r[i]] = v.z; Bs[buf][b_c[i] + 3][b_r[i]] = v.w; }
+    else *reinterpret_cast<float4*>(&Bs[buf][b_r[i]][b_c[i]]) = v;
+  };
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+  float4 ra[2], rb[2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) { ra[i] = load_a(0, i); rb[i] = load_b(0, i); }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) { store_a(0, i, ra[i]); store_b(0, i, rb[i]); }
+  __syncthreads();
+  int buf = 0;
+  for (int p0 = 0; p0 < P; p0 += BKS) {
+    const bool more = p0 + BKS < P;
+    if (more) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) { ra[i] = load_a(p0 + BKS, i); rb[i] = load_b(p0 + BKS, i); }
+    }
+#pragma unroll
+    for (int p = 0; p < BKS; ++p) {
+      float a[8], b[8];
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][p][ty * 4]), a1 = *reinterpret_cast<const float4*>(&As[buf][p][64 + ty * 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][p][tx * 4]), b1 = *reinterpret_cast<const float4*>(&Bs[buf][p][64 + tx * 4]);
+      a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w; a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
+      b[0] = b0.x; b[1] = b0.y; b[2] = b0.z; b[3] = b0.w; b[4] = b1.x; b[5] = b1.y; b[6] = b1.z; b[7] = b1.w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    if (more) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) { store_a(buf ^ 1, i, ra[i]); store_b(buf ^ 1, i, rb[i]); }
+    }
+    __syncthreads();
+    buf ^= 1;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int gm = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + i - 4);
+    float* row = C + (int64_t)gm * ldc + n0;
+    *reinterpret_cast<float4*>(row + tx * 4) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    *reinterpret_cast<float4*>(row + 64 + tx * 4) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+  }
+}
+
 cudaError_t sgemm(cudaStream_t st, int M, int N, int P, const float* A, int lda, bool ta, const float* B, int ldb, bool tb, float* C, int ldc) {
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
-  k_sgemm<<<grid, 256, 0, st>>>(M, N, P, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc);
+  const bool full = M % BM == 0 && N % BN == 0 && P % BKS == 0 && lda % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
+                    ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15) == 0;
+  if (full) {
+    if (ta && tb) k_sgemm_full<true, true><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    else if (ta) k_sgemm_full<true, false><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    else if (tb) k_sgemm_full<false, true><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    else k_sgemm_full<false, false><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+  } else {
+    k_sgemm<<<grid, 256, 0, st>>>(M, N, P, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc);
+  }
   return cudaGetLastError();
 }
 
@@ -92,28 +181,30 @@ __global__ void k_sub(const float* __restrict__ a, const float* __restrict__ b, 
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) c[i] = a[i] - b[i];
 }
 
-// A fixed start for the iteration: values in (-1, 1) from a counter hash (any full-rank start converges).
-__global__ void k_init(float* y, int64_t n) {
+// A fixed start for the iteration: values in (-1, 1) from a counter hash (any full-rank start converges).  The iterate
+// is stored with a leading dimension ld >= m (a multiple of the SGEMM tile); the columns past m are zero and stay zero.
+__global__ void k_init(float* y, int rows, int m, int ld) {
+  const int64_t n = (int64_t)rows * ld;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     uint64_t z = (uint64_t)i * 0x9E3779B97F4A7C15ull + 0xD1B54A32D192ED03ull;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
     z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
     z ^= z >> 31;
-    y[i] = (float)((double)(z >> 11) * (2.0 / 9007199254740992.0) - 1.0);
+    y[i] = (int)(i % ld) < m ? (float)((double)(z >> 11) * (2.0 / 9007199254740992.0) - 1.0) : 0.f;
   }
 }
 
 // S[i][j] = sum_row A[row][i] B[row][j]  for two [rows][m] fp32 matrices, products and sums in fp64.
-// One CTA per 16 x 16 block of S; its 256 threads stride over the rows and meet in a shared-memory reduction.
-__global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, const float* __restrict__ B, int rows, int m, double* __restrict__ S) {
+// One CTA per 16 x 16 block of S, one thread per element; slices of 16 rows go through shared memory.
+__global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, const float* __restrict__ B, int rows, int m, int ld, double* __restrict__ S) {
   __shared__ float sa[16][17], sb[16][17];
   const int i0 = blockIdx.y * 16, j0 = blockIdx.x * 16, t = threadIdx.x, ti = t >> 4, tj = t & 15;
   double acc = 0.0;
   for (int r0 = 0; r0 < rows; r0 += 16) {
     {
       const int rr = r0 + ti;
-      sa[ti][tj] = (rr < rows && i0 + tj < m) ? A[(int64_t)rr * m + i0 + tj] : 0.f;
-      sb[ti][tj] = (rr < rows && j0 + tj < m) ? B[(int64_t)rr * m + j0 + tj] : 0.f;
+      sa[ti][tj] = (rr < rows && i0 + tj < m) ? A[(int64_t)rr * ld + i0 + tj] : 0.f;
+      sb[ti][tj] = (rr < rows && j0 + tj < m) ? B[(int64_t)rr * ld + j0 + tj] : 0.f;
     }
     __syncthreads();
 #pragma unroll
@@ -123,11 +214,21 @@ __global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, con
   if (i0 + ti < m && j0 + tj < m) S[(int64_t)(i0 + ti) * m + j0 + tj] = acc;
 }
 
-// In-place Cholesky S = L L^T (lower triangle, fp64) of an m x m matrix in global memory by one CTA.
-// A small multiple of the trace is added to the diagonal first, so that a rank-deficient iterate still factors.
-__global__ void __launch_bounds__(1024) k_chol64(double* S, int m) {
+// Cholesky S = L L^T (fp64) of an m x m Gram matrix and the inverse of the factor, by one CTA: writes W = L^{-T} as fp32
+// into an [ld][ld] matrix (zero outside its upper triangle), so that Q = Y W is orth(Y).  The matrix is worked on in
+// shared memory when it fits (m <= kCholSmem), else in place in global memory.  A small multiple of the trace is added
+// to the diagonal first, so that a rank-deficient iterate still factors.
+constexpr int kCholSmem = 160;
+__global__ void __launch_bounds__(1024) k_chol_inv64(double* Sg, int m, float* W, int ld) {
+  extern __shared__ double sm[];
   __shared__ double shift_s;
   const int t = threadIdx.x, nt = blockDim.x;
+  const bool in_smem = m <= kCholSmem;
+  double* S = in_smem ? sm : Sg;
+  if (in_smem) {
+    for (int e = t; e < m * m; e += nt) sm[e] = Sg[e];
+    __syncthreads();
+  }
   if (t == 0) {
     double tr = 0.0;
     for (int i = 0; i < m; ++i) tr += S[(int64_t)i * m + i];
@@ -153,18 +254,25 @@ __global__ void __launch_bounds__(1024) k_chol64(double* S, int m) {
     }
     __syncthreads();
   }
-}
-
-// Q = Y L^{-T}: every row q of Q solves q L^T = y by forward substitution (one thread per row; L is read by all).
-__global__ void k_trsm_rows(const float* __restrict__ Y, const double* __restrict__ L, int rows, int m, float* __restrict__ Q) {
-  const int row = blockIdx.x * blockDim.x + threadIdx.x;
-  if (row >= rows) return;
-  const float* y = Y + (int64_t)row * m;
-  float* q = Q + (int64_t)row * m;
-  for (int j = 0; j < m; ++j) {
-    double v = (double)y[j];
-    for (int i = 0; i < j; ++i) v -= (double)q[i] * L[(int64_t)j * m + i];
-    q[j] = (float)(v / L[(int64_t)j * m + j]);
+  // X = L^{-1}, one thread per column j (forward substitution down the column), kept in the strict upper triangle of S
+  // (free after the factorisation) as S[j][i] = X[i][j] for i > j; the diagonal of X is 1 / L[j][j].
+  for (int j = t; j < m; j += nt) {
+    for (int i = j + 1; i < m; ++i) {
+      double acc = S[(int64_t)i * m + j] / S[(int64_t)j * m + j];                   // L[i][j] X[j][j]
+      for (int q = j + 1; q < i; ++q) acc += S[(int64_t)i * m + q] * S[(int64_t)j * m + q];   // L[i][q] X[q][j]
+      S[(int64_t)j * m + i] = -acc / S[(int64_t)i * m + i];
+    }
+  }
+  __syncthreads();
+  // W[j][i] = X[i][j] (upper triangle of W = L^{-T}); everything else zero
+  for (int e = t; e < ld * ld; e += nt) {
+    const int j = e / ld, i = e % ld;
+    float v = 0.f;
+    if (j < m && i < m) {
+      if (i == j) v = (float)(1.0 / S[(int64_t)j * m + j]);
+      else if (i > j) v = (float)S[(int64_t)j * m + i];
+    }
+    W[e] = v;
   }
 }
 
@@ -197,7 +305,7 @@ __global__ void __launch_bounds__(1024) k_jacobi64(double* H, double* V, int m, 
         for (int o = 16; o > 0; o >>= 1) {
           al += __shfl_xor_sync(0xffffffffu, al, o); be += __shfl_xor_sync(0xffffffffu, be, o); ga += __shfl_xor_sync(0xffffffffu, ga, o);
         }
-        if (fabs(ga) <= 1e-15 * sqrt(al * be) || ga == 0.0) continue;
+        if (fabs(ga) <= 1e-11 * sqrt(al * be) || ga == 0.0) continue;      // orthogonal far beyond what the fp32 operands carry
         const double zeta = (be - al) / (2.0 * ga);
         const double tt = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
         const double c = 1.0 / sqrt(1.0 + tt * tt), s = c * tt;
@@ -210,7 +318,7 @@ __global__ void __launch_bounds__(1024) k_jacobi64(double* H, double* V, int m, 
           const double a = vp[i], b = vq[i];
           vp[i] = c * a - s * b; vq[i] = s * a + c * b;
         }
-        if (lane == 0 && fabs(ga) > 1e-13 * sqrt(al * be)) moved_s = 1;
+        if (lane == 0) moved_s = 1;
       }
       __syncthreads();
     }
@@ -273,8 +381,8 @@ __global__ void k_axpy_neg(float* __restrict__ c, const float* __restrict__ a, i
 
 // ------------------------------------------------------------------------------------------------ workspace
 struct Plan {
-  int d, k, n, r, m, iters;
-  size_t off_dw, off_g, off_t, off_m, off_y, off_q, off_z, off_u, off_s, off_h, off_v, off_lam, off_vf, total;
+  int d, k, n, r, m, ldm, iters;       // ldm: leading dimension of the iterates (m rounded up to the SGEMM tile)
+  size_t off_w, off_dw, off_g, off_t, off_m, off_y, off_q, off_z, off_u, off_s, off_h, off_v, off_lam, off_vf, total;
 };
 size_t up256(size_t v) { return (v + 255) & ~size_t(255); }
 bool make_plan(const eora_solve_config* c, Plan& p) {
@@ -285,15 +393,17 @@ bool make_plan(const eora_solve_config* c, Plan& p) {
   if (p.m > p.d) p.m = p.d;
   if (p.r > p.m || p.m > 512) return false;
   p.iters = c->iters > 0 ? c->iters : 24;
+  p.ldm = (p.m + BN - 1) / BN * BN;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += up256(bytes); return at; };
   p.off_dw = take((size_t)p.d * p.k * 4);
   p.off_g = take((size_t)p.k * p.k * 4);
   p.off_t = take((size_t)p.d * (p.k > p.n ? p.k : p.n) * 4);      // T = dW G; the loss check keeps dW X~ here
   p.off_m = take((size_t)p.d * p.d * 4);
-  p.off_y = take((size_t)p.d * p.m * 4);
-  p.off_q = take((size_t)p.d * p.m * 4);
-  p.off_z = take((size_t)p.d * p.m * 4);
+  p.off_y = take((size_t)p.d * p.ldm * 4);
+  p.off_q = take((size_t)p.d * p.ldm * 4);
+  p.off_z = take((size_t)p.d * p.ldm * 4);
+  p.off_w = take((size_t)p.ldm * p.ldm * 4);
   p.off_u = take((size_t)p.d * p.r * 4);
   p.off_s = take((size_t)p.m * p.m * 8);
   p.off_h = take((size_t)p.m * p.m * 8);
@@ -307,13 +417,21 @@ inline bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 
 
 #define CK(x) do { cudaError_t e__ = (x); if (e__ != cudaSuccess) return EORA_ERR_CUDA; } while (0)
 
-// Q = orth(Y) by Cholesky-QR, Gram matrix and factor in fp64.
-int orthonormalise(cudaStream_t st, const Plan& p, const float* Y, float* Q, double* S) {
+// Q = orth(Y) by Cholesky-QR: Gram matrix, factor and its inverse in fp64, then Q = Y L^{-T} as a contraction.
+int orthonormalise(cudaStream_t st, const Plan& p, const float* Y, float* Q, double* S, float* W) {
   dim3 g((p.m + 15) / 16, (p.m + 15) / 16);
-  k_gram64<<<g, 256, 0, st>>>(Y, Y, p.d, p.m, S);
-  k_chol64<<<1, 1024, 0, st>>>(S, p.m);
-  k_trsm_rows<<<(p.d + 127) / 128, 128, 0, st>>>(Y, S, p.d, p.m, Q);
+  k_gram64<<<g, 256, 0, st>>>(Y, Y, p.d, p.m, p.ldm, S);
+  static bool attr_set[64] = {};
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return EORA_ERR_CUDA;
+  const int smem = p.m <= kCholSmem ? p.m * p.m * 8 : 0;
+  if (!attr_set[device]) {
+    CK(cudaFuncSetAttribute(k_chol_inv64, cudaFuncAttributeMaxDynamicSharedMemorySize, kCholSmem * kCholSmem * 8));
+    attr_set[device] = true;
+  }
+  k_chol_inv64<<<1, 1024, smem, st>>>(S, p.m, W, p.ldm);
   CK(cudaGetLastError());
+  CK(sgemm(st, p.d, p.ldm, p.ldm, Y, p.ldm, false, W, p.ldm, false, Q, p.ldm));
   return EORA_OK;
 }
 
@@ -341,13 +459,14 @@ int eora_solve(const eora_solve_config* cfg, const float* w, const float* w_hat,
   float* Y = reinterpret_cast<float*>(ws + p.off_y);
   float* Q = reinterpret_cast<float*>(ws + p.off_q);
   float* Z = reinterpret_cast<float*>(ws + p.off_z);
+  float* Wm = reinterpret_cast<float*>(ws + p.off_w);
   float* U = reinterpret_cast<float*>(ws + p.off_u);
   double* S = reinterpret_cast<double*>(ws + p.off_s);
   double* H = reinterpret_cast<double*>(ws + p.off_h);
   double* V = reinterpret_cast<double*>(ws + p.off_v);
   double* lam = reinterpret_cast<double*>(ws + p.off_lam);
   float* Vf = reinterpret_cast<float*>(ws + p.off_vf);
-  const int d = p.d, k = p.k, n = p.n, r = p.r, m = p.m;
+  const int d = p.d, k = p.k, n = p.n, r = p.r, m = p.m, ldm = p.ldm;
 
   // step 1
   k_sub<<<592, 256, 0, st>>>(w, w_hat, dW, (int64_t)d * k);
@@ -356,22 +475,22 @@ int eora_solve(const eora_solve_config* cfg, const float* w, const float* w_hat,
   CK(sgemm(st, d, k, k, dW, k, false, G, k, false, T, k));                    // T = dW G
   CK(sgemm(st, d, d, k, T, k, false, dW, k, true, Mm, d));                    // Mm = T dW^T
   // step 5: subspace iteration
-  k_init<<<592, 256, 0, st>>>(Y, (int64_t)d * m);
-  if (int rc = orthonormalise(st, p, Y, Q, S)) return rc;
+  k_init<<<592, 256, 0, st>>>(Y, d, m, ldm);
+  if (int rc = orthonormalise(st, p, Y, Q, S, Wm)) return rc;
   for (int it = 0; it < p.iters; ++it) {
-    CK(sgemm(st, d, m, d, Mm, d, false, Q, m, false, Y, m));                  // Y = Mm Q
-    if (int rc = orthonormalise(st, p, Y, Q, S)) return rc;
+    CK(sgemm(st, d, ldm, d, Mm, d, false, Q, ldm, false, Y, ldm));            // Y = Mm Q
+    if (int rc = orthonormalise(st, p, Y, Q, S, Wm)) return rc;
   }
-  if (int rc = orthonormalise(st, p, Q, Y, S)) return rc;                     // second pass: orthogonal to fp32 rounding
+  if (int rc = orthonormalise(st, p, Q, Y, S, Wm)) return rc;                 // second pass: orthogonal to fp32 rounding
   // Rayleigh-Ritz on span(Y)
-  CK(sgemm(st, d, m, d, Mm, d, false, Y, m, false, Z, m));                    // Z = Mm Y
+  CK(sgemm(st, d, ldm, d, Mm, d, false, Y, ldm, false, Z, ldm));              // Z = Mm Y
   {
     dim3 g((m + 15) / 16, (m + 15) / 16);
-    k_gram64<<<g, 256, 0, st>>>(Y, Z, d, m, H);                               // H = Y^T Mm Y
+    k_gram64<<<g, 256, 0, st>>>(Y, Z, d, m, ldm, H);                          // H = Y^T Mm Y
   }
   k_jacobi64<<<1, 1024, 0, st>>>(H, V, m, lam, Vf, 40);
   CK(cudaGetLastError());
-  CK(sgemm(st, d, r, m, Y, m, false, Vf, m, false, U, r));                    // U' = Y V[:, :r]
+  CK(sgemm(st, d, r, m, Y, ldm, false, Vf, m, false, U, r));                  // U' = Y V[:, :r]
   // step 6
   k_finish_b<<<296, 256, 0, st>>>(U, lam, d, r, b_prime, sigma);
   CK(sgemm(st, r, k, d, U, r, true, dW, k, false, a, k));                     // U'^T dW
