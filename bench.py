@@ -455,6 +455,48 @@ def time_single_layer(device: str, K: int, N: int, w: str, r: int, M: int, copie
     return e0.elapsed_time(e1) / (iters * copies)
 
 
+# Peak of the fp32 FMA pipe: 148 SMs x 128 lanes x 2 flops x 1.965 GHz (unit counts and maximum clock of the part).
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def time_solve(device: str, d: int = 4096, k: int = 4096, n: int = 2048, r: int = 128, reps: int = 3, cpu: bool = True):
+    """Extra: the offline solve (Algorithm 1 steps 1-6) of one q-shaped layer: weight 4096 x 4096, 2048 calibration
+    columns, rank 128, library defaults (32 extra vectors, 24 iterations).  Flops = those of the contractions the
+    library runs (Gram matrix, the two products that form dW' dW'^T, one product per iteration plus its
+    orthonormalisation, Rayleigh-Ritz, A); the small fp64 problems are not counted."""
+    import torch
+    import paper_2410_21271_b200 as eora
+    w, w_hat, x = gen.make_solve_case(31, d, k, n)
+    tw, th, tx = (torch.from_numpy(v).to(device) for v in (w, w_hat, x))
+    b, a, s = eora.solve(tw, th, tx, r)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        b, a, s = eora.solve(tw, th, tx, r)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    m, iters = r + 32, 24
+    ldm = (m + 127) // 128 * 128
+    flops = 2.0 * k * k * n + 2.0 * d * k * k + 2.0 * d * d * k + (iters + 1) * 2.0 * d * d * ldm + (iters + 2) * 2.0 * d * ldm * ldm + 2.0 * r * d * k
+    loss = eora.solve_loss(tw, th, tx, b, a)
+    uncompensated = float(torch.linalg.norm((tw - th).double() @ tx.double()))
+    out = {"workload": f"one layer {d}x{k}, {n} calibration columns, rank {r}", "ms": ms, "layers_per_s": 1e3 / ms,
+           "gflop": flops / 1e9, "tflops": flops / ms / 1e9, "bound": "alu", "peak_tflops_fp32": FP32_PEAK_TFLOPS,
+           "frac_of_fp32_peak": flops / ms / 1e9 / FP32_PEAK_TFLOPS,
+           "remaining_loss_over_uncompensated": loss / uncompensated, "dtype": "f32 (f64 for the small problems)"}
+    if cpu:
+        from oracle import eora_solve_oracle as sol
+        dc, kc, nc = 1024, 1024, 512
+        wc, whc, xc = gen.make_solve_case(31, dc, kc, nc)
+        t0 = time.perf_counter()
+        sol.solve(wc, whc, xc, r)
+        sec = time.perf_counter() - t0
+        out["cpu_baseline"] = {"kind": "oracle", "seconds": sec, "sample": f"one layer {dc}x{kc}, {nc} calibration columns, rank {r} (64 times fewer flops than the GPU workload)"}
+    return out
+
+
 PREFILL_SHAPES = {"q,o": (4096, 4096, 2), "k,v": (4096, 1024, 2), "gate,up": (4096, 14336, 2), "down": (14336, 4096, 1)}
 
 
@@ -634,6 +676,7 @@ def main():
     ap.add_argument("--unfused", action="store_true", help="one launch per layer (224 per token) instead of fusing q|k|v and gate|up")
     ap.add_argument("--only-prefill", action="store_true", help="run the prefill leg alone (for profiling) and print its result")
     ap.add_argument("--single-stream", action="store_true", help="launch all layers of a block in stream order")
+    ap.add_argument("--only-solve", action="store_true", help="run the offline solve leg alone (for profiling) and print its result")
     ap.add_argument("--only-few-tokens", action="store_true",
                     help="run the 64-token q-shaped layer alone (for profiling the split-reduction launches) and print its time")
     args = ap.parse_args()
@@ -676,6 +719,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(device))
         _DIST["on"] = True
 
+    if args.only_solve:
+        if rank == 0:
+            print(json.dumps({"solve": time_solve(device, cpu=False)}))
+        return
     if args.only_few_tokens:
         if rank == 0:
             ms = time_single_layer(device, 4096, 4096, "q4", RANK, 64, copies=8, iters=5)
@@ -723,6 +770,10 @@ def main():
             line["configs"] = all_configs(device, local_rank, peaks)
         except Exception as e:  # the decode line must still be printed
             line["configs"] = {"error": repr(e)}
+        try:
+            line["solve"] = time_solve(device, cpu=(world == 1))
+        except Exception as e:
+            line["solve"] = {"error": repr(e)}
     if rank == 0:
         print(json.dumps(line))
     if _DIST["on"]:

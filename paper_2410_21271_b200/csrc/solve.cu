@@ -247,20 +247,29 @@ __global__ void __launch_bounds__(1024) k_chol_inv64(double* Sg, int m, float* W
     for (int i = j + 1 + t; i < m; i += nt) S[(int64_t)i * m + j] /= ljj;
     __syncthreads();
     // trailing update of the lower triangle: S[i][c] -= L[i][j] L[c][j] for j < c <= i
-    const int rem = m - j - 1;
-    for (int e = t; e < rem * rem; e += nt) {
-      const int i = j + 1 + e / rem, c = j + 1 + e % rem;
-      if (c <= i) S[(int64_t)i * m + c] -= S[(int64_t)i * m + j] * S[(int64_t)c * m + j];
+    for (int i = j + 1 + (t >> 5); i < m; i += nt >> 5) {
+      const double lij = S[(int64_t)i * m + j];
+      for (int c = j + 1 + (t & 31); c <= i; c += 32) S[(int64_t)i * m + c] -= lij * S[(int64_t)c * m + j];
     }
     __syncthreads();
   }
-  // X = L^{-1}, one thread per column j (forward substitution down the column), kept in the strict upper triangle of S
-  // (free after the factorisation) as S[j][i] = X[i][j] for i > j; the diagonal of X is 1 / L[j][j].
-  for (int j = t; j < m; j += nt) {
-    for (int i = j + 1; i < m; ++i) {
-      double acc = S[(int64_t)i * m + j] / S[(int64_t)j * m + j];                   // L[i][j] X[j][j]
-      for (int q = j + 1; q < i; ++q) acc += S[(int64_t)i * m + q] * S[(int64_t)j * m + q];   // L[i][q] X[q][j]
-      S[(int64_t)j * m + i] = -acc / S[(int64_t)i * m + i];
+  // X = L^{-1}, one warp per column j (forward substitution down the column, the lanes share each dot product), kept
+  // in the strict upper triangle of S (free after the factorisation) as S[j][i] = X[i][j] for i > j; the diagonal of X
+  // is 1 / L[j][j].
+  {
+    const int warp = t >> 5, lane = t & 31, nwarp = nt >> 5;
+    for (int j = warp; j < m; j += nwarp) {
+      const double xjj = 1.0 / S[(int64_t)j * m + j];
+      for (int i = j + 1; i < m; ++i) {
+        double acc = 0.0;
+        for (int q = j + 1 + lane; q < i; q += 32) acc += S[(int64_t)i * m + q] * S[(int64_t)j * m + q];   // L[i][q] X[q][j]
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        acc += S[(int64_t)i * m + j] * xjj;                                                                // L[i][j] X[j][j]
+        __syncwarp();
+        if (lane == 0) S[(int64_t)j * m + i] = -acc / S[(int64_t)i * m + i];
+        __syncwarp();
+      }
     }
   }
   __syncthreads();
@@ -280,11 +289,14 @@ __global__ void __launch_bounds__(1024) k_chol_inv64(double* Sg, int m, float* W
 // CTA: pairs of columns of H are rotated until they are orthogonal; then lam_i = ||h_i|| and V holds the rotations.
 // Pairs follow the round-robin tournament (m' / 2 disjoint pairs per step, m' - 1 steps per sweep); a warp takes a pair.
 // Output: eigenvalues in descending order (lam) and the matching eigenvectors as fp32 columns of Vf ([m][m] row-major).
-__global__ void __launch_bounds__(1024) k_jacobi64(double* H, double* V, int m, double* lam, float* Vf, int max_sweeps) {
+__global__ void __launch_bounds__(1024) k_jacobi64(double* Hg, double* V, int m, double* lam, float* Vf, int max_sweeps) {
+  extern __shared__ double smj[];
   __shared__ int moved_s;
   __shared__ int rank_s[512];
   const int t = threadIdx.x, nt = blockDim.x, warp = t >> 5, lane = t & 31, nwarp = nt >> 5;
-  for (int e = t; e < m * m; e += nt) V[e] = (e / m == e % m) ? 1.0 : 0.0;
+  // the matrix whose columns are rotated is read three times per pair: in shared memory when it fits
+  double* H = m <= kCholSmem ? smj : Hg;
+  for (int e = t; e < m * m; e += nt) { V[e] = (e / m == e % m) ? 1.0 : 0.0; if (m <= kCholSmem) smj[e] = Hg[e]; }
   __syncthreads();
   const int mp = (m + 1) & ~1;                       // players of the tournament (one bye if m is odd)
   for (int sweep = 0; sweep < max_sweeps; ++sweep) {
@@ -488,7 +500,13 @@ int eora_solve(const eora_solve_config* cfg, const float* w, const float* w_hat,
     dim3 g((m + 15) / 16, (m + 15) / 16);
     k_gram64<<<g, 256, 0, st>>>(Y, Z, d, m, ldm, H);                          // H = Y^T Mm Y
   }
-  k_jacobi64<<<1, 1024, 0, st>>>(H, V, m, lam, Vf, 40);
+  {
+    static bool jattr[64] = {};
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return EORA_ERR_CUDA;
+    if (!jattr[device]) { CK(cudaFuncSetAttribute(k_jacobi64, cudaFuncAttributeMaxDynamicSharedMemorySize, kCholSmem * kCholSmem * 8)); jattr[device] = true; }
+    k_jacobi64<<<1, 1024, m <= kCholSmem ? m * m * 8 : 0, st>>>(H, V, m, lam, Vf, 40);
+  }
   CK(cudaGetLastError());
   CK(sgemm(st, d, r, m, Y, ldm, false, Vf, m, false, U, r));                  // U' = Y V[:, :r]
   // step 6

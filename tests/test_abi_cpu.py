@@ -18,14 +18,21 @@ def lib():
 
 
 def declared_functions():
-    text = open(eora.HEADER_PATH).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(eora_[a-z0-9_]+)\s*\(", text)))
+    inc = os.path.dirname(eora.HEADER_PATH)
+    names = set()
+    for h in sorted(os.listdir(inc)):                       # every header of include/
+        if not h.endswith(".h"):
+            continue
+        text = open(os.path.join(inc, h)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(eora_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol(lib):
     names = declared_functions()
-    assert {"eora_linear_create", "eora_linear_forward", "eora_linear_destroy"} <= set(names)
+    assert {"eora_linear_create", "eora_linear_forward", "eora_linear_destroy", "eora_solve", "eora_solve_loss",
+            "eora_solve_workspace_bytes"} <= set(names)
     for n in names:
         assert hasattr(lib, n), n
     assert lib.eora_version() >= 100
@@ -39,6 +46,23 @@ def test_struct_layout_matches_header():
     body = hdr[hdr.index("typedef struct {", hdr.index("} eora_linear_config;")):hdr.index("} eora_linear_weights;")]
     names = re.findall(r"const void\* (\w+);", body)
     assert names == [f[0] for f in eora.eora_linear_weights._fields_]
+
+
+def test_solve_config_layout_and_argument_checks(lib):
+    assert ctypes.sizeof(eora.eora_solve_config) == 6 * 4
+    hdr = open(os.path.join(os.path.dirname(eora.HEADER_PATH), "eora_solve.h")).read()
+    body = hdr[hdr.index("typedef struct {"):hdr.index("} eora_solve_config;")]
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    fields = [f.strip() for decl in re.findall(r"int32_t ([^;]+);", body) for f in decl.split(",")]
+    assert fields == [f[0] for f in eora.eora_solve_config._fields_]
+    good = eora.eora_solve_config(256, 128, 64, 16, 0, 0)
+    assert eora.eora_solve_workspace_bytes(good) > 4 * (256 * 128 + 128 * 128 + 256 * 256)
+    for bad in (eora.eora_solve_config(0, 128, 64, 16, 0, 0), eora.eora_solve_config(256, 128, 64, 0, 0, 0),
+                eora.eora_solve_config(256, 128, 64, 500, 100, 0), eora.eora_solve_config(8, 128, 64, 16, 0, 0)):
+        assert eora.eora_solve_workspace_bytes(bad) == 0
+    assert lib.eora_solve_workspace_bytes(None) == 0
+    assert lib.eora_solve(None, None, None, None, None, None, None, None, 0, None) == eora.EORA_ERR_NULL_ARG
+    assert lib.eora_solve_loss(None, None, None, None, None, None, None, None, 0, None) == eora.EORA_ERR_NULL_ARG
 
 
 def test_status_strings(lib):
