@@ -219,25 +219,50 @@ def time_decode(layers, xs, ys, steps: int, warmup: int, device_index: int, use_
     return ms, cs.summary(), graph is not None
 
 
-def time_e2e(layers, steps: int, warmup: int):
-    """The same step through eora_linear_forward_host: pinned host X in, host Y out, per layer."""
+def time_e2e(layers, steps: int, warmup: int, mode: str = "graph"):
+    """The same step through the host-buffer entry points: pinned host X in, host Y out, per launch unit.
+    mode "sync_each": every unit is a synchronous eora_linear_forward_host / _fused_host.
+    mode "enqueue": the launch units of a token are enqueued back to back (eora_linear_forward_host_async /
+    _fused_host_async) and the stream is synchronised once per token.
+    mode "graph": the same enqueue-only calls captured once into a CUDA graph (the copies from and to the pinned host
+    buffers are nodes of the graph); a token is one replay and one synchronisation."""
     import torch
     hx = {name: torch.from_numpy(gen.make_x(7, M_DECODE, K)).pin_memory() for name, (K, N) in LAYERS}
     hy = {name: torch.empty((M_DECODE, N), dtype=torch.float16).pin_memory() for name, (K, N) in LAYERS}
-    def step():
+
+    def enqueue(stream, sync):
         for names, K, Ns, obj in layers:
             if len(names) == 1:
-                obj.forward_host(hx[names[0]], hy[names[0]])
+                obj.forward_host(hx[names[0]], hy[names[0]], stream=stream, sync=sync)
             else:
-                obj.forward_host(hx[names[0]], [hy[n] for n in names])
-    for _ in range(max(1, warmup)):
-        step()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        step()
-    torch.cuda.synchronize()
-    sec = (time.perf_counter() - t0) / steps
+                obj.forward_host(hx[names[0]], [hy[n] for n in names], stream=stream, sync=sync)
+
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        enqueue(st, mode == "sync_each")          # first call: the handles allocate their staging buffers
+        st.synchronize()
+        if mode == "graph":
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                enqueue(st, False)
+            def step():
+                g.replay()
+                st.synchronize()
+        elif mode == "enqueue":
+            def step():
+                enqueue(st, False)
+                st.synchronize()
+        else:
+            def step():
+                enqueue(st, True)
+        for _ in range(max(1, warmup)):
+            step()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            step()
+        torch.cuda.synchronize()
+        sec = (time.perf_counter() - t0) / steps
     h2d = sum(2 * M_DECODE * K for _, K, Ns, _ in layers)
     d2h = sum(2 * M_DECODE * N for _, K, Ns, _ in layers for N in Ns)
     return sec, h2d, d2h
@@ -753,10 +778,21 @@ def main():
             "gpu_launches": n_launch_step * args.steps, "cuda_graph": graphed, "roofline": roofline}
 
     if not args.no_extras:
-        sec, h2d, d2h = time_e2e(layers, max(2, min(args.steps, 10)), 1)
+        n_e2e = max(2, min(args.steps, 10))
+        try:
+            sec, h2d, d2h = time_e2e(layers, n_e2e, 3, "graph")
+            how = "captured once into a CUDA graph, one replay and one stream synchronisation per token"
+        except Exception:                           # capture refused: enqueue directly
+            sec, h2d, d2h = time_e2e(layers, n_e2e, 3, "enqueue")
+            how = "one stream synchronisation per token"
         sec = max_over_ranks(sec)
+        sec_enq = max_over_ranks(time_e2e(layers, n_e2e, 1, "enqueue")[0])
+        sec_sync = max_over_ranks(time_e2e(layers, n_e2e, 1, "sync_each")[0])
         line["e2e"] = {"value": world * M_DECODE / sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                       "note": "per launch unit: pinned host X -> device, the layer(s), Y -> host, stream sync"}
+                       "note": "per launch unit: pinned host X -> device, the layer(s), Y -> pinned host, enqueued with "
+                               "eora_linear_forward_host_async / _fused_host_async; " + how,
+                       "enqueued_without_graph": world * M_DECODE / sec_enq,
+                       "with_a_synchronisation_per_launch_unit": world * M_DECODE / sec_sync}
     for _, _, _, obj in layers:
         obj.close()
     if not args.no_extras and rank == 0:

@@ -184,6 +184,17 @@ int eora_linear_forward_fused_host(eora_linear_t h, const void* x_host, int32_t 
  */
 int eora_linear_forward_host(eora_linear_t h, const void* x_host, int32_t m, void* y_host, void* stream);
 
+/*
+ * The host-buffer forwards without the synchronisation at the end: the copy of x_host, the launch(es) and the copy (or
+ * the kernel's own stores) into y_host / ys_host are enqueued on `stream` and the call returns.  x_host must stay
+ * unchanged and y_host unread until the caller has synchronised the stream; both should be page-locked (pageable
+ * memory makes the copies synchronous).  The staging buffers belong to the handle, so calls on ONE handle must use
+ * one stream (they are then ordered); different handles are independent.  A token's worth of layers can so be
+ * enqueued back to back and synchronised once.
+ */
+int eora_linear_forward_host_async(eora_linear_t h, const void* x_host, int32_t m, void* y_host, void* stream);
+int eora_linear_forward_fused_host_async(eora_linear_t h, const void* x_host, int32_t m, void* const* ys_host, void* stream);
+
 /* Free everything the handle owns.  NULL is a no-op.  The caller must have synchronised. */
 int eora_linear_destroy(eora_linear_t h);
 

@@ -70,6 +70,10 @@ def lib() -> ctypes.CDLL:
         L.eora_linear_forward_fused.restype = c_int
         L.eora_linear_forward_fused_host.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
         L.eora_linear_forward_fused_host.restype = c_int
+        L.eora_linear_forward_host_async.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_forward_host_async.restype = c_int
+        L.eora_linear_forward_fused_host_async.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
+        L.eora_linear_forward_fused_host_async.restype = c_int
         L.eora_linear_create_multi.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p]
         L.eora_linear_create_multi.restype = c_int
         L.eora_linear_forward_multi.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p]
@@ -166,6 +170,21 @@ def eora_linear_forward(handle: int, x, m: int, y, stream=None, check: bool = Tr
     st = lib().eora_linear_forward(handle, _ptr(x), int(m), _ptr(y), _stream(stream))
     if check and st != EORA_OK:
         raise EoraError(st, "eora_linear_forward")
+    return st
+
+
+def eora_linear_forward_host_async(handle: int, x_host, m: int, y_host, stream=None, check: bool = True) -> int:
+    st = lib().eora_linear_forward_host_async(handle, _ptr(x_host), int(m), _ptr(y_host), _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward_host_async")
+    return st
+
+
+def eora_linear_forward_fused_host_async(handle: int, x_host, m: int, ys_host, stream=None, check: bool = True) -> int:
+    arr = (c_void_p * len(ys_host))(*[_ptr(y) for y in ys_host])
+    st = lib().eora_linear_forward_fused_host_async(handle, _ptr(x_host), int(m), arr, _stream(stream))
+    if check and st != EORA_OK:
+        raise EoraError(st, "eora_linear_forward_fused_host_async")
     return st
 
 
@@ -381,8 +400,8 @@ class Layer:
         eora_linear_forward(self.handle, x, m, y, stream)
         return y
 
-    def forward_host(self, x_host, y_host, stream=None):
-        eora_linear_forward_host(self.handle, x_host, x_host.shape[0], y_host, stream)
+    def forward_host(self, x_host, y_host, stream=None, sync: bool = True):
+        (eora_linear_forward_host if sync else eora_linear_forward_host_async)(self.handle, x_host, x_host.shape[0], y_host, stream)
         return y_host
 
     def path(self, m: int) -> int:
@@ -442,8 +461,8 @@ class FusedLayers:
         eora_linear_forward_fused(self.handle, x, m, ys, stream)
         return ys
 
-    def forward_host(self, x_host, ys_host, stream=None):
-        eora_linear_forward_fused_host(self.handle, x_host, x_host.shape[0], ys_host, stream)
+    def forward_host(self, x_host, ys_host, stream=None, sync: bool = True):
+        (eora_linear_forward_fused_host if sync else eora_linear_forward_fused_host_async)(self.handle, x_host, x_host.shape[0], ys_host, stream)
         return ys_host
 
     def launches(self, m: int) -> int:

@@ -79,3 +79,31 @@ def test_multi_adapter_handle_is_refused_by_the_fused_entry_points():
     assert eora.eora_linear_forward(Lm.handle, x, 2, y, check=False) == eora.EORA_ERR_UNSUPPORTED
     torch.cuda.synchronize()
     Lm.close()
+
+
+def test_host_forwards_enqueued_back_to_back():
+    """The enqueue-only host-buffer forwards: several layers and a fused pair on one stream, one synchronisation, every
+    result against the oracle; a second round reuses the handles' staging buffers."""
+    import torch
+    K = 512
+    cases = [make_case(60 + i, K, N, 64, w="q4") for i, N in enumerate((96, 256, 160))]
+    Ls = [eora.Layer(wf, af, bf, max_m=8) for wf, af, bf in cases]
+    fused = [make_case(70 + i, K, N, 64, w="q3") for i, N in enumerate((128, 64))]
+    F = eora.FusedLayers(fused, max_m=8)
+    for M in (1, 5):
+        xs = [gen.make_x(80 + i, M, K) for i in range(4)]
+        hx = [torch.from_numpy(x.copy()).pin_memory() for x in xs]
+        hy = [torch.zeros((M, N), dtype=torch.float16).pin_memory() for N in (96, 256, 160)]
+        hf = [torch.zeros((M, N), dtype=torch.float16).pin_memory() for N in (128, 64)]
+        for L, x, y in zip(Ls, hx, hy):
+            L.forward_host(x, y, sync=False)
+        F.forward_host(hx[3], hf, sync=False)
+        torch.cuda.synchronize()
+        for (wf, af, bf), x, y in zip(cases, xs, hy):
+            check_parity(y.numpy().astype(np.float64), orc.forward(x, "f16", wf, af, bf), f"enqueued M{M}")
+        for (wf, af, bf), y in zip(fused, hf):
+            check_parity(y.numpy().astype(np.float64), orc.forward(xs[3], "f16", wf, af, bf), f"enqueued fused M{M}")
+    for L in Ls:
+        assert L.device_status() == 0
+        L.close()
+    F.close()
