@@ -219,69 +219,83 @@ __global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, con
 // shared memory when it fits (m <= kCholSmem), else in place in global memory.  A small multiple of the trace is added
 // to the diagonal first, so that a rank-deficient iterate still factors.
 constexpr int kCholSmem = 160;
+// The factorisation proper on a matrix S with row stride m (shared or global memory, the code is the same).
+__device__ __forceinline__ void chol_inverse_in_place(double* S, const int m, double* shift_slot) {
+  const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+  if (warp == 0) {
+    double tr = 0.0;
+    for (int i = lane; i < m; i += 32) tr += S[i * m + i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
+    if (lane == 0) *shift_slot = 1e-13 * tr + 1e-300;
+  }
+  __syncthreads();
+  const double shift = *shift_slot;
+  for (int i = t; i < m; i += 1024) S[i * m + i] += shift;
+  __syncthreads();
+  for (int j = 0; j < m; ++j) {
+    // every thread computes the pivot itself (one barrier less per column)
+    const double v = S[j * m + j];
+    const double ljj = sqrt(v > shift * 1e-3 ? v : shift * 1e-3);
+    const double inv = 1.0 / ljj;
+    __syncthreads();                                   // everybody has read the pivot before it is overwritten
+    if (t == 0) S[j * m + j] = ljj;
+    for (int i = j + 1 + t; i < m; i += 1024) S[i * m + j] *= inv;
+    __syncthreads();
+    // trailing update of the lower triangle, a warp per row: S[i][c] -= L[i][j] L[c][j] for j < c <= i
+    for (int i = j + 1 + warp; i < m; i += 32) {
+      double* row = S + i * m;
+      const double lij = row[j];
+      for (int c = j + 1 + lane; c <= i; c += 32) row[c] -= lij * S[c * m + j];
+    }
+    __syncthreads();
+  }
+  // X = L^{-1}, a warp per column j (forward substitution down the column, the lanes share each dot product), kept in
+  // the strict upper triangle of S (free after the factorisation) as S[j][i] = X[i][j]; the diagonal of X is 1 / L[j][j].
+  for (int j = warp; j < m; j += 32) {
+    double* xr = S + j * m;                            // row j of the upper triangle: X[.][j]
+    const double xjj = 1.0 / xr[j];
+    for (int i = j + 1; i < m; ++i) {
+      const double* li = S + i * m;
+      double acc = 0.0;
+      for (int q = j + 1 + lane; q < i; q += 32) acc += li[q] * xr[q];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      __syncwarp();
+      if (lane == 0) xr[i] = -(acc + li[j] * xjj) / li[i];
+      __syncwarp();
+    }
+  }
+  __syncthreads();
+}
+
+// Cholesky S = L L^T (fp64) of an m x m Gram matrix and the inverse of the factor, by one CTA: writes W = L^{-T} as fp32
+// into an [ld][ld] matrix (zero outside its upper triangle), so that Q = Y W is orth(Y).  The matrix is worked on in
+// shared memory when it fits (m <= kCholSmem), else in place in global memory.  A small multiple of the trace is added
+// to the diagonal first, so that a rank-deficient iterate still factors.
 __global__ void __launch_bounds__(1024) k_chol_inv64(double* Sg, int m, float* W, int ld) {
   extern __shared__ double sm[];
   __shared__ double shift_s;
-  const int t = threadIdx.x, nt = blockDim.x;
+  const int t = threadIdx.x;
   const bool in_smem = m <= kCholSmem;
-  double* S = in_smem ? sm : Sg;
   if (in_smem) {
-    for (int e = t; e < m * m; e += nt) sm[e] = Sg[e];
+    for (int e = t; e < m * m; e += 1024) sm[e] = Sg[e];
     __syncthreads();
+    chol_inverse_in_place(sm, m, &shift_s);
+  } else {
+    chol_inverse_in_place(Sg, m, &shift_s);
   }
-  if (t == 0) {
-    double tr = 0.0;
-    for (int i = 0; i < m; ++i) tr += S[(int64_t)i * m + i];
-    shift_s = 1e-13 * tr + 1e-300;
-  }
-  __syncthreads();
-  for (int i = t; i < m; i += nt) S[(int64_t)i * m + i] += shift_s;
-  __syncthreads();
-  for (int j = 0; j < m; ++j) {
-    if (t == 0) {
-      const double v = S[(int64_t)j * m + j];
-      S[(int64_t)j * m + j] = sqrt(v > shift_s * 1e-3 ? v : shift_s * 1e-3);
-    }
-    __syncthreads();
-    const double ljj = S[(int64_t)j * m + j];
-    for (int i = j + 1 + t; i < m; i += nt) S[(int64_t)i * m + j] /= ljj;
-    __syncthreads();
-    // trailing update of the lower triangle: S[i][c] -= L[i][j] L[c][j] for j < c <= i
-    for (int i = j + 1 + (t >> 5); i < m; i += nt >> 5) {
-      const double lij = S[(int64_t)i * m + j];
-      for (int c = j + 1 + (t & 31); c <= i; c += 32) S[(int64_t)i * m + c] -= lij * S[(int64_t)c * m + j];
-    }
-    __syncthreads();
-  }
-  // X = L^{-1}, one warp per column j (forward substitution down the column, the lanes share each dot product), kept
-  // in the strict upper triangle of S (free after the factorisation) as S[j][i] = X[i][j] for i > j; the diagonal of X
-  // is 1 / L[j][j].
-  {
-    const int warp = t >> 5, lane = t & 31, nwarp = nt >> 5;
-    for (int j = warp; j < m; j += nwarp) {
-      const double xjj = 1.0 / S[(int64_t)j * m + j];
-      for (int i = j + 1; i < m; ++i) {
-        double acc = 0.0;
-        for (int q = j + 1 + lane; q < i; q += 32) acc += S[(int64_t)i * m + q] * S[(int64_t)j * m + q];   // L[i][q] X[q][j]
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        acc += S[(int64_t)i * m + j] * xjj;                                                                // L[i][j] X[j][j]
-        __syncwarp();
-        if (lane == 0) S[(int64_t)j * m + i] = -acc / S[(int64_t)i * m + i];
-        __syncwarp();
-      }
-    }
-  }
-  __syncthreads();
+  const double* S = in_smem ? sm : Sg;
   // W[j][i] = X[i][j] (upper triangle of W = L^{-T}); everything else zero
-  for (int e = t; e < ld * ld; e += nt) {
-    const int j = e / ld, i = e % ld;
-    float v = 0.f;
-    if (j < m && i < m) {
-      if (i == j) v = (float)(1.0 / S[(int64_t)j * m + j]);
-      else if (i > j) v = (float)S[(int64_t)j * m + i];
+  for (int j = t >> 5; j < ld; j += 32) {
+    for (int i = t & 31; i < ld; i += 32) {
+      float v = 0.f;
+      if (j < m && i < m) {
+        if (i == j) v = (float)(1.0 / S[j * m + j]);
+        else if (i > j) v = (float)S[j * m + i];
+      }
+      W[j * ld + i] = v;
     }
-    W[e] = v;
   }
 }
 
