@@ -279,7 +279,8 @@ __device__ __forceinline__ void finish_row_tile(const DecodeArgs& p, uint32_t ti
 }
 
 // One segment: `n` consecutive blobs of one matrix starting at blob index b0.
-template <int FMT, bool HILO, int OUT>
+// I8M: backbone blobs of a launch with two to eight tokens go through the integer product (blob_product_i8m).
+template <int FMT, bool HILO, int OUT, bool I8M = false>
 __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32_t b0, uint32_t n, uint32_t nt, uint32_t blob_b,
                                             uint32_t per_copy, uint32_t sz2, int lane) {
   if constexpr (FMT == FMT_NONE) {
@@ -288,6 +289,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
     if (n == 0) return true;
     uint32_t pair = b0 / nt, tile = b0 - pair * nt;
     uint32_t xr[16], xl[16];
+    XI8M xm;
+    const bool x_bf16 = p.x_dtype == EORA_X_BF16;
     uint32_t sub = 0, sub_end = nt;
     Flush fl = OUT == OUT_T ? make_flush(p.d_t, p.r_pad, p.m, lane) : make_flush(p.y_ws, p.n_pad, p.m, lane);
     if constexpr (HILO) {
@@ -304,6 +307,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
         if (i < p.n_sub && tile >= p.sub_tile0[i]) sub = i;
       sub_end = p.sub_tile0[sub + 1];
       load_t_pair(xr, xl, p, sub * p.b_np + pair, lane);
+    } else if constexpr (I8M) {
+      load_x_i8m<FMT>(xm, p.x, x_bf16, p.m, p.d_in, pair, lane);
     } else {
       load_x_pair(xr, p, pair, lane);
     }
@@ -343,7 +348,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
 #pragma unroll 2
       for (uint32_t j = 0; j < cn; ++j) {
         float tot[4];
-        blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
+        if constexpr (I8M) blob_product_i8m<FMT>(src + j * blob_b, lane, sz2, xm, tot);
+        else blob_product<FMT, HILO>(src + j * blob_b, lane, sz2, xr, xl, tot, r.aux);
         if constexpr (OUT == OUT_T) {
           flush_sums(fl, tile, tot);
           ++flushed;
@@ -359,6 +365,8 @@ __device__ __forceinline__ bool run_segment(const DecodeArgs& p, Ring& r, uint32
             if constexpr (HILO) {
               sub = 0; sub_end = p.sub_tile0[1];
               load_t_pair(xr, xl, p, pair, lane);
+            } else if constexpr (I8M) {
+              load_x_i8m<FMT>(xm, p.x, x_bf16, p.m, p.d_in, pair, lane);
             } else {
               load_x_pair(xr, p, pair, lane);
             }
@@ -495,17 +503,20 @@ __device__ __forceinline__ bool run_backbone_i8(const DecodeArgs& p, Ring& r, Wa
   return true;
 }
 
-template <int WF, bool I8>
+template <int WF, int I8>
 __device__ __forceinline__ bool run_backbone(const DecodeArgs& p, Ring& r, WalkI8& w, uint32_t first, uint32_t count, uint32_t blob_w, int lane) {
-  if constexpr (I8) {
+  if constexpr (I8 == 2) {
+    return run_segment<WF, false, OUT_Y, true>(p, r, first, count, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
+  } else if constexpr (I8 == 1) {
     return p.w_sz2 ? run_backbone_i8<WF, true>(p, r, w, first, count, lane) : run_backbone_i8<WF, false>(p, r, w, first, count, lane);
   } else {
     return run_segment<WF, false, OUT_Y>(p, r, first, count, p.w_nt, blob_w, p.w_per_copy, p.w_sz2, lane);
   }
 }
 
-// I8: the launch has one token and the backbone goes through the integer inner product.
-template <int WF, int ABF, bool I8>
+// I8: the backbone goes through the integer inner product -- 1: one token (the walk above), 2: two to eight tokens
+// (tokens as the columns of the narrow operand, two byte planes = two MMAs per weight fragment), 0: fp16 product.
+template <int WF, int ABF, int I8>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_constant__ DecodeArgs p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -587,7 +598,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   if (tr && lane == 0) tr[1] = globaltimer_ns();
 
   WalkI8 wk;
-  if constexpr (I8) {
+  if constexpr (I8 == 1) {
     wk.pair = kNone; wk.next_b = kNone; wk.tile = 0; wk.yb = p.y_ws; wk.my_tile = 0; wk.batch_n = 0; wk.tk_n = 0; wk.tk_old = 0; wk.tk_tile = 0;
   }
   bool ok = true;
@@ -598,7 +609,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
     if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
     if (ok) ok = run_backbone<WF, I8>(p, r, wk, w0 + wf, wn - wf, blob_w, lane);
   }
-  if constexpr (I8) {
+  if constexpr (I8 == 1) {
     if (ok) { tickets_take(p, wk, lane); tickets_resolve(p, wk, lane); }
   }
   if (!ok) {
@@ -625,7 +636,7 @@ cudaError_t launch_kernel(const cudaLaunchConfig_t& cfg, const DecodeArgs& args,
 // Formats whose backbone blobs have an integer inner product.
 constexpr bool has_i8(int fmt) { return fmt == FMT_Q4 || fmt == FMT_Q3; }
 
-template <int WF, bool I8>
+template <int WF, int I8>
 cudaError_t launch_ab2(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf, int device) {
   switch (abf) {
     case FMT_F16: return launch_kernel<k_decode<WF, FMT_F16, I8>>(cfg, args, device);
@@ -638,9 +649,10 @@ cudaError_t launch_ab2(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, in
 template <int WF>
 cudaError_t launch_ab(const cudaLaunchConfig_t& cfg, const DecodeArgs& args, int abf, int device) {
   if constexpr (has_i8(WF)) {
-    if (args.m == 1) return launch_ab2<WF, true>(cfg, args, abf, device);
+    if (args.m == 1) return launch_ab2<WF, 1>(cfg, args, abf, device);
+    return launch_ab2<WF, 2>(cfg, args, abf, device);
   }
-  return launch_ab2<WF, false>(cfg, args, abf, device);
+  return launch_ab2<WF, 0>(cfg, args, abf, device);
 }
 
 // Relative cost of one blob (time a warp spends on it); only the ratios matter.
@@ -722,7 +734,7 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
   const uint32_t nw = (uint32_t)grid * kWarps;
   if (ab) {
     // with one token the backbone blobs go through the integer inner product, which is cheaper
-    const bool i8 = m == 1 && (h->w.fmt == FMT_Q4 || h->w.fmt == FMT_Q3);
+    const bool i8 = h->w.fmt == FMT_Q4 || h->w.fmt == FMT_Q3;       // (one to eight tokens: this function's passes)
     uint32_t n1 = a.a_blobs < nw / 3 ? a.a_blobs : nw / 3;
     uint32_t n3 = b_blobs < nw / 3 ? b_blobs : nw / 3;
     if (n1 < 1) n1 = 1;

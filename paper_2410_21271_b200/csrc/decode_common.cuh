@@ -495,6 +495,126 @@ __device__ __forceinline__ void blob_product_i8(const uint8_t* blob_l, const uin
   }
 }
 
+// ---- the same integer product for two to eight tokens -------------------------------------------------------------
+// Tokens are the columns of the MMA's narrow operand: lane (g, t) holds, for token g, the eight reduction elements
+// 32 j + 8 t .. + 7 of MMA j -- exactly the sixteen bytes per MMA that it loads from its token's row -- as a low and a
+// high byte plane (two MMAs per weight fragment instead of one).  Every token has its own block scale and sums; the
+// accumulator of lane (g, t) belongs to tokens 2t and 2t + 1, whose scale and sums it fetches once per pair.
+struct XI8M {
+  uint32_t lo[4][2], hi[4][2];   // narrow-operand registers of the four MMAs of a pair, low and high plane (token g)
+  float scale[2];                // 2^e of tokens 2t, 2t + 1
+  int sum[2][2];                 // [token 2t + i][tile c]: sum of v over the tile
+};
+
+template <int FMT>
+__device__ __forceinline__ void load_x_i8m(XI8M& xm, const void* x, bool bf16, int m, int d_in, uint32_t pair, int lane) {
+  const int g = lane >> 2, t = lane & 3;
+  float f[4][8];
+  if (g < m) {
+    const uint16_t* src = reinterpret_cast<const uint16_t*>(x) + (size_t)g * d_in + pair * 128 + 8 * t;
+    uint4 u[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(u[j].x), "=r"(u[j].y), "=r"(u[j].z), "=r"(u[j].w) : "l"(src + 32 * j) : "memory");
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t w[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (bf16) { f[j][2 * e] = __uint_as_float(w[e] << 16); f[j][2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u); }
+        else { const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&w[e])); f[j][2 * e] = v.x; f[j][2 * e + 1] = v.y; }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[j][e] = 0.f;
+  }
+  float am = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) am = fmaxf(am, fabsf(f[j][e]));
+  am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, 1));
+  am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, 2));               // the token's 128 elements sit in its four lanes
+  const uint32_t eb = __float_as_uint(am * 1.00396f) >> 23;
+  const bool live = eb >= 15u && eb < 255u;
+  const float inv = live ? __uint_as_float((268u - eb) << 23) : 0.f;
+  const float my_scale = live ? __uint_as_float((eb - 14u) << 23) : 0.f;
+  int my_sum[2] = {0, 0};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    int v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { v[e] = __float2int_rn(f[j][e] * inv); my_sum[j >> 1] += v[e]; }
+    uint32_t l0 = prmt(prmt(v[0], v[1], 0x0040u), prmt(v[2], v[3], 0x0040u), 0x5410u);
+    uint32_t l1 = prmt(prmt(v[4], v[5], 0x0040u), prmt(v[6], v[7], 0x0040u), 0x5410u);
+    uint32_t h0 = prmt(prmt(v[0] + 128, v[1] + 128, 0x0051u), prmt(v[2] + 128, v[3] + 128, 0x0051u), 0x5410u);
+    uint32_t h1 = prmt(prmt(v[4] + 128, v[5] + 128, 0x0051u), prmt(v[6] + 128, v[7] + 128, 0x0051u), 0x5410u);
+    if constexpr (FMT == FMT_Q4) {                 // the and-or delivers the codes as (0, 4, 1, 5) and (2, 6, 3, 7)
+      const uint32_t a = prmt(l0, l1, 0x5140u), b = prmt(l0, l1, 0x7362u), c = prmt(h0, h1, 0x5140u), d = prmt(h0, h1, 0x7362u);
+      l0 = a; l1 = b; h0 = c; h1 = d;
+    }
+    xm.lo[j][0] = l0; xm.lo[j][1] = l1; xm.hi[j][0] = h0; xm.hi[j][1] = h1;
+  }
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    my_sum[c] += __shfl_xor_sync(0xffffffffu, my_sum[c], 1);
+    my_sum[c] += __shfl_xor_sync(0xffffffffu, my_sum[c], 2);
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {                    // what belongs to the accumulator's columns: tokens 2t and 2t + 1
+    const int from = (2 * t + i) * 4;
+    xm.scale[i] = __shfl_sync(0xffffffffu, my_scale, from);
+    xm.sum[i][0] = __shfl_sync(0xffffffffu, my_sum[0], from);
+    xm.sum[i][1] = __shfl_sync(0xffffffffu, my_sum[1], from);
+  }
+}
+
+// tot[i] as the accumulator of mma.m16n8k16: (row g, token 2t), (row g, token 2t + 1), (row g + 8, token 2t), (row g + 8, 2t + 1).
+template <int FMT>
+__device__ __forceinline__ void blob_product_i8m(const uint8_t* blob, int lane, uint32_t sz2, const XI8M& xm, float (&tot)[4]) {
+  constexpr int tb = tile_bytes(FMT);
+  const int g = lane >> 2;
+  const uint8_t* blob_l = blob + (FMT == FMT_Q4 ? 16 : 8) * lane;
+  const uint8_t* blob_g = blob + 4 * g;
+  tot[0] = tot[1] = tot[2] = tot[3] = 0.f;
+  int z_a = 0, z_b = 0;
+  float s_a = 0.f, s_b = 0.f;
+  int zs[2] = {0, 0};                    // sum of v over the tiles of the current scale entry, tokens 2t and 2t + 1
+  int dl[4] = {0, 0, 0, 0}, dh[4] = {0, 0, 0, 0};
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    if (c == 0 || sz2) {
+      const uint8_t* sz = blob_g + 2 * tb + c * kSzEntryBytes;
+      const uint32_t s2 = *reinterpret_cast<const uint32_t*>(sz);
+      const uint32_t z2 = *reinterpret_cast<const uint16_t*>(sz + 32 - 2 * g);
+      z_a = (int)(z2 & 255u); z_b = (int)(z2 >> 8);
+      const float2 sf = __half22float2(*reinterpret_cast<const __half2*>(&s2));
+      s_a = sf.x; s_b = sf.y;
+      zs[0] = zs[1] = 0;
+    }
+    zs[0] += xm.sum[0][c];
+    zs[1] += xm.sum[1][c];
+    uint32_t q[4][2];
+    tile_quads<FMT>(blob_l + c * tb, lane, q);
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+      mma16832_s8(dl, q[2 * blk][0], q[2 * blk + 1][0], q[2 * blk][1], q[2 * blk + 1][1], xm.lo[2 * c + blk][0], xm.lo[2 * c + blk][1]);
+      mma16832_s8(dh, q[2 * blk][0], q[2 * blk + 1][0], q[2 * blk][1], q[2 * blk + 1][1], xm.hi[2 * c + blk][0], xm.hi[2 * c + blk][1]);
+    }
+    if (c == 1 || sz2) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int tok = i & 1, z = i < 2 ? z_a : z_b;
+        const float s = (i < 2 ? s_a : s_b) * xm.scale[tok];
+        tot[i] = fmaf((float)(dh[i] * 256 + dl[i] - z * zs[tok]), s, tot[i]);
+        dl[i] = 0; dh[i] = 0;
+      }
+    }
+  }
+}
+
 __device__ __forceinline__ void store_y(void* y, int dtype, int64_t i, float v) {
   if (dtype == EORA_Y_F16) reinterpret_cast<__half*>(y)[i] = __float2half_rn(v);
   else if (dtype == EORA_Y_BF16) reinterpret_cast<__nv_bfloat16*>(y)[i] = __float2bfloat16_rn(v);
