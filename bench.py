@@ -318,11 +318,16 @@ def time_prefill(device: str, steps: int = 10, warmup: int = 3, layer_set: bool 
 
 
 def kernel_sources_sha() -> str:
-    """Hash of the decode kernel's sources: the DRAM traffic taken with ncu is only valid for the code it was taken on."""
+    """Hash of the decode kernel's code (comments and white space left out): the DRAM traffic taken with ncu is only
+    valid for the code it was taken on."""
     import hashlib
+    import re
     h = hashlib.sha256()
     for f in ("decode.cu", "decode_common.cuh", "eora_common.cuh"):
-        h.update(open(os.path.join(ROOT, "paper_2410_21271_b200", "csrc", f), "rb").read())
+        text = open(os.path.join(ROOT, "paper_2410_21271_b200", "csrc", f)).read()
+        text = re.sub(r"/\*.*?\*/", " ", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", " ", text)
+        h.update(" ".join(text.split()).encode())
     return h.hexdigest()[:16]
 
 

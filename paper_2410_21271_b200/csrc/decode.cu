@@ -5,8 +5,11 @@
 // Work decomposition.  All three matrices are stored as blobs of 16 rows x 128 reduction elements,
 // ordered pair-major (see eora_common.cuh), and every blob is an independent piece of work: a warp
 // multiplies it with the 128 activations it needs (kept in registers as tensor-core operand
-// fragments, tokens as the n8 side of mma.m16n8k16) and adds the 16 x m partial sums to an fp32
-// accumulator array in global memory with red.add.  Warps are fully independent: each owns a
+// fragments, tokens as the n8 side of the MMA) and adds the 16 x m partial sums to an fp32
+// accumulator array in global memory with red.add.  Blobs of a 3/4-bit backbone go through an integer
+// product (mma.m16n8k32 on the byte codes against two byte planes of 16-bit block fixed point activations,
+// see decode_common.cuh), all other blobs (adapters, 2:4 backbones) are dequantised to exact fp16 integers
+// and go through mma.m16n8k16.  Warps are fully independent: each owns a
 // contiguous run of blobs of up to three matrices, fetches it with its own bulk copies into its own
 // shared-memory ring and never synchronises with another warp of its CTA.
 //
@@ -587,9 +590,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
     r.ptr[2] = p.w_q + (size_t)(w0 + wf) * blob_w; r.rem[2] = wn - wf; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
   }
 
-  // Before the dependency resolves only two of the three first copies per warp are requested:
-  // the activations are read right after the wait, and their loads would otherwise queue behind 29 MB of
-  // weight requests.
+  // Before the dependency resolves at most two first copies per warp are requested (with a deeper ring the others
+  // follow the loads of the activations, which are read right after the wait and would otherwise queue behind the
+  // weight requests).
   ring_issue(r, 0, lane);
   ring_issue(r, 1, lane);
   r.deferred = kRing - 2;
