@@ -14,8 +14,9 @@
 // shared-memory ring and never synchronises with another warp of its CTA.
 //
 //   * the first warps ("A owners") take the blobs of A first (t += X . A, sums in d_t) and then a share of W,
-//   * the last warps ("B owners") take a share of W, then their blobs of B, for which the activations are t
+//   * the last warps ("B owners") take one copy of W, then their blobs of B, for which the activations are t
 //     (read back as fp32 and split into an fp16 high and low part, so that t keeps fp32-like accuracy),
+//     then the rest of their share of W,
 //   * the warps in between take backbone blobs only.
 // The only wait in the kernel is the one before the B share: all of A must have been added to t.  A
 // owners never wait, and they sit in the first half of the CTAs, which are dispatched first and hold no B
@@ -575,18 +576,18 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
     bb0 = share_lo(p.sh_b, i); bn = share_n(p.sh_b, i);
   }
   const uint32_t blob_a = blob_bytes(ABF, p.a_sz2), blob_w = blob_bytes(WF, p.w_sz2), blob_b = blob_bytes(ABF, p.b_sz2);
-  // Order of the runs.  A owners: A, then W.  B owners: W, then B: by then t is complete more often than not (with B
-  // in the middle of the W share, as it was, a B owner of a small layer stood waiting for t with work left to do),
-  // and the deal gives them fewer backbone blobs to make up for the round trips that end their run (reading t back,
-  // their own tickets).
+  // Order of the runs.  A owners: A, then W.  The others: the first copy's worth of W, then B, then the
+  // rest of W: by then t is complete, and the round trips of the B share (reading t back, its tickets)
+  // are hidden behind the other warps' W work instead of sitting at the end of the kernel.
+  const uint32_t wf = !b_owner ? wn : (wn < p.w_per_copy ? wn : p.w_per_copy);
   if (!b_owner) {
     r.ptr[0] = p.a_q + (size_t)a0 * blob_a; r.rem[0] = an; r.blob[0] = blob_a; r.per[0] = p.a_per_copy;
     r.ptr[1] = p.w_q + (size_t)w0 * blob_w; r.rem[1] = wn; r.blob[1] = blob_w; r.per[1] = p.w_per_copy;
     r.ptr[2] = p.w_q; r.rem[2] = 0; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
   } else {
-    r.ptr[0] = p.w_q + (size_t)w0 * blob_w; r.rem[0] = wn; r.blob[0] = blob_w; r.per[0] = p.w_per_copy;
+    r.ptr[0] = p.w_q + (size_t)w0 * blob_w; r.rem[0] = wf; r.blob[0] = blob_w; r.per[0] = p.w_per_copy;
     r.ptr[1] = p.b_q + (size_t)bb0 * blob_b; r.rem[1] = bn; r.blob[1] = blob_b; r.per[1] = p.b_per_copy;
-    r.ptr[2] = p.w_q; r.rem[2] = 0; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
+    r.ptr[2] = p.w_q + (size_t)(w0 + wf) * blob_w; r.rem[2] = wn - wf; r.blob[2] = blob_w; r.per[2] = p.w_per_copy;
   }
 
   // Before the dependency resolves at most two first copies per warp are requested (with a deeper ring the others
@@ -605,10 +606,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) k_decode(const __grid_co
   }
   bool ok = true;
   if (a_owner) ok = run_segment<ABF, false, OUT_T>(p, r, a0, an, p.a_nt, blob_a, p.a_per_copy, p.a_sz2, lane);
-  if (ok) ok = run_backbone<WF, I8>(p, r, wk, w0, wn, blob_w, lane);
+  if (ok) ok = run_backbone<WF, I8>(p, r, wk, w0, wf, blob_w, lane);
   if (tr && lane == 0) tr[2] = globaltimer_ns();
   if (b_owner) {
     if (ok) ok = run_segment<ABF, true, OUT_Y>(p, r, bb0, bn, p.w_nt, blob_b, p.b_per_copy, p.b_sz2, lane);
+    if (ok) ok = run_backbone<WF, I8>(p, r, wk, w0 + wf, wn - wf, blob_w, lane);
   }
   if constexpr (I8 == 1) {
     if (ok) { tickets_take(p, wk, lane); tickets_resolve(p, wk, lane); }
@@ -749,7 +751,7 @@ cudaError_t launch_decode_forward(const Handle* h, const void* x, int m, void* c
     // fixed extra cost: the A owners fetch a second set of activations, the B owners read t back and end
     // with their own round of tickets, which is latency that a warp cannot hide from itself.
     const double cw1 = blob_cost(h->w.fmt, false) * (i8 ? 0.75 : 1.0);
-    const double fixed_a = i8 ? 4.0 : 2.0, fixed_b = 13.0;
+    const double fixed_a = i8 ? 4.0 : 2.0, fixed_b = 9.0;
     const double e1 = fixed_a + (double)a.a_blobs / n1 * blob_cost(h->a.fmt, false);
     const double e3 = fixed_b + (double)b_blobs / n3 * blob_cost(h->b.fmt, true);
     const double T = (w_blobs * cw1 + n1 * e1 + n3 * e3) / nw;      // finishing time of every warp
