@@ -42,7 +42,7 @@ constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 constexpr int kCtasPerSm = 1;
 constexpr int kRing = 2;                  // bulk copies in flight per warp
-constexpr int kSlotBytes = 4352;          // one ring slot = one bulk copy (a run of whole blobs)
+constexpr int kSlotBytes = 6528;          // one ring slot = one bulk copy (a run of whole blobs: eight 3-bit, six 4-bit ones)
 constexpr int kBarBytes = 512;            // kWarps * kRing mbarriers
 constexpr int kSmemBytes = kWarps * kRing * kSlotBytes + kBarBytes + kSp24LutBytes;
 
