@@ -707,6 +707,8 @@ def main():
     ap.add_argument("--only-prefill", action="store_true", help="run the prefill leg alone (for profiling) and print its result")
     ap.add_argument("--single-stream", action="store_true", help="launch all layers of a block in stream order")
     ap.add_argument("--only-solve", action="store_true", help="run the offline solve leg alone (for profiling) and print its result")
+    ap.add_argument("--only-tmem-decode", action="store_true",
+                    help="run one block with the opt-in tensor-memory decode family at M = 1 and 16 (for profiling) and print the times")
     ap.add_argument("--only-few-tokens", action="store_true",
                     help="run the 64-token q-shaped layer alone (for profiling the split-reduction launches) and print its time")
     args = ap.parse_args()
@@ -749,6 +751,14 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(device))
         _DIST["on"] = True
 
+    if args.only_tmem_decode:
+        if rank == 0:
+            out = {}
+            res = time_decode_config(device, "q3", "f16", RANK, (1, 16), copies=2, iters=3, policy=eora.EORA_POLICY_TMEM_DECODE)
+            for M, (ms, nl) in res.items():
+                out[f"M{M}"] = {"ms_per_block": ms, "launches_per_block": nl, "GB/s": block_bytes("q3", "f16", RANK, M, True) / ms / 1e6}
+            print(json.dumps({"tmem_decode": out}))
+        return
     if args.only_solve:
         if rank == 0:
             print(json.dumps({"solve": time_solve(device, cpu=False)}))
