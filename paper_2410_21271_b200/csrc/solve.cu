@@ -214,59 +214,117 @@ __global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, con
   if (i0 + ti < m && j0 + tj < m) S[(int64_t)(i0 + ti) * m + j0 + tj] = acc;
 }
 
-// Cholesky S = L L^T (fp64) of an m x m Gram matrix and the inverse of the factor, by one CTA: writes W = L^{-T} as fp32
-// into an [ld][ld] matrix (zero outside its upper triangle), so that Q = Y W is orth(Y).  The matrix is worked on in
-// shared memory when it fits (m <= kCholSmem), else in place in global memory.  A small multiple of the trace is added
-// to the diagonal first, so that a rank-deficient iterate still factors.
+// Largest m for which the one-CTA kernels below keep their fp64 matrix in shared memory.
 constexpr int kCholSmem = 160;
-// The factorisation proper on a matrix S with row stride m (shared or global memory, the code is the same).
-__device__ __forceinline__ void chol_inverse_in_place(double* S, const int m, double* shift_slot) {
+// The factorisation proper on an m x m matrix S with row stride ls (shared or global memory, the code is the same).
+// In shared memory ls is odd: threads that walk down a column (one row each) would otherwise all hit one bank when m
+// is a multiple of 16.
+__device__ __forceinline__ void chol_inverse_in_place(double* S, const int m, const int ls, double* shift_slot, double* scratch) {
   const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
   if (warp == 0) {
     double tr = 0.0;
-    for (int i = lane; i < m; i += 32) tr += S[i * m + i];
+    for (int i = lane; i < m; i += 32) tr += S[i * ls + i];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
     if (lane == 0) *shift_slot = 1e-13 * tr + 1e-300;
   }
   __syncthreads();
   const double shift = *shift_slot;
-  for (int i = t; i < m; i += 1024) S[i * m + i] += shift;
+  for (int i = t; i < m; i += 1024) S[i * ls + i] += shift;
   __syncthreads();
-  for (int j = 0; j < m; ++j) {
-    // every thread computes the pivot itself (one barrier less per column)
-    const double v = S[j * m + j];
-    const double ljj = sqrt(v > shift * 1e-3 ? v : shift * 1e-3);
-    const double inv = 1.0 / ljj;
-    __syncthreads();                                   // everybody has read the pivot before it is overwritten
-    if (t == 0) S[j * m + j] = ljj;
-    for (int i = j + 1 + t; i < m; i += 1024) S[i * m + j] *= inv;
-    __syncthreads();
-    // trailing update of the lower triangle, a warp per row: S[i][c] -= L[i][j] L[c][j] for j < c <= i
-    for (int i = j + 1 + warp; i < m; i += 32) {
-      double* row = S + i * m;
-      const double lij = row[j];
-      for (int c = j + 1 + lane; c <= i; c += 32) row[c] -= lij * S[c * m + j];
+  // Blocked right-looking factorisation, panels of 16 columns: (A) the 16 x 16 diagonal block by one warp, (B) the rows
+  // below it by one thread per row (forward substitution against the block), (C) the rank-16 update of the trailing
+  // lower triangle by everybody -- three barriers per panel instead of three per column.
+  constexpr int NB = 16;
+  for (int j0 = 0; j0 < m; j0 += NB) {
+    const int jb = m - j0 < NB ? m - j0 : NB;
+    if (warp == 0) {
+      for (int j = 0; j < jb; ++j) {
+        double* dj = S + (j0 + j) * ls + j0;                 // row j0 + j of the block
+        const double v = dj[j];
+        const double ljj = sqrt(v > shift * 1e-3 ? v : shift * 1e-3);
+        __syncwarp();
+        if (lane == 0) dj[j] = ljj;
+        if (lane > j && lane < jb) S[(j0 + lane) * ls + j0 + j] /= ljj;
+        __syncwarp();
+        if (lane > j && lane < jb) {
+          double* dr = S + (j0 + lane) * ls + j0;
+          const double lrj = dr[j];
+          for (int c = j + 1; c <= lane; ++c) dr[c] -= lrj * S[(j0 + c) * ls + j0 + j];
+        }
+        __syncwarp();
+      }
     }
     __syncthreads();
-  }
-  // X = L^{-1}, a warp per column j (forward substitution down the column, the lanes share each dot product), kept in
-  // the strict upper triangle of S (free after the factorisation) as S[j][i] = X[i][j]; the diagonal of X is 1 / L[j][j].
-  for (int j = warp; j < m; j += 32) {
-    double* xr = S + j * m;                            // row j of the upper triangle: X[.][j]
-    const double xjj = 1.0 / xr[j];
-    for (int i = j + 1; i < m; ++i) {
-      const double* li = S + i * m;
-      double acc = 0.0;
-      for (int q = j + 1 + lane; q < i; q += 32) acc += li[q] * xr[q];
+    for (int i = j0 + jb + t; i < m; i += 1024) {           // (B)
+      double* ri = S + i * ls + j0;
+      for (int j = 0; j < jb; ++j) {
+        const double* dj = S + (j0 + j) * ls + j0;
+        double v = ri[j];
+        for (int q = 0; q < j; ++q) v -= ri[q] * dj[q];
+        ri[j] = v / dj[j];
+      }
+    }
+    __syncthreads();
+    for (int i = j0 + jb + warp; i < m; i += 32) {          // (C)
+      const double* li = S + i * ls + j0;
+      double lr[NB];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      __syncwarp();
-      if (lane == 0) xr[i] = -(acc + li[j] * xjj) / li[i];
-      __syncwarp();
+      for (int q = 0; q < NB; ++q) lr[q] = q < jb ? li[q] : 0.0;
+      for (int c = j0 + jb + lane; c <= i; c += 32) {
+        const double* lc = S + c * ls + j0;
+        double acc = 0.0;
+#pragma unroll
+        for (int q = 0; q < NB; ++q) acc += q < jb ? lr[q] * lc[q] : 0.0;
+        S[i * ls + c] -= acc;
+      }
+    }
+    __syncthreads();
+  }
+  // X = L^{-1} by blocks of 16, kept transposed in the strict upper triangle of S (free after the factorisation):
+  // S[j][i] = X[i][j] for i > j; the diagonal of X is 1 / L[j][j].
+  //   diagonal blocks: X_bb = L_bb^{-1}, one thread per column (16 steps of forward substitution);
+  //   then block diagonal by block diagonal (distance dd = 1, 2, ...: the blocks of one diagonal are independent):
+  //     P = sum_{kb = jb}^{ib - 1} L_{ib,kb} X_{kb,jb}   (into the scratch, one thread per element),
+  //     X_{ib,jb} = - X_{ib,ib} P.
+  const int nblk = (m + NB - 1) / NB;
+  auto X_at = [&](int i, int j) -> double {               // X[i][j], i >= j
+    return i == j ? 1.0 / S[j * ls + j] : S[j * ls + i];
+  };
+  for (int j = t; j < m; j += 1024) {
+    const int b0 = (j / NB) * NB, b1 = b0 + NB < m ? b0 + NB : m;
+    const double xjj = 1.0 / S[j * ls + j];
+    for (int i = j + 1; i < b1; ++i) {
+      double acc = S[i * ls + j] * xjj;
+      for (int q = j + 1; q < i; ++q) acc += S[i * ls + q] * S[j * ls + q];
+      S[j * ls + i] = -acc / S[i * ls + i];
     }
   }
   __syncthreads();
+  for (int dd = 1; dd < nblk; ++dd) {
+    const int nb_d = nblk - dd;                            // blocks on this diagonal: (ib, jb) = (jb + dd, jb)
+    for (int e = t; e < nb_d * NB * NB; e += 1024) {
+      const int jb = e / (NB * NB), r = (e / NB) % NB, c = e % NB, ib = jb + dd;
+      const int i = ib * NB + r, j = jb * NB + c;
+      double acc = 0.0;
+      if (i < m && j < m) {
+        const double* li = S + i * ls;
+        for (int q = j; q < ib * NB; ++q) acc += li[q] * X_at(q, j);      // X[q][j] = 0 for q < j
+      }
+      scratch[e] = acc;
+    }
+    __syncthreads();
+    for (int e = t; e < nb_d * NB * NB; e += 1024) {
+      const int jb = e / (NB * NB), r = (e / NB) % NB, c = e % NB, ib = jb + dd;
+      const int i = ib * NB + r, j = jb * NB + c;
+      if (i < m && j < m) {
+        double acc = 0.0;
+        for (int q = 0; q <= r; ++q) acc += X_at(i, ib * NB + q) * scratch[(jb * NB + q) * NB + c];
+        S[j * ls + i] = -acc;
+      }
+    }
+    __syncthreads();
+  }
 }
 
 // Cholesky S = L L^T (fp64) of an m x m Gram matrix and the inverse of the factor, by one CTA: writes W = L^{-T} as fp32
@@ -278,12 +336,13 @@ __global__ void __launch_bounds__(1024) k_chol_inv64(double* Sg, int m, float* W
   __shared__ double shift_s;
   const int t = threadIdx.x;
   const bool in_smem = m <= kCholSmem;
+  const int ls = in_smem ? (m | 1) : m;
   if (in_smem) {
-    for (int e = t; e < m * m; e += 1024) sm[e] = Sg[e];
+    for (int e = t; e < m * m; e += 1024) sm[(e / m) * ls + e % m] = Sg[e];
     __syncthreads();
-    chol_inverse_in_place(sm, m, &shift_s);
+    chol_inverse_in_place(sm, m, ls, &shift_s, sm + m * ls);
   } else {
-    chol_inverse_in_place(Sg, m, &shift_s);
+    chol_inverse_in_place(Sg, m, ls, &shift_s, sm);
   }
   const double* S = in_smem ? sm : Sg;
   // W[j][i] = X[i][j] (upper triangle of W = L^{-T}); everything else zero
@@ -291,8 +350,8 @@ __global__ void __launch_bounds__(1024) k_chol_inv64(double* Sg, int m, float* W
     for (int i = t & 31; i < ld; i += 32) {
       float v = 0.f;
       if (j < m && i < m) {
-        if (i == j) v = (float)(1.0 / S[j * m + j]);
-        else if (i > j) v = (float)S[j * m + i];
+        if (i == j) v = (float)(1.0 / S[j * ls + j]);
+        else if (i > j) v = (float)S[j * ls + i];
       }
       W[j * ld + i] = v;
     }
@@ -450,9 +509,9 @@ int orthonormalise(cudaStream_t st, const Plan& p, const float* Y, float* Q, dou
   static bool attr_set[64] = {};
   int device = 0;
   if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return EORA_ERR_CUDA;
-  const int smem = p.m <= kCholSmem ? p.m * p.m * 8 : 0;
+  const int smem = (p.m <= kCholSmem ? p.m * (p.m | 1) * 8 : 0) + ((p.m + 15) / 16) * 16 * 16 * 8;     // the matrix (if it fits) and the scratch of the block inverse
   if (!attr_set[device]) {
-    CK(cudaFuncSetAttribute(k_chol_inv64, cudaFuncAttributeMaxDynamicSharedMemorySize, kCholSmem * kCholSmem * 8));
+    CK(cudaFuncSetAttribute(k_chol_inv64, cudaFuncAttributeMaxDynamicSharedMemorySize, kCholSmem * (kCholSmem | 1) * 8 + ((kCholSmem + 15) / 16) * 16 * 16 * 8));
     attr_set[device] = true;
   }
   k_chol_inv64<<<1, 1024, smem, st>>>(S, p.m, W, p.ldm);
