@@ -83,20 +83,24 @@ __global__ void __launch_bounds__(256) k_sgemm(int M, int N, int P, const float*
 
 // The same product for whole tiles (M, N multiples of 128, P of 16, rows 16-byte aligned): 16-byte global loads, the
 // next k-slice fetched into registers while the current one is multiplied.
-template <bool TA, bool TB>
+// TM: output rows per thread (8: tiles of 128 rows; 4: tiles of 64 rows, for products with few tiles).
+template <bool TA, bool TB, int TM>
 __global__ void __launch_bounds__(256) k_sgemm_full(int P, const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
                                                     float* __restrict__ C, int ldc) {
-  __shared__ __align__(16) float As[2][BKS][BM + PAD];
+  constexpr int BMT = 16 * TM, NA = TM / 4;          // tile rows; 16-byte pieces of the A tile per thread
+  __shared__ __align__(16) float As[2][BKS][BMT + PAD];
   __shared__ __align__(16) float Bs[2][BKS][BN + PAD];
   const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
-  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const int m0 = blockIdx.y * BMT, n0 = blockIdx.x * BN;
   // this thread's two 16-byte pieces of each operand tile
   // A not transposed: tile rows m (128) x 16 p: piece = (row, p4), 4 pieces per row;  transposed: A[p][m]: (p, m4), 32 per p
-  int a_r[2], a_c[2], b_r[2], b_c[2];
+  int a_r[NA], a_c[NA], b_r[2], b_c[2];
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     const int e = t + 256 * i;
-    if (TA) { a_r[i] = e >> 5; a_c[i] = (e & 31) * 4; } else { a_r[i] = e >> 2; a_c[i] = (e & 3) * 4; }
+    if (i < NA) {
+      if (TA) { a_r[i] = e / (BMT / 4); a_c[i] = (e % (BMT / 4)) * 4; } else { a_r[i] = e >> 2; a_c[i] = (e & 3) * 4; }
+    }
     if (TB) { b_r[i] = e >> 2; b_c[i] = (e & 3) * 4; } else { b_r[i] = e >> 5; b_c[i] = (e & 31) * 4; }
   }
   auto load_a = [&](int p0, int i) -> float4 {
@@ -115,46 +119,47 @@ __global__ void __launch_bounds__(256) k_sgemm_full(int P, const float* __restri
     if (TB) { Bs[buf][b_c[i]][b_r[i]] = v.x; Bs[buf][b_c[i] + 1][b_r[i]] = v.y; Bs[buf][b_c[i] + 2][b_r[i]] = v.z; Bs[buf][b_c[i] + 3][b_r[i]] = v.w; }
     else *reinterpret_cast<float4*>(&Bs[buf][b_r[i]][b_c[i]]) = v;
   };
-  float acc[8][8];
+  float acc[TM][8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
+  for (int i = 0; i < TM; ++i)
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
-  float4 ra[2], rb[2];
+  float4 ra[NA], rb[2];
 #pragma unroll
-  for (int i = 0; i < 2; ++i) { ra[i] = load_a(0, i); rb[i] = load_b(0, i); }
+  for (int i = 0; i < 2; ++i) { if (i < NA) ra[i] = load_a(0, i); rb[i] = load_b(0, i); }
 #pragma unroll
-  for (int i = 0; i < 2; ++i) { store_a(0, i, ra[i]); store_b(0, i, rb[i]); }
+  for (int i = 0; i < 2; ++i) { if (i < NA) store_a(0, i, ra[i]); store_b(0, i, rb[i]); }
   __syncthreads();
   int buf = 0;
   for (int p0 = 0; p0 < P; p0 += BKS) {
     const bool more = p0 + BKS < P;
     if (more) {
 #pragma unroll
-      for (int i = 0; i < 2; ++i) { ra[i] = load_a(p0 + BKS, i); rb[i] = load_b(p0 + BKS, i); }
+      for (int i = 0; i < 2; ++i) { if (i < NA) ra[i] = load_a(p0 + BKS, i); rb[i] = load_b(p0 + BKS, i); }
     }
 #pragma unroll
     for (int p = 0; p < BKS; ++p) {
       float a[8], b[8];
-      const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][p][ty * 4]), a1 = *reinterpret_cast<const float4*>(&As[buf][p][64 + ty * 4]);
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[buf][p][ty * 4]);
+      const float4 a1 = TM == 8 ? *reinterpret_cast<const float4*>(&As[buf][p][(BMT / 2) + ty * 4]) : a0;
       const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][p][tx * 4]), b1 = *reinterpret_cast<const float4*>(&Bs[buf][p][64 + tx * 4]);
       a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w; a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
       b[0] = b0.x; b[1] = b0.y; b[2] = b0.z; b[3] = b0.w; b[4] = b1.x; b[5] = b1.y; b[6] = b1.z; b[7] = b1.w;
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < TM; ++i)
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
     if (more) {
 #pragma unroll
-      for (int i = 0; i < 2; ++i) { store_a(buf ^ 1, i, ra[i]); store_b(buf ^ 1, i, rb[i]); }
+      for (int i = 0; i < 2; ++i) { if (i < NA) store_a(buf ^ 1, i, ra[i]); store_b(buf ^ 1, i, rb[i]); }
     }
     __syncthreads();
     buf ^= 1;
   }
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int gm = m0 + (i < 4 ? ty * 4 + i : 64 + ty * 4 + i - 4);
+  for (int i = 0; i < TM; ++i) {
+    const int gm = m0 + (i < 4 ? ty * 4 + i : (BMT / 2) + ty * 4 + i - 4);
     float* row = C + (int64_t)gm * ldc + n0;
     *reinterpret_cast<float4*>(row + tx * 4) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
     *reinterpret_cast<float4*>(row + 64 + tx * 4) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
@@ -166,10 +171,18 @@ cudaError_t sgemm(cudaStream_t st, int M, int N, int P, const float* A, int lda,
   const bool full = M % BM == 0 && N % BN == 0 && P % BKS == 0 && lda % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
                     ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15) == 0;
   if (full) {
-    if (ta && tb) k_sgemm_full<true, true><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
-    else if (ta) k_sgemm_full<true, false><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
-    else if (tb) k_sgemm_full<false, true><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
-    else k_sgemm_full<false, false><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    // products with few tiles (the 4096 x 256 iterates: 64 tiles of 128 rows on 148 SMs) take tiles of 64 rows
+    const bool half = (int)(grid.x * grid.y) < 120;
+    if (half) {
+      dim3 g2(grid.x, M / 64);
+      if (ta && tb) k_sgemm_full<true, true, 4><<<g2, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+      else if (ta) k_sgemm_full<true, false, 4><<<g2, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+      else if (tb) k_sgemm_full<false, true, 4><<<g2, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+      else k_sgemm_full<false, false, 4><<<g2, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    } else if (ta && tb) k_sgemm_full<true, true, 8><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    else if (ta) k_sgemm_full<true, false, 8><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    else if (tb) k_sgemm_full<false, true, 8><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    else k_sgemm_full<false, false, 8><<<grid, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
   } else {
     k_sgemm<<<grid, 256, 0, st>>>(M, N, P, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc);
   }
@@ -197,18 +210,20 @@ __global__ void k_init(float* y, int rows, int m, int ld) {
 // S[i][j] = sum_row A[row][i] B[row][j]  for two [rows][m] fp32 matrices, products and sums in fp64.
 // One CTA per 16 x 16 block of S, one thread per element; slices of 16 rows go through shared memory.
 __global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, const float* __restrict__ B, int rows, int m, int ld, double* __restrict__ S) {
-  __shared__ float sa[16][17], sb[16][17];
+  constexpr int RS = 64;                               // rows per slice
+  __shared__ float sa[RS][17], sb[RS][17];
   const int i0 = blockIdx.y * 16, j0 = blockIdx.x * 16, t = threadIdx.x, ti = t >> 4, tj = t & 15;
   double acc = 0.0;
-  for (int r0 = 0; r0 < rows; r0 += 16) {
-    {
-      const int rr = r0 + ti;
-      sa[ti][tj] = (rr < rows && i0 + tj < m) ? A[(int64_t)rr * ld + i0 + tj] : 0.f;
-      sb[ti][tj] = (rr < rows && j0 + tj < m) ? B[(int64_t)rr * ld + j0 + tj] : 0.f;
+  for (int r0 = 0; r0 < rows; r0 += RS) {
+#pragma unroll
+    for (int k = 0; k < RS / 16; ++k) {
+      const int rr = r0 + ti + 16 * k;
+      sa[ti + 16 * k][tj] = (rr < rows && i0 + tj < m) ? A[(int64_t)rr * ld + i0 + tj] : 0.f;
+      sb[ti + 16 * k][tj] = (rr < rows && j0 + tj < m) ? B[(int64_t)rr * ld + j0 + tj] : 0.f;
     }
     __syncthreads();
-#pragma unroll
-    for (int r = 0; r < 16; ++r) acc += (double)sa[r][ti] * (double)sb[r][tj];
+#pragma unroll 16
+    for (int r = 0; r < RS; ++r) acc += (double)sa[r][ti] * (double)sb[r][tj];
     __syncthreads();
   }
   if (i0 + ti < m && j0 + tj < m) S[(int64_t)(i0 + ti) * m + j0 + tj] = acc;
