@@ -374,7 +374,10 @@ __global__ void __launch_bounds__(1024) k_chol_inv64(double* Sg, int m, float* W
 }
 
 // Symmetric positive semi-definite eigenproblem H = V diag(lam) V^T, m x m, fp64, by one-sided (Hestenes) Jacobi in one
-// CTA: pairs of columns of H are rotated until they are orthogonal; then lam_i = ||h_i|| and V holds the rotations.
+// CTA: pairs of rows of H (= columns, H is symmetric) are rotated until they are orthogonal.  With J the product of the
+// rotations the result is J^T H = diag(lam) J^T: row i has norm lam_i and direction v_i, so the eigenvectors are the
+// normalised rows and no separate accumulation of the rotations is needed (a row whose norm is zero up to rounding has
+// no direction; its eigenvalue is far below the ones that are kept).
 // Pairs follow the round-robin tournament (m' / 2 disjoint pairs per step, m' - 1 steps per sweep); a warp takes a pair.
 // Output: eigenvalues in descending order (lam) and the matching eigenvectors as fp32 columns of Vf ([m][m] row-major).
 __global__ void __launch_bounds__(1024) k_jacobi64(double* Hg, double* V, int m, double* lam, float* Vf, int max_sweeps) {
@@ -384,7 +387,8 @@ __global__ void __launch_bounds__(1024) k_jacobi64(double* Hg, double* V, int m,
   const int t = threadIdx.x, nt = blockDim.x, warp = t >> 5, lane = t & 31, nwarp = nt >> 5;
   // the matrix whose columns are rotated is read three times per pair: in shared memory when it fits
   double* H = m <= kCholSmem ? smj : Hg;
-  for (int e = t; e < m * m; e += nt) { V[e] = (e / m == e % m) ? 1.0 : 0.0; if (m <= kCholSmem) smj[e] = Hg[e]; }
+  (void)V;
+  if (m <= kCholSmem) for (int e = t; e < m * m; e += nt) smj[e] = Hg[e];
   __syncthreads();
   const int mp = (m + 1) & ~1;                       // players of the tournament (one bye if m is odd)
   for (int sweep = 0; sweep < max_sweeps; ++sweep) {
@@ -413,11 +417,6 @@ __global__ void __launch_bounds__(1024) k_jacobi64(double* Hg, double* V, int m,
           const double a = hp[i], b = hq[i];
           hp[i] = c * a - s * b; hq[i] = s * a + c * b;
         }
-        double* vp = V + (int64_t)p * m; double* vq = V + (int64_t)q * m;
-        for (int i = lane; i < m; i += 32) {
-          const double a = vp[i], b = vq[i];
-          vp[i] = c * a - s * b; vq[i] = s * a + c * b;
-        }
         if (lane == 0) moved_s = 1;
       }
       __syncthreads();
@@ -443,9 +442,11 @@ __global__ void __launch_bounds__(1024) k_jacobi64(double* Hg, double* V, int m,
   }
   __syncthreads();
   for (int c = t; c < m; c += nt) lam[rank_s[c]] = lam[m + c];
+  __syncthreads();
   for (int e = t; e < m * m; e += nt) {
     const int c = e / m, i = e % m;                  // eigenvector c, component i  ->  Vf[i][rank of c]
-    Vf[(int64_t)i * m + rank_s[c]] = (float)V[e];
+    const double nrm = lam[rank_s[c]];
+    Vf[(int64_t)i * m + rank_s[c]] = nrm > 0.0 ? (float)(H[e] / nrm) : 0.f;
   }
 }
 
