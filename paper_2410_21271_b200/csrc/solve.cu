@@ -10,8 +10,9 @@
 //   6.  B' = U' S',  A = S'^{-1} U'^T dW
 //
 // Every kernel here is plain fp32 / fp64 CUDA-core arithmetic: the large contractions are tiled SGEMMs
-// (128 x 128 x 16 tiles through shared memory, 8 x 8 outputs per thread); fp32 because the quality of the
-// eigenvectors near the cut depends on the small differences between neighbouring eigenvalues of Mm.
+// (128 x 128 x 16 tiles through shared memory, 8 x 8 outputs per thread; 64 x 128 tiles for the skinny products of
+// the iteration); fp32 because the quality of the eigenvectors near the cut depends on the small differences
+// between neighbouring eigenvalues of Mm.  The (r + oversample)^2 problems run in fp64 in one CTA each.
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include "../../include/eora_linear.h"
