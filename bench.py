@@ -516,6 +516,35 @@ def time_solve(device: str, d: int = 4096, k: int = 4096, n: int = 2048, r: int 
            "gflop": flops / 1e9, "tflops": flops / ms / 1e9, "bound": "alu", "peak_tflops_fp32": FP32_PEAK_TFLOPS,
            "frac_of_fp32_peak": flops / ms / 1e9 / FP32_PEAK_TFLOPS,
            "remaining_loss_over_uncompensated": loss / uncompensated, "dtype": "f32 (f64 for the small problems)"}
+    # Independent layers (q, k, v share one input; gate and up another) can be solved side by side: each solve is a
+    # chain of launches on its own stream with its own workspace, and the one-CTA factorisations of one layer run beside
+    # the contractions of the others.
+    n_streams, per_stream = 4, 2
+    cfg = eora.eora_solve_config(d, k, n, r, 0, 0)
+    nbytes = eora.eora_solve_workspace_bytes(cfg)
+    streams = [torch.cuda.Stream(device=device) for _ in range(n_streams)]
+    bufs = [(torch.empty(nbytes, dtype=torch.uint8, device=device), torch.empty((d, r), dtype=torch.float32, device=device),
+             torch.empty((r, k), dtype=torch.float32, device=device), torch.empty(r, dtype=torch.float32, device=device))
+            for _ in range(n_streams)]
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    e0.record()
+    for st in streams:
+        st.wait_stream(cur)
+    for _ in range(per_stream):
+        for st, (ws, bb, aa, ss) in zip(streams, bufs):
+            eora.eora_solve(cfg, tw, th, tx, bb, aa, ss, ws, st)
+    for st in streams:
+        cur.wait_stream(st)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_c = e0.elapsed_time(e1) / (n_streams * per_stream)
+    same = all(bool(torch.equal(bb, b)) and bool(torch.equal(aa, a)) for _, bb, aa, _ in bufs)
+    out["side_by_side"] = {"streams": n_streams, "solves": n_streams * per_stream, "ms_per_layer": ms_c, "layers_per_s": 1e3 / ms_c,
+                           "tflops": flops / ms_c / 1e9, "frac_of_fp32_peak": flops / ms_c / 1e9 / FP32_PEAK_TFLOPS,
+                           "results_equal_to_the_single_stream_solve": same}
+    del bufs
     if cpu:
         from oracle import eora_solve_oracle as sol
         dc, kc, nc = 1024, 1024, 512

@@ -109,3 +109,28 @@ def test_solve_large_against_oracle():
     assert opt * (1 - 1e-6) <= got <= opt * (1 + LOSS_RTOL), (got, opt)
     assert np.isclose(loss_dev, got, rtol=1e-3)
     assert np.allclose(s, ref["sigma"], rtol=SIGMA_RTOL)
+
+
+def test_solves_side_by_side_on_three_streams():
+    """Three different layers solved at the same time, each on its own stream with its own workspace: every one meets the
+    oracle's optimum, so the solves share no state."""
+    import torch
+    cases = [(200, 160, 120, 16, 21), (256, 256, 512, 64, 22), (130, 300, 260, 24, 23)]
+    streams = [torch.cuda.Stream() for _ in cases]
+    ins, outs = [], []
+    for (d, k, n, r, seed) in cases:
+        w, w_hat, x = gen.make_solve_case(seed, d, k, n)
+        ins.append((w, w_hat, x, tuple(torch.from_numpy(np.ascontiguousarray(v)).cuda() for v in (w, w_hat, x))))
+    torch.cuda.synchronize()
+    for rep in range(2):                                  # the second round runs with every stream already busy
+        outs = []
+        for st, (d, k, n, r, _), (_, _, _, dev) in zip(streams, cases, ins):
+            with torch.cuda.stream(st):
+                outs.append(eora.solve(dev[0], dev[1], dev[2], r, stream=st))
+    torch.cuda.synchronize()
+    for (d, k, n, r, _), (w, w_hat, x, _), (b, a, s) in zip(cases, ins, outs):
+        ref = sol.solve(w, w_hat, x, r)
+        opt = sol.layer_loss(ref["dW"], ref["B"], ref["A"], x)
+        got = sol.layer_loss(ref["dW"], b.cpu().numpy(), a.cpu().numpy(), x)
+        assert opt * (1 - 1e-6) <= got <= opt * (1 + LOSS_RTOL), (d, k, n, r, got, opt)
+        assert np.allclose(s.cpu().numpy(), ref["sigma"], rtol=SIGMA_RTOL)
