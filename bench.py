@@ -678,6 +678,38 @@ def time_prefill_config(device: str, w: str, r: int, xd: str, M: int = 2048, ite
     return out
 
 
+def time_prefill_fused(device: str, r: int = 128, M: int = 2048, copies: int = 4, iters: int = 100) -> dict:
+    """The launches of a block that share their input behind one fused handle each (q|k|v, gate|up), M = 2048, 4-bit
+    backbone: one launch pair per group, every layer's tiles written to its own output."""
+    import torch
+    import paper_2410_21271_b200 as eora
+    shapes = dict(LAYERS)
+    out = {}
+    for names in (("q", "k", "v"), ("gate", "up")):
+        K = shapes[names[0]][0]
+        parts = [(gen.make_backbone_quant(5 + i, K, shapes[nm][1], 4, 128),) + tuple(gen.make_ab_f16(5 + i, K, shapes[nm][1], r))
+                 for i, nm in enumerate(names)]
+        Fs = [eora.FusedLayers(parts, max_m=M, device=device) for _ in range(copies)]
+        xh = gen.make_x(6, M, K, "f16")
+        xs = [torch.from_numpy(xh).to(device) for _ in range(copies)]
+        ys = [[torch.empty((M, shapes[nm][1]), dtype=torch.float16, device=device) for nm in names] for _ in range(copies)]
+        for F, x, y in zip(Fs, xs, ys):
+            F.forward(x, y)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            Fs[i % copies].forward(xs[i % copies], ys[i % copies])
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        fl = sum(traffic.forward_flops(K, shapes[nm][1], r, M) for nm in names)
+        out["|".join(names)] = {"ms": ms, "tflops": fl / ms / 1e9, "launches": Fs[0].launches(M)}
+        for F in Fs:
+            F.close()
+    return out
+
+
 def all_configs(device: str, device_index: int, peaks: dict) -> list:
     """Every configuration of the benchmark definition that the headline does not cover, device-timed."""
     import paper_2410_21271_b200 as eora
@@ -729,6 +761,10 @@ def all_configs(device: str, device_index: int, peaks: dict) -> list:
             if "sustained" in sb:
                 sb["sustained"]["frac_of_measured_bf16_sustained"] = sb["sustained"]["tflops_block"] / sust
         out.append(e)
+    fz = time_prefill_fused(device)
+    for v in fz.values():
+        v["frac_of_measured_bf16_burst"] = v["tflops"] / burst
+    out.append({"config": 4, "workload": "llama3-8b fused groups/q4-g128/eora-f16-r128/X-f16/M2048", "kind": "prefill-fused", "per_group": fz})
     # config 5 at M = 2048: dense-equivalent flops against 1x and 2x the dense peak (a sparse tensor path could reach 2x)
     res = time_prefill_config(device, "sp24", 128, "f16")
     out.append({"config": 5, "workload": "llama3-8b-block/sp24/eora-f16-r128/M2048", "kind": "prefill", **res,

@@ -140,13 +140,14 @@ int eora_linear_forward(eora_linear_t h, const void* x, int32_t m, void* y, void
  * (Section 3), and several of them read the same activations: q/k/v of an attention block, gate/up
  * of an MLP.  eora_linear_create_fused builds ONE handle for n_layers (2..4) such layers, given as
  * arrays of configs and weights; they must agree in everything but d_out (same d_in, rank, formats,
- * groups, dtypes, max_m <= 64, policy AUTO; any backbone format).  eora_linear_forward_fused computes
+ * groups, dtypes, max_m, policy AUTO; any backbone format).  eora_linear_forward_fused computes
  *     ys[i][M][d_out_i] = X . deq(Wq_i) + (X . A_i) . B_i      for every layer i
  * with ONE kernel launch for up to eight tokens: X is read once, and the launch latency is paid once.
- * ys: host array of n_layers device pointers (16-byte aligned, caller-owned).  The handle serves
- * M <= 64: the decode family, and for 9..64 tokens the tensor-core family (two launches, the first for
- * t = X . A of all layers) if every d_out_i is a multiple of 128, else ceil(M / 8) decode passes;
- * eora_linear_forward / _forward_host on it return
+ * ys: host array of n_layers device pointers (16-byte aligned, caller-owned).  M <= 8: the decode
+ * family; more tokens: the tensor-core family (two launches, the first for t = X . A of all layers) if
+ * every d_out_i is a multiple of 128 (and the group size of 64), else ceil(M / 8) decode passes up to
+ * M = 64.  max_m > 64 therefore needs the tensor-core family: create returns EORA_ERR_UNSUPPORTED
+ * otherwise.  eora_linear_forward / _forward_host on it return
  * EORA_ERR_UNSUPPORTED, everything else (destroy, launches, last_device_status, dump of the
  * stacked matrices) works as for a plain handle.  Errors as for create / forward.
  */

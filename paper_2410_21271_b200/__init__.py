@@ -436,7 +436,7 @@ class Layer:
 
 class FusedLayers:
     """Several layers that read the same X (q/k/v, gate/up) behind ONE handle and one launch per forward.
-    Decode only (max_m <= 64).  Methods only marshal arguments."""
+    max_m > 64 needs every d_out to be a multiple of 128 (the tensor-core family).  Methods only marshal arguments."""
 
     def __init__(self, layers, *, max_m: int, x_dtype: str = "f16", y_dtype: str = "f16",
                  kernel_policy: int = EORA_POLICY_AUTO, device="cuda:0"):
@@ -485,7 +485,7 @@ class FusedLayers:
 
 class MultiAdapterLayer:
     """One backbone with several adapters; every token of a forward names the adapter it uses (-1: none).
-    Decode only (max_m <= 64).  Methods only marshal arguments."""
+    max_m > 64 needs every d_out to be a multiple of 128 (the tensor-core family).  Methods only marshal arguments."""
 
     def __init__(self, w_fmt: dict, adapters, *, max_m: int, x_dtype: str = "f16", y_dtype: str = "f16", device="cuda:0"):
         import torch

@@ -160,7 +160,7 @@ WMat pair_view(const WMat& m, int p0, int n_pairs) {
 // pointers are taken from wts[0]).
 int create_multi_impl(const eora_linear_config* cfg, const eora_linear_weights* wts, int n, void* stream, eora_linear_t* out);
 
-// One layer (n == 1) or n layers that share X, stacked along the output axis (fused, decode only).
+// One layer (n == 1) or n layers that share X, stacked along the output axis (fused).
 int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, int n, void* stream, eora_linear_t* out) {
   if (out) *out = nullptr;
   if (!cfgs || !wts || !out) return EORA_ERR_NULL_ARG;
@@ -180,7 +180,7 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
     d_out_total += ci.d_out;
   }
   const bool fused = n > 1;
-  if (fused && (c.max_m > 64 || c.kernel_policy == EORA_POLICY_GENERIC)) return EORA_ERR_UNSUPPORTED;
+  if (fused && c.kernel_policy == EORA_POLICY_GENERIC) return EORA_ERR_UNSUPPORTED;
   c.d_out = d_out_total;
 
   eora_linear* obj = new (std::nothrow) eora_linear();
@@ -284,6 +284,8 @@ int create_impl(const eora_linear_config* cfgs, const eora_linear_weights* wts, 
   if (prefill_init(h) != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (decode_tc_init(h, s) != cudaSuccess) return fail(EORA_ERR_CUDA);
   if (fused && !decode_supported(h, 1) && !decode_tc_supported(h, 1)) return fail(EORA_ERR_UNSUPPORTED);
+  // more than 64 tokens on a fused handle: the tensor-core family only (every layer a whole number of 128-row tiles)
+  if (fused && c.max_m > 64 && !prefill_supported(h, c.max_m)) return fail(EORA_ERR_UNSUPPORTED);
   if (cudaStreamSynchronize(s) != cudaSuccess) return fail(EORA_ERR_CUDA);
   *out = obj;
   return EORA_OK;

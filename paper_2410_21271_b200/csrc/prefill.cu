@@ -57,7 +57,7 @@ struct PrefillArgs {
   // first one also takes the K-extension).  Each adds its accumulator to ws (fp32, [tokens][ld_ws], zero between
   // launches) and takes a ticket of its tile; the CTA that takes the last one converts the sums to `out` and puts
   // ws and the ticket back to zero.  ksplit == 1: the accumulator goes straight to `out`.
-  // Fused layers (stacked along the weight rows, few tokens only): layer i owns rows [sub_row0[i], sub_row0[i + 1]),
+  // Fused layers (stacked along the weight rows): layer i owns rows [sub_row0[i], sub_row0[i + 1]),
   // writes to outs[i] (leading dimension sub_ld[i]) and takes columns [i * t_sub, (i + 1) * t_sub) of t in the
   // K-extension.  A plain layer: n_sub = 1, sub_row0 = {0, n_valid}, outs[0] = out.
   int n_sub;
@@ -754,8 +754,7 @@ int token_tile(int m) {                // the MMA N: a multiple of 16 up to 256
 bool prefill_supported(const Handle* h, int m) {
   if (m <= 8) return false;              // one decode pass is always cheaper
   if (h->multi) return false;            // per-token adapters: decode family only
-  if (h->n_sub > 1) {                    // fused layers: launches of few tokens only, tiles of 128 rows must not straddle two layers
-    if (m > kThinTokens) return false;
+  if (h->n_sub > 1) {                    // fused layers: tiles of 128 rows must not straddle two layers
     for (int i = 0; i < h->n_sub; ++i)
       if (h->sub_dout[i] % BN_W) return false;
   }
@@ -907,6 +906,8 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
   a.nkb_w = c.d_in / BK; a.nkb_b = ab ? h->r_pad / BK : 0; a.dev_status = h->dev_status;
   a.trace = reinterpret_cast<long long*>(h->trace);
   a.rows = cta_rows(n_valid, m, bt, h->sm_count);
+  for (int i = 0; i < h->n_sub && h->n_sub > 1; ++i)          // fused layers: every layer a whole number of tiles
+    if (h->sub_dout[i] % (2 * BN_W)) a.rows = BN_W;
   a.n_small = 0; a.small_x = 1; a.n_split = n_valid; a.big_x = (n_valid + a.rows - 1) / a.rows;
   a.ksplit = 1; a.kchunk = a.nkb_w; a.ws = nullptr; a.ld_ws = 0; a.tickets = nullptr;
   if (thin) {
@@ -937,7 +938,7 @@ cudaError_t launch_prefill_forward(const Handle* h, const void* x, int m, void* 
       a.small_x = (n_valid - a.n_split + kSmallTile - 1) / kSmallTile;
       a.n_small = a.small_x * ((m + kSmallTile - 1) / kSmallTile);
       if (!make_map(&tm_xs, x16, m, c.d_in, c.d_in, kSmallTile)) return cudaErrorInvalidValue;
-      if (ab && !make_map(&tm_ts, h->t16, m, h->r_pad, h->r_pad, kSmallTile)) return cudaErrorInvalidValue;
+      if (ab && !make_map(&tm_ts, h->t16, m, h->t_cols, h->t_cols, kSmallTile)) return cudaErrorInvalidValue;
       if (!ab) tm_ts = tm_xs;
     }
   }

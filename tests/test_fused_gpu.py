@@ -143,3 +143,58 @@ def test_fused_argument_errors():
     assert eora.eora_linear_forward_fused(F.handle, x, 1, [y, None], check=False) == eora.EORA_ERR_NULL_ARG
     torch.cuda.synchronize()
     F.close()
+
+
+@pytest.mark.parametrize("w,ab,K,Ns,r,M,xd", [
+    ("q4", "f16", 1024, [256, 128, 128], 128, 65, "f16"),     # a 128-row layer: tiles of 128 rows throughout
+    ("q3", "q4", 512, [512, 256], 64, 300, "f16"),            # whole 256-row tiles, two token tiles with a ragged tail
+    ("q4", "q8", 1024, [128, 384], 256, 130, "bf16"),
+    ("q4", "f16", 768, [256, 256], 0, 257, "f16"),            # no adapter
+    ("sp24", "f16", 512, [128, 256], 128, 96, "f16"),
+])
+def test_fused_many_tokens_tensor_core_family(w, ab, K, Ns, r, M, xd):
+    """More than 64 tokens on a fused handle: the tensor-core family writes every layer's tiles to that layer's output
+    and takes that layer's slice of t; compared with the oracle's forward of each layer, whole outputs."""
+    layers = [make_case(90 + i, K, N, r, w=w, ab=ab) for i, N in enumerate(Ns)]
+    x = gen.make_x(91, M, K, xd)
+    F = eora.FusedLayers(layers, max_m=M, x_dtype=xd)
+    assert F.launches(M) <= 3
+    for rep in range(2):
+        ys = run_fused(F, x, xd)
+        for i, (wf, af, bf) in enumerate(layers):
+            check_parity(ys[i], orc.forward(x, xd, wf, af, bf), f"layer {i} call {rep}")
+    for m2 in (1, 8, 40):                                   # and the other families on the same handle
+        x2 = gen.make_x(92, m2, K, xd)
+        ys = run_fused(F, x2, xd)
+        for i, (wf, af, bf) in enumerate(layers):
+            check_parity(ys[i], orc.forward(x2, xd, wf, af, bf), f"layer {i} M={m2}")
+    F.close()
+
+
+@pytest.mark.parametrize("names", [("q", "k", "v"), ("gate", "up")])
+def test_fused_fullsize_prefill_sampled(names):
+    """M = 2048 at the full sizes (gate | up takes the launch whose last row tiles are covered by small tiles): sampled
+    outputs of every layer, with the corners, the last columns and both sides of tile borders among them."""
+    import torch
+    K = SHAPES[names[0]][0]
+    M = 2048
+    layers = [make_case(95 + i, K, SHAPES[nm][1], 128, w="q4") for i, nm in enumerate(names)]
+    x = gen.make_x(96, M, K)
+    F = eora.FusedLayers(layers, max_m=M)
+    assert F.launches(M) == 2
+    ys = run_fused(F, x, "f16")
+    rng = np.random.default_rng(5)
+    for i, (wf, af, bf) in enumerate(layers):
+        y = ys[i]
+        N = y.shape[1]
+        mi = rng.integers(0, M, 64); ni = rng.integers(0, N, 64)
+        mi[:4] = [0, M - 1, 0, M - 1]; ni[:4] = [0, 0, N - 1, N - 1]
+        ni[4:16] = N - 1 - rng.integers(0, min(N, 512), 12)
+        ni[16:24] = np.clip(128 * rng.integers(1, max(2, N // 128), 8) - rng.integers(0, 2, 8), 0, N - 1)
+        mi[24:32] = np.clip(128 * rng.integers(1, max(2, M // 128), 8) - rng.integers(0, 2, 8), 0, M - 1)
+        ref = orc.forward_at(x, "f16", wf, af, bf, mi, ni)
+        d = y[mi, ni] - ref
+        assert np.all(np.isfinite(y)), names[i]
+        assert np.linalg.norm(d) / np.linalg.norm(ref) <= 2e-3, names[i]
+        assert np.abs(d).max() <= 1e-2 * np.abs(ref).max(), names[i]
+    F.close()
