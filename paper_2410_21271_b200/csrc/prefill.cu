@@ -737,11 +737,19 @@ int fill_stages(PrefillArgs& a) {      // returns the dynamic shared memory to r
   return a.w_off + a.sw * 2 * BN_W * 128 + 1024;
 }
 
-// Weight rows per CTA: 256, or 128 when 256-row tiles would leave more than half of the SMs without a CTA
-// (the dequantisation of a CTA's rows is what bounds its k-block period, so halving the rows halves its time).
+// Weight rows per CTA: 256 or 128, whichever tiling needs less time counted in waves of sm_count CTAs (a CTA needs an SM
+// of its own).  The dequantisation of a CTA's rows is what bounds its k-block period (1200 cycles for 256 rows, 763 for
+// 128), so a 128-row tile costs 0.64 of a 256-row one.  A last partial wave of 256-row tiles that is at most a quarter
+// of the SMs is covered by small tiles inside the first wave (launch_prefill_forward), counted as half a wave.
 int cta_rows(int n_rows, int m, int bt, int sm_count) {
-  const int tiles = ((n_rows + 2 * BN_W - 1) / (2 * BN_W)) * ((m + bt - 1) / bt);
-  return (n_rows > BN_W && 2 * tiles <= sm_count) ? BN_W : 2 * BN_W;
+  if (n_rows <= BN_W) return 2 * BN_W;
+  const int ty = (m + bt - 1) / bt;
+  const int t256 = ((n_rows + 2 * BN_W - 1) / (2 * BN_W)) * ty, t128 = ((n_rows + BN_W - 1) / BN_W) * ty;
+  const int over = t256 % sm_count;
+  float w256 = (float)(t256 / sm_count);
+  if (over > 0) w256 += (bt == 256 && t256 > sm_count && 4 * over <= sm_count) ? 0.5f : 1.0f;
+  const float w128 = 0.64f * (float)((t128 + sm_count - 1) / sm_count);
+  return w128 < w256 ? BN_W : 2 * BN_W;
 }
 
 int token_tile(int m) {                // the MMA N: a multiple of 16 up to 256
