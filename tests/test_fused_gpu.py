@@ -198,3 +198,20 @@ def test_fused_fullsize_prefill_sampled(names):
         assert np.linalg.norm(d) / np.linalg.norm(ref) <= 2e-3, names[i]
         assert np.abs(d).max() <= 1e-2 * np.abs(ref).max(), names[i]
     F.close()
+
+
+def test_fused_forward_host_many_tokens():
+    """The host entry point above 64 tokens: results go through the staging buffer (side by side) and the copy engine."""
+    import torch
+    K, Ns, r, M = 512, [128, 256], 64, 100
+    layers = [make_case(97 + i, K, N, r, w="q4") for i, N in enumerate(Ns)]
+    x = gen.make_x(98, M, K)
+    F = eora.FusedLayers(layers, max_m=M)
+    xh = torch.from_numpy(x.copy()).pin_memory()
+    yh = [torch.full((M, N), float("nan"), dtype=torch.float16).pin_memory() for N in Ns]
+    for rep in range(2):
+        F.forward_host(xh, yh)
+        assert F.device_status() == 0
+        for i, (wf, af, bf) in enumerate(layers):
+            check_parity(yh[i].float().numpy().astype(np.float64), orc.forward(x, "f16", wf, af, bf), f"layer {i} call {rep}")
+    F.close()
