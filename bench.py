@@ -508,7 +508,7 @@ def time_solve(device: str, d: int = 4096, k: int = 4096, n: int = 2048, r: int 
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / reps
     m, iters = r + 32, 24
-    ldm = (m + 127) // 128 * 128
+    ldm = 160 if (128 < m <= 160 and d % 32 == 0) else (m + 127) // 128 * 128      # width the library's iterates are stored with
     flops = 2.0 * k * k * n + 2.0 * d * k * k + 2.0 * d * d * k + (iters + 1) * 2.0 * d * d * ldm + (iters + 2) * 2.0 * d * ldm * ldm + 2.0 * r * d * k
     loss = eora.solve_loss(tw, th, tx, b, a)
     uncompensated = float(torch.linalg.norm((tw - th).double() @ tx.double()))

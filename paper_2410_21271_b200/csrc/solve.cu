@@ -10,8 +10,8 @@
 //   6.  B' = U' S',  A = S'^{-1} U'^T dW
 //
 // Every kernel here is plain fp32 / fp64 CUDA-core arithmetic: the large contractions are tiled SGEMMs
-// (128 x 128 x 16 tiles through shared memory, 8 x 8 outputs per thread; 64 x 128 tiles for the skinny products of
-// the iteration); fp32 because the quality of the eigenvectors near the cut depends on the small differences
+// (128 x 128 x 16 tiles through shared memory, 8 x 8 outputs per thread; for the skinny products of the iteration
+// 32 x 160 tiles at the default width of 160 vectors, else 64 x 128); fp32 because the quality of the eigenvectors near the cut depends on the small differences
 // between neighbouring eigenvalues of Mm.  The (r + oversample)^2 problems run in fp64 in one CTA each.
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -167,10 +167,85 @@ __global__ void __launch_bounds__(256) k_sgemm_full(int P, const float* __restri
   }
 }
 
+// C[M][160] = A[M][P] B[P][160] (nothing transposed; M a multiple of 32, P of 16, rows 16-byte aligned): the products of the
+// subspace iteration with its default width of 160 vectors.  Tiles of 32 rows x all 160 columns, so that a product
+// with 4096 rows is 128 CTAs and no flop goes into padding columns; 2 x 10 outputs per thread.
+constexpr int NQ = 160, BMQ = 32;
+__global__ void __launch_bounds__(256) k_sgemm_n160(int P, const float* __restrict__ A, int lda, const float* __restrict__ B, int ldb,
+                                                    float* __restrict__ C, int ldc) {
+  __shared__ __align__(16) float As[2][BKS][BMQ + PAD];
+  __shared__ __align__(16) float Bs[2][BKS][NQ + PAD];
+  const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+  const int m0 = blockIdx.x * BMQ;
+  // 16-byte pieces: A tile 32 rows x 16 p = 128 pieces (threads 0..127), B tile 16 p x 160 = 640 pieces (2.5 per thread)
+  const int a_r = (t & 127) >> 2, a_c = (t & 3) * 4;
+  int b_r[3], b_c[3];
+#pragma unroll
+  for (int i = 0; i < 3; ++i) { const int e = t + 256 * i; b_r[i] = e / (NQ / 4); b_c[i] = (e % (NQ / 4)) * 4; }
+  const bool has_a = t < 128, has_b2 = t + 512 < BKS * NQ / 4;
+  auto load_a = [&](int p0) -> float4 { return *reinterpret_cast<const float4*>(A + (int64_t)(m0 + a_r) * lda + p0 + a_c); };
+  auto load_b = [&](int p0, int i) -> float4 { return *reinterpret_cast<const float4*>(B + (int64_t)(p0 + b_r[i]) * ldb + b_c[i]); };
+  auto store_a = [&](int buf, const float4& v) {
+    As[buf][a_c][a_r] = v.x; As[buf][a_c + 1][a_r] = v.y; As[buf][a_c + 2][a_r] = v.z; As[buf][a_c + 3][a_r] = v.w;
+  };
+  auto store_b = [&](int buf, int i, const float4& v) { *reinterpret_cast<float4*>(&Bs[buf][b_r[i]][b_c[i]]) = v; };
+  float acc[2][10];
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < 10; ++j) acc[i][j] = 0.f;
+  float4 ra = make_float4(0.f, 0.f, 0.f, 0.f), rb[3];
+  if (has_a) ra = load_a(0);
+#pragma unroll
+  for (int i = 0; i < 3; ++i) if (i < 2 || has_b2) rb[i] = load_b(0, i);
+  if (has_a) store_a(0, ra);
+#pragma unroll
+  for (int i = 0; i < 3; ++i) if (i < 2 || has_b2) store_b(0, i, rb[i]);
+  __syncthreads();
+  int buf = 0;
+  for (int p0 = 0; p0 < P; p0 += BKS) {
+    const bool more = p0 + BKS < P;
+    if (more) {
+      if (has_a) ra = load_a(p0 + BKS);
+#pragma unroll
+      for (int i = 0; i < 3; ++i) if (i < 2 || has_b2) rb[i] = load_b(p0 + BKS, i);
+    }
+#pragma unroll
+    for (int p = 0; p < BKS; ++p) {
+      const float2 a = *reinterpret_cast<const float2*>(&As[buf][p][ty * 2]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[buf][p][tx * 4]), b1 = *reinterpret_cast<const float4*>(&Bs[buf][p][64 + tx * 4]);
+      const float2 b2 = *reinterpret_cast<const float2*>(&Bs[buf][p][128 + tx * 2]);
+      const float b[10] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w, b2.x, b2.y};
+#pragma unroll
+      for (int j = 0; j < 10; ++j) { acc[0][j] = fmaf(a.x, b[j], acc[0][j]); acc[1][j] = fmaf(a.y, b[j], acc[1][j]); }
+    }
+    if (more) {
+      if (has_a) store_a(buf ^ 1, ra);
+#pragma unroll
+      for (int i = 0; i < 3; ++i) if (i < 2 || has_b2) store_b(buf ^ 1, i, rb[i]);
+    }
+    __syncthreads();
+    buf ^= 1;
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    float* row = C + (int64_t)(m0 + ty * 2 + i) * ldc;
+    *reinterpret_cast<float4*>(row + tx * 4) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    *reinterpret_cast<float4*>(row + 64 + tx * 4) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
+    *reinterpret_cast<float2*>(row + 128 + tx * 2) = make_float2(acc[i][8], acc[i][9]);
+  }
+}
+
 cudaError_t sgemm(cudaStream_t st, int M, int N, int P, const float* A, int lda, bool ta, const float* B, int ldb, bool tb, float* C, int ldc) {
   dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
   const bool full = M % BM == 0 && N % BN == 0 && P % BKS == 0 && lda % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
                     ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15) == 0;
+  const bool al = lda % 4 == 0 && ldb % 4 == 0 && ldc % 4 == 0 &&
+                  ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15) == 0;
+  if (N == NQ && !ta && !tb && M % BMQ == 0 && P % BKS == 0 && al) {
+    k_sgemm_n160<<<M / BMQ, 256, 0, st>>>(P, A, lda, B, ldb, C, ldc);
+    return cudaGetLastError();
+  }
   if (full) {
     // products with few tiles (the 4096 x 256 iterates: 64 tiles of 128 rows on 148 SMs) take tiles of 64 rows
     const bool half = (int)(grid.x * grid.y) < 120;
@@ -483,7 +558,7 @@ __global__ void k_axpy_neg(float* __restrict__ c, const float* __restrict__ a, i
 
 // ------------------------------------------------------------------------------------------------ workspace
 struct Plan {
-  int d, k, n, r, m, ldm, iters;       // ldm: leading dimension of the iterates (m rounded up to the SGEMM tile)
+  int d, k, n, r, m, ldm, iters;       // ldm: leading dimension of the iterates (m rounded up to the SGEMM tile, or 160)
   size_t off_w, off_dw, off_g, off_t, off_m, off_y, off_q, off_z, off_u, off_s, off_h, off_v, off_lam, off_vf, total;
 };
 size_t up256(size_t v) { return (v + 255) & ~size_t(255); }
@@ -496,6 +571,7 @@ bool make_plan(const eora_solve_config* c, Plan& p) {
   if (p.r > p.m || p.m > 512) return false;
   p.iters = c->iters > 0 ? c->iters : 24;
   p.ldm = (p.m + BN - 1) / BN * BN;
+  if (p.m > BN && p.m <= NQ && p.d % BMQ == 0) p.ldm = NQ;          // the default width: its own kernel, no padding columns
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += up256(bytes); return at; };
   p.off_dw = take((size_t)p.d * p.k * 4);

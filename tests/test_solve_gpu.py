@@ -27,7 +27,8 @@ def run_solve(w, w_hat, x, r, **kw):
     return b.cpu().numpy().astype(np.float64), a.cpu().numpy().astype(np.float64), s.cpu().numpy().astype(np.float64), loss_dev
 
 
-@pytest.mark.parametrize("d,k,n,r", [(96, 64, 200, 8), (200, 160, 120, 16), (130, 70, 33, 5), (64, 300, 500, 12), (256, 256, 512, 64)])
+@pytest.mark.parametrize("d,k,n,r", [(96, 64, 200, 8), (200, 160, 120, 16), (130, 70, 33, 5), (64, 300, 500, 12), (256, 256, 512, 64),
+                                     (256, 192, 300, 120), (320, 256, 400, 128), (264, 192, 300, 128)])   # iterates 152 and 160 wide: the 160-column product; 264 rows: the padded one
 def test_solve_matches_oracle_loss_and_spectrum(d, k, n, r):
     w, w_hat, x = gen.make_solve_case(11, d, k, n)
     ref = sol.solve(w, w_hat, x, r)
