@@ -284,25 +284,45 @@ __global__ void k_init(float* y, int rows, int m, int ld) {
 }
 
 // S[i][j] = sum_row A[row][i] B[row][j]  for two [rows][m] fp32 matrices, products and sums in fp64.
-// One CTA per 16 x 16 block of S, one thread per element; slices of 16 rows go through shared memory.
-__global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, const float* __restrict__ B, int rows, int m, int ld, double* __restrict__ S) {
+// One CTA per 16 x 16 block of S and per part of the rows (blockIdx.z; `chunk` rows each, a multiple of the slice), one
+// thread per element; slices of 64 rows go through shared memory.  Part z writes its sums to parts[z][m][m];
+// k_sum_parts adds the parts in a fixed order, so the result does not depend on the order the CTAs ran in.
+constexpr int kGramParts = 4;
+__global__ void __launch_bounds__(256) k_gram64(const float* __restrict__ A, const float* __restrict__ B, int rows, int chunk, int m, int ld,
+                                                double* __restrict__ parts) {
   constexpr int RS = 64;                               // rows per slice
   __shared__ float sa[RS][17], sb[RS][17];
   const int i0 = blockIdx.y * 16, j0 = blockIdx.x * 16, t = threadIdx.x, ti = t >> 4, tj = t & 15;
+  const int r_lo = blockIdx.z * chunk, r_hi = min(rows, r_lo + chunk);
   double acc = 0.0;
-  for (int r0 = 0; r0 < rows; r0 += RS) {
+  for (int r0 = r_lo; r0 < r_hi; r0 += RS) {
 #pragma unroll
     for (int k = 0; k < RS / 16; ++k) {
       const int rr = r0 + ti + 16 * k;
-      sa[ti + 16 * k][tj] = (rr < rows && i0 + tj < m) ? A[(int64_t)rr * ld + i0 + tj] : 0.f;
-      sb[ti + 16 * k][tj] = (rr < rows && j0 + tj < m) ? B[(int64_t)rr * ld + j0 + tj] : 0.f;
+      sa[ti + 16 * k][tj] = (rr < r_hi && i0 + tj < m) ? A[(int64_t)rr * ld + i0 + tj] : 0.f;
+      sb[ti + 16 * k][tj] = (rr < r_hi && j0 + tj < m) ? B[(int64_t)rr * ld + j0 + tj] : 0.f;
     }
     __syncthreads();
 #pragma unroll 16
     for (int r = 0; r < RS; ++r) acc += (double)sa[r][ti] * (double)sb[r][tj];
     __syncthreads();
   }
-  if (i0 + ti < m && j0 + tj < m) S[(int64_t)(i0 + ti) * m + j0 + tj] = acc;
+  if (i0 + ti < m && j0 + tj < m) parts[((int64_t)blockIdx.z * m + i0 + ti) * m + j0 + tj] = acc;
+}
+__global__ void k_sum_parts(const double* __restrict__ parts, int n_parts, int n, double* __restrict__ S) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  double v = parts[i];
+  for (int z = 1; z < n_parts; ++z) v += parts[(int64_t)z * n + i];
+  S[i] = v;
+}
+// S = A^T B over all rows: the parts, then their sum.
+cudaError_t gram64(cudaStream_t st, const float* A, const float* B, int rows, int m, int ld, double* parts, double* S) {
+  const int chunk = ((rows + kGramParts - 1) / kGramParts + 63) / 64 * 64;
+  dim3 g((m + 15) / 16, (m + 15) / 16, kGramParts);
+  k_gram64<<<g, 256, 0, st>>>(A, B, rows, chunk, m, ld, parts);
+  k_sum_parts<<<(m * m + 255) / 256, 256, 0, st>>>(parts, kGramParts, m * m, S);
+  return cudaGetLastError();
 }
 
 // Largest m for which the one-CTA kernels below keep their fp64 matrix in shared memory.
@@ -559,7 +579,7 @@ __global__ void k_axpy_neg(float* __restrict__ c, const float* __restrict__ a, i
 // ------------------------------------------------------------------------------------------------ workspace
 struct Plan {
   int d, k, n, r, m, ldm, iters;       // ldm: leading dimension of the iterates (m rounded up to the SGEMM tile, or 160)
-  size_t off_w, off_dw, off_g, off_t, off_m, off_y, off_q, off_z, off_u, off_s, off_h, off_v, off_lam, off_vf, total;
+  size_t off_w, off_dw, off_g, off_t, off_m, off_y, off_q, off_z, off_u, off_s, off_sp, off_h, off_v, off_lam, off_vf, total;
 };
 size_t up256(size_t v) { return (v + 255) & ~size_t(255); }
 bool make_plan(const eora_solve_config* c, Plan& p) {
@@ -584,6 +604,7 @@ bool make_plan(const eora_solve_config* c, Plan& p) {
   p.off_w = take((size_t)p.ldm * p.ldm * 4);
   p.off_u = take((size_t)p.d * p.r * 4);
   p.off_s = take((size_t)p.m * p.m * 8);
+  p.off_sp = take((size_t)kGramParts * p.m * p.m * 8);
   p.off_h = take((size_t)p.m * p.m * 8);
   p.off_v = take((size_t)p.m * p.m * 8);
   p.off_lam = take((size_t)2 * p.m * 8);
@@ -596,9 +617,8 @@ inline bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 
 #define CK(x) do { cudaError_t e__ = (x); if (e__ != cudaSuccess) return EORA_ERR_CUDA; } while (0)
 
 // Q = orth(Y) by Cholesky-QR: Gram matrix, factor and its inverse in fp64, then Q = Y L^{-T} as a contraction.
-int orthonormalise(cudaStream_t st, const Plan& p, const float* Y, float* Q, double* S, float* W) {
-  dim3 g((p.m + 15) / 16, (p.m + 15) / 16);
-  k_gram64<<<g, 256, 0, st>>>(Y, Y, p.d, p.m, p.ldm, S);
+int orthonormalise(cudaStream_t st, const Plan& p, const float* Y, float* Q, double* S, double* parts, float* W) {
+  CK(gram64(st, Y, Y, p.d, p.m, p.ldm, parts, S));
   static bool attr_set[64] = {};
   int device = 0;
   if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return EORA_ERR_CUDA;
@@ -640,6 +660,7 @@ int eora_solve(const eora_solve_config* cfg, const float* w, const float* w_hat,
   float* Wm = reinterpret_cast<float*>(ws + p.off_w);
   float* U = reinterpret_cast<float*>(ws + p.off_u);
   double* S = reinterpret_cast<double*>(ws + p.off_s);
+  double* Sp = reinterpret_cast<double*>(ws + p.off_sp);
   double* H = reinterpret_cast<double*>(ws + p.off_h);
   double* V = reinterpret_cast<double*>(ws + p.off_v);
   double* lam = reinterpret_cast<double*>(ws + p.off_lam);
@@ -654,18 +675,15 @@ int eora_solve(const eora_solve_config* cfg, const float* w, const float* w_hat,
   CK(sgemm(st, d, d, k, T, k, false, dW, k, true, Mm, d));                    // Mm = T dW^T
   // step 5: subspace iteration
   k_init<<<592, 256, 0, st>>>(Y, d, m, ldm);
-  if (int rc = orthonormalise(st, p, Y, Q, S, Wm)) return rc;
+  if (int rc = orthonormalise(st, p, Y, Q, S, Sp, Wm)) return rc;
   for (int it = 0; it < p.iters; ++it) {
     CK(sgemm(st, d, ldm, d, Mm, d, false, Q, ldm, false, Y, ldm));            // Y = Mm Q
-    if (int rc = orthonormalise(st, p, Y, Q, S, Wm)) return rc;
+    if (int rc = orthonormalise(st, p, Y, Q, S, Sp, Wm)) return rc;
   }
-  if (int rc = orthonormalise(st, p, Q, Y, S, Wm)) return rc;                 // second pass: orthogonal to fp32 rounding
+  if (int rc = orthonormalise(st, p, Q, Y, S, Sp, Wm)) return rc;                 // second pass: orthogonal to fp32 rounding
   // Rayleigh-Ritz on span(Y)
   CK(sgemm(st, d, ldm, d, Mm, d, false, Y, ldm, false, Z, ldm));              // Z = Mm Y
-  {
-    dim3 g((m + 15) / 16, (m + 15) / 16);
-    k_gram64<<<g, 256, 0, st>>>(Y, Z, d, m, ldm, H);                          // H = Y^T Mm Y
-  }
+  CK(gram64(st, Y, Z, d, m, ldm, Sp, H));                                     // H = Y^T Mm Y
   {
     static bool jattr[64] = {};
     int device = 0;
