@@ -264,3 +264,16 @@ def test_fused_qkv_fullsize_eight_tokens():
     for (w, a, b), y in zip(parts, ys):
         check_parity(y.float().cpu().numpy().astype(np.float64), orc.forward(x, "f16", w, a, b), "fused q|k|v M8")
     F.close()
+
+
+@pytest.mark.parametrize("name,M", [("q", 3072), ("q", 1536), ("k", 4096), ("gate", 1024)])
+def test_prefill_other_token_counts_sampled(name, M):
+    """Token counts at which the launch picks another tiling than at M = 2048 (rows per CTA are chosen by counting the
+    waves of both tilings; q at M = 3072 takes tiles of 128 rows)."""
+    K, N = SHAPES[name]
+    wf, af, bf = make_case(41, K, N, 128, w="q4")
+    x = gen.make_x(42, M, K)
+    L = eora.Layer(wf, af, bf, max_m=M)
+    assert L.path(M) == eora.EORA_PATH_PREFILL
+    sampled_check(L, wf, af, bf, x, "f16")
+    L.close()
