@@ -671,7 +671,7 @@ int eora_solve(const eora_solve_config* cfg, const float* w, const float* w_hat,
   k_sub<<<592, 256, 0, st>>>(w, w_hat, dW, (int64_t)d * k);
   // steps 2-4, as the d x d matrix dW' dW'^T = dW (X~ X~^T) dW^T
   CK(sgemm(st, k, k, n, x_tilde, n, false, x_tilde, n, true, G, k));          // G = X~ X~^T
-  CK(sgemm(st, d, k, k, dW, k, false, G, k, false, T, k));                    // T = dW G
+  CK(sgemm(st, d, k, k, dW, k, false, G, k, true, T, k));                     // T = dW G = dW G^T (G is symmetric; the row-by-row form of the product is the faster one)
   CK(sgemm(st, d, d, k, T, k, false, dW, k, true, Mm, d));                    // Mm = T dW^T
   // step 5: subspace iteration
   k_init<<<592, 256, 0, st>>>(Y, d, m, ldm);
