@@ -500,7 +500,22 @@ __global__ void __launch_bounds__(1024) k_jacobi64(double* Hg, double* V, int m,
         // columns p and q of H (column c of the symmetric start is stored as row c: H[c * m + i])
         double* hp = H + (int64_t)p * m; double* hq = H + (int64_t)q * m;
         double al = 0.0, be = 0.0, ga = 0.0;
-        for (int i = lane; i < m; i += 32) { const double a = hp[i], b = hq[i]; al += a * a; be += b * b; ga += a * b; }
+        // up to 160 columns a lane keeps its five elements of both rows in registers between the products and the
+        // rotation: the kernel is bound by shared-memory traffic, and this takes a third of it away
+        constexpr int KE = 5;
+        const bool keep = m <= 32 * KE;
+        double av[KE], bv[KE];
+        if (keep) {
+#pragma unroll
+          for (int e = 0; e < KE; ++e) {
+            const int i = lane + 32 * e;
+            const double a = i < m ? hp[i] : 0.0, b = i < m ? hq[i] : 0.0;
+            av[e] = a; bv[e] = b;
+            al += a * a; be += b * b; ga += a * b;
+          }
+        } else {
+          for (int i = lane; i < m; i += 32) { const double a = hp[i], b = hq[i]; al += a * a; be += b * b; ga += a * b; }
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           al += __shfl_xor_sync(0xffffffffu, al, o); be += __shfl_xor_sync(0xffffffffu, be, o); ga += __shfl_xor_sync(0xffffffffu, ga, o);
@@ -509,9 +524,17 @@ __global__ void __launch_bounds__(1024) k_jacobi64(double* Hg, double* V, int m,
         const double zeta = (be - al) / (2.0 * ga);
         const double tt = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
         const double c = 1.0 / sqrt(1.0 + tt * tt), s = c * tt;
-        for (int i = lane; i < m; i += 32) {
-          const double a = hp[i], b = hq[i];
-          hp[i] = c * a - s * b; hq[i] = s * a + c * b;
+        if (keep) {
+#pragma unroll
+          for (int e = 0; e < KE; ++e) {
+            const int i = lane + 32 * e;
+            if (i < m) { hp[i] = c * av[e] - s * bv[e]; hq[i] = s * av[e] + c * bv[e]; }
+          }
+        } else {
+          for (int i = lane; i < m; i += 32) {
+            const double a = hp[i], b = hq[i];
+            hp[i] = c * a - s * b; hq[i] = s * a + c * b;
+          }
         }
         if (lane == 0) moved_s = 1;
       }
